@@ -1,0 +1,145 @@
+/*
+ * moc_ffn.h -- C ABI of the B200 (sm_100a) Mixture-of-Channels FFN operator.
+ *
+ * The operator (paper Section 3.2, Eqs. (Moc-1), the Top-K mask, (MoC-2)):
+ *     G = X W_gate,  M = TopK_row(G),  S' = SiLU(G) . M,  Z' = S' . U on M (U = X W_up),  D = Z' W_down
+ * Only the K selected channels of every token are formed, and only the compact triple
+ * (channel index, gate value, up value) is kept for the backward pass (Section 4, Table 1,
+ * column "MoC+GCP": G.M, U.M and M stored; S.M and Z.M recomputed).
+ *
+ * Conventions that hold for every entry point
+ * -------------------------------------------
+ * Pointers   All data pointers are DEVICE pointers on the current CUDA device, 16-byte aligned;
+ *            `desc` is a HOST pointer; `cuda_stream` is a cudaStream_t passed as void* (NULL = the
+ *            legacy default stream).  The caller owns every buffer, including the workspace.  The
+ *            library allocates no device memory.
+ * Layouts    x, out, grad_out, grad_x : [tokens, d_model] row-major.
+ *            w_gate, w_up, w_down and their gradients : CHANNEL-MAJOR [d_ff_ld, d_model] row-major,
+ *            row j = the d_model-vector of channel j.  For gate/up that is column j of the paper's
+ *            W in R^{d x d_ffn}; for down it is row j of the paper's W_down in R^{d_ffn x d}.  Rows
+ *            d_ff .. d_ff_ld-1 are padding: never selected, never read as channels, and their
+ *            gradient rows are written as zero.
+ *            topk_idx [tokens, k] int16, ascending within a token; topk_gate / topk_up [tokens, k]
+ *            in the storage dtype: the pre-SiLU gate value g and the up value u of each kept channel.
+ * Selection  The K channels with the largest SIGNED pre-SiLU gate values, compared on the fp32
+ *            accumulator of the gate projection.  Ties at the K-th value go to the lower channel;
+ *            -0.0 equals +0.0; NaN orders as -infinity.
+ * Arithmetic Storage dtype per `dtype`; every contraction accumulates in fp32.
+ * Async      Calls enqueue work on `cuda_stream` and return without synchronising.  Errors the host
+ *            can see (bad descriptor, NULL or misaligned pointer, workspace too small) are returned
+ *            as a negative status BEFORE anything is launched.  Conditions only the device can see
+ *            (a saved index outside [0, d_ff), a bounded wait that expired) make the kernel skip the
+ *            offending work without touching out-of-range memory and raise a sticky per-device status
+ *            word that moc_last_device_status() reports.
+ * Threads    Entry points may be called from several host threads on different streams as long as
+ *            their buffers (workspace included) do not overlap.
+ */
+#ifndef MOC_FFN_H_
+#define MOC_FFN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(_WIN32)
+#define MOC_API
+#else
+#define MOC_API __attribute__((visibility("default")))
+#endif
+
+typedef enum {
+    MOC_OK = 0,
+    MOC_ERR_INVALID_ARG = -1, /* NULL/misaligned pointer, k outside [1, d_ff], negative sizes ...   */
+    MOC_ERR_UNSUPPORTED = -2, /* d_ff > 32768 (int16 indices), d_model % 8 != 0, decode tokens > 16 */
+    MOC_ERR_WORKSPACE = -3,   /* workspace pointer NULL or smaller than moc_ffn_workspace_bytes()    */
+    MOC_ERR_CUDA = -4,        /* a CUDA runtime call or a launch failed                             */
+    MOC_ERR_TIMEOUT = -5,     /* device status: a bounded wait inside a kernel expired              */
+    MOC_ERR_BAD_INDEX = -6    /* device status: a saved channel index was outside [0, d_ff)         */
+} moc_status;
+
+typedef enum { MOC_F32 = 0, MOC_BF16 = 1 } moc_dtype;
+
+typedef enum { MOC_OP_FORWARD = 0, MOC_OP_BACKWARD = 1, MOC_OP_DECODE = 2 } moc_op;
+
+/* bit 0 of moc_ffn_desc.flags: add into grad_w_* instead of overwriting them */
+#define MOC_FLAG_ACCUMULATE_WGRAD 1u
+
+typedef struct moc_ffn_desc {
+    int64_t tokens;   /* T = batch * seq, >= 0 (0 is a no-op)                                   */
+    int32_t d_model;  /* d, multiple of 8                                                        */
+    int32_t d_ff;     /* F, logical channel count, 1 <= F <= 32768                               */
+    int32_t d_ff_ld;  /* rows allocated in each weight array, >= d_ff                            */
+    int32_t k;        /* channels kept per token, 1 <= k <= d_ff; k == d_ff is dense SwiGLU      */
+    int32_t dtype;    /* moc_dtype of x, weights, out, topk_gate/topk_up and all gradients       */
+    uint32_t flags;   /* MOC_FLAG_*                                                              */
+} moc_ffn_desc;
+
+/*
+ * Bytes of caller-provided workspace that `op` needs for this descriptor (0 on an invalid
+ * descriptor).  The workspace holds transient buffers only (gate projection of a token chunk,
+ * per-channel token lists for the weight gradients ...); nothing in it outlives the call.
+ */
+MOC_API size_t moc_ffn_workspace_bytes(const moc_ffn_desc *desc, int op);
+
+/*
+ * Forward, Eqs. (Moc-1), mask, (MoC-2).
+ *   in : x [T,d], w_gate / w_up / w_down [d_ff_ld, d]
+ *   out: out [T,d]; topk_idx [T,k] int16, topk_gate [T,k], topk_up [T,k] -- the compact saved
+ *        activations of Table 1 ("MoC+GCP").  The three saved outputs may all be NULL (inference:
+ *        nothing is kept); passing only some of them is MOC_ERR_INVALID_ARG.
+ * Returns MOC_OK or a negative moc_status; nothing is launched on error.
+ */
+MOC_API int moc_ffn_forward(const moc_ffn_desc *desc, const void *x, const void *w_gate, const void *w_up,
+                            const void *w_down, void *out, int16_t *topk_idx, void *topk_gate, void *topk_up,
+                            void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * Backward, Eqs. (bp-1)..(bp-5), from the saved compact activations (S' and Z' are recomputed
+ * element-wise from topk_gate / topk_up; the mask is a constant, no gradient flows through it).
+ *   in : x, weights, topk_idx / topk_gate / topk_up as written by moc_ffn_forward, grad_out [T,d]
+ *   out: grad_x [T,d]; grad_w_gate / grad_w_up / grad_w_down [d_ff_ld, d].  Any of the four may be
+ *        NULL (skipped).  Weight gradients are overwritten unless MOC_FLAG_ACCUMULATE_WGRAD is set.
+ * A saved index outside [0, d_ff) is skipped and reported through moc_last_device_status().
+ */
+MOC_API int moc_ffn_backward(const moc_ffn_desc *desc, const void *x, const void *w_gate, const void *w_up,
+                             const void *w_down, const int16_t *topk_idx, const void *topk_gate,
+                             const void *topk_up, const void *grad_out, void *grad_x, void *grad_w_gate,
+                             void *grad_w_up, void *grad_w_down, void *workspace, size_t workspace_bytes,
+                             void *cuda_stream);
+
+/*
+ * Small-batch inference (Section 5): the same forward for tokens <= 16, organised so that only the
+ * gate matrix and the selected rows of w_up / w_down are read from HBM
+ * (d d_ffn + 2 K d weight elements per token instead of 3 d d_ffn).  Nothing is saved.
+ */
+MOC_API int moc_ffn_decode(const moc_ffn_desc *desc, const void *x, const void *w_gate, const void *w_up,
+                           const void *w_down, void *out, void *workspace, size_t workspace_bytes,
+                           void *cuda_stream);
+
+/*
+ * The Top-K selector alone (the mask definition of Section 3.2), exposed so that it can be checked
+ * bit-exactly: gate [rows, n_ld] fp32 on the device, only the first n columns of a row are channels;
+ * idx_out [rows, k] int16 ascending.  Needs no workspace.
+ */
+MOC_API int moc_topk_select(int64_t rows, int32_t n, int32_t n_ld, int32_t k, const float *gate,
+                            int16_t *idx_out, void *cuda_stream);
+
+/*
+ * Synchronises `cuda_stream`, then returns and clears the current device's sticky status word:
+ * MOC_OK, MOC_ERR_TIMEOUT or MOC_ERR_BAD_INDEX (MOC_ERR_CUDA if the synchronisation itself failed).
+ */
+MOC_API int moc_last_device_status(void *cuda_stream);
+
+/* Bytes per token that stay alive between forward and backward: k * (2 + 2 * sizeof(dtype)). */
+MOC_API size_t moc_ffn_saved_bytes_per_token(const moc_ffn_desc *desc);
+
+/* Static, NUL-terminated description of a moc_status value. */
+MOC_API const char *moc_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MOC_FFN_H_ */

@@ -1,0 +1,220 @@
+"""ctypes binding of the MoC FFN C ABI (``include/moc_ffn.h``).
+
+Argument marshalling only: every step of the operator runs in the CUDA library.  PyTorch is
+used for device memory and streams.  There is no fallback: if ``libmoc_ffn.so`` has not been
+built (``python -m paper_2511_09323_b200.build``) or cannot be loaded, the first call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libmoc_ffn.so")
+
+MOC_OK = 0
+MOC_ERR_INVALID_ARG = -1
+MOC_ERR_UNSUPPORTED = -2
+MOC_ERR_WORKSPACE = -3
+MOC_ERR_CUDA = -4
+MOC_ERR_TIMEOUT = -5
+MOC_ERR_BAD_INDEX = -6
+MOC_F32, MOC_BF16 = 0, 1
+MOC_OP_FORWARD, MOC_OP_BACKWARD, MOC_OP_DECODE = 0, 1, 2
+MOC_FLAG_ACCUMULATE_WGRAD = 1
+
+EXPORTED = (
+    "moc_ffn_workspace_bytes", "moc_ffn_forward", "moc_ffn_backward", "moc_ffn_decode", "moc_topk_select",
+    "moc_last_device_status", "moc_ffn_saved_bytes_per_token", "moc_status_string",
+)
+
+
+class MocFfnDesc(ctypes.Structure):
+    _fields_ = [
+        ("tokens", ctypes.c_int64), ("d_model", ctypes.c_int32), ("d_ff", ctypes.c_int32),
+        ("d_ff_ld", ctypes.c_int32), ("k", ctypes.c_int32), ("dtype", ctypes.c_int32),
+        ("flags", ctypes.c_uint32),
+    ]
+
+
+class MocError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} ({status})")
+
+
+_lib = None
+
+
+def load() -> ctypes.CDLL:
+    """Loads the CUDA library; raises if it is missing (there is no CPU path)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} not found: build it with `python -m paper_2511_09323_b200.build`")
+        lib = ctypes.CDLL(LIB_PATH)
+        vp, sz = ctypes.c_void_p, ctypes.c_size_t
+        dp = ctypes.POINTER(MocFfnDesc)
+        lib.moc_ffn_workspace_bytes.restype = sz
+        lib.moc_ffn_workspace_bytes.argtypes = [dp, ctypes.c_int]
+        lib.moc_ffn_saved_bytes_per_token.restype = sz
+        lib.moc_ffn_saved_bytes_per_token.argtypes = [dp]
+        lib.moc_ffn_forward.restype = ctypes.c_int
+        lib.moc_ffn_forward.argtypes = [dp] + [vp] * 9 + [sz, vp]
+        lib.moc_ffn_backward.restype = ctypes.c_int
+        lib.moc_ffn_backward.argtypes = [dp] + [vp] * 13 + [sz, vp]
+        lib.moc_ffn_decode.restype = ctypes.c_int
+        lib.moc_ffn_decode.argtypes = [dp] + [vp] * 6 + [sz, vp]
+        lib.moc_topk_select.restype = ctypes.c_int
+        lib.moc_topk_select.argtypes = [ctypes.c_int64, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, vp, vp, vp]
+        lib.moc_last_device_status.restype = ctypes.c_int
+        lib.moc_last_device_status.argtypes = [vp]
+        lib.moc_status_string.restype = ctypes.c_char_p
+        lib.moc_status_string.argtypes = [ctypes.c_int]
+        _lib = lib
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return load().moc_status_string(int(status)).decode()
+
+
+def _dtype_code(t: torch.dtype) -> int:
+    if t == torch.float32:
+        return MOC_F32
+    if t == torch.bfloat16:
+        return MOC_BF16
+    raise TypeError(f"unsupported storage dtype {t}")
+
+
+def make_desc(tokens, d_model, d_ff, k, dtype, d_ff_ld=None, flags=0) -> MocFfnDesc:
+    code = dtype if isinstance(dtype, int) else _dtype_code(dtype)
+    return MocFfnDesc(int(tokens), int(d_model), int(d_ff), int(d_ff if d_ff_ld is None else d_ff_ld), int(k),
+                      code, int(flags))
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream_ptr(stream=None):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _check_dev(*tensors):
+    for t in tensors:
+        if t is None:
+            continue
+        if not t.is_cuda:
+            raise ValueError("expected CUDA tensors")
+        if not t.is_contiguous():
+            raise ValueError("expected contiguous tensors")
+
+
+def moc_ffn_workspace_bytes(desc: MocFfnDesc, op: int) -> int:
+    return int(load().moc_ffn_workspace_bytes(ctypes.byref(desc), int(op)))
+
+
+def moc_ffn_saved_bytes_per_token(desc: MocFfnDesc) -> int:
+    return int(load().moc_ffn_saved_bytes_per_token(ctypes.byref(desc)))
+
+
+def alloc_workspace(desc: MocFfnDesc, op: int, device=None) -> torch.Tensor:
+    n = moc_ffn_workspace_bytes(desc, op)
+    return torch.empty(max(n, 16), dtype=torch.uint8, device=device or torch.device("cuda"))
+
+
+def moc_ffn_forward(x, w_gate, w_up, w_down, k, d_ff=None, save=True, out=None, saved=None, workspace=None,
+                    stream=None):
+    """Returns (out, topk_idx, topk_gate, topk_up); the last three are None when save=False."""
+    _check_dev(x, w_gate, w_up, w_down, out, workspace)
+    T, d = x.shape
+    F_ld = w_gate.shape[0]
+    desc = make_desc(T, d, F_ld if d_ff is None else d_ff, k, x.dtype, d_ff_ld=F_ld)
+    if out is None:
+        out = torch.empty_like(x)
+    if save:
+        if saved is None:
+            saved = (torch.empty((T, k), dtype=torch.int16, device=x.device),
+                     torch.empty((T, k), dtype=x.dtype, device=x.device),
+                     torch.empty((T, k), dtype=x.dtype, device=x.device))
+        idx, tg, tu = saved
+    else:
+        idx = tg = tu = None
+    if workspace is None:
+        workspace = alloc_workspace(desc, MOC_OP_FORWARD, x.device)
+    rc = load().moc_ffn_forward(ctypes.byref(desc), _ptr(x), _ptr(w_gate), _ptr(w_up), _ptr(w_down), _ptr(out),
+                                _ptr(idx), _ptr(tg), _ptr(tu), _ptr(workspace), workspace.numel(),
+                                _stream_ptr(stream))
+    if rc != MOC_OK:
+        raise MocError(rc, "moc_ffn_forward")
+    return out, idx, tg, tu
+
+
+def moc_ffn_backward(x, w_gate, w_up, w_down, topk_idx, topk_gate, topk_up, grad_out, d_ff=None,
+                     want=("x", "w_gate", "w_up", "w_down"), grads=None, accumulate=False, workspace=None,
+                     stream=None):
+    """Returns dict(grad_x, grad_w_gate, grad_w_up, grad_w_down) (None for entries not in `want`)."""
+    _check_dev(x, w_gate, w_up, w_down, topk_idx, topk_gate, topk_up, grad_out, workspace)
+    T, d = x.shape
+    F_ld = w_gate.shape[0]
+    k = topk_idx.shape[1]
+    desc = make_desc(T, d, F_ld if d_ff is None else d_ff, k, x.dtype, d_ff_ld=F_ld,
+                     flags=MOC_FLAG_ACCUMULATE_WGRAD if accumulate else 0)
+    grads = dict(grads or {})
+    res = {}
+    for name, like in (("x", x), ("w_gate", w_gate), ("w_up", w_up), ("w_down", w_down)):
+        key = "grad_" + name
+        if name in want:
+            res[key] = grads.get(key)
+            if res[key] is None:
+                res[key] = torch.empty_like(like)
+        else:
+            res[key] = None
+    _check_dev(*res.values())
+    if workspace is None:
+        workspace = alloc_workspace(desc, MOC_OP_BACKWARD, x.device)
+    rc = load().moc_ffn_backward(ctypes.byref(desc), _ptr(x), _ptr(w_gate), _ptr(w_up), _ptr(w_down),
+                                 _ptr(topk_idx), _ptr(topk_gate), _ptr(topk_up), _ptr(grad_out),
+                                 _ptr(res["grad_x"]), _ptr(res["grad_w_gate"]), _ptr(res["grad_w_up"]),
+                                 _ptr(res["grad_w_down"]), _ptr(workspace), workspace.numel(), _stream_ptr(stream))
+    if rc != MOC_OK:
+        raise MocError(rc, "moc_ffn_backward")
+    return res
+
+
+def moc_ffn_decode(x, w_gate, w_up, w_down, k, d_ff=None, out=None, workspace=None, stream=None):
+    _check_dev(x, w_gate, w_up, w_down, out, workspace)
+    T, d = x.shape
+    F_ld = w_gate.shape[0]
+    desc = make_desc(T, d, F_ld if d_ff is None else d_ff, k, x.dtype, d_ff_ld=F_ld)
+    if out is None:
+        out = torch.empty_like(x)
+    if workspace is None:
+        workspace = alloc_workspace(desc, MOC_OP_DECODE, x.device)
+    rc = load().moc_ffn_decode(ctypes.byref(desc), _ptr(x), _ptr(w_gate), _ptr(w_up), _ptr(w_down), _ptr(out),
+                               _ptr(workspace), workspace.numel(), _stream_ptr(stream))
+    if rc != MOC_OK:
+        raise MocError(rc, "moc_ffn_decode")
+    return out
+
+
+def moc_topk_select(gate: torch.Tensor, k: int, n: int | None = None, stream=None) -> torch.Tensor:
+    """gate [rows, n_ld] fp32 on the device -> idx [rows, k] int16 (ascending)."""
+    _check_dev(gate)
+    if gate.dtype != torch.float32 or gate.dim() != 2:
+        raise TypeError("gate must be a 2-D fp32 tensor")
+    rows, n_ld = gate.shape
+    n = n_ld if n is None else n
+    idx = torch.empty((rows, k), dtype=torch.int16, device=gate.device)
+    rc = load().moc_topk_select(rows, n, n_ld, k, _ptr(gate), _ptr(idx), _stream_ptr(stream))
+    if rc != MOC_OK:
+        raise MocError(rc, "moc_topk_select")
+    return idx
+
+
+def moc_last_device_status(stream=None) -> int:
+    return int(load().moc_last_device_status(_stream_ptr(stream)))

@@ -1,0 +1,350 @@
+// C ABI of the MoC FFN library: argument validation, workspace carving, kernel plans.
+// Everything here is host code that only enqueues kernels on the caller's stream.
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstdint>
+#include <cstring>
+
+#include "gather_kernels.cuh"
+#include "moc_common.cuh"
+#include "topk_select.cuh"
+
+namespace moc {
+
+// ---- device status word ---------------------------------------------------------------------------
+__device__ int g_status_word = 0;
+
+int *device_status_ptr() {
+    // the symbol has one instance per device; its address is looked up once per device
+    static int *cache[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (!cache[dev]) {
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_status_word) != cudaSuccess) return nullptr;
+        cache[dev] = static_cast<int *>(p);
+    }
+    return cache[dev];
+}
+
+namespace {
+
+constexpr size_t kAlign = 256;
+constexpr int kMaxDynSmem = 227 * 1024;
+
+inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline bool good_ptr(const void *p) { return p != nullptr && aligned16(p); }
+inline size_t esize(int dtype) { return dtype == MOC_BF16 ? 2 : 4; }
+
+int check_desc(const moc_ffn_desc *d) {
+    if (!d) return MOC_ERR_INVALID_ARG;
+    if (d->tokens < 0 || d->d_model < 1 || d->d_ff < 1 || d->d_ff_ld < d->d_ff || d->k < 1 || d->k > d->d_ff)
+        return MOC_ERR_INVALID_ARG;
+    if (d->dtype != MOC_F32 && d->dtype != MOC_BF16) return MOC_ERR_UNSUPPORTED;
+    if (d->flags & ~MOC_FLAG_ACCUMULATE_WGRAD) return MOC_ERR_INVALID_ARG;
+    if (d->d_ff > 32768) return MOC_ERR_UNSUPPORTED;     // int16 channel indices
+    if (d->d_model % 8 != 0) return MOC_ERR_UNSUPPORTED;  // 16-byte row vectors
+    if ((double)d->tokens * (double)d->k >= 4294967296.0) return MOC_ERR_UNSUPPORTED;  // 32-bit pair ids
+    return MOC_OK;
+}
+
+// ---- workspace layouts ------------------------------------------------------------------------------
+struct Carver {
+    size_t off = 0;
+    size_t take(size_t bytes) {
+        size_t o = off;
+        off = align_up(off + bytes, kAlign);
+        return o;
+    }
+};
+
+struct ForwardPlan {
+    int64_t chunk;   // tokens per gate-projection chunk
+    size_t off_g;    // fp32 [chunk, F]
+    size_t off_idx;  // int16 [T, K] when the caller keeps nothing
+    size_t total;
+};
+
+ForwardPlan plan_forward(const moc_ffn_desc &d) {
+    ForwardPlan p{};
+    const size_t row = (size_t)d.d_ff * 4;
+    int64_t chunk = (int64_t)std::max<size_t>(1, ((size_t)256 << 20) / row);
+    chunk = std::min<int64_t>(chunk, 1 << 20);  // keeps the gate GEMM's grid.y in range
+    p.chunk = std::max<int64_t>(1, std::min<int64_t>(d.tokens, chunk));
+    Carver c;
+    p.off_g = c.take((size_t)p.chunk * row);
+    p.off_idx = c.take((size_t)d.tokens * d.k * sizeof(int16_t));
+    p.total = c.off;
+    return p;
+}
+
+struct BackwardPlan {
+    int tb, nb;  // tokens per block / number of token blocks of the channel-list build
+    size_t off_coef, off_counts, off_totals, off_rowstart, off_pairs, total;
+};
+
+BackwardPlan plan_backward(const moc_ffn_desc &d) {
+    BackwardPlan p{};
+    const int64_t T = d.tokens;
+    int64_t nb = std::min<int64_t>(1184, (T + 7) / 8);
+    nb = std::max<int64_t>(1, nb);
+    p.tb = (int)((T + nb - 1) / nb);
+    if (p.tb < 1) p.tb = 1;
+    p.nb = (int)((T + p.tb - 1) / p.tb);
+    if (p.nb < 1) p.nb = 1;
+    const size_t TK = (size_t)T * d.k;
+    Carver c;
+    p.off_coef = c.take(3 * TK * sizeof(float));
+    p.off_counts = c.take((size_t)p.nb * d.d_ff * sizeof(uint32_t));
+    p.off_totals = c.take((size_t)d.d_ff * sizeof(uint32_t));
+    p.off_rowstart = c.take(((size_t)d.d_ff + 1) * sizeof(uint32_t));
+    p.off_pairs = c.take(TK * sizeof(uint32_t));
+    p.total = c.off;
+    return p;
+}
+
+template <typename K>
+int set_smem(K kernel, size_t bytes) {
+    if (bytes > (size_t)kMaxDynSmem) return MOC_ERR_UNSUPPORTED;
+    if (bytes > 48 * 1024) {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess)
+            return MOC_ERR_CUDA;
+    }
+    return MOC_OK;
+}
+
+inline int launch_ok() { return cudaGetLastError() == cudaSuccess ? MOC_OK : MOC_ERR_CUDA; }
+
+size_t token_red_floats(int d) {
+    const int nvec = d / 8;
+    const int lanes_v = std::min(nvec, kTokenThreads);
+    const int G = kTokenThreads / lanes_v;
+    return G > 1 ? (size_t)G * d : 0;
+}
+
+// ---- forward (gathered plan) -------------------------------------------------------------------------
+template <typename T>
+int forward_gather(const moc_ffn_desc &d, const T *x, const T *wg, const T *wu, const T *wd, T *out,
+                   int16_t *idx, T *tg, T *tu, char *ws, cudaStream_t st) {
+    const ForwardPlan p = plan_forward(d);
+    float *G = reinterpret_cast<float *>(ws + p.off_g);
+    if (!idx) idx = reinterpret_cast<int16_t *>(ws + p.off_idx);
+    const int F = d.d_ff, K = d.k, dm = d.d_model;
+
+    const size_t sel_smem = (size_t)F * sizeof(uint32_t);
+    int rc = set_smem(select_rows_kernel<T>, sel_smem);
+    if (rc != MOC_OK) return rc;
+    const size_t tok_smem = ((size_t)dm + 2 * (size_t)K + token_red_floats(dm)) * sizeof(float);
+    rc = set_smem(forward_token_kernel<T>, tok_smem);
+    if (rc != MOC_OK) return rc;
+
+    for (int64_t t0 = 0; t0 < d.tokens; t0 += p.chunk) {
+        const int64_t n = std::min<int64_t>(p.chunk, d.tokens - t0);
+        dim3 grid((F + 63) / 64, (unsigned)((n + 63) / 64));
+        gemm_nt_alu_kernel<T><<<grid, 256, 0, st>>>(x + t0 * dm, wg, G, (int)n, F, dm, F);
+        if ((rc = launch_ok()) != MOC_OK) return rc;
+        const unsigned sel_grid = (unsigned)std::min<int64_t>(n, 148 * 32);
+        select_rows_kernel<T><<<sel_grid, kSelectThreads, sel_smem, st>>>(G, n, F, F, K, idx + t0 * K,
+                                                                           tg ? tg + t0 * K : nullptr);
+        if ((rc = launch_ok()) != MOC_OK) return rc;
+        forward_token_kernel<T><<<(unsigned)n, kTokenThreads, tok_smem, st>>>(
+            x + t0 * dm, wu, wd, G, F, idx + t0 * K, dm, K, out + t0 * dm, tu ? tu + t0 * K : nullptr, 0);
+        if ((rc = launch_ok()) != MOC_OK) return rc;
+    }
+    return MOC_OK;
+}
+
+// ---- backward (gathered plan) ------------------------------------------------------------------------
+template <typename T>
+int backward_gather(const moc_ffn_desc &d, const T *x, const T *wg, const T *wu, const T *wd,
+                    const int16_t *idx, const T *tg, const T *tu, const T *dout, T *gx, T *gwg, T *gwu, T *gwd,
+                    char *ws, cudaStream_t st) {
+    const BackwardPlan p = plan_backward(d);
+    const int F = d.d_ff, K = d.k, dm = d.d_model;
+    const int64_t TK = d.tokens * (int64_t)K;
+    const bool want_w = gwg || gwu || gwd;
+    float *coef = reinterpret_cast<float *>(ws + p.off_coef);
+    int *status = device_status_ptr();
+    if (!status) return MOC_ERR_CUDA;
+
+    const size_t tok_smem = ((size_t)dm + 3 * (size_t)K + token_red_floats(dm)) * sizeof(float);
+    int rc = set_smem(backward_token_kernel<T>, tok_smem);
+    if (rc != MOC_OK) return rc;
+    backward_token_kernel<T><<<(unsigned)d.tokens, kTokenThreads, tok_smem, st>>>(
+        wg, wu, wd, idx, tg, tu, dout, dm, F, K, TK, gx, want_w ? coef : nullptr, status);
+    if ((rc = launch_ok()) != MOC_OK) return rc;
+    if (!want_w) return MOC_OK;
+
+    uint32_t *counts = reinterpret_cast<uint32_t *>(ws + p.off_counts);
+    uint32_t *totals = reinterpret_cast<uint32_t *>(ws + p.off_totals);
+    uint32_t *row_start = reinterpret_cast<uint32_t *>(ws + p.off_rowstart);
+    uint32_t *pairs = reinterpret_cast<uint32_t *>(ws + p.off_pairs);
+    const size_t f_smem = (size_t)F * sizeof(uint32_t);
+    if ((rc = set_smem(csr_count_kernel, f_smem)) != MOC_OK) return rc;
+    if ((rc = set_smem(csr_fill_kernel, f_smem)) != MOC_OK) return rc;
+    csr_count_kernel<<<p.nb, 256, f_smem, st>>>(idx, d.tokens, K, F, p.tb, counts);
+    if ((rc = launch_ok()) != MOC_OK) return rc;
+    csr_scan_blocks_kernel<<<(F + 255) / 256, 256, 0, st>>>(counts, p.nb, F, totals);
+    if ((rc = launch_ok()) != MOC_OK) return rc;
+    csr_scan_channels_kernel<<<1, 1024, 0, st>>>(totals, F, row_start);
+    if ((rc = launch_ok()) != MOC_OK) return rc;
+    csr_fill_kernel<<<p.nb, 256, f_smem, st>>>(idx, d.tokens, K, F, p.tb, counts, row_start, pairs);
+    if ((rc = launch_ok()) != MOC_OK) return rc;
+
+    const size_t red = token_red_floats(dm) * 3 * sizeof(float);
+    if ((rc = set_smem(wgrad_rows_kernel<T>, red)) != MOC_OK) return rc;
+    wgrad_rows_kernel<T><<<d.d_ff_ld, kTokenThreads, red, st>>>(x, dout, coef, TK, row_start, pairs, dm, F, K, gwg,
+                                                                  gwu, gwd,
+                                                                  (d.flags & MOC_FLAG_ACCUMULATE_WGRAD) ? 1 : 0);
+    return launch_ok();
+}
+
+}  // namespace
+}  // namespace moc
+
+using namespace moc;
+
+// =====================================================================================================
+extern "C" {
+
+size_t moc_ffn_workspace_bytes(const moc_ffn_desc *desc, int op) {
+    if (check_desc(desc) != MOC_OK) return 0;
+    if (desc->tokens == 0) return 0;
+    switch (op) {
+        case MOC_OP_FORWARD:
+            return plan_forward(*desc).total;
+        case MOC_OP_DECODE:
+            if (desc->tokens > 16) return 0;
+            return plan_forward(*desc).total;
+        case MOC_OP_BACKWARD:
+            return plan_backward(*desc).total;
+        default:
+            return 0;
+    }
+}
+
+size_t moc_ffn_saved_bytes_per_token(const moc_ffn_desc *desc) {
+    if (check_desc(desc) != MOC_OK) return 0;
+    return (size_t)desc->k * (sizeof(int16_t) + 2 * esize(desc->dtype));
+}
+
+int moc_ffn_forward(const moc_ffn_desc *desc, const void *x, const void *w_gate, const void *w_up,
+                    const void *w_down, void *out, int16_t *topk_idx, void *topk_gate, void *topk_up,
+                    void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    int rc = check_desc(desc);
+    if (rc != MOC_OK) return rc;
+    const bool save_all = topk_idx && topk_gate && topk_up;
+    const bool save_none = !topk_idx && !topk_gate && !topk_up;
+    if (!save_all && !save_none) return MOC_ERR_INVALID_ARG;
+    if (desc->tokens == 0) return MOC_OK;
+    if (!good_ptr(x) || !good_ptr(w_gate) || !good_ptr(w_up) || !good_ptr(w_down) || !good_ptr(out))
+        return MOC_ERR_INVALID_ARG;
+    if (save_all && (!aligned16(topk_idx) || !aligned16(topk_gate) || !aligned16(topk_up)))
+        return MOC_ERR_INVALID_ARG;
+    const size_t need = moc_ffn_workspace_bytes(desc, MOC_OP_FORWARD);
+    if (need && (!good_ptr(workspace) || workspace_bytes < need)) return MOC_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    char *ws = static_cast<char *>(workspace);
+    if (desc->dtype == MOC_BF16) {
+        using T = __nv_bfloat16;
+        return forward_gather<T>(*desc, (const T *)x, (const T *)w_gate, (const T *)w_up, (const T *)w_down,
+                                 (T *)out, topk_idx, (T *)topk_gate, (T *)topk_up, ws, st);
+    }
+    return forward_gather<float>(*desc, (const float *)x, (const float *)w_gate, (const float *)w_up,
+                                 (const float *)w_down, (float *)out, topk_idx, (float *)topk_gate,
+                                 (float *)topk_up, ws, st);
+}
+
+int moc_ffn_backward(const moc_ffn_desc *desc, const void *x, const void *w_gate, const void *w_up,
+                     const void *w_down, const int16_t *topk_idx, const void *topk_gate, const void *topk_up,
+                     const void *grad_out, void *grad_x, void *grad_w_gate, void *grad_w_up, void *grad_w_down,
+                     void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    int rc = check_desc(desc);
+    if (rc != MOC_OK) return rc;
+    if (desc->tokens == 0) {
+        // no tokens: weight gradients are zero unless they accumulate
+        if (desc->flags & MOC_FLAG_ACCUMULATE_WGRAD) return MOC_OK;
+        cudaStream_t st0 = static_cast<cudaStream_t>(cuda_stream);
+        const size_t wbytes = (size_t)desc->d_ff_ld * desc->d_model * esize(desc->dtype);
+        void *gw[3] = {grad_w_gate, grad_w_up, grad_w_down};
+        for (void *g : gw) {
+            if (g && !aligned16(g)) return MOC_ERR_INVALID_ARG;
+        }
+        for (void *g : gw) {
+            if (g && cudaMemsetAsync(g, 0, wbytes, st0) != cudaSuccess) return MOC_ERR_CUDA;
+        }
+        return MOC_OK;
+    }
+    if (!good_ptr(x) || !good_ptr(w_gate) || !good_ptr(w_up) || !good_ptr(w_down) || !good_ptr(topk_idx) ||
+        !good_ptr(topk_gate) || !good_ptr(topk_up) || !good_ptr(grad_out))
+        return MOC_ERR_INVALID_ARG;
+    if (!aligned16(grad_x) || !aligned16(grad_w_gate) || !aligned16(grad_w_up) || !aligned16(grad_w_down))
+        return MOC_ERR_INVALID_ARG;
+    if (!grad_x && !grad_w_gate && !grad_w_up && !grad_w_down) return MOC_OK;
+    const size_t need = moc_ffn_workspace_bytes(desc, MOC_OP_BACKWARD);
+    if (need && (!good_ptr(workspace) || workspace_bytes < need)) return MOC_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    char *ws = static_cast<char *>(workspace);
+    if (desc->dtype == MOC_BF16) {
+        using T = __nv_bfloat16;
+        return backward_gather<T>(*desc, (const T *)x, (const T *)w_gate, (const T *)w_up, (const T *)w_down,
+                                  topk_idx, (const T *)topk_gate, (const T *)topk_up, (const T *)grad_out,
+                                  (T *)grad_x, (T *)grad_w_gate, (T *)grad_w_up, (T *)grad_w_down, ws, st);
+    }
+    using T = float;
+    return backward_gather<T>(*desc, (const T *)x, (const T *)w_gate, (const T *)w_up, (const T *)w_down,
+                              topk_idx, (const T *)topk_gate, (const T *)topk_up, (const T *)grad_out,
+                              (T *)grad_x, (T *)grad_w_gate, (T *)grad_w_up, (T *)grad_w_down, ws, st);
+}
+
+int moc_ffn_decode(const moc_ffn_desc *desc, const void *x, const void *w_gate, const void *w_up,
+                   const void *w_down, void *out, void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    int rc = check_desc(desc);
+    if (rc != MOC_OK) return rc;
+    if (desc->tokens > 16) return MOC_ERR_UNSUPPORTED;
+    return moc_ffn_forward(desc, x, w_gate, w_up, w_down, out, nullptr, nullptr, nullptr, workspace,
+                           workspace_bytes, cuda_stream);
+}
+
+int moc_topk_select(int64_t rows, int32_t n, int32_t n_ld, int32_t k, const float *gate, int16_t *idx_out,
+                    void *cuda_stream) {
+    if (rows < 0 || n < 1 || n_ld < n || k < 1 || k > n) return MOC_ERR_INVALID_ARG;
+    if (n > 32768) return MOC_ERR_UNSUPPORTED;
+    if (rows == 0) return MOC_OK;
+    if (!good_ptr(gate) || !idx_out || (reinterpret_cast<uintptr_t>(idx_out) & 1u)) return MOC_ERR_INVALID_ARG;
+    const size_t smem = (size_t)n * sizeof(uint32_t);
+    int rc = set_smem(topk_select_kernel<kSelectThreads>, smem);
+    if (rc != MOC_OK) return rc;
+    const unsigned grid = (unsigned)std::min<int64_t>(rows, 148 * 32);
+    topk_select_kernel<kSelectThreads><<<grid, kSelectThreads, smem, static_cast<cudaStream_t>(cuda_stream)>>>(
+        gate, rows, n, n_ld, k, idx_out);
+    return launch_ok();
+}
+
+int moc_last_device_status(void *cuda_stream) {
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return MOC_ERR_CUDA;
+    int *p = device_status_ptr();
+    if (!p) return MOC_ERR_CUDA;
+    int v = 0;
+    if (cudaMemcpy(&v, p, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return MOC_ERR_CUDA;
+    if (v != 0) {
+        if (cudaMemset(p, 0, sizeof(int)) != cudaSuccess) return MOC_ERR_CUDA;
+    }
+    return v;
+}
+
+const char *moc_status_string(int status) {
+    switch (status) {
+        case MOC_OK: return "ok";
+        case MOC_ERR_INVALID_ARG: return "invalid argument";
+        case MOC_ERR_UNSUPPORTED: return "unsupported shape or type";
+        case MOC_ERR_WORKSPACE: return "workspace missing or too small";
+        case MOC_ERR_CUDA: return "CUDA runtime error";
+        case MOC_ERR_TIMEOUT: return "a bounded device-side wait expired";
+        case MOC_ERR_BAD_INDEX: return "saved channel index out of range";
+        default: return "unknown status";
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,273 @@
+"""Parity of the CUDA library (called through its C ABI) with the CPU oracle on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import moc_oracle as orc
+from oracle import parity
+from paper_2511_09323_b200 import binding as B
+from paper_2511_09323_b200 import build as moc_build
+from paper_2511_09323_b200 import synthetic as syn
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    moc_build.build()
+    B.load()
+    assert B.moc_last_device_status() == B.MOC_OK
+    yield
+    assert B.moc_last_device_status() == B.MOC_OK
+
+
+def _dev(t):
+    return t.to("cuda")
+
+
+def _problem(w: syn.Workload):
+    wg, wu, wd = syn.make_weights(w)
+    x = syn.make_x(w)
+    dD = syn.make_grad_out(w)
+    return x, wg, wu, wd, dD
+
+
+def _run_forward_backward(w: syn.Workload, decode=False):
+    x, wg, wu, wd, dD = _problem(w)
+    xd, wgd, wud, wdd, dDd = map(_dev, (x, wg, wu, wd, dD))
+    out, idx, tg, tu = B.moc_ffn_forward(xd, wgd, wud, wdd, w.k, d_ff=w.d_ff)
+    torch.cuda.synchronize()
+    x64, wg64, wu64, wd64, dD64 = map(syn.to_f64, (x, wg, wu, wd, dD))
+    dev = dict(out=syn.to_f64(out), idx=idx.cpu().numpy(), gval=syn.to_f64(tg), uval=syn.to_f64(tu))
+    rep = parity.check_forward(dev, x64, wg64, wu64, wd64, w.k, w.d_ff, w.dtype)
+    grads = B.moc_ffn_backward(xd, wgd, wud, wdd, idx, tg, tu, dDd, d_ff=w.d_ff)
+    torch.cuda.synchronize()
+    gdev = {k: syn.to_f64(v) for k, v in grads.items()}
+    rep.update(parity.check_backward(gdev, x64, wg64, wu64, wd64, dev["idx"], dev["gval"], dev["uval"], dD64,
+                                     w.d_ff, w.dtype))
+    return rep, (xd, wgd, wud, wdd, dDd), (out, idx, tg, tu), grads
+
+
+# ------------------------------------------------------------------ selector alone: bit exact
+
+
+def _adversarial_rows(n):
+    r = np.arange(n, dtype=np.float32)
+    rows = [
+        np.zeros(n, np.float32),
+        r.copy(),
+        -r,
+        np.where(r % 3 == 0, 1.0, -1.0).astype(np.float32),
+        np.where(r % 2 == 0, 0.0, -0.0).astype(np.float32),
+        np.concatenate([[np.inf, -np.inf], np.linspace(-1, 1, n - 2)]).astype(np.float32),
+        np.full(n, -np.inf, np.float32),
+        np.where(r % 5 == 0, np.nan, np.sin(r)).astype(np.float32),
+        (np.round(np.random.default_rng(1).standard_normal(n) * 16) / 16).astype(np.float32),  # many duplicates
+        np.random.default_rng(2).standard_normal(n).astype(np.float32) * 1e-30,               # tiny magnitudes
+        np.float32(1e30) * np.random.default_rng(3).standard_normal(n).astype(np.float32),
+    ]
+    return np.stack(rows)
+
+
+@pytest.mark.parametrize("n,n_ld", [(1, 4), (37, 40), (256, 256), (257, 264), (2048, 2048), (5461, 5504), (32768, 32768)])
+def test_selector_bit_exact_adversarial(n, n_ld):
+    rows = _adversarial_rows(max(n, 3))[:, :n] if n >= 3 else np.zeros((3, n), np.float32)
+    g = np.full((rows.shape[0], n_ld), 1e9, np.float32)  # padding columns hold large values: must be ignored
+    g[:, :n] = rows
+    gd = torch.from_numpy(g).cuda()
+    for k in sorted({1, 2, max(1, n // 8), max(1, n - 1), n}):
+        if k > n:
+            continue
+        got = B.moc_topk_select(gd, k, n=n).cpu().numpy().astype(np.int32)
+        np.testing.assert_array_equal(got, orc.topk(g, k, F=n), err_msg=f"n={n} k={k}")
+
+
+@pytest.mark.parametrize("name", ["C1", "C2", "C3", "C4"])
+def test_selector_bit_exact_on_oracle_gate_values(name):
+    """The selector is fed float32(oracle gate values) of the configuration's shape."""
+    w = syn.WORKLOADS[name]
+    T = 48 if w.d_ff > 4000 else 96
+    wg, _, _ = syn.make_weights(w)
+    x = syn.make_x(w, tokens=T)
+    g64 = syn.to_f64(x) @ syn.to_f64(wg)[: w.d_ff].T
+    g32 = np.zeros((T, w.d_ff_ld), np.float32)
+    g32[:, : w.d_ff] = g64.astype(np.float32)
+    got = B.moc_topk_select(torch.from_numpy(g32).cuda(), w.k, n=w.d_ff).cpu().numpy().astype(np.int32)
+    np.testing.assert_array_equal(got, orc.topk(g32, w.k, F=w.d_ff))
+
+
+def test_selector_many_rows_grid_stride():
+    rng = np.random.default_rng(7)
+    g = rng.standard_normal((6000, 96)).astype(np.float32)  # more rows than the selector's grid
+    got = B.moc_topk_select(torch.from_numpy(g).cuda(), 12).cpu().numpy().astype(np.int32)
+    np.testing.assert_array_equal(got, orc.topk(g, 12))
+
+
+# ------------------------------------------------------------------ forward + backward
+
+
+def test_c1_tiny_fp32_forward_backward():
+    rep, *_ = _run_forward_backward(syn.C1)
+    assert rep["out"][0] <= 1e-4 * rep["out"][1]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("T,d,F,F_ld,K", [
+    (1, 8, 8, 8, 1),            # smallest legal shape
+    (3, 16, 40, 40, 39),        # K = F - 1
+    (5, 24, 33, 40, 33),        # K = F (dense SwiGLU) with a padded tail
+    (70, 264, 333, 336, 41),    # nothing a multiple of a tile
+    (300, 768, 520, 520, 65),   # several tiles + ragged tails
+])
+def test_ragged_shapes(dtype, T, d, F, F_ld, K):
+    w = syn.Workload(f"rag-{T}-{d}-{F}-{K}", dtype, T, d, F, F_ld, K, seed=100 + T)
+    _run_forward_backward(w)
+
+
+def test_llama130m_shape_bf16_slice():
+    """C2's layer shape on a token slice the oracle finishes in seconds."""
+    w = syn.C2.with_tokens(640)
+    rep, *_ = _run_forward_backward(w)
+    assert rep["tokens_with_band_picks"] <= 64
+
+
+def test_llama1b_shape_bf16_padded_slice():
+    """C3's layer shape: d_ff = 5461 in arrays of 5504 rows; the oracle runs the unpadded problem."""
+    w = syn.C3.with_tokens(96)
+    _run_forward_backward(w)
+
+
+def test_k_equals_dff_matches_dense_swiglu_formula():
+    w = syn.Workload("dense", "f32", 33, 64, 96, 96, 96, seed=5)
+    x, wg, wu, wd, _ = _problem(w)
+    out, idx, tg, tu = B.moc_ffn_forward(_dev(x), _dev(wg), _dev(wu), _dev(wd), w.k)
+    x64, wg64, wu64, wd64 = map(syn.to_f64, (x, wg, wu, wd))
+    G, U = x64 @ wg64.T, x64 @ wu64.T
+    dense = (G / (1 + np.exp(-G)) * U) @ wd64
+    parity.assert_close(syn.to_f64(out), dense, "f32", "dense SwiGLU")
+    np.testing.assert_array_equal(idx.cpu().numpy(), np.tile(np.arange(96, dtype=np.int16), (33, 1)))
+
+
+def test_inference_forward_saves_nothing_and_matches_training_forward():
+    w = syn.Workload("inf", "bf16", 50, 128, 256, 256, 32, seed=9)
+    x, wg, wu, wd, _ = map(_dev, _problem(w))
+    out_a, *_ = B.moc_ffn_forward(x, wg, wu, wd, w.k, save=True)
+    out_b, idx, tg, tu = B.moc_ffn_forward(x, wg, wu, wd, w.k, save=False)
+    assert idx is None and tg is None and tu is None
+    assert torch.equal(out_a, out_b)
+
+
+def test_forward_and_backward_are_deterministic():
+    w = syn.Workload("det", "bf16", 257, 128, 300, 304, 40, seed=3)
+    _, (x, wg, wu, wd, dD), (out, idx, tg, tu), g1 = _run_forward_backward(w)
+    out2, idx2, tg2, tu2 = B.moc_ffn_forward(x, wg, wu, wd, w.k, d_ff=w.d_ff)
+    assert torch.equal(out, out2) and torch.equal(idx, idx2) and torch.equal(tg, tg2) and torch.equal(tu, tu2)
+    g2 = B.moc_ffn_backward(x, wg, wu, wd, idx, tg, tu, dD, d_ff=w.d_ff)
+    for k in g1:
+        assert torch.equal(g1[k], g2[k]), k
+
+
+def test_backward_partial_outputs_and_accumulate_flag():
+    w = syn.Workload("acc", "f32", 64, 64, 128, 128, 16, seed=8)
+    _, (x, wg, wu, wd, dD), (out, idx, tg, tu), full = _run_forward_backward(w)
+    part = B.moc_ffn_backward(x, wg, wu, wd, idx, tg, tu, dD, want=("w_up",))
+    assert part["grad_x"] is None and part["grad_w_down"] is None
+    assert torch.equal(part["grad_w_up"], full["grad_w_up"])
+    only_x = B.moc_ffn_backward(x, wg, wu, wd, idx, tg, tu, dD, want=("x",))
+    assert torch.equal(only_x["grad_x"], full["grad_x"])
+    base = {k: torch.full_like(v, 0.5) for k, v in full.items() if k != "grad_x"}
+    acc = B.moc_ffn_backward(x, wg, wu, wd, idx, tg, tu, dD, want=("w_gate", "w_up", "w_down"), grads=base,
+                             accumulate=True)
+    for k in ("grad_w_gate", "grad_w_up", "grad_w_down"):
+        torch.testing.assert_close(acc[k], full[k] + 0.5, rtol=1e-6, atol=1e-6)
+    # rows of channels no token selected are exactly zero
+    used = torch.zeros(w.d_ff, dtype=torch.bool, device="cuda")
+    used[idx.long().flatten()] = True
+    if (~used).any():
+        for k in ("grad_w_gate", "grad_w_up", "grad_w_down"):
+            assert torch.all(full[k][~used] == 0)
+
+
+def test_corrupted_saved_index_is_skipped_and_reported():
+    w = syn.Workload("bad", "bf16", 40, 64, 96, 96, 8, seed=12)
+    _, (x, wg, wu, wd, dD), (out, idx, tg, tu), full = _run_forward_backward(w)
+    bad = idx.clone()
+    bad[3, 2] = 96       # == d_ff: out of range
+    bad[7, 0] = -5
+    assert B.moc_last_device_status() == B.MOC_OK
+    g = B.moc_ffn_backward(x, wg, wu, wd, bad, tg, tu, dD)
+    assert B.moc_last_device_status() == B.MOC_ERR_BAD_INDEX
+    assert B.moc_last_device_status() == B.MOC_OK      # reading clears it
+    # the other tokens' grad_x rows are untouched by the corruption
+    keep = torch.ones(w.tokens, dtype=torch.bool, device="cuda")
+    keep[3] = keep[7] = False
+    assert torch.equal(g["grad_x"][keep], full["grad_x"][keep])
+    assert torch.isfinite(g["grad_w_down"].float()).all()
+
+
+def test_host_errors_raise_before_launch():
+    w = syn.Workload("err", "bf16", 8, 64, 96, 96, 8, seed=1)
+    x, wg, wu, wd, _ = map(_dev, _problem(w))
+    with pytest.raises(B.MocError) as e:
+        B.moc_ffn_forward(x, wg, wu, wd, 97)
+    assert e.value.status == B.MOC_ERR_INVALID_ARG
+    with pytest.raises(B.MocError) as e:
+        B.moc_ffn_forward(x, wg, wu, wd, 8, workspace=torch.empty(16, dtype=torch.uint8, device="cuda"))
+    assert e.value.status == B.MOC_ERR_WORKSPACE
+    with pytest.raises(B.MocError) as e:
+        B.moc_ffn_decode(_dev(syn.make_x(w, tokens=17)), wg, wu, wd, 8)
+    assert e.value.status == B.MOC_ERR_UNSUPPORTED
+    assert B.moc_last_device_status() == B.MOC_OK
+
+
+def test_zero_tokens_is_a_noop():
+    x = torch.empty((0, 64), dtype=torch.bfloat16, device="cuda")
+    wg = torch.zeros((32, 64), dtype=torch.bfloat16, device="cuda")
+    out, idx, tg, tu = B.moc_ffn_forward(x, wg, wg, wg, 4)
+    assert out.shape == (0, 64) and idx.shape == (0, 4)
+
+
+# ------------------------------------------------------------------ decode
+
+
+def _check_decode(out64, x64, wg64, wu64, wd64, K, dtype, what):
+    """Decode returns no indices, so the comparison is with the oracle's own picks.  Where a token's margin
+    between its K-th and (K+1)-th gate value is below 1e-4 (inside the 1e-3 exclusion band) the swapped pick
+    is accepted as well; every other token must match within the tolerance."""
+    full = orc.forward(x64, wg64, wu64, wd64, K, want_g=True)
+    F = wg64.shape[0]
+    scale = np.abs(full["out"]).max()
+    tol = parity.REL_TOL[dtype] * scale
+    for t in range(x64.shape[0]):
+        err = np.abs(out64[t] - full["out"][t]).max()
+        if err <= tol:
+            continue
+        g = full["g"][t]
+        order = np.lexsort((np.arange(F), -g))
+        assert K < F and g[order[K - 1]] - g[order[K]] <= 1e-4, f"{what}: token {t} error {err:.3e} > {tol:.3e}"
+        alt = np.sort(np.concatenate([order[: K - 1], order[K: K + 1]])).astype(np.int32)[None]
+        ref = orc.forward_given_idx(x64[t: t + 1], wg64, wu64, wd64, alt)["out"][0]
+        assert np.abs(out64[t] - ref).max() <= tol, f"{what}: token {t} matches neither pick"
+
+
+@pytest.mark.parametrize("T", [1, 4, 16])
+def test_decode_llama7b_shape(T):
+    w = syn.C4.with_tokens(T)
+    wg, wu, wd = syn.make_weights(w)
+    x = syn.make_x(w)
+    out = B.moc_ffn_decode(_dev(x), _dev(wg), _dev(wu), _dev(wd), w.k)
+    torch.cuda.synchronize()
+    x64, wg64, wu64, wd64 = map(syn.to_f64, (x, wg, wu, wd))
+    _check_decode(syn.to_f64(out), x64, wg64, wu64, wd64, w.k, "bf16", f"decode T={T}")
+
+
+@pytest.mark.parametrize("dtype,T,d,F,K", [("f32", 3, 64, 200, 25), ("bf16", 16, 256, 1000, 125), ("bf16", 7, 520, 777, 97)])
+def test_decode_small_shapes(dtype, T, d, F, K):
+    w = syn.Workload("dec", dtype, T, d, F, F, K, seed=77, decode=True)
+    wg, wu, wd = syn.make_weights(w)
+    x = syn.make_x(w)
+    out = B.moc_ffn_decode(_dev(x), _dev(wg), _dev(wu), _dev(wd), K)
+    out_f, *_ = B.moc_ffn_forward(_dev(x), _dev(wg), _dev(wu), _dev(wd), K, save=False)
+    x64, wg64, wu64, wd64 = map(syn.to_f64, (x, wg, wu, wd))
+    _check_decode(syn.to_f64(out), x64, wg64, wu64, wd64, K, dtype, "decode")
+    _check_decode(syn.to_f64(out_f), x64, wg64, wu64, wd64, K, dtype, "forward(save=False)")
