@@ -1,0 +1,498 @@
+#!/usr/bin/env python
+"""Benchmark of the MoC FFN hot path on B200.
+
+One "step" is one pass of the training hot path -- moc_ffn_forward followed by moc_ffn_backward
+(all four gradients) -- over one batch of the LLaMA-130M-shaped workload (16384 tokens, d_model 768,
+d_ff 2048, K 256, bf16 storage with fp32 accumulation), called through the C ABI.  The line printed
+by rank 0 also carries: the end-to-end number with host buffers (``e2e``), the roofline of the
+dominant kernel measured with CUDA events inside the timed region (``roofline``), the CPU oracle
+timed on this machine's host cores (``cpu_baseline``), small-batch decode latencies on the LLaMA-7B
+shape (``decode``) and the saved-activation bytes (``act_bytes``).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+With N > 1 it is launched by torchrun, one rank per GPU; every rank runs the same per-GPU batch
+(weak scaling, tokens are independent, no data-path collective).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "moc_ffn_fwd_bwd_tokens_per_s"
+UNIT = "tokens/s"
+ALU_FP32_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12   # 148 SMs x 128 FMA lanes x 2 flop x max SM clock
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def parse_args():
+    p = argparse.ArgumentParser()
+    p.add_argument("--gpus", type=int, default=1)
+    p.add_argument("--steps", type=int, default=20)
+    p.add_argument("--warmup", type=int, default=5)
+    p.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    p.add_argument("--workload", default="C2", choices=["C1", "C2", "C3", "C5"])
+    p.add_argument("--tokens", type=int, default=0, help="override the workload's token count (debugging)")
+    p.add_argument("--no-decode", action="store_true")
+    p.add_argument("--no-cpu-baseline", action="store_true")
+    p.add_argument("--cpu-seconds", type=float, default=15.0, help="target seconds of oracle work")
+    return p.parse_args()
+
+
+# ------------------------------------------------------------------------------------------------ helpers
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            d = json.load(fh)
+        return {k: float(d[k]) for k in FALLBACK_PEAKS if k in d} | {"source": "measured"}
+    return dict(FALLBACK_PEAKS) | {"source": "fallback"}
+
+
+def shard_plan(world: int, rank: int, tokens_per_gpu: int):
+    """Weak scaling: every rank owns `tokens_per_gpu` independent tokens; returns (global offset, count)."""
+    if world < 1 or not 0 <= rank < world:
+        raise ValueError("bad world/rank")
+    return rank * tokens_per_gpu, tokens_per_gpu
+
+
+def aggregate(total_ms_per_rank, tokens_per_rank, steps):
+    """Whole-job throughput from per-rank timings: all tokens / slowest rank's time."""
+    worst = max(total_ms_per_rank)
+    tokens = sum(tokens_per_rank) * steps
+    return tokens / (worst / 1e3), worst / steps
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons of one GPU while a region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, uuid: str | None):
+        self.uuid = uuid
+        self.proc = None
+        self.tmp = None
+
+    def start(self):
+        try:
+            self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+            cmd = ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100"]
+            if self.uuid:
+                cmd.insert(1, f"--id={self.uuid}")
+            self.proc = subprocess.Popen(cmd, stdout=self.tmp, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if not self.proc:
+            return out
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.tmp.flush()
+        self.tmp.seek(0)
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.tmp.read().splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                smax.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        self.tmp.close()
+        try:
+            os.unlink(self.tmp.name)
+        except OSError:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(smax), reasons=sorted(reasons),
+                       samples=len(sm))
+        return out
+
+
+def kernel_work(name: str, T: int, d: int, F: int, K: int, e: int):
+    """Algorithmic work of one step's launches of a kernel: (bound, amount, unit of amount).
+
+    Per-token figures (d = d_model, F = d_ff, e = bytes per element):
+      gate projection 2dF flop; selection reads F fp32 and writes K (idx + value);
+      gathered up + down 4Kd flop; backward per-token part 6Kd flop (dz, and both terms of grad_x);
+      weight gradients 6Kd flop.
+    """
+    table = {
+        "gate_gemm_alu": ("tensor", 2.0 * T * d * F, "flop"),
+        "gate_up_gemm_tc": ("tensor", 4.0 * T * d * F, "flop"),
+        "select_rows": ("hbm", T * F * 4.0 + T * K * (2.0 + e), "byte"),
+        "forward_token": ("alu", 4.0 * T * K * d, "flop"),
+        "backward_token": ("alu", 6.0 * T * K * d, "flop"),
+        "wgrad_rows": ("alu", 6.0 * T * K * d, "flop"),
+        "csr_count": ("hbm", T * K * 2.0, "byte"),
+        "csr_fill": ("hbm", T * K * 6.0, "byte"),
+    }
+    return table.get(name)
+
+
+# ------------------------------------------------------------------------------------------------ reference arm
+
+
+def oracle_step_fn(w, tokens):
+    """Returns (callable running the oracle's forward+backward on `tokens` tokens, thread count)."""
+    import numpy as np
+    from oracle import moc_oracle as orc
+    from paper_2511_09323_b200 import synthetic as syn
+    wg, wu, wd = (syn.to_f64(t) for t in syn.make_weights(w))
+    x = syn.to_f64(syn.make_x(w, tokens=tokens))
+    dD = syn.to_f64(syn.make_grad_out(w, tokens=tokens))
+
+    def run():
+        f = orc.forward(x, wg, wu, wd, w.k, F=w.d_ff)
+        gv = syn.round_to(f["gval"], w.dtype)
+        uv = syn.round_to(f["uval"], w.dtype)
+        g = orc.backward(x, wg, wu, wd, f["idx"], gv, uv, dD, F=w.d_ff)
+        return float(np.abs(g["grad_x"]).max())
+
+    return run, orc.num_threads()
+
+
+def calibrate_oracle_tokens(w, target_s, cap):
+    """Token count whose oracle forward+backward takes about target_s on this host."""
+    probe = min(cap, 64)
+    run, threads = oracle_step_fn(w, probe)
+    t0 = time.perf_counter()
+    run()
+    dt = max(time.perf_counter() - t0, 1e-4)
+    # the weight-gradient phase has a fixed F*d cost; scale only the per-token part conservatively
+    n = int(max(probe, min(cap, probe * target_s / dt)))
+    return max(16, n - n % 16), threads
+
+
+def run_reference(args):
+    from paper_2511_09323_b200 import synthetic as syn
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    w = syn.WORKLOADS[args.workload]
+    per_step_target = max(0.5, min(4.0, 120.0 / max(1, args.steps + args.warmup)))
+    n, threads = calibrate_oracle_tokens(w, per_step_target, w.tokens)
+    run, threads = oracle_step_fn(w, n)
+    for _ in range(args.warmup):
+        run()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        run()
+    dt = time.perf_counter() - t0
+    value = n * args.steps / dt
+    sample = f"first {n} of {w.tokens} tokens of {w.name} per step, fp64 oracle forward+backward"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(w, w.tokens, {"reference_sample_tokens_per_step": n}),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+    return 0
+
+
+def workload_config(w, tokens, extra=None):
+    cfg = {"workload": f"{w.name}: MoC FFN forward+backward, tokens={tokens}"
+                       + (f" (batch {w.batch} x seq {w.seq})" if w.batch and tokens == w.tokens else ""),
+           "tokens_per_gpu": tokens, "d_model": w.d_model, "d_ff": w.d_ff, "d_ff_ld": w.d_ff_ld, "k": w.k,
+           "storage": w.dtype, "accumulate": "f32"}
+    if extra:
+        cfg.update(extra)
+    return cfg
+
+
+# ------------------------------------------------------------------------------------------------ our arm
+
+
+def run_ours(args):
+    import torch
+    from paper_2511_09323_b200 import binding as B
+    from paper_2511_09323_b200 import build as moc_build
+    from paper_2511_09323_b200 import synthetic as syn
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device (there is no CPU path)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=dev)
+    if rank == 0:
+        moc_build.build()
+    if dist:
+        dist.barrier()
+    B.load()
+
+    w = syn.WORKLOADS[args.workload]
+    T = args.tokens or w.tokens
+    _, T = shard_plan(world, rank, T)
+    e = 2 if w.dtype == "bf16" else 4
+    wg, wu, wd = (t.to(dev) for t in syn.make_weights(w))
+    x_h = syn.make_x(w, tokens=T).pin_memory()
+    dD_h = syn.make_grad_out(w, tokens=T).pin_memory()
+    x, dD = x_h.to(dev), dD_h.to(dev)
+    out = torch.empty_like(x)
+    saved = (torch.empty((T, w.k), dtype=torch.int16, device=dev), torch.empty((T, w.k), dtype=x.dtype, device=dev),
+             torch.empty((T, w.k), dtype=x.dtype, device=dev))
+    grads = {"grad_x": torch.empty_like(x), "grad_w_gate": torch.empty_like(wg),
+             "grad_w_up": torch.empty_like(wu), "grad_w_down": torch.empty_like(wd)}
+    desc = B.make_desc(T, w.d_model, w.d_ff, w.k, x.dtype, d_ff_ld=w.d_ff_ld)
+    ws_f = B.alloc_workspace(desc, B.MOC_OP_FORWARD, dev)
+    ws_b = B.alloc_workspace(desc, B.MOC_OP_BACKWARD, dev)
+    out_h = torch.empty_like(x_h).pin_memory()
+    gx_h = torch.empty_like(x_h).pin_memory()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)   # 2 x L2
+
+    def step(xd, dd):
+        B.moc_ffn_forward(xd, wg, wu, wd, w.k, d_ff=w.d_ff, out=out, saved=saved, workspace=ws_f)
+        B.moc_ffn_backward(xd, wg, wu, wd, saved[0], saved[1], saved[2], dd, d_ff=w.d_ff, grads=grads,
+                           workspace=ws_b)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        flush.zero_()
+        step(x, dD)
+    barrier()
+    if B.moc_last_device_status() != B.MOC_OK:
+        raise RuntimeError("device status raised during warm-up")
+
+    # ---- timed region: K steps, L2 flushed between steps (outside the event pairs) -------------
+    uuid = None
+    try:
+        uuid = "GPU-" + str(torch.cuda.get_device_properties(dev).uuid)
+    except Exception:
+        pass
+    sampler = ClockSampler(uuid)
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    launches0 = B.moc_launch_count()
+    B.moc_profile_enable(True)
+    barrier()
+    sampler.start()
+    for s, t in ev:
+        flush.zero_()
+        s.record()
+        step(x, dD)
+        t.record()
+    barrier()
+    clocks = sampler.stop()
+    prof = B.moc_profile_collect()
+    B.moc_profile_enable(False)
+    launches = B.moc_launch_count() - launches0
+    step_ms = [s.elapsed_time(t) for s, t in ev]
+    total_ms = sum(step_ms)
+
+    # ---- end to end: host buffers in, host buffers out, copies inside the timed region ----------
+    x_d2, dD_d2 = torch.empty_like(x), torch.empty_like(dD)
+    ev2 = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+
+    def e2e_step():
+        x_d2.copy_(x_h, non_blocking=True)
+        dD_d2.copy_(dD_h, non_blocking=True)
+        step(x_d2, dD_d2)
+        out_h.copy_(out, non_blocking=True)
+        gx_h.copy_(grads["grad_x"], non_blocking=True)
+
+    e2e_step()
+    barrier()
+    for s, t in ev2:
+        flush.zero_()
+        s.record()
+        e2e_step()
+        t.record()
+    barrier()
+    e2e_total_ms = sum(s.elapsed_time(t) for s, t in ev2)
+    h2d = x_h.numel() * e * 2
+    d2h = out_h.numel() * e * 2
+
+    # ---- aggregate over ranks (max time, sum tokens) ---------------------------------------------
+    tot = torch.tensor([total_ms, e2e_total_ms], dtype=torch.float64, device=dev)
+    if dist:
+        dist.all_reduce(tot, op=dist.ReduceOp.MAX)
+    worst_ms, worst_e2e_ms = tot.tolist()
+    value = world * T * args.steps / (worst_ms / 1e3)
+    e2e_value = world * T * args.steps / (worst_e2e_ms / 1e3)
+
+    status = B.moc_last_device_status()
+    if status != B.MOC_OK:
+        raise RuntimeError(f"device status {status} after the timed region")
+
+    line = None
+    if rank == 0:
+        peaks = load_peaks()
+        roof, kernels = roofline_report(prof, args.steps, T, w, e, peaks)
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": worst_ms / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32",
+            "data": "synthetic",
+            "config": workload_config(w, T, {"l2": "flushed between steps by a 256 MiB write outside the timed events",
+                                             "parallelism": f"token-sharded x{world}, no collective"}),
+            "clocks": {k: clocks[k] for k in ("sm_mhz", "sm_max_mhz", "reasons")},
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "ms_per_step": worst_e2e_ms / args.steps},
+            "gpu_launches": launches,
+            "roofline": roof,
+            "kernels": kernels,
+            "step_ms_min_median": [min(step_ms), statistics.median(step_ms)],
+            "act_bytes": act_bytes_report(w, T, e, saved, B, desc),
+            "strict_roofline": strict_roofline(w, T, e, worst_ms / args.steps, peaks),
+        }
+    # ---- decode (rank 0, after the training timing) ----------------------------------------------
+    if rank == 0 and not args.no_decode:
+        del flush, ws_f, ws_b
+        torch.cuda.empty_cache()
+        try:
+            line["decode"] = decode_report(torch, B, syn, dev, load_peaks())
+        except Exception as exc:  # the training number stands on its own
+            line["decode"] = {"error": repr(exc)}
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        n, threads = calibrate_oracle_tokens(w, args.cpu_seconds, T)
+        run, threads = oracle_step_fn(w, n)
+        t0 = time.perf_counter()
+        run()
+        dt = time.perf_counter() - t0
+        line["cpu_baseline"] = {"value": n / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
+                                "sample": f"first {n} of {T} tokens, fp64 oracle forward+backward, {dt:.1f} s"}
+    if dist:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(line))
+    return 0
+
+
+def roofline_report(prof, steps, T, w, e, peaks):
+    """Roofline of the kernel with the largest share of the timed region + a per-kernel table."""
+    kernels = {}
+    total = sum(ms for k, (n, ms) in prof.items() if not k.startswith("_")) or 1.0
+    for name, (n, ms) in prof.items():
+        if name.startswith("_"):
+            continue
+        kernels[name] = {"launches": n, "total_ms": round(ms, 4), "share": round(ms / total, 4)}
+    if not kernels:
+        return None, kernels
+    top = max(kernels, key=lambda k: kernels[k]["total_ms"])
+    n, ms = prof[top]
+    work = kernel_work(top, T, w.d_model, w.d_ff, w.k, e)
+    roof = {"kernel": top, "launches": n, "avg_ms": ms / n}
+    if work:
+        bound, amount, unit = work
+        per_launch = amount * steps / n          # `amount` is per step
+        rate = per_launch / (ms / n / 1e3)
+        if bound == "hbm":
+            roof.update(bound="hbm", achieved=rate / 1e9, peak=peaks["hbm_gbs"], unit="GB/s")
+        elif bound == "tensor":
+            roof.update(bound="tensor", achieved=rate / 1e12, peak=peaks["bf16_tflops_sustained"], unit="TFLOP/s")
+        else:
+            roof.update(bound="alu", achieved=rate / 1e12, peak=ALU_FP32_PEAK_TFLOPS, unit="TFLOP/s")
+        roof["frac"] = roof["achieved"] / roof["peak"]
+        roof["peak_source"] = peaks["source"] if bound != "alu" else "derived: 148 SM x 128 lanes x 2 x 1.965 GHz"
+        roof["algorithmic_per_launch"] = per_launch
+    roof["traffic"] = None
+    return roof, kernels
+
+
+def strict_roofline(w, T, e, ms_per_step, peaks):
+    """Whole-step figures: strict roofline = max(gate GEMM at tensor peak, compulsory bytes at HBM rate)."""
+    d, F, K = w.d_model, w.d_ff, w.k
+    gate = 2.0 * T * d * F
+    sparse = 16.0 * T * K * d
+    comp_bytes = (T * d * e * 2 + 3 * F * d * e + T * K * (2 + 2 * e)) + \
+                 (2 * T * d * e + 3 * F * d * e + T * K * (2 + 2 * e) + T * d * e + 3 * F * d * e)
+    r_gate = gate / (peaks["bf16_tflops"] * 1e12) * 1e3
+    r_bytes = comp_bytes / (peaks["hbm_gbs"] * 1e9) * 1e3
+    r_strict = max(r_gate, r_bytes)
+    return {"r_gate_ms": r_gate, "r_bytes_ms": r_bytes, "strict_frac": r_strict / ms_per_step,
+            "algorithmic_tflops": (gate + sparse) / (ms_per_step / 1e3) / 1e12,
+            "dense_equiv_tflops": 18.0 * T * d * F / (ms_per_step / 1e3) / 1e12,
+            "peak_source": peaks["source"]}
+
+
+def act_bytes_report(w, T, e, saved, B, desc):
+    measured = sum(t.numel() * t.element_size() for t in saved)
+    return {"moc_saved_per_token": B.moc_ffn_saved_bytes_per_token(desc), "measured_saved_total": measured,
+            "measured_saved_per_token": measured / T, "dense_swiglu_per_token": 4 * w.d_ff * e,
+            "dense_gcp_per_token": 2 * w.d_ff * e, "x_and_out_per_token_each": w.d_model * e}
+
+
+def decode_report(torch, B, syn, dev, peaks, iters=48, sets=4):
+    """moc_ffn_decode on the LLaMA-7B shape for 1/4/16 tokens; weight sets rotate so that every call
+    streams its weights from HBM (4 sets x 270 MB > L2)."""
+    w = syn.C4
+    weights = [tuple(t.to(dev) for t in syn.make_weights(w, seed_offset=s)) for s in range(sets)]
+    rep = {"weight_sets": sets, "iters": iters}
+    e = 2
+    for T in syn.C4_BATCHES:
+        x = syn.make_x(w, tokens=T).to(dev)
+        out = torch.empty_like(x)
+        desc = B.make_desc(T, w.d_model, w.d_ff, w.k, x.dtype, d_ff_ld=w.d_ff_ld)
+        ws = B.alloc_workspace(desc, B.MOC_OP_DECODE, dev)
+        for i in range(sets):
+            B.moc_ffn_decode(x, *weights[i], w.k, out=out, workspace=ws)
+        torch.cuda.synchronize()
+        s, t = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s.record()
+        for i in range(iters):
+            B.moc_ffn_decode(x, *weights[i % sets], w.k, out=out, workspace=ws)
+        t.record()
+        torch.cuda.synchronize()
+        us = s.elapsed_time(t) * 1e3 / iters
+        # union of selected channels from an extra saved forward on set 0
+        _, idx, _, _ = B.moc_ffn_forward(x, *weights[0], w.k)
+        union = int(torch.unique(idx.long()).numel())
+        algo = w.d_ff * w.d_model * e + 2 * union * w.d_model * e + 2 * T * w.d_model * e
+        roof_us = algo / (peaks["hbm_gbs"] * 1e9) * 1e6
+        rep[f"T{T}"] = {"us_per_step": us, "us_per_token": us / T, "union_channels": union,
+                        "algorithmic_bytes": algo, "roofline_us": roof_us, "frac": roof_us / us,
+                        "achieved_gbs": algo / (us * 1e-6) / 1e9}
+        del ws
+    return rep
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

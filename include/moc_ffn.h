@@ -136,6 +136,27 @@ MOC_API int moc_last_device_status(void *cuda_stream);
 /* Bytes per token that stay alive between forward and backward: k * (2 + 2 * sizeof(dtype)). */
 MOC_API size_t moc_ffn_saved_bytes_per_token(const moc_ffn_desc *desc);
 
+/*
+ * Diagnostics (no counterpart in the paper; they exist so that a benchmark can attribute device
+ * time to kernels without a profiler attached).  Not thread-safe against concurrent entry-point
+ * calls: open a window, run the calls to be measured on ONE stream, collect, read.
+ *   moc_launch_count          kernels launched by this library in this process so far.
+ *   moc_profile_enable(1)     opens a window and clears the accumulators; while it is open every
+ *                             kernel launch is bracketed by a pair of CUDA events on its stream
+ *                             (at most 8192 launches per collect; later ones are not recorded).
+ *   moc_profile_enable(0)     closes the window.
+ *   moc_profile_collect       synchronises `cuda_stream`, folds the recorded pairs into per-kernel
+ *                             totals; returns the number of launches that were not recorded (>= 0)
+ *                             or a negative moc_status.
+ *   moc_profile_kernel_count / _name / _read   enumerate kernels and read launches + total ms.
+ */
+MOC_API int64_t moc_launch_count(void);
+MOC_API int moc_profile_enable(int on);
+MOC_API int moc_profile_collect(void *cuda_stream);
+MOC_API int moc_profile_kernel_count(void);
+MOC_API const char *moc_profile_kernel_name(int id);
+MOC_API int moc_profile_read(int id, int64_t *launches, double *total_ms);
+
 /* Static, NUL-terminated description of a moc_status value. */
 MOC_API const char *moc_status_string(int status);
 

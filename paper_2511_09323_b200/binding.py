@@ -27,7 +27,9 @@ MOC_FLAG_ACCUMULATE_WGRAD = 1
 
 EXPORTED = (
     "moc_ffn_workspace_bytes", "moc_ffn_forward", "moc_ffn_backward", "moc_ffn_decode", "moc_topk_select",
-    "moc_last_device_status", "moc_ffn_saved_bytes_per_token", "moc_status_string",
+    "moc_last_device_status", "moc_ffn_saved_bytes_per_token", "moc_status_string", "moc_launch_count",
+    "moc_profile_enable", "moc_profile_collect", "moc_profile_kernel_count", "moc_profile_kernel_name",
+    "moc_profile_read",
 )
 
 
@@ -73,6 +75,19 @@ def load() -> ctypes.CDLL:
         lib.moc_last_device_status.argtypes = [vp]
         lib.moc_status_string.restype = ctypes.c_char_p
         lib.moc_status_string.argtypes = [ctypes.c_int]
+        lib.moc_launch_count.restype = ctypes.c_int64
+        lib.moc_launch_count.argtypes = []
+        lib.moc_profile_enable.restype = ctypes.c_int
+        lib.moc_profile_enable.argtypes = [ctypes.c_int]
+        lib.moc_profile_collect.restype = ctypes.c_int
+        lib.moc_profile_collect.argtypes = [vp]
+        lib.moc_profile_kernel_count.restype = ctypes.c_int
+        lib.moc_profile_kernel_count.argtypes = []
+        lib.moc_profile_kernel_name.restype = ctypes.c_char_p
+        lib.moc_profile_kernel_name.argtypes = [ctypes.c_int]
+        lib.moc_profile_read.restype = ctypes.c_int
+        lib.moc_profile_read.argtypes = [ctypes.c_int, ctypes.POINTER(ctypes.c_int64),
+                                         ctypes.POINTER(ctypes.c_double)]
         _lib = lib
     return _lib
 
@@ -218,3 +233,29 @@ def moc_topk_select(gate: torch.Tensor, k: int, n: int | None = None, stream=Non
 
 def moc_last_device_status(stream=None) -> int:
     return int(load().moc_last_device_status(_stream_ptr(stream)))
+
+
+def moc_launch_count() -> int:
+    return int(load().moc_launch_count())
+
+
+def moc_profile_enable(on: bool) -> None:
+    rc = load().moc_profile_enable(1 if on else 0)
+    if rc != MOC_OK:
+        raise MocError(rc, "moc_profile_enable")
+
+
+def moc_profile_collect(stream=None) -> dict:
+    """Synchronises the stream and returns {kernel name: (launches, total_ms)} for the open window."""
+    lib = load()
+    rc = lib.moc_profile_collect(_stream_ptr(stream))
+    if rc < 0:
+        raise MocError(rc, "moc_profile_collect")
+    out = {}
+    for i in range(lib.moc_profile_kernel_count()):
+        n, ms = ctypes.c_int64(0), ctypes.c_double(0.0)
+        lib.moc_profile_read(i, ctypes.byref(n), ctypes.byref(ms))
+        if n.value:
+            out[lib.moc_profile_kernel_name(i).decode()] = (int(n.value), float(ms.value))
+    out["_dropped"] = (rc, 0.0)
+    return out

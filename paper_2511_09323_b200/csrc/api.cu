@@ -3,8 +3,10 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <atomic>
 #include <cstdint>
 #include <cstring>
+#include <vector>
 
 #include "gather_kernels.cuh"
 #include "moc_common.cuh"
@@ -27,6 +29,62 @@ int *device_status_ptr() {
     }
     return cache[dev];
 }
+
+// ---- launch bookkeeping --------------------------------------------------------------------------
+// Every kernel the library launches goes through MOC_LAUNCH: it counts the launch and, while a
+// profiling window is open, brackets it with a pair of CUDA events on the caller's stream so that
+// a benchmark can read per-kernel device time without a profiler attached.
+enum KernelId {
+    KID_GATE_GEMM_ALU = 0,
+    KID_SELECT_ROWS,
+    KID_FORWARD_TOKEN,
+    KID_BACKWARD_TOKEN,
+    KID_CSR_COUNT,
+    KID_CSR_SCAN_BLOCKS,
+    KID_CSR_SCAN_CHANNELS,
+    KID_CSR_FILL,
+    KID_WGRAD_ROWS,
+    KID_TOPK_SELECT,
+    KID_COUNT
+};
+static const char *const kKernelNames[KID_COUNT] = {
+    "gate_gemm_alu", "select_rows",       "forward_token", "backward_token", "csr_count",
+    "csr_scan_blocks", "csr_scan_channels", "csr_fill",      "wgrad_rows",     "topk_select",
+};
+
+struct Profiler {
+    static constexpr int kMaxPairs = 8192;
+    std::atomic<int64_t> launches{0};
+    bool on = false;
+    std::vector<cudaEvent_t> ev;  // 2 * kMaxPairs, created on first use
+    int used = 0, dropped = 0;
+    int ids[kMaxPairs];
+    double ms[KID_COUNT] = {};
+    int64_t count[KID_COUNT] = {};
+};
+static Profiler g_prof;
+
+static bool prof_begin(int kid, cudaStream_t st) {
+    g_prof.launches.fetch_add(1, std::memory_order_relaxed);
+    if (!g_prof.on) return false;
+    if (g_prof.used >= Profiler::kMaxPairs) {
+        ++g_prof.dropped;
+        return false;
+    }
+    g_prof.ids[g_prof.used] = kid;
+    return cudaEventRecord(g_prof.ev[2 * g_prof.used], st) == cudaSuccess;
+}
+static void prof_end(bool rec, cudaStream_t st) {
+    if (!rec) return;
+    cudaEventRecord(g_prof.ev[2 * g_prof.used + 1], st);
+    ++g_prof.used;
+}
+#define MOC_LAUNCH(kid, st, ...)                   \
+    do {                                           \
+        const bool moc_rec_ = prof_begin(kid, st); \
+        __VA_ARGS__;                               \
+        prof_end(moc_rec_, st);                    \
+    } while (0)
 
 namespace {
 
@@ -142,14 +200,17 @@ int forward_gather(const moc_ffn_desc &d, const T *x, const T *wg, const T *wu, 
     for (int64_t t0 = 0; t0 < d.tokens; t0 += p.chunk) {
         const int64_t n = std::min<int64_t>(p.chunk, d.tokens - t0);
         dim3 grid((F + 63) / 64, (unsigned)((n + 63) / 64));
-        gemm_nt_alu_kernel<T><<<grid, 256, 0, st>>>(x + t0 * dm, wg, G, (int)n, F, dm, F);
+        MOC_LAUNCH(KID_GATE_GEMM_ALU, st, (gemm_nt_alu_kernel<T><<<grid, 256, 0, st>>>(x + t0 * dm, wg, G, (int)n, F, dm, F)));
         if ((rc = launch_ok()) != MOC_OK) return rc;
         const unsigned sel_grid = (unsigned)std::min<int64_t>(n, 148 * 32);
-        select_rows_kernel<T><<<sel_grid, kSelectThreads, sel_smem, st>>>(G, n, F, F, K, idx + t0 * K,
-                                                                           tg ? tg + t0 * K : nullptr);
+        MOC_LAUNCH(KID_SELECT_ROWS, st,
+                   (select_rows_kernel<T><<<sel_grid, kSelectThreads, sel_smem, st>>>(
+                       G, n, F, F, K, idx + t0 * K, tg ? tg + t0 * K : nullptr)));
         if ((rc = launch_ok()) != MOC_OK) return rc;
-        forward_token_kernel<T><<<(unsigned)n, kTokenThreads, tok_smem, st>>>(
-            x + t0 * dm, wu, wd, G, F, idx + t0 * K, dm, K, out + t0 * dm, tu ? tu + t0 * K : nullptr, 0);
+        MOC_LAUNCH(KID_FORWARD_TOKEN, st,
+                   (forward_token_kernel<T><<<(unsigned)n, kTokenThreads, tok_smem, st>>>(
+                       x + t0 * dm, wu, wd, G, F, idx + t0 * K, dm, K, out + t0 * dm, tu ? tu + t0 * K : nullptr,
+                       0)));
         if ((rc = launch_ok()) != MOC_OK) return rc;
     }
     return MOC_OK;
@@ -171,8 +232,9 @@ int backward_gather(const moc_ffn_desc &d, const T *x, const T *wg, const T *wu,
     const size_t tok_smem = ((size_t)dm + 3 * (size_t)K + token_red_floats(dm)) * sizeof(float);
     int rc = set_smem(backward_token_kernel<T>, tok_smem);
     if (rc != MOC_OK) return rc;
-    backward_token_kernel<T><<<(unsigned)d.tokens, kTokenThreads, tok_smem, st>>>(
-        wg, wu, wd, idx, tg, tu, dout, dm, F, K, TK, gx, want_w ? coef : nullptr, status);
+    MOC_LAUNCH(KID_BACKWARD_TOKEN, st,
+               (backward_token_kernel<T><<<(unsigned)d.tokens, kTokenThreads, tok_smem, st>>>(
+                   wg, wu, wd, idx, tg, tu, dout, dm, F, K, TK, gx, want_w ? coef : nullptr, status)));
     if ((rc = launch_ok()) != MOC_OK) return rc;
     if (!want_w) return MOC_OK;
 
@@ -183,20 +245,23 @@ int backward_gather(const moc_ffn_desc &d, const T *x, const T *wg, const T *wu,
     const size_t f_smem = (size_t)F * sizeof(uint32_t);
     if ((rc = set_smem(csr_count_kernel, f_smem)) != MOC_OK) return rc;
     if ((rc = set_smem(csr_fill_kernel, f_smem)) != MOC_OK) return rc;
-    csr_count_kernel<<<p.nb, 256, f_smem, st>>>(idx, d.tokens, K, F, p.tb, counts);
+    MOC_LAUNCH(KID_CSR_COUNT, st, (csr_count_kernel<<<p.nb, 256, f_smem, st>>>(idx, d.tokens, K, F, p.tb, counts)));
     if ((rc = launch_ok()) != MOC_OK) return rc;
-    csr_scan_blocks_kernel<<<(F + 255) / 256, 256, 0, st>>>(counts, p.nb, F, totals);
+    MOC_LAUNCH(KID_CSR_SCAN_BLOCKS, st,
+               (csr_scan_blocks_kernel<<<(F + 255) / 256, 256, 0, st>>>(counts, p.nb, F, totals)));
     if ((rc = launch_ok()) != MOC_OK) return rc;
-    csr_scan_channels_kernel<<<1, 1024, 0, st>>>(totals, F, row_start);
+    MOC_LAUNCH(KID_CSR_SCAN_CHANNELS, st, (csr_scan_channels_kernel<<<1, 1024, 0, st>>>(totals, F, row_start)));
     if ((rc = launch_ok()) != MOC_OK) return rc;
-    csr_fill_kernel<<<p.nb, 256, f_smem, st>>>(idx, d.tokens, K, F, p.tb, counts, row_start, pairs);
+    MOC_LAUNCH(KID_CSR_FILL, st,
+               (csr_fill_kernel<<<p.nb, 256, f_smem, st>>>(idx, d.tokens, K, F, p.tb, counts, row_start, pairs)));
     if ((rc = launch_ok()) != MOC_OK) return rc;
 
     const size_t red = token_red_floats(dm) * 3 * sizeof(float);
     if ((rc = set_smem(wgrad_rows_kernel<T>, red)) != MOC_OK) return rc;
-    wgrad_rows_kernel<T><<<d.d_ff_ld, kTokenThreads, red, st>>>(x, dout, coef, TK, row_start, pairs, dm, F, K, gwg,
-                                                                  gwu, gwd,
-                                                                  (d.flags & MOC_FLAG_ACCUMULATE_WGRAD) ? 1 : 0);
+    MOC_LAUNCH(KID_WGRAD_ROWS, st,
+               (wgrad_rows_kernel<T><<<d.d_ff_ld, kTokenThreads, red, st>>>(
+                   x, dout, coef, TK, row_start, pairs, dm, F, K, gwg, gwu, gwd,
+                   (d.flags & MOC_FLAG_ACCUMULATE_WGRAD) ? 1 : 0)));
     return launch_ok();
 }
 
@@ -317,8 +382,10 @@ int moc_topk_select(int64_t rows, int32_t n, int32_t n_ld, int32_t k, const floa
     int rc = set_smem(topk_select_kernel<kSelectThreads>, smem);
     if (rc != MOC_OK) return rc;
     const unsigned grid = (unsigned)std::min<int64_t>(rows, 148 * 32);
-    topk_select_kernel<kSelectThreads><<<grid, kSelectThreads, smem, static_cast<cudaStream_t>(cuda_stream)>>>(
-        gate, rows, n, n_ld, k, idx_out);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    MOC_LAUNCH(KID_TOPK_SELECT, st,
+               (topk_select_kernel<kSelectThreads><<<grid, kSelectThreads, smem, st>>>(gate, rows, n, n_ld, k,
+                                                                                        idx_out)));
     return launch_ok();
 }
 
@@ -332,6 +399,53 @@ int moc_last_device_status(void *cuda_stream) {
         if (cudaMemset(p, 0, sizeof(int)) != cudaSuccess) return MOC_ERR_CUDA;
     }
     return v;
+}
+
+int64_t moc_launch_count(void) { return g_prof.launches.load(std::memory_order_relaxed); }
+
+int moc_profile_enable(int on) {
+    if (on) {
+        if (g_prof.ev.empty()) {
+            g_prof.ev.resize(2 * Profiler::kMaxPairs);
+            for (auto &e : g_prof.ev) {
+                if (cudaEventCreate(&e) != cudaSuccess) {
+                    g_prof.ev.clear();
+                    return MOC_ERR_CUDA;
+                }
+            }
+        }
+        g_prof.used = g_prof.dropped = 0;
+        for (int i = 0; i < KID_COUNT; ++i) {
+            g_prof.ms[i] = 0.0;
+            g_prof.count[i] = 0;
+        }
+    }
+    g_prof.on = on != 0;
+    return MOC_OK;
+}
+
+int moc_profile_collect(void *cuda_stream) {
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return MOC_ERR_CUDA;
+    for (int i = 0; i < g_prof.used; ++i) {
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, g_prof.ev[2 * i], g_prof.ev[2 * i + 1]) != cudaSuccess) return MOC_ERR_CUDA;
+        g_prof.ms[g_prof.ids[i]] += ms;
+        g_prof.count[g_prof.ids[i]] += 1;
+    }
+    const int dropped = g_prof.dropped;
+    g_prof.used = g_prof.dropped = 0;
+    return dropped;
+}
+
+int moc_profile_kernel_count(void) { return KID_COUNT; }
+
+const char *moc_profile_kernel_name(int id) { return (id >= 0 && id < KID_COUNT) ? kKernelNames[id] : ""; }
+
+int moc_profile_read(int id, int64_t *launches, double *total_ms) {
+    if (id < 0 || id >= KID_COUNT || !launches || !total_ms) return MOC_ERR_INVALID_ARG;
+    *launches = g_prof.count[id];
+    *total_ms = g_prof.ms[id];
+    return MOC_OK;
 }
 
 const char *moc_status_string(int status) {
