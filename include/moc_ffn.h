@@ -57,7 +57,8 @@ typedef enum {
     MOC_ERR_WORKSPACE = -3,   /* workspace pointer NULL or smaller than moc_ffn_workspace_bytes()    */
     MOC_ERR_CUDA = -4,        /* a CUDA runtime call or a launch failed                             */
     MOC_ERR_TIMEOUT = -5,     /* device status: a bounded wait inside a kernel expired              */
-    MOC_ERR_BAD_INDEX = -6    /* device status: a saved channel index was outside [0, d_ff)         */
+    MOC_ERR_BAD_INDEX = -6,   /* device status: a saved channel index was outside [0, d_ff)         */
+    MOC_ERR_STATIC_LIMIT = -7 /* problem larger than the built-in scratch of moc_ffn_decode_static   */
 } moc_status;
 
 typedef enum { MOC_F32 = 0, MOC_BF16 = 1 } moc_dtype;
@@ -118,6 +119,38 @@ MOC_API int moc_ffn_backward(const moc_ffn_desc *desc, const void *x, const void
 MOC_API int moc_ffn_decode(const moc_ffn_desc *desc, const void *x, const void *w_gate, const void *w_up,
                            const void *w_down, void *out, void *workspace, size_t workspace_bytes,
                            void *cuda_stream);
+
+/*
+ * moc_ffn_decode for callers that must not allocate.  (The paper has no counterpart: this is a
+ * packaging variant of the decode path, not a different computation.)
+ *
+ * Who needs it: code that runs where device allocation is off the table -- an inference server
+ * that handed all free HBM to its KV-cache pool at start-up, so a cudaMalloc in the decode loop
+ * would fail; a latency-critical loop that cannot afford cudaMalloc/cudaFree because they
+ * synchronise the whole device; a plug-in that is handed tensors but no allocator.  Such callers
+ * still pass their inputs and the output buffer, but no workspace: the transient buffers (the fp32
+ * gate projection of the batch and its channel indices) live in an array that is part of the
+ * library image, MOC_STATIC_SCRATCH_BYTES long.  Every GPU that loads the library holds that array
+ * from load until the process exits, whether or not this entry point is ever called.
+ *
+ * Limits  tokens <= MOC_STATIC_MAX_TOKENS and d_ff <= MOC_STATIC_MAX_DFF; anything larger returns
+ *         MOC_ERR_STATIC_LIMIT and launches nothing (use moc_ffn_decode with a workspace instead).
+ *         All other argument rules are those of moc_ffn_decode.
+ * Set-up  The first call on each device looks up the device address of the array (no allocation,
+ *         but a runtime query): make that first call during start-up, before any stream capture.
+ * Sharing All calls on a device use the SAME array.  Calls on one stream are ordered and safe;
+ *         calls whose kernels can overlap on the GPU (different streams or host threads without an
+ *         ordering between them) race on it and give undefined results.  The array keeps whatever
+ *         the previous call left; nothing in it needs to start at zero, because each call writes
+ *         the whole region it later reads.
+ * It calls neither cudaMalloc nor cudaFree nor any allocating library routine.
+ */
+#define MOC_STATIC_MAX_TOKENS 16
+#define MOC_STATIC_MAX_DFF 16384
+#define MOC_STATIC_SCRATCH_BYTES \
+    ((size_t)MOC_STATIC_MAX_TOKENS * MOC_STATIC_MAX_DFF * (sizeof(float) + sizeof(int16_t)) + 512)
+MOC_API int moc_ffn_decode_static(const moc_ffn_desc *desc, const void *x, const void *w_gate,
+                                  const void *w_up, const void *w_down, void *out, void *cuda_stream);
 
 /*
  * The Top-K selector alone (the mask definition of Section 3.2), exposed so that it can be checked

@@ -21,6 +21,8 @@ MOC_ERR_WORKSPACE = -3
 MOC_ERR_CUDA = -4
 MOC_ERR_TIMEOUT = -5
 MOC_ERR_BAD_INDEX = -6
+MOC_ERR_STATIC_LIMIT = -7
+MOC_STATIC_MAX_TOKENS, MOC_STATIC_MAX_DFF = 16, 16384
 MOC_F32, MOC_BF16 = 0, 1
 MOC_OP_FORWARD, MOC_OP_BACKWARD, MOC_OP_DECODE = 0, 1, 2
 MOC_FLAG_ACCUMULATE_WGRAD = 1
@@ -29,7 +31,7 @@ EXPORTED = (
     "moc_ffn_workspace_bytes", "moc_ffn_forward", "moc_ffn_backward", "moc_ffn_decode", "moc_topk_select",
     "moc_last_device_status", "moc_ffn_saved_bytes_per_token", "moc_status_string", "moc_launch_count",
     "moc_profile_enable", "moc_profile_collect", "moc_profile_kernel_count", "moc_profile_kernel_name",
-    "moc_profile_read",
+    "moc_profile_read", "moc_ffn_decode_static",
 )
 
 
@@ -69,6 +71,8 @@ def load() -> ctypes.CDLL:
         lib.moc_ffn_backward.argtypes = [dp] + [vp] * 13 + [sz, vp]
         lib.moc_ffn_decode.restype = ctypes.c_int
         lib.moc_ffn_decode.argtypes = [dp] + [vp] * 6 + [sz, vp]
+        lib.moc_ffn_decode_static.restype = ctypes.c_int
+        lib.moc_ffn_decode_static.argtypes = [dp] + [vp] * 5 + [vp]
         lib.moc_topk_select.restype = ctypes.c_int
         lib.moc_topk_select.argtypes = [ctypes.c_int64, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, vp, vp, vp]
         lib.moc_last_device_status.restype = ctypes.c_int
@@ -214,6 +218,21 @@ def moc_ffn_decode(x, w_gate, w_up, w_down, k, d_ff=None, out=None, workspace=No
                                _ptr(workspace), workspace.numel(), _stream_ptr(stream))
     if rc != MOC_OK:
         raise MocError(rc, "moc_ffn_decode")
+    return out
+
+
+def moc_ffn_decode_static(x, w_gate, w_up, w_down, k, out, d_ff=None, stream=None):
+    """Decode for callers that cannot allocate: no workspace argument, and `out` must be supplied, so that
+    nothing on this call path asks any allocator (torch's included) for memory.  The transient buffers
+    live in an array inside the library; see the limits and the sharing rules in include/moc_ffn.h."""
+    _check_dev(x, w_gate, w_up, w_down, out)
+    T, d = x.shape
+    F_ld = w_gate.shape[0]
+    desc = make_desc(T, d, F_ld if d_ff is None else d_ff, k, x.dtype, d_ff_ld=F_ld)
+    rc = load().moc_ffn_decode_static(ctypes.byref(desc), _ptr(x), _ptr(w_gate), _ptr(w_up), _ptr(w_down),
+                                      _ptr(out), _stream_ptr(stream))
+    if rc != MOC_OK:
+        raise MocError(rc, "moc_ffn_decode_static")
     return out
 
 

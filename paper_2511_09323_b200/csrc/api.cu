@@ -389,6 +389,45 @@ int moc_topk_select(int64_t rows, int32_t n, int32_t n_ld, int32_t k, const floa
     return launch_ok();
 }
 
+// ---- decode without a caller workspace --------------------------------------------------------------
+// Scratch for moc_ffn_decode_static.  In host code the name below is only a handle for the runtime,
+// not a device address: the address is asked for once per device and that pointer goes to the kernels.
+static __device__ __align__(256) unsigned char g_static_scratch[MOC_STATIC_SCRATCH_BYTES];
+
+static char *static_scratch_ptr() {
+    static char *cache[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (!cache[dev]) {
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return nullptr;
+        cache[dev] = static_cast<char *>(p);
+    }
+    return cache[dev];
+}
+
+int moc_ffn_decode_static(const moc_ffn_desc *desc, const void *x, const void *w_gate, const void *w_up,
+                          const void *w_down, void *out, void *cuda_stream) {
+    int rc = check_desc(desc);
+    if (rc != MOC_OK) return rc;
+    if (desc->tokens > MOC_STATIC_MAX_TOKENS || desc->d_ff > MOC_STATIC_MAX_DFF) return MOC_ERR_STATIC_LIMIT;
+    if (desc->tokens == 0) return MOC_OK;
+    if (!good_ptr(x) || !good_ptr(w_gate) || !good_ptr(w_up) || !good_ptr(w_down) || !good_ptr(out))
+        return MOC_ERR_INVALID_ARG;
+    // same carving as the workspace variant; the limits above bound it by the array's size
+    if (plan_forward(*desc).total > MOC_STATIC_SCRATCH_BYTES) return MOC_ERR_STATIC_LIMIT;
+    char *ws = static_scratch_ptr();
+    if (!ws) return MOC_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (desc->dtype == MOC_BF16) {
+        using T = __nv_bfloat16;
+        return forward_gather<T>(*desc, (const T *)x, (const T *)w_gate, (const T *)w_up, (const T *)w_down,
+                                 (T *)out, nullptr, nullptr, nullptr, ws, st);
+    }
+    return forward_gather<float>(*desc, (const float *)x, (const float *)w_gate, (const float *)w_up,
+                                 (const float *)w_down, (float *)out, nullptr, nullptr, nullptr, ws, st);
+}
+
 int moc_last_device_status(void *cuda_stream) {
     if (cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return MOC_ERR_CUDA;
     int *p = device_status_ptr();
@@ -457,6 +496,7 @@ const char *moc_status_string(int status) {
         case MOC_ERR_CUDA: return "CUDA runtime error";
         case MOC_ERR_TIMEOUT: return "a bounded device-side wait expired";
         case MOC_ERR_BAD_INDEX: return "saved channel index out of range";
+        case MOC_ERR_STATIC_LIMIT: return "problem exceeds the built-in scratch of moc_ffn_decode_static";
         default: return "unknown status";
     }
 }
