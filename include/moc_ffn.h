@@ -161,6 +161,18 @@ MOC_API int moc_topk_select(int64_t rows, int32_t n, int32_t n_ld, int32_t k, co
                             int16_t *idx_out, void *cuda_stream);
 
 /*
+ * The dense bf16 contraction used for the gate projection G = X W_gate of Eq. (Moc-1) and for every
+ * other contraction of the tensor-core plan, exposed so that it can be checked on its own:
+ *     C[m, n] (fp32, row-major, leading dimension ldc) = sum_k A(m, k) * B(n, k),  fp32 accumulation.
+ * A is stored [m, k] row-major (lda >= k) when a_mn_major == 0, or [k, m] row-major (lda >= m) when
+ * a_mn_major != 0; B likewise as [n, k] or [k, n].  lda and ldb are in elements and multiples of 8.
+ * Runs on the tcgen05 tensor cores (one persistent CTA per SM, TMA-fed, TMEM accumulators).
+ */
+MOC_API int moc_tc_gemm_bf16(int64_t m, int64_t n, int64_t k, const void *a, int a_mn_major, int64_t lda,
+                             const void *b, int b_mn_major, int64_t ldb, float *c, int64_t ldc,
+                             void *cuda_stream);
+
+/*
  * Synchronises `cuda_stream`, then returns and clears the current device's sticky status word:
  * MOC_OK, MOC_ERR_TIMEOUT or MOC_ERR_BAD_INDEX (MOC_ERR_CUDA if the synchronisation itself failed).
  */

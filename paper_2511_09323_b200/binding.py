@@ -31,7 +31,7 @@ EXPORTED = (
     "moc_ffn_workspace_bytes", "moc_ffn_forward", "moc_ffn_backward", "moc_ffn_decode", "moc_topk_select",
     "moc_last_device_status", "moc_ffn_saved_bytes_per_token", "moc_status_string", "moc_launch_count",
     "moc_profile_enable", "moc_profile_collect", "moc_profile_kernel_count", "moc_profile_kernel_name",
-    "moc_profile_read", "moc_ffn_decode_static",
+    "moc_profile_read", "moc_ffn_decode_static", "moc_tc_gemm_bf16",
 )
 
 
@@ -73,6 +73,9 @@ def load() -> ctypes.CDLL:
         lib.moc_ffn_decode.argtypes = [dp] + [vp] * 6 + [sz, vp]
         lib.moc_ffn_decode_static.restype = ctypes.c_int
         lib.moc_ffn_decode_static.argtypes = [dp] + [vp] * 5 + [vp]
+        lib.moc_tc_gemm_bf16.restype = ctypes.c_int
+        lib.moc_tc_gemm_bf16.argtypes = [ctypes.c_int64] * 3 + [vp, ctypes.c_int, ctypes.c_int64, vp, ctypes.c_int,
+                                                                ctypes.c_int64, vp, ctypes.c_int64, vp]
         lib.moc_topk_select.restype = ctypes.c_int
         lib.moc_topk_select.argtypes = [ctypes.c_int64, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, vp, vp, vp]
         lib.moc_last_device_status.restype = ctypes.c_int
@@ -278,3 +281,21 @@ def moc_profile_collect(stream=None) -> dict:
             out[lib.moc_profile_kernel_name(i).decode()] = (int(n.value), float(ms.value))
     out["_dropped"] = (rc, 0.0)
     return out
+
+
+def moc_tc_gemm_bf16(a: torch.Tensor, b: torch.Tensor, a_mn_major: bool = False, b_mn_major: bool = False,
+                     stream=None) -> torch.Tensor:
+    """C[m,n] fp32 = sum_k A(m,k) B(n,k).  a is [m,k] (or [k,m] when a_mn_major), b is [n,k] (or [k,n])."""
+    _check_dev(a, b)
+    if a.dtype != torch.bfloat16 or b.dtype != torch.bfloat16:
+        raise TypeError("bf16 operands expected")
+    m, k = (a.shape[1], a.shape[0]) if a_mn_major else a.shape
+    n, kb = (b.shape[1], b.shape[0]) if b_mn_major else b.shape
+    if k != kb:
+        raise ValueError("contraction sizes differ")
+    c = torch.empty((m, n), dtype=torch.float32, device=a.device)
+    rc = load().moc_tc_gemm_bf16(m, n, k, _ptr(a), int(a_mn_major), a.stride(0), _ptr(b), int(b_mn_major),
+                                 b.stride(0), _ptr(c), n, _stream_ptr(stream))
+    if rc != MOC_OK:
+        raise MocError(rc, "moc_tc_gemm_bf16")
+    return c

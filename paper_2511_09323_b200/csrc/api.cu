@@ -10,6 +10,8 @@
 
 #include "gather_kernels.cuh"
 #include "moc_common.cuh"
+#include "tc_gemm.cuh"
+#include "tc_plan.cuh"
 #include "topk_select.cuh"
 
 namespace moc {
@@ -45,11 +47,21 @@ enum KernelId {
     KID_CSR_FILL,
     KID_WGRAD_ROWS,
     KID_TOPK_SELECT,
+    KID_TC_GATE_UP_GEMM,
+    KID_TC_SELECT_MASK,
+    KID_TC_DOWN_GEMM,
+    KID_TC_TILE_START,
+    KID_TC_DZ_GEMM,
+    KID_TC_WGRAD_GEMM,
+    KID_TC_DX_GEMM,
+    KID_TC_TEST_GEMM,
     KID_COUNT
 };
 static const char *const kKernelNames[KID_COUNT] = {
     "gate_gemm_alu", "select_rows",       "forward_token", "backward_token", "csr_count",
     "csr_scan_blocks", "csr_scan_channels", "csr_fill",      "wgrad_rows",     "topk_select",
+    "tc_gate_up_gemm", "tc_select_mask",  "tc_down_gemm",  "tc_tile_start",  "tc_dz_gemm",
+    "tc_wgrad_gemm",   "tc_dx_gemm",      "tc_test_gemm",
 };
 
 struct Profiler {
@@ -265,6 +277,175 @@ int backward_gather(const moc_ffn_desc &d, const T *x, const T *wg, const T *wu,
     return launch_ok();
 }
 
+// ---- tensor-core plan (bf16 training shapes) ---------------------------------------------------------
+bool use_tc_plan(const moc_ffn_desc &d) {
+    if (d.dtype != MOC_BF16 || d.tokens < 256) return false;
+    // the forward selector keeps F keys and K packed entries in shared memory
+    return ((size_t)d.d_ff + (size_t)d.k) * 4 <= 200 * 1024;
+}
+
+inline int ceil_div(int64_t a, int64_t b) { return (int)((a + b - 1) / b); }
+
+int forward_tc(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat16 *wg, const __nv_bfloat16 *wu,
+               const __nv_bfloat16 *wd, __nv_bfloat16 *out, int16_t *idx, __nv_bfloat16 *tg, __nv_bfloat16 *tu,
+               char *ws, cudaStream_t st) {
+    using namespace tc;
+    const TcForwardLayout L = tc_forward_layout(d);
+    float *G = reinterpret_cast<float *>(ws + L.off_g);
+    __nv_bfloat16 *U = reinterpret_cast<__nv_bfloat16 *>(ws + L.off_u);
+    const int F = d.d_ff, K = d.k, dm = d.d_model;
+    const int64_t T = d.tokens;
+    const int f_tiles = ceil_div(F, BN);
+
+    const size_t sel_smem = ((size_t)F + K) * sizeof(uint32_t);
+    int rc = set_smem(select_mask_rows_kernel, sel_smem);
+    if (rc != MOC_OK) return rc;
+
+    int *status = device_status_ptr();
+    if (!status) return MOC_ERR_CUDA;
+    Params p;
+    init_params(p);
+    if (!map_k_major(&p.b_map[0], wg, F, dm, dm, BN) || !map_k_major(&p.b_map[1], wu, F, dm, dm, BN))
+        return MOC_ERR_CUDA;
+    p.status = status;
+    p.num_problems = 2;
+    p.b_idx[1][0] = 1;
+    p.k_blocks = ceil_div(dm, BK);
+    p.N = F;
+    p.n_tiles = f_tiles;
+    p.ldc[0] = p.ldc[1] = L.ldf;
+    for (int64_t t0 = 0; t0 < T; t0 += L.chunk) {
+        const int64_t n = std::min<int64_t>(L.chunk, T - t0);
+        if (!map_k_major(&p.a_map[0], x + t0 * dm, n, dm, dm, BM)) return MOC_ERR_CUDA;
+        p.M = (int)n;
+        p.m_tiles = ceil_div(n, BM);
+        p.c[0] = G;
+        p.c[1] = U + t0 * L.ldf;
+        MOC_LAUNCH(KID_TC_GATE_UP_GEMM, st, (rc = launch_gemm<false, false, EPI_GATE_UP>(p, st)));
+        if (rc != MOC_OK) return rc;
+        const unsigned grid = (unsigned)std::min<int64_t>(n, (int64_t)sm_count() * 8);
+        MOC_LAUNCH(KID_TC_SELECT_MASK, st,
+                   (select_mask_rows_kernel<<<grid, kSelectThreads, sel_smem, st>>>(
+                       G, L.ldf, U + t0 * L.ldf, L.ldf, n, F, K, idx ? idx + t0 * K : nullptr,
+                       idx ? tg + t0 * K : nullptr, idx ? tu + t0 * K : nullptr)));
+        if ((rc = launch_ok()) != MOC_OK) return rc;
+    }
+    // D = Z' W_down over all tokens: A = Z' [T, F] (K-major), B = Wd [F, d] (its contiguous dimension is N)
+    Params q;
+    init_params(q);
+    if (!map_k_major(&q.a_map[0], U, T, F, L.ldf, BM) || !map_mn_major(&q.b_map[0], wd, F, dm, dm))
+        return MOC_ERR_CUDA;
+    q.k_blocks = ceil_div(F, BK);
+    q.M = (int)T;
+    q.N = dm;
+    q.m_tiles = ceil_div(T, BM);
+    q.n_tiles = ceil_div(dm, BN);
+    q.c[0] = out;
+    q.ldc[0] = dm;
+    q.status = status;
+    MOC_LAUNCH(KID_TC_DOWN_GEMM, st, (rc = launch_gemm<false, true, EPI_BF16>(q, st)));
+    return rc;
+}
+
+int backward_tc(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat16 *wg, const __nv_bfloat16 *wu,
+                const __nv_bfloat16 *wd, const int16_t *idx, const __nv_bfloat16 *tg, const __nv_bfloat16 *tu,
+                const __nv_bfloat16 *dout, __nv_bfloat16 *gx, __nv_bfloat16 *gwg, __nv_bfloat16 *gwu,
+                __nv_bfloat16 *gwd, char *ws, cudaStream_t st) {
+    using namespace tc;
+    const TcBackwardLayout L = tc_backward_layout(d);
+    __nv_bfloat16 *Zp = reinterpret_cast<__nv_bfloat16 *>(ws + L.off_z);
+    __nv_bfloat16 *dUp = reinterpret_cast<__nv_bfloat16 *>(ws + L.off_du);
+    __nv_bfloat16 *dGp = reinterpret_cast<__nv_bfloat16 *>(ws + L.off_dg);
+    int32_t *tile_start = reinterpret_cast<int32_t *>(ws + L.off_tile_start);
+    const int F = d.d_ff, K = d.k, dm = d.d_model;
+    const int64_t T = d.tokens;
+    int *status = device_status_ptr();
+    if (!status) return MOC_ERR_CUDA;
+    int rc;
+
+    MOC_LAUNCH(KID_TC_TILE_START, st,
+               (tile_start_kernel<<<(unsigned)((T + 7) / 8), 256, 0, st>>>(idx, T, K, F, L.n_tiles, tile_start,
+                                                                          status)));
+    if ((rc = launch_ok()) != MOC_OK) return rc;
+
+    // dZ = dD Wd^T sampled at the saved indices -> dense masked Z', dU', dG'   (Eqs. (bp-1)..(bp-3))
+    {
+        Params p;
+        init_params(p);
+        if (!map_k_major(&p.a_map[0], dout, T, dm, dm, BM) || !map_k_major(&p.b_map[0], wd, F, dm, dm, BN))
+            return MOC_ERR_CUDA;
+        p.k_blocks = ceil_div(dm, BK);
+        p.M = (int)T;
+        p.N = F;
+        p.m_tiles = ceil_div(T, BM);
+        p.n_tiles = L.n_tiles;
+        p.c[0] = Zp;
+        p.c[1] = dUp;
+        p.c[2] = dGp;
+        p.ldc[0] = p.ldc[1] = p.ldc[2] = L.ldf;
+        p.idx = idx;
+        p.gval = tg;
+        p.uval = tu;
+        p.tile_start = tile_start;
+        p.topk = K;
+        p.d_ff = F;
+        p.status = status;
+        MOC_LAUNCH(KID_TC_DZ_GEMM, st, (rc = launch_gemm<false, false, EPI_DZ_SAMPLE>(p, st)));
+        if (rc != MOC_OK) return rc;
+    }
+    // weight gradients: dWd = Z'^T dD, dWu = dU'^T x, dWg = dG'^T x   (Eqs. (bp-1), (bp-4)); contraction over tokens
+    if (gwd || gwu || gwg) {
+        Params p;
+        init_params(p);
+        if (!map_mn_major(&p.b_map[0], dout, T, dm, dm) || !map_mn_major(&p.b_map[1], x, T, dm, dm))
+            return MOC_ERR_CUDA;
+        int np = 0;
+        auto add = [&](__nv_bfloat16 *dst, const __nv_bfloat16 *a, int bsel) {
+            if (!dst) return true;
+            if (!map_mn_major(&p.a_map[np], a, T, F, L.ldf)) return false;
+            p.a_idx[np][0] = (int8_t)np;
+            p.b_idx[np][0] = (int8_t)bsel;
+            p.c[np] = dst;
+            p.ldc[np] = dm;
+            ++np;
+            return true;
+        };
+        if (!add(gwd, Zp, 0) || !add(gwu, dUp, 1) || !add(gwg, dGp, 1)) return MOC_ERR_CUDA;
+        p.num_problems = np;
+        p.k_blocks = ceil_div(T, BK);
+        p.M = d.d_ff_ld;  // padding rows read zeros from the maps and are written as zeros
+        p.N = dm;
+        p.m_tiles = ceil_div(d.d_ff_ld, BM);
+        p.n_tiles = ceil_div(dm, BN);
+        p.accumulate = (d.flags & MOC_FLAG_ACCUMULATE_WGRAD) ? 1 : 0;
+        p.status = status;
+        MOC_LAUNCH(KID_TC_WGRAD_GEMM, st, (rc = launch_gemm<true, true, EPI_BF16>(p, st)));
+        if (rc != MOC_OK) return rc;
+    }
+    // dX = dG' Wg + dU' Wu   (Eq. (bp-5)): one accumulator, two contraction segments
+    if (gx) {
+        Params p;
+        init_params(p);
+        if (!map_k_major(&p.a_map[0], dGp, T, F, L.ldf, BM) || !map_k_major(&p.a_map[1], dUp, T, F, L.ldf, BM) ||
+            !map_mn_major(&p.b_map[0], wg, F, dm, dm) || !map_mn_major(&p.b_map[1], wu, F, dm, dm))
+            return MOC_ERR_CUDA;
+        p.k_segments = 2;
+        p.a_idx[0][1] = 1;
+        p.b_idx[0][1] = 1;
+        p.k_blocks = ceil_div(F, BK);
+        p.M = (int)T;
+        p.N = dm;
+        p.m_tiles = ceil_div(T, BM);
+        p.n_tiles = ceil_div(dm, BN);
+        p.c[0] = gx;
+        p.ldc[0] = dm;
+        p.status = status;
+        MOC_LAUNCH(KID_TC_DX_GEMM, st, (rc = launch_gemm<false, true, EPI_BF16>(p, st)));
+        if (rc != MOC_OK) return rc;
+    }
+    return MOC_OK;
+}
+
 }  // namespace
 }  // namespace moc
 
@@ -278,12 +459,12 @@ size_t moc_ffn_workspace_bytes(const moc_ffn_desc *desc, int op) {
     if (desc->tokens == 0) return 0;
     switch (op) {
         case MOC_OP_FORWARD:
-            return plan_forward(*desc).total;
+            return use_tc_plan(*desc) ? tc::tc_forward_layout(*desc).total : plan_forward(*desc).total;
         case MOC_OP_DECODE:
             if (desc->tokens > 16) return 0;
             return plan_forward(*desc).total;
         case MOC_OP_BACKWARD:
-            return plan_backward(*desc).total;
+            return use_tc_plan(*desc) ? tc::tc_backward_layout(*desc).total : plan_backward(*desc).total;
         default:
             return 0;
     }
@@ -313,6 +494,9 @@ int moc_ffn_forward(const moc_ffn_desc *desc, const void *x, const void *w_gate,
     char *ws = static_cast<char *>(workspace);
     if (desc->dtype == MOC_BF16) {
         using T = __nv_bfloat16;
+        if (use_tc_plan(*desc))
+            return forward_tc(*desc, (const T *)x, (const T *)w_gate, (const T *)w_up, (const T *)w_down, (T *)out,
+                              topk_idx, (T *)topk_gate, (T *)topk_up, ws, st);
         return forward_gather<T>(*desc, (const T *)x, (const T *)w_gate, (const T *)w_up, (const T *)w_down,
                                  (T *)out, topk_idx, (T *)topk_gate, (T *)topk_up, ws, st);
     }
@@ -353,6 +537,10 @@ int moc_ffn_backward(const moc_ffn_desc *desc, const void *x, const void *w_gate
     char *ws = static_cast<char *>(workspace);
     if (desc->dtype == MOC_BF16) {
         using T = __nv_bfloat16;
+        if (use_tc_plan(*desc))
+            return backward_tc(*desc, (const T *)x, (const T *)w_gate, (const T *)w_up, (const T *)w_down, topk_idx,
+                               (const T *)topk_gate, (const T *)topk_up, (const T *)grad_out, (T *)grad_x,
+                               (T *)grad_w_gate, (T *)grad_w_up, (T *)grad_w_down, ws, st);
         return backward_gather<T>(*desc, (const T *)x, (const T *)w_gate, (const T *)w_up, (const T *)w_down,
                                   topk_idx, (const T *)topk_gate, (const T *)topk_up, (const T *)grad_out,
                                   (T *)grad_x, (T *)grad_w_gate, (T *)grad_w_up, (T *)grad_w_down, ws, st);
@@ -426,6 +614,39 @@ int moc_ffn_decode_static(const moc_ffn_desc *desc, const void *x, const void *w
     }
     return forward_gather<float>(*desc, (const float *)x, (const float *)w_gate, (const float *)w_up,
                                  (const float *)w_down, (float *)out, nullptr, nullptr, nullptr, ws, st);
+}
+
+int moc_tc_gemm_bf16(int64_t m, int64_t n, int64_t k, const void *a, int a_mn_major, int64_t lda, const void *b,
+                     int b_mn_major, int64_t ldb, float *c, int64_t ldc, void *cuda_stream) {
+    using namespace tc;
+    if (m < 1 || n < 1 || k < 1 || m > INT32_MAX || n > INT32_MAX || k > INT32_MAX) return MOC_ERR_INVALID_ARG;
+    if (!good_ptr(a) || !good_ptr(b) || !good_ptr(c) || lda % 8 || ldb % 8 || ldc < n) return MOC_ERR_INVALID_ARG;
+    int *status = device_status_ptr();
+    if (!status) return MOC_ERR_CUDA;
+    Params p;
+    init_params(p);
+    const bool ok_a = a_mn_major ? map_mn_major(&p.a_map[0], a, k, m, lda) : map_k_major(&p.a_map[0], a, m, k, lda, BM);
+    const bool ok_b = b_mn_major ? map_mn_major(&p.b_map[0], b, k, n, ldb) : map_k_major(&p.b_map[0], b, n, k, ldb, BN);
+    if (!ok_a || !ok_b) return MOC_ERR_CUDA;
+    p.k_blocks = ceil_div(k, BK);
+    p.M = (int)m;
+    p.N = (int)n;
+    p.m_tiles = ceil_div(m, BM);
+    p.n_tiles = ceil_div(n, BN);
+    p.c[0] = c;
+    p.ldc[0] = (int)ldc;
+    p.status = status;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    int rc = MOC_OK;
+    if (!a_mn_major && !b_mn_major)
+        MOC_LAUNCH(KID_TC_TEST_GEMM, st, (rc = launch_gemm<false, false, EPI_F32>(p, st)));
+    else if (!a_mn_major && b_mn_major)
+        MOC_LAUNCH(KID_TC_TEST_GEMM, st, (rc = launch_gemm<false, true, EPI_F32>(p, st)));
+    else if (a_mn_major && b_mn_major)
+        MOC_LAUNCH(KID_TC_TEST_GEMM, st, (rc = launch_gemm<true, true, EPI_F32>(p, st)));
+    else
+        MOC_LAUNCH(KID_TC_TEST_GEMM, st, (rc = launch_gemm<true, false, EPI_F32>(p, st)));
+    return rc;
 }
 
 int moc_last_device_status(void *cuda_stream) {

@@ -1,0 +1,458 @@
+// bf16 tensor-core GEMM for sm_100a: tcgen05.mma with TMEM accumulators, TMA-fed operands.
+//
+// One persistent CTA per SM (192 threads): warp 0 issues TMA loads, warp 1 issues tcgen05.mma and
+// owns the TMEM allocation, warps 2..5 run the epilogue.  Output tile 128 x 256, K step 64, four
+// shared-memory stages (48 KiB each), two accumulator stages in TMEM (2 x 256 columns) so that the
+// epilogue of tile i overlaps the main loop of tile i+1.
+//
+// Operands may be K-major (rows of 64 contraction elements = one 128-byte swizzle row) or MN-major
+// (the tensor's contiguous dimension is M or N; loaded as 64-wide boxes of 64 contraction rows).
+// Several "problems" (up to 3) can share one launch, and a problem's contraction may run over two
+// segments with different operand tensors; that is how the MoC contractions are batched:
+//   forward   [G | U]          = x  * [Wg ; Wu]^T        two problems, shared A
+//   forward   D                = Z' * Wd                 B is MN-major
+//   backward  dZ               = dD * Wd^T               epilogue samples at the saved indices
+//   backward  dWd | dWu | dWg  = Z'^T dD | dU'^T x | dG'^T x    three problems, both operands MN-major
+//   backward  dX               = dG' * Wg + dU' * Wu     two contraction segments, B is MN-major
+//
+// Every wait on an mbarrier is bounded: when the bound expires the kernel raises MOC_ERR_TIMEOUT in
+// the device status word, all roles leave their loops, the CTA waits a fixed time for copies in
+// flight, frees its TMEM and returns.
+#pragma once
+
+#include <cuda.h>
+
+#include "moc_common.cuh"
+
+namespace moc {
+namespace tc {
+
+constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4, ACC_STAGES = 2;
+constexpr int THREADS = 192;
+constexpr uint32_t A_STAGE_BYTES = BM * BK * 2, B_STAGE_BYTES = BN * BK * 2;
+constexpr uint32_t STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
+constexpr uint32_t TMEM_COLS = ACC_STAGES * BN;  // 512
+constexpr size_t SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)STAGES * STAGE_BYTES + 256 /*barriers*/;
+
+enum Epilogue : int {
+    EPI_F32 = 0,       // C fp32 [M, ldc]
+    EPI_GATE_UP = 1,   // problem 0 -> fp32 G [M, ldg]; problem 1 -> bf16 U [M, ldu]
+    EPI_BF16 = 2,      // C bf16 [M, ldc]  (optionally accumulating into C)
+    EPI_DZ_SAMPLE = 3  // dZ tile sampled at the saved indices -> dense masked Z', dU', dG' bf16 [M, ldz]
+};
+
+struct Params {
+    CUtensorMap a_map[3];
+    CUtensorMap b_map[3];
+    int8_t a_idx[3][2];  // [problem][segment] -> tensor map index
+    int8_t b_idx[3][2];
+    int num_problems;    // 1..3
+    int k_segments;      // 1..2
+    int k_blocks;        // 64-wide contraction blocks per segment
+    int M, N;            // output extent of one problem (rows = A-side, cols = B-side)
+    int m_tiles, n_tiles;
+    int accumulate;      // EPI_BF16: add the previous content of C
+    // outputs
+    void *c[3];          // per problem
+    int ldc[3];
+    // EPI_DZ_SAMPLE
+    const int16_t *idx;            // [M, K]
+    const __nv_bfloat16 *gval;     // [M, K]
+    const __nv_bfloat16 *uval;     // [M, K]
+    const int32_t *tile_start;     // [M, n_tiles]: first position p with idx[t,p] >= n_blk*BN
+    int topk;
+    int d_ff;                      // indices >= d_ff are invalid
+    int *status;
+};
+
+// ---------------------------------------------------------------------------------------------- PTX
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait (about two seconds of SM clock).  Returns false when it gave up or another role already did.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    uint32_t spins = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++spins & 0x3ff) == 0) {
+            if (*abort_flag) return false;
+            if (clock64() - t0 > 4000000000LL) {
+                *abort_flag = 1;
+                raise_status(status, MOC_ERR_TIMEOUT);
+                return false;
+            }
+        }
+    }
+    return true;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y)
+        : "memory");
+}
+__device__ __forceinline__ void prefetch_tmap(const CUtensorMap *map) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols)
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                          uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
+                 : "memory");
+}
+
+// 32 consecutive fp32 columns of this thread's TMEM lane
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// ---------------------------------------------------------------------------------------------- descriptors
+// Shared-memory matrix descriptor, 128-byte swizzle, version 1 (sm_100).
+//   K-major : rows of 128 bytes, 8-row groups 1024 bytes apart            (LBO unused, SBO = 1024)
+//   MN-major: 64-element (128-byte) rows along MN, one row per k; 8 k-rows = 1024 bytes (SBO);
+//             the next 64 elements along MN live in the next 64 x BK box (LBO = BK * 128 bytes)
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3ffffu) >> 4);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3fffu) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3fffu) << 32;
+    d |= (uint64_t)1 << 46;  // descriptor version
+    d |= (uint64_t)2 << 61;  // SWIZZLE_128B
+    return d;
+}
+
+template <bool A_MN, bool B_MN>
+__device__ __forceinline__ constexpr uint32_t make_idesc() {
+    return (1u << 4)                        // D format: fp32
+           | (1u << 7) | (1u << 10)         // A, B format: bf16
+           | ((A_MN ? 1u : 0u) << 15) | ((B_MN ? 1u : 0u) << 16)
+           | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+}
+
+// ---------------------------------------------------------------------------------------------- epilogue helpers
+__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
+    __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+    return *reinterpret_cast<uint32_t *>(&h);
+}
+
+// store 32 consecutive outputs of one row; full vector path when the chunk is inside the row and aligned
+__device__ __forceinline__ void store_row_f32(float *dst, const uint32_t (&r)[32], int valid) {
+    if (valid >= 32 && ((reinterpret_cast<uintptr_t>(dst) & 15u) == 0)) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+            reinterpret_cast<uint4 *>(dst)[i] = make_uint4(r[4 * i], r[4 * i + 1], r[4 * i + 2], r[4 * i + 3]);
+    } else {
+#pragma unroll
+        for (int i = 0; i < 32; ++i)
+            if (i < valid) dst[i] = __uint_as_float(r[i]);
+    }
+}
+__device__ __forceinline__ void store_row_bf16(__nv_bfloat16 *dst, const float (&v)[32], int valid) {
+    if (valid >= 32 && ((reinterpret_cast<uintptr_t>(dst) & 15u) == 0)) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            reinterpret_cast<uint4 *>(dst)[i] =
+                make_uint4(pack_bf16(v[8 * i], v[8 * i + 1]), pack_bf16(v[8 * i + 2], v[8 * i + 3]),
+                           pack_bf16(v[8 * i + 4], v[8 * i + 5]), pack_bf16(v[8 * i + 6], v[8 * i + 7]));
+    } else {
+#pragma unroll
+        for (int i = 0; i < 32; ++i)
+            if (i < valid) dst[i] = __float2bfloat16_rn(v[i]);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------- kernel
+template <bool A_MN, bool B_MN, int EPI>
+__global__ void __launch_bounds__(THREADS, 1) gemm_kernel(const __grid_constant__ Params p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;  // 128-byte swizzle atoms need 1024-byte alignment
+    uint8_t *smem = smem_raw + (base - raw);
+    const uint32_t bar_base = base + STAGES * STAGE_BYTES;
+    auto full_bar = [&](int s) { return bar_base + 8u * s; };
+    auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
+    auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
+    auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + ACC_STAGES + a); };
+    volatile uint32_t *tmem_holder =
+        reinterpret_cast<volatile uint32_t *>(smem + STAGES * STAGE_BYTES + 8 * (2 * STAGES + 2 * ACC_STAGES));
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_holder + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int tiles_per_problem = p.m_tiles * p.n_tiles;
+    const int total_tiles = tiles_per_problem * p.num_problems;
+    const int kb_total = p.k_blocks * p.k_segments;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(full_bar(s), 1);
+            mbar_init(empty_bar(s), 1);
+        }
+        for (int a = 0; a < ACC_STAGES; ++a) {
+            mbar_init(tfull_bar(a), 1);
+            mbar_init(tempty_bar(a), 4);  // one arrival per epilogue warp
+        }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(const_cast<uint32_t *>(tmem_holder)), TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_holder;
+
+    // tile id -> (m block, problem, n block): all tiles of one m block are adjacent, so CTAs running at
+    // the same time share A rows and the (small) B operands stay in L2
+    auto decode_tile = [&](int tile, int &m_blk, int &prob, int &n_blk) {
+        const int per_m = p.num_problems * p.n_tiles;
+        m_blk = tile / per_m;
+        const int r = tile - m_blk * per_m;
+        prob = r / p.n_tiles;
+        n_blk = r - prob * p.n_tiles;
+    };
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            for (int i = 0; i < 3; ++i) {
+                prefetch_tmap(&p.a_map[i]);
+                prefetch_tmap(&p.b_map[i]);
+            }
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+                int m_blk, prob, n_blk;
+                decode_tile(tile, m_blk, prob, n_blk);
+                for (int kb = 0; kb < kb_total; ++kb) {
+                    if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status)) {
+                        ok = false;
+                        break;
+                    }
+                    const int seg = kb / p.k_blocks, kk = (kb - seg * p.k_blocks) * BK;
+                    const CUtensorMap *am = &p.a_map[p.a_idx[prob][seg]];
+                    const CUtensorMap *bm = &p.b_map[p.b_idx[prob][seg]];
+                    const uint32_t sa = base + stage * STAGE_BYTES, sb = sa + A_STAGE_BYTES;
+                    mbar_expect_tx(full_bar(stage), STAGE_BYTES);
+                    if (A_MN) {
+#pragma unroll
+                        for (int i = 0; i < BM / 64; ++i)
+                            tma_load_2d(sa + i * (64 * BK * 2), am, full_bar(stage), m_blk * BM + i * 64, kk);
+                    } else {
+                        tma_load_2d(sa, am, full_bar(stage), kk, m_blk * BM);
+                    }
+                    if (B_MN) {
+#pragma unroll
+                        for (int i = 0; i < BN / 64; ++i)
+                            tma_load_2d(sb + i * (64 * BK * 2), bm, full_bar(stage), n_blk * BN + i * 64, kk);
+                    } else {
+                        tma_load_2d(sb, bm, full_bar(stage), kk, n_blk * BN);
+                    }
+                    if (++stage == STAGES) {
+                        stage = 0;
+                        phase ^= 1u;
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = make_idesc<A_MN, B_MN>();
+            int stage = 0, acc = 0;
+            uint32_t phase = 0, acc_phase = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+                if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, p.status)) break;
+                tc_fence_after();
+                const uint32_t tmem_d = tmem_base + (uint32_t)acc * BN;
+                for (int kb = 0; kb < kb_total; ++kb) {
+                    if (!mbar_wait(full_bar(stage), phase, abort_flag, p.status)) {
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint32_t sa = base + stage * STAGE_BYTES, sb = sa + A_STAGE_BYTES;
+#pragma unroll
+                    for (int k = 0; k < BK / 16; ++k) {
+                        // one instruction consumes 16 contraction elements: 32 bytes along a K-major row,
+                        // or 16 rows of 128 bytes in an MN-major box
+                        const uint64_t ad = A_MN ? make_smem_desc(sa + k * 2048, BK * 128, 1024)
+                                                 : make_smem_desc(sa + k * 32, 16, 1024);
+                        const uint64_t bd = B_MN ? make_smem_desc(sb + k * 2048, BK * 128, 1024)
+                                                 : make_smem_desc(sb + k * 32, 16, 1024);
+                        umma_bf16(tmem_d, ad, bd, idesc, (kb | k) != 0 ? 1u : 0u);
+                    }
+                    umma_commit(empty_bar(stage));  // frees the stage once these MMAs have read it
+                    if (++stage == STAGES) {
+                        stage = 0;
+                        phase ^= 1u;
+                    }
+                }
+                if (!ok) break;
+                umma_commit(tfull_bar(acc));  // accumulator complete
+                if (++acc == ACC_STAGES) {
+                    acc = 0;
+                    acc_phase ^= 1u;
+                }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue (warps 2..5)
+        const int quarter = warp & 3;  // TMEM lanes 32*quarter .. +31 are the ones this warp may read
+        int acc = 0;
+        uint32_t acc_phase = 0;
+        for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+            int m_blk, prob, n_blk;
+            decode_tile(tile, m_blk, prob, n_blk);
+            // the whole warp must agree: the TMEM loads below are warp-collective
+            if (!__all_sync(0xffffffffu, mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.status))) break;
+            tc_fence_after();
+            const int row = m_blk * BM + quarter * 32 + lane;
+            const bool row_ok = row < p.M;
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)acc * BN;
+            const int n0 = n_blk * BN;
+
+            // EPI_DZ_SAMPLE: walk this row's saved (ascending) indices in step with the columns
+            int pos = 0, next_j = 0x7fffffff;
+            const int16_t *irow = nullptr;
+            if (EPI == EPI_DZ_SAMPLE && row_ok) {
+                irow = p.idx + (int64_t)row * p.topk;
+                pos = p.tile_start[(int64_t)row * p.n_tiles + n_blk];
+                if (pos < p.topk) next_j = irow[pos];
+            }
+
+#pragma unroll 1
+            for (int c0 = 0; c0 < BN; c0 += 32) {
+                uint32_t r[32];
+                __syncwarp();
+                tmem_ld32(taddr + (uint32_t)c0, r);
+                tmem_ld_wait();
+                const int col = n0 + c0;
+                const int valid = p.N - col;  // columns of this chunk inside the problem
+                if (!row_ok || valid <= 0) continue;
+                if (EPI == EPI_F32 || (EPI == EPI_GATE_UP && prob == 0)) {
+                    float *dst = static_cast<float *>(p.c[prob]) + (int64_t)row * p.ldc[prob] + col;
+                    store_row_f32(dst, r, valid);
+                } else if (EPI == EPI_BF16 || EPI == EPI_GATE_UP) {
+                    __nv_bfloat16 *dst = static_cast<__nv_bfloat16 *>(p.c[prob]) + (int64_t)row * p.ldc[prob] + col;
+                    float v[32];
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+                    if (EPI == EPI_BF16 && p.accumulate) {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            if (i < valid) v[i] += __bfloat162float(dst[i]);
+                    }
+                    store_row_bf16(dst, v, valid);
+                } else {  // EPI_DZ_SAMPLE
+                    float vz[32], vu[32], vg[32];
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        vz[i] = 0.f;
+                        vu[i] = 0.f;
+                        vg[i] = 0.f;
+                        if (next_j == col + i) {
+                            const float dz = __uint_as_float(r[i]);
+                            const float g = __bfloat162float(p.gval[(int64_t)row * p.topk + pos]);
+                            const float u = __bfloat162float(p.uval[(int64_t)row * p.topk + pos]);
+                            const float s = silu_f(g);
+                            vz[i] = s * u;                  // Z' = S' . U          (recomputed)
+                            vu[i] = s * dz;                 // dU = S' . dZ'
+                            vg[i] = u * dz * dsilu_f(g);    // dG = (U.M) . dZ' . SiLU'(G)
+                            ++pos;
+                            next_j = pos < p.topk ? (int)irow[pos] : 0x7fffffff;
+                        }
+                    }
+                    const int64_t o = (int64_t)row * p.ldc[0] + col;
+                    store_row_bf16(static_cast<__nv_bfloat16 *>(p.c[0]) + o, vz, valid);
+                    store_row_bf16(static_cast<__nv_bfloat16 *>(p.c[1]) + o, vu, valid);
+                    store_row_bf16(static_cast<__nv_bfloat16 *>(p.c[2]) + o, vg, valid);
+                }
+            }
+            if (EPI == EPI_DZ_SAMPLE && row_ok && next_j < n0 + BN && next_j < p.d_ff) {
+                // an index inside this tile was not consumed: the saved list is not ascending
+                raise_status(p.status, MOC_ERR_BAD_INDEX);
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tempty_bar(acc));
+            if (++acc == ACC_STAGES) {
+                acc = 0;
+                acc_phase ^= 1u;
+            }
+        }
+    }
+
+    // ---------------------------------------------------------------------- teardown
+    __syncwarp();
+    if (*abort_flag) {
+        // give copies and MMAs still in flight time to land before shared memory and TMEM go away
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000LL) __nanosleep(1000);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+}  // namespace tc
+}  // namespace moc
