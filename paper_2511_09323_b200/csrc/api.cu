@@ -50,18 +50,19 @@ enum KernelId {
     KID_TC_GATE_UP_GEMM,
     KID_TC_SELECT_MASK,
     KID_TC_DOWN_GEMM,
-    KID_TC_TILE_START,
+    KID_TC_BWD_SAMPLE,
     KID_TC_DZ_GEMM,
     KID_TC_WGRAD_GEMM,
     KID_TC_DX_GEMM,
     KID_TC_TEST_GEMM,
+    KID_TC_SELECT_HINT,
     KID_COUNT
 };
 static const char *const kKernelNames[KID_COUNT] = {
     "gate_gemm_alu", "select_rows",       "forward_token", "backward_token", "csr_count",
     "csr_scan_blocks", "csr_scan_channels", "csr_fill",      "wgrad_rows",     "topk_select",
-    "tc_gate_up_gemm", "tc_select_mask",  "tc_down_gemm",  "tc_tile_start",  "tc_dz_gemm",
-    "tc_wgrad_gemm",   "tc_dx_gemm",      "tc_test_gemm",
+    "tc_gate_up_gemm", "tc_select_mask",  "tc_down_gemm",  "tc_bwd_sample",  "tc_dz_gemm",
+    "tc_wgrad_gemm",   "tc_dx_gemm",      "tc_test_gemm",  "tc_select_hint",
 };
 
 struct Profiler {
@@ -176,8 +177,10 @@ BackwardPlan plan_backward(const moc_ffn_desc &d) {
 
 template <typename K>
 int set_smem(K kernel, size_t bytes) {
-    if (bytes > (size_t)kMaxDynSmem) return MOC_ERR_UNSUPPORTED;
-    if (bytes > 48 * 1024) {
+    // kernels that use the selector also hold its static shared state (about 14 KiB)
+    constexpr size_t kStaticReserve = 16 * 1024;
+    if (bytes + kStaticReserve > (size_t)kMaxDynSmem) return MOC_ERR_UNSUPPORTED;
+    if (bytes + kStaticReserve > 48 * 1024) {
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess)
             return MOC_ERR_CUDA;
     }
@@ -297,9 +300,22 @@ int forward_tc(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat1
     const int64_t T = d.tokens;
     const int f_tiles = ceil_div(F, BN);
 
-    const size_t sel_smem = ((size_t)F + K) * sizeof(uint32_t);
-    int rc = set_smem(select_mask_rows_kernel, sel_smem);
+    // selector: one warp per token while a row fits in registers (F <= 4096), else one CTA per token
+    const int nv = F <= 1024 ? 8 : (F <= 2048 ? 16 : (F <= 4096 ? 32 : 0));
+    const size_t warp_smem = 8 * ((size_t)kWarpSelCand + 2 * (size_t)K) * sizeof(uint32_t);
+    const size_t cta_smem = ((size_t)F + K) * sizeof(uint32_t);
+    const bool warp_select = nv != 0 && warp_smem + 16 * 1024 <= (size_t)kMaxDynSmem;
+    float *hint = reinterpret_cast<float *>(ws + L.off_hint);
+    int rc = MOC_OK;
+    if (warp_select) {
+        if (nv == 8) rc = set_smem(select_mask_rows_warp_kernel<8>, warp_smem);
+        if (nv == 16) rc = set_smem(select_mask_rows_warp_kernel<16>, warp_smem);
+        if (nv == 32) rc = set_smem(select_mask_rows_warp_kernel<32>, warp_smem);
+    } else {
+        rc = set_smem(select_mask_rows_kernel, cta_smem);
+    }
     if (rc != MOC_OK) return rc;
+    if ((rc = set_smem(select_hint_kernel, (size_t)F * sizeof(uint32_t))) != MOC_OK) return rc;
 
     int *status = device_status_ptr();
     if (!status) return MOC_ERR_CUDA;
@@ -323,11 +339,34 @@ int forward_tc(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat1
         p.c[1] = U + t0 * L.ldf;
         MOC_LAUNCH(KID_TC_GATE_UP_GEMM, st, (rc = launch_gemm<false, false, EPI_GATE_UP>(p, st)));
         if (rc != MOC_OK) return rc;
-        const unsigned grid = (unsigned)std::min<int64_t>(n, (int64_t)sm_count() * 8);
-        MOC_LAUNCH(KID_TC_SELECT_MASK, st,
-                   (select_mask_rows_kernel<<<grid, kSelectThreads, sel_smem, st>>>(
-                       G, L.ldf, U + t0 * L.ldf, L.ldf, n, F, K, idx ? idx + t0 * K : nullptr,
-                       idx ? tg + t0 * K : nullptr, idx ? tu + t0 * K : nullptr)));
+        if (t0 == 0) {
+            MOC_LAUNCH(KID_TC_SELECT_HINT, st,
+                       (select_hint_kernel<<<1, kSelectThreads, (size_t)F * sizeof(uint32_t), st>>>(G, F, K, hint)));
+            if ((rc = launch_ok()) != MOC_OK) return rc;
+        }
+        int16_t *o_idx = idx ? idx + t0 * K : nullptr;
+        __nv_bfloat16 *o_g = idx ? tg + t0 * K : nullptr, *o_u = idx ? tu + t0 * K : nullptr;
+        __nv_bfloat16 *Uc = U + t0 * L.ldf;
+        if (warp_select) {
+            const unsigned grid = (unsigned)std::min<int64_t>((n + 7) / 8, (int64_t)sm_count() * 4);
+            if (nv == 8)
+                MOC_LAUNCH(KID_TC_SELECT_MASK, st,
+                           (select_mask_rows_warp_kernel<8><<<grid, 256, warp_smem, st>>>(G, L.ldf, Uc, L.ldf, n, F, K,
+                                                                                           o_idx, o_g, o_u, hint)));
+            else if (nv == 16)
+                MOC_LAUNCH(KID_TC_SELECT_MASK, st,
+                           (select_mask_rows_warp_kernel<16><<<grid, 256, warp_smem, st>>>(G, L.ldf, Uc, L.ldf, n, F, K,
+                                                                                            o_idx, o_g, o_u, hint)));
+            else
+                MOC_LAUNCH(KID_TC_SELECT_MASK, st,
+                           (select_mask_rows_warp_kernel<32><<<grid, 256, warp_smem, st>>>(G, L.ldf, Uc, L.ldf, n, F, K,
+                                                                                            o_idx, o_g, o_u, hint)));
+        } else {
+            const unsigned grid = (unsigned)std::min<int64_t>(n, (int64_t)sm_count() * 6);
+            MOC_LAUNCH(KID_TC_SELECT_MASK, st,
+                       (select_mask_rows_kernel<<<grid, kSelectThreads, cta_smem, st>>>(G, L.ldf, Uc, L.ldf, n, F, K,
+                                                                                         o_idx, o_g, o_u, hint)));
+        }
         if ((rc = launch_ok()) != MOC_OK) return rc;
     }
     // D = Z' W_down over all tokens: A = Z' [T, F] (K-major), B = Wd [F, d] (its contiguous dimension is N)
@@ -356,19 +395,13 @@ int backward_tc(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat
     __nv_bfloat16 *Zp = reinterpret_cast<__nv_bfloat16 *>(ws + L.off_z);
     __nv_bfloat16 *dUp = reinterpret_cast<__nv_bfloat16 *>(ws + L.off_du);
     __nv_bfloat16 *dGp = reinterpret_cast<__nv_bfloat16 *>(ws + L.off_dg);
-    int32_t *tile_start = reinterpret_cast<int32_t *>(ws + L.off_tile_start);
     const int F = d.d_ff, K = d.k, dm = d.d_model;
     const int64_t T = d.tokens;
     int *status = device_status_ptr();
     if (!status) return MOC_ERR_CUDA;
     int rc;
 
-    MOC_LAUNCH(KID_TC_TILE_START, st,
-               (tile_start_kernel<<<(unsigned)((T + 7) / 8), 256, 0, st>>>(idx, T, K, F, L.n_tiles, tile_start,
-                                                                          status)));
-    if ((rc = launch_ok()) != MOC_OK) return rc;
-
-    // dZ = dD Wd^T sampled at the saved indices -> dense masked Z', dU', dG'   (Eqs. (bp-1)..(bp-3))
+    // dZ = dD Wd^T (dense, bf16), then the element-wise step at the saved indices -> masked Z', dU', dG'
     {
         Params p;
         init_params(p);
@@ -378,20 +411,19 @@ int backward_tc(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat
         p.M = (int)T;
         p.N = F;
         p.m_tiles = ceil_div(T, BM);
-        p.n_tiles = L.n_tiles;
+        p.n_tiles = ceil_div(F, BN);
         p.c[0] = Zp;
-        p.c[1] = dUp;
-        p.c[2] = dGp;
-        p.ldc[0] = p.ldc[1] = p.ldc[2] = L.ldf;
-        p.idx = idx;
-        p.gval = tg;
-        p.uval = tu;
-        p.tile_start = tile_start;
-        p.topk = K;
-        p.d_ff = F;
+        p.ldc[0] = L.ldf;
         p.status = status;
-        MOC_LAUNCH(KID_TC_DZ_GEMM, st, (rc = launch_gemm<false, false, EPI_DZ_SAMPLE>(p, st)));
+        MOC_LAUNCH(KID_TC_DZ_GEMM, st, (rc = launch_gemm<false, false, EPI_BF16>(p, st)));
         if (rc != MOC_OK) return rc;
+        const size_t smem = (size_t)K * 8;
+        if ((rc = set_smem(backward_sample_rows_kernel, smem)) != MOC_OK) return rc;
+        const unsigned grid = (unsigned)std::min<int64_t>(T, (int64_t)sm_count() * 8);
+        MOC_LAUNCH(KID_TC_BWD_SAMPLE, st,
+                   (backward_sample_rows_kernel<<<grid, 256, smem, st>>>(idx, tg, tu, T, K, F, L.ldf, Zp, dUp, dGp,
+                                                                         status)));
+        if ((rc = launch_ok()) != MOC_OK) return rc;
     }
     // weight gradients: dWd = Z'^T dD, dWu = dU'^T x, dWg = dG'^T x   (Eqs. (bp-1), (bp-4)); contraction over tokens
     if (gwd || gwu || gwg) {

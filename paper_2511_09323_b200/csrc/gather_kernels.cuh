@@ -80,18 +80,19 @@ __global__ void __launch_bounds__(kSelectThreads) select_rows_kernel(const float
                                                                       T *__restrict__ topk_gate) {
     extern __shared__ __align__(16) uint32_t select_keys[];
     __shared__ SelectSmem sm;
+    SelectGuess guess;
     for (int64_t r = blockIdx.x; r < rows; r += gridDim.x) {
         const float *g = G + r * (int64_t)ldg;
-        for (int j = threadIdx.x; j < F; j += kSelectThreads) select_keys[j] = gate_key(g[j]);
-        __syncthreads();
         uint32_t tau;
         int need;
-        block_radix_threshold<kSelectThreads>(select_keys, F, K, sm, tau, need);
+        block_select_row<kSelectThreads>(g, F, K, select_keys, sm, guess, tau, need);
         int16_t *o = idx_out + r * (int64_t)K;
         T *og = topk_gate ? topk_gate + r * (int64_t)K : nullptr;
         block_ordered_emit<kSelectThreads>(select_keys, F, tau, need, sm, [&](int pos, int j) {
             o[pos] = (int16_t)j;
-            if (og) og[pos] = from_f32<T>(g[j]);
+            // the value comes back from the key in shared memory: a global load inside the ordered walk
+            // would cost a memory round trip per chunk
+            if (og) og[pos] = from_f32<T>(key_to_float(select_keys[j]));
         });
         __syncthreads();
     }

@@ -11,7 +11,7 @@
 // segments with different operand tensors; that is how the MoC contractions are batched:
 //   forward   [G | U]          = x  * [Wg ; Wu]^T        two problems, shared A
 //   forward   D                = Z' * Wd                 B is MN-major
-//   backward  dZ               = dD * Wd^T               epilogue samples at the saved indices
+//   backward  dZ               = dD * Wd^T
 //   backward  dWd | dWu | dWg  = Z'^T dD | dU'^T x | dG'^T x    three problems, both operands MN-major
 //   backward  dX               = dG' * Wg + dU' * Wu     two contraction segments, B is MN-major
 //
@@ -37,8 +37,7 @@ constexpr size_t SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)STAGES * STAGE_
 enum Epilogue : int {
     EPI_F32 = 0,       // C fp32 [M, ldc]
     EPI_GATE_UP = 1,   // problem 0 -> fp32 G [M, ldg]; problem 1 -> bf16 U [M, ldu]
-    EPI_BF16 = 2,      // C bf16 [M, ldc]  (optionally accumulating into C)
-    EPI_DZ_SAMPLE = 3  // dZ tile sampled at the saved indices -> dense masked Z', dU', dG' bf16 [M, ldz]
+    EPI_BF16 = 2       // C bf16 [M, ldc]  (optionally accumulating into C)
 };
 
 struct Params {
@@ -55,13 +54,6 @@ struct Params {
     // outputs
     void *c[3];          // per problem
     int ldc[3];
-    // EPI_DZ_SAMPLE
-    const int16_t *idx;            // [M, K]
-    const __nv_bfloat16 *gval;     // [M, K]
-    const __nv_bfloat16 *uval;     // [M, K]
-    const int32_t *tile_start;     // [M, n_tiles]: first position p with idx[t,p] >= n_blk*BN
-    int topk;
-    int d_ff;                      // indices >= d_ff are invalid
     int *status;
 };
 
@@ -368,15 +360,6 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_kernel(const __grid_constant_
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)acc * BN;
             const int n0 = n_blk * BN;
 
-            // EPI_DZ_SAMPLE: walk this row's saved (ascending) indices in step with the columns
-            int pos = 0, next_j = 0x7fffffff;
-            const int16_t *irow = nullptr;
-            if (EPI == EPI_DZ_SAMPLE && row_ok) {
-                irow = p.idx + (int64_t)row * p.topk;
-                pos = p.tile_start[(int64_t)row * p.n_tiles + n_blk];
-                if (pos < p.topk) next_j = irow[pos];
-            }
-
 #pragma unroll 1
             for (int c0 = 0; c0 < BN; c0 += 32) {
                 uint32_t r[32];
@@ -400,34 +383,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_kernel(const __grid_constant_
                             if (i < valid) v[i] += __bfloat162float(dst[i]);
                     }
                     store_row_bf16(dst, v, valid);
-                } else {  // EPI_DZ_SAMPLE
-                    float vz[32], vu[32], vg[32];
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        vz[i] = 0.f;
-                        vu[i] = 0.f;
-                        vg[i] = 0.f;
-                        if (next_j == col + i) {
-                            const float dz = __uint_as_float(r[i]);
-                            const float g = __bfloat162float(p.gval[(int64_t)row * p.topk + pos]);
-                            const float u = __bfloat162float(p.uval[(int64_t)row * p.topk + pos]);
-                            const float s = silu_f(g);
-                            vz[i] = s * u;                  // Z' = S' . U          (recomputed)
-                            vu[i] = s * dz;                 // dU = S' . dZ'
-                            vg[i] = u * dz * dsilu_f(g);    // dG = (U.M) . dZ' . SiLU'(G)
-                            ++pos;
-                            next_j = pos < p.topk ? (int)irow[pos] : 0x7fffffff;
-                        }
-                    }
-                    const int64_t o = (int64_t)row * p.ldc[0] + col;
-                    store_row_bf16(static_cast<__nv_bfloat16 *>(p.c[0]) + o, vz, valid);
-                    store_row_bf16(static_cast<__nv_bfloat16 *>(p.c[1]) + o, vu, valid);
-                    store_row_bf16(static_cast<__nv_bfloat16 *>(p.c[2]) + o, vg, valid);
                 }
-            }
-            if (EPI == EPI_DZ_SAMPLE && row_ok && next_j < n0 + BN && next_j < p.d_ff) {
-                // an index inside this tile was not consumed: the saved list is not ascending
-                raise_status(p.status, MOC_ERR_BAD_INDEX);
             }
             tc_fence_before();
             __syncwarp();
