@@ -8,6 +8,7 @@
 #include <cstring>
 #include <vector>
 
+#include "decode_kernels.cuh"
 #include "gather_kernels.cuh"
 #include "moc_common.cuh"
 #include "tc_gemm.cuh"
@@ -56,13 +57,18 @@ enum KernelId {
     KID_TC_DX_GEMM,
     KID_TC_TEST_GEMM,
     KID_TC_SELECT_HINT,
+    KID_DEC_GATE_GEMV,
+    KID_DEC_SELECT,
+    KID_DEC_UP,
+    KID_DEC_DOWN,
     KID_COUNT
 };
 static const char *const kKernelNames[KID_COUNT] = {
     "gate_gemm_alu", "select_rows",       "forward_token", "backward_token", "csr_count",
     "csr_scan_blocks", "csr_scan_channels", "csr_fill",      "wgrad_rows",     "topk_select",
     "tc_gate_up_gemm", "tc_select_mask",  "tc_down_gemm",  "tc_bwd_sample",  "tc_dz_gemm",
-    "tc_wgrad_gemm",   "tc_dx_gemm",      "tc_test_gemm",  "tc_select_hint",
+    "tc_wgrad_gemm",   "tc_dx_gemm",      "tc_test_gemm",  "tc_select_hint", "dec_gate_gemv",
+    "dec_select",      "dec_up",          "dec_down",
 };
 
 struct Profiler {
@@ -177,8 +183,8 @@ BackwardPlan plan_backward(const moc_ffn_desc &d) {
 
 template <typename K>
 int set_smem(K kernel, size_t bytes) {
-    // kernels that use the selector also hold its static shared state (about 14 KiB)
-    constexpr size_t kStaticReserve = 16 * 1024;
+    // kernels that use the selector also hold its static shared state (up to 47 KiB with 1024 threads)
+    constexpr size_t kStaticReserve = 48 * 1024;
     if (bytes + kStaticReserve > (size_t)kMaxDynSmem) return MOC_ERR_UNSUPPORTED;
     if (bytes + kStaticReserve > 48 * 1024) {
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess)
@@ -284,7 +290,7 @@ int backward_gather(const moc_ffn_desc &d, const T *x, const T *wg, const T *wu,
 bool use_tc_plan(const moc_ffn_desc &d) {
     if (d.dtype != MOC_BF16 || d.tokens < 256) return false;
     // the forward selector keeps F keys and K packed entries in shared memory
-    return ((size_t)d.d_ff + (size_t)d.k) * 4 <= 200 * 1024;
+    return ((size_t)d.d_ff + (size_t)d.k) * 4 <= 170 * 1024;
 }
 
 inline int ceil_div(int64_t a, int64_t b) { return (int)((a + b - 1) / b); }
@@ -304,7 +310,7 @@ int forward_tc(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat1
     const int nv = F <= 1024 ? 8 : (F <= 2048 ? 16 : (F <= 4096 ? 32 : 0));
     const size_t warp_smem = 8 * ((size_t)kWarpSelCand + 2 * (size_t)K) * sizeof(uint32_t);
     const size_t cta_smem = ((size_t)F + K) * sizeof(uint32_t);
-    const bool warp_select = nv != 0 && warp_smem + 16 * 1024 <= (size_t)kMaxDynSmem;
+    const bool warp_select = nv != 0 && warp_smem + 48 * 1024 <= (size_t)kMaxDynSmem;
     float *hint = reinterpret_cast<float *>(ws + L.off_hint);
     int rc = MOC_OK;
     if (warp_select) {
@@ -478,6 +484,70 @@ int backward_tc(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat
     return MOC_OK;
 }
 
+// ---- decode plan (bf16, tokens <= 16) ------------------------------------------------------------------
+struct DecodeLayout {
+    int ldf, slices, parts, gemv_grid;
+    size_t off_g, off_zc, off_mask, off_list, off_count, off_acc, off_cnt, total;
+};
+
+DecodeLayout decode_layout(const moc_ffn_desc &d) {
+    DecodeLayout L{};
+    L.ldf = (d.d_ff + 7) & ~7;
+    L.slices = (d.d_model + dec::kSliceCols - 1) / dec::kSliceCols;
+    // about two CTAs per SM in the down kernel; a CTA's share of the list is bounded by its shared arrays
+    const int sms = tc::sm_count();
+    L.parts = std::max(std::max(1, 2 * sms / L.slices), (d.d_ff + dec::kMaxPart - 1) / dec::kMaxPart);
+    // gate GEMV: two CTAs per SM, at most 64 channels each
+    L.gemv_grid = std::max(std::min(2 * sms, (d.d_ff + 7) / 8), (d.d_ff + 63) / 64);
+    Carver c;
+    L.off_g = c.take((size_t)d.tokens * L.ldf * sizeof(float));
+    L.off_zc = c.take((size_t)d.d_ff * 16 * sizeof(float));
+    L.off_mask = c.take((size_t)d.d_ff * sizeof(uint32_t));
+    L.off_list = c.take((size_t)d.d_ff * sizeof(uint16_t));
+    L.off_count = c.take(sizeof(int));
+    L.off_acc = c.take((size_t)d.tokens * d.d_model * sizeof(float));
+    L.off_cnt = c.take((size_t)L.slices * sizeof(int));
+    L.total = c.off;
+    return L;
+}
+
+bool use_decode_plan(const moc_ffn_desc &d) {
+    return d.dtype == MOC_BF16 && d.tokens >= 1 && d.tokens <= 16 && d.d_model <= 256 * dec::kSliceCols;
+}
+
+int decode_bf16(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat16 *wg, const __nv_bfloat16 *wu,
+                const __nv_bfloat16 *wd, __nv_bfloat16 *out, char *wsp, cudaStream_t st) {
+    const DecodeLayout L = decode_layout(d);
+    const int T = (int)d.tokens, F = d.d_ff, K = d.k, dm = d.d_model;
+    int *status = device_status_ptr();
+    if (!status) return MOC_ERR_CUDA;
+    dec::Workspace ws;
+    ws.G = reinterpret_cast<float *>(wsp + L.off_g);
+    ws.Zc = reinterpret_cast<float *>(wsp + L.off_zc);
+    ws.chmask = reinterpret_cast<uint32_t *>(wsp + L.off_mask);
+    ws.list = reinterpret_cast<uint16_t *>(wsp + L.off_list);
+    ws.list_count = reinterpret_cast<int *>(wsp + L.off_count);
+    ws.out_acc = reinterpret_cast<float *>(wsp + L.off_acc);
+    ws.counters = reinterpret_cast<int *>(wsp + L.off_cnt);
+    ws.ldf = L.ldf;
+    int rc;
+    const size_t sel_smem = (size_t)F * sizeof(uint32_t);
+    if ((rc = set_smem(dec::select_mask_kernel, sel_smem)) != MOC_OK) return rc;
+    const size_t down_smem = 2 * dec::kBatchRows * 1024 + (size_t)dec::kMaxPart * (16 * sizeof(float) + 4);
+    if ((rc = set_smem(dec::down_rows_kernel, down_smem)) != MOC_OK) return rc;
+
+    MOC_LAUNCH(KID_DEC_GATE_GEMV, st,
+               (dec::gate_gemv_kernel<<<L.gemv_grid, 256, 0, st>>>(x, wg, T, dm, F, ws, L.slices)));
+    if ((rc = launch_ok()) != MOC_OK) return rc;
+    MOC_LAUNCH(KID_DEC_SELECT, st, (dec::select_mask_kernel<<<T, dec::kSelThreads, sel_smem, st>>>(ws, F, K)));
+    if ((rc = launch_ok()) != MOC_OK) return rc;
+    MOC_LAUNCH(KID_DEC_UP, st, (dec::up_rows_kernel<<<2 * tc::sm_count(), 256, 0, st>>>(x, wu, T, dm, F, ws)));
+    if ((rc = launch_ok()) != MOC_OK) return rc;
+    MOC_LAUNCH(KID_DEC_DOWN, st,
+               (dec::down_rows_kernel<<<dim3(L.slices, L.parts), 256, down_smem, st>>>(wd, T, dm, F, ws, out, status)));
+    return launch_ok();
+}
+
 }  // namespace
 }  // namespace moc
 
@@ -494,7 +564,7 @@ size_t moc_ffn_workspace_bytes(const moc_ffn_desc *desc, int op) {
             return use_tc_plan(*desc) ? tc::tc_forward_layout(*desc).total : plan_forward(*desc).total;
         case MOC_OP_DECODE:
             if (desc->tokens > 16) return 0;
-            return plan_forward(*desc).total;
+            return use_decode_plan(*desc) ? decode_layout(*desc).total : plan_forward(*desc).total;
         case MOC_OP_BACKWARD:
             return use_tc_plan(*desc) ? tc::tc_backward_layout(*desc).total : plan_backward(*desc).total;
         default:
@@ -588,8 +658,16 @@ int moc_ffn_decode(const moc_ffn_desc *desc, const void *x, const void *w_gate, 
     int rc = check_desc(desc);
     if (rc != MOC_OK) return rc;
     if (desc->tokens > 16) return MOC_ERR_UNSUPPORTED;
-    return moc_ffn_forward(desc, x, w_gate, w_up, w_down, out, nullptr, nullptr, nullptr, workspace,
-                           workspace_bytes, cuda_stream);
+    if (!use_decode_plan(*desc))  // fp32 storage: the gathered forward with nothing saved
+        return moc_ffn_forward(desc, x, w_gate, w_up, w_down, out, nullptr, nullptr, nullptr, workspace,
+                               workspace_bytes, cuda_stream);
+    if (!good_ptr(x) || !good_ptr(w_gate) || !good_ptr(w_up) || !good_ptr(w_down) || !good_ptr(out))
+        return MOC_ERR_INVALID_ARG;
+    const size_t need = decode_layout(*desc).total;
+    if (!good_ptr(workspace) || workspace_bytes < need) return MOC_ERR_WORKSPACE;
+    using T = __nv_bfloat16;
+    return decode_bf16(*desc, (const T *)x, (const T *)w_gate, (const T *)w_up, (const T *)w_down, (T *)out,
+                       static_cast<char *>(workspace), static_cast<cudaStream_t>(cuda_stream));
 }
 
 int moc_topk_select(int64_t rows, int32_t n, int32_t n_ld, int32_t k, const float *gate, int16_t *idx_out,

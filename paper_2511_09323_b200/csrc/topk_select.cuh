@@ -9,9 +9,9 @@
 // and can be compared bit for bit.
 //
 // Cost control:
-//  * histogram updates are aggregated per warp (lanes with the same digit elect one lane that adds
-//    their count), because gate values of one row share sign and exponent and would otherwise
-//    serialise on a handful of bins;
+//  * the first pass counts into one private histogram per warp (padded so that equal bins of different
+//    warps sit in different banks), because gate values of one row share sign and exponent and would
+//    otherwise serialise on a handful of counters;
 //  * after the first pass only the keys of the chosen bin are still candidates; when they fit, they
 //    are copied to a short list and passes 2..4 read the list instead of the whole row;
 //  * the ordered emission needs only a fixed number of block barriers: per-(chunk, warp) counts go to
@@ -27,27 +27,25 @@ constexpr int kSelectMaxN = 32768;                      // int16 channel indices
 constexpr int kSelectCandCap = 2048;                    // candidate list entries
 constexpr int kSelectTable = kSelectMaxN / 256 * 8;     // (chunk, warp) slots: 128 chunks x 8 warps
 
-struct SelectSmem {
+constexpr int kPrivStride = 257;  // per-warp histogram stride: equal bins of different warps hit different banks
+
+template <int NW>
+struct SelectSmemT {
     uint32_t hist[256];
     uint32_t warp_tot[32];
     uint32_t cand[kSelectCandCap];
     uint32_t table[kSelectTable];
+    uint32_t priv[NW * kPrivStride];  // one private first-pass histogram per warp
     uint32_t chosen_bin;
     uint32_t remaining;
     uint32_t cand_count;
 };
-
-// adds 1 to hist[bin] for every lane with active == true, one shared-memory atomic per distinct bin
-__device__ __forceinline__ void warp_hist_add(uint32_t *hist, uint32_t bin, bool active) {
-    const uint32_t key = active ? bin : 0xffffffffu;
-    const uint32_t peers = __match_any_sync(0xffffffffu, key);
-    if (active && (__ffs(peers) - 1) == (int)(threadIdx.x & 31)) atomicAdd(&hist[bin], (uint32_t)__popc(peers));
-}
+using SelectSmem = SelectSmemT<kSelectThreads / 32>;
 
 // From hist[256] and sm.remaining: the bin holding the remaining-th largest, and how many lie above it.
 // Result in sm.chosen_bin = bin | (count_above << 8).  All threads call; contains block barriers.
 template <int THREADS>
-__device__ __forceinline__ void block_pick_bin(SelectSmem &sm) {
+__device__ __forceinline__ void block_pick_bin(SelectSmemT<THREADS / 32> &sm) {
     const int tid = threadIdx.x;
     uint32_t h = 0, s = 0;
     if (tid < 256) {
@@ -72,23 +70,28 @@ __device__ __forceinline__ void block_pick_bin(SelectSmem &sm) {
 // Finds tau (key of the K-th largest) and need (how many keys == tau are to be kept).
 // keys: shared memory, n entries.  All threads of the CTA must call it.  THREADS >= 256.
 template <int THREADS>
-__device__ __forceinline__ void block_radix_threshold(const uint32_t *keys, int n, int k, SelectSmem &sm,
-                                                      uint32_t &tau, int &need) {
+__device__ __forceinline__ void block_radix_threshold(const uint32_t *keys, int n, int k,
+                                                      SelectSmemT<THREADS / 32> &sm, uint32_t &tau, int &need) {
     static_assert(THREADS >= 256 && THREADS % 32 == 0, "selector needs at least 256 threads");
-    const int tid = threadIdx.x;
-    // ---- pass 1 over the whole row: top 8 bits
-    if (tid < 256) sm.hist[tid] = 0;
+    constexpr int NW = THREADS / 32;
+    const int tid = threadIdx.x, warp = tid >> 5;
+    // ---- pass 1 over the whole row: top 8 bits (sign and exponent).  The gate values of a row share
+    // these bits almost entirely, so a single histogram would serialise on a few counters: every warp
+    // counts into its own copy and the copies are summed afterwards.
+    for (int i = tid; i < NW * kPrivStride; i += THREADS) sm.priv[i] = 0;
     if (tid == 0) {
         sm.remaining = (uint32_t)k;
         sm.cand_count = 0;
     }
     __syncthreads();
-    for (int base = 0; base < n; base += THREADS) {
-        const int j = base + tid;
-        const bool in = j < n;
-        warp_hist_add(sm.hist, in ? (keys[j] >> 24) : 0u, in);
-    }
+    for (int j = tid; j < n; j += THREADS) atomicAdd(&sm.priv[warp * kPrivStride + (keys[j] >> 24)], 1u);
     __syncthreads();
+    if (tid < 256) {
+        uint32_t h = 0;
+#pragma unroll 8
+        for (int w = 0; w < NW; ++w) h += sm.priv[w * kPrivStride + tid];
+        sm.hist[tid] = h;
+    }
     block_pick_bin<THREADS>(sm);
     uint32_t cb = sm.chosen_bin;
     uint32_t prefix = (cb & 255u) << 24, mask = 255u << 24;
@@ -118,10 +121,9 @@ __device__ __forceinline__ void block_radix_threshold(const uint32_t *keys, int 
         const int shift = 24 - 8 * pass;
         if (tid < 256) sm.hist[tid] = 0;
         __syncthreads();
-        for (int base = 0; base < m; base += THREADS) {
-            const int j = base + tid;
-            const uint32_t key = j < m ? src[j] : 0u;
-            warp_hist_add(sm.hist, (key >> shift) & 255u, j < m && (key & mask) == prefix);
+        for (int j = tid; j < m; j += THREADS) {
+            const uint32_t key = src[j];
+            if ((key & mask) == prefix) atomicAdd(&sm.hist[(key >> shift) & 255u], 1u);
         }
         __syncthreads();
         block_pick_bin<THREADS>(sm);
@@ -159,7 +161,8 @@ __device__ __forceinline__ float key_to_float(uint32_t key) {
 // All threads call; `guess` must hold the same values in every thread (it is updated uniformly).
 template <int THREADS>
 __device__ __forceinline__ void block_select_row(const float *__restrict__ g, int n, int k, uint32_t *keys,
-                                                 SelectSmem &sm, SelectGuess &guess, uint32_t &tau, int &need) {
+                                                 SelectSmemT<THREADS / 32> &sm, SelectGuess &guess, uint32_t &tau,
+                                                 int &need) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     uint32_t lo = 1u, hi = 0u;  // empty bracket
     if (guess.valid) {
@@ -256,19 +259,20 @@ __device__ __forceinline__ void block_select_row(const float *__restrict__ g, in
 // among the kept channels in ascending channel order (0 <= pos < k).
 template <int THREADS, typename Emit>
 __device__ __forceinline__ void block_ordered_emit(const uint32_t *keys, int n, uint32_t tau, int need,
-                                                   SelectSmem &sm, Emit emit) {
-    static_assert(THREADS == 256, "table layout assumes 8 warps");
+                                                   SelectSmemT<THREADS / 32> &sm, Emit emit) {
+    static_assert(THREADS == 256 || THREADS == 1024, "table holds (n / THREADS) x (THREADS / 32) <= 1024 slots");
+    constexpr int NW = THREADS / 32;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t lt_mask = (1u << lane) - 1u;
     const int chunks = (n + THREADS - 1) / THREADS;
-    const int slots = chunks * 8;
+    const int slots = chunks * NW;
     // sweep 1: per (chunk, warp) counts of key > tau (low half) and key == tau (high half)
     for (int c = 0; c < chunks; ++c) {
         const int j = c * THREADS + tid;
         const uint32_t key = j < n ? keys[j] : 0u;
         const uint32_t bg = __ballot_sync(0xffffffffu, j < n && key > tau);
         const uint32_t be = __ballot_sync(0xffffffffu, j < n && key == tau);
-        if (lane == 0) sm.table[c * 8 + warp] = (uint32_t)__popc(bg) | ((uint32_t)__popc(be) << 16);
+        if (lane == 0) sm.table[c * NW + warp] = (uint32_t)__popc(bg) | ((uint32_t)__popc(be) << 16);
     }
     __syncthreads();
     // exclusive scan of the table in slot order; thread t owns slots [per*t, per*t + per)
@@ -304,7 +308,7 @@ __device__ __forceinline__ void block_ordered_emit(const uint32_t *keys, int n, 
         const bool gt = j < n && key > tau;
         const bool eq = j < n && key == tau;
         const uint32_t bg = __ballot_sync(0xffffffffu, gt), be = __ballot_sync(0xffffffffu, eq);
-        const uint32_t before = sm.table[c * 8 + warp];
+        const uint32_t before = sm.table[c * NW + warp];
         const uint32_t gt_before = (before & 0xffffu) + (uint32_t)__popc(bg & lt_mask);
         const uint32_t eq_before = (before >> 16) + (uint32_t)__popc(be & lt_mask);
         if (gt || (eq && eq_before < (uint32_t)need)) emit((int)(gt_before + min(eq_before, (uint32_t)need)), j);
