@@ -6,6 +6,8 @@
 #include <atomic>
 #include <cstdint>
 #include <cstring>
+#include <mutex>
+#include <unordered_map>
 #include <vector>
 
 #include "decode_kernels.cuh"
@@ -187,8 +189,16 @@ int set_smem(K kernel, size_t bytes) {
     constexpr size_t kStaticReserve = 48 * 1024;
     if (bytes + kStaticReserve > (size_t)kMaxDynSmem) return MOC_ERR_UNSUPPORTED;
     if (bytes + kStaticReserve > 48 * 1024) {
-        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess)
-            return MOC_ERR_CUDA;
+        // the attribute only ever grows; remember what was set so that steady-state calls make no driver call
+        static std::mutex mu;
+        static std::unordered_map<const void *, size_t> configured;
+        std::lock_guard<std::mutex> lock(mu);
+        size_t &have = configured[reinterpret_cast<const void *>(kernel)];
+        if (have < bytes) {
+            if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess)
+                return MOC_ERR_CUDA;
+            have = bytes;
+        }
     }
     return MOC_OK;
 }
@@ -487,7 +497,7 @@ int backward_tc(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat
 // ---- decode plan (bf16, tokens <= 16) ------------------------------------------------------------------
 struct DecodeLayout {
     int ldf, slices, parts, gemv_grid;
-    size_t off_g, off_zc, off_mask, off_list, off_count, off_acc, off_cnt, total;
+    size_t off_g, off_zb, off_mask, off_list, off_count, off_acc, off_cnt, total;
 };
 
 DecodeLayout decode_layout(const moc_ffn_desc &d) {
@@ -497,11 +507,11 @@ DecodeLayout decode_layout(const moc_ffn_desc &d) {
     // about two CTAs per SM in the down kernel; a CTA's share of the list is bounded by its shared arrays
     const int sms = tc::sm_count();
     L.parts = std::max(std::max(1, 2 * sms / L.slices), (d.d_ff + dec::kMaxPart - 1) / dec::kMaxPart);
-    // gate GEMV: two CTAs per SM, at most 64 channels each
-    L.gemv_grid = std::max(std::min(2 * sms, (d.d_ff + 7) / 8), (d.d_ff + 63) / 64);
+    // GEMV kernels: two CTAs per SM, never more than 64 rows per CTA
+    L.gemv_grid = std::max(std::max(1, std::min(2 * sms, (d.d_ff + 7) / 8)), (d.d_ff + 63) / 64);
     Carver c;
     L.off_g = c.take((size_t)d.tokens * L.ldf * sizeof(float));
-    L.off_zc = c.take((size_t)d.d_ff * 16 * sizeof(float));
+    L.off_zb = c.take((size_t)((d.d_ff + 15) / 16) * 256 * sizeof(__nv_bfloat16));
     L.off_mask = c.take((size_t)d.d_ff * sizeof(uint32_t));
     L.off_list = c.take((size_t)d.d_ff * sizeof(uint16_t));
     L.off_count = c.take(sizeof(int));
@@ -523,7 +533,7 @@ int decode_bf16(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat
     if (!status) return MOC_ERR_CUDA;
     dec::Workspace ws;
     ws.G = reinterpret_cast<float *>(wsp + L.off_g);
-    ws.Zc = reinterpret_cast<float *>(wsp + L.off_zc);
+    ws.Zb = reinterpret_cast<__nv_bfloat16 *>(wsp + L.off_zb);
     ws.chmask = reinterpret_cast<uint32_t *>(wsp + L.off_mask);
     ws.list = reinterpret_cast<uint16_t *>(wsp + L.off_list);
     ws.list_count = reinterpret_cast<int *>(wsp + L.off_count);
@@ -531,20 +541,25 @@ int decode_bf16(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat
     ws.counters = reinterpret_cast<int *>(wsp + L.off_cnt);
     ws.ldf = L.ldf;
     int rc;
-    const size_t sel_smem = (size_t)F * sizeof(uint32_t);
+    const size_t sel_smem = ((size_t)F + 2 * dec::kSelListCap) * sizeof(uint32_t);
     if ((rc = set_smem(dec::select_mask_kernel, sel_smem)) != MOC_OK) return rc;
-    const size_t down_smem = 2 * dec::kBatchRows * 1024 + (size_t)dec::kMaxPart * (16 * sizeof(float) + 4);
-    if ((rc = set_smem(dec::down_rows_kernel, down_smem)) != MOC_OK) return rc;
+    if ((rc = set_smem(dec::down_rows_kernel, dec::kDownSmem)) != MOC_OK) return rc;
+    if ((rc = set_smem(dec::gemv_rows_kernel<false>, dec::kGemvSmem)) != MOC_OK) return rc;
+    if ((rc = set_smem(dec::gemv_rows_kernel<true>, dec::kGemvSmem)) != MOC_OK) return rc;
 
     MOC_LAUNCH(KID_DEC_GATE_GEMV, st,
-               (dec::gate_gemv_kernel<<<L.gemv_grid, 256, 0, st>>>(x, wg, T, dm, F, ws, L.slices)));
+               (dec::gemv_rows_kernel<false><<<L.gemv_grid, dec::kGemvThreads, dec::kGemvSmem, st>>>(
+                   x, wg, T, dm, F, ws, L.slices, status)));
     if ((rc = launch_ok()) != MOC_OK) return rc;
     MOC_LAUNCH(KID_DEC_SELECT, st, (dec::select_mask_kernel<<<T, dec::kSelThreads, sel_smem, st>>>(ws, F, K)));
     if ((rc = launch_ok()) != MOC_OK) return rc;
-    MOC_LAUNCH(KID_DEC_UP, st, (dec::up_rows_kernel<<<2 * tc::sm_count(), 256, 0, st>>>(x, wu, T, dm, F, ws)));
+    MOC_LAUNCH(KID_DEC_UP, st,
+               (dec::gemv_rows_kernel<true><<<L.gemv_grid, dec::kGemvThreads, dec::kGemvSmem, st>>>(
+                   x, wu, T, dm, F, ws, L.slices, status)));
     if ((rc = launch_ok()) != MOC_OK) return rc;
     MOC_LAUNCH(KID_DEC_DOWN, st,
-               (dec::down_rows_kernel<<<dim3(L.slices, L.parts), 256, down_smem, st>>>(wd, T, dm, F, ws, out, status)));
+               (dec::down_rows_kernel<<<dim3(L.slices, L.parts), dec::kGemvThreads, dec::kDownSmem, st>>>(
+                   wd, T, dm, F, ws, out, status)));
     return launch_ok();
 }
 

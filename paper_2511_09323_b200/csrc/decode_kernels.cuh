@@ -3,20 +3,22 @@
 // Decode is bound by reading weights from HBM once: the whole gate matrix (F*d elements) plus the
 // selected rows of W_up and W_down.  With several tokens, a row selected by more than one token is
 // read once (the union of the tokens' channel sets), which is what keeps a batch of 16 cheaper than
-// a dense FFN.  Four kernels, all streaming:
-//   1. gate GEMV   : the channels are dealt out evenly to two CTAs per SM; a CTA's 8 warps split the
-//                    contraction into contiguous parts; the tokens are the M dimension of m16n8k16
-//                    tensor-core MMAs so that 16 tokens cost no more issue slots than one (one FMA per
-//                    loaded weight and token would be ALU-bound at 16 tokens).
-//   2. select      : one 1024-thread CTA per token, exact Top-K (same selector as training); sets the
-//                    token's bit in a per-channel mask and appends a channel to the list of used
-//                    channels the first time any token selects it.
-//   3. up          : one warp per used channel, u = x . Wu[j,:] for the tokens in its mask,
-//                    z = SiLU(g) u, stored next to the channel's list position.
-//   4. down        : CTA = (512-column slice, part of the list); rows arrive through a double-buffered
-//                    shared-memory ring filled by bulk async copies; per-slice partial sums are added to
-//                    an fp32 accumulator with atomics and the last CTA of a slice writes the bf16 output
-//                    (summation order across CTAs is not fixed, so the last bit of `out` may vary).
+// a dense FFN.  Four kernels, all streaming through shared-memory rings filled by bulk async copies
+// (the bytes in flight live in shared memory, not in registers):
+//   1. gate GEMV   : rows of W_gate dealt out evenly to two CTAs per SM; a producer warp copies
+//                    8-row x 1 KiB stages, 8 consumer warps split each stage along the contraction.
+//                    The tokens are the M dimension of m16n8k16 tensor-core MMAs, so 16 tokens cost no
+//                    more issue slots than one (one FMA per loaded weight and token would be ALU-bound).
+//   2. select      : one 1024-thread CTA per token, exact Top-K by a radix select whose digits are taken
+//                    relative to the range the candidates lie in (see the kernel).  Decode needs the set,
+//                    not the order: the token's bit is set in a per-channel mask.
+//   3. up          : the same GEMV over the listed rows of W_up; z = SiLU(g) u for the tokens in each
+//                    channel's mask (zero for the others), stored as bf16 in MMA-ready blocks.
+//   4. down        : CTA = (512-column slice, part of the list).  Stages of 16 rows x 1 KiB; the rows are
+//                    the contraction index, so the B fragments are read transposed with ldmatrix.
+//                    Per-slice partial sums are added to an fp32 accumulator with atomics and the last
+//                    CTA of a slice writes the bf16 output (the summation order across CTAs is not
+//                    fixed, so the last bit of `out` may vary from run to run).
 #pragma once
 
 #include "moc_common.cuh"
@@ -26,303 +28,600 @@
 namespace moc {
 namespace dec {
 
-constexpr int kGemvMaxTiles = 8;   // 8-channel MMA tiles per CTA (<= 64 channels)
 constexpr int kSelThreads = 1024;
-constexpr int kSliceCols = 512;    // down projection: columns per CTA (1 KiB of a bf16 row)
-constexpr int kBatchRows = 32;     // rows per ring buffer
-constexpr int kMaxPart = 512;      // list entries per down CTA (bound of its shared arrays)
+constexpr int kSelListCap = 4096;   // candidate list entries (two lists)
+constexpr int kSliceCols = 512;     // down projection: columns per CTA (1 KiB of a bf16 row)
+constexpr int kMaxPart = 512;       // list entries per down CTA (bound of its shared arrays)
+
+// GEMV ring: a stage is 8 rows x 512 contraction elements; rows are padded to 1088 bytes so that the
+// 16-byte fragment loads of a quarter warp fall into distinct bank groups
+constexpr int kGemvChunk = 512, kGemvPitch = 1088, kGemvStageBytes = 8 * kGemvPitch, kGemvStages = 11;
+constexpr int kGemvThreads = 288;   // 8 consumer warps + 1 producer warp
+constexpr int kGemvMaxTiles = 8;    // 8-row tiles per CTA: the host sizes the grid so that a CTA owns <= 64 rows
+constexpr int kGemvMaxRows = kGemvMaxTiles * 8;
+constexpr size_t kGemvSmem = (size_t)kGemvStages * kGemvStageBytes + 128;
+// down ring: a stage is 16 rows x 1 KiB, pitch 1040 so that ldmatrix rows fall into distinct bank groups
+constexpr int kDownPitch = 1040, kDownStageBytes = 16 * kDownPitch, kDownStages = 4;
+constexpr size_t kDownSmem = (size_t)kDownStages * kDownStageBytes + (size_t)kMaxPart * (32 + 2) + 128;
 
 struct Workspace {
-    float *G;           // [T, ldf] gate projection
-    float *Zc;          // [list position][16] z = SiLU(g) u per token
-    uint32_t *chmask;   // [F] bit t set: token t selected the channel
-    uint16_t *list;     // [F] used channels in order of first selection
-    int *list_count;    // number of used channels
-    float *out_acc;     // [T, d]
-    int *counters;      // [slices] arrival counters of the down kernel
+    float *G;             // [T, ldf] gate projection
+    __nv_bfloat16 *Zb;    // [list position / 16][16 tokens][16 positions] z = SiLU(g) u (0 where not selected)
+    uint32_t *chmask;     // [F] bit t set: token t selected the channel
+    uint16_t *list;       // [F] used channels in order of first selection
+    int *list_count;      // number of used channels
+    float *out_acc;       // [T, d]
+    int *counters;        // [slices] arrival counters of the down kernel
     int ldf;
 };
 
-__device__ __forceinline__ uint4 ld_stream16(const void *p) {
-    uint4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-                 : "l"(p));
-    return v;
-}
 __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                                uint32_t b0, uint32_t b1) {
-    asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
         "{%0, %1, %2, %3};"
         : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
+__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+__device__ __forceinline__ void consumer_bar_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 
-// ---------------------------------------------------------------------------------------------- 1. gate GEMV
-// G[t, j] = sum_i x[t,i] Wg[j,i]   (Eq. (Moc-1), per token as in Section 5).
-// CTA b owns channels [b F / grid, (b+1) F / grid).  Each lane loads 16 contiguous bytes (8 contraction
-// elements) of a weight row per step; the same permutation of the contraction index is applied to the
-// x fragment, so no data movement is needed to form the MMA operands.
-__global__ void __launch_bounds__(256, 2) gate_gemv_kernel(const __nv_bfloat16 *__restrict__ x,
-                                                           const __nv_bfloat16 *__restrict__ wg, int T, int d, int F,
-                                                           Workspace ws, int slices) {
-    __shared__ float red[8][16][kGemvMaxTiles * 8 + 1];
+// ---------------------------------------------------------------------------------------------- 1 + 3. GEMV
+// R[t, r] = sum_i x[t,i] W[row(r), i] for the CTA's share of the rows, all tokens at once.
+//   GATHER == false: rows are the channels 0..F-1 of W_gate; result -> G          (Eq. (Moc-1))
+//   GATHER == true : rows are the listed channels of W_up;   result -> z = SiLU(g) u on the masks
+// CTA b owns row slots [b n / grid, (b+1) n / grid).  Each lane reads 16 contiguous bytes (8 contraction
+// elements) of a weight row per fragment; the same permutation of the contraction index is applied to the
+// x fragment, so the MMA operands need no data movement.
+template <bool GATHER>
+__global__ void __launch_bounds__(kGemvThreads, 2) gemv_rows_kernel(const __nv_bfloat16 *__restrict__ x,
+                                                                    const __nv_bfloat16 *__restrict__ w, int T, int d,
+                                                                    int F, Workspace ws, int slices,
+                                                                    int *__restrict__ status) {
+    extern __shared__ __align__(128) uint8_t gsm[];
+    __shared__ uint64_t bars[2 * kGemvStages];
+    __shared__ int s_abort;
+    __shared__ int s_scan[(kSelectMaxN / kGemvThreads + 2) * 9 + 1];  // (chunk, warp) counts of used channels
+    __shared__ uint16_t s_rows[kGemvMaxRows];                          // this CTA's rows when gathering
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int g = lane >> 2, q = lane & 3;
-    const int r0 = (int)(((int64_t)blockIdx.x * F) / gridDim.x);
-    const int r1 = (int)(((int64_t)(blockIdx.x + 1) * F) / gridDim.x);
-    const int nt = (r1 - r0 + 7) >> 3;
-    // housekeeping for the later kernels: clear masks, accumulators, counters
-    for (int j = r0 + tid; j < r1; j += 256) ws.chmask[j] = 0u;
-    for (int64_t i = (int64_t)blockIdx.x * 256 + tid; i < (int64_t)T * d; i += (int64_t)gridDim.x * 256)
-        ws.out_acc[i] = 0.f;
-    if (blockIdx.x == 0) {
-        if (tid < slices) ws.counters[tid] = 0;
-        if (tid == 0) *ws.list_count = 0;
-    }
-
-    float acc[kGemvMaxTiles][4];
+    int n = F;
+    uint32_t used_bits[4] = {0u, 0u, 0u, 0u};  // bit c: this thread's channel of chunk c is used
+    if (GATHER) {
+        // Every CTA derives the list of used channels (ascending) from the masks: per (chunk, warp) counts,
+        // one scan, then each used channel knows its list position.  A CTA keeps the positions of its own
+        // share; CTA 0 also writes the whole list for the down kernel.
+        const int chunks = (F + kGemvThreads - 1) / kGemvThreads;  // <= 114
+        // masks are fetched in groups of 16 independent loads; the "used" flags stay in registers
+        for (int c0 = 0; c0 < chunks; c0 += 16) {
+            uint32_t m[16];
 #pragma unroll
-    for (int nb = 0; nb < kGemvMaxTiles; ++nb)
+            for (int u = 0; u < 16; ++u) {
+                const int j = (c0 + u) * kGemvThreads + tid;
+                m[u] = (c0 + u < chunks && j < F) ? ws.chmask[j] : 0u;
+            }
 #pragma unroll
-        for (int e = 0; e < 4; ++e) acc[nb][e] = 0.f;
-    const int ksteps = (d + 31) >> 5;
-    const int per_warp = (ksteps + 7) >> 3;
-    const int s_begin = warp * per_warp, s_end = min(ksteps, s_begin + per_warp);
-    const __nv_bfloat16 *xa_row = x + (int64_t)g * d, *xb_row = x + (int64_t)(g + 8) * d;
-    const bool has_a = g < T, has_b = g + 8 < T;
-    const __nv_bfloat16 *wrow[kGemvMaxTiles];
-    bool wok[kGemvMaxTiles];
-#pragma unroll
-    for (int nb = 0; nb < kGemvMaxTiles; ++nb) {
-        const int ch = r0 + nb * 8 + g;
-        wok[nb] = nb < nt && ch < r1;
-        wrow[nb] = wg + (int64_t)(wok[nb] ? ch : r0) * d;
-    }
-#pragma unroll 2
-    for (int s = s_begin; s < s_end; ++s) {
-        const int koff = (s << 5) + (q << 3);
-        const bool kv = koff < d;
-        uint4 wv[kGemvMaxTiles];
-#pragma unroll
-        for (int nb = 0; nb < kGemvMaxTiles; ++nb) {
-            wv[nb] = make_uint4(0, 0, 0, 0);
-            if (kv && wok[nb]) wv[nb] = ld_stream16(wrow[nb] + koff);
+            for (int u = 0; u < 16; ++u) {
+                if (c0 + u < chunks) {
+                    const uint32_t b = __ballot_sync(0xffffffffu, m[u] != 0u);
+                    if (lane == 0) s_scan[(c0 + u) * 9 + warp] = __popc(b);
+                    if (m[u] != 0u) used_bits[(c0 + u) >> 5] |= 1u << ((c0 + u) & 31);
+                }
+            }
         }
-        uint4 xa = make_uint4(0, 0, 0, 0), xb = make_uint4(0, 0, 0, 0);
-        if (kv && has_a) xa = *reinterpret_cast<const uint4 *>(xa_row + koff);
-        if (kv && has_b) xb = *reinterpret_cast<const uint4 *>(xb_row + koff);
+        __syncthreads();
+        // exclusive scan in (chunk, warp) order: thread c scans chunk c's 9 counts, the chunk totals are
+        // scanned across the block (chunks <= 114 < threads)
+        __shared__ int s_wsum[9];
+        int ctot = 0;
+        if (tid < chunks)
+            for (int i = 0; i < 9; ++i) ctot += s_scan[tid * 9 + i];
+        int inc = ctot;
 #pragma unroll
-        for (int nb = 0; nb < kGemvMaxTiles; ++nb) {
-            if (nb < nt) {  // uniform
-                mma_bf16_16816(acc[nb], xa.x, xb.x, xa.y, xb.y, wv[nb].x, wv[nb].y);
-                mma_bf16_16816(acc[nb], xa.z, xb.z, xa.w, xb.w, wv[nb].z, wv[nb].w);
+        for (int o = 1; o < 32; o <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, inc, o);
+            if (lane >= o) inc += v;
+        }
+        if (lane == 31) s_wsum[warp] = inc;
+        __syncthreads();
+        int before = inc - ctot;
+        for (int wi = 0; wi < warp; ++wi) before += s_wsum[wi];
+        if (tid < chunks) {
+            int run = before;
+            for (int i = 0; i < 9; ++i) {
+                const int v = s_scan[tid * 9 + i];
+                s_scan[tid * 9 + i] = run;
+                run += v;
+            }
+            if (tid == chunks - 1) s_scan[chunks * 9] = run;
+        }
+        __syncthreads();
+        n = s_scan[chunks * 9];
+    }
+    const int r0 = (int)(((int64_t)blockIdx.x * n) / gridDim.x);
+    const int r1 = (int)(((int64_t)(blockIdx.x + 1) * n) / gridDim.x);
+    const int tiles = (r1 - r0 + 7) >> 3;
+    if (GATHER) {
+        const int chunks = (F + kGemvThreads - 1) / kGemvThreads;
+        for (int c = 0; c < chunks; ++c) {
+            const int j = c * kGemvThreads + tid;
+            const bool used = (used_bits[c >> 5] >> (c & 31)) & 1u;
+            const uint32_t b = __ballot_sync(0xffffffffu, used);
+            if (used) {
+                const int pos = s_scan[c * 9 + warp] + __popc(b & ((1u << lane) - 1u));
+                if (pos >= r0 && pos < r1 && pos - r0 < kGemvMaxRows) s_rows[pos - r0] = (uint16_t)j;
+                if (blockIdx.x == 0) ws.list[pos] = (uint16_t)j;
+            }
+        }
+        if (blockIdx.x == 0 && tid == 0) *ws.list_count = n;
+    }
+    const int nkc = (d + kGemvChunk - 1) / kGemvChunk;
+    const uint32_t ring = tc::smem_u32(gsm);
+    auto full_bar = [&](int s) { return tc::smem_u32(&bars[s]); };
+    auto empty_bar = [&](int s) { return tc::smem_u32(&bars[kGemvStages + s]); };
+
+    if (!GATHER) {
+        // housekeeping for the later kernels: clear masks, accumulators, counters
+        for (int j = r0 + tid; j < r1; j += kGemvThreads) ws.chmask[j] = 0u;
+        for (int64_t i = (int64_t)blockIdx.x * kGemvThreads + tid; i < (int64_t)T * d;
+             i += (int64_t)gridDim.x * kGemvThreads)
+            ws.out_acc[i] = 0.f;
+        if (blockIdx.x == 0 && tid < slices) ws.counters[tid] = 0;
+    }
+    // When the last chunk of a row is short, the bytes it leaves untouched are multiplied by zero x entries and
+    // must therefore be finite: the ring then starts out as zeros.  (Rows of a partial tile that are never
+    // copied only feed outputs that are never written.)
+    if (d % kGemvChunk != 0)
+        for (int i = tid; i < (int)(kGemvStages * kGemvStageBytes / 16); i += kGemvThreads)
+            reinterpret_cast<uint4 *>(gsm)[i] = make_uint4(0, 0, 0, 0);
+    if (tid == 0) {
+        for (int s = 0; s < kGemvStages; ++s) {
+            tc::mbar_init(full_bar(s), 1);
+            tc::mbar_init(empty_bar(s), 8);
+        }
+        s_abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // zero fill before the async copies
+    __syncthreads();
+    if (tiles <= 0) return;
+
+    if (warp == 8) {
+        // ------------------------------------------------------------------ producer
+        int stage = 0;
+        uint32_t phase = 0;
+        bool ok = true;
+        for (int tile = 0; tile < tiles && ok; ++tile) {
+            const int slot = r0 + tile * 8 + lane;  // lanes 0..7 own one row each
+            const bool valid = lane < 8 && slot < r1;
+            const int row = valid ? (GATHER ? (int)s_rows[slot - r0] : slot) : 0;
+            const int nvalid = min(8, r1 - (r0 + tile * 8));
+            for (int kc = 0; kc < nkc; ++kc) {
+                if (!__all_sync(0xffffffffu, tc::mbar_wait(empty_bar(stage), phase ^ 1u, &s_abort, status))) {
+                    ok = false;
+                    break;
+                }
+                const int k0 = kc * kGemvChunk;
+                const uint32_t bytes = (uint32_t)min(kGemvChunk, d - k0) * 2;
+                if (lane == 0) tc::mbar_expect_tx(full_bar(stage), bytes * (uint32_t)nvalid);
+                __syncwarp();
+                if (valid)
+                    bulk_copy_g2s(ring + stage * kGemvStageBytes + lane * kGemvPitch, w + (int64_t)row * d + k0,
+                                  bytes, full_bar(stage));
+                if (++stage == kGemvStages) {
+                    stage = 0;
+                    phase ^= 1u;
+                }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ consumers (warps 0..7)
+        // The partial sums of all the CTA's tiles (at most kGemvMaxTiles, the host sizes the grid for that)
+        // stay in registers; the eight warps' sums are combined once, after the last stage, in the ring's
+        // memory (idle by then).
+        const int g = lane >> 2, q = lane & 3;
+        const __nv_bfloat16 *xa_row = x + (int64_t)g * d, *xb_row = x + (int64_t)(g + 8) * d;
+        const bool has_a = g < T, has_b = g + 8 < T;
+        int stage = 0;
+        uint32_t phase = 0;
+        bool ok = true;
+        float acc[kGemvMaxTiles][4];
+#pragma unroll
+        for (int ti = 0; ti < kGemvMaxTiles; ++ti) acc[ti][0] = acc[ti][1] = acc[ti][2] = acc[ti][3] = 0.f;
+#pragma unroll
+        for (int ti = 0; ti < kGemvMaxTiles; ++ti) {
+            if (ti < tiles && ok) {  // uniform
+                for (int kc = 0; kc < nkc; ++kc) {
+                    // this warp's 64 contraction elements of the chunk: two 16-byte fragments per lane
+                    const int k0 = kc * kGemvChunk + warp * 64 + q * 8;
+                    uint4 xa0 = make_uint4(0, 0, 0, 0), xa1 = xa0, xb0 = xa0, xb1 = xa0;
+                    if (has_a) {
+                        if (k0 < d) xa0 = *reinterpret_cast<const uint4 *>(xa_row + k0);
+                        if (k0 + 32 < d) xa1 = *reinterpret_cast<const uint4 *>(xa_row + k0 + 32);
+                    }
+                    if (has_b) {
+                        if (k0 < d) xb0 = *reinterpret_cast<const uint4 *>(xb_row + k0);
+                        if (k0 + 32 < d) xb1 = *reinterpret_cast<const uint4 *>(xb_row + k0 + 32);
+                    }
+                    if (!__all_sync(0xffffffffu, tc::mbar_wait(full_bar(stage), phase, &s_abort, status))) {
+                        ok = false;
+                        break;
+                    }
+                    const uint8_t *src = gsm + stage * kGemvStageBytes + g * kGemvPitch + warp * 128 + q * 16;
+                    const uint4 w0 = *reinterpret_cast<const uint4 *>(src);
+                    const uint4 w1 = *reinterpret_cast<const uint4 *>(src + 64);
+#ifdef MOC_EXP_NOMMA
+                    acc[ti][0] += __uint_as_float((w0.x ^ w1.y ^ xa0.x ^ xa1.y ^ xb0.x ^ xb1.x) & 0x3f800000u);
+#else
+                    mma_bf16_16816(acc[ti], xa0.x, xb0.x, xa0.y, xb0.y, w0.x, w0.y);
+                    mma_bf16_16816(acc[ti], xa0.z, xb0.z, xa0.w, xb0.w, w0.z, w0.w);
+                    mma_bf16_16816(acc[ti], xa1.x, xb1.x, xa1.y, xb1.y, w1.x, w1.y);
+                    mma_bf16_16816(acc[ti], xa1.z, xb1.z, xa1.w, xb1.w, w1.z, w1.w);
+#endif
+                    __syncwarp();
+                    if (lane == 0) tc::mbar_arrive(empty_bar(stage));
+                    if (++stage == kGemvStages) {
+                        stage = 0;
+                        phase ^= 1u;
+                    }
+                }
+            }
+        }
+        // every warp passes both barriers, also after a failed wait
+        consumer_bar_sync();
+        float *red = reinterpret_cast<float *>(gsm);  // [8 warps][16 tokens][kGemvMaxTiles * 8 + 1]
+        constexpr int RP = kGemvMaxTiles * 8 + 1;
+#pragma unroll
+        for (int ti = 0; ti < kGemvMaxTiles; ++ti) {
+            float *r = red + (warp * 16) * RP + ti * 8 + 2 * q;
+            r[g * RP] = acc[ti][0];
+            r[g * RP + 1] = acc[ti][1];
+            r[(g + 8) * RP] = acc[ti][2];
+            r[(g + 8) * RP + 1] = acc[ti][3];
+        }
+        consumer_bar_sync();
+        ok = ok && !s_abort;
+        const int width = r1 - r0;
+        for (int o = tid; ok && o < 16 * width; o += 256) {
+            const int t = o / width, c = o - t * width;
+            const int slot = r0 + c;
+            float sum = 0.f;
+#pragma unroll
+            for (int wi = 0; wi < 8; ++wi) sum += red[(wi * 16 + t) * RP + c];
+            if (!GATHER) {
+                if (t < T) ws.G[(int64_t)t * ws.ldf + slot] = sum;
+            } else {
+                const int j = s_rows[c];
+                float z = 0.f;
+                if (t < T && ((ws.chmask[j] >> t) & 1u)) z = silu_f(ws.G[(int64_t)t * ws.ldf + j]) * sum;
+                ws.Zb[((int64_t)(slot >> 4) * 16 + t) * 16 + (slot & 15)] = __float2bfloat16_rn(z);
             }
         }
     }
-#pragma unroll
-    for (int nb = 0; nb < kGemvMaxTiles; ++nb) {
-        red[warp][g][nb * 8 + 2 * q] = acc[nb][0];
-        red[warp][g][nb * 8 + 2 * q + 1] = acc[nb][1];
-        red[warp][g + 8][nb * 8 + 2 * q] = acc[nb][2];
-        red[warp][g + 8][nb * 8 + 2 * q + 1] = acc[nb][3];
-    }
-    __syncthreads();
-    const int width = r1 - r0;
-    for (int o = tid; o < T * width; o += 256) {
-        const int t = o / width, c = o - t * width;
-        float s = 0.f;
-#pragma unroll
-        for (int w = 0; w < 8; ++w) s += red[w][t][c];
-        ws.G[(int64_t)t * ws.ldf + r0 + c] = s;
+    __syncwarp();
+    if (s_abort) {
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000LL) __nanosleep(1000);
     }
 }
 
 // ---------------------------------------------------------------------------------------------- 2. select
-// One CTA per token: exact Top-K of G[t, 0..F).
-__global__ void __launch_bounds__(kSelThreads) select_mask_kernel(Workspace ws, int F, int K) {
-    extern __shared__ __align__(16) uint32_t select_keys[];
-    __shared__ SelectSmemT<kSelThreads / 32> sm;
-    const int t = blockIdx.x;
-    const float *g = ws.G + (int64_t)t * ws.ldf;
-    for (int j = threadIdx.x; j < F; j += kSelThreads) select_keys[j] = gate_key(g[j]);
-    __syncthreads();
-    uint32_t tau;
-    int need;
-    block_radix_threshold<kSelThreads>(select_keys, F, K, sm, tau, need);
-    const uint32_t bit = 1u << t;
-    block_ordered_emit<kSelThreads>(select_keys, F, tau, need, sm, [&](int, int j) {
-        if (atomicOr(&ws.chmask[j], bit) == 0u) ws.list[atomicAdd(ws.list_count, 1)] = (uint16_t)j;
-    });
-}
+// One CTA per token: exact Top-K set of G[t, 0..F).
+//
+// A single CTA has to find the K-th largest of ~10^4 keys with as few block-wide steps as possible.
+// Radix select with digits taken from the top of the key fails at that here: the keys of one row share
+// sign and exponent, so the first digits put almost everything into a few bins (serialised counters) and
+// narrow the candidates very slowly.  Instead the digits are taken relative to the range the candidates
+// are known to lie in: with [lo, hi] the current range, bin = (key - lo) >> shift with shift chosen so
+// that the range maps onto at most 2048 bins.  The first level uses the row's minimum and maximum key;
+// the bin that holds the K-th largest then holds a handful of keys, which are copied to a short list and
+// ranked directly.  Further levels (only for very uneven data) repeat the step on the list.
+// Decode needs the set, not the order: the token's bit is set in a per-channel mask with plain
+// reductions; only when ties at the threshold must be cut does the ordered emission run.
+struct SelectLevel {
+    uint32_t lo, hi;  // candidates lie in [lo, hi]
+    uint32_t m;       // the m-th largest of them is wanted
+    uint32_t count;   // number of candidates
+};
 
-// ---------------------------------------------------------------------------------------------- 3. up
-// One warp per used channel j: u_t = x_t . Wu[j,:] for every token t in the channel's mask,
-// z_t = SiLU(G[t,j]) u_t.   (Eq. (MoC-2) on the mask.)
-__global__ void __launch_bounds__(256) up_rows_kernel(const __nv_bfloat16 *__restrict__ x,
-                                                      const __nv_bfloat16 *__restrict__ wu, int T, int d, int F,
-                                                      Workspace ws) {
-    const int lane = threadIdx.x & 31;
-    const int gw = blockIdx.x * 8 + (threadIdx.x >> 5), nw = gridDim.x * 8;
-    const int nvec = d >> 3;  // 16-byte vectors per row
-    const int count = min(*ws.list_count, F);
-    for (int p = gw; p < count; p += nw) {
-        const int j = ws.list[p];
-        const uint32_t m = ws.chmask[j];
-        const __nv_bfloat16 *row = wu + (int64_t)j * d;
-        float part[16];
-#pragma unroll
-        for (int t = 0; t < 16; ++t) part[t] = 0.f;
-        // the row is consumed in segments of 8 vectors per lane (2048 elements), weights in registers
-        for (int v0 = 0; v0 < nvec; v0 += 256) {
-            uint4 w[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const int v = v0 + i * 32 + lane;
-                w[i] = make_uint4(0, 0, 0, 0);
-                if (v < nvec) w[i] = ld_stream16(row + 8 * v);
-            }
-#pragma unroll
-            for (int t = 0; t < 16; ++t) {
-                if (!((m >> t) & 1u)) continue;  // uniform across the warp
-                const __nv_bfloat16 *xt = x + (int64_t)t * d;
-                float a = 0.f;
-#pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    const int v = v0 + i * 32 + lane;
-                    if (v < nvec) {
-                        const uint4 xv = *reinterpret_cast<const uint4 *>(xt + 8 * v);
-                        const uint32_t ww[4] = {w[i].x, w[i].y, w[i].z, w[i].w};
-                        const uint32_t xx[4] = {xv.x, xv.y, xv.z, xv.w};
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            a = fmaf(__uint_as_float(ww[e] << 16), __uint_as_float(xx[e] << 16), a);
-                            a = fmaf(__uint_as_float(ww[e] & 0xffff0000u), __uint_as_float(xx[e] & 0xffff0000u), a);
-                        }
-                    }
+__global__ void __launch_bounds__(kSelThreads) select_mask_kernel(Workspace ws, int F, int K) {
+    extern __shared__ __align__(16) uint32_t dyn[];  // keys [F] | candidate lists 2 x [kSelListCap]
+    __shared__ SelectSmemT<kSelThreads / 32> sm;      // full radix select (fallback); its arrays double as scratch
+    __shared__ uint32_t s_min[32], s_max[32], s_pick, s_above, s_inbin, s_n;
+    uint32_t *keys = dyn;
+    uint32_t *lists[2] = {dyn + F, dyn + F + kSelListCap};
+    uint32_t *hist = sm.priv;  // 2048 entries
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    constexpr int NW = kSelThreads / 32;
+    const int t = blockIdx.x;
+    const uint32_t bit = 1u << t;
+    const float *g = ws.G + (int64_t)t * ws.ldf;
+
+    // ---- keys, minimum and maximum
+    uint32_t kmin = 0xffffffffu, kmax = 0u;
+    for (int j = tid; j < F; j += kSelThreads) {
+        const uint32_t key = gate_key(g[j]);
+        keys[j] = key;
+        kmin = min(kmin, key);
+        kmax = max(kmax, key);
+    }
+    kmin = __reduce_min_sync(0xffffffffu, kmin);
+    kmax = __reduce_max_sync(0xffffffffu, kmax);
+    if (lane == 0) {
+        s_min[warp] = kmin;
+        s_max[warp] = kmax;
+    }
+    for (int i = tid; i < 2048; i += kSelThreads) hist[i] = 0;
+    if (tid == 0) s_n = 0;
+    __syncthreads();
+    kmin = s_min[lane];
+    kmax = s_max[lane];
+    kmin = __reduce_min_sync(0xffffffffu, kmin);
+    kmax = __reduce_max_sync(0xffffffffu, kmax);
+
+    SelectLevel lv{kmin, kmax, (uint32_t)K, (uint32_t)F};
+    const uint32_t *src = keys;
+    int which = 0;
+    bool failed = false;
+    uint32_t tau = 0, in_bin = 0;
+    int need = 0;
+    // ---- range-relative radix levels
+    while (true) {
+        const uint32_t span = lv.hi - lv.lo;
+        if (span == 0) {  // all candidates equal
+            tau = lv.lo;
+            need = (int)lv.m;
+            in_bin = lv.count;
+            break;
+        }
+        if (lv.count <= 64 && src != keys) {
+            // rank the few candidates directly: candidate i is the answer when exactly m-1 others precede it
+            // in (value descending, position ascending) order
+            if (tid < (int)lv.count) {
+                const uint32_t mine = src[tid];
+                uint32_t before = 0, equal = 0;
+                for (uint32_t i = 0; i < lv.count; ++i) {
+                    const uint32_t o = src[i];
+                    before += (o > mine || (o == mine && i < (uint32_t)tid)) ? 1u : 0u;
+                    equal += o == mine ? 1u : 0u;
                 }
-                part[t] += a;
+                if (before == lv.m - 1) {
+                    uint32_t gt = 0;
+                    for (uint32_t i = 0; i < lv.count; ++i) gt += src[i] > mine ? 1u : 0u;
+                    s_pick = mine;
+                    s_above = lv.m - gt;  // how many keys equal to tau are wanted
+                    s_inbin = equal;
+                }
             }
+            __syncthreads();
+            tau = s_pick;
+            need = (int)s_above;
+            in_bin = s_inbin;
+            break;
         }
+        const int bits = 32 - __clz(span);
+        const int shift = bits > 11 ? bits - 11 : 0;
+        // histogram of (key - lo) >> shift over the candidates (hist is zero on entry)
+        for (uint32_t i = tid; i < lv.count; i += kSelThreads) {
+            const uint32_t key = src[i];
+            if (key >= lv.lo && key <= lv.hi) atomicAdd(&hist[(key - lv.lo) >> shift], 1u);
+        }
+        __syncthreads();
+        // suffix sums: thread i owns bins 2i, 2i+1
+        const uint32_t h0 = hist[2 * tid], h1 = hist[2 * tid + 1];
+        uint32_t s = h0 + h1;
 #pragma unroll
-        for (int t = 0; t < 16; ++t) {
-            if (!((m >> t) & 1u)) continue;
-            const float u = warp_sum(part[t]);
-            if (lane == 0) ws.Zc[(int64_t)p * 16 + t] = silu_f(ws.G[(int64_t)t * ws.ldf + j]) * u;
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t v = __shfl_down_sync(0xffffffffu, s, o);
+            if (lane + o < 32) s += v;
         }
+        if (lane == 0) sm.warp_tot[warp] = s;
+        __syncthreads();
+        {
+            // totals of the warps after this one: a second-level suffix scan done by every warp on its own
+            uint32_t w = sm.warp_tot[lane];
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t v = __shfl_down_sync(0xffffffffu, w, o);
+                if (lane + o < 32) w += v;
+            }
+            const uint32_t after = __shfl_sync(0xffffffffu, w, (warp + 1) & 31);
+            if (warp + 1 < NW) s += after;
+        }
+        if (s - h0 >= lv.m && s - h0 - h1 < lv.m) {
+            s_pick = 2 * tid + 1;
+            s_above = s - h0 - h1;
+            s_inbin = h1;
+        } else if (s >= lv.m && s - h0 < lv.m) {
+            s_pick = 2 * tid;
+            s_above = s - h0;
+            s_inbin = h0;
+        }
+        __syncthreads();
+        const uint32_t bin = s_pick;
+        const uint32_t new_lo = lv.lo + (bin << shift);
+        const uint32_t new_hi = shift ? min(lv.hi, new_lo + ((1u << shift) - 1u)) : new_lo;
+        const uint32_t new_m = lv.m - s_above, new_count = s_inbin;
+        if (shift == 0) {  // the bin is a single key value
+            tau = new_lo;
+            need = (int)new_m;
+            in_bin = new_count;
+            break;
+        }
+        if (new_count > (uint32_t)kSelListCap) {
+            failed = true;
+            break;
+        }
+        // copy the bin's keys to the other list and clear the histogram for the next level
+        uint32_t *dst = lists[which];
+        for (uint32_t i = tid; i < lv.count; i += kSelThreads) {
+            const uint32_t key = src[i];
+            if (key >= new_lo && key <= new_hi) dst[atomicAdd(&s_n, 1u)] = key;
+        }
+        for (int i = tid; i < 2048; i += kSelThreads) hist[i] = 0;
+        __syncthreads();
+        if (tid == 0) s_n = 0;
+        lv = SelectLevel{new_lo, new_hi, new_m, new_count};
+        src = dst;
+        which ^= 1;
+        __syncthreads();
+    }
+    bool ties_cut = true;  // true: some keys equal to tau must be left out -> ordered emission
+    if (failed)
+        block_radix_threshold<kSelThreads>(keys, F, K, sm, tau, need);
+    else
+        ties_cut = in_bin != (uint32_t)need;
+    if (!ties_cut) {
+        // every key >= tau is kept; no order is needed and nothing is read back (plain reductions)
+        for (int j = tid; j < F; j += kSelThreads)
+            if (keys[j] >= tau) atomicOr(&ws.chmask[j], bit);
+    } else {
+        block_ordered_emit<kSelThreads>(keys, F, tau, need, sm, [&](int, int j) { atomicOr(&ws.chmask[j], bit); });
     }
 }
 
 // ---------------------------------------------------------------------------------------------- 4. down
-// out[t, c] = sum_{j in C_t} z[t,j] Wd[j, c]   (Section 5, final output), for the CTA's column slice
-// and its part of the list of used channels.  grid = (slices, parts).
-__global__ void __launch_bounds__(256) down_rows_kernel(const __nv_bfloat16 *__restrict__ wd, int T, int d, int F,
-                                                        Workspace ws, __nv_bfloat16 *__restrict__ out,
-                                                        int *__restrict__ status) {
+// out[t, c] = sum_{j in C_t} z[t,j] Wd[j, c]   (Section 5, final output) for the CTA's column slice and its
+// part of the list of used channels.  grid = (slices, parts).  Tokens are the M dimension of the MMA, the
+// listed channels its contraction index: B[k = channel][n = column] is row-major in shared memory and is
+// read transposed with ldmatrix.
+__global__ void __launch_bounds__(kGemvThreads, 2) down_rows_kernel(const __nv_bfloat16 *__restrict__ wd, int T, int d,
+                                                                    int F, Workspace ws,
+                                                                    __nv_bfloat16 *__restrict__ out,
+                                                                    int *__restrict__ status) {
     extern __shared__ __align__(128) uint8_t dsm[];
-    // layout: ring [2][kBatchRows][1 KiB] | z [kMaxPart][16] floats | channel [kMaxPart] u16 | mask [kMaxPart] u16
+    // layout: ring [kDownStages][16][kDownPitch] | z blocks [kMaxPart / 16][16 tokens][16] bf16 | channel [kMaxPart]
     uint8_t *ring = dsm;
-    float *zl = reinterpret_cast<float *>(dsm + 2 * kBatchRows * 1024);
+    __nv_bfloat16 *zl = reinterpret_cast<__nv_bfloat16 *>(dsm + kDownStages * kDownStageBytes);
     uint16_t *lch = reinterpret_cast<uint16_t *>(zl + kMaxPart * 16);
-    uint16_t *lmask = lch + kMaxPart;
-    __shared__ uint64_t bars[2];
+    __shared__ uint64_t bars[2 * kDownStages];
     __shared__ int s_abort, s_last;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int slice = blockIdx.x, c0 = slice * kSliceCols;
     const int cols = min(kSliceCols, d - c0);       // multiple of 8
     const uint32_t row_bytes = (uint32_t)cols * 2;  // multiple of 16
     const int total = min(*ws.list_count, F);
-    const int per = min(kMaxPart, (total + (int)gridDim.y - 1) / (int)gridDim.y);
-    const int p0 = min(total, (int)blockIdx.y * per);
-    const int count = min(per, total - p0);
+    // parts are whole 16-position blocks, so that a part's z blocks are the ones the up kernel wrote
+    const int blocks_total = (total + 15) >> 4;
+    const int per_blocks = min(kMaxPart / 16, (blocks_total + (int)gridDim.y - 1) / (int)gridDim.y);
+    const int b0 = min(blocks_total, (int)blockIdx.y * per_blocks);
+    const int nblocks = min(per_blocks, blocks_total - b0);
+    const int p0 = b0 * 16;
+    const int count = min(nblocks * 16, total - p0);
+    auto full_bar = [&](int s) { return tc::smem_u32(&bars[s]); };
+    auto empty_bar = [&](int s) { return tc::smem_u32(&bars[kDownStages + s]); };
 
+    for (int i = tid; i < (int)(kDownStages * kDownStageBytes / 16); i += kGemvThreads)
+        reinterpret_cast<uint4 *>(ring)[i] = make_uint4(0, 0, 0, 0);
     if (tid == 0) {
-        tc::mbar_init(tc::smem_u32(&bars[0]), 1);
-        tc::mbar_init(tc::smem_u32(&bars[1]), 1);
+        for (int s = 0; s < kDownStages; ++s) {
+            tc::mbar_init(full_bar(s), 1);
+            tc::mbar_init(empty_bar(s), 8);
+        }
         s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    for (int i = tid; i < count; i += 256) {
-        const int j = ws.list[p0 + i];
-        lch[i] = (uint16_t)j;
-        lmask[i] = (uint16_t)ws.chmask[j];
+    for (int i = tid; i < count; i += kGemvThreads) lch[i] = ws.list[p0 + i];
+    // z blocks of this part: nblocks x 512 bytes, contiguous
+    for (int i = tid; i < nblocks * 32; i += kGemvThreads)
+        reinterpret_cast<uint4 *>(zl)[i] = reinterpret_cast<const uint4 *>(ws.Zb + (int64_t)b0 * 256)[i];
+    __syncthreads();
+    // positions past the end of the list were never written by the up kernel: they must count as zero
+    if (nblocks > 0 && count < nblocks * 16) {
+        for (int i = tid; i < 256; i += kGemvThreads)
+            if ((nblocks - 1) * 16 + (i & 15) >= count) zl[(nblocks - 1) * 256 + i] = __float2bfloat16_rn(0.f);
     }
-    for (int i = tid; i < count * 16; i += 256) zl[i] = ws.Zc[(int64_t)p0 * 16 + i];
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     __syncthreads();
 
-    const int batches = (count + kBatchRows - 1) / kBatchRows;
-    auto issue = [&](int b) {  // warp 0: one bulk copy per lane
-        const int buf = b & 1;
-        const int rows = min(kBatchRows, count - b * kBatchRows);
-        const uint32_t bar = tc::smem_u32(&bars[buf]);
-        if (lane == 0) tc::mbar_expect_tx(bar, (uint32_t)rows * row_bytes);
-        __syncwarp();
-        if (lane < rows) {
-            const int j = lch[b * kBatchRows + lane];
-            const uint32_t dst = tc::smem_u32(ring + ((size_t)buf * kBatchRows + lane) * 1024);
-            const __nv_bfloat16 *src = wd + (int64_t)j * d + c0;
-            asm volatile(
-                "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                ::"r"(dst), "l"(src), "r"(row_bytes), "r"(bar)
-                : "memory");
+    if (warp == 8) {
+        // ------------------------------------------------------------------ producer: 16 rows per stage
+        int stage = 0;
+        uint32_t phase = 0;
+        for (int blk = 0; blk < nblocks; ++blk) {
+            if (!__all_sync(0xffffffffu, tc::mbar_wait(empty_bar(stage), phase ^ 1u, &s_abort, status))) break;
+            const int p = blk * 16 + lane;
+            const bool valid = lane < 16 && p < count;
+            const int nvalid = min(16, count - blk * 16);
+            if (lane == 0) tc::mbar_expect_tx(full_bar(stage), row_bytes * (uint32_t)nvalid);
+            __syncwarp();
+            if (valid)
+                bulk_copy_g2s(tc::smem_u32(ring + stage * kDownStageBytes + lane * kDownPitch),
+                              wd + (int64_t)lch[p] * d + c0, row_bytes, full_bar(stage));
+            if (++stage == kDownStages) {
+                stage = 0;
+                phase ^= 1u;
+            }
         }
-    };
-    float acc[16][2];
+    } else {
+        // ------------------------------------------------------------------ consumers: warp w owns columns 64w..64w+63
+        const int g = lane >> 2, q = lane & 3;
+        float acc[8][4];
 #pragma unroll
-    for (int t = 0; t < 16; ++t) acc[t][0] = acc[t][1] = 0.f;
-    if (warp == 0 && batches > 0) issue(0);
-    uint32_t phase0 = 0, phase1 = 0;
-    for (int b = 0; b < batches; ++b) {
-        const int buf = b & 1;
-        if (warp == 0 && b + 1 < batches) issue(b + 1);  // the other buffer was released by the barrier below
-        const bool ok = tc::mbar_wait(tc::smem_u32(&bars[buf]), buf ? phase1 : phase0, &s_abort, status);
-        if (buf) phase1 ^= 1u; else phase0 ^= 1u;
-        if (!__syncthreads_and(ok)) break;
-        const int rows = min(kBatchRows, count - b * kBatchRows);
-        if (2 * tid < cols) {
-            for (int r = 0; r < rows; ++r) {
-                const int p = b * kBatchRows + r;
-                const uint32_t w2 =
-                    *reinterpret_cast<const uint32_t *>(ring + ((size_t)buf * kBatchRows + r) * 1024 + 4 * tid);
-                const float w0 = __uint_as_float(w2 << 16), w1 = __uint_as_float(w2 & 0xffff0000u);
-                const uint32_t m = lmask[p];
-                const float *zp = zl + p * 16;
+        for (int nb = 0; nb < 8; ++nb)
 #pragma unroll
-                for (int t = 0; t < 16; ++t) {
-                    if ((m >> t) & 1u) {
-                        const float z = zp[t];
-                        acc[t][0] = fmaf(z, w0, acc[t][0]);
-                        acc[t][1] = fmaf(z, w1, acc[t][1]);
+            for (int e = 0; e < 4; ++e) acc[nb][e] = 0.f;
+        int stage = 0;
+        uint32_t phase = 0;
+        for (int blk = 0; blk < nblocks; ++blk) {
+            // A fragment: z[t][position] of this block (tokens g and g+8, positions 2q.. and 2q+8..)
+            const uint32_t *zb = reinterpret_cast<const uint32_t *>(zl + blk * 256);
+            const uint32_t a0 = zb[g * 8 + q], a1 = zb[(g + 8) * 8 + q];
+            const uint32_t a2 = zb[g * 8 + 4 + q], a3 = zb[(g + 8) * 8 + 4 + q];
+            if (!__all_sync(0xffffffffu, tc::mbar_wait(full_bar(stage), phase, &s_abort, status))) break;
+            // ldmatrix.x4.trans: lanes 0..15 address rows k = 0..15 at this column pair's first tile,
+            // lanes 16..31 the same rows 8 columns further: one instruction yields two n-tiles
+            const uint32_t base = tc::smem_u32(ring + stage * kDownStageBytes) + (uint32_t)(lane & 15) * kDownPitch +
+                                  (uint32_t)(warp * 128 + (lane >> 4) * 16);
+#pragma unroll
+            for (int pr = 0; pr < 4; ++pr) {
+                uint32_t b0r, b1r, b2r, b3r;
+                asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                             : "=r"(b0r), "=r"(b1r), "=r"(b2r), "=r"(b3r)
+                             : "r"(base + pr * 32));
+                mma_bf16_16816(acc[2 * pr], a0, a1, a2, a3, b0r, b1r);
+                mma_bf16_16816(acc[2 * pr + 1], a0, a1, a2, a3, b2r, b3r);
+            }
+            __syncwarp();
+            if (lane == 0) tc::mbar_arrive(empty_bar(stage));
+            if (++stage == kDownStages) {
+                stage = 0;
+                phase ^= 1u;
+            }
+        }
+        // add this CTA's partial sums: rows g / g+8 = tokens, columns 64 warp + 8 nb + 2q, +1
+        if (nblocks > 0) {
+#pragma unroll
+            for (int nb = 0; nb < 8; ++nb) {
+                const int c = warp * 64 + nb * 8 + 2 * q;
+                if (c < cols) {
+                    if (g < T) {
+                        atomicAdd(ws.out_acc + (int64_t)g * d + c0 + c, acc[nb][0]);
+                        atomicAdd(ws.out_acc + (int64_t)g * d + c0 + c + 1, acc[nb][1]);
+                    }
+                    if (g + 8 < T) {
+                        atomicAdd(ws.out_acc + (int64_t)(g + 8) * d + c0 + c, acc[nb][2]);
+                        atomicAdd(ws.out_acc + (int64_t)(g + 8) * d + c0 + c + 1, acc[nb][3]);
                     }
                 }
             }
         }
-        __syncthreads();  // everyone is done with `buf` before it is refilled
     }
+    __syncwarp();
     if (s_abort) {
         const long long t0 = clock64();
         while (clock64() - t0 < 2000000LL) __nanosleep(1000);
     }
-    // add this CTA's partial sums, then the last CTA of the slice converts the totals to bf16
-    if (2 * tid < cols && count > 0) {
-#pragma unroll
-        for (int t = 0; t < 16; ++t) {
-            if (t < T) {
-                float *o = ws.out_acc + (int64_t)t * d + c0 + 2 * tid;
-                if (acc[t][0] != 0.f) atomicAdd(o, acc[t][0]);
-                if (acc[t][1] != 0.f) atomicAdd(o + 1, acc[t][1]);
-            }
-        }
-    }
+    // the last CTA of the slice converts the totals to bf16
     __threadfence();
     __syncthreads();
     if (tid == 0) s_last = atomicAdd(&ws.counters[slice], 1) == (int)gridDim.y - 1;
     __syncthreads();
     if (s_last) {
         __threadfence();
-        for (int i = tid; i < T * (cols >> 1); i += 256) {
+        for (int i = tid; i < T * (cols >> 1); i += kGemvThreads) {
             const int t = i / (cols >> 1), c = (i % (cols >> 1)) * 2;
             const float *a = ws.out_acc + (int64_t)t * d + c0 + c;
             const float v0 = __ldcg(a), v1 = __ldcg(a + 1);
