@@ -135,22 +135,33 @@ class ClockSampler:
 
 
 def kernel_work(name: str, T: int, d: int, F: int, K: int, e: int):
-    """Algorithmic work of one step's launches of a kernel: (bound, amount, unit of amount).
+    """Work of one step's launches of a kernel: (bound, algorithmic amount, executed amount, unit).
 
-    Per-token figures (d = d_model, F = d_ff, e = bytes per element):
-      gate projection 2dF flop; selection reads F fp32 and writes K (idx + value);
-      gathered up + down 4Kd flop; backward per-token part 6Kd flop (dz, and both terms of grad_x);
-      weight gradients 6Kd flop.
+    Algorithmic = what the operator needs (per token, d = d_model, F = d_ff, e = bytes per element):
+      gate projection 2dF flop; every contraction with a Top-K operand 2Kd flop per term
+      (up, down, dZ: 2Kd each; three weight gradients 6Kd; two terms of grad_x 4Kd);
+      selection reads the fp32 gate row (4F B) and the K kept up values (eK) and writes idx/g/u (K(2+2e) B).
+    Executed = what the tensor-core plan runs: every contraction dense over F (2dF per term), and the dense
+    masked arrays it writes for the next contraction.
     """
     table = {
-        "gate_gemm_alu": ("tensor", 2.0 * T * d * F, "flop"),
-        "gate_up_gemm_tc": ("tensor", 4.0 * T * d * F, "flop"),
-        "select_rows": ("hbm", T * F * 4.0 + T * K * (2.0 + e), "byte"),
-        "forward_token": ("alu", 4.0 * T * K * d, "flop"),
-        "backward_token": ("alu", 6.0 * T * K * d, "flop"),
-        "wgrad_rows": ("alu", 6.0 * T * K * d, "flop"),
-        "csr_count": ("hbm", T * K * 2.0, "byte"),
-        "csr_fill": ("hbm", T * K * 6.0, "byte"),
+        # gathered plan
+        "gate_gemm_alu": ("tensor", 2.0 * T * d * F, 2.0 * T * d * F, "flop"),
+        "select_rows": ("hbm", T * F * 4.0 + T * K * (2.0 + e), T * F * 4.0 + T * K * (2.0 + e), "byte"),
+        "forward_token": ("alu", 4.0 * T * K * d, 4.0 * T * K * d, "flop"),
+        "backward_token": ("alu", 6.0 * T * K * d, 6.0 * T * K * d, "flop"),
+        "wgrad_rows": ("alu", 6.0 * T * K * d, 6.0 * T * K * d, "flop"),
+        "csr_count": ("hbm", T * K * 2.0, T * K * 2.0, "byte"),
+        "csr_fill": ("hbm", T * K * 6.0, T * K * 6.0, "byte"),
+        # tensor-core plan
+        "tc_gate_up_gemm": ("tensor", 2.0 * T * d * F + 2.0 * T * K * d, 4.0 * T * d * F, "flop"),
+        "tc_select_mask": ("hbm", T * (4.0 * F + e * K + K * (2.0 + 2 * e)),
+                           T * (4.0 * F + e * K + K * (2.0 + 2 * e) + 2.0 * F), "byte"),
+        "tc_down_gemm": ("tensor", 2.0 * T * K * d, 2.0 * T * d * F, "flop"),
+        "tc_dz_gemm": ("tensor", 2.0 * T * K * d, 2.0 * T * d * F, "flop"),
+        "tc_bwd_sample": ("hbm", T * K * (2.0 + 2 * e + e), T * (K * (2.0 + 3 * e) + 6.0 * F), "byte"),
+        "tc_wgrad_gemm": ("tensor", 6.0 * T * K * d, 6.0 * T * d * F, "flop"),
+        "tc_dx_gemm": ("tensor", 4.0 * T * K * d, 4.0 * T * d * F, "flop"),
     }
     return table.get(name)
 
@@ -414,9 +425,11 @@ def roofline_report(prof, steps, T, w, e, peaks):
     work = kernel_work(top, T, w.d_model, w.d_ff, w.k, e)
     roof = {"kernel": top, "launches": n, "avg_ms": ms / n}
     if work:
-        bound, amount, unit = work
+        bound, amount, executed, unit = work
         per_launch = amount * steps / n          # `amount` is per step
         rate = per_launch / (ms / n / 1e3)
+        roof["executed_per_launch"] = executed * steps / n
+        roof["executed_rate"] = executed * steps / n / (ms / n / 1e3) / (1e9 if bound == "hbm" else 1e12)
         if bound == "hbm":
             roof.update(bound="hbm", achieved=rate / 1e9, peak=peaks["hbm_gbs"], unit="GB/s")
         elif bound == "tensor":
@@ -453,37 +466,52 @@ def act_bytes_report(w, T, e, saved, B, desc):
             "dense_gcp_per_token": 2 * w.d_ff * e, "x_and_out_per_token_each": w.d_model * e}
 
 
-def decode_report(torch, B, syn, dev, peaks, iters=48, sets=4):
-    """moc_ffn_decode on the LLaMA-7B shape for 1/4/16 tokens; weight sets rotate so that every call
-    streams its weights from HBM (4 sets x 270 MB > L2)."""
+def decode_report(torch, B, syn, dev, peaks, calls=32, sets=4, replays=5):
+    """moc_ffn_decode on the LLaMA-7B shape for 1/4/16 tokens.  One CUDA graph holds `calls` back-to-back calls
+    that rotate through `sets` distinct weight sets (4 x 270 MB > L2), so every call streams its weights from
+    HBM and launch overhead is what a served model would see; the graph is replayed `replays` times."""
     w = syn.C4
     weights = [tuple(t.to(dev) for t in syn.make_weights(w, seed_offset=s)) for s in range(sets)]
-    rep = {"weight_sets": sets, "iters": iters}
+    rep = {"weight_sets": sets, "calls_per_graph": calls, "replays": replays, "timing": "CUDA graph replay"}
     e = 2
+    stream = torch.cuda.Stream(device=dev)
     for T in syn.C4_BATCHES:
         x = syn.make_x(w, tokens=T).to(dev)
         out = torch.empty_like(x)
         desc = B.make_desc(T, w.d_model, w.d_ff, w.k, x.dtype, d_ff_ld=w.d_ff_ld)
         ws = B.alloc_workspace(desc, B.MOC_OP_DECODE, dev)
-        for i in range(sets):
+        for i in range(sets):   # warm-up; also performs every one-time set-up outside the capture
             B.moc_ffn_decode(x, *weights[i], w.k, out=out, workspace=ws)
+        torch.cuda.synchronize()
+        launches0 = B.moc_launch_count()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(stream):
+            with torch.cuda.graph(graph, stream=stream):
+                for i in range(calls):
+                    B.moc_ffn_decode(x, *weights[i % sets], w.k, out=out, workspace=ws, stream=stream)
+        launches = (B.moc_launch_count() - launches0) // calls
+        torch.cuda.synchronize()
+        graph.replay()
         torch.cuda.synchronize()
         s, t = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         s.record()
-        for i in range(iters):
-            B.moc_ffn_decode(x, *weights[i % sets], w.k, out=out, workspace=ws)
+        for _ in range(replays):
+            graph.replay()
         t.record()
         torch.cuda.synchronize()
-        us = s.elapsed_time(t) * 1e3 / iters
-        # union of selected channels from an extra saved forward on set 0
+        us = s.elapsed_time(t) * 1e3 / (calls * replays)
+        # union of selected channels from a saved forward on set 0 (same selection rule)
         _, idx, _, _ = B.moc_ffn_forward(x, *weights[0], w.k)
         union = int(torch.unique(idx.long()).numel())
         algo = w.d_ff * w.d_model * e + 2 * union * w.d_model * e + 2 * T * w.d_model * e
         roof_us = algo / (peaks["hbm_gbs"] * 1e9) * 1e6
         rep[f"T{T}"] = {"us_per_step": us, "us_per_token": us / T, "union_channels": union,
                         "algorithmic_bytes": algo, "roofline_us": roof_us, "frac": roof_us / us,
-                        "achieved_gbs": algo / (us * 1e-6) / 1e9}
-        del ws
+                        "achieved_gbs": algo / (us * 1e-6) / 1e9, "kernels_per_call": launches,
+                        "dense_ffn_bytes": 3 * w.d_ff * w.d_model * e}
+        del ws, graph
+    if B.moc_last_device_status() != B.MOC_OK:
+        raise RuntimeError("device status raised during decode")
     return rep
 
 

@@ -26,11 +26,18 @@ def test_shard_plan_and_aggregate_single_process():
 
 def test_kernel_work_table_matches_per_token_formulas():
     T, d, F, K, e = 16384, 768, 2048, 256, 2
-    assert bench.kernel_work("gate_gemm_alu", T, d, F, K, e) == ("tensor", 2.0 * T * d * F, "flop")
+    assert bench.kernel_work("gate_gemm_alu", T, d, F, K, e)[:2] == ("tensor", 2.0 * T * d * F)
     assert bench.kernel_work("select_rows", T, d, F, K, e)[1] == T * F * 4 + T * K * 4
-    # forward + backward sparse work adds up to the 16 T K d of the operator
+    # gathered plan: forward + backward sparse work adds up to the 16 T K d of the operator
     total = sum(bench.kernel_work(k, T, d, F, K, e)[1] for k in ("forward_token", "backward_token", "wgrad_rows"))
     assert total == 16.0 * T * K * d
+    # tensor-core plan: algorithmic flops = gate 2TdF + 16TKd; executed flops = 18TdF (every contraction dense)
+    gemms = ("tc_gate_up_gemm", "tc_down_gemm", "tc_dz_gemm", "tc_wgrad_gemm", "tc_dx_gemm")
+    assert sum(bench.kernel_work(k, T, d, F, K, e)[1] for k in gemms) == 2.0 * T * d * F + 16.0 * T * K * d
+    assert sum(bench.kernel_work(k, T, d, F, K, e)[2] for k in gemms) == 18.0 * T * d * F
+    for k in gemms:
+        bound, algo, executed, unit = bench.kernel_work(k, T, d, F, K, e)
+        assert bound == "tensor" and unit == "flop" and executed >= algo
     assert bench.kernel_work("nonexistent", T, d, F, K, e) is None
 
 

@@ -271,3 +271,118 @@ def test_decode_small_shapes(dtype, T, d, F, K):
     x64, wg64, wu64, wd64 = map(syn.to_f64, (x, wg, wu, wd))
     _check_decode(syn.to_f64(out), x64, wg64, wu64, wd64, K, dtype, "decode")
     _check_decode(syn.to_f64(out_f), x64, wg64, wu64, wd64, K, dtype, "forward(save=False)")
+
+
+# ------------------------------------------------------------------ tensor-core plan (bf16, tokens >= 256)
+
+
+@pytest.mark.parametrize("T,d,F,F_ld,K", [
+    (513, 264, 1100, 1104, 137),   # d not a multiple of 64, F not a multiple of 256, ragged token tile
+    (256, 128, 96, 96, 96),        # K = F: dense SwiGLU through the tensor-core plan
+    (384, 512, 4500, 4504, 563),   # more than 4096 channels: CTA-per-token selector
+])
+def test_tc_plan_shapes(T, d, F, F_ld, K):
+    w = syn.Workload(f"tc-{T}-{d}-{F}-{K}", "bf16", T, d, F, F_ld, K, seed=200 + T)
+    _run_forward_backward(w)
+
+
+def test_tc_plan_llama1b_padded_slice():
+    """C3's layer (d_ff = 5461 in arrays of 5504 rows) on enough tokens to take the tensor-core plan."""
+    _run_forward_backward(syn.C3.with_tokens(384))
+
+
+def test_tc_plan_sweep_k_fractions():
+    """C5's K fractions d_ff/16, d_ff/8, d_ff/4 on a 1B-shaped layer narrowed to keep the oracle fast."""
+    for K in (64, 128, 256):
+        w = syn.Workload(f"c5-{K}", "bf16", 320, 512, 1024, 1024, K, seed=500 + K)
+        _run_forward_backward(w)
+
+
+def test_ties_go_to_the_lower_channel_on_both_plans():
+    """Duplicated gate rows give bit-identical gate values; when only one of a pair fits, it must be the lower."""
+    for T in (64, 320):   # gathered plan, tensor-core plan
+        w = syn.Workload("ties", "bf16", T, 128, 512, 512, 65, seed=77)
+        wg, wu, wd = syn.make_weights(w)
+        wg[1::2] = wg[0::2]          # channels 2i and 2i+1 share their gate row
+        x = syn.make_x(w)
+        out, idx, tg, tu = B.moc_ffn_forward(_dev(x), _dev(wg), _dev(wu), _dev(wd), w.k)
+        idx = idx.cpu().numpy().astype(np.int64)
+        split = 0
+        for t in range(T):
+            sel = set(idx[t].tolist())
+            for j in idx[t]:
+                if j % 2 == 1:
+                    assert j - 1 in sel, f"token {t}: channel {j} kept without its equal lower twin {j - 1}"
+                elif j + 1 not in sel:
+                    split += 1
+        assert split > 0   # K is odd: every token splits exactly one pair
+        x64, wg64, wu64, wd64 = map(syn.to_f64, (x, wg, wu, wd))
+        dev = dict(out=syn.to_f64(out), idx=idx, gval=syn.to_f64(tg), uval=syn.to_f64(tu))
+        parity.check_forward(dev, x64, wg64, wu64, wd64, w.k, w.d_ff, w.dtype)
+
+
+def test_tc_plan_backward_options_and_determinism():
+    w = syn.Workload("tc-opts", "bf16", 384, 256, 768, 768, 96, seed=41)
+    _, (x, wg, wu, wd, dD), (out, idx, tg, tu), full = _run_forward_backward(w)
+    out2, idx2, tg2, tu2 = B.moc_ffn_forward(x, wg, wu, wd, w.k)
+    assert torch.equal(out, out2) and torch.equal(idx, idx2) and torch.equal(tg, tg2) and torch.equal(tu, tu2)
+    again = B.moc_ffn_backward(x, wg, wu, wd, idx, tg, tu, dD)
+    for k in full:
+        assert torch.equal(full[k], again[k]), k
+    part = B.moc_ffn_backward(x, wg, wu, wd, idx, tg, tu, dD, want=("w_down", "x"))
+    assert part["grad_w_gate"] is None and part["grad_w_up"] is None
+    assert torch.equal(part["grad_w_down"], full["grad_w_down"]) and torch.equal(part["grad_x"], full["grad_x"])
+    base = {k: torch.full_like(v, 0.25) for k, v in full.items() if k != "grad_x"}
+    acc = B.moc_ffn_backward(x, wg, wu, wd, idx, tg, tu, dD, want=("w_gate", "w_up", "w_down"), grads=base,
+                             accumulate=True)
+    for k in ("grad_w_gate", "grad_w_up", "grad_w_down"):
+        ref = full[k].float() + 0.25
+        assert (acc[k].float() - ref).abs().max() <= 1e-2 * ref.abs().max()
+    inf_out, *_ = B.moc_ffn_forward(x, wg, wu, wd, w.k, save=False)
+    assert torch.equal(inf_out, out)
+
+
+def test_tc_plan_corrupted_saved_index_is_skipped_and_reported():
+    w = syn.Workload("tc-bad", "bf16", 300, 128, 256, 256, 32, seed=13)
+    _, (x, wg, wu, wd, dD), (out, idx, tg, tu), full = _run_forward_backward(w)
+    bad = idx.clone()
+    bad[5, 3] = 256
+    bad[9, 0] = -1
+    g = B.moc_ffn_backward(x, wg, wu, wd, bad, tg, tu, dD)
+    assert B.moc_last_device_status() == B.MOC_ERR_BAD_INDEX
+    assert B.moc_last_device_status() == B.MOC_OK
+    keep = torch.ones(w.tokens, dtype=torch.bool, device="cuda")
+    keep[5] = keep[9] = False
+    assert torch.equal(g["grad_x"][keep], full["grad_x"][keep])
+    for k in g:
+        assert torch.isfinite(g[k].float()).all()
+
+
+def test_full_size_bench_workload_sampled_against_oracle():
+    """C2 at its full 16384 tokens, in the configuration bench.py times: sampled tokens of out / saved values /
+    grad_x and sampled rows of the weight gradients are recomputed one by one by the oracle."""
+    w = syn.C2
+    x, wg, wu, wd, dD = _problem(w)
+    xd, wgd, wud, wdd, dDd = map(_dev, (x, wg, wu, wd, dD))
+    out, idx, tg, tu = B.moc_ffn_forward(xd, wgd, wud, wdd, w.k)
+    grads = B.moc_ffn_backward(xd, wgd, wud, wdd, idx, tg, tu, dDd)
+    torch.cuda.synchronize()
+    assert B.moc_last_device_status() == B.MOC_OK
+    rng = np.random.default_rng(0)
+    toks = np.sort(rng.choice(w.tokens, 96, replace=False))
+    wg64, wu64, wd64 = map(syn.to_f64, (wg, wu, wd))
+    x64s, dD64s = syn.to_f64(x[toks]), syn.to_f64(dD[toks])
+    idx_np = idx.cpu().numpy()
+    dev = dict(out=syn.to_f64(out[toks]), idx=idx_np[toks], gval=syn.to_f64(tg[toks]), uval=syn.to_f64(tu[toks]))
+    parity.check_forward(dev, x64s, wg64, wu64, wd64, w.k, w.d_ff, w.dtype)
+    ref = orc.backward(x64s, wg64, wu64, wd64, idx_np[toks].astype(np.int32), dev["gval"], dev["uval"], dD64s,
+                       want=("x",))
+    parity.assert_close(syn.to_f64(grads["grad_x"][toks]), ref["grad_x"], w.dtype, "grad_x (sampled tokens)")
+    rows = np.sort(rng.choice(w.d_ff, 24, replace=False)).astype(np.int32)
+    wrows = orc.backward_weight_rows(syn.to_f64(x), wd64, idx_np.astype(np.int32), syn.to_f64(tg), syn.to_f64(tu),
+                                     syn.to_f64(dD), rows, w.d_ff)
+    for name in ("grad_w_gate", "grad_w_up", "grad_w_down"):
+        got = syn.to_f64(grads[name][torch.from_numpy(rows.astype(np.int64)).cuda()])
+        parity.assert_close(got, wrows[name], w.dtype, name + " (sampled rows)")
+    # structural properties at full size
+    parity.check_index_sets(idx_np, w.d_ff)
