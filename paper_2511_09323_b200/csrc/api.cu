@@ -184,9 +184,9 @@ BackwardPlan plan_backward(const moc_ffn_desc &d) {
 }
 
 template <typename K>
-int set_smem(K kernel, size_t bytes) {
-    // kernels that use the selector also hold its static shared state (up to 47 KiB with 1024 threads)
-    constexpr size_t kStaticReserve = 48 * 1024;
+int set_smem(K kernel, size_t bytes, size_t kStaticReserve = 48 * 1024) {
+    // by default room is left for the selector's static shared state (up to 47 KiB with 1024 threads), which
+    // most kernels that call this hold
     if (bytes + kStaticReserve > (size_t)kMaxDynSmem) return MOC_ERR_UNSUPPORTED;
     if (bytes + kStaticReserve > 48 * 1024) {
         // the attribute only ever grows; remember what was set so that steady-state calls make no driver call
@@ -318,20 +318,37 @@ int forward_tc(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat1
 
     // selector: one warp per token while a row fits in registers (F <= 4096), else one CTA per token
     const int nv = F <= 1024 ? 8 : (F <= 2048 ? 16 : (F <= 4096 ? 32 : 0));
-    const size_t warp_smem = 8 * ((size_t)kWarpSelCand + 2 * (size_t)K) * sizeof(uint32_t);
+    // each warp stages its token's rows in its own slice of shared memory: as many warps per SM as fit, in one
+    // or two CTAs
+    const size_t warp_bytes = nv ? warp_select_words(nv, K) * sizeof(uint32_t) : 0;
+    const int warps_per_sm = nv ? (int)std::min<size_t>((size_t)220 * 1024 / warp_bytes, 2 * kWarpSelMaxWarps) : 0;
+    const int sel_ctas_per_sm = warps_per_sm > 4 ? 2 : 1;
+    const int sel_wpc = warps_per_sm / sel_ctas_per_sm;
+    const size_t warp_smem = (size_t)sel_wpc * warp_bytes;
     const size_t cta_smem = ((size_t)F + K) * sizeof(uint32_t);
-    const bool warp_select = nv != 0 && warp_smem + 48 * 1024 <= (size_t)kMaxDynSmem;
+    const bool warp_select = nv != 0 && sel_wpc >= 1;
     float *hint = reinterpret_cast<float *>(ws + L.off_hint);
     int rc = MOC_OK;
     if (warp_select) {
-        if (nv == 8) rc = set_smem(select_mask_rows_warp_kernel<8>, warp_smem);
-        if (nv == 16) rc = set_smem(select_mask_rows_warp_kernel<16>, warp_smem);
-        if (nv == 32) rc = set_smem(select_mask_rows_warp_kernel<32>, warp_smem);
+        if (nv == 8) rc = set_smem(select_mask_rows_warp_kernel<8>, warp_smem, 2048);
+        if (nv == 16) rc = set_smem(select_mask_rows_warp_kernel<16>, warp_smem, 2048);
+        if (nv == 32) rc = set_smem(select_mask_rows_warp_kernel<32>, warp_smem, 2048);
     } else {
         rc = set_smem(select_mask_rows_kernel, cta_smem);
     }
     if (rc != MOC_OK) return rc;
     if ((rc = set_smem(select_hint_kernel, (size_t)F * sizeof(uint32_t))) != MOC_OK) return rc;
+    // Warp selector: every launch works with one bracket kept in the workspace ({center, width, tag} at
+    // hint[0..2]); it gathers the statistics of its thresholds (hint[4..6], CTA counter at hint[8]) and its last
+    // CTA rewrites the bracket for the next launch.  The bracket is only a hint: a stale or garbage one costs
+    // time (rows take the slow exact path), never correctness.  The statistics are cleared per call.
+    SelectMeta meta{};
+    if (warp_select) {
+        meta.bracket = hint;
+        meta.acc = hint + 4;
+        meta.done = reinterpret_cast<unsigned int *>(hint + 8);
+        if (cudaMemsetAsync(hint + 4, 0, 32, st) != cudaSuccess) return MOC_ERR_CUDA;
+    }
 
     int *status = device_status_ptr();
     if (!status) return MOC_ERR_CUDA;
@@ -355,7 +372,7 @@ int forward_tc(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat1
         p.c[1] = U + t0 * L.ldf;
         MOC_LAUNCH(KID_TC_GATE_UP_GEMM, st, (rc = launch_gemm<false, false, EPI_GATE_UP>(p, st)));
         if (rc != MOC_OK) return rc;
-        if (t0 == 0) {
+        if (t0 == 0 && !warp_select) {
             MOC_LAUNCH(KID_TC_SELECT_HINT, st,
                        (select_hint_kernel<<<1, kSelectThreads, (size_t)F * sizeof(uint32_t), st>>>(G, F, K, hint)));
             if ((rc = launch_ok()) != MOC_OK) return rc;
@@ -364,19 +381,20 @@ int forward_tc(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat1
         __nv_bfloat16 *o_g = idx ? tg + t0 * K : nullptr, *o_u = idx ? tu + t0 * K : nullptr;
         __nv_bfloat16 *Uc = U + t0 * L.ldf;
         if (warp_select) {
-            const unsigned grid = (unsigned)std::min<int64_t>((n + 7) / 8, (int64_t)sm_count() * 4);
+            const unsigned grid =
+                (unsigned)std::min<int64_t>((n + sel_wpc - 1) / sel_wpc, (int64_t)sm_count() * sel_ctas_per_sm);
             if (nv == 8)
                 MOC_LAUNCH(KID_TC_SELECT_MASK, st,
-                           (select_mask_rows_warp_kernel<8><<<grid, 256, warp_smem, st>>>(G, L.ldf, Uc, L.ldf, n, F, K,
-                                                                                           o_idx, o_g, o_u, hint)));
+                           (select_mask_rows_warp_kernel<8><<<grid, sel_wpc * 32, warp_smem, st>>>(G, L.ldf, Uc, L.ldf, n, F, K,
+                                                                                           o_idx, o_g, o_u, meta, status)));
             else if (nv == 16)
                 MOC_LAUNCH(KID_TC_SELECT_MASK, st,
-                           (select_mask_rows_warp_kernel<16><<<grid, 256, warp_smem, st>>>(G, L.ldf, Uc, L.ldf, n, F, K,
-                                                                                            o_idx, o_g, o_u, hint)));
+                           (select_mask_rows_warp_kernel<16><<<grid, sel_wpc * 32, warp_smem, st>>>(G, L.ldf, Uc, L.ldf, n, F, K,
+                                                                                            o_idx, o_g, o_u, meta, status)));
             else
                 MOC_LAUNCH(KID_TC_SELECT_MASK, st,
-                           (select_mask_rows_warp_kernel<32><<<grid, 256, warp_smem, st>>>(G, L.ldf, Uc, L.ldf, n, F, K,
-                                                                                            o_idx, o_g, o_u, hint)));
+                           (select_mask_rows_warp_kernel<32><<<grid, sel_wpc * 32, warp_smem, st>>>(G, L.ldf, Uc, L.ldf, n, F, K,
+                                                                                            o_idx, o_g, o_u, meta, status)));
         } else {
             const unsigned grid = (unsigned)std::min<int64_t>(n, (int64_t)sm_count() * 6);
             MOC_LAUNCH(KID_TC_SELECT_MASK, st,
@@ -848,3 +866,5 @@ const char *moc_status_string(int status) {
 }
 
 }  // extern "C"
+
+

@@ -124,190 +124,395 @@ __global__ void __launch_bounds__(kSelectThreads) select_hint_kernel(const float
 }
 
 // ------------------------------------------------------------------------------------------------
-// Forward selector for rows of at most NV * 128 channels: ONE WARP per token, the row's keys live in
-// registers (NV float4 loads per lane), no block barriers.  Same outputs as the CTA-per-token kernel
-// below.  Threshold: bracket from the hint / the warp's previous row, verified by counting; inside
-// the bracket an exact bitwise search over the few keys it holds; if the bracket fails, the same
-// bitwise search over all registers.  Emission is an ordered warp scan, so indices come out
-// ascending and ties go to the lower channel.
-constexpr int kWarpSelCand = 384;
+// Forward selector for rows of at most NV * 128 channels: ONE WARP per token, no block barriers.
+// Same outputs as the CTA-per-token kernel below.
+//
+// Every warp owns a slice of shared memory into which lane 0 bulk-copies the token's gate row (fp32) and up
+// row (bf16); the warp works on those copies, turns the up row into the masked Z' row in place and
+// bulk-stores it back.  All global traffic of a row is therefore three asynchronous, fully coalesced
+// copies plus the compact outputs, and the scattered accesses of the method (K values per token) stay in
+// shared memory.
+//
+// The launch starts from one bracket [center - width, center + width] that is expected to contain every
+// row's threshold; it comes from the thresholds of the previous launch (kept in the workspace).  A row whose
+// threshold lies outside moves the bracket (tripling its reach on that side) and tries again; without a
+// bracket from an earlier launch a warp derives one from the first threshold it finds.  Per row:
+//   1. the gate values are classified with plain float compares: values above the bracket are counted,
+//      values inside it are parked (raw bits) in the lane's column of shared memory;
+//   2. if the counts prove that the K-th largest value is a parked one, a 64-bin histogram over the
+//      bracket's key range finds its bin and the few keys of that bin are ranked exactly: threshold tau;
+//   3. when no tie has to be cut, the kept set is {g >= tau}: one compare per value, four flags per
+//      lane and 128-channel group go to a shared bitmap, which is then enumerated in ascending order;
+//   4. values of the kept channels, compact outputs, masked row.
+// Rows for which 1-3 do not apply (no bracket yet, too many parked keys, ties to cut, non-finite
+// threshold, inconsistent counts) take the general exact path (8-bit radix selection over the
+// staged row).  Either way the result is exact: indices ascending, ties to the lower channel.
+constexpr int kWarpSelSlots = 14;                        // parked keys per lane
+constexpr int kWarpSelCand = (kWarpSelSlots + 1) * 32;   // one more row absorbs the overflow of a column
+constexpr int kWarpSelWords = 128;                       // bitmap words (4096 channels)
+constexpr float kBracketTag = 20251109.0f;
+constexpr int kWarpSelMaxWarps = 8;                      // warps per CTA, at most
 
-template <int NV>
-__global__ void __launch_bounds__(256) select_mask_rows_warp_kernel(
-    const float *__restrict__ G, int ldg, __nv_bfloat16 *__restrict__ U, int ldu, int64_t rows, int F, int K,
-    int16_t *__restrict__ idx_out, __nv_bfloat16 *__restrict__ g_out, __nv_bfloat16 *__restrict__ u_out,
-    const float *__restrict__ hint) {
-    extern __shared__ __align__(16) uint32_t warp_sel_smem[];  // per warp: kWarpSelCand + 2 K words
-    const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
-    uint32_t *cand = warp_sel_smem + (size_t)wib * (kWarpSelCand + 2 * K);
-    uint32_t *packed = cand + kWarpSelCand;  // [K] key of the kept channel, later its z (bf16 bits)
-    uint32_t *packed_j = packed + K;         // [K] channel
+// Words of shared memory one warp needs: gate row, up row, parked keys, bitmap, kept list, mbarrier.
+__host__ __device__ constexpr size_t warp_select_words(int nv, int K) {
+    return (size_t)nv * 128 + (size_t)nv * 64 + kWarpSelCand + kWarpSelWords + (size_t)((K + 3) & ~3) + 4;
+}
+
+struct SelectMeta {
+    float *bracket;      // {center, half width, tag}; rewritten by the last CTA of the launch
+    float *acc;          // {sum of thresholds, sum of |threshold - center|, rows}: this launch's statistics
+    unsigned int *done;  // CTAs finished
+};
+
+__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_copy_s2g(void *dst, uint32_t src, uint32_t bytes) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src), "r"(bytes)
+                 : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+__device__ __forceinline__ void bulk_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// General exact path for one staged row: most-significant-digit radix selection with 8-bit digits.
+// g: the row in shared memory (ncols values, channels past the end hold -inf and are never counted because
+// only the first F are visited); hist: 256 words of the warp's shared memory.  Leaves the kept channels
+// (ascending) in kept[0..K) and returns the threshold key.
+__device__ __noinline__ uint32_t warp_select_row_general(const float *g, int F, int K, uint32_t *hist,
+                                                         uint32_t *kept) {
+    const int lane = threadIdx.x & 31;
     const uint32_t lt_mask = (1u << lane) - 1u;
-    const int64_t gw = (int64_t)blockIdx.x * 8 + wib, nw = (int64_t)gridDim.x * 8;
-    SelectGuess guess = guess_from_hint(hint);
-
-    for (int64_t r = gw; r < rows; r += nw) {
-        const float *g = G + r * (int64_t)ldg;
-        __nv_bfloat16 *u = U + r * (int64_t)ldu;
-        // ---- keys: lane holds channels (v*32 + lane)*4 .. +3 of every 128-channel group v
-        uint32_t key[NV][4];
-#pragma unroll
-        for (int v = 0; v < NV; ++v) {
-            const int c0 = (v * 32 + lane) * 4;
-            float4 f = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (c0 < F) f = *reinterpret_cast<const float4 *>(g + c0);
-            key[v][0] = c0 + 0 < F ? gate_key(f.x) : 0u;
-            key[v][1] = c0 + 1 < F ? gate_key(f.y) : 0u;
-            key[v][2] = c0 + 2 < F ? gate_key(f.z) : 0u;
-            key[v][3] = c0 + 3 < F ? gate_key(f.w) : 0u;
-        }
-        // ---- bracket: count and collect
-        uint32_t tau = 0;
-        int need = 0;
-        bool solved = false, overflow = false;
-        if (guess.valid) {
-            const uint32_t lo = gate_key(guess.center - guess.delta), hi = gate_key(guess.center + guess.delta);
-            uint32_t cnt = 0, n_band = 0;
-#pragma unroll
-            for (int v = 0; v < NV; ++v) {
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const uint32_t k32 = key[v][e];
-                    const bool above = k32 > hi, not_below = k32 >= lo;
-                    cnt += (above ? 1u : 0u) + (not_below ? 0x10000u : 0u);
-                    const bool band = not_below && !above;
-                    const uint32_t b = __ballot_sync(0xffffffffu, band);
-                    if (b) {
-                        const uint32_t slot = n_band + (uint32_t)__popc(b & lt_mask);
-                        if (band && slot < (uint32_t)kWarpSelCand) cand[slot] = k32;
-                        n_band += (uint32_t)__popc(b);
-                    }
-                }
-            }
-            cnt = __reduce_add_sync(0xffffffffu, cnt);
-            const uint32_t c_hi = cnt & 0xffffu, c_lo = cnt >> 16;
-            overflow = n_band > (uint32_t)kWarpSelCand;
-            solved = c_hi < (uint32_t)K && c_lo >= (uint32_t)K && !overflow;
-            if (solved) {
-                __syncwarp();
-                const uint32_t m = (uint32_t)K - c_hi;
-                uint32_t res = hi;
-                if (lo != hi) {
-                    const int top = 31 - __clz(lo ^ hi);
-                    res = hi & ~((2u << top) - 1u);
-                    for (int bit = top; bit >= 0; --bit) {
-                        const uint32_t trial = res | (1u << bit);
-                        uint32_t c = 0;
-                        for (uint32_t i = lane; i < n_band; i += 32) c += cand[i] >= trial ? 1u : 0u;
-                        c = __reduce_add_sync(0xffffffffu, c);
-                        if (c >= m) res = trial;
-                    }
-                }
-                uint32_t gt = 0;
-                for (uint32_t i = lane; i < n_band; i += 32) gt += cand[i] > res ? 1u : 0u;
-                gt = __reduce_add_sync(0xffffffffu, gt);
-                tau = res;
-                need = (int)(m - gt);
-            }
-        }
-        if (!solved) {
-            // exact K-th largest by bitwise search over the registers
-            uint32_t res = 0;
-#pragma unroll 1
-            for (int bit = 31; bit >= 0; --bit) {
-                const uint32_t trial = res | (1u << bit);
-                uint32_t c = 0;
-#pragma unroll
-                for (int v = 0; v < NV; ++v)
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) c += key[v][e] >= trial ? 1u : 0u;
-                c = __reduce_add_sync(0xffffffffu, c);
-                if (c >= (uint32_t)K) res = trial;
-            }
-            uint32_t gt = 0;
-#pragma unroll
-            for (int v = 0; v < NV; ++v)
-#pragma unroll
-                for (int e = 0; e < 4; ++e) gt += key[v][e] > res ? 1u : 0u;
-            gt = __reduce_add_sync(0xffffffffu, gt);
-            tau = res;
-            need = K - (int)gt;
-        }
-        // ---- ordered emission (group v, then lane, then element)
-        uint32_t run_gt = 0, run_eq = 0;
-#pragma unroll
-        for (int v = 0; v < NV; ++v) {
-            uint32_t local = 0;
-#pragma unroll
-            for (int e = 0; e < 4; ++e)
-                local += (key[v][e] > tau ? 1u : 0u) + (key[v][e] == tau ? 0x10000u : 0u);
-            uint32_t inc = local;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const uint32_t nb = __shfl_up_sync(0xffffffffu, inc, o);
-                if (lane >= o) inc += nb;
-            }
-            const uint32_t total = __shfl_sync(0xffffffffu, inc, 31);
-            if (local) {
-                uint32_t gt_b = run_gt + ((inc - local) & 0xffffu), eq_b = run_eq + ((inc - local) >> 16);
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const uint32_t k32 = key[v][e];
-                    const bool gt = k32 > tau, eq = k32 == tau;
-                    if (gt || (eq && eq_b < (uint32_t)need)) {
-                        // only shared-memory stores here: global loads inside this ordered walk would
-                        // serialise one memory round trip per element
-                        const int pos = (int)(gt_b + min(eq_b, (uint32_t)need));
-                        packed[pos] = k32;
-                        packed_j[pos] = (uint32_t)((v * 32 + lane) * 4 + e);
-                    }
-                    gt_b += gt ? 1u : 0u;
-                    eq_b += eq ? 1u : 0u;
-                }
-            }
-            run_gt += total & 0xffffu;
-            run_eq += total >> 16;
+    uint32_t prefix = 0, kk = (uint32_t)K;  // kk: rank of the threshold among the keys that share the prefix
+    for (int pass = 0; pass < 4; ++pass) {
+        const int shift = 24 - 8 * pass;
+        for (int i = lane; i < 256; i += 32) hist[i] = 0u;
+        __syncwarp();
+        for (int j = lane; j < F; j += 32) {
+            const uint32_t key = gate_key(g[j]);
+            if (pass == 0 || (key >> (shift + 8)) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
         }
         __syncwarp();
-        // ---- values of the kept channels: independent iterations, so the scattered loads of u overlap;
-        //      the compact outputs are written with consecutive lanes on consecutive slots
+        // lane owns digits 8 lane .. 8 lane + 7; counts of all higher digits come from a suffix scan over lanes
+        uint32_t h[8], tot = 0;
+#pragma unroll
+        for (int b = 0; b < 8; ++b) {
+            h[b] = hist[lane * 8 + b];
+            tot += h[b];
+        }
+        uint32_t suf = tot;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t nb = __shfl_down_sync(0xffffffffu, suf, o);
+            if (lane + o < 32) suf += nb;
+        }
+        uint32_t gt = suf - tot, digit = 0, next_kk = 0;
+        bool found = false;
+#pragma unroll
+        for (int b = 7; b >= 0; --b) {
+            const uint32_t ge = gt + h[b];
+            if (gt < kk && kk <= ge) {
+                found = true;
+                digit = (uint32_t)(lane * 8 + b);
+                next_kk = kk - gt;
+            }
+            gt = ge;
+        }
+        const int src = __ffs(__ballot_sync(0xffffffffu, found)) - 1;  // exactly one lane, since 1 <= kk <= keys left
+        digit = __shfl_sync(0xffffffffu, digit, src);
+        kk = __shfl_sync(0xffffffffu, next_kk, src);
+        prefix = (prefix << 8) | digit;
+        __syncwarp();
+    }
+    const uint32_t res = prefix, need = kk;  // kk keys equal to the threshold are kept, lowest channels first
+    uint32_t run_gt = 0, run_eq = 0;
+    for (int base = 0; base < F; base += 32) {
+        const int j = base + lane;
+        const uint32_t key = j < F ? gate_key(g[j]) : 0u;
+        const bool isgt = j < F && key > res, iseq = j < F && key == res;
+        const uint32_t bg = __ballot_sync(0xffffffffu, isgt), be = __ballot_sync(0xffffffffu, iseq);
+        const uint32_t gt_b = run_gt + (uint32_t)__popc(bg & lt_mask), eq_b = run_eq + (uint32_t)__popc(be & lt_mask);
+        if (isgt || (iseq && eq_b < need)) kept[gt_b + min(eq_b, need)] = (uint32_t)j;
+        run_gt += (uint32_t)__popc(bg);
+        run_eq += (uint32_t)__popc(be);
+    }
+    __syncwarp();
+    return res;
+}
+
+template <int NV>
+__global__ void __launch_bounds__(kWarpSelMaxWarps * 32) select_mask_rows_warp_kernel(
+    const float *__restrict__ G, int ldg, __nv_bfloat16 *__restrict__ U, int ldu, int64_t rows, int F, int K,
+    int16_t *__restrict__ idx_out, __nv_bfloat16 *__restrict__ g_out, __nv_bfloat16 *__restrict__ u_out,
+    SelectMeta meta, int *status) {
+    extern __shared__ __align__(128) uint32_t warp_sel_smem[];
+    __shared__ float s_stat[kWarpSelMaxWarps][3];
+    __shared__ int s_abort;
+    const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5, wpc = blockDim.x >> 5;
+    uint32_t *base = warp_sel_smem + (size_t)wib * warp_select_words(NV, K);
+    float *sg = reinterpret_cast<float *>(base);                                // [NV * 128] gate row
+    __nv_bfloat16 *su = reinterpret_cast<__nv_bfloat16 *>(base + NV * 128);     // [NV * 128] up row -> Z' row
+    uint32_t *cand = base + NV * 128 + NV * 64;                                 // [slot][lane] parked values
+    uint32_t *bitmap = cand + kWarpSelCand;                                     // kept-channel bitmap
+    uint32_t *kept = bitmap + kWarpSelWords;                                    // [K] channel | z bits << 16
+    uint64_t *bar_mem = reinterpret_cast<uint64_t *>(kept + ((K + 3) & ~3));
+    const uint32_t bar = smem_u32(bar_mem);
+    const int64_t gw = (int64_t)blockIdx.x * wpc + wib, nw = (int64_t)gridDim.x * wpc;
+    const float b_center = meta.bracket[0], b_width = meta.bracket[1];
+    const bool have_bracket = meta.bracket[2] == kBracketTag && b_width > 0.f && fabsf(b_center) <= 3.0e38f;
+    float cen = b_center, wid = b_width;  // this warp's bracket
+    bool have = have_bracket;
+    float st_sum = 0.f, st_abs = 0.f, st_n = 0.f;
+    const int words = (F + 31) >> 5;
+    const uint32_t g_bytes = (uint32_t)ldg * 4u, u_bytes = (uint32_t)ldu * 2u;  // multiples of 16: ld % 8 == 0
+
+    if (threadIdx.x == 0) s_abort = 0;
+    if (lane == 0) mbar_init(bar, 1);
+    // channels the copies never write read as -inf for good
+    for (int c = ldg + lane; c < NV * 128; c += 32) sg[c] = -INFINITY;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    __syncthreads();
+    uint32_t phase = 0;
+    bool dead = false;
+
+    for (int64_t r = gw; r < rows && !dead; r += nw) {
+        const float *g = G + r * (int64_t)ldg;
+        __nv_bfloat16 *u = U + r * (int64_t)ldu;
+        // ---- stage the two rows (the previous row's store has to have read the up buffer first)
+        if (lane == 0) {
+            bulk_store_wait_read();
+            fence_async_smem();
+            mbar_expect_tx(bar, g_bytes + u_bytes);
+            bulk_copy_g2s(smem_u32(sg), g, g_bytes, bar);
+            bulk_copy_g2s(smem_u32(su), u, u_bytes, bar);
+        }
+        if (!__all_sync(0xffffffffu, mbar_wait(bar, phase, &s_abort, status))) {
+            dead = true;
+            break;
+        }
+        phase ^= 1u;
+        for (int c = F + lane; c < ldg; c += 32) sg[c] = -INFINITY;  // padding columns of this row
+        __syncwarp();
+
+        uint32_t tau = 0, res = 0;
+        bool fast = false, settled = false, no_cut = false;
+        float lo_f = cen - wid, hi_f = cen + wid;
+        for (int attempt = 0; have && attempt < 8; ++attempt) {
+            // ---- 1. classify: lane reads channels (v*32 + lane)*4 .. +3 of every 128-channel group v
+            uint32_t n_above = 0, n_mine = 0;
 #pragma unroll 4
+            for (int v = 0; v < NV; ++v) {
+                const float4 q = *reinterpret_cast<const float4 *>(sg + (v * 32 + lane) * 4);
+                const float e4[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float x = e4[e];
+                    n_above += x > hi_f ? 1u : 0u;
+                    const bool inside = x >= lo_f && x <= hi_f;
+                    if (inside) cand[min(n_mine, (uint32_t)kWarpSelSlots) * 32 + lane] = __float_as_uint(x);
+                    n_mine += inside ? 1u : 0u;
+                }
+            }
+            const uint32_t c_hi = __reduce_add_sync(0xffffffffu, n_above);
+            const uint32_t n_band = __reduce_add_sync(0xffffffffu, n_mine);
+            const uint32_t max_mine = __reduce_max_sync(0xffffffffu, n_mine);
+            if (max_mine > (uint32_t)kWarpSelSlots) {  // too many values inside: halve the bracket
+                const float c = 0.5f * (lo_f + hi_f), w = 0.25f * (hi_f - lo_f);
+                lo_f = c - w;
+                hi_f = c + w;
+                continue;
+            }
+            if (c_hi >= (uint32_t)K) {  // the threshold is above the bracket
+                const float w = hi_f - lo_f;
+                lo_f = hi_f;
+                hi_f += 2.f * w;
+                continue;
+            }
+            if (c_hi + n_band < (uint32_t)K) {  // ... below it
+                const float w = hi_f - lo_f;
+                hi_f = lo_f;
+                lo_f -= 2.f * w;
+                continue;
+            }
+            // ---- 2. the m-th largest parked key: a 64-bin histogram over the bracket's key range finds its
+            //         bin, the (few) keys of that bin are ranked against each other
+            const uint32_t lo_k = gate_key(lo_f), hi_k = gate_key(hi_f);
+            const uint32_t m = (uint32_t)K - c_hi;
+            uint32_t *hist = bitmap, *list = bitmap + 64, *list_n = bitmap + 96;
+            const uint32_t span = hi_k - lo_k;
+            const int shift = max(0, 26 - __clz(span | 1u));  // (span >> shift) < 64
+            hist[lane] = 0u;
+            hist[lane + 32] = 0u;
+            if (lane == 0) *list_n = 0u;
+            __syncwarp();
+            for (uint32_t s = 0; s < n_mine; ++s) {
+                const uint32_t key = gate_key(__uint_as_float(cand[s * 32 + lane]));
+                atomicAdd(&hist[(key - lo_k) >> shift], 1u);
+            }
+            __syncwarp();
+            const uint32_t h0 = hist[2 * lane], h1 = hist[2 * lane + 1], tot = h0 + h1;
+            uint32_t suf = tot;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t nb = __shfl_down_sync(0xffffffffu, suf, o);
+                if (lane + o < 32) suf += nb;
+            }
+            const uint32_t above = suf - tot;  // keys in bins above 2 lane + 1
+            const bool f1 = above < m && m <= above + h1, f0 = above + h1 < m && m <= above + tot;
+            const int src = __ffs(__ballot_sync(0xffffffffu, f0 || f1)) - 1;  // one lane: 1 <= m <= n_band
+            const uint32_t tbin = __shfl_sync(0xffffffffu, (uint32_t)(2 * lane + (f1 ? 1 : 0)), src);
+            const uint32_t m2 = m - __shfl_sync(0xffffffffu, f1 ? above : above + h1, src);
+            const uint32_t nbin = __shfl_sync(0xffffffffu, f1 ? h1 : h0, src);
+            if (nbin <= 32u) {
+                for (uint32_t s = 0; s < n_mine; ++s) {
+                    const uint32_t key = gate_key(__uint_as_float(cand[s * 32 + lane]));
+                    if (((key - lo_k) >> shift) == tbin) list[atomicAdd(list_n, 1u)] = key;
+                }
+                __syncwarp();
+                const uint32_t mykey = (uint32_t)lane < nbin ? list[lane] : 0u;
+                uint32_t n_gt = 0, n_eq = 0;
+                for (uint32_t i = 0; i < nbin; ++i) {
+                    const uint32_t o = list[i];
+                    n_gt += o > mykey ? 1u : 0u;
+                    n_eq += o == mykey ? 1u : 0u;
+                }
+                const bool is_tau = (uint32_t)lane < nbin && n_gt < m2 && m2 <= n_gt + n_eq;
+                const int tl = __ffs(__ballot_sync(0xffffffffu, is_tau)) - 1;
+                res = __shfl_sync(0xffffffffu, mykey, tl);
+                // no tie to cut iff every key equal to the threshold is kept
+                no_cut = __shfl_sync(0xffffffffu, n_gt + n_eq, tl) == m2;
+                settled = true;
+            }
+            break;
+        }
+        __syncwarp();
+        const float tau_f = key_to_float(res);
+        if (settled && no_cut && fabsf(tau_f) <= 3.0e38f) {
+            // ---- 3. kept set = {g >= tau}.  Four flags per group go to the shared bitmap (channel
+            //         (v*32 + lane)*4 + e is bit (lane & 7) * 4 + e of word v*4 + lane / 8)
+            for (int w = lane; w < words; w += 32) bitmap[w] = 0u;
+            __syncwarp();
+#pragma unroll 4
+            for (int v = 0; v < NV; ++v) {
+                const float4 q = *reinterpret_cast<const float4 *>(sg + (v * 32 + lane) * 4);
+                const uint32_t nib = (q.x >= tau_f ? 1u : 0u) | (q.y >= tau_f ? 2u : 0u) |
+                                     (q.z >= tau_f ? 4u : 0u) | (q.w >= tau_f ? 8u : 0u);
+                if (nib) atomicOr(&bitmap[v * 4 + (lane >> 3)], nib << ((lane & 7) * 4));
+            }
+            __syncwarp();
+            // enumerate in ascending channel order: lane l owns words [l*wpl, (l+1)*wpl)
+            const int wpl = (words + 31) >> 5;
+            uint32_t mine = 0;
+            for (int i = 0; i < wpl; ++i) {
+                const int w = lane * wpl + i;
+                mine += w < words ? (uint32_t)__popc(bitmap[w]) : 0u;
+            }
+            uint32_t pre = mine;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t nb = __shfl_up_sync(0xffffffffu, pre, o);
+                if (lane >= o) pre += nb;
+            }
+            if (__shfl_sync(0xffffffffu, pre, 31) == (uint32_t)K) {  // counts and compares agree
+                uint32_t pos = pre - mine;
+                for (int i = 0; i < wpl; ++i) {
+                    const int w = lane * wpl + i;
+                    uint32_t bits = w < words ? bitmap[w] : 0u;
+                    while (bits) {
+                        const int b = __ffs(bits) - 1;
+                        bits &= bits - 1u;
+                        kept[pos++] = (uint32_t)(w * 32 + b);
+                    }
+                }
+                tau = res;
+                fast = true;
+            }
+        }
+        __syncwarp();
+        if (!fast) tau = warp_select_row_general(sg, F, K, cand, kept);
+        __syncwarp();
+        // ---- 4. values of the kept channels (shared-memory gathers); the compact outputs are written with
+        //         consecutive lanes on consecutive slots
         for (int i = lane; i < K; i += 32) {
-            const uint32_t j = packed_j[i];
-            const float gv = key_to_float(packed[i]);
-            const __nv_bfloat16 ub = u[j];
-            const __nv_bfloat16 zb = __float2bfloat16_rn(silu_f(gv) * __bfloat162float(ub));
-            packed[i] = (uint32_t)(*reinterpret_cast<const uint16_t *>(&zb));
+            const uint32_t j = kept[i];
+            const float gval = sg[j];
+            const __nv_bfloat16 ub = su[j];
+            const __nv_bfloat16 zb = __float2bfloat16_rn(silu_f(gval) * __bfloat162float(ub));
+            kept[i] = j | ((uint32_t)(*reinterpret_cast<const uint16_t *>(&zb)) << 16);
             if (idx_out) {
                 idx_out[r * K + i] = (int16_t)j;
-                g_out[r * K + i] = __float2bfloat16_rn(gv);
+                g_out[r * K + i] = __float2bfloat16_rn(gval);
                 u_out[r * K + i] = ub;
             }
         }
         __syncwarp();
-        // ---- U row -> masked Z' in place
-        uint4 *row16 = reinterpret_cast<uint4 *>(u);
+        // ---- up row -> masked Z' row, in shared memory, then one bulk store
+        uint4 *row16 = reinterpret_cast<uint4 *>(su);
         for (int i = lane; i < (ldu >> 3); i += 32) row16[i] = make_uint4(0, 0, 0, 0);
         __syncwarp();
         for (int i = lane; i < K; i += 32) {
-            const uint16_t zb = (uint16_t)packed[i];
-            u[packed_j[i]] = *reinterpret_cast<const __nv_bfloat16 *>(&zb);
+            const uint32_t e = kept[i];
+            const uint16_t zb = (uint16_t)(e >> 16);
+            su[e & 0xffffu] = *reinterpret_cast<const __nv_bfloat16 *>(&zb);
         }
+        fence_async_smem();
         __syncwarp();
-        // ---- next row's bracket
+        if (lane == 0) bulk_copy_s2g(u, smem_u32(su), u_bytes);
+        // ---- statistics for the next launch's bracket
         const float t = key_to_float(tau);
-        if (!(fabsf(t) <= 3.0e38f)) {
-            guess.valid = false;
-        } else if (!guess.valid) {
-            guess.center = t;
-            guess.delta = 0.15f * fabsf(t) + 1e-30f;
-            guess.valid = true;
-        } else {
-            const float err = fabsf(t - guess.center);
-            guess.delta = solved ? 0.9f * guess.delta + 0.44f * err
-                                 : (overflow ? 0.5f * guess.delta : 2.0f * err + guess.delta);
-            guess.delta = fminf(fmaxf(guess.delta, 1e-30f), 1.0e37f);
-            guess.center = t;
+        if (fabsf(t) <= 3.0e38f) {
+            st_sum += t;
+            st_abs += have_bracket ? fabsf(t - b_center) : 0.f;
+            st_n += 1.f;
+            if (!have) {  // no bracket from an earlier launch: the warp makes its own from its first threshold
+                cen = t;
+                wid = 0.15f * fabsf(t) + 1e-30f;
+                have = true;
+            }
+        }
+    }
+    if (lane == 0) bulk_store_wait_all();
+    // ---- publish: per CTA one set of atomics; the last CTA turns the launch's statistics into the next bracket
+    if (lane == 0) {
+        s_stat[wib][0] = st_sum;
+        s_stat[wib][1] = st_abs;
+        s_stat[wib][2] = st_n;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float a = 0.f, b = 0.f, c = 0.f;
+        for (int w = 0; w < wpc; ++w) {
+            a += s_stat[w][0];
+            b += s_stat[w][1];
+            c += s_stat[w][2];
+        }
+        if (c > 0.f) {
+            atomicAdd(&meta.acc[0], a);
+            atomicAdd(&meta.acc[1], b);
+            atomicAdd(&meta.acc[2], c);
+        }
+        __threadfence();
+        if (atomicAdd(meta.done, 1u) == gridDim.x - 1) {
+            __threadfence();
+            const float sum = atomicAdd(&meta.acc[0], 0.f), dev = atomicAdd(&meta.acc[1], 0.f),
+                        n = atomicAdd(&meta.acc[2], 0.f);
+            if (n > 0.f) {
+                const float center = sum / n;
+                // five mean absolute deviations (about four standard deviations) once a center existed to
+                // measure them against; 15 % of the center otherwise; never narrower than 2 %
+                float width = have_bracket ? 5.0f * dev / n : 0.15f * fabsf(center);
+                width = fmaxf(width, 0.02f * fabsf(center) + 1e-30f);
+                meta.bracket[0] = center;
+                meta.bracket[1] = width;
+                meta.bracket[2] = kBracketTag;
+            } else {
+                meta.bracket[2] = 0.f;
+            }
+            meta.acc[0] = meta.acc[1] = meta.acc[2] = 0.f;
+            *meta.done = 0u;
         }
     }
 }
@@ -424,7 +629,7 @@ struct TcForwardLayout {
     int ldf;        // leading dimension of the dense [*, F] arrays (multiple of 8)
     size_t off_g;   // fp32 G of one chunk [chunk, ldf]
     size_t off_u;   // bf16 U, rewritten in place into Z', for ALL tokens [T, ldf]
-    size_t off_hint;  // two floats: threshold hint of the call (see select_hint_kernel)
+    size_t off_hint;  // bracket {center, width, tag}, statistics {sum, sum|dev|, rows}, CTA counter
     size_t total;
 };
 struct TcBackwardLayout {
