@@ -32,7 +32,10 @@ constexpr int THREADS = 192;
 constexpr uint32_t A_STAGE_BYTES = BM * BK * 2, B_STAGE_BYTES = BN * BK * 2;
 constexpr uint32_t STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
 constexpr uint32_t TMEM_COLS = ACC_STAGES * BN;  // 512
-constexpr size_t SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)STAGES * STAGE_BYTES + 256 /*barriers*/;
+// epilogue staging: per epilogue warp two 32-row x 128-byte boxes (128-byte swizzle atoms, 1024-byte aligned)
+constexpr uint32_t EPI_BOX_BYTES = 32 * 128, EPI_BUFS = 2, BAR_REGION_BYTES = 1024;
+constexpr size_t SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)STAGES * STAGE_BYTES + BAR_REGION_BYTES +
+                              4 * EPI_BUFS * EPI_BOX_BYTES;
 
 enum Epilogue : int {
     EPI_F32 = 0,       // C fp32 [M, ldc]
@@ -54,6 +57,8 @@ struct Params {
     // outputs
     void *c[3];          // per problem
     int ldc[3];
+    CUtensorMap c_map[3];  // per problem: [M, N] with 32-row boxes of 128 bytes (32 fp32 or 64 bf16 columns)
+    int direct_store;      // 1: the output cannot be described by a tensor map; threads store their rows
     int *status;
 };
 
@@ -103,6 +108,33 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
         "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
         ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y)
         : "memory");
+}
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, uint32_t src, int x, int y) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"(map), "r"(src),
+                 "r"(x), "r"(y)
+                 : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+// 1-D bulk copies: global -> shared (completes on an mbarrier) and shared -> global (bulk group of the thread)
+__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_copy_s2g(void *dst, uint32_t src, uint32_t bytes) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src), "r"(bytes)
+                 : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+// the issuing thread's bulk stores: all but the newest `Keep` groups have read their shared-memory source
+template <int Keep>
+__device__ __forceinline__ void bulk_store_wait_read() {
+    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(Keep) : "memory");
+}
+__device__ __forceinline__ void bulk_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap *map) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
@@ -213,6 +245,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_kernel(const __grid_constant_
     const uint32_t base = (raw + 1023u) & ~1023u;  // 128-byte swizzle atoms need 1024-byte alignment
     uint8_t *smem = smem_raw + (base - raw);
     const uint32_t bar_base = base + STAGES * STAGE_BYTES;
+    const uint32_t epi_base = bar_base + BAR_REGION_BYTES;
     auto full_bar = [&](int s) { return bar_base + 8u * s; };
     auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
     auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
@@ -347,7 +380,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_kernel(const __grid_constant_
     } else {
         // ------------------------------------------------------------------ epilogue (warps 2..5)
         const int quarter = warp & 3;  // TMEM lanes 32*quarter .. +31 are the ones this warp may read
-        int acc = 0;
+        int acc = 0, ebuf = 0;
         uint32_t acc_phase = 0;
         for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
             int m_blk, prob, n_blk;
@@ -360,29 +393,89 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_kernel(const __grid_constant_
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)acc * BN;
             const int n0 = n_blk * BN;
 
+            const bool f32_out = EPI == EPI_F32 || (EPI == EPI_GATE_UP && prob == 0);
+            const bool direct = p.direct_store != 0 || (EPI == EPI_BF16 && p.accumulate);
+            const int row0 = m_blk * BM + quarter * 32;  // first row of this warp's 32
+            if (direct) {
+                // ---- every thread stores its own row (outputs a tensor map cannot describe, accumulation)
 #pragma unroll 1
-            for (int c0 = 0; c0 < BN; c0 += 32) {
-                uint32_t r[32];
-                __syncwarp();
-                tmem_ld32(taddr + (uint32_t)c0, r);
-                tmem_ld_wait();
-                const int col = n0 + c0;
-                const int valid = p.N - col;  // columns of this chunk inside the problem
-                if (!row_ok || valid <= 0) continue;
-                if (EPI == EPI_F32 || (EPI == EPI_GATE_UP && prob == 0)) {
-                    float *dst = static_cast<float *>(p.c[prob]) + (int64_t)row * p.ldc[prob] + col;
-                    store_row_f32(dst, r, valid);
-                } else if (EPI == EPI_BF16 || EPI == EPI_GATE_UP) {
-                    __nv_bfloat16 *dst = static_cast<__nv_bfloat16 *>(p.c[prob]) + (int64_t)row * p.ldc[prob] + col;
-                    float v[32];
+                for (int c0 = 0; c0 < BN; c0 += 32) {
+                    uint32_t r[32];
+                    __syncwarp();
+                    tmem_ld32(taddr + (uint32_t)c0, r);
+                    tmem_ld_wait();
+                    const int col = n0 + c0;
+                    const int valid = p.N - col;  // columns of this chunk inside the problem
+                    if (!row_ok || valid <= 0) continue;
+                    if (f32_out) {
+                        float *dst = static_cast<float *>(p.c[prob]) + (int64_t)row * p.ldc[prob] + col;
+                        store_row_f32(dst, r, valid);
+                    } else {
+                        __nv_bfloat16 *dst =
+                            static_cast<__nv_bfloat16 *>(p.c[prob]) + (int64_t)row * p.ldc[prob] + col;
+                        float v[32];
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
-                    if (EPI == EPI_BF16 && p.accumulate) {
+                        for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+                        if (EPI == EPI_BF16 && p.accumulate) {
 #pragma unroll
-                        for (int i = 0; i < 32; ++i)
-                            if (i < valid) v[i] += __bfloat162float(dst[i]);
+                            for (int i = 0; i < 32; ++i)
+                                if (i < valid) v[i] += __bfloat162float(dst[i]);
+                        }
+                        store_row_bf16(dst, v, valid);
                     }
-                    store_row_bf16(dst, v, valid);
+                }
+            } else if (row0 < p.M) {
+                // ---- 32-row boxes of 128 bytes go through shared memory (thread = row, 16-byte pieces swizzled
+                //      the way the tensor map expects) and leave as bulk tensor stores, which clip at M and N
+                const uint32_t my_row = (uint32_t)lane * 128u, sw = (uint32_t)(lane & 7);
+                if (f32_out) {
+#pragma unroll 1
+                    for (int c0 = 0; c0 < BN && n0 + c0 < p.N; c0 += 32) {
+                        uint32_t r[32];
+                        __syncwarp();
+                        tmem_ld32(taddr + (uint32_t)c0, r);
+                        tmem_ld_wait();
+                        if (lane == 0) bulk_store_wait_read<EPI_BUFS - 1>();  // the box about to be refilled is free
+                        __syncwarp();
+                        const uint32_t box = epi_base + (uint32_t)(quarter * EPI_BUFS + ebuf) * EPI_BOX_BYTES;
+#pragma unroll
+                        for (int i = 0; i < 8; ++i)
+                            st_shared_v4(box + my_row + (((uint32_t)i ^ sw) << 4), r[4 * i], r[4 * i + 1], r[4 * i + 2],
+                                         r[4 * i + 3]);
+                        fence_async_smem();
+                        __syncwarp();
+                        if (lane == 0) tma_store_2d(&p.c_map[prob], box, n0 + c0, row0);
+                        ebuf ^= 1;
+                    }
+                } else {
+#pragma unroll 1
+                    for (int c0 = 0; c0 < BN && n0 + c0 < p.N; c0 += 64) {
+                        uint32_t r[32], q[32];
+                        __syncwarp();
+                        tmem_ld32(taddr + (uint32_t)c0, r);
+                        tmem_ld32(taddr + (uint32_t)c0 + 32u, q);
+                        tmem_ld_wait();
+                        if (lane == 0) bulk_store_wait_read<EPI_BUFS - 1>();
+                        __syncwarp();
+                        const uint32_t box = epi_base + (uint32_t)(quarter * EPI_BUFS + ebuf) * EPI_BOX_BYTES;
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            st_shared_v4(box + my_row + (((uint32_t)i ^ sw) << 4),
+                                         pack_bf16(__uint_as_float(r[8 * i]), __uint_as_float(r[8 * i + 1])),
+                                         pack_bf16(__uint_as_float(r[8 * i + 2]), __uint_as_float(r[8 * i + 3])),
+                                         pack_bf16(__uint_as_float(r[8 * i + 4]), __uint_as_float(r[8 * i + 5])),
+                                         pack_bf16(__uint_as_float(r[8 * i + 6]), __uint_as_float(r[8 * i + 7])));
+                            st_shared_v4(box + my_row + (((uint32_t)(i + 4) ^ sw) << 4),
+                                         pack_bf16(__uint_as_float(q[8 * i]), __uint_as_float(q[8 * i + 1])),
+                                         pack_bf16(__uint_as_float(q[8 * i + 2]), __uint_as_float(q[8 * i + 3])),
+                                         pack_bf16(__uint_as_float(q[8 * i + 4]), __uint_as_float(q[8 * i + 5])),
+                                         pack_bf16(__uint_as_float(q[8 * i + 6]), __uint_as_float(q[8 * i + 7])));
+                        }
+                        fence_async_smem();
+                        __syncwarp();
+                        if (lane == 0) tma_store_2d(&p.c_map[prob], box, n0 + c0, row0);
+                        ebuf ^= 1;
+                    }
                 }
             }
             tc_fence_before();
@@ -397,6 +490,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_kernel(const __grid_constant_
 
     // ---------------------------------------------------------------------- teardown
     __syncwarp();
+    if (warp >= 2 && lane == 0) bulk_store_wait_all();  // shared memory must outlive the stores that read it
     if (*abort_flag) {
         // give copies and MMAs still in flight time to land before shared memory and TMEM go away
         const long long t0 = clock64();

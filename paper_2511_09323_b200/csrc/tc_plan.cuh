@@ -73,8 +73,30 @@ inline void init_params(Params &p) {
     p.k_segments = 1;
 }
 
+// Output [rows, cols] with leading dimension ld as 32-row boxes of 128 bytes.  False when the tensor-map rules
+// (16-byte aligned base and row pitch) do not hold.
+inline bool make_out_map(CUtensorMap *m, void *ptr, int64_t rows, int64_t cols, int64_t ld, bool f32) {
+    EncodeTiledFn fn = encode_fn();
+    const size_t esz = f32 ? 4 : 2;
+    if (!fn || (reinterpret_cast<uintptr_t>(ptr) & 15u) || ((size_t)ld * esz) % 16 != 0 || rows <= 0 || cols <= 0)
+        return false;
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)ld * esz};
+    cuuint32_t box[2] = {(cuuint32_t)(128 / esz), 32};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(m, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, ptr, dims, strides, box,
+              estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 template <bool A_MN, bool B_MN, int EPI>
-inline int launch_gemm(const Params &p, cudaStream_t st) {
+inline int launch_gemm(const Params &p_in, cudaStream_t st) {
+    Params p = p_in;
+    p.direct_store = 0;
+    for (int i = 0; i < p.num_problems && !p.direct_store; ++i) {
+        const bool f32 = EPI == EPI_F32 || (EPI == EPI_GATE_UP && i == 0);
+        if (!make_out_map(&p.c_map[i], p.c[i], p.M, p.N, p.ldc[i], f32)) p.direct_store = 1;
+    }
     auto kern = gemm_kernel<A_MN, B_MN, EPI>;
     static bool configured = false;
     if (!configured) {
@@ -163,20 +185,6 @@ struct SelectMeta {
     float *acc;          // {sum of thresholds, sum of |threshold - center|, rows}: this launch's statistics
     unsigned int *done;  // CTAs finished
 };
-
-__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
-                 : "memory");
-}
-__device__ __forceinline__ void bulk_copy_s2g(void *dst, uint32_t src, uint32_t bytes) {
-    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src), "r"(bytes)
-                 : "memory");
-    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-}
-__device__ __forceinline__ void bulk_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
-__device__ __forceinline__ void bulk_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 // General exact path for one staged row: most-significant-digit radix selection with 8-bit digits.
 // g: the row in shared memory (ncols values, channels past the end hold -inf and are never counted because
@@ -283,7 +291,7 @@ __global__ void __launch_bounds__(kWarpSelMaxWarps * 32) select_mask_rows_warp_k
         __nv_bfloat16 *u = U + r * (int64_t)ldu;
         // ---- stage the two rows (the previous row's store has to have read the up buffer first)
         if (lane == 0) {
-            bulk_store_wait_read();
+            bulk_store_wait_read<0>();
             fence_async_smem();
             mbar_expect_tx(bar, g_bytes + u_bytes);
             bulk_copy_g2s(smem_u32(sg), g, g_bytes, bar);
