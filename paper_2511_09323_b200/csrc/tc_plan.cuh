@@ -632,6 +632,129 @@ __global__ void __launch_bounds__(256) backward_sample_rows_kernel(
 }
 
 // ------------------------------------------------------------------------------------------------
+// The same step with ONE WARP per token and the rows staged in the warp's slice of shared memory: the dZ
+// row arrives by a bulk copy (the next token's row is already in flight while this one is worked on), the
+// three masked rows are built in shared memory and leave as bulk stores.  Global traffic is fully
+// coalesced and the scattered accesses stay on chip.  Used when the four rows of a token fit a slice.
+__host__ __device__ constexpr size_t sample_warp_words(int ld, int K) {
+    return (size_t)2 * ld /* four bf16 rows */ + (size_t)2 * ((K + 1) & ~1) /* entries */ + 4 /* two mbarriers */;
+}
+constexpr int kSampleMaxWarps = 8;
+
+__global__ void __launch_bounds__(kSampleMaxWarps * 32) backward_sample_rows_warp_kernel(
+    const int16_t *__restrict__ idx, const __nv_bfloat16 *__restrict__ gval, const __nv_bfloat16 *__restrict__ uval,
+    int64_t T, int K, int F, int ld, __nv_bfloat16 *__restrict__ dz_z, __nv_bfloat16 *__restrict__ du,
+    __nv_bfloat16 *__restrict__ dg, int *__restrict__ status) {
+    extern __shared__ __align__(128) uint32_t sample_warp_smem[];
+    __shared__ int s_abort;
+    const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5, wpc = blockDim.x >> 5;
+    uint32_t *base = sample_warp_smem + (size_t)wib * sample_warp_words(ld, K);
+    const int row_words = ld >> 1;  // ld is a multiple of 8: rows are multiples of 16 bytes
+    __nv_bfloat16 *zbuf0 = reinterpret_cast<__nv_bfloat16 *>(base);  // two dZ rows, used alternately
+    __nv_bfloat16 *ubuf = reinterpret_cast<__nv_bfloat16 *>(base + 2 * row_words);
+    __nv_bfloat16 *gbuf = reinterpret_cast<__nv_bfloat16 *>(base + 3 * row_words);
+    uint32_t *entry = base + 4 * row_words;  // K x {j | z << 16, dU | dG << 16}
+    uint64_t *bar_mem = reinterpret_cast<uint64_t *>(entry + 2 * ((K + 1) & ~1));
+    const uint32_t bar0 = smem_u32(bar_mem);  // two mbarriers, 8 bytes apart
+    const uint32_t row_bytes = (uint32_t)ld * 2u;
+    const int64_t gw = (int64_t)blockIdx.x * wpc + wib, nw = (int64_t)gridDim.x * wpc;
+
+    if (threadIdx.x == 0) s_abort = 0;
+    if (lane == 0) {
+        mbar_init(bar0, 1);
+        mbar_init(bar0 + 8u, 1);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    __syncthreads();
+    uint32_t phases = 0;  // bit b: parity to wait for on barrier b
+    if (lane == 0 && gw < T) {
+        mbar_expect_tx(bar0, row_bytes);
+        bulk_copy_g2s(smem_u32(zbuf0), dz_z + gw * (int64_t)ld, row_bytes, bar0);
+    }
+    int b = 0;
+    for (int64_t t = gw; t < T; t += nw, b ^= 1) {
+        if (!__all_sync(0xffffffffu, mbar_wait(bar0 + 8u * (uint32_t)b, (phases >> b) & 1u, &s_abort, status))) break;
+        phases ^= 1u << b;
+        __nv_bfloat16 *zr = zbuf0 + (size_t)b * ld;
+        for (int k0 = 0; k0 < K; k0 += 256) {
+            // eight saved entries per lane, their loads issued together
+            int jv[8];
+            __nv_bfloat16 gb[8], ub[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int k = k0 + i * 32 + lane;
+                jv[i] = -1;
+                if (k < K) {
+                    jv[i] = idx[t * K + k];
+                    gb[i] = gval[t * K + k];
+                    ub[i] = uval[t * K + k];
+                }
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int k = k0 + i * 32 + lane;
+                if (k >= K) continue;
+                const int j = jv[i];
+                uint32_t w0 = 0xffffu, w1 = 0;  // j = 0xffff marks a skipped entry
+                if (j >= 0 && j < F) {
+                    const float dz = __bfloat162float(zr[j]);
+                    const float g = __bfloat162float(gb[i]);
+                    const float u = __bfloat162float(ub[i]);
+                    const float s = silu_f(g);
+                    const __nv_bfloat16 zb = __float2bfloat16_rn(s * u);
+                    w0 = (uint32_t)j | ((uint32_t)(*reinterpret_cast<const uint16_t *>(&zb)) << 16);
+                    w1 = pack_bf16(s * dz, u * dz * dsilu_f(g));
+                } else {
+                    raise_status(status, MOC_ERR_BAD_INDEX);
+                }
+                entry[2 * k] = w0;
+                entry[2 * k + 1] = w1;
+            }
+        }
+        // by now the stores of the previous token have read their rows: the other dZ buffer (next token's row goes
+        // there) and the dU / dG rows are free
+        if (lane == 0) {
+            bulk_store_wait_read<0>();
+            fence_async_smem();
+            if (t + nw < T) {
+                const uint32_t nbar = bar0 + 8u * (uint32_t)(b ^ 1);
+                mbar_expect_tx(nbar, row_bytes);
+                bulk_copy_g2s(smem_u32(zbuf0 + (size_t)(b ^ 1) * ld), dz_z + (t + nw) * (int64_t)ld, row_bytes, nbar);
+            }
+        }
+        __syncwarp();
+        {
+            uint4 *z16 = reinterpret_cast<uint4 *>(zr), *u16 = reinterpret_cast<uint4 *>(ubuf),
+                  *g16 = reinterpret_cast<uint4 *>(gbuf);
+            const uint4 zero = make_uint4(0, 0, 0, 0);
+            for (int v = lane; v < (ld >> 3); v += 32) {
+                z16[v] = zero;
+                u16[v] = zero;
+                g16[v] = zero;
+            }
+        }
+        __syncwarp();
+        for (int k = lane; k < K; k += 32) {
+            const uint32_t w0 = entry[2 * k], w1 = entry[2 * k + 1];
+            const uint32_t j = w0 & 0xffffu;
+            if (j == 0xffffu) continue;
+            const uint16_t zb = (uint16_t)(w0 >> 16), ub = (uint16_t)(w1 & 0xffffu), gb = (uint16_t)(w1 >> 16);
+            zr[j] = *reinterpret_cast<const __nv_bfloat16 *>(&zb);
+            ubuf[j] = *reinterpret_cast<const __nv_bfloat16 *>(&ub);
+            gbuf[j] = *reinterpret_cast<const __nv_bfloat16 *>(&gb);
+        }
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+            bulk_copy_s2g(dz_z + t * (int64_t)ld, smem_u32(zr), row_bytes);
+            bulk_copy_s2g(du + t * (int64_t)ld, smem_u32(ubuf), row_bytes);
+            bulk_copy_s2g(dg + t * (int64_t)ld, smem_u32(gbuf), row_bytes);
+        }
+    }
+    if (lane == 0) bulk_store_wait_all();
+}
+
+// ------------------------------------------------------------------------------------------------
 struct TcForwardLayout {
     int64_t chunk;  // tokens per gate/up pass
     int ldf;        // leading dimension of the dense [*, F] arrays (multiple of 8)
