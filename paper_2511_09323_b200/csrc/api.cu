@@ -316,23 +316,27 @@ int forward_tc(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat1
     const int64_t T = d.tokens;
     const int f_tiles = ceil_div(F, BN);
 
-    // selector: one warp per token while a row fits in registers (F <= 4096), else one CTA per token
-    const int nv = F <= 1024 ? 8 : (F <= 2048 ? 16 : (F <= 4096 ? 32 : 0));
+    // selector: one warp per token while at least four warps' rows fit an SM's shared memory, else one CTA per token
+    const int nv = ceil_div(F, 128);  // 128-channel groups of a row
     // each warp stages its token's rows in its own slice of shared memory: as many warps per SM as fit, in one
     // or two CTAs
-    const size_t warp_bytes = nv ? warp_select_words(nv, K) * sizeof(uint32_t) : 0;
-    const int warps_per_sm = nv ? (int)std::min<size_t>((size_t)220 * 1024 / warp_bytes, 2 * kWarpSelMaxWarps) : 0;
-    const int sel_ctas_per_sm = warps_per_sm > 4 ? 2 : 1;
+    const size_t warp_bytes = warp_select_words(nv, K) * sizeof(uint32_t);
+    const int warps_per_sm = (int)std::min<size_t>((size_t)220 * 1024 / warp_bytes, 2 * kWarpSelMaxWarps);
+    const int sel_ctas_per_sm = warps_per_sm > kWarpSelMaxWarps ? 2 : 1;
     const int sel_wpc = warps_per_sm / sel_ctas_per_sm;
     const size_t warp_smem = (size_t)sel_wpc * warp_bytes;
     const size_t cta_smem = ((size_t)F + K) * sizeof(uint32_t);
-    const bool warp_select = nv != 0 && sel_wpc >= 1;
+    const bool warp_select = warps_per_sm >= 4;
     float *hint = reinterpret_cast<float *>(ws + L.off_hint);
     int rc = MOC_OK;
     if (warp_select) {
-        if (nv == 8) rc = set_smem(select_mask_rows_warp_kernel<8>, warp_smem, 2048);
-        if (nv == 16) rc = set_smem(select_mask_rows_warp_kernel<16>, warp_smem, 2048);
-        if (nv == 32) rc = set_smem(select_mask_rows_warp_kernel<32>, warp_smem, 2048);
+        switch (nv) {
+            case 8: rc = set_smem(select_mask_rows_warp_kernel<8>, warp_smem, 2048); break;
+            case 16: rc = set_smem(select_mask_rows_warp_kernel<16>, warp_smem, 2048); break;
+            case 32: rc = set_smem(select_mask_rows_warp_kernel<32>, warp_smem, 2048); break;
+            case 43: rc = set_smem(select_mask_rows_warp_kernel<43>, warp_smem, 2048); break;
+            default: rc = set_smem(select_mask_rows_warp_kernel<0>, warp_smem, 2048); break;
+        }
     } else {
         rc = set_smem(select_mask_rows_kernel, cta_smem);
     }
@@ -341,13 +345,13 @@ int forward_tc(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat1
     // Warp selector: every launch works with one bracket kept in the workspace ({center, width, tag} at
     // hint[0..2]); it gathers the statistics of its thresholds (hint[4..6], CTA counter at hint[8]) and its last
     // CTA rewrites the bracket for the next launch.  The bracket is only a hint: a stale or garbage one costs
-    // time (rows take the slow exact path), never correctness.  The statistics are cleared per call.
+    // time (rows take the general exact path), never correctness; the statistics and the counter reset themselves
+    // at the end of every launch.
     SelectMeta meta{};
     if (warp_select) {
         meta.bracket = hint;
         meta.acc = hint + 4;
         meta.done = reinterpret_cast<unsigned int *>(hint + 8);
-        if (cudaMemsetAsync(hint + 4, 0, 32, st) != cudaSuccess) return MOC_ERR_CUDA;
     }
 
     int *status = device_status_ptr();
@@ -383,18 +387,18 @@ int forward_tc(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat1
         if (warp_select) {
             const unsigned grid =
                 (unsigned)std::min<int64_t>((n + sel_wpc - 1) / sel_wpc, (int64_t)sm_count() * sel_ctas_per_sm);
-            if (nv == 8)
-                MOC_LAUNCH(KID_TC_SELECT_MASK, st,
-                           (select_mask_rows_warp_kernel<8><<<grid, sel_wpc * 32, warp_smem, st>>>(G, L.ldf, Uc, L.ldf, n, F, K,
-                                                                                           o_idx, o_g, o_u, meta, status)));
-            else if (nv == 16)
-                MOC_LAUNCH(KID_TC_SELECT_MASK, st,
-                           (select_mask_rows_warp_kernel<16><<<grid, sel_wpc * 32, warp_smem, st>>>(G, L.ldf, Uc, L.ldf, n, F, K,
-                                                                                            o_idx, o_g, o_u, meta, status)));
-            else
-                MOC_LAUNCH(KID_TC_SELECT_MASK, st,
-                           (select_mask_rows_warp_kernel<32><<<grid, sel_wpc * 32, warp_smem, st>>>(G, L.ldf, Uc, L.ldf, n, F, K,
-                                                                                            o_idx, o_g, o_u, meta, status)));
+#define MOC_WARP_SELECT(NV)                                                                    \
+    MOC_LAUNCH(KID_TC_SELECT_MASK, st,                                                         \
+               (select_mask_rows_warp_kernel<NV><<<grid, sel_wpc * 32, warp_smem, st>>>(       \
+                   G, L.ldf, Uc, L.ldf, n, F, nv, K, o_idx, o_g, o_u, meta, status)))
+            switch (nv) {  // the usual row lengths get their loops unrolled
+                case 8: MOC_WARP_SELECT(8); break;
+                case 16: MOC_WARP_SELECT(16); break;
+                case 32: MOC_WARP_SELECT(32); break;
+                case 43: MOC_WARP_SELECT(43); break;
+                default: MOC_WARP_SELECT(0); break;
+            }
+#undef MOC_WARP_SELECT
         } else {
             const unsigned grid = (unsigned)std::min<int64_t>(n, (int64_t)sm_count() * 6);
             MOC_LAUNCH(KID_TC_SELECT_MASK, st,

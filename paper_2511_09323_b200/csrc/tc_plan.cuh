@@ -146,7 +146,8 @@ __global__ void __launch_bounds__(kSelectThreads) select_hint_kernel(const float
 }
 
 // ------------------------------------------------------------------------------------------------
-// Forward selector for rows of at most NV * 128 channels: ONE WARP per token, no block barriers.
+// Forward selector for rows that fit a warp's slice of shared memory: ONE WARP per token, no block barriers.
+// nv = number of 128-channel groups of a row.
 // Same outputs as the CTA-per-token kernel below.
 //
 // Every warp owns a slice of shared memory into which lane 0 bulk-copies the token's gate row (fp32) and up
@@ -169,15 +170,25 @@ __global__ void __launch_bounds__(kSelectThreads) select_hint_kernel(const float
 // Rows for which 1-3 do not apply (no bracket yet, too many parked keys, ties to cut, non-finite
 // threshold, inconsistent counts) take the general exact path (8-bit radix selection over the
 // staged row).  Either way the result is exact: indices ascending, ties to the lower channel.
-constexpr int kWarpSelSlots = 14;                        // parked keys per lane
-constexpr int kWarpSelCand = (kWarpSelSlots + 1) * 32;   // one more row absorbs the overflow of a column
-constexpr int kWarpSelWords = 128;                       // bitmap words (4096 channels)
+// Parked values per lane: 14 for rows of up to 2048 channels, growing with the square root of the row length
+// (the spread of a row's threshold shrinks with the square root, so the values inside the bracket grow likewise).
+__host__ __device__ constexpr int warp_select_slots(int nv) {
+    int s = 14;
+    while (s * s * 16 < 196 * nv) ++s;  // s >= 14 sqrt(nv / 16)
+    return s;
+}
+__host__ __device__ constexpr int warp_select_cand_words(int nv) {
+    return (warp_select_slots(nv) + 1) * 32;  // one more row absorbs the overflow of a column (>= 256: histogram)
+}
+constexpr int kWarpSelWords = 128;                       // bitmap words, at least (also scratch of the search)
 constexpr float kBracketTag = 20251109.0f;
 constexpr int kWarpSelMaxWarps = 8;                      // warps per CTA, at most
 
 // Words of shared memory one warp needs: gate row, up row, parked keys, bitmap, kept list, mbarrier.
+__host__ __device__ constexpr int warp_select_bitmap_words(int nv) { return nv * 4 > kWarpSelWords ? nv * 4 : kWarpSelWords; }
 __host__ __device__ constexpr size_t warp_select_words(int nv, int K) {
-    return (size_t)nv * 128 + (size_t)nv * 64 + kWarpSelCand + kWarpSelWords + (size_t)((K + 3) & ~3) + 4;
+    return (size_t)nv * 128 + (size_t)nv * 64 + warp_select_cand_words(nv) + warp_select_bitmap_words(nv) +
+           (size_t)((K + 3) & ~3) + 4;
 }
 
 struct SelectMeta {
@@ -251,21 +262,23 @@ __device__ __noinline__ uint32_t warp_select_row_general(const float *g, int F, 
     return res;
 }
 
-template <int NV>
+template <int NV>  // number of 128-channel groups when known at compile time, 0: taken from nv_runtime
 __global__ void __launch_bounds__(kWarpSelMaxWarps * 32) select_mask_rows_warp_kernel(
-    const float *__restrict__ G, int ldg, __nv_bfloat16 *__restrict__ U, int ldu, int64_t rows, int F, int K,
+    const float *__restrict__ G, int ldg, __nv_bfloat16 *__restrict__ U, int ldu, int64_t rows, int F, int nv_runtime, int K,
     int16_t *__restrict__ idx_out, __nv_bfloat16 *__restrict__ g_out, __nv_bfloat16 *__restrict__ u_out,
     SelectMeta meta, int *status) {
     extern __shared__ __align__(128) uint32_t warp_sel_smem[];
     __shared__ float s_stat[kWarpSelMaxWarps][3];
     __shared__ int s_abort;
+    const int nv = NV > 0 ? NV : nv_runtime;
+    const int slots = warp_select_slots(nv);
     const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5, wpc = blockDim.x >> 5;
-    uint32_t *base = warp_sel_smem + (size_t)wib * warp_select_words(NV, K);
-    float *sg = reinterpret_cast<float *>(base);                                // [NV * 128] gate row
-    __nv_bfloat16 *su = reinterpret_cast<__nv_bfloat16 *>(base + NV * 128);     // [NV * 128] up row -> Z' row
-    uint32_t *cand = base + NV * 128 + NV * 64;                                 // [slot][lane] parked values
-    uint32_t *bitmap = cand + kWarpSelCand;                                     // kept-channel bitmap
-    uint32_t *kept = bitmap + kWarpSelWords;                                    // [K] channel | z bits << 16
+    uint32_t *base = warp_sel_smem + (size_t)wib * warp_select_words(nv, K);
+    float *sg = reinterpret_cast<float *>(base);                                // [nv * 128] gate row
+    __nv_bfloat16 *su = reinterpret_cast<__nv_bfloat16 *>(base + nv * 128);     // [nv * 128] up row -> Z' row
+    uint32_t *cand = base + nv * 128 + nv * 64;                                 // [slot][lane] parked values
+    uint32_t *bitmap = cand + warp_select_cand_words(nv);                                     // kept-channel bitmap
+    uint32_t *kept = bitmap + warp_select_bitmap_words(nv);                                    // [K] channel | z bits << 16
     uint64_t *bar_mem = reinterpret_cast<uint64_t *>(kept + ((K + 3) & ~3));
     const uint32_t bar = smem_u32(bar_mem);
     const int64_t gw = (int64_t)blockIdx.x * wpc + wib, nw = (int64_t)gridDim.x * wpc;
@@ -280,7 +293,7 @@ __global__ void __launch_bounds__(kWarpSelMaxWarps * 32) select_mask_rows_warp_k
     if (threadIdx.x == 0) s_abort = 0;
     if (lane == 0) mbar_init(bar, 1);
     // channels the copies never write read as -inf for good
-    for (int c = ldg + lane; c < NV * 128; c += 32) sg[c] = -INFINITY;
+    for (int c = ldg + lane; c < nv * 128; c += 32) sg[c] = -INFINITY;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     __syncthreads();
     uint32_t phase = 0;
@@ -312,7 +325,7 @@ __global__ void __launch_bounds__(kWarpSelMaxWarps * 32) select_mask_rows_warp_k
             // ---- 1. classify: lane reads channels (v*32 + lane)*4 .. +3 of every 128-channel group v
             uint32_t n_above = 0, n_mine = 0;
 #pragma unroll 4
-            for (int v = 0; v < NV; ++v) {
+            for (int v = 0; v < nv; ++v) {
                 const float4 q = *reinterpret_cast<const float4 *>(sg + (v * 32 + lane) * 4);
                 const float e4[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
@@ -320,14 +333,14 @@ __global__ void __launch_bounds__(kWarpSelMaxWarps * 32) select_mask_rows_warp_k
                     const float x = e4[e];
                     n_above += x > hi_f ? 1u : 0u;
                     const bool inside = x >= lo_f && x <= hi_f;
-                    if (inside) cand[min(n_mine, (uint32_t)kWarpSelSlots) * 32 + lane] = __float_as_uint(x);
+                    if (inside) cand[min(n_mine, (uint32_t)slots) * 32 + lane] = __float_as_uint(x);
                     n_mine += inside ? 1u : 0u;
                 }
             }
             const uint32_t c_hi = __reduce_add_sync(0xffffffffu, n_above);
             const uint32_t n_band = __reduce_add_sync(0xffffffffu, n_mine);
             const uint32_t max_mine = __reduce_max_sync(0xffffffffu, n_mine);
-            if (max_mine > (uint32_t)kWarpSelSlots) {  // too many values inside: halve the bracket
+            if (max_mine > (uint32_t)slots) {  // too many values inside: halve the bracket
                 const float c = 0.5f * (lo_f + hi_f), w = 0.25f * (hi_f - lo_f);
                 lo_f = c - w;
                 hi_f = c + w;
@@ -404,7 +417,7 @@ __global__ void __launch_bounds__(kWarpSelMaxWarps * 32) select_mask_rows_warp_k
             for (int w = lane; w < words; w += 32) bitmap[w] = 0u;
             __syncwarp();
 #pragma unroll 4
-            for (int v = 0; v < NV; ++v) {
+            for (int v = 0; v < nv; ++v) {
                 const float4 q = *reinterpret_cast<const float4 *>(sg + (v * 32 + lane) * 4);
                 const uint32_t nib = (q.x >= tau_f ? 1u : 0u) | (q.y >= tau_f ? 2u : 0u) |
                                      (q.z >= tau_f ? 4u : 0u) | (q.w >= tau_f ? 8u : 0u);
@@ -503,7 +516,8 @@ __global__ void __launch_bounds__(kWarpSelMaxWarps * 32) select_mask_rows_warp_k
             atomicAdd(&meta.acc[2], c);
         }
         __threadfence();
-        if (atomicAdd(meta.done, 1u) == gridDim.x - 1) {
+        // wrapping counter: back at zero after the last CTA, whatever it held when the workspace was new
+        if (atomicInc(meta.done, gridDim.x - 1) == gridDim.x - 1) {
             __threadfence();
             const float sum = atomicAdd(&meta.acc[0], 0.f), dev = atomicAdd(&meta.acc[1], 0.f),
                         n = atomicAdd(&meta.acc[2], 0.f);
@@ -520,7 +534,6 @@ __global__ void __launch_bounds__(kWarpSelMaxWarps * 32) select_mask_rows_warp_k
                 meta.bracket[2] = 0.f;
             }
             meta.acc[0] = meta.acc[1] = meta.acc[2] = 0.f;
-            *meta.done = 0u;
         }
     }
 }
