@@ -358,7 +358,7 @@ int forward_tc(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat1
     if (!status) return MOC_ERR_CUDA;
     Params p;
     init_params(p);
-    if (!map_k_major(&p.b_map[0], wg, F, dm, dm, BN) || !map_k_major(&p.b_map[1], wu, F, dm, dm, BN))
+    if (!map_k_major(&p.b_map[0], wg, F, dm, dm, b_box_rows()) || !map_k_major(&p.b_map[1], wu, F, dm, dm, b_box_rows()))
         return MOC_ERR_CUDA;
     p.status = status;
     p.num_problems = 2;
@@ -443,7 +443,7 @@ int backward_tc(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat
     {
         Params p;
         init_params(p);
-        if (!map_k_major(&p.a_map[0], dout, T, dm, dm, BM) || !map_k_major(&p.b_map[0], wd, F, dm, dm, BN))
+        if (!map_k_major(&p.a_map[0], dout, T, dm, dm, BM) || !map_k_major(&p.b_map[0], wd, F, dm, dm, b_box_rows()))
             return MOC_ERR_CUDA;
         p.k_blocks = ceil_div(dm, BK);
         p.M = (int)T;
@@ -502,6 +502,8 @@ int backward_tc(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat
         p.m_tiles = ceil_div(d.d_ff_ld, BM);
         p.n_tiles = ceil_div(dm, BN);
         p.accumulate = (d.flags & MOC_FLAG_ACCUMULATE_WGRAD) ? 1 : 0;
+        // long contraction, few tiles: the finer tile granularity of single CTAs fills the last wave better
+        p.single_cta = 1;
         p.status = status;
         MOC_LAUNCH(KID_TC_WGRAD_GEMM, st, (rc = launch_gemm<true, true, EPI_BF16>(p, st)));
         if (rc != MOC_OK) return rc;
@@ -787,7 +789,7 @@ int moc_tc_gemm_bf16(int64_t m, int64_t n, int64_t k, const void *a, int a_mn_ma
     Params p;
     init_params(p);
     const bool ok_a = a_mn_major ? map_mn_major(&p.a_map[0], a, k, m, lda) : map_k_major(&p.a_map[0], a, m, k, lda, BM);
-    const bool ok_b = b_mn_major ? map_mn_major(&p.b_map[0], b, k, n, ldb) : map_k_major(&p.b_map[0], b, n, k, ldb, BN);
+    const bool ok_b = b_mn_major ? map_mn_major(&p.b_map[0], b, k, n, ldb) : map_k_major(&p.b_map[0], b, n, k, ldb, b_box_rows());
     if (!ok_a || !ok_b) return MOC_ERR_CUDA;
     p.k_blocks = ceil_div(k, BK);
     p.M = (int)m;

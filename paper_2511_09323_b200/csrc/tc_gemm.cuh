@@ -59,6 +59,7 @@ struct Params {
     int ldc[3];
     CUtensorMap c_map[3];  // per problem: [M, N] with 32-row boxes of 128 bytes (32 fp32 or 64 bf16 columns)
     int direct_store;      // 1: the output cannot be described by a tensor map; threads store their rows
+    int single_cta;        // 1: one CTA per tile even where CTA pairs are available (set by the caller)
     int *status;
 };
 
@@ -167,6 +168,59 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
                  : "memory");
 }
 
+// ---- CTA pairs (cta_group::2): one MMA spans the tensor cores, shared memory and TMEM of two CTAs of a cluster
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// shared::cluster address of the same shared-memory location in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// tile load whose completion bytes are counted by an mbarrier of the pair's leading CTA (no multicast: every CTA
+// fetches its own boxes)
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, uint32_t leader_bar, int x, int y) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(leader_bar), "r"(x), "r"(y)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t dst_smem, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols)
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                               uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// arrives (once the MMAs issued so far have completed) on the barrier at this shared-memory offset in both CTAs
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+    asm volatile(
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar),
+        "h"((uint16_t)3)
+        : "memory");
+}
+
 // 32 consecutive fp32 columns of this thread's TMEM lane
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
     asm volatile(
@@ -197,12 +251,12 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr, uint32_t 
     return d;
 }
 
-template <bool A_MN, bool B_MN>
+template <bool A_MN, bool B_MN, int M_INSTR = BM>
 __device__ __forceinline__ constexpr uint32_t make_idesc() {
     return (1u << 4)                        // D format: fp32
            | (1u << 7) | (1u << 10)         // A, B format: bf16
            | ((A_MN ? 1u : 0u) << 15) | ((B_MN ? 1u : 0u) << 16)
-           | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+           | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(M_INSTR >> 4) << 24);
 }
 
 // ---------------------------------------------------------------------------------------------- epilogue helpers
@@ -234,6 +288,102 @@ __device__ __forceinline__ void store_row_bf16(__nv_bfloat16 *dst, const float (
 #pragma unroll
         for (int i = 0; i < 32; ++i)
             if (i < valid) dst[i] = __float2bfloat16_rn(v[i]);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------- epilogue
+// One warp moves its 32 rows x BN columns of a finished accumulator (TMEM lanes of the warp, columns at taddr) to
+// the output of problem `prob`: rows row0.., columns n0...  warp_boxes: the warp's EPI_BUFS staging boxes.
+template <int EPI>
+__device__ __forceinline__ void epilogue_tile(const Params &p, int prob, int row0, int n0, uint32_t taddr,
+                                              uint32_t warp_boxes, int &ebuf) {
+    const int lane = threadIdx.x & 31;
+    const int row = row0 + lane;
+    const bool row_ok = row < p.M;
+
+    const bool f32_out = EPI == EPI_F32 || (EPI == EPI_GATE_UP && prob == 0);
+    const bool direct = p.direct_store != 0 || (EPI == EPI_BF16 && p.accumulate);
+    if (direct) {
+        // ---- every thread stores its own row (outputs a tensor map cannot describe, accumulation)
+#pragma unroll 1
+        for (int c0 = 0; c0 < BN; c0 += 32) {
+            uint32_t r[32];
+            __syncwarp();
+            tmem_ld32(taddr + (uint32_t)c0, r);
+            tmem_ld_wait();
+            const int col = n0 + c0;
+            const int valid = p.N - col;  // columns of this chunk inside the problem
+            if (!row_ok || valid <= 0) continue;
+            if (f32_out) {
+                float *dst = static_cast<float *>(p.c[prob]) + (int64_t)row * p.ldc[prob] + col;
+                store_row_f32(dst, r, valid);
+            } else {
+                __nv_bfloat16 *dst =
+                    static_cast<__nv_bfloat16 *>(p.c[prob]) + (int64_t)row * p.ldc[prob] + col;
+                float v[32];
+#pragma unroll
+                for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+                if (EPI == EPI_BF16 && p.accumulate) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        if (i < valid) v[i] += __bfloat162float(dst[i]);
+                }
+                store_row_bf16(dst, v, valid);
+            }
+        }
+    } else if (row0 < p.M) {
+        // ---- 32-row boxes of 128 bytes go through shared memory (thread = row, 16-byte pieces swizzled
+        //      the way the tensor map expects) and leave as bulk tensor stores, which clip at M and N
+        const uint32_t my_row = (uint32_t)lane * 128u, sw = (uint32_t)(lane & 7);
+        if (f32_out) {
+#pragma unroll 1
+            for (int c0 = 0; c0 < BN && n0 + c0 < p.N; c0 += 32) {
+                uint32_t r[32];
+                __syncwarp();
+                tmem_ld32(taddr + (uint32_t)c0, r);
+                tmem_ld_wait();
+                if (lane == 0) bulk_store_wait_read<EPI_BUFS - 1>();  // the box about to be refilled is free
+                __syncwarp();
+                const uint32_t box = warp_boxes + (uint32_t)ebuf * EPI_BOX_BYTES;
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    st_shared_v4(box + my_row + (((uint32_t)i ^ sw) << 4), r[4 * i], r[4 * i + 1], r[4 * i + 2],
+                                 r[4 * i + 3]);
+                fence_async_smem();
+                __syncwarp();
+                if (lane == 0) tma_store_2d(&p.c_map[prob], box, n0 + c0, row0);
+                ebuf ^= 1;
+            }
+        } else {
+#pragma unroll 1
+            for (int c0 = 0; c0 < BN && n0 + c0 < p.N; c0 += 64) {
+                uint32_t r[32], q[32];
+                __syncwarp();
+                tmem_ld32(taddr + (uint32_t)c0, r);
+                tmem_ld32(taddr + (uint32_t)c0 + 32u, q);
+                tmem_ld_wait();
+                if (lane == 0) bulk_store_wait_read<EPI_BUFS - 1>();
+                __syncwarp();
+                const uint32_t box = warp_boxes + (uint32_t)ebuf * EPI_BOX_BYTES;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    st_shared_v4(box + my_row + (((uint32_t)i ^ sw) << 4),
+                                 pack_bf16(__uint_as_float(r[8 * i]), __uint_as_float(r[8 * i + 1])),
+                                 pack_bf16(__uint_as_float(r[8 * i + 2]), __uint_as_float(r[8 * i + 3])),
+                                 pack_bf16(__uint_as_float(r[8 * i + 4]), __uint_as_float(r[8 * i + 5])),
+                                 pack_bf16(__uint_as_float(r[8 * i + 6]), __uint_as_float(r[8 * i + 7])));
+                    st_shared_v4(box + my_row + (((uint32_t)(i + 4) ^ sw) << 4),
+                                 pack_bf16(__uint_as_float(q[8 * i]), __uint_as_float(q[8 * i + 1])),
+                                 pack_bf16(__uint_as_float(q[8 * i + 2]), __uint_as_float(q[8 * i + 3])),
+                                 pack_bf16(__uint_as_float(q[8 * i + 4]), __uint_as_float(q[8 * i + 5])),
+                                 pack_bf16(__uint_as_float(q[8 * i + 6]), __uint_as_float(q[8 * i + 7])));
+                }
+                fence_async_smem();
+                __syncwarp();
+                if (lane == 0) tma_store_2d(&p.c_map[prob], box, n0 + c0, row0);
+                ebuf ^= 1;
+            }
+        }
     }
 }
 
@@ -388,96 +538,9 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_kernel(const __grid_constant_
             // the whole warp must agree: the TMEM loads below are warp-collective
             if (!__all_sync(0xffffffffu, mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.status))) break;
             tc_fence_after();
-            const int row = m_blk * BM + quarter * 32 + lane;
-            const bool row_ok = row < p.M;
-            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)acc * BN;
-            const int n0 = n_blk * BN;
-
-            const bool f32_out = EPI == EPI_F32 || (EPI == EPI_GATE_UP && prob == 0);
-            const bool direct = p.direct_store != 0 || (EPI == EPI_BF16 && p.accumulate);
-            const int row0 = m_blk * BM + quarter * 32;  // first row of this warp's 32
-            if (direct) {
-                // ---- every thread stores its own row (outputs a tensor map cannot describe, accumulation)
-#pragma unroll 1
-                for (int c0 = 0; c0 < BN; c0 += 32) {
-                    uint32_t r[32];
-                    __syncwarp();
-                    tmem_ld32(taddr + (uint32_t)c0, r);
-                    tmem_ld_wait();
-                    const int col = n0 + c0;
-                    const int valid = p.N - col;  // columns of this chunk inside the problem
-                    if (!row_ok || valid <= 0) continue;
-                    if (f32_out) {
-                        float *dst = static_cast<float *>(p.c[prob]) + (int64_t)row * p.ldc[prob] + col;
-                        store_row_f32(dst, r, valid);
-                    } else {
-                        __nv_bfloat16 *dst =
-                            static_cast<__nv_bfloat16 *>(p.c[prob]) + (int64_t)row * p.ldc[prob] + col;
-                        float v[32];
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
-                        if (EPI == EPI_BF16 && p.accumulate) {
-#pragma unroll
-                            for (int i = 0; i < 32; ++i)
-                                if (i < valid) v[i] += __bfloat162float(dst[i]);
-                        }
-                        store_row_bf16(dst, v, valid);
-                    }
-                }
-            } else if (row0 < p.M) {
-                // ---- 32-row boxes of 128 bytes go through shared memory (thread = row, 16-byte pieces swizzled
-                //      the way the tensor map expects) and leave as bulk tensor stores, which clip at M and N
-                const uint32_t my_row = (uint32_t)lane * 128u, sw = (uint32_t)(lane & 7);
-                if (f32_out) {
-#pragma unroll 1
-                    for (int c0 = 0; c0 < BN && n0 + c0 < p.N; c0 += 32) {
-                        uint32_t r[32];
-                        __syncwarp();
-                        tmem_ld32(taddr + (uint32_t)c0, r);
-                        tmem_ld_wait();
-                        if (lane == 0) bulk_store_wait_read<EPI_BUFS - 1>();  // the box about to be refilled is free
-                        __syncwarp();
-                        const uint32_t box = epi_base + (uint32_t)(quarter * EPI_BUFS + ebuf) * EPI_BOX_BYTES;
-#pragma unroll
-                        for (int i = 0; i < 8; ++i)
-                            st_shared_v4(box + my_row + (((uint32_t)i ^ sw) << 4), r[4 * i], r[4 * i + 1], r[4 * i + 2],
-                                         r[4 * i + 3]);
-                        fence_async_smem();
-                        __syncwarp();
-                        if (lane == 0) tma_store_2d(&p.c_map[prob], box, n0 + c0, row0);
-                        ebuf ^= 1;
-                    }
-                } else {
-#pragma unroll 1
-                    for (int c0 = 0; c0 < BN && n0 + c0 < p.N; c0 += 64) {
-                        uint32_t r[32], q[32];
-                        __syncwarp();
-                        tmem_ld32(taddr + (uint32_t)c0, r);
-                        tmem_ld32(taddr + (uint32_t)c0 + 32u, q);
-                        tmem_ld_wait();
-                        if (lane == 0) bulk_store_wait_read<EPI_BUFS - 1>();
-                        __syncwarp();
-                        const uint32_t box = epi_base + (uint32_t)(quarter * EPI_BUFS + ebuf) * EPI_BOX_BYTES;
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            st_shared_v4(box + my_row + (((uint32_t)i ^ sw) << 4),
-                                         pack_bf16(__uint_as_float(r[8 * i]), __uint_as_float(r[8 * i + 1])),
-                                         pack_bf16(__uint_as_float(r[8 * i + 2]), __uint_as_float(r[8 * i + 3])),
-                                         pack_bf16(__uint_as_float(r[8 * i + 4]), __uint_as_float(r[8 * i + 5])),
-                                         pack_bf16(__uint_as_float(r[8 * i + 6]), __uint_as_float(r[8 * i + 7])));
-                            st_shared_v4(box + my_row + (((uint32_t)(i + 4) ^ sw) << 4),
-                                         pack_bf16(__uint_as_float(q[8 * i]), __uint_as_float(q[8 * i + 1])),
-                                         pack_bf16(__uint_as_float(q[8 * i + 2]), __uint_as_float(q[8 * i + 3])),
-                                         pack_bf16(__uint_as_float(q[8 * i + 4]), __uint_as_float(q[8 * i + 5])),
-                                         pack_bf16(__uint_as_float(q[8 * i + 6]), __uint_as_float(q[8 * i + 7])));
-                        }
-                        fence_async_smem();
-                        __syncwarp();
-                        if (lane == 0) tma_store_2d(&p.c_map[prob], box, n0 + c0, row0);
-                        ebuf ^= 1;
-                    }
-                }
-            }
+            epilogue_tile<EPI>(p, prob, m_blk * BM + quarter * 32, n_blk * BN,
+                               tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)acc * BN,
+                               epi_base + (uint32_t)quarter * EPI_BUFS * EPI_BOX_BYTES, ebuf);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(tempty_bar(acc));
@@ -501,6 +564,201 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_kernel(const __grid_constant_
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+
+// ---------------------------------------------------------------------------------------------- pair kernel
+// The same GEMM with the CTAs working in pairs (clusters of two, `cta_group::2`): a pair owns a 256 x 256 output
+// tile; each CTA stages its own 128 rows of A and HALF of the B tile (128 of the 256 columns), and one
+// `tcgen05.mma.cta_group::2` issued by the pair's leading CTA multiplies both A halves with both B halves, each
+// CTA's TMEM receiving its 128 rows.  Per CTA and k-block that is 32 KiB of operands instead of 48 KiB: a third
+// less traffic from L2 and a six-deep ring in the same shared memory.
+//   full[s]   (leader's)  : counts the bytes both CTAs' loads bring in for stage s
+//   empty[s]  (each CTA's): the leader's commit arrives on it in both CTAs when the MMAs have read stage s
+//   tfull[a]  (each CTA's): ... when accumulator a is complete
+//   tempty[a] (leader's)  : the eight epilogue warps of the pair arrive when they have drained accumulator a
+constexpr int PAIR_STAGES = 6;
+constexpr uint32_t PAIR_B_STAGE_BYTES = (BN / 2) * BK * 2, PAIR_STAGE_BYTES = A_STAGE_BYTES + PAIR_B_STAGE_BYTES;
+static_assert(PAIR_STAGES * PAIR_STAGE_BYTES == STAGES * STAGE_BYTES, "both kernels use the same shared-memory layout");
+
+template <bool A_MN, bool B_MN, int EPI>
+__global__ void __launch_bounds__(THREADS, 1) gemm_pair_kernel(const __grid_constant__ Params p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;  // 128-byte swizzle atoms need 1024-byte alignment
+    uint8_t *smem = smem_raw + (base - raw);
+    const uint32_t bar_base = base + PAIR_STAGES * PAIR_STAGE_BYTES;
+    const uint32_t epi_base = bar_base + BAR_REGION_BYTES;
+    auto full_bar = [&](int s) { return bar_base + 8u * s; };
+    auto empty_bar = [&](int s) { return bar_base + 8u * (PAIR_STAGES + s); };
+    auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * PAIR_STAGES + a); };
+    auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * PAIR_STAGES + ACC_STAGES + a); };
+    volatile uint32_t *tmem_holder = reinterpret_cast<volatile uint32_t *>(
+        smem + PAIR_STAGES * PAIR_STAGE_BYTES + 8 * (2 * PAIR_STAGES + 2 * ACC_STAGES));
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_holder + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();  // 0: the pair's leading CTA
+    const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
+    const int m_pairs = (p.m_tiles + 1) >> 1;  // 256-row blocks
+    const int total_tiles = m_pairs * p.n_tiles * p.num_problems;
+    const int kb_total = p.k_blocks * p.k_segments;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < PAIR_STAGES; ++s) {
+            mbar_init(full_bar(s), 1);
+            mbar_init(empty_bar(s), 1);
+        }
+        for (int a = 0; a < ACC_STAGES; ++a) {
+            mbar_init(tfull_bar(a), 1);
+            mbar_init(tempty_bar(a), 8);  // one arrival per epilogue warp of the pair
+        }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        tmem_alloc_pair(smem_u32(const_cast<uint32_t *>(tmem_holder)), TMEM_COLS);
+        tmem_relinquish_pair();
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();  // the partner's barriers exist before anything signals them
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_holder;
+
+    auto decode_tile = [&](int tile, int &m_blk, int &prob, int &n_blk) {
+        const int per_m = p.num_problems * p.n_tiles;
+        m_blk = tile / per_m;
+        const int r = tile - m_blk * per_m;
+        prob = r / p.n_tiles;
+        n_blk = r - prob * p.n_tiles;
+    };
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer (one per CTA)
+        if (lane == 0) {
+            for (int i = 0; i < 3; ++i) {
+                prefetch_tmap(&p.a_map[i]);
+                prefetch_tmap(&p.b_map[i]);
+            }
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int tile = pair; tile < total_tiles && ok; tile += num_pairs) {
+                int m_blk, prob, n_blk;
+                decode_tile(tile, m_blk, prob, n_blk);
+                const int m0 = m_blk * (2 * BM) + (int)rank * BM;          // this CTA's rows of A
+                const int nb0 = n_blk * BN + (int)rank * (BN / 2);         // this CTA's half of the B tile
+                for (int kb = 0; kb < kb_total; ++kb) {
+                    if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status)) {
+                        ok = false;
+                        break;
+                    }
+                    const int seg = kb / p.k_blocks, kk = (kb - seg * p.k_blocks) * BK;
+                    const CUtensorMap *am = &p.a_map[p.a_idx[prob][seg]];
+                    const CUtensorMap *bm = &p.b_map[p.b_idx[prob][seg]];
+                    const uint32_t sa = base + stage * PAIR_STAGE_BYTES, sb = sa + A_STAGE_BYTES;
+                    const uint32_t lead_full = map_to_cta(full_bar(stage), 0);
+                    if (rank == 0) mbar_expect_tx(full_bar(stage), 2 * PAIR_STAGE_BYTES);
+                    if (A_MN) {
+#pragma unroll
+                        for (int i = 0; i < BM / 64; ++i)
+                            tma_load_2d_pair(sa + i * (64 * BK * 2), am, lead_full, m0 + i * 64, kk);
+                    } else {
+                        tma_load_2d_pair(sa, am, lead_full, kk, m0);
+                    }
+                    if (B_MN) {
+#pragma unroll
+                        for (int i = 0; i < BN / 128; ++i)
+                            tma_load_2d_pair(sb + i * (64 * BK * 2), bm, lead_full, nb0 + i * 64, kk);
+                    } else {
+                        tma_load_2d_pair(sb, bm, lead_full, kk, nb0);
+                    }
+                    if (++stage == PAIR_STAGES) {
+                        stage = 0;
+                        phase ^= 1u;
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer (leading CTA only)
+        if (lane == 0 && rank == 0) {
+            constexpr uint32_t idesc = make_idesc<A_MN, B_MN, 2 * BM>();
+            int stage = 0, acc = 0;
+            uint32_t phase = 0, acc_phase = 0;
+            bool ok = true;
+            for (int tile = pair; tile < total_tiles && ok; tile += num_pairs) {
+                if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, p.status)) break;
+                tc_fence_after();
+                const uint32_t tmem_d = tmem_base + (uint32_t)acc * BN;
+                for (int kb = 0; kb < kb_total; ++kb) {
+                    if (!mbar_wait(full_bar(stage), phase, abort_flag, p.status)) {
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint32_t sa = base + stage * PAIR_STAGE_BYTES, sb = sa + A_STAGE_BYTES;
+#pragma unroll
+                    for (int k = 0; k < BK / 16; ++k) {
+                        const uint64_t ad = A_MN ? make_smem_desc(sa + k * 2048, BK * 128, 1024)
+                                                 : make_smem_desc(sa + k * 32, 16, 1024);
+                        const uint64_t bd = B_MN ? make_smem_desc(sb + k * 2048, BK * 128, 1024)
+                                                 : make_smem_desc(sb + k * 32, 16, 1024);
+                        umma_bf16_pair(tmem_d, ad, bd, idesc, (kb | k) != 0 ? 1u : 0u);
+                    }
+                    umma_commit_pair(empty_bar(stage));  // frees the stage in both CTAs
+                    if (++stage == PAIR_STAGES) {
+                        stage = 0;
+                        phase ^= 1u;
+                    }
+                }
+                if (!ok) break;
+                umma_commit_pair(tfull_bar(acc));  // accumulator complete, in both CTAs
+                if (++acc == ACC_STAGES) {
+                    acc = 0;
+                    acc_phase ^= 1u;
+                }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue (warps 2..5 of each CTA)
+        const int quarter = warp & 3;
+        int acc = 0, ebuf = 0;
+        uint32_t acc_phase = 0;
+        for (int tile = pair; tile < total_tiles; tile += num_pairs) {
+            int m_blk, prob, n_blk;
+            decode_tile(tile, m_blk, prob, n_blk);
+            if (!__all_sync(0xffffffffu, mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.status))) break;
+            tc_fence_after();
+            epilogue_tile<EPI>(p, prob, m_blk * (2 * BM) + (int)rank * BM + quarter * 32, n_blk * BN,
+                               tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)acc * BN,
+                               epi_base + (uint32_t)quarter * EPI_BUFS * EPI_BOX_BYTES, ebuf);
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(map_to_cta(tempty_bar(acc), 0));
+            if (++acc == ACC_STAGES) {
+                acc = 0;
+                acc_phase ^= 1u;
+            }
+        }
+    }
+
+    // ---------------------------------------------------------------------- teardown
+    __syncwarp();
+    if (warp >= 2 && lane == 0) bulk_store_wait_all();  // shared memory must outlive the stores that read it
+    if (*abort_flag) {
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000LL) __nanosleep(1000);
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();  // neither CTA leaves while the partner may still read its shared memory or signal it
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc_pair(tmem_base, TMEM_COLS);
     }
 }
 

@@ -8,6 +8,8 @@
 #pragma once
 
 #include <cuda.h>
+#include <cstdlib>
+#include <cstring>
 #include <cuda_runtime.h>
 
 #include "moc_common.cuh"
@@ -57,6 +59,19 @@ inline bool map_mn_major(CUtensorMap *m, const void *ptr, int64_t k, int64_t mn,
     return make_map(m, ptr, k, mn, ld, 64, BK);
 }
 
+// CTA pairs (clusters of two, one MMA across both) are the default; MOC_FFN_GEMM=single in the environment selects
+// the one-CTA kernel (kept for comparison and for devices that refuse the cluster launch).
+inline bool pair_mode() {
+    static int mode = -1;
+    if (mode < 0) {
+        const char *e = getenv("MOC_FFN_GEMM");
+        mode = (e && strcmp(e, "single") == 0) ? 0 : 1;
+    }
+    return mode == 1;
+}
+// rows of a K-major B box: a CTA of a pair stages half of the 256 B rows of a tile
+inline int b_box_rows() { return pair_mode() ? BN / 2 : BN; }
+
 inline int sm_count() {
     static int n = 0;
     if (!n) {
@@ -96,6 +111,34 @@ inline int launch_gemm(const Params &p_in, cudaStream_t st) {
     for (int i = 0; i < p.num_problems && !p.direct_store; ++i) {
         const bool f32 = EPI == EPI_F32 || (EPI == EPI_GATE_UP && i == 0);
         if (!make_out_map(&p.c_map[i], p.c[i], p.M, p.N, p.ldc[i], f32)) p.direct_store = 1;
+    }
+    if (pair_mode() && !(p.single_cta && A_MN && B_MN)) {  // K-major B boxes are sized for the mode: no choice there
+        auto kern = gemm_pair_kernel<A_MN, B_MN, EPI>;
+        cudaLaunchConfig_t cfg = {};
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.blockDim = dim3(THREADS);
+        cfg.dynamicSmemBytes = SMEM_BYTES;
+        cfg.stream = st;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        static int max_pairs = 0;  // pairs that can be resident at once
+        if (!max_pairs) {
+            if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES) != cudaSuccess)
+                return MOC_ERR_CUDA;
+            cfg.gridDim = dim3(2 * (unsigned)sm_count());
+            int n = 0;
+            if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess || n <= 0) return MOC_ERR_CUDA;
+            max_pairs = n;
+        }
+        const int tiles = ((p.m_tiles + 1) / 2) * p.n_tiles * p.num_problems;
+        const int pairs = tiles < max_pairs ? tiles : max_pairs;
+        if (pairs <= 0) return MOC_OK;
+        cfg.gridDim = dim3(2 * (unsigned)pairs);
+        return cudaLaunchKernelEx(&cfg, kern, p) == cudaSuccess ? MOC_OK : MOC_ERR_CUDA;
     }
     auto kern = gemm_kernel<A_MN, B_MN, EPI>;
     static bool configured = false;
