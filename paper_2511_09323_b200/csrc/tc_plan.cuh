@@ -834,7 +834,13 @@ inline TcForwardLayout tc_forward_layout(const moc_ffn_desc &d) {
     // stay in L2: LLaMA-130M shapes 0.109 -> 0.087 ms for the GEMM and 0.114 -> 0.091 ms for the selector.)
     const size_t per_token = (size_t)L.ldf * 6;
     const int64_t all_m = (d.tokens + BM - 1) / BM;
-    int64_t hi = std::max<int64_t>(1, (int64_t)(((size_t)1280 << 20) / per_token) / BM);
+    // MOC_FFN_FWD_CHUNK_MIB in the environment overrides the bound (smaller workspace, more launches)
+    size_t bound_mib = 1280;
+    if (const char *e = getenv("MOC_FFN_FWD_CHUNK_MIB")) {
+        const long v = atol(e);
+        if (v >= 1 && v <= (1 << 20)) bound_mib = (size_t)v;
+    }
+    int64_t hi = std::max<int64_t>(1, (int64_t)((bound_mib << 20) / per_token) / BM);
     hi = std::min(hi, all_m);
     const int64_t n_chunks = (all_m + hi - 1) / hi;
     const int64_t best = (all_m + n_chunks - 1) / n_chunks;  // equal chunks

@@ -279,10 +279,19 @@ def test_decode_small_shapes(dtype, T, d, F, K):
 @pytest.mark.parametrize("T,d,F,F_ld,K", [
     (513, 264, 1100, 1104, 137),   # d not a multiple of 64, F not a multiple of 256, ragged token tile
     (256, 128, 96, 96, 96),        # K = F: dense SwiGLU through the tensor-core plan
-    (384, 512, 4500, 4504, 563),   # more than 4096 channels: CTA-per-token selector
+    (384, 512, 4500, 4504, 563),   # more than 4096 channels: few warps per SM in the warp-per-token selector
+    (300, 128, 9000, 9000, 700),   # rows too long for a warp's shared-memory slice: CTA-per-token selector
 ])
 def test_tc_plan_shapes(T, d, F, F_ld, K):
     w = syn.Workload(f"tc-{T}-{d}-{F}-{K}", "bf16", T, d, F, F_ld, K, seed=200 + T)
+    _run_forward_backward(w)
+
+
+def test_tc_plan_forward_in_several_token_chunks(monkeypatch):
+    """A 1 MiB bound on the transient gate array makes the forward run its GEMM + selector over five token chunks
+    (the last one ragged); results must not depend on the chunking."""
+    monkeypatch.setenv("MOC_FFN_FWD_CHUNK_MIB", "1")
+    w = syn.Workload("tc-chunked", "bf16", 513, 264, 1100, 1104, 137, seed=713)
     _run_forward_backward(w)
 
 
