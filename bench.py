@@ -33,6 +33,12 @@ METRIC = "moc_ffn_fwd_bwd_tokens_per_s"
 UNIT = "tokens/s"
 ALU_FP32_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12   # 148 SMs x 128 FMA lanes x 2 flop x max SM clock
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of each kernel of the step on the default C2 workload, from one
+# `ncu --set full` capture of this program (profiles/tensor_core_plan_kernels_C2.md); reported as `roofline.traffic`
+NCU_DRAM_BYTES_C2 = {
+    "tc_gate_up_gemm": 176.2e6, "tc_select_mask": 257.3e6, "tc_down_gemm": 75.0e6, "tc_bwd_sample": 234.3e6,
+    "tc_dz_gemm": 42.9e6, "tc_wgrad_gemm": 255.2e6, "tc_dx_gemm": 158.9e6,
+}
 
 
 def parse_args():
@@ -439,7 +445,9 @@ def roofline_report(prof, steps, T, w, e, peaks):
         roof["frac"] = roof["achieved"] / roof["peak"]
         roof["peak_source"] = peaks["source"] if bound != "alu" else "derived: 148 SM x 128 lanes x 2 x 1.965 GHz"
         roof["algorithmic_per_launch"] = per_launch
-    roof["traffic"] = None
+    # measured DRAM bytes per launch exist for the default workload only (one launch of each kernel per step there)
+    at_default = w.name == syn.C2.name and T == syn.C2.tokens and n == steps
+    roof["traffic"] = NCU_DRAM_BYTES_C2.get(top) if at_default else None
     return roof, kernels
 
 
