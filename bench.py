@@ -446,7 +446,7 @@ def roofline_report(prof, steps, T, w, e, peaks):
         roof["peak_source"] = peaks["source"] if bound != "alu" else "derived: 148 SM x 128 lanes x 2 x 1.965 GHz"
         roof["algorithmic_per_launch"] = per_launch
     # measured DRAM bytes per launch exist for the default workload only (one launch of each kernel per step there)
-    at_default = w.name == syn.C2.name and T == syn.C2.tokens and n == steps
+    at_default = w.name.startswith("C2-") and T == 64 * 256 and n == steps
     roof["traffic"] = NCU_DRAM_BYTES_C2.get(top) if at_default else None
     return roof, kernels
 

@@ -554,7 +554,7 @@ DecodeLayout decode_layout(const moc_ffn_desc &d) {
     L.off_list = c.take((size_t)d.d_ff * sizeof(uint16_t));
     L.off_count = c.take(sizeof(int));
     L.off_acc = c.take((size_t)d.tokens * d.d_model * sizeof(float));
-    L.off_cnt = c.take((size_t)L.slices * sizeof(int));
+    L.off_cnt = c.take((size_t)(L.slices + 1) * sizeof(int));  // + arrivals of the select kernel
     L.total = c.off;
     return L;
 }
@@ -589,7 +589,7 @@ int decode_bf16(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat
                (dec::gemv_rows_kernel<false><<<L.gemv_grid, dec::kGemvThreads, dec::kGemvSmem, st>>>(
                    x, wg, T, dm, F, ws, L.slices, status)));
     if ((rc = launch_ok()) != MOC_OK) return rc;
-    MOC_LAUNCH(KID_DEC_SELECT, st, (dec::select_mask_kernel<<<T, dec::kSelThreads, sel_smem, st>>>(ws, F, K)));
+    MOC_LAUNCH(KID_DEC_SELECT, st, (dec::select_mask_kernel<<<T, dec::kSelThreads, sel_smem, st>>>(ws, F, K, ws.counters + L.slices)));
     if ((rc = launch_ok()) != MOC_OK) return rc;
     MOC_LAUNCH(KID_DEC_UP, st,
                (dec::gemv_rows_kernel<true><<<L.gemv_grid, dec::kGemvThreads, dec::kGemvSmem, st>>>(

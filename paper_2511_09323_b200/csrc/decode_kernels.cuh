@@ -84,79 +84,15 @@ __global__ void __launch_bounds__(kGemvThreads, 2) gemv_rows_kernel(const __nv_b
     extern __shared__ __align__(128) uint8_t gsm[];
     __shared__ uint64_t bars[2 * kGemvStages];
     __shared__ int s_abort;
-    __shared__ int s_scan[(kSelectMaxN / kGemvThreads + 2) * 9 + 1];  // (chunk, warp) counts of used channels
     __shared__ uint16_t s_rows[kGemvMaxRows];                          // this CTA's rows when gathering
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    int n = F;
-    uint32_t used_bits[4] = {0u, 0u, 0u, 0u};  // bit c: this thread's channel of chunk c is used
-    if (GATHER) {
-        // Every CTA derives the list of used channels (ascending) from the masks: per (chunk, warp) counts,
-        // one scan, then each used channel knows its list position.  A CTA keeps the positions of its own
-        // share; CTA 0 also writes the whole list for the down kernel.
-        const int chunks = (F + kGemvThreads - 1) / kGemvThreads;  // <= 114
-        // masks are fetched in groups of 16 independent loads; the "used" flags stay in registers
-        for (int c0 = 0; c0 < chunks; c0 += 16) {
-            uint32_t m[16];
-#pragma unroll
-            for (int u = 0; u < 16; ++u) {
-                const int j = (c0 + u) * kGemvThreads + tid;
-                m[u] = (c0 + u < chunks && j < F) ? ws.chmask[j] : 0u;
-            }
-#pragma unroll
-            for (int u = 0; u < 16; ++u) {
-                if (c0 + u < chunks) {
-                    const uint32_t b = __ballot_sync(0xffffffffu, m[u] != 0u);
-                    if (lane == 0) s_scan[(c0 + u) * 9 + warp] = __popc(b);
-                    if (m[u] != 0u) used_bits[(c0 + u) >> 5] |= 1u << ((c0 + u) & 31);
-                }
-            }
-        }
-        __syncthreads();
-        // exclusive scan in (chunk, warp) order: thread c scans chunk c's 9 counts, the chunk totals are
-        // scanned across the block (chunks <= 114 < threads)
-        __shared__ int s_wsum[9];
-        int ctot = 0;
-        if (tid < chunks)
-            for (int i = 0; i < 9; ++i) ctot += s_scan[tid * 9 + i];
-        int inc = ctot;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int v = __shfl_up_sync(0xffffffffu, inc, o);
-            if (lane >= o) inc += v;
-        }
-        if (lane == 31) s_wsum[warp] = inc;
-        __syncthreads();
-        int before = inc - ctot;
-        for (int wi = 0; wi < warp; ++wi) before += s_wsum[wi];
-        if (tid < chunks) {
-            int run = before;
-            for (int i = 0; i < 9; ++i) {
-                const int v = s_scan[tid * 9 + i];
-                s_scan[tid * 9 + i] = run;
-                run += v;
-            }
-            if (tid == chunks - 1) s_scan[chunks * 9] = run;
-        }
-        __syncthreads();
-        n = s_scan[chunks * 9];
-    }
+    // gathering: the used channels (ascending) were listed by the select kernel
+    const int n = GATHER ? min(*ws.list_count, F) : F;
     const int r0 = (int)(((int64_t)blockIdx.x * n) / gridDim.x);
     const int r1 = (int)(((int64_t)(blockIdx.x + 1) * n) / gridDim.x);
     const int tiles = (r1 - r0 + 7) >> 3;
-    if (GATHER) {
-        const int chunks = (F + kGemvThreads - 1) / kGemvThreads;
-        for (int c = 0; c < chunks; ++c) {
-            const int j = c * kGemvThreads + tid;
-            const bool used = (used_bits[c >> 5] >> (c & 31)) & 1u;
-            const uint32_t b = __ballot_sync(0xffffffffu, used);
-            if (used) {
-                const int pos = s_scan[c * 9 + warp] + __popc(b & ((1u << lane) - 1u));
-                if (pos >= r0 && pos < r1 && pos - r0 < kGemvMaxRows) s_rows[pos - r0] = (uint16_t)j;
-                if (blockIdx.x == 0) ws.list[pos] = (uint16_t)j;
-            }
-        }
-        if (blockIdx.x == 0 && tid == 0) *ws.list_count = n;
-    }
+    if (GATHER)
+        for (int i = tid; i < r1 - r0 && i < kGemvMaxRows; i += kGemvThreads) s_rows[i] = ws.list[r0 + i];
     const int nkc = (d + kGemvChunk - 1) / kGemvChunk;
     const uint32_t ring = tc::smem_u32(gsm);
     auto full_bar = [&](int s) { return tc::smem_u32(&bars[s]); };
@@ -168,7 +104,7 @@ __global__ void __launch_bounds__(kGemvThreads, 2) gemv_rows_kernel(const __nv_b
         for (int64_t i = (int64_t)blockIdx.x * kGemvThreads + tid; i < (int64_t)T * d;
              i += (int64_t)gridDim.x * kGemvThreads)
             ws.out_acc[i] = 0.f;
-        if (blockIdx.x == 0 && tid < slices) ws.counters[tid] = 0;
+        if (blockIdx.x == 0 && tid <= slices) ws.counters[tid] = 0;  // [slices]: arrivals of the select kernel
     }
     // When the last chunk of a row is short, the bytes it leaves untouched are multiplied by zero x entries and
     // must therefore be finite: the ring then starts out as zeros.  (Rows of a partial tile that are never
@@ -193,18 +129,20 @@ __global__ void __launch_bounds__(kGemvThreads, 2) gemv_rows_kernel(const __nv_b
         int stage = 0;
         uint32_t phase = 0;
         bool ok = true;
-        for (int tile = 0; tile < tiles && ok; ++tile) {
-            const int slot = r0 + tile * 8 + lane;  // lanes 0..7 own one row each
-            const bool valid = lane < 8 && slot < r1;
-            const int row = valid ? (GATHER ? (int)s_rows[slot - r0] : slot) : 0;
-            const int nvalid = min(8, r1 - (r0 + tile * 8));
-            for (int kc = 0; kc < nkc; ++kc) {
+        // stages go chunk by chunk of the contraction index, all the CTA's row tiles within a chunk (the
+        // consumers keep a chunk's x fragments in registers across the tiles)
+        for (int kc = 0; kc < nkc && ok; ++kc) {
+            const int k0 = kc * kGemvChunk;
+            const uint32_t bytes = (uint32_t)min(kGemvChunk, d - k0) * 2;
+            for (int tile = 0; tile < tiles; ++tile) {
+                const int slot = r0 + tile * 8 + lane;  // lanes 0..7 own one row each
+                const bool valid = lane < 8 && slot < r1;
+                const int row = valid ? (GATHER ? (int)s_rows[slot - r0] : slot) : 0;
+                const int nvalid = min(8, r1 - (r0 + tile * 8));
                 if (!__all_sync(0xffffffffu, tc::mbar_wait(empty_bar(stage), phase ^ 1u, &s_abort, status))) {
                     ok = false;
                     break;
                 }
-                const int k0 = kc * kGemvChunk;
-                const uint32_t bytes = (uint32_t)min(kGemvChunk, d - k0) * 2;
                 if (lane == 0) tc::mbar_expect_tx(full_bar(stage), bytes * (uint32_t)nvalid);
                 __syncwarp();
                 if (valid)
@@ -230,21 +168,21 @@ __global__ void __launch_bounds__(kGemvThreads, 2) gemv_rows_kernel(const __nv_b
         float acc[kGemvMaxTiles][4];
 #pragma unroll
         for (int ti = 0; ti < kGemvMaxTiles; ++ti) acc[ti][0] = acc[ti][1] = acc[ti][2] = acc[ti][3] = 0.f;
+        for (int kc = 0; kc < nkc && ok; ++kc) {
+            // this warp's 64 contraction elements of the chunk: two 16-byte fragments per lane and token row
+            const int k0 = kc * kGemvChunk + warp * 64 + q * 8;
+            uint4 xa0 = make_uint4(0, 0, 0, 0), xa1 = xa0, xb0 = xa0, xb1 = xa0;
+            if (has_a) {
+                if (k0 < d) xa0 = *reinterpret_cast<const uint4 *>(xa_row + k0);
+                if (k0 + 32 < d) xa1 = *reinterpret_cast<const uint4 *>(xa_row + k0 + 32);
+            }
+            if (has_b) {
+                if (k0 < d) xb0 = *reinterpret_cast<const uint4 *>(xb_row + k0);
+                if (k0 + 32 < d) xb1 = *reinterpret_cast<const uint4 *>(xb_row + k0 + 32);
+            }
 #pragma unroll
-        for (int ti = 0; ti < kGemvMaxTiles; ++ti) {
-            if (ti < tiles && ok) {  // uniform
-                for (int kc = 0; kc < nkc; ++kc) {
-                    // this warp's 64 contraction elements of the chunk: two 16-byte fragments per lane
-                    const int k0 = kc * kGemvChunk + warp * 64 + q * 8;
-                    uint4 xa0 = make_uint4(0, 0, 0, 0), xa1 = xa0, xb0 = xa0, xb1 = xa0;
-                    if (has_a) {
-                        if (k0 < d) xa0 = *reinterpret_cast<const uint4 *>(xa_row + k0);
-                        if (k0 + 32 < d) xa1 = *reinterpret_cast<const uint4 *>(xa_row + k0 + 32);
-                    }
-                    if (has_b) {
-                        if (k0 < d) xb0 = *reinterpret_cast<const uint4 *>(xb_row + k0);
-                        if (k0 + 32 < d) xb1 = *reinterpret_cast<const uint4 *>(xb_row + k0 + 32);
-                    }
+            for (int ti = 0; ti < kGemvMaxTiles; ++ti) {
+                if (ti < tiles && ok) {  // uniform
                     if (!__all_sync(0xffffffffu, tc::mbar_wait(full_bar(stage), phase, &s_abort, status))) {
                         ok = false;
                         break;
@@ -252,14 +190,10 @@ __global__ void __launch_bounds__(kGemvThreads, 2) gemv_rows_kernel(const __nv_b
                     const uint8_t *src = gsm + stage * kGemvStageBytes + g * kGemvPitch + warp * 128 + q * 16;
                     const uint4 w0 = *reinterpret_cast<const uint4 *>(src);
                     const uint4 w1 = *reinterpret_cast<const uint4 *>(src + 64);
-#ifdef MOC_EXP_NOMMA
-                    acc[ti][0] += __uint_as_float((w0.x ^ w1.y ^ xa0.x ^ xa1.y ^ xb0.x ^ xb1.x) & 0x3f800000u);
-#else
                     mma_bf16_16816(acc[ti], xa0.x, xb0.x, xa0.y, xb0.y, w0.x, w0.y);
                     mma_bf16_16816(acc[ti], xa0.z, xb0.z, xa0.w, xb0.w, w0.z, w0.w);
                     mma_bf16_16816(acc[ti], xa1.x, xb1.x, xa1.y, xb1.y, w1.x, w1.y);
                     mma_bf16_16816(acc[ti], xa1.z, xb1.z, xa1.w, xb1.w, w1.z, w1.w);
-#endif
                     __syncwarp();
                     if (lane == 0) tc::mbar_arrive(empty_bar(stage));
                     if (++stage == kGemvStages) {
@@ -326,7 +260,8 @@ struct SelectLevel {
     uint32_t count;   // number of candidates
 };
 
-__global__ void __launch_bounds__(kSelThreads) select_mask_kernel(Workspace ws, int F, int K) {
+__global__ void __launch_bounds__(kSelThreads) select_mask_kernel(Workspace ws, int F, int K, int *arrivals) {
+    static_assert(kSelThreads == 1024, "the listing step scans one count per lane");
     extern __shared__ __align__(16) uint32_t dyn[];  // keys [F] | candidate lists 2 x [kSelListCap]
     __shared__ SelectSmemT<kSelThreads / 32> sm;      // full radix select (fallback); its arrays double as scratch
     __shared__ uint32_t s_min[32], s_max[32], s_pick, s_above, s_inbin, s_n;
@@ -480,6 +415,42 @@ __global__ void __launch_bounds__(kSelThreads) select_mask_kernel(Workspace ws, 
     } else {
         block_ordered_emit<kSelThreads>(keys, F, tau, need, sm, [&](int, int j) { atomicOr(&ws.chmask[j], bit); });
     }
+    // ---- the last CTA to get here lists the used channels (ascending) for the up and down kernels
+    __shared__ int s_is_last, s_warp_cnt[NW], s_base;
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        s_is_last = atomicAdd(arrivals, 1) == (int)gridDim.x - 1;
+        s_base = 0;
+    }
+    __syncthreads();
+    if (!s_is_last) return;
+    __threadfence();
+    constexpr int kMaxChunks = (kSelectMaxN + kSelThreads - 1) / kSelThreads;
+    uint32_t used_bits = 0;  // bit c: channel c * kSelThreads + tid is used (all loads issued together)
+#pragma unroll
+    for (int c = 0; c < kMaxChunks; ++c) {
+        const int j = c * kSelThreads + tid;
+        if (j < F && __ldcg(&ws.chmask[j]) != 0u) used_bits |= 1u << c;
+    }
+    for (int c = 0; c * kSelThreads < F; ++c) {
+        const bool used = (used_bits >> c) & 1u;
+        const uint32_t b = __ballot_sync(0xffffffffu, used);
+        if (lane == 0) s_warp_cnt[warp] = __popc(b);
+        __syncthreads();
+        int w = s_warp_cnt[lane], inc = w;  // NW == 32: one count per lane
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, inc, o);
+            if (lane >= o) inc += v;
+        }
+        const int before = __shfl_sync(0xffffffffu, inc - w, warp), total = __shfl_sync(0xffffffffu, inc, 31);
+        if (used) ws.list[s_base + before + __popc(b & ((1u << lane) - 1u))] = (uint16_t)(c * kSelThreads + tid);
+        __syncthreads();
+        if (tid == 0) s_base += total;
+        __syncthreads();
+    }
+    if (tid == 0) *ws.list_count = s_base;
 }
 
 // ---------------------------------------------------------------------------------------------- 4. down

@@ -41,6 +41,22 @@ def test_kernel_work_table_matches_per_token_formulas():
     assert bench.kernel_work("nonexistent", T, d, F, K, e) is None
 
 
+def test_roofline_report_picks_the_largest_kernel_and_fills_every_key():
+    from paper_2511_09323_b200 import synthetic as syn
+    w, steps = syn.C2, 4
+    peaks = {"hbm_gbs": 6550.7, "bf16_tflops": 1647.5, "bf16_tflops_sustained": 1388.1, "source": "measured"}
+    prof = {"tc_wgrad_gemm": (steps, 0.48), "tc_select_mask": (steps, 0.36), "_hidden": (1, 9.0)}
+    roof, kernels = bench.roofline_report(prof, steps, w.tokens, w, 2, peaks)
+    assert roof["kernel"] == "tc_wgrad_gemm" and set(kernels) == {"tc_wgrad_gemm", "tc_select_mask"}
+    assert roof["bound"] == "tensor" and roof["peak"] == 1388.1 and roof["unit"] == "TFLOP/s"
+    assert roof["frac"] == pytest.approx(roof["achieved"] / roof["peak"])
+    assert roof["achieved"] == pytest.approx(6.0 * w.tokens * w.k * w.d_model / 0.12e-3 / 1e12)
+    assert roof["traffic"] == bench.NCU_DRAM_BYTES_C2["tc_wgrad_gemm"]          # default workload: measured bytes
+    roof2, _ = bench.roofline_report(prof, steps, 1024, w, 2, peaks)            # any other size: no measurement
+    assert roof2["traffic"] is None
+    assert kernels["tc_select_mask"]["share"] == pytest.approx(0.36 / 0.84, abs=1e-3)
+
+
 def _worker(rank, world, port, q):
     os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
     dist.init_process_group("gloo", rank=rank, world_size=world)
