@@ -550,8 +550,8 @@ DecodeLayout decode_layout(const moc_ffn_desc &d) {
     Carver c;
     L.off_g = c.take((size_t)d.tokens * L.ldf * sizeof(float));
     L.off_zb = c.take((size_t)((d.d_ff + 15) / 16) * 256 * sizeof(__nv_bfloat16));
-    L.off_mask = c.take((size_t)d.d_ff * sizeof(uint32_t));
-    L.off_list = c.take((size_t)d.d_ff * sizeof(uint16_t));
+    L.off_mask = c.take((size_t)d.tokens * ((d.d_ff + 31) / 32) * sizeof(uint32_t));  // per-token selection bitmaps
+    L.off_list = c.take((size_t)(d.d_ff + 1) * sizeof(uint16_t));
     L.off_count = c.take(sizeof(int));
     L.off_acc = c.take((size_t)d.tokens * d.d_model * sizeof(float));
     L.off_cnt = c.take((size_t)(L.slices + 1) * sizeof(int));  // + arrivals of the select kernel
@@ -572,7 +572,8 @@ int decode_bf16(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat
     dec::Workspace ws;
     ws.G = reinterpret_cast<float *>(wsp + L.off_g);
     ws.Zb = reinterpret_cast<__nv_bfloat16 *>(wsp + L.off_zb);
-    ws.chmask = reinterpret_cast<uint32_t *>(wsp + L.off_mask);
+    ws.sel_bits = reinterpret_cast<uint32_t *>(wsp + L.off_mask);
+    ws.sel_words = (F + 31) / 32;
     ws.list = reinterpret_cast<uint16_t *>(wsp + L.off_list);
     ws.list_count = reinterpret_cast<int *>(wsp + L.off_count);
     ws.out_acc = reinterpret_cast<float *>(wsp + L.off_acc);
@@ -886,5 +887,6 @@ const char *moc_status_string(int status) {
 }
 
 }  // extern "C"
+
 
 

@@ -47,7 +47,8 @@ constexpr size_t kDownSmem = (size_t)kDownStages * kDownStageBytes + (size_t)kMa
 struct Workspace {
     float *G;             // [T, ldf] gate projection
     __nv_bfloat16 *Zb;    // [list position / 16][16 tokens][16 positions] z = SiLU(g) u (0 where not selected)
-    uint32_t *chmask;     // [F] bit t set: token t selected the channel
+    uint32_t *sel_bits;   // [T][sel_words] bit j % 32 of word j / 32: token t selected channel j
+    int sel_words;        // ceil(F / 32)
     uint16_t *list;       // [F] used channels in order of first selection
     int *list_count;      // number of used channels
     float *out_acc;       // [T, d]
@@ -100,7 +101,6 @@ __global__ void __launch_bounds__(kGemvThreads, 2) gemv_rows_kernel(const __nv_b
 
     if (!GATHER) {
         // housekeeping for the later kernels: clear masks, accumulators, counters
-        for (int j = r0 + tid; j < r1; j += kGemvThreads) ws.chmask[j] = 0u;
         for (int64_t i = (int64_t)blockIdx.x * kGemvThreads + tid; i < (int64_t)T * d;
              i += (int64_t)gridDim.x * kGemvThreads)
             ws.out_acc[i] = 0.f;
@@ -229,7 +229,8 @@ __global__ void __launch_bounds__(kGemvThreads, 2) gemv_rows_kernel(const __nv_b
             } else {
                 const int j = s_rows[c];
                 float z = 0.f;
-                if (t < T && ((ws.chmask[j] >> t) & 1u)) z = silu_f(ws.G[(int64_t)t * ws.ldf + j]) * sum;
+                if (t < T && ((ws.sel_bits[t * ws.sel_words + (j >> 5)] >> (j & 31)) & 1u))
+                    z = silu_f(ws.G[(int64_t)t * ws.ldf + j]) * sum;
                 ws.Zb[((int64_t)(slot >> 4) * 16 + t) * 16 + (slot & 15)] = __float2bfloat16_rn(z);
             }
         }
@@ -271,7 +272,6 @@ __global__ void __launch_bounds__(kSelThreads) select_mask_kernel(Workspace ws, 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     constexpr int NW = kSelThreads / 32;
     const int t = blockIdx.x;
-    const uint32_t bit = 1u << t;
     const float *g = ws.G + (int64_t)t * ws.ldf;
 
     // ---- keys, minimum and maximum
@@ -408,49 +408,73 @@ __global__ void __launch_bounds__(kSelThreads) select_mask_kernel(Workspace ws, 
         block_radix_threshold<kSelThreads>(keys, F, K, sm, tau, need);
     else
         ties_cut = in_bin != (uint32_t)need;
+    uint32_t *my_bits = ws.sel_bits + (int64_t)t * ws.sel_words;
+    const int nch = (F + kSelThreads - 1) / kSelThreads;
     if (!ties_cut) {
-        // every key >= tau is kept; no order is needed and nothing is read back (plain reductions)
-        for (int j = tid; j < F; j += kSelThreads)
-            if (keys[j] >= tau) atomicOr(&ws.chmask[j], bit);
+        // every key >= tau is kept: consecutive lanes hold consecutive channels, so a ballot IS a word of the
+        // token's selection bitmap (plain stores, no atomics, nothing read back)
+        for (int c = 0; c < nch; ++c) {
+            const int j = c * kSelThreads + tid;
+            const uint32_t b = __ballot_sync(0xffffffffu, j < F && keys[j] >= tau);
+            if (lane == 0 && c * kSelThreads + warp * 32 < F) my_bits[c * NW + warp] = b;
+        }
     } else {
-        block_ordered_emit<kSelThreads>(keys, F, tau, need, sm, [&](int, int j) { atomicOr(&ws.chmask[j], bit); });
+        for (int i = tid; i < ws.sel_words; i += kSelThreads) my_bits[i] = 0u;
+        __syncthreads();
+        block_ordered_emit<kSelThreads>(keys, F, tau, need, sm,
+                                        [&](int, int j) { atomicOr(&my_bits[j >> 5], 1u << (j & 31)); });
     }
     // ---- the last CTA to get here lists the used channels (ascending) for the up and down kernels
-    __shared__ int s_is_last, s_warp_cnt[NW], s_base;
+    __shared__ int s_is_last, s_warp_cnt[NW];
     __threadfence();
     __syncthreads();
     if (tid == 0) {
         s_is_last = atomicAdd(arrivals, 1) == (int)gridDim.x - 1;
-        s_base = 0;
     }
     __syncthreads();
     if (!s_is_last) return;
     __threadfence();
-    constexpr int kMaxChunks = (kSelectMaxN + kSelThreads - 1) / kSelThreads;
-    uint32_t used_bits = 0;  // bit c: channel c * kSelThreads + tid is used (all loads issued together)
+    // union of the tokens' bitmaps, one word per thread (at most 1024 words), block-wide exclusive scan of the
+    // popcounts, then every thread writes the channels of its word
+    uint32_t word = 0;
+    if (tid < ws.sel_words) {
+        uint32_t part[16];  // at most 16 tokens: all loads in flight together
 #pragma unroll
-    for (int c = 0; c < kMaxChunks; ++c) {
-        const int j = c * kSelThreads + tid;
-        if (j < F && __ldcg(&ws.chmask[j]) != 0u) used_bits |= 1u << c;
-    }
-    for (int c = 0; c * kSelThreads < F; ++c) {
-        const bool used = (used_bits >> c) & 1u;
-        const uint32_t b = __ballot_sync(0xffffffffu, used);
-        if (lane == 0) s_warp_cnt[warp] = __popc(b);
-        __syncthreads();
-        int w = s_warp_cnt[lane], inc = w;  // NW == 32: one count per lane
+        for (int tt = 0; tt < 16; ++tt)
+            part[tt] = tt < (int)gridDim.x ? __ldcg(&ws.sel_bits[(int64_t)tt * ws.sel_words + tid]) : 0u;
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int v = __shfl_up_sync(0xffffffffu, inc, o);
-            if (lane >= o) inc += v;
-        }
-        const int before = __shfl_sync(0xffffffffu, inc - w, warp), total = __shfl_sync(0xffffffffu, inc, 31);
-        if (used) ws.list[s_base + before + __popc(b & ((1u << lane) - 1u))] = (uint16_t)(c * kSelThreads + tid);
-        __syncthreads();
-        if (tid == 0) s_base += total;
-        __syncthreads();
+        for (int tt = 0; tt < 16; ++tt) word |= part[tt];
     }
-    if (tid == 0) *ws.list_count = s_base;
+    const int v = __popc(word);
+    int inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int u = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += u;
+    }
+    if (lane == 31) s_warp_cnt[warp] = inc;
+    __syncthreads();
+    int wt = s_warp_cnt[lane], winc = wt;  // NW == 32: one warp total per lane
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int u = __shfl_up_sync(0xffffffffu, winc, o);
+        if (lane >= o) winc += u;
+    }
+    const int before_warp = __shfl_sync(0xffffffffu, winc - wt, warp), total = __shfl_sync(0xffffffffu, winc, 31);
+    // the list is put together in shared memory (the keys' memory, free by now) and leaves in whole words:
+    // consecutive 2-byte stores of one thread to global memory serialise on their sector
+    uint16_t *slist = reinterpret_cast<uint16_t *>(dyn);
+    __syncthreads();  // all threads are done with the keys
+    int pos = before_warp + inc - v;
+    while (word) {
+        const int bpos = __ffs(word) - 1;
+        word &= word - 1u;
+        slist[pos++] = (uint16_t)(tid * 32 + bpos);
+    }
+    __syncthreads();
+    for (int i = tid; i < (total + 1) / 2; i += kSelThreads)  // the list array holds F (rounded up to even) entries
+        reinterpret_cast<uint32_t *>(ws.list)[i] = reinterpret_cast<const uint32_t *>(slist)[i];
+    if (tid == 0) *ws.list_count = total;
 }
 
 // ---------------------------------------------------------------------------------------------- 4. down
@@ -562,19 +586,31 @@ __global__ void __launch_bounds__(kGemvThreads, 2) down_rows_kernel(const __nv_b
                 phase ^= 1u;
             }
         }
-        // add this CTA's partial sums: rows g / g+8 = tokens, columns 64 warp + 8 nb + 2q, +1
+        // add this CTA's partial sums.  A lane holds columns 64 warp + 8 nb + 2q, +1 of tokens g and g + 8; lanes q
+        // and q ^ 1 swap halves so that an even lane owns four consecutive columns of token g and an odd lane of
+        // token g + 8: one 16-byte vector reduction each instead of four scalar ones
         if (nblocks > 0) {
+            const bool odd = q & 1;
+            const int tok = odd ? g + 8 : g;
 #pragma unroll
             for (int nb = 0; nb < 8; ++nb) {
-                const int c = warp * 64 + nb * 8 + 2 * q;
-                if (c < cols) {
-                    if (g < T) {
-                        atomicAdd(ws.out_acc + (int64_t)g * d + c0 + c, acc[nb][0]);
-                        atomicAdd(ws.out_acc + (int64_t)g * d + c0 + c + 1, acc[nb][1]);
-                    }
-                    if (g + 8 < T) {
-                        atomicAdd(ws.out_acc + (int64_t)(g + 8) * d + c0 + c, acc[nb][2]);
-                        atomicAdd(ws.out_acc + (int64_t)(g + 8) * d + c0 + c + 1, acc[nb][3]);
+                const float s0 = odd ? acc[nb][0] : acc[nb][2], s1 = odd ? acc[nb][1] : acc[nb][3];
+                const float r0v = __shfl_xor_sync(0xffffffffu, s0, 1), r1v = __shfl_xor_sync(0xffffffffu, s1, 1);
+                const float k0 = odd ? acc[nb][2] : acc[nb][0], k1 = odd ? acc[nb][3] : acc[nb][1];
+                // even lane: (own, partner's) = columns c .. c+3; odd lane: (partner's, own) = columns c-2 .. c+1
+                const float v0 = odd ? r0v : k0, v1 = odd ? r1v : k1, v2 = odd ? k0 : r0v, v3 = odd ? k1 : r1v;
+                const int c = warp * 64 + nb * 8 + 2 * (q & ~1);
+                if (tok < T) {
+                    float *dst = ws.out_acc + (int64_t)tok * d + c0 + c;
+                    if (c + 3 < cols) {
+                        asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst), "f"(v0), "f"(v1), "f"(v2),
+                                     "f"(v3)
+                                     : "memory");
+                    } else {
+                        if (c < cols) atomicAdd(dst, v0);
+                        if (c + 1 < cols) atomicAdd(dst + 1, v1);
+                        if (c + 2 < cols) atomicAdd(dst + 2, v2);
+                        if (c + 3 < cols) atomicAdd(dst + 3, v3);
                     }
                 }
             }
