@@ -563,6 +563,23 @@ bool use_decode_plan(const moc_ffn_desc &d) {
     return d.dtype == MOC_BF16 && d.tokens >= 1 && d.tokens <= 16 && d.d_model <= 256 * dec::kSliceCols;
 }
 
+// Launch with programmatic stream serialization allowed: the kernel may become resident while its predecessor in
+// the stream drains (every kernel launched this way calls pdl_wait before it touches global data).
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, unsigned block, size_t smem, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+}
+
 int decode_bf16(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat16 *wg, const __nv_bfloat16 *wu,
                 const __nv_bfloat16 *wd, __nv_bfloat16 *out, char *wsp, cudaStream_t st) {
     const DecodeLayout L = decode_layout(d);
@@ -587,18 +604,20 @@ int decode_bf16(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat
     if ((rc = set_smem(dec::gemv_rows_kernel<true>, dec::kGemvSmem)) != MOC_OK) return rc;
 
     MOC_LAUNCH(KID_DEC_GATE_GEMV, st,
-               (dec::gemv_rows_kernel<false><<<L.gemv_grid, dec::kGemvThreads, dec::kGemvSmem, st>>>(
-                   x, wg, T, dm, F, ws, L.slices, status)));
+               launch_pdl(dec::gemv_rows_kernel<false>, dim3(L.gemv_grid), dec::kGemvThreads, dec::kGemvSmem, st, x, wg, T,
+                          dm, F, ws, L.slices, status));
     if ((rc = launch_ok()) != MOC_OK) return rc;
-    MOC_LAUNCH(KID_DEC_SELECT, st, (dec::select_mask_kernel<<<T, dec::kSelThreads, sel_smem, st>>>(ws, F, K, ws.counters + L.slices)));
+    MOC_LAUNCH(KID_DEC_SELECT, st,
+               launch_pdl(dec::select_mask_kernel, dim3(T), dec::kSelThreads, sel_smem, st, ws, F, K,
+                          ws.counters + L.slices));
     if ((rc = launch_ok()) != MOC_OK) return rc;
     MOC_LAUNCH(KID_DEC_UP, st,
-               (dec::gemv_rows_kernel<true><<<L.gemv_grid, dec::kGemvThreads, dec::kGemvSmem, st>>>(
-                   x, wu, T, dm, F, ws, L.slices, status)));
+               launch_pdl(dec::gemv_rows_kernel<true>, dim3(L.gemv_grid), dec::kGemvThreads, dec::kGemvSmem, st, x, wu, T,
+                          dm, F, ws, L.slices, status));
     if ((rc = launch_ok()) != MOC_OK) return rc;
     MOC_LAUNCH(KID_DEC_DOWN, st,
-               (dec::down_rows_kernel<<<dim3(L.slices, L.parts), dec::kGemvThreads, dec::kDownSmem, st>>>(
-                   wd, T, dm, F, ws, out, status)));
+               launch_pdl(dec::down_rows_kernel, dim3(L.slices, L.parts), dec::kGemvThreads, dec::kDownSmem, st, wd, T, dm,
+                          F, ws, out, status));
     return launch_ok();
 }
 

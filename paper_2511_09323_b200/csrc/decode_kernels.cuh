@@ -87,7 +87,12 @@ __global__ void __launch_bounds__(kGemvThreads, 2) gemv_rows_kernel(const __nv_b
     __shared__ int s_abort;
     __shared__ uint16_t s_rows[kGemvMaxRows];                          // this CTA's rows when gathering
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    // gathering: the used channels (ascending) were listed by the select kernel
+    tc::pdl_launch_dependents();
+    // Gathering: the list of used channels comes from the select kernel, so every thread waits for it here.
+    // Gate projection: the weights do not depend on earlier kernels, so the producer warp starts streaming them
+    // at once (while the previous kernel of the stream may still be draining); only the consumers wait, before
+    // they touch x or the workspace.
+    if (GATHER) tc::pdl_wait();
     const int n = GATHER ? min(*ws.list_count, F) : F;
     const int r0 = (int)(((int64_t)blockIdx.x * n) / gridDim.x);
     const int r1 = (int)(((int64_t)(blockIdx.x + 1) * n) / gridDim.x);
@@ -99,13 +104,6 @@ __global__ void __launch_bounds__(kGemvThreads, 2) gemv_rows_kernel(const __nv_b
     auto full_bar = [&](int s) { return tc::smem_u32(&bars[s]); };
     auto empty_bar = [&](int s) { return tc::smem_u32(&bars[kGemvStages + s]); };
 
-    if (!GATHER) {
-        // housekeeping for the later kernels: clear masks, accumulators, counters
-        for (int64_t i = (int64_t)blockIdx.x * kGemvThreads + tid; i < (int64_t)T * d;
-             i += (int64_t)gridDim.x * kGemvThreads)
-            ws.out_acc[i] = 0.f;
-        if (blockIdx.x == 0 && tid <= slices) ws.counters[tid] = 0;  // [slices]: arrivals of the select kernel
-    }
     // When the last chunk of a row is short, the bytes it leaves untouched are multiplied by zero x entries and
     // must therefore be finite: the ring then starts out as zeros.  (Rows of a partial tile that are never
     // copied only feed outputs that are never written.)
@@ -122,7 +120,7 @@ __global__ void __launch_bounds__(kGemvThreads, 2) gemv_rows_kernel(const __nv_b
     }
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // zero fill before the async copies
     __syncthreads();
-    if (tiles <= 0) return;
+    if (tiles <= 0 && GATHER) return;  // (the gate kernel's grid never leaves a CTA without rows)
 
     if (warp == 8) {
         // ------------------------------------------------------------------ producer
@@ -159,6 +157,14 @@ __global__ void __launch_bounds__(kGemvThreads, 2) gemv_rows_kernel(const __nv_b
         // The partial sums of all the CTA's tiles (at most kGemvMaxTiles, the host sizes the grid for that)
         // stay in registers; the eight warps' sums are combined once, after the last stage, in the ring's
         // memory (idle by then).
+        if (!GATHER) {
+            tc::pdl_wait();
+            // housekeeping for the later kernels: clear the accumulators and the arrival counters
+            for (int64_t i = (int64_t)blockIdx.x * 256 + tid; i < (int64_t)T * d; i += (int64_t)gridDim.x * 256)
+                ws.out_acc[i] = 0.f;
+            if (blockIdx.x == 0)
+                for (int i = tid; i <= slices; i += 256) ws.counters[i] = 0;  // [slices]: arrivals of the select kernel
+        }
         const int g = lane >> 2, q = lane & 3;
         const __nv_bfloat16 *xa_row = x + (int64_t)g * d, *xb_row = x + (int64_t)(g + 8) * d;
         const bool has_a = g < T, has_b = g + 8 < T;
@@ -272,6 +278,8 @@ __global__ void __launch_bounds__(kSelThreads) select_mask_kernel(Workspace ws, 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     constexpr int NW = kSelThreads / 32;
     const int t = blockIdx.x;
+    tc::pdl_launch_dependents();
+    tc::pdl_wait();
     const float *g = ws.G + (int64_t)t * ws.ldf;
 
     // ---- keys, minimum and maximum
@@ -497,17 +505,9 @@ __global__ void __launch_bounds__(kGemvThreads, 2) down_rows_kernel(const __nv_b
     const int slice = blockIdx.x, c0 = slice * kSliceCols;
     const int cols = min(kSliceCols, d - c0);       // multiple of 8
     const uint32_t row_bytes = (uint32_t)cols * 2;  // multiple of 16
-    const int total = min(*ws.list_count, F);
-    // parts are whole 16-position blocks, so that a part's z blocks are the ones the up kernel wrote
-    const int blocks_total = (total + 15) >> 4;
-    const int per_blocks = min(kMaxPart / 16, (blocks_total + (int)gridDim.y - 1) / (int)gridDim.y);
-    const int b0 = min(blocks_total, (int)blockIdx.y * per_blocks);
-    const int nblocks = min(per_blocks, blocks_total - b0);
-    const int p0 = b0 * 16;
-    const int count = min(nblocks * 16, total - p0);
+    tc::pdl_launch_dependents();
     auto full_bar = [&](int s) { return tc::smem_u32(&bars[s]); };
     auto empty_bar = [&](int s) { return tc::smem_u32(&bars[kDownStages + s]); };
-
     for (int i = tid; i < (int)(kDownStages * kDownStageBytes / 16); i += kGemvThreads)
         reinterpret_cast<uint4 *>(ring)[i] = make_uint4(0, 0, 0, 0);
     if (tid == 0) {
@@ -518,6 +518,15 @@ __global__ void __launch_bounds__(kGemvThreads, 2) down_rows_kernel(const __nv_b
         s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    tc::pdl_wait();  // the list and z come from the kernels before
+    const int total = min(*ws.list_count, F);
+    // parts are whole 16-position blocks, so that a part's z blocks are the ones the up kernel wrote
+    const int blocks_total = (total + 15) >> 4;
+    const int per_blocks = min(kMaxPart / 16, (blocks_total + (int)gridDim.y - 1) / (int)gridDim.y);
+    const int b0 = min(blocks_total, (int)blockIdx.y * per_blocks);
+    const int nblocks = min(per_blocks, blocks_total - b0);
+    const int p0 = b0 * 16;
+    const int count = min(nblocks * 16, total - p0);
     for (int i = tid; i < count; i += kGemvThreads) lch[i] = ws.list[p0 + i];
     // z blocks of this part: nblocks x 512 bytes, contiguous
     for (int i = tid; i < nblocks * 32; i += kGemvThreads)
