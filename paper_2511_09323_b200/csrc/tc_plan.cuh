@@ -323,7 +323,11 @@ __global__ void __launch_bounds__(kWarpSelMaxWarps * 32) select_mask_rows_warp_k
     uint32_t *bitmap = cand + warp_select_cand_words(nv);                                     // kept-channel bitmap
     uint32_t *kept = bitmap + warp_select_bitmap_words(nv);                                    // [K] channel | z bits << 16
     uint64_t *bar_mem = reinterpret_cast<uint64_t *>(kept + ((K + 3) & ~3));
-    const uint32_t bar = smem_u32(bar_mem);
+    const uint32_t bar_g = smem_u32(bar_mem), bar_u = smem_u32(bar_mem + 1);  // gate row / up row arrived
+    // the kept channels' gate values are parked in the search scratch (free by then) when it is large enough: the
+    // gate buffer can then take the next token's row while this token's values are still being worked on
+    float *gkept = reinterpret_cast<float *>(cand);
+    const bool early_gate = K <= warp_select_cand_words(nv) + warp_select_bitmap_words(nv);
     const int64_t gw = (int64_t)blockIdx.x * wpc + wib, nw = (int64_t)gridDim.x * wpc;
     const float b_center = meta.bracket[0], b_width = meta.bracket[1];
     const bool have_bracket = meta.bracket[2] == kBracketTag && b_width > 0.f && fabsf(b_center) <= 3.0e38f;
@@ -334,30 +338,35 @@ __global__ void __launch_bounds__(kWarpSelMaxWarps * 32) select_mask_rows_warp_k
     const uint32_t g_bytes = (uint32_t)ldg * 4u, u_bytes = (uint32_t)ldu * 2u;  // multiples of 16: ld % 8 == 0
 
     if (threadIdx.x == 0) s_abort = 0;
-    if (lane == 0) mbar_init(bar, 1);
+    if (lane == 0) {
+        mbar_init(bar_g, 1);
+        mbar_init(bar_u, 1);
+    }
     // channels the copies never write read as -inf for good
     for (int c = ldg + lane; c < nv * 128; c += 32) sg[c] = -INFINITY;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     __syncthreads();
-    uint32_t phase = 0;
+    uint32_t phase = 0;  // both barriers complete once per token
     bool dead = false;
+    if (lane == 0 && gw < rows) {
+        mbar_expect_tx(bar_g, g_bytes);
+        bulk_copy_g2s(smem_u32(sg), G + gw * (int64_t)ldg, g_bytes, bar_g);
+    }
 
     for (int64_t r = gw; r < rows && !dead; r += nw) {
-        const float *g = G + r * (int64_t)ldg;
         __nv_bfloat16 *u = U + r * (int64_t)ldu;
-        // ---- stage the two rows (the previous row's store has to have read the up buffer first)
+        // ---- the up row is needed only in step 4: its copy starts now (once the previous token's store has read
+        //      the buffer) and lands while steps 1-3 run; the gate row was requested during the previous token
         if (lane == 0) {
             bulk_store_wait_read<0>();
             fence_async_smem();
-            mbar_expect_tx(bar, g_bytes + u_bytes);
-            bulk_copy_g2s(smem_u32(sg), g, g_bytes, bar);
-            bulk_copy_g2s(smem_u32(su), u, u_bytes, bar);
+            mbar_expect_tx(bar_u, u_bytes);
+            bulk_copy_g2s(smem_u32(su), u, u_bytes, bar_u);
         }
-        if (!__all_sync(0xffffffffu, mbar_wait(bar, phase, &s_abort, status))) {
+        if (!__all_sync(0xffffffffu, mbar_wait(bar_g, phase, &s_abort, status))) {
             dead = true;
             break;
         }
-        phase ^= 1u;
         for (int c = F + lane; c < ldg; c += 32) sg[c] = -INFINITY;  // padding columns of this row
         __syncwarp();
 
@@ -498,11 +507,29 @@ __global__ void __launch_bounds__(kWarpSelMaxWarps * 32) select_mask_rows_warp_k
         __syncwarp();
         if (!fast) tau = warp_select_row_general(sg, F, K, cand, kept);
         __syncwarp();
-        // ---- 4. values of the kept channels (shared-memory gathers); the compact outputs are written with
-        //         consecutive lanes on consecutive slots
+        // ---- 4. values of the kept channels (shared-memory gathers).  Gate values first, so that the gate buffer
+        //         can be handed to the next token's copy
+        auto request_next_gate = [&]() {
+            if (lane == 0 && r + nw < rows) {
+                fence_async_smem();
+                mbar_expect_tx(bar_g, g_bytes);
+                bulk_copy_g2s(smem_u32(sg), G + (r + nw) * (int64_t)ldg, g_bytes, bar_g);
+            }
+        };
+        if (early_gate) {
+            for (int i = lane; i < K; i += 32) gkept[i] = sg[kept[i]];
+            __syncwarp();
+            request_next_gate();
+        }
+        if (!__all_sync(0xffffffffu, mbar_wait(bar_u, phase, &s_abort, status))) {
+            dead = true;
+            break;
+        }
+        phase ^= 1u;
+        //         the compact outputs are written with consecutive lanes on consecutive slots
         for (int i = lane; i < K; i += 32) {
             const uint32_t j = kept[i];
-            const float gval = sg[j];
+            const float gval = early_gate ? gkept[i] : sg[j];
             const __nv_bfloat16 ub = su[j];
             const __nv_bfloat16 zb = __float2bfloat16_rn(silu_f(gval) * __bfloat162float(ub));
             kept[i] = j | ((uint32_t)(*reinterpret_cast<const uint16_t *>(&zb)) << 16);
@@ -513,6 +540,7 @@ __global__ void __launch_bounds__(kWarpSelMaxWarps * 32) select_mask_rows_warp_k
             }
         }
         __syncwarp();
+        if (!early_gate) request_next_gate();
         // ---- up row -> masked Z' row, in shared memory, then one bulk store
         uint4 *row16 = reinterpret_cast<uint4 *>(su);
         for (int i = lane; i < (ldu >> 3); i += 32) row16[i] = make_uint4(0, 0, 0, 0);
