@@ -324,15 +324,15 @@ __global__ void __launch_bounds__(kSelThreads) select_mask_kernel(Workspace ws, 
             // in (value descending, position ascending) order
             if (tid < (int)lv.count) {
                 const uint32_t mine = src[tid];
-                uint32_t before = 0, equal = 0;
-                for (uint32_t i = 0; i < lv.count; ++i) {
+                uint32_t before = 0, equal = 0, gt = 0;
+#pragma unroll 8
+                for (uint32_t i = 0; i < lv.count; ++i) {  // independent broadcast loads, eight in flight
                     const uint32_t o = src[i];
+                    gt += o > mine ? 1u : 0u;
                     before += (o > mine || (o == mine && i < (uint32_t)tid)) ? 1u : 0u;
                     equal += o == mine ? 1u : 0u;
                 }
                 if (before == lv.m - 1) {
-                    uint32_t gt = 0;
-                    for (uint32_t i = 0; i < lv.count; ++i) gt += src[i] > mine ? 1u : 0u;
                     s_pick = mine;
                     s_above = lv.m - gt;  // how many keys equal to tau are wanted
                     s_inbin = equal;
