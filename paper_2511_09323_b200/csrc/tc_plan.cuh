@@ -721,7 +721,8 @@ __global__ void __launch_bounds__(256) backward_sample_rows_kernel(
 // three masked rows are built in shared memory and leave as bulk stores.  Global traffic is fully
 // coalesced and the scattered accesses stay on chip.  Used when the four rows of a token fit a slice.
 __host__ __device__ constexpr size_t sample_warp_words(int ld, int K) {
-    return (size_t)2 * ld /* four bf16 rows */ + (size_t)2 * ((K + 1) & ~1) /* entries */ + 4 /* two mbarriers */;
+    return (size_t)2 * ld /* four bf16 rows */ + (size_t)2 * ((K + 1) & ~1) /* entries */ +
+           (size_t)3 * ((K + 7) & ~7) /* saved idx, g, u of two tokens */ + 4 /* two mbarriers */;
 }
 constexpr int kSampleMaxWarps = 8;
 
@@ -738,9 +739,14 @@ __global__ void __launch_bounds__(kSampleMaxWarps * 32) backward_sample_rows_war
     __nv_bfloat16 *ubuf = reinterpret_cast<__nv_bfloat16 *>(base + 2 * row_words);
     __nv_bfloat16 *gbuf = reinterpret_cast<__nv_bfloat16 *>(base + 3 * row_words);
     uint32_t *entry = base + 4 * row_words;  // K x {j | z << 16, dU | dG << 16}
-    uint64_t *bar_mem = reinterpret_cast<uint64_t *>(entry + 2 * ((K + 1) & ~1));
+    // saved idx | g | u rows of the two tokens in flight, K8 16-bit entries each (arrive with the dZ row when K is a
+    // multiple of 8, i.e. when the rows are 16-byte multiples; plain loads otherwise)
+    const int K8 = (K + 7) & ~7;
+    uint16_t *saved0 = reinterpret_cast<uint16_t *>(entry + 2 * ((K + 1) & ~1));
+    const bool staged_saved = (K & 7) == 0;
+    uint64_t *bar_mem = reinterpret_cast<uint64_t *>(saved0 + 6 * K8);
     const uint32_t bar0 = smem_u32(bar_mem);  // two mbarriers, 8 bytes apart
-    const uint32_t row_bytes = (uint32_t)ld * 2u;
+    const uint32_t row_bytes = (uint32_t)ld * 2u, saved_bytes = (uint32_t)K * 2u;
     const int64_t gw = (int64_t)blockIdx.x * wpc + wib, nw = (int64_t)gridDim.x * wpc;
 
     if (threadIdx.x == 0) s_abort = 0;
@@ -751,15 +757,24 @@ __global__ void __launch_bounds__(kSampleMaxWarps * 32) backward_sample_rows_war
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     __syncthreads();
     uint32_t phases = 0;  // bit b: parity to wait for on barrier b
-    if (lane == 0 && gw < T) {
-        mbar_expect_tx(bar0, row_bytes);
-        bulk_copy_g2s(smem_u32(zbuf0), dz_z + gw * (int64_t)ld, row_bytes, bar0);
-    }
+    auto request = [&](int64_t tok, int buf) {  // lane 0: dZ row (+ saved rows) of a token into buffer `buf`
+        const uint32_t nbar = bar0 + 8u * (uint32_t)buf;
+        mbar_expect_tx(nbar, row_bytes + (staged_saved ? 3u * saved_bytes : 0u));
+        bulk_copy_g2s(smem_u32(zbuf0 + (size_t)buf * ld), dz_z + tok * (int64_t)ld, row_bytes, nbar);
+        if (staged_saved) {
+            uint16_t *sv = saved0 + (size_t)buf * 3 * K8;
+            bulk_copy_g2s(smem_u32(sv), idx + tok * K, saved_bytes, nbar);
+            bulk_copy_g2s(smem_u32(sv + K8), gval + tok * K, saved_bytes, nbar);
+            bulk_copy_g2s(smem_u32(sv + 2 * K8), uval + tok * K, saved_bytes, nbar);
+        }
+    };
+    if (lane == 0 && gw < T) request(gw, 0);
     int b = 0;
     for (int64_t t = gw; t < T; t += nw, b ^= 1) {
         if (!__all_sync(0xffffffffu, mbar_wait(bar0 + 8u * (uint32_t)b, (phases >> b) & 1u, &s_abort, status))) break;
         phases ^= 1u << b;
         __nv_bfloat16 *zr = zbuf0 + (size_t)b * ld;
+        const uint16_t *sv = saved0 + (size_t)b * 3 * K8;
         for (int k0 = 0; k0 < K; k0 += 256) {
             // eight saved entries per lane, their loads issued together
             int jv[8];
@@ -769,9 +784,15 @@ __global__ void __launch_bounds__(kSampleMaxWarps * 32) backward_sample_rows_war
                 const int k = k0 + i * 32 + lane;
                 jv[i] = -1;
                 if (k < K) {
-                    jv[i] = idx[t * K + k];
-                    gb[i] = gval[t * K + k];
-                    ub[i] = uval[t * K + k];
+                    if (staged_saved) {
+                        jv[i] = (int16_t)sv[k];
+                        gb[i] = *reinterpret_cast<const __nv_bfloat16 *>(sv + K8 + k);
+                        ub[i] = *reinterpret_cast<const __nv_bfloat16 *>(sv + 2 * K8 + k);
+                    } else {
+                        jv[i] = idx[t * K + k];
+                        gb[i] = gval[t * K + k];
+                        ub[i] = uval[t * K + k];
+                    }
                 }
             }
 #pragma unroll
@@ -800,11 +821,7 @@ __global__ void __launch_bounds__(kSampleMaxWarps * 32) backward_sample_rows_war
         if (lane == 0) {
             bulk_store_wait_read<0>();
             fence_async_smem();
-            if (t + nw < T) {
-                const uint32_t nbar = bar0 + 8u * (uint32_t)(b ^ 1);
-                mbar_expect_tx(nbar, row_bytes);
-                bulk_copy_g2s(smem_u32(zbuf0 + (size_t)(b ^ 1) * ld), dz_z + (t + nw) * (int64_t)ld, row_bytes, nbar);
-            }
+            if (t + nw < T) request(t + nw, b ^ 1);
         }
         __syncwarp();
         {
