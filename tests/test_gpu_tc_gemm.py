@@ -67,3 +67,23 @@ def test_ragged_edges(m, n, k, a_mn, b_mn):
 def test_many_tiles_persistent_schedule_and_padding(a_mn, b_mn):
     # more tiles than SMs, long contraction (pipeline wraps many times), leading dimension > extent
     _run(2500, 1300, 1544, a_mn, b_mn, pad=8)
+
+
+def test_output_pitch_a_tensor_map_cannot_describe():
+    # 250 fp32 columns = 1000-byte rows: not a multiple of 16 bytes, so the epilogue stores rows thread by thread
+    _run(200, 250, 136, False, False)
+    _run(200, 250, 136, True, True)
+
+
+def test_single_cta_kernel_selected_by_environment():
+    """MOC_FFN_GEMM=single (read once per process) routes every GEMM to the one-CTA kernel: run the exact-tile and
+    ragged cases again in a child process with it set."""
+    import os
+    import subprocess
+    import sys
+    env = dict(os.environ, MOC_FFN_GEMM="single")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    r = subprocess.run([sys.executable, "-m", "pytest", os.path.join(root, "tests", "test_gpu_tc_gemm.py"), "-q", "-x",
+                        "-m", "gpu", "-k", "exact_tiles or ragged_edges or output_pitch"],
+                       cwd=root, env=env, capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
