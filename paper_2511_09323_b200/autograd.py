@@ -1,0 +1,79 @@
+"""`torch.autograd` front end of the MoC FFN operator: marshalling only, every step runs in the CUDA library.
+
+`moc_ffn(x, w_gate, w_up, w_down, k)` is the layer of Section 3.2 (Eqs. (Moc-1)..(Moc-3)) with the backward of Section 3.3
+(Eqs. (bp-1)..(bp-5)); between forward and backward only the compact Top-K activations are kept alive (int16 channel
+indices and the gate / up values of the K selected channels per token, Section 3.4), plus `x` for the weight gradients.
+`MoCFFN` is a drop-in module holding the three weight matrices channel-major (`[d_ff, d_model]` each, the layout of
+`nn.Linear.weight` for gate / up and of its transpose for down).
+
+No gradient flows through the choice of channels (the mask is a constant in the backward equations).
+"""
+from __future__ import annotations
+
+import torch
+
+from . import binding as B
+
+
+class _MoCFFNFunction(torch.autograd.Function):
+    @staticmethod
+    def forward(ctx, x, w_gate, w_up, w_down, k, d_ff):
+        shape = x.shape
+        x2 = x.reshape(-1, shape[-1]).contiguous()
+        save = any(ctx.needs_input_grad[:4])
+        out, idx, tg, tu = B.moc_ffn_forward(x2, w_gate, w_up, w_down, int(k), d_ff=d_ff, save=save)
+        if save:
+            ctx.save_for_backward(x2, w_gate, w_up, w_down, idx, tg, tu)
+            ctx.d_ff = d_ff
+            ctx.x_shape = shape
+        return out.reshape(shape)
+
+    @staticmethod
+    def backward(ctx, grad_out):
+        x2, w_gate, w_up, w_down, idx, tg, tu = ctx.saved_tensors
+        names = ("x", "w_gate", "w_up", "w_down")
+        want = tuple(n for n, need in zip(names, ctx.needs_input_grad[:4]) if need)
+        go = grad_out.reshape(-1, grad_out.shape[-1]).contiguous()
+        res = B.moc_ffn_backward(x2, w_gate, w_up, w_down, idx, tg, tu, go, d_ff=ctx.d_ff, want=want)
+        gx = res["grad_x"]
+        return (None if gx is None else gx.reshape(ctx.x_shape), res["grad_w_gate"], res["grad_w_up"],
+                res["grad_w_down"], None, None)
+
+
+def moc_ffn(x: torch.Tensor, w_gate: torch.Tensor, w_up: torch.Tensor, w_down: torch.Tensor, k: int,
+            d_ff: int | None = None) -> torch.Tensor:
+    """out[..., :] = sum over the k channels j with the largest pre-SiLU gate value x.w_gate[j] of
+    SiLU(x.w_gate[j]) * (x.w_up[j]) * w_down[j, :].  `x` is `[..., d_model]`, the weights `[d_ff_ld, d_model]` (rows at and
+    past `d_ff`, when given, are padding and never selected)."""
+    return _MoCFFNFunction.apply(x, w_gate, w_up, w_down, k, d_ff)
+
+
+class MoCFFN(torch.nn.Module):
+    """SwiGLU feed-forward block with Top-K channel selection on the gate (Section 3.2)."""
+
+    def __init__(self, d_model: int, d_ff: int, k: int, dtype=torch.bfloat16, device="cuda", init_std: float = 0.02):
+        super().__init__()
+        if not 1 <= k <= d_ff:
+            raise ValueError("k must be in [1, d_ff]")
+        self.d_model, self.d_ff, self.k = int(d_model), int(d_ff), int(k)
+        mk = lambda: torch.nn.Parameter(torch.empty(d_ff, d_model, dtype=dtype, device=device))
+        self.w_gate, self.w_up, self.w_down = mk(), mk(), mk()
+        self.reset_parameters(init_std)
+
+    def reset_parameters(self, std: float = 0.02) -> None:
+        for p in (self.w_gate, self.w_up, self.w_down):
+            torch.nn.init.normal_(p, mean=0.0, std=std)
+
+    def forward(self, x: torch.Tensor) -> torch.Tensor:
+        return moc_ffn(x, self.w_gate, self.w_up, self.w_down, self.k)
+
+    def saved_bytes_per_token(self) -> int:
+        """Bytes of activations alive between forward and backward per token, besides x and the output."""
+        e = torch.empty((), dtype=self.w_gate.dtype).element_size()
+        return self.k * (2 + 2 * e)
+
+    def extra_repr(self) -> str:
+        return f"d_model={self.d_model}, d_ff={self.d_ff}, k={self.k} ({100.0 * self.k / self.d_ff:.1f} % of channels)"
+
+
+__all__ = ["moc_ffn", "MoCFFN"]
