@@ -367,31 +367,48 @@ def test_tc_plan_corrupted_saved_index_is_skipped_and_reported():
         assert torch.isfinite(g[k].float()).all()
 
 
-def test_full_size_bench_workload_sampled_against_oracle():
-    """C2 at its full 16384 tokens, in the configuration bench.py times: sampled tokens of out / saved values /
-    grad_x and sampled rows of the weight gradients are recomputed one by one by the oracle."""
-    w = syn.C2
+def _full_size_sampled(w, n_tokens, n_rows):
     x, wg, wu, wd, dD = _problem(w)
     xd, wgd, wud, wdd, dDd = map(_dev, (x, wg, wu, wd, dD))
-    out, idx, tg, tu = B.moc_ffn_forward(xd, wgd, wud, wdd, w.k)
-    grads = B.moc_ffn_backward(xd, wgd, wud, wdd, idx, tg, tu, dDd)
+    out, idx, tg, tu = B.moc_ffn_forward(xd, wgd, wud, wdd, w.k, d_ff=w.d_ff)
+    grads = B.moc_ffn_backward(xd, wgd, wud, wdd, idx, tg, tu, dDd, d_ff=w.d_ff)
     torch.cuda.synchronize()
     assert B.moc_last_device_status() == B.MOC_OK
     rng = np.random.default_rng(0)
-    toks = np.sort(rng.choice(w.tokens, 96, replace=False))
+    toks = np.sort(rng.choice(w.tokens, n_tokens, replace=False))
     wg64, wu64, wd64 = map(syn.to_f64, (wg, wu, wd))
     x64s, dD64s = syn.to_f64(x[toks]), syn.to_f64(dD[toks])
     idx_np = idx.cpu().numpy()
     dev = dict(out=syn.to_f64(out[toks]), idx=idx_np[toks], gval=syn.to_f64(tg[toks]), uval=syn.to_f64(tu[toks]))
     parity.check_forward(dev, x64s, wg64, wu64, wd64, w.k, w.d_ff, w.dtype)
     ref = orc.backward(x64s, wg64, wu64, wd64, idx_np[toks].astype(np.int32), dev["gval"], dev["uval"], dD64s,
-                       want=("x",))
+                       F=w.d_ff, want=("x",))
     parity.assert_close(syn.to_f64(grads["grad_x"][toks]), ref["grad_x"], w.dtype, "grad_x (sampled tokens)")
-    rows = np.sort(rng.choice(w.d_ff, 24, replace=False)).astype(np.int32)
+    rows = np.sort(rng.choice(w.d_ff, n_rows, replace=False)).astype(np.int32)
     wrows = orc.backward_weight_rows(syn.to_f64(x), wd64, idx_np.astype(np.int32), syn.to_f64(tg), syn.to_f64(tu),
                                      syn.to_f64(dD), rows, w.d_ff)
     for name in ("grad_w_gate", "grad_w_up", "grad_w_down"):
         got = syn.to_f64(grads[name][torch.from_numpy(rows.astype(np.int64)).cuda()])
         parity.assert_close(got, wrows[name], w.dtype, name + " (sampled rows)")
+        if w.d_ff_ld > w.d_ff:   # padding rows of the weight gradients stay exactly zero
+            assert torch.all(grads[name][w.d_ff:] == 0), name
     # structural properties at full size
     parity.check_index_sets(idx_np, w.d_ff)
+
+
+def test_full_size_bench_workload_sampled_against_oracle():
+    """C2 at its full 16384 tokens, in the configuration bench.py times: sampled tokens of out / saved values /
+    grad_x and sampled rows of the weight gradients are recomputed one by one by the oracle."""
+    _full_size_sampled(syn.C2, 96, 24)
+
+
+def test_full_size_llama1b_padded_sampled_against_oracle():
+    """C3 at its full 32768 tokens (d_ff = 5461 in arrays of 5504 rows): the same sampled comparison."""
+    _full_size_sampled(syn.C3, 64, 16)
+
+
+@pytest.mark.parametrize("K", [344, 1376])
+def test_full_size_sweep_workload_sampled_against_oracle(K):
+    """C5 at its full 65536 tokens with the smallest and the largest K of the sweep (d_ff / 16 and d_ff / 4)."""
+    import dataclasses
+    _full_size_sampled(dataclasses.replace(syn.C5, k=K, name=f"C5-k{K}"), 32, 8)
