@@ -273,7 +273,7 @@ def test_decode_small_shapes(dtype, T, d, F, K):
     _check_decode(syn.to_f64(out_f), x64, wg64, wu64, wd64, K, dtype, "forward(save=False)")
 
 
-# ------------------------------------------------------------------ tensor-core plan (bf16, tokens >= 256)
+# ------------------------------------------------------------------ tensor-core plan (bf16)
 
 
 @pytest.mark.parametrize("T,d,F,F_ld,K", [
@@ -284,6 +284,12 @@ def test_decode_small_shapes(dtype, T, d, F, K):
 ])
 def test_tc_plan_shapes(T, d, F, F_ld, K):
     w = syn.Workload(f"tc-{T}-{d}-{F}-{K}", "bf16", T, d, F, F_ld, K, seed=200 + T)
+    _run_forward_backward(w)
+
+
+def test_bf16_rows_too_long_for_the_tensor_core_selector_take_the_gathered_plan():
+    """(d_ff + k) * 4 bytes beyond the selector's shared memory: bf16 falls back to the exact gathered kernels."""
+    w = syn.Workload("bf16-gathered", "bf16", 5, 64, 32768, 32768, 11008, seed=77)
     _run_forward_backward(w)
 
 
