@@ -190,7 +190,7 @@ __device__ __forceinline__ void cluster_sync_all() {
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
-// tile load whose completion bytes are counted by an mbarrier of the pair's leading CTA (no multicast: every CTA
+// tile load whose completion bytes are counted by an mbarrier of the pair's leading CTA (nothing is broadcast: every CTA
 // fetches its own boxes)
 __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, uint32_t leader_bar, int x, int y) {
     asm volatile(
