@@ -322,8 +322,14 @@ int forward_tc(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat1
     const int nv = ceil_div(F, 128);  // 128-channel groups of a row
     // each warp stages its token's rows in its own slice of shared memory: as many warps per SM as fit, in one
     // or two CTAs
-    const size_t warp_bytes = warp_select_words(nv, K) * sizeof(uint32_t);
-    const int warps_per_sm = (int)std::min<size_t>((size_t)220 * 1024 / warp_bytes, 2 * kWarpSelMaxWarps);
+    // (rows too long for that with separate gate and up buffers let the two rows share one buffer)
+    const auto warps_fit = [&](bool shared) {
+        return (int)std::min<size_t>((size_t)220 * 1024 / (warp_select_words(nv, K, shared) * sizeof(uint32_t)),
+                                     2 * kWarpSelMaxWarps);
+    };
+    const bool sel_shared_u = warps_fit(false) < 4 && warp_select_parks_gates(nv, K) && warps_fit(true) >= 4;
+    const size_t warp_bytes = warp_select_words(nv, K, sel_shared_u) * sizeof(uint32_t);
+    const int warps_per_sm = warps_fit(sel_shared_u);
     const int sel_ctas_per_sm = warps_per_sm > kWarpSelMaxWarps ? 2 : 1;
     const int sel_wpc = warps_per_sm / sel_ctas_per_sm;
     const size_t warp_smem = (size_t)sel_wpc * warp_bytes;
@@ -332,12 +338,16 @@ int forward_tc(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat1
     float *hint = reinterpret_cast<float *>(ws + L.off_hint);
     int rc = MOC_OK;
     if (warp_select) {
-        switch (nv) {
-            case 8: rc = set_smem(select_mask_rows_warp_kernel<8>, warp_smem, 2048); break;
-            case 16: rc = set_smem(select_mask_rows_warp_kernel<16>, warp_smem, 2048); break;
-            case 32: rc = set_smem(select_mask_rows_warp_kernel<32>, warp_smem, 2048); break;
-            case 43: rc = set_smem(select_mask_rows_warp_kernel<43>, warp_smem, 2048); break;
-            default: rc = set_smem(select_mask_rows_warp_kernel<0>, warp_smem, 2048); break;
+        if (sel_shared_u) {
+            rc = set_smem(select_mask_rows_warp_kernel<0, true>, warp_smem, 2048);
+        } else {
+            switch (nv) {
+                case 8: rc = set_smem(select_mask_rows_warp_kernel<8, false>, warp_smem, 2048); break;
+                case 16: rc = set_smem(select_mask_rows_warp_kernel<16, false>, warp_smem, 2048); break;
+                case 32: rc = set_smem(select_mask_rows_warp_kernel<32, false>, warp_smem, 2048); break;
+                case 43: rc = set_smem(select_mask_rows_warp_kernel<43, false>, warp_smem, 2048); break;
+                default: rc = set_smem(select_mask_rows_warp_kernel<0, false>, warp_smem, 2048); break;
+            }
         }
     } else {
         rc = set_smem(select_mask_rows_kernel, cta_smem);
@@ -389,16 +399,20 @@ int forward_tc(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat1
         if (warp_select) {
             const unsigned grid =
                 (unsigned)std::min<int64_t>((n + sel_wpc - 1) / sel_wpc, (int64_t)sm_count() * sel_ctas_per_sm);
-#define MOC_WARP_SELECT(NV)                                                                    \
-    MOC_LAUNCH(KID_TC_SELECT_MASK, st,                                                         \
-               (select_mask_rows_warp_kernel<NV><<<grid, sel_wpc * 32, warp_smem, st>>>(       \
+#define MOC_WARP_SELECT(NV, SHARED)                                                                    \
+    MOC_LAUNCH(KID_TC_SELECT_MASK, st,                                                                 \
+               (select_mask_rows_warp_kernel<NV, SHARED><<<grid, sel_wpc * 32, warp_smem, st>>>(       \
                    G, L.ldf, Uc, L.ldf, n, F, nv, K, o_idx, o_g, o_u, meta, status)))
-            switch (nv) {  // the usual row lengths get their loops unrolled
-                case 8: MOC_WARP_SELECT(8); break;
-                case 16: MOC_WARP_SELECT(16); break;
-                case 32: MOC_WARP_SELECT(32); break;
-                case 43: MOC_WARP_SELECT(43); break;
-                default: MOC_WARP_SELECT(0); break;
+            if (sel_shared_u) {
+                MOC_WARP_SELECT(0, true);
+            } else {
+                switch (nv) {  // the usual row lengths get their loops unrolled
+                    case 8: MOC_WARP_SELECT(8, false); break;
+                    case 16: MOC_WARP_SELECT(16, false); break;
+                    case 32: MOC_WARP_SELECT(32, false); break;
+                    case 43: MOC_WARP_SELECT(43, false); break;
+                    default: MOC_WARP_SELECT(0, false); break;
+                }
             }
 #undef MOC_WARP_SELECT
         } else {

@@ -229,9 +229,15 @@ constexpr int kWarpSelMaxWarps = 8;                      // warps per CTA, at mo
 
 // Words of shared memory one warp needs: gate row, up row, parked keys, bitmap, kept list, mbarrier.
 __host__ __device__ constexpr int warp_select_bitmap_words(int nv) { return nv * 4 > kWarpSelWords ? nv * 4 : kWarpSelWords; }
-__host__ __device__ constexpr size_t warp_select_words(int nv, int K) {
-    return (size_t)nv * 128 + (size_t)nv * 64 + warp_select_cand_words(nv) + warp_select_bitmap_words(nv) +
-           (size_t)((K + 3) & ~3) + 4;
+// shared_u: the up row is copied into the gate row's buffer once the gate values are no longer needed there
+// (less shared memory per warp, so longer rows still get several warps per SM; no prefetch of the next gate row)
+__host__ __device__ constexpr size_t warp_select_words(int nv, int K, bool shared_u = false) {
+    return (size_t)nv * 128 + (shared_u ? 0 : (size_t)nv * 64) + warp_select_cand_words(nv) +
+           warp_select_bitmap_words(nv) + (size_t)((K + 3) & ~3) + 4;
+}
+// whether the kept channels' gate values fit the search scratch (see the kernel); shared_u needs it
+__host__ __device__ constexpr bool warp_select_parks_gates(int nv, int K) {
+    return K <= warp_select_cand_words(nv) + warp_select_bitmap_words(nv);
 }
 
 struct SelectMeta {
@@ -305,7 +311,9 @@ __device__ __noinline__ uint32_t warp_select_row_general(const float *g, int F, 
     return res;
 }
 
-template <int NV>  // number of 128-channel groups when known at compile time, 0: taken from nv_runtime
+// NV: number of 128-channel groups when known at compile time, 0: taken from nv_runtime
+// shared_u: one buffer for the gate row and, after step 3, the up row (see warp_select_words)
+template <int NV, bool shared_u>
 __global__ void __launch_bounds__(kWarpSelMaxWarps * 32) select_mask_rows_warp_kernel(
     const float *__restrict__ G, int ldg, __nv_bfloat16 *__restrict__ U, int ldu, int64_t rows, int F, int nv_runtime, int K,
     int16_t *__restrict__ idx_out, __nv_bfloat16 *__restrict__ g_out, __nv_bfloat16 *__restrict__ u_out,
@@ -316,10 +324,10 @@ __global__ void __launch_bounds__(kWarpSelMaxWarps * 32) select_mask_rows_warp_k
     const int nv = NV > 0 ? NV : nv_runtime;
     const int slots = warp_select_slots(nv);
     const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5, wpc = blockDim.x >> 5;
-    uint32_t *base = warp_sel_smem + (size_t)wib * warp_select_words(nv, K);
+    uint32_t *base = warp_sel_smem + (size_t)wib * warp_select_words(nv, K, shared_u);
     float *sg = reinterpret_cast<float *>(base);                                // [nv * 128] gate row
-    __nv_bfloat16 *su = reinterpret_cast<__nv_bfloat16 *>(base + nv * 128);     // [nv * 128] up row -> Z' row
-    uint32_t *cand = base + nv * 128 + nv * 64;                                 // [slot][lane] parked values
+    __nv_bfloat16 *su = reinterpret_cast<__nv_bfloat16 *>(shared_u ? base : base + nv * 128);  // up row -> Z' row
+    uint32_t *cand = base + nv * 128 + (shared_u ? 0 : nv * 64);                                 // [slot][lane] parked values
     uint32_t *bitmap = cand + warp_select_cand_words(nv);                                     // kept-channel bitmap
     uint32_t *kept = bitmap + warp_select_bitmap_words(nv);                                    // [K] channel | z bits << 16
     uint64_t *bar_mem = reinterpret_cast<uint64_t *>(kept + ((K + 3) & ~3));
@@ -327,7 +335,7 @@ __global__ void __launch_bounds__(kWarpSelMaxWarps * 32) select_mask_rows_warp_k
     // the kept channels' gate values are parked in the search scratch (free by then) when it is large enough: the
     // gate buffer can then take the next token's row while this token's values are still being worked on
     float *gkept = reinterpret_cast<float *>(cand);
-    const bool early_gate = K <= warp_select_cand_words(nv) + warp_select_bitmap_words(nv);
+    const bool early_gate = warp_select_parks_gates(nv, K);  // (the host only asks for shared_u when this holds)
     const int64_t gw = (int64_t)blockIdx.x * wpc + wib, nw = (int64_t)gridDim.x * wpc;
     const float b_center = meta.bracket[0], b_width = meta.bracket[1];
     const bool have_bracket = meta.bracket[2] == kBracketTag && b_width > 0.f && fabsf(b_center) <= 3.0e38f;
@@ -348,7 +356,7 @@ __global__ void __launch_bounds__(kWarpSelMaxWarps * 32) select_mask_rows_warp_k
     __syncthreads();
     uint32_t phase = 0;  // both barriers complete once per token
     bool dead = false;
-    if (lane == 0 && gw < rows) {
+    if (lane == 0 && gw < rows && !shared_u) {
         mbar_expect_tx(bar_g, g_bytes);
         bulk_copy_g2s(smem_u32(sg), G + gw * (int64_t)ldg, g_bytes, bar_g);
     }
@@ -357,11 +365,17 @@ __global__ void __launch_bounds__(kWarpSelMaxWarps * 32) select_mask_rows_warp_k
         __nv_bfloat16 *u = U + r * (int64_t)ldu;
         // ---- the up row is needed only in step 4: its copy starts now (once the previous token's store has read
         //      the buffer) and lands while steps 1-3 run; the gate row was requested during the previous token
+        //      (one buffer for both rows: the gate row is requested here and the up row after step 3)
         if (lane == 0) {
             bulk_store_wait_read<0>();
             fence_async_smem();
-            mbar_expect_tx(bar_u, u_bytes);
-            bulk_copy_g2s(smem_u32(su), u, u_bytes, bar_u);
+            if (shared_u) {
+                mbar_expect_tx(bar_g, g_bytes);
+                bulk_copy_g2s(smem_u32(sg), G + r * (int64_t)ldg, g_bytes, bar_g);
+            } else {
+                mbar_expect_tx(bar_u, u_bytes);
+                bulk_copy_g2s(smem_u32(su), u, u_bytes, bar_u);
+            }
         }
         if (!__all_sync(0xffffffffu, mbar_wait(bar_g, phase, &s_abort, status))) {
             dead = true;
@@ -519,7 +533,13 @@ __global__ void __launch_bounds__(kWarpSelMaxWarps * 32) select_mask_rows_warp_k
         if (early_gate) {
             for (int i = lane; i < K; i += 32) gkept[i] = sg[kept[i]];
             __syncwarp();
-            request_next_gate();
+            if (!shared_u) {
+                request_next_gate();
+            } else if (lane == 0) {
+                fence_async_smem();
+                mbar_expect_tx(bar_u, u_bytes);
+                bulk_copy_g2s(smem_u32(su), u, u_bytes, bar_u);
+            }
         }
         if (!__all_sync(0xffffffffu, mbar_wait(bar_u, phase, &s_abort, status))) {
             dead = true;
