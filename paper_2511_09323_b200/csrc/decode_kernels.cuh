@@ -165,6 +165,21 @@ __global__ void __launch_bounds__(kGemvThreads, 2) gemv_rows_kernel(const __nv_b
             if (blockIdx.x == 0)
                 for (int i = tid; i <= slices; i += 256) ws.counters[i] = 0;  // [slices]: arrivals of the select kernel
         }
+        // gathering: the factor SiLU(g) of every output this thread will write (0 where the token did not select
+        // the channel) is fetched now, so that the loads are long done when the sums are ready
+        const int width = r1 - r0;
+        float sfac[4] = {0.f, 0.f, 0.f, 0.f};  // 16 tokens x at most 64 rows / 256 threads
+        if (GATHER) {
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int o = tid + 256 * k;
+                if (o < 16 * width) {
+                    const int t = o / width, j = s_rows[o - t * width];
+                    if (t < T && ((ws.sel_bits[t * ws.sel_words + (j >> 5)] >> (j & 31)) & 1u))
+                        sfac[k] = silu_f(ws.G[(int64_t)t * ws.ldf + j]);
+                }
+            }
+        }
         const int g = lane >> 2, q = lane & 3;
         const __nv_bfloat16 *xa_row = x + (int64_t)g * d, *xb_row = x + (int64_t)(g + 8) * d;
         const bool has_a = g < T, has_b = g + 8 < T;
@@ -223,21 +238,20 @@ __global__ void __launch_bounds__(kGemvThreads, 2) gemv_rows_kernel(const __nv_b
         }
         consumer_bar_sync();
         ok = ok && !s_abort;
-        const int width = r1 - r0;
-        for (int o = tid; ok && o < 16 * width; o += 256) {
-            const int t = o / width, c = o - t * width;
-            const int slot = r0 + c;
-            float sum = 0.f;
 #pragma unroll
-            for (int wi = 0; wi < 8; ++wi) sum += red[(wi * 16 + t) * RP + c];
-            if (!GATHER) {
-                if (t < T) ws.G[(int64_t)t * ws.ldf + slot] = sum;
-            } else {
-                const int j = s_rows[c];
-                float z = 0.f;
-                if (t < T && ((ws.sel_bits[t * ws.sel_words + (j >> 5)] >> (j & 31)) & 1u))
-                    z = silu_f(ws.G[(int64_t)t * ws.ldf + j]) * sum;
-                ws.Zb[((int64_t)(slot >> 4) * 16 + t) * 16 + (slot & 15)] = __float2bfloat16_rn(z);
+        for (int k = 0; k < 4; ++k) {
+            const int o = tid + 256 * k;
+            if (ok && o < 16 * width) {
+                const int t = o / width, c = o - t * width;
+                const int slot = r0 + c;
+                float sum = 0.f;
+#pragma unroll
+                for (int wi = 0; wi < 8; ++wi) sum += red[(wi * 16 + t) * RP + c];
+                if (!GATHER) {
+                    if (t < T) ws.G[(int64_t)t * ws.ldf + slot] = sum;
+                } else {
+                    ws.Zb[((int64_t)(slot >> 4) * 16 + t) * 16 + (slot & 15)] = __float2bfloat16_rn(sfac[k] * sum);
+                }
             }
         }
     }
