@@ -322,23 +322,41 @@ int forward_tc(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat1
     const int nv = ceil_div(F, 128);  // 128-channel groups of a row
     // each warp stages its token's rows in its own slice of shared memory: as many warps per SM as fit, in one
     // or two CTAs
-    // (rows too long for that with separate gate and up buffers let the two rows share one buffer)
-    const auto warps_fit = [&](bool shared) {
-        return (int)std::min<size_t>((size_t)220 * 1024 / (warp_select_words(nv, K, shared) * sizeof(uint32_t)),
-                                     2 * kWarpSelMaxWarps);
+    // (rows too long for that with separate gate and up buffers let the two rows share one buffer).  Two warps
+    // work on a token (MOC_FFN_SELECT=warp in the environment: one warp per token, kept for comparison).
+    static const bool sel_pairs = !(getenv("MOC_FFN_SELECT") && strcmp(getenv("MOC_FFN_SELECT"), "warp") == 0);
+    const auto units_fit = [&](bool shared) {  // tokens in flight per SM
+        const size_t words = sel_pairs ? pair_select_words(nv, K, shared) : warp_select_words(nv, K, shared);
+        return (int)std::min<size_t>((size_t)220 * 1024 / (words * sizeof(uint32_t)), 16);
     };
-    const bool sel_shared_u = warps_fit(false) < 4 && warp_select_parks_gates(nv, K) && warps_fit(true) >= 4;
-    const size_t warp_bytes = warp_select_words(nv, K, sel_shared_u) * sizeof(uint32_t);
-    const int warps_per_sm = warps_fit(sel_shared_u);
-    const int sel_ctas_per_sm = warps_per_sm > kWarpSelMaxWarps ? 2 : 1;
-    const int sel_wpc = warps_per_sm / sel_ctas_per_sm;
+    const bool parks = sel_pairs ? pair_select_parks_gates(nv, K) : warp_select_parks_gates(nv, K);
+    const int min_units = sel_pairs ? 2 : 4;  // at least four warps per SM
+    const bool sel_shared_u = units_fit(false) < min_units && parks && units_fit(true) >= min_units;
+    const size_t warp_bytes = (sel_pairs ? pair_select_words(nv, K, sel_shared_u) : warp_select_words(nv, K, sel_shared_u)) *
+                              sizeof(uint32_t);
+    const int warps_per_sm = units_fit(sel_shared_u);  // tokens in flight per SM (a warp or a pair of warps each)
+    const int sel_units_per_cta = sel_pairs ? kPairSelMaxWarps / 2 : kWarpSelMaxWarps;
+    const int sel_ctas_per_sm = warps_per_sm > sel_units_per_cta ? 2 : 1;
+    const int sel_wpc = std::min(warps_per_sm / sel_ctas_per_sm, sel_units_per_cta);  // tokens per CTA
     const size_t warp_smem = (size_t)sel_wpc * warp_bytes;
     const size_t cta_smem = ((size_t)F + K) * sizeof(uint32_t);
-    const bool warp_select = warps_per_sm >= 4;
+    const bool warp_select = warps_per_sm >= min_units;
     float *hint = reinterpret_cast<float *>(ws + L.off_hint);
     int rc = MOC_OK;
     if (warp_select) {
-        if (sel_shared_u) {
+        if (sel_pairs) {
+            if (sel_shared_u) {
+                rc = set_smem(select_mask_rows_pair_kernel<0, true>, warp_smem, 2048);
+            } else {
+                switch (nv) {
+                    case 8: rc = set_smem(select_mask_rows_pair_kernel<8, false>, warp_smem, 2048); break;
+                    case 16: rc = set_smem(select_mask_rows_pair_kernel<16, false>, warp_smem, 2048); break;
+                    case 32: rc = set_smem(select_mask_rows_pair_kernel<32, false>, warp_smem, 2048); break;
+                    case 43: rc = set_smem(select_mask_rows_pair_kernel<43, false>, warp_smem, 2048); break;
+                    default: rc = set_smem(select_mask_rows_pair_kernel<0, false>, warp_smem, 2048); break;
+                }
+            }
+        } else if (sel_shared_u) {
             rc = set_smem(select_mask_rows_warp_kernel<0, true>, warp_smem, 2048);
         } else {
             switch (nv) {
@@ -399,21 +417,28 @@ int forward_tc(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat1
         if (warp_select) {
             const unsigned grid =
                 (unsigned)std::min<int64_t>((n + sel_wpc - 1) / sel_wpc, (int64_t)sm_count() * sel_ctas_per_sm);
-#define MOC_WARP_SELECT(NV, SHARED)                                                                    \
-    MOC_LAUNCH(KID_TC_SELECT_MASK, st,                                                                 \
-               (select_mask_rows_warp_kernel<NV, SHARED><<<grid, sel_wpc * 32, warp_smem, st>>>(       \
+#define MOC_WARP_SELECT(KERNEL, NV, SHARED, THREADS_PER_TOKEN)                                               \
+    MOC_LAUNCH(KID_TC_SELECT_MASK, st,                                                                          \
+               (KERNEL<NV, SHARED><<<grid, sel_wpc * THREADS_PER_TOKEN, warp_smem, st>>>(                        \
                    G, L.ldf, Uc, L.ldf, n, F, nv, K, o_idx, o_g, o_u, meta, status)))
-            if (sel_shared_u) {
-                MOC_WARP_SELECT(0, true);
+#define MOC_SELECT_BY_WIDTH(KERNEL, TPT)                                       \
+    if (sel_shared_u) {                                                        \
+        MOC_WARP_SELECT(KERNEL, 0, true, TPT);                                 \
+    } else {                                                                   \
+        switch (nv) { /* the usual row lengths get their loops unrolled */     \
+            case 8: MOC_WARP_SELECT(KERNEL, 8, false, TPT); break;             \
+            case 16: MOC_WARP_SELECT(KERNEL, 16, false, TPT); break;           \
+            case 32: MOC_WARP_SELECT(KERNEL, 32, false, TPT); break;           \
+            case 43: MOC_WARP_SELECT(KERNEL, 43, false, TPT); break;           \
+            default: MOC_WARP_SELECT(KERNEL, 0, false, TPT); break;            \
+        }                                                                      \
+    }
+            if (sel_pairs) {
+                MOC_SELECT_BY_WIDTH(select_mask_rows_pair_kernel, 64)
             } else {
-                switch (nv) {  // the usual row lengths get their loops unrolled
-                    case 8: MOC_WARP_SELECT(8, false); break;
-                    case 16: MOC_WARP_SELECT(16, false); break;
-                    case 32: MOC_WARP_SELECT(32, false); break;
-                    case 43: MOC_WARP_SELECT(43, false); break;
-                    default: MOC_WARP_SELECT(0, false); break;
-                }
+                MOC_SELECT_BY_WIDTH(select_mask_rows_warp_kernel, 32)
             }
+#undef MOC_SELECT_BY_WIDTH
 #undef MOC_WARP_SELECT
         } else {
             const unsigned grid = (unsigned)std::min<int64_t>(n, (int64_t)sm_count() * 6);

@@ -630,6 +630,353 @@ __global__ void __launch_bounds__(kWarpSelMaxWarps * 32) select_mask_rows_warp_k
 }
 
 // ------------------------------------------------------------------------------------------------
+// The same selector with TWO WARPS per token (same staging, same steps, same exactness): the pair shares one
+// slice of shared memory, each warp takes every other 128-channel group in steps 1 and 3 and half of the kept
+// channels in step 4, and the two meet at a named barrier of their own between the steps.  A token's rows
+// occupy the slice for about half as long, so the shared memory of an SM (which bounds the tokens in flight)
+// feeds twice as many warps.
+__host__ __device__ constexpr size_t pair_select_words(int nv, int K, bool shared_u) {
+    return (size_t)nv * 128 + (shared_u ? 0 : (size_t)nv * 64) + 2 * (size_t)warp_select_cand_words(nv) +
+           warp_select_bitmap_words(nv) + (size_t)((K + 3) & ~3) + 16 /* exchange */ + 4 /* two mbarriers */;
+}
+__host__ __device__ constexpr bool pair_select_parks_gates(int nv, int K) {
+    return K <= 2 * warp_select_cand_words(nv) + warp_select_bitmap_words(nv);
+}
+constexpr int kPairSelMaxWarps = 12;  // warps per CTA, at most (six pairs: named barriers 1..6; two CTAs per SM)
+
+template <int NV, bool shared_u>
+__global__ void __launch_bounds__(kPairSelMaxWarps * 32, 2) select_mask_rows_pair_kernel(
+    const float *__restrict__ G, int ldg, __nv_bfloat16 *__restrict__ U, int ldu, int64_t rows, int F, int nv_runtime, int K,
+    int16_t *__restrict__ idx_out, __nv_bfloat16 *__restrict__ g_out, __nv_bfloat16 *__restrict__ u_out,
+    SelectMeta meta, int *status) {
+    extern __shared__ __align__(128) uint32_t warp_sel_smem[];
+    __shared__ float s_stat[kPairSelMaxWarps / 2][3];
+    __shared__ int s_abort;
+    const int nv = NV > 0 ? NV : nv_runtime;
+    const int slots = warp_select_slots(nv), cw = warp_select_cand_words(nv);
+    const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5, ppc = blockDim.x >> 6;  // pairs per CTA
+    const int pair = wib >> 1, w = wib & 1, pl = (w << 5) | lane;                      // pl: 0..63 within the pair
+    uint32_t *base = warp_sel_smem + (size_t)pair * pair_select_words(nv, K, shared_u);
+    float *sg = reinterpret_cast<float *>(base);
+    __nv_bfloat16 *su = reinterpret_cast<__nv_bfloat16 *>(shared_u ? base : base + nv * 128);
+    uint32_t *cand0 = base + nv * 128 + (shared_u ? 0 : nv * 64);  // [2 warps][slot][lane] parked values
+    uint32_t *cand = cand0 + w * cw;
+    uint32_t *bitmap = cand0 + 2 * cw;
+    uint32_t *kept = bitmap + warp_select_bitmap_words(nv);
+    uint32_t *xch = kept + ((K + 3) & ~3);  // [2 parities][2 warps][4] counts exchanged between the warps
+    uint64_t *bar_mem = reinterpret_cast<uint64_t *>(xch + 16);
+    const uint32_t bar_g = smem_u32(bar_mem), bar_u = smem_u32(bar_mem + 1);
+    float *gkept = reinterpret_cast<float *>(cand0);
+    const bool early_gate = pair_select_parks_gates(nv, K);
+    auto pair_sync = [&]() { asm volatile("bar.sync %0, 64;" ::"r"(pair + 1) : "memory"); };
+    const int64_t gp = (int64_t)blockIdx.x * ppc + pair, np = (int64_t)gridDim.x * ppc;
+    const float b_center = meta.bracket[0], b_width = meta.bracket[1];
+    const bool have_bracket = meta.bracket[2] == kBracketTag && b_width > 0.f && fabsf(b_center) <= 3.0e38f;
+    float cen = b_center, wid = b_width;
+    bool have = have_bracket;
+    float st_sum = 0.f, st_abs = 0.f, st_n = 0.f;
+    const int words = (F + 31) >> 5;
+    const uint32_t g_bytes = (uint32_t)ldg * 4u, u_bytes = (uint32_t)ldu * 2u;
+
+    if (threadIdx.x == 0) s_abort = 0;
+    if (pl == 0) {
+        mbar_init(bar_g, 1);
+        mbar_init(bar_u, 1);
+    }
+    for (int c = ldg + pl; c < nv * 128; c += 64) sg[c] = -INFINITY;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    __syncthreads();
+    uint32_t phase = 0;
+    int xp = 0;  // parity of the exchange slot in use
+    bool dead = false;
+    if (pl == 0 && gp < rows && !shared_u) {
+        mbar_expect_tx(bar_g, g_bytes);
+        bulk_copy_g2s(smem_u32(sg), G + gp * (int64_t)ldg, g_bytes, bar_g);
+    }
+    // both warps of a pair take every branch below together: all conditions come from values they share
+
+    for (int64_t r = gp; r < rows && !dead; r += np) {
+        __nv_bfloat16 *u = U + r * (int64_t)ldu;
+        if (pl == 0) {
+            bulk_store_wait_read<0>();
+            fence_async_smem();
+            if (shared_u) {
+                mbar_expect_tx(bar_g, g_bytes);
+                bulk_copy_g2s(smem_u32(sg), G + r * (int64_t)ldg, g_bytes, bar_g);
+            } else {
+                mbar_expect_tx(bar_u, u_bytes);
+                bulk_copy_g2s(smem_u32(su), u, u_bytes, bar_u);
+            }
+        }
+        if (!__all_sync(0xffffffffu, mbar_wait(bar_g, phase, &s_abort, status))) dead = true;
+        if (!dead)
+            for (int c = F + pl; c < ldg; c += 64) sg[c] = -INFINITY;
+        // the partner must see the same verdict: a failed wait ends the pair (s_abort is set block-wide)
+        pair_sync();
+        if (s_abort) dead = true;
+        if (dead) break;
+
+        uint32_t tau = 0, res = 0;
+        bool fast = false, settled = false, no_cut = false;
+        float lo_f = cen - wid, hi_f = cen + wid;
+        for (int attempt = 0; have && attempt < 8; ++attempt) {
+            // ---- 1. classify: this warp's groups v = w, w + 2, ...
+            uint32_t n_above = 0, n_mine = 0;
+#pragma unroll 4
+            for (int v = w; v < nv; v += 2) {
+                const float4 q = *reinterpret_cast<const float4 *>(sg + (v * 32 + lane) * 4);
+                const float e4[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float x = e4[e];
+                    n_above += x > hi_f ? 1u : 0u;
+                    const bool inside = x >= lo_f && x <= hi_f;
+                    if (inside) cand[min(n_mine, (uint32_t)slots) * 32 + lane] = __float_as_uint(x);
+                    n_mine += inside ? 1u : 0u;
+                }
+            }
+            const uint32_t my_hi = __reduce_add_sync(0xffffffffu, n_above);
+            const uint32_t my_band = __reduce_add_sync(0xffffffffu, n_mine);
+            const uint32_t my_max = __reduce_max_sync(0xffffffffu, n_mine);
+            uint32_t *xs = xch + xp * 8;
+            xp ^= 1;
+            if (lane == 0) {
+                xs[w * 4 + 0] = my_hi;
+                xs[w * 4 + 1] = my_band;
+                xs[w * 4 + 2] = my_max;
+            }
+            // scratch of the search, cleared here so that the barrier below also publishes it
+            uint32_t *hist = bitmap, *list = bitmap + 64, *list_n = bitmap + 96;
+            hist[pl] = 0u;
+            if (pl == 0) *list_n = 0u;
+            pair_sync();
+            const uint32_t c_hi = xs[0] + xs[4], n_band = xs[1] + xs[5], max_mine = max(xs[2], xs[6]);
+            if (max_mine > (uint32_t)slots) {  // too many values inside: halve the bracket
+                const float c = 0.5f * (lo_f + hi_f), wd = 0.25f * (hi_f - lo_f);
+                lo_f = c - wd;
+                hi_f = c + wd;
+                continue;
+            }
+            if (c_hi >= (uint32_t)K) {
+                const float wd = hi_f - lo_f;
+                lo_f = hi_f;
+                hi_f += 2.f * wd;
+                continue;
+            }
+            if (c_hi + n_band < (uint32_t)K) {
+                const float wd = hi_f - lo_f;
+                hi_f = lo_f;
+                lo_f -= 2.f * wd;
+                continue;
+            }
+            // ---- 2. histogram of both warps' parked keys, bin of the m-th largest, exact ranking inside it
+            //         (both warps compute the scan and the ranking: same inputs, same result, no exchange)
+            const uint32_t lo_k = gate_key(lo_f), hi_k = gate_key(hi_f);
+            const uint32_t m = (uint32_t)K - c_hi;
+            const uint32_t span = hi_k - lo_k;
+            const int shift = max(0, 26 - __clz(span | 1u));
+            for (uint32_t s = 0; s < n_mine; ++s) {
+                const uint32_t key = gate_key(__uint_as_float(cand[s * 32 + lane]));
+                atomicAdd(&hist[(key - lo_k) >> shift], 1u);
+            }
+            pair_sync();
+            const uint32_t h0 = hist[2 * lane], h1 = hist[2 * lane + 1], tot = h0 + h1;
+            uint32_t suf = tot;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t nb = __shfl_down_sync(0xffffffffu, suf, o);
+                if (lane + o < 32) suf += nb;
+            }
+            const uint32_t above = suf - tot;
+            const bool f1 = above < m && m <= above + h1, f0 = above + h1 < m && m <= above + tot;
+            const int src = __ffs(__ballot_sync(0xffffffffu, f0 || f1)) - 1;
+            const uint32_t tbin = __shfl_sync(0xffffffffu, (uint32_t)(2 * lane + (f1 ? 1 : 0)), src);
+            const uint32_t m2 = m - __shfl_sync(0xffffffffu, f1 ? above : above + h1, src);
+            const uint32_t nbin = __shfl_sync(0xffffffffu, f1 ? h1 : h0, src);
+            if (nbin <= 32u) {
+                for (uint32_t s = 0; s < n_mine; ++s) {
+                    const uint32_t key = gate_key(__uint_as_float(cand[s * 32 + lane]));
+                    if (((key - lo_k) >> shift) == tbin) list[atomicAdd(list_n, 1u)] = key;
+                }
+                pair_sync();
+                const uint32_t mykey = (uint32_t)lane < nbin ? list[lane] : 0u;
+                uint32_t n_gt = 0, n_eq = 0;
+                for (uint32_t i = 0; i < nbin; ++i) {
+                    const uint32_t o = list[i];
+                    n_gt += o > mykey ? 1u : 0u;
+                    n_eq += o == mykey ? 1u : 0u;
+                }
+                const bool is_tau = (uint32_t)lane < nbin && n_gt < m2 && m2 <= n_gt + n_eq;
+                const int tl = __ffs(__ballot_sync(0xffffffffu, is_tau)) - 1;
+                res = __shfl_sync(0xffffffffu, mykey, tl);
+                no_cut = __shfl_sync(0xffffffffu, n_gt + n_eq, tl) == m2;
+                settled = true;
+            }
+            break;
+        }
+        pair_sync();  // the search scratch is about to become the bitmap
+        const float tau_f = key_to_float(res);
+        if (settled && no_cut && fabsf(tau_f) <= 3.0e38f) {
+            // ---- 3. kept set = {g >= tau}: each warp writes the bitmap words of its own groups
+            for (int v = w; v < nv; v += 2)
+                if (lane < 4 && v * 4 + lane < warp_select_bitmap_words(nv)) bitmap[v * 4 + lane] = 0u;
+            __syncwarp();
+#pragma unroll 4
+            for (int v = w; v < nv; v += 2) {
+                const float4 q = *reinterpret_cast<const float4 *>(sg + (v * 32 + lane) * 4);
+                const uint32_t nib = (q.x >= tau_f ? 1u : 0u) | (q.y >= tau_f ? 2u : 0u) |
+                                     (q.z >= tau_f ? 4u : 0u) | (q.w >= tau_f ? 8u : 0u);
+                if (nib) atomicOr(&bitmap[v * 4 + (lane >> 3)], nib << ((lane & 7) * 4));
+            }
+            pair_sync();
+            // enumerate in ascending channel order: thread pl of the pair owns words [pl*wpl, (pl+1)*wpl)
+            const int wpl = (words + 63) >> 6;
+            uint32_t mine = 0;
+            for (int i = 0; i < wpl; ++i) {
+                const int wd = pl * wpl + i;
+                mine += wd < words ? (uint32_t)__popc(bitmap[wd]) : 0u;
+            }
+            uint32_t pre = mine;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t nb = __shfl_up_sync(0xffffffffu, pre, o);
+                if (lane >= o) pre += nb;
+            }
+            uint32_t *xs = xch + xp * 8;
+            xp ^= 1;
+            if (lane == 31) xs[w * 4 + 3] = pre;  // this warp's total
+            pair_sync();
+            const uint32_t tot0 = xs[3], tot1 = xs[7];
+            if (tot0 + tot1 == (uint32_t)K) {  // counts and compares agree
+                uint32_t pos = pre - mine + (w ? tot0 : 0u);
+                for (int i = 0; i < wpl; ++i) {
+                    const int wd = pl * wpl + i;
+                    uint32_t bits = wd < words ? bitmap[wd] : 0u;
+                    while (bits) {
+                        const int b = __ffs(bits) - 1;
+                        bits &= bits - 1u;
+                        kept[pos++] = (uint32_t)(wd * 32 + b);
+                    }
+                }
+                tau = res;
+                fast = true;
+            }
+        }
+        pair_sync();
+        if (!fast) {
+            // general exact path (rare): one warp works on the whole row, its partner waits
+            if (w == 0) {
+                const uint32_t t0 = warp_select_row_general(sg, F, K, cand0, kept);
+                if (lane == 0) xch[0] = t0;
+            }
+            xp = 0;
+            pair_sync();
+            tau = xch[0];
+            pair_sync();
+        }
+        // ---- 4. values of the kept channels, entries pl, pl + 64, ...
+        auto request_next_gate = [&]() {
+            if (pl == 0 && r + np < rows) {
+                fence_async_smem();
+                mbar_expect_tx(bar_g, g_bytes);
+                bulk_copy_g2s(smem_u32(sg), G + (r + np) * (int64_t)ldg, g_bytes, bar_g);
+            }
+        };
+        if (early_gate) {
+            for (int i = pl; i < K; i += 64) gkept[i] = sg[kept[i]];
+            pair_sync();
+            if (!shared_u) {
+                request_next_gate();
+            } else if (pl == 0) {
+                fence_async_smem();
+                mbar_expect_tx(bar_u, u_bytes);
+                bulk_copy_g2s(smem_u32(su), u, u_bytes, bar_u);
+            }
+        }
+        if (!__all_sync(0xffffffffu, mbar_wait(bar_u, phase, &s_abort, status))) dead = true;
+        pair_sync();
+        if (s_abort) dead = true;
+        if (dead) break;
+        phase ^= 1u;
+        for (int i = pl; i < K; i += 64) {
+            const uint32_t j = kept[i];
+            const float gval = early_gate ? gkept[i] : sg[j];
+            const __nv_bfloat16 ub = su[j];
+            const __nv_bfloat16 zb = __float2bfloat16_rn(silu_f(gval) * __bfloat162float(ub));
+            kept[i] = j | ((uint32_t)(*reinterpret_cast<const uint16_t *>(&zb)) << 16);
+            if (idx_out) {
+                idx_out[r * K + i] = (int16_t)j;
+                g_out[r * K + i] = __float2bfloat16_rn(gval);
+                u_out[r * K + i] = ub;
+            }
+        }
+        pair_sync();
+        if (!early_gate) request_next_gate();
+        // ---- up row -> masked Z' row, in shared memory, then one bulk store
+        uint4 *row16 = reinterpret_cast<uint4 *>(su);
+        for (int i = pl; i < (ldu >> 3); i += 64) row16[i] = make_uint4(0, 0, 0, 0);
+        pair_sync();
+        for (int i = pl; i < K; i += 64) {
+            const uint32_t e = kept[i];
+            const uint16_t zb = (uint16_t)(e >> 16);
+            su[e & 0xffffu] = *reinterpret_cast<const __nv_bfloat16 *>(&zb);
+        }
+        fence_async_smem();
+        pair_sync();
+        if (pl == 0) bulk_copy_s2g(u, smem_u32(su), u_bytes);
+        // ---- statistics for the next launch's bracket (kept by both warps, published by the first)
+        const float t = key_to_float(tau);
+        if (fabsf(t) <= 3.0e38f) {
+            st_sum += t;
+            st_abs += have_bracket ? fabsf(t - b_center) : 0.f;
+            st_n += 1.f;
+            if (!have) {
+                cen = t;
+                wid = 0.15f * fabsf(t) + 1e-30f;
+                have = true;
+            }
+        }
+    }
+    if (pl == 0) bulk_store_wait_all();
+    if (pl == 0) {
+        s_stat[pair][0] = st_sum;
+        s_stat[pair][1] = st_abs;
+        s_stat[pair][2] = st_n;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float a = 0.f, b = 0.f, c = 0.f;
+        for (int i = 0; i < ppc; ++i) {
+            a += s_stat[i][0];
+            b += s_stat[i][1];
+            c += s_stat[i][2];
+        }
+        if (c > 0.f) {
+            atomicAdd(&meta.acc[0], a);
+            atomicAdd(&meta.acc[1], b);
+            atomicAdd(&meta.acc[2], c);
+        }
+        __threadfence();
+        if (atomicInc(meta.done, gridDim.x - 1) == gridDim.x - 1) {
+            __threadfence();
+            const float sum = atomicAdd(&meta.acc[0], 0.f), dev = atomicAdd(&meta.acc[1], 0.f),
+                        n = atomicAdd(&meta.acc[2], 0.f);
+            if (n > 0.f) {
+                const float center = sum / n;
+                float width = have_bracket ? 5.0f * dev / n : 0.15f * fabsf(center);
+                width = fmaxf(width, 0.02f * fabsf(center) + 1e-30f);
+                meta.bracket[0] = center;
+                meta.bracket[1] = width;
+                meta.bracket[2] = kBracketTag;
+            } else {
+                meta.bracket[2] = 0.f;
+            }
+            meta.acc[0] = meta.acc[1] = meta.acc[2] = 0.f;
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
 // Forward selector of the tensor-core plan, one CTA per token.
 //   G [rows, ldg] fp32 and U [rows, ldu] bf16 are the dense projections of the token chunk.
 //   Emits idx / g / u of the K kept channels (when saving) and rewrites the token's U row IN PLACE
