@@ -337,6 +337,33 @@ def test_ties_go_to_the_lower_channel_on_both_plans():
         parity.check_forward(dev, x64, wg64, wu64, wd64, w.k, w.d_ff, w.dtype)
 
 
+def test_tc_plan_degenerate_and_badly_scaled_tokens():
+    """Tokens the selector's bracket cannot anticipate: all-zero rows (every gate value ties: channels 0..K-1 are
+    kept), rows scaled by 1e3 and by 1e-3 between ordinary ones (the bracket has to move far and back), and a
+    batch whose first launch has no bracket at all (fresh workspace filled with NaN bytes)."""
+    w = syn.Workload("odd-tokens", "bf16", 600, 256, 2048, 2048, 256, seed=4242)
+    wg, wu, wd = syn.make_weights(w)
+    x = syn.make_x(w).float()
+    x[5::50] = 0.0
+    x[7::50] *= 1.0e3
+    x[11::50] *= 1.0e-3
+    x = x.to(torch.bfloat16)
+    xd, wgd, wud, wdd = map(_dev, (x, wg, wu, wd))
+    desc = B.make_desc(w.tokens, w.d_model, w.d_ff, w.k, xd.dtype)
+    ws = B.alloc_workspace(desc, B.MOC_OP_FORWARD)
+    ws.fill_(0xFF)      # whatever a new workspace holds must not matter
+    for attempt in range(2):   # second call: the bracket left by the first one is in the workspace
+        out, idx, tg, tu = B.moc_ffn_forward(xd, wgd, wud, wdd, w.k, workspace=ws)
+        torch.cuda.synchronize()
+        assert B.moc_last_device_status() == B.MOC_OK
+        idx_np = idx.cpu().numpy().astype(np.int64)
+        for t in range(5, w.tokens, 50):
+            assert np.array_equal(idx_np[t], np.arange(w.k)), f"zero token {t}"
+        x64, wg64, wu64, wd64 = map(syn.to_f64, (x, wg, wu, wd))
+        dev = dict(out=syn.to_f64(out), idx=idx_np, gval=syn.to_f64(tg), uval=syn.to_f64(tu))
+        parity.check_forward(dev, x64, wg64, wu64, wd64, w.k, w.d_ff, w.dtype)
+
+
 def test_tc_plan_backward_options_and_determinism():
     w = syn.Workload("tc-opts", "bf16", 384, 256, 768, 768, 96, seed=41)
     _, (x, wg, wu, wd, dD), (out, idx, tg, tu), full = _run_forward_backward(w)
@@ -430,6 +457,6 @@ def test_one_warp_per_token_selector_selected_by_environment():
     env = dict(os.environ, MOC_FFN_SELECT="warp")
     root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
     r = subprocess.run([sys.executable, "-m", "pytest", os.path.join(root, "tests", "test_gpu_parity.py"), "-q", "-x",
-                        "-m", "gpu", "-k", "tc_plan_shapes or ties_go or several_token_chunks or llama1b_padded_slice"],
+                        "-m", "gpu", "-k", "tc_plan_shapes or ties_go or several_token_chunks or llama1b_padded_slice or degenerate"],
                        cwd=root, env=env, capture_output=True, text=True, timeout=900)
     assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
