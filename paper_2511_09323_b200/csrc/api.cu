@@ -325,17 +325,22 @@ int forward_tc(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat1
     // (rows too long for that with separate gate and up buffers let the two rows share one buffer).  Two warps
     // work on a token (MOC_FFN_SELECT=warp in the environment: one warp per token, kept for comparison).
     static const bool sel_pairs = !(getenv("MOC_FFN_SELECT") && strcmp(getenv("MOC_FFN_SELECT"), "warp") == 0);
+    // teams of four warps for long rows (few tokens fit an SM there), pairs otherwise
+    // (measured: LLaMA-1B width 0.59 -> 0.50 ms and LLaMA-7B width 0.56 -> 0.41 ms with four; 2048 channels 0.080 ->
+    // 0.124 ms, so short rows keep pairs)
+    const int sel_team = nv >= 40 ? 4 : 2;
     const auto units_fit = [&](bool shared) {  // tokens in flight per SM
-        const size_t words = sel_pairs ? pair_select_words(nv, K, shared) : warp_select_words(nv, K, shared);
+        const size_t words = sel_pairs ? pair_select_words(nv, K, shared, sel_team) : warp_select_words(nv, K, shared);
         return (int)std::min<size_t>((size_t)220 * 1024 / (words * sizeof(uint32_t)), 16);
     };
-    const bool parks = sel_pairs ? pair_select_parks_gates(nv, K) : warp_select_parks_gates(nv, K);
+    const bool parks = sel_pairs ? pair_select_parks_gates(nv, K, sel_team) : warp_select_parks_gates(nv, K);
     const int min_units = sel_pairs ? 2 : 4;  // at least four warps per SM
     const bool sel_shared_u = units_fit(false) < min_units && parks && units_fit(true) >= min_units;
-    const size_t warp_bytes = (sel_pairs ? pair_select_words(nv, K, sel_shared_u) : warp_select_words(nv, K, sel_shared_u)) *
-                              sizeof(uint32_t);
+    const size_t warp_bytes =
+        (sel_pairs ? pair_select_words(nv, K, sel_shared_u, sel_team) : warp_select_words(nv, K, sel_shared_u)) *
+        sizeof(uint32_t);
     const int warps_per_sm = units_fit(sel_shared_u);  // tokens in flight per SM (a warp or a pair of warps each)
-    const int sel_units_per_cta = sel_pairs ? kPairSelMaxWarps / 2 : kWarpSelMaxWarps;
+    const int sel_units_per_cta = sel_pairs ? kPairSelMaxWarps / sel_team : kWarpSelMaxWarps;
     const int sel_ctas_per_sm = warps_per_sm > sel_units_per_cta ? 2 : 1;
     const int sel_wpc = std::min(warps_per_sm / sel_ctas_per_sm, sel_units_per_cta);  // tokens per CTA
     const size_t warp_smem = (size_t)sel_wpc * warp_bytes;
@@ -344,16 +349,23 @@ int forward_tc(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat1
     float *hint = reinterpret_cast<float *>(ws + L.off_hint);
     int rc = MOC_OK;
     if (warp_select) {
-        if (sel_pairs) {
+        if (sel_pairs && sel_team == 4) {
             if (sel_shared_u) {
-                rc = set_smem(select_mask_rows_pair_kernel<0, true>, warp_smem, 2048);
+                rc = set_smem(select_mask_rows_pair_kernel<0, true, 4>, warp_smem, 2048);
+            } else if (nv == 43) {
+                rc = set_smem(select_mask_rows_pair_kernel<43, false, 4>, warp_smem, 2048);
+            } else {
+                rc = set_smem(select_mask_rows_pair_kernel<0, false, 4>, warp_smem, 2048);
+            }
+        } else if (sel_pairs) {
+            if (sel_shared_u) {
+                rc = set_smem(select_mask_rows_pair_kernel<0, true, 2>, warp_smem, 2048);
             } else {
                 switch (nv) {
-                    case 8: rc = set_smem(select_mask_rows_pair_kernel<8, false>, warp_smem, 2048); break;
-                    case 16: rc = set_smem(select_mask_rows_pair_kernel<16, false>, warp_smem, 2048); break;
-                    case 32: rc = set_smem(select_mask_rows_pair_kernel<32, false>, warp_smem, 2048); break;
-                    case 43: rc = set_smem(select_mask_rows_pair_kernel<43, false>, warp_smem, 2048); break;
-                    default: rc = set_smem(select_mask_rows_pair_kernel<0, false>, warp_smem, 2048); break;
+                    case 8: rc = set_smem(select_mask_rows_pair_kernel<8, false, 2>, warp_smem, 2048); break;
+                    case 16: rc = set_smem(select_mask_rows_pair_kernel<16, false, 2>, warp_smem, 2048); break;
+                    case 32: rc = set_smem(select_mask_rows_pair_kernel<32, false, 2>, warp_smem, 2048); break;
+                    default: rc = set_smem(select_mask_rows_pair_kernel<0, false, 2>, warp_smem, 2048); break;
                 }
             }
         } else if (sel_shared_u) {
@@ -417,29 +429,30 @@ int forward_tc(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat1
         if (warp_select) {
             const unsigned grid =
                 (unsigned)std::min<int64_t>((n + sel_wpc - 1) / sel_wpc, (int64_t)sm_count() * sel_ctas_per_sm);
-#define MOC_WARP_SELECT(KERNEL, NV, SHARED, THREADS_PER_TOKEN)                                               \
-    MOC_LAUNCH(KID_TC_SELECT_MASK, st,                                                                          \
-               (KERNEL<NV, SHARED><<<grid, sel_wpc * THREADS_PER_TOKEN, warp_smem, st>>>(                        \
+#define MOC_SELECT_LAUNCH(THREADS_PER_TOKEN, ...)                                                          \
+    MOC_LAUNCH(KID_TC_SELECT_MASK, st,                                                                     \
+               (__VA_ARGS__<<<grid, sel_wpc * THREADS_PER_TOKEN, warp_smem, st>>>(                          \
                    G, L.ldf, Uc, L.ldf, n, F, nv, K, o_idx, o_g, o_u, meta, status)))
-#define MOC_SELECT_BY_WIDTH(KERNEL, TPT)                                       \
-    if (sel_shared_u) {                                                        \
-        MOC_WARP_SELECT(KERNEL, 0, true, TPT);                                 \
-    } else {                                                                   \
-        switch (nv) { /* the usual row lengths get their loops unrolled */     \
-            case 8: MOC_WARP_SELECT(KERNEL, 8, false, TPT); break;             \
-            case 16: MOC_WARP_SELECT(KERNEL, 16, false, TPT); break;           \
-            case 32: MOC_WARP_SELECT(KERNEL, 32, false, TPT); break;           \
-            case 43: MOC_WARP_SELECT(KERNEL, 43, false, TPT); break;           \
-            default: MOC_WARP_SELECT(KERNEL, 0, false, TPT); break;            \
-        }                                                                      \
-    }
-            if (sel_pairs) {
-                MOC_SELECT_BY_WIDTH(select_mask_rows_pair_kernel, 64)
+            // the usual row lengths get their loops unrolled
+            if (sel_pairs && sel_team == 4) {
+                if (sel_shared_u) MOC_SELECT_LAUNCH(128, select_mask_rows_pair_kernel<0, true, 4>);
+                else if (nv == 43) MOC_SELECT_LAUNCH(128, select_mask_rows_pair_kernel<43, false, 4>);
+                else MOC_SELECT_LAUNCH(128, select_mask_rows_pair_kernel<0, false, 4>);
+            } else if (sel_pairs) {
+                if (sel_shared_u) MOC_SELECT_LAUNCH(64, select_mask_rows_pair_kernel<0, true, 2>);
+                else if (nv == 8) MOC_SELECT_LAUNCH(64, select_mask_rows_pair_kernel<8, false, 2>);
+                else if (nv == 16) MOC_SELECT_LAUNCH(64, select_mask_rows_pair_kernel<16, false, 2>);
+                else if (nv == 32) MOC_SELECT_LAUNCH(64, select_mask_rows_pair_kernel<32, false, 2>);
+                else MOC_SELECT_LAUNCH(64, select_mask_rows_pair_kernel<0, false, 2>);
             } else {
-                MOC_SELECT_BY_WIDTH(select_mask_rows_warp_kernel, 32)
+                if (sel_shared_u) MOC_SELECT_LAUNCH(32, select_mask_rows_warp_kernel<0, true>);
+                else if (nv == 8) MOC_SELECT_LAUNCH(32, select_mask_rows_warp_kernel<8, false>);
+                else if (nv == 16) MOC_SELECT_LAUNCH(32, select_mask_rows_warp_kernel<16, false>);
+                else if (nv == 32) MOC_SELECT_LAUNCH(32, select_mask_rows_warp_kernel<32, false>);
+                else if (nv == 43) MOC_SELECT_LAUNCH(32, select_mask_rows_warp_kernel<43, false>);
+                else MOC_SELECT_LAUNCH(32, select_mask_rows_warp_kernel<0, false>);
             }
-#undef MOC_SELECT_BY_WIDTH
-#undef MOC_WARP_SELECT
+#undef MOC_SELECT_LAUNCH
         } else {
             const unsigned grid = (unsigned)std::min<int64_t>(n, (int64_t)sm_count() * 6);
             MOC_LAUNCH(KID_TC_SELECT_MASK, st,

@@ -630,45 +630,47 @@ __global__ void __launch_bounds__(kWarpSelMaxWarps * 32) select_mask_rows_warp_k
 }
 
 // ------------------------------------------------------------------------------------------------
-// The same selector with TWO WARPS per token (same staging, same steps, same exactness): the pair shares one
-// slice of shared memory, each warp takes every other 128-channel group in steps 1 and 3 and half of the kept
-// channels in step 4, and the two meet at a named barrier of their own between the steps.  A token's rows
-// occupy the slice for about half as long, so the shared memory of an SM (which bounds the tokens in flight)
-// feeds twice as many warps.
-__host__ __device__ constexpr size_t pair_select_words(int nv, int K, bool shared_u) {
-    return (size_t)nv * 128 + (shared_u ? 0 : (size_t)nv * 64) + 2 * (size_t)warp_select_cand_words(nv) +
-           warp_select_bitmap_words(nv) + (size_t)((K + 3) & ~3) + 16 /* exchange */ + 4 /* two mbarriers */;
+// The same selector with a TEAM of W = 2 or 4 warps per token (same staging, same steps, same exactness): the
+// team shares one slice of shared memory, warp w takes the 128-channel groups w, w + W, ... in steps 1 and 3 and
+// every W-th batch of kept channels in step 4, and the warps meet at a named barrier of their own between the
+// steps.  A token's rows occupy the slice for a fraction of the time, so the shared memory of an SM (which
+// bounds the tokens in flight) feeds W times as many warps.
+__host__ __device__ constexpr size_t pair_select_words(int nv, int K, bool shared_u, int W = 2) {
+    return (size_t)nv * 128 + (shared_u ? 0 : (size_t)nv * 64) + (size_t)W * warp_select_cand_words(nv) +
+           warp_select_bitmap_words(nv) + (size_t)((K + 3) & ~3) + 32 /* exchange */ + 4 /* two mbarriers */;
 }
-__host__ __device__ constexpr bool pair_select_parks_gates(int nv, int K) {
-    return K <= 2 * warp_select_cand_words(nv) + warp_select_bitmap_words(nv);
+__host__ __device__ constexpr bool pair_select_parks_gates(int nv, int K, int W = 2) {
+    return K <= W * warp_select_cand_words(nv) + warp_select_bitmap_words(nv);
 }
-constexpr int kPairSelMaxWarps = 12;  // warps per CTA, at most (six pairs: named barriers 1..6; two CTAs per SM)
+constexpr int kPairSelMaxWarps = 12;  // warps per CTA, at most (six pairs or three teams of four; two CTAs per SM)
 
-template <int NV, bool shared_u>
+template <int NV, bool shared_u, int W>
 __global__ void __launch_bounds__(kPairSelMaxWarps * 32, 2) select_mask_rows_pair_kernel(
     const float *__restrict__ G, int ldg, __nv_bfloat16 *__restrict__ U, int ldu, int64_t rows, int F, int nv_runtime, int K,
     int16_t *__restrict__ idx_out, __nv_bfloat16 *__restrict__ g_out, __nv_bfloat16 *__restrict__ u_out,
     SelectMeta meta, int *status) {
     extern __shared__ __align__(128) uint32_t warp_sel_smem[];
+    static_assert(W == 2 || W == 4, "teams of two or four warps");
+    constexpr int TT = 32 * W;  // threads of a team
     __shared__ float s_stat[kPairSelMaxWarps / 2][3];
     __shared__ int s_abort;
     const int nv = NV > 0 ? NV : nv_runtime;
     const int slots = warp_select_slots(nv), cw = warp_select_cand_words(nv);
-    const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5, ppc = blockDim.x >> 6;  // pairs per CTA
-    const int pair = wib >> 1, w = wib & 1, pl = (w << 5) | lane;                      // pl: 0..63 within the pair
-    uint32_t *base = warp_sel_smem + (size_t)pair * pair_select_words(nv, K, shared_u);
+    const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5, ppc = blockDim.x / TT;  // teams per CTA
+    const int pair = wib / W, w = wib % W, pl = (w << 5) | lane;                       // pl: thread index within the team
+    uint32_t *base = warp_sel_smem + (size_t)pair * pair_select_words(nv, K, shared_u, W);
     float *sg = reinterpret_cast<float *>(base);
     __nv_bfloat16 *su = reinterpret_cast<__nv_bfloat16 *>(shared_u ? base : base + nv * 128);
-    uint32_t *cand0 = base + nv * 128 + (shared_u ? 0 : nv * 64);  // [2 warps][slot][lane] parked values
+    uint32_t *cand0 = base + nv * 128 + (shared_u ? 0 : nv * 64);  // [W warps][slot][lane] parked values
     uint32_t *cand = cand0 + w * cw;
-    uint32_t *bitmap = cand0 + 2 * cw;
+    uint32_t *bitmap = cand0 + W * cw;
     uint32_t *kept = bitmap + warp_select_bitmap_words(nv);
-    uint32_t *xch = kept + ((K + 3) & ~3);  // [2 parities][2 warps][4] counts exchanged between the warps
-    uint64_t *bar_mem = reinterpret_cast<uint64_t *>(xch + 16);
+    uint32_t *xch = kept + ((K + 3) & ~3);  // [2 parities][W warps][4] counts exchanged between the warps
+    uint64_t *bar_mem = reinterpret_cast<uint64_t *>(xch + 32);
     const uint32_t bar_g = smem_u32(bar_mem), bar_u = smem_u32(bar_mem + 1);
     float *gkept = reinterpret_cast<float *>(cand0);
-    const bool early_gate = pair_select_parks_gates(nv, K);
-    auto pair_sync = [&]() { asm volatile("bar.sync %0, 64;" ::"r"(pair + 1) : "memory"); };
+    const bool early_gate = pair_select_parks_gates(nv, K, W);
+    auto pair_sync = [&]() { asm volatile("bar.sync %0, %1;" ::"r"(pair + 1), "n"(TT) : "memory"); };
     const int64_t gp = (int64_t)blockIdx.x * ppc + pair, np = (int64_t)gridDim.x * ppc;
     const float b_center = meta.bracket[0], b_width = meta.bracket[1];
     const bool have_bracket = meta.bracket[2] == kBracketTag && b_width > 0.f && fabsf(b_center) <= 3.0e38f;
@@ -683,7 +685,7 @@ __global__ void __launch_bounds__(kPairSelMaxWarps * 32, 2) select_mask_rows_pai
         mbar_init(bar_g, 1);
         mbar_init(bar_u, 1);
     }
-    for (int c = ldg + pl; c < nv * 128; c += 64) sg[c] = -INFINITY;
+    for (int c = ldg + pl; c < nv * 128; c += TT) sg[c] = -INFINITY;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     __syncthreads();
     uint32_t phase = 0;
@@ -693,7 +695,7 @@ __global__ void __launch_bounds__(kPairSelMaxWarps * 32, 2) select_mask_rows_pai
         mbar_expect_tx(bar_g, g_bytes);
         bulk_copy_g2s(smem_u32(sg), G + gp * (int64_t)ldg, g_bytes, bar_g);
     }
-    // both warps of a pair take every branch below together: all conditions come from values they share
+    // the warps of a team take every branch below together: all conditions come from values they share
 
     for (int64_t r = gp; r < rows && !dead; r += np) {
         __nv_bfloat16 *u = U + r * (int64_t)ldu;
@@ -710,7 +712,7 @@ __global__ void __launch_bounds__(kPairSelMaxWarps * 32, 2) select_mask_rows_pai
         }
         if (!__all_sync(0xffffffffu, mbar_wait(bar_g, phase, &s_abort, status))) dead = true;
         if (!dead)
-            for (int c = F + pl; c < ldg; c += 64) sg[c] = -INFINITY;
+            for (int c = F + pl; c < ldg; c += TT) sg[c] = -INFINITY;
         // the partner must see the same verdict: a failed wait ends the pair (s_abort is set block-wide)
         pair_sync();
         if (s_abort) dead = true;
@@ -723,7 +725,7 @@ __global__ void __launch_bounds__(kPairSelMaxWarps * 32, 2) select_mask_rows_pai
             // ---- 1. classify: this warp's groups v = w, w + 2, ...
             uint32_t n_above = 0, n_mine = 0;
 #pragma unroll 4
-            for (int v = w; v < nv; v += 2) {
+            for (int v = w; v < nv; v += W) {
                 const float4 q = *reinterpret_cast<const float4 *>(sg + (v * 32 + lane) * 4);
                 const float e4[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
@@ -738,7 +740,7 @@ __global__ void __launch_bounds__(kPairSelMaxWarps * 32, 2) select_mask_rows_pai
             const uint32_t my_hi = __reduce_add_sync(0xffffffffu, n_above);
             const uint32_t my_band = __reduce_add_sync(0xffffffffu, n_mine);
             const uint32_t my_max = __reduce_max_sync(0xffffffffu, n_mine);
-            uint32_t *xs = xch + xp * 8;
+            uint32_t *xs = xch + xp * (4 * W);
             xp ^= 1;
             if (lane == 0) {
                 xs[w * 4 + 0] = my_hi;
@@ -747,10 +749,16 @@ __global__ void __launch_bounds__(kPairSelMaxWarps * 32, 2) select_mask_rows_pai
             }
             // scratch of the search, cleared here so that the barrier below also publishes it
             uint32_t *hist = bitmap, *list = bitmap + 64, *list_n = bitmap + 96;
-            hist[pl] = 0u;
+            if (pl < 64) hist[pl] = 0u;
             if (pl == 0) *list_n = 0u;
             pair_sync();
-            const uint32_t c_hi = xs[0] + xs[4], n_band = xs[1] + xs[5], max_mine = max(xs[2], xs[6]);
+            uint32_t c_hi = 0, n_band = 0, max_mine = 0;
+#pragma unroll
+            for (int i = 0; i < W; ++i) {
+                c_hi += xs[4 * i];
+                n_band += xs[4 * i + 1];
+                max_mine = max(max_mine, xs[4 * i + 2]);
+            }
             if (max_mine > (uint32_t)slots) {  // too many values inside: halve the bracket
                 const float c = 0.5f * (lo_f + hi_f), wd = 0.25f * (hi_f - lo_f);
                 lo_f = c - wd;
@@ -818,11 +826,11 @@ __global__ void __launch_bounds__(kPairSelMaxWarps * 32, 2) select_mask_rows_pai
         const float tau_f = key_to_float(res);
         if (settled && no_cut && fabsf(tau_f) <= 3.0e38f) {
             // ---- 3. kept set = {g >= tau}: each warp writes the bitmap words of its own groups
-            for (int v = w; v < nv; v += 2)
+            for (int v = w; v < nv; v += W)
                 if (lane < 4 && v * 4 + lane < warp_select_bitmap_words(nv)) bitmap[v * 4 + lane] = 0u;
             __syncwarp();
 #pragma unroll 4
-            for (int v = w; v < nv; v += 2) {
+            for (int v = w; v < nv; v += W) {
                 const float4 q = *reinterpret_cast<const float4 *>(sg + (v * 32 + lane) * 4);
                 const uint32_t nib = (q.x >= tau_f ? 1u : 0u) | (q.y >= tau_f ? 2u : 0u) |
                                      (q.z >= tau_f ? 4u : 0u) | (q.w >= tau_f ? 8u : 0u);
@@ -830,7 +838,7 @@ __global__ void __launch_bounds__(kPairSelMaxWarps * 32, 2) select_mask_rows_pai
             }
             pair_sync();
             // enumerate in ascending channel order: thread pl of the pair owns words [pl*wpl, (pl+1)*wpl)
-            const int wpl = (words + 63) >> 6;
+            const int wpl = (words + TT - 1) / TT;
             uint32_t mine = 0;
             for (int i = 0; i < wpl; ++i) {
                 const int wd = pl * wpl + i;
@@ -842,13 +850,18 @@ __global__ void __launch_bounds__(kPairSelMaxWarps * 32, 2) select_mask_rows_pai
                 const uint32_t nb = __shfl_up_sync(0xffffffffu, pre, o);
                 if (lane >= o) pre += nb;
             }
-            uint32_t *xs = xch + xp * 8;
+            uint32_t *xs = xch + xp * (4 * W);
             xp ^= 1;
             if (lane == 31) xs[w * 4 + 3] = pre;  // this warp's total
             pair_sync();
-            const uint32_t tot0 = xs[3], tot1 = xs[7];
-            if (tot0 + tot1 == (uint32_t)K) {  // counts and compares agree
-                uint32_t pos = pre - mine + (w ? tot0 : 0u);
+            uint32_t total = 0, before = 0;
+#pragma unroll
+            for (int i = 0; i < W; ++i) {
+                total += xs[4 * i + 3];
+                before += i < w ? xs[4 * i + 3] : 0u;
+            }
+            if (total == (uint32_t)K) {  // counts and compares agree
+                uint32_t pos = pre - mine + before;
                 for (int i = 0; i < wpl; ++i) {
                     const int wd = pl * wpl + i;
                     uint32_t bits = wd < words ? bitmap[wd] : 0u;
@@ -883,7 +896,7 @@ __global__ void __launch_bounds__(kPairSelMaxWarps * 32, 2) select_mask_rows_pai
             }
         };
         if (early_gate) {
-            for (int i = pl; i < K; i += 64) gkept[i] = sg[kept[i]];
+            for (int i = pl; i < K; i += TT) gkept[i] = sg[kept[i]];
             pair_sync();
             if (!shared_u) {
                 request_next_gate();
@@ -898,7 +911,7 @@ __global__ void __launch_bounds__(kPairSelMaxWarps * 32, 2) select_mask_rows_pai
         if (s_abort) dead = true;
         if (dead) break;
         phase ^= 1u;
-        for (int i = pl; i < K; i += 64) {
+        for (int i = pl; i < K; i += TT) {
             const uint32_t j = kept[i];
             const float gval = early_gate ? gkept[i] : sg[j];
             const __nv_bfloat16 ub = su[j];
@@ -914,9 +927,9 @@ __global__ void __launch_bounds__(kPairSelMaxWarps * 32, 2) select_mask_rows_pai
         if (!early_gate) request_next_gate();
         // ---- up row -> masked Z' row, in shared memory, then one bulk store
         uint4 *row16 = reinterpret_cast<uint4 *>(su);
-        for (int i = pl; i < (ldu >> 3); i += 64) row16[i] = make_uint4(0, 0, 0, 0);
+        for (int i = pl; i < (ldu >> 3); i += TT) row16[i] = make_uint4(0, 0, 0, 0);
         pair_sync();
-        for (int i = pl; i < K; i += 64) {
+        for (int i = pl; i < K; i += TT) {
             const uint32_t e = kept[i];
             const uint16_t zb = (uint16_t)(e >> 16);
             su[e & 0xffffu] = *reinterpret_cast<const __nv_bfloat16 *>(&zb);
