@@ -280,8 +280,9 @@ def test_decode_small_shapes(dtype, T, d, F, K):
     (513, 264, 1100, 1104, 137),   # d not a multiple of 64, F not a multiple of 256, ragged token tile
     (256, 128, 96, 96, 96),        # K = F: dense SwiGLU through the tensor-core plan
     (384, 512, 4500, 4504, 563),   # more than 4096 channels: few warps per SM in the warp-per-token selector
-    (300, 128, 9000, 9000, 700),   # rows too long for separate gate and up buffers: both rows share one buffer
-    (260, 64, 20000, 20000, 1500), # rows too long for any warp slice: CTA-per-token selector
+    (300, 128, 9000, 9000, 700),   # long rows: teams of four warps, two tokens in flight per SM
+    (260, 64, 16000, 16000, 1200), # rows too long for separate gate and up buffers: both rows share one buffer
+    (260, 64, 24000, 24000, 1500), # rows too long for any shared-memory slice: CTA-per-token selector
 ])
 def test_tc_plan_shapes(T, d, F, F_ld, K):
     w = syn.Workload(f"tc-{T}-{d}-{F}-{K}", "bf16", T, d, F, F_ld, K, seed=200 + T)
