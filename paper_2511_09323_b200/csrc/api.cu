@@ -512,15 +512,18 @@ int backward_tc(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat
         // one warp per token with the token's rows staged in shared memory while at least four such warps fit an
         // SM; else one CTA per token working in global memory
         const size_t sw_bytes = sample_warp_words(L.ldf, K) * sizeof(uint32_t);
-        const int sw_per_sm = (int)std::min<size_t>((size_t)220 * 1024 / sw_bytes, 2 * kSampleMaxWarps);
-        if (sw_per_sm >= 4 && F <= 65535) {
-            const int ctas_per_sm = sw_per_sm > 4 ? 2 : 1, wpc = sw_per_sm / ctas_per_sm;
+        const int sw_per_sm = (int)std::min<size_t>((size_t)220 * 1024 / sw_bytes, 2 * kSampleMaxWarps);  // tokens in flight
+        if (sw_per_sm >= 2 && F <= 65535) {
+            // two warps per token unless that many tokens fit that one warp each already fills the SM
+            const int team = sw_per_sm <= 12 ? 2 : 1;
+            const int per_cta_max = kSampleMaxWarps / team;
+            const int ctas_per_sm = (sw_per_sm + per_cta_max - 1) / per_cta_max, wpc = sw_per_sm / ctas_per_sm;
             const size_t smem = (size_t)wpc * sw_bytes;
-            if ((rc = set_smem(backward_sample_rows_warp_kernel, smem, 2048)) != MOC_OK) return rc;
+            auto kern = team == 2 ? backward_sample_rows_warp_kernel<2> : backward_sample_rows_warp_kernel<1>;
+            if ((rc = set_smem(kern, smem, 2048)) != MOC_OK) return rc;
             const unsigned grid = (unsigned)std::min<int64_t>((T + wpc - 1) / wpc, (int64_t)sm_count() * ctas_per_sm);
             MOC_LAUNCH(KID_TC_BWD_SAMPLE, st,
-                       (backward_sample_rows_warp_kernel<<<grid, wpc * 32, smem, st>>>(idx, tg, tu, T, K, F, L.ldf, Zp,
-                                                                                        dUp, dGp, status)));
+                       (kern<<<grid, wpc * team * 32, smem, st>>>(idx, tg, tu, T, K, F, L.ldf, Zp, dUp, dGp, status)));
         } else {
             const size_t smem = (size_t)K * 8;
             if ((rc = set_smem(backward_sample_rows_kernel, smem)) != MOC_OK) return rc;

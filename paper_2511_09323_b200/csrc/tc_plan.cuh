@@ -1104,16 +1104,25 @@ __host__ __device__ constexpr size_t sample_warp_words(int ld, int K) {
     return (size_t)2 * ld /* four bf16 rows */ + (size_t)2 * ((K + 1) & ~1) /* entries */ +
            (size_t)3 * ((K + 7) & ~7) /* saved idx, g, u of two tokens */ + 4 /* two mbarriers */;
 }
-constexpr int kSampleMaxWarps = 8;
+constexpr int kSampleMaxWarps = 10;
 
+// W warps work on a token (W = 1 or 2: with two, the token's rows occupy the slice for about half as long and the
+// same shared memory feeds twice the warps); they meet at a named barrier of their own between the phases.
+template <int W>
 __global__ void __launch_bounds__(kSampleMaxWarps * 32) backward_sample_rows_warp_kernel(
     const int16_t *__restrict__ idx, const __nv_bfloat16 *__restrict__ gval, const __nv_bfloat16 *__restrict__ uval,
     int64_t T, int K, int F, int ld, __nv_bfloat16 *__restrict__ dz_z, __nv_bfloat16 *__restrict__ du,
     __nv_bfloat16 *__restrict__ dg, int *__restrict__ status) {
     extern __shared__ __align__(128) uint32_t sample_warp_smem[];
     __shared__ int s_abort;
-    const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5, wpc = blockDim.x >> 5;
-    uint32_t *base = sample_warp_smem + (size_t)wib * sample_warp_words(ld, K);
+    constexpr int TT = 32 * W;  // threads of a team
+    const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5, wpc = blockDim.x / TT;  // teams per CTA
+    const int team = wib / W, pl = ((wib % W) << 5) | lane;                            // pl: thread index within the team
+    auto team_sync = [&]() {
+        if (W == 1) __syncwarp();
+        else asm volatile("bar.sync %0, %1;" ::"r"(team + 1), "n"(TT) : "memory");
+    };
+    uint32_t *base = sample_warp_smem + (size_t)team * sample_warp_words(ld, K);
     const int row_words = ld >> 1;  // ld is a multiple of 8: rows are multiples of 16 bytes
     __nv_bfloat16 *zbuf0 = reinterpret_cast<__nv_bfloat16 *>(base);  // two dZ rows, used alternately
     __nv_bfloat16 *ubuf = reinterpret_cast<__nv_bfloat16 *>(base + 2 * row_words);
@@ -1127,10 +1136,10 @@ __global__ void __launch_bounds__(kSampleMaxWarps * 32) backward_sample_rows_war
     uint64_t *bar_mem = reinterpret_cast<uint64_t *>(saved0 + 6 * K8);
     const uint32_t bar0 = smem_u32(bar_mem);  // two mbarriers, 8 bytes apart
     const uint32_t row_bytes = (uint32_t)ld * 2u, saved_bytes = (uint32_t)K * 2u;
-    const int64_t gw = (int64_t)blockIdx.x * wpc + wib, nw = (int64_t)gridDim.x * wpc;
+    const int64_t gw = (int64_t)blockIdx.x * wpc + team, nw = (int64_t)gridDim.x * wpc;
 
     if (threadIdx.x == 0) s_abort = 0;
-    if (lane == 0) {
+    if (pl == 0) {
         mbar_init(bar0, 1);
         mbar_init(bar0 + 8u, 1);
     }
@@ -1148,20 +1157,22 @@ __global__ void __launch_bounds__(kSampleMaxWarps * 32) backward_sample_rows_war
             bulk_copy_g2s(smem_u32(sv + 2 * K8), uval + tok * K, saved_bytes, nbar);
         }
     };
-    if (lane == 0 && gw < T) request(gw, 0);
+    if (pl == 0 && gw < T) request(gw, 0);
     int b = 0;
     for (int64_t t = gw; t < T; t += nw, b ^= 1) {
-        if (!__all_sync(0xffffffffu, mbar_wait(bar0 + 8u * (uint32_t)b, (phases >> b) & 1u, &s_abort, status))) break;
+        mbar_wait(bar0 + 8u * (uint32_t)b, (phases >> b) & 1u, &s_abort, status);  // a failed wait sets s_abort
+        team_sync();
+        if (s_abort) break;  // the whole team sees the same flag after the barrier
         phases ^= 1u << b;
         __nv_bfloat16 *zr = zbuf0 + (size_t)b * ld;
         const uint16_t *sv = saved0 + (size_t)b * 3 * K8;
-        for (int k0 = 0; k0 < K; k0 += 256) {
+        for (int k0 = 0; k0 < K; k0 += 8 * TT) {
             // eight saved entries per lane, their loads issued together
             int jv[8];
             __nv_bfloat16 gb[8], ub[8];
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
-                const int k = k0 + i * 32 + lane;
+                const int k = k0 + i * TT + pl;
                 jv[i] = -1;
                 if (k < K) {
                     if (staged_saved) {
@@ -1177,7 +1188,7 @@ __global__ void __launch_bounds__(kSampleMaxWarps * 32) backward_sample_rows_war
             }
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
-                const int k = k0 + i * 32 + lane;
+                const int k = k0 + i * TT + pl;
                 if (k >= K) continue;
                 const int j = jv[i];
                 uint32_t w0 = 0xffffu, w1 = 0;  // j = 0xffff marks a skipped entry
@@ -1198,24 +1209,25 @@ __global__ void __launch_bounds__(kSampleMaxWarps * 32) backward_sample_rows_war
         }
         // by now the stores of the previous token have read their rows: the other dZ buffer (next token's row goes
         // there) and the dU / dG rows are free
-        if (lane == 0) {
+        team_sync();  // every thread has sampled the dZ row
+        if (pl == 0) {
             bulk_store_wait_read<0>();
             fence_async_smem();
             if (t + nw < T) request(t + nw, b ^ 1);
         }
-        __syncwarp();
+        team_sync();
         {
             uint4 *z16 = reinterpret_cast<uint4 *>(zr), *u16 = reinterpret_cast<uint4 *>(ubuf),
                   *g16 = reinterpret_cast<uint4 *>(gbuf);
             const uint4 zero = make_uint4(0, 0, 0, 0);
-            for (int v = lane; v < (ld >> 3); v += 32) {
+            for (int v = pl; v < (ld >> 3); v += TT) {
                 z16[v] = zero;
                 u16[v] = zero;
                 g16[v] = zero;
             }
         }
-        __syncwarp();
-        for (int k = lane; k < K; k += 32) {
+        team_sync();
+        for (int k = pl; k < K; k += TT) {
             const uint32_t w0 = entry[2 * k], w1 = entry[2 * k + 1];
             const uint32_t j = w0 & 0xffffu;
             if (j == 0xffffu) continue;
@@ -1225,14 +1237,14 @@ __global__ void __launch_bounds__(kSampleMaxWarps * 32) backward_sample_rows_war
             gbuf[j] = *reinterpret_cast<const __nv_bfloat16 *>(&gb);
         }
         fence_async_smem();
-        __syncwarp();
-        if (lane == 0) {
+        team_sync();
+        if (pl == 0) {
             bulk_copy_s2g(dz_z + t * (int64_t)ld, smem_u32(zr), row_bytes);
             bulk_copy_s2g(du + t * (int64_t)ld, smem_u32(ubuf), row_bytes);
             bulk_copy_s2g(dg + t * (int64_t)ld, smem_u32(gbuf), row_bytes);
         }
     }
-    if (lane == 0) bulk_store_wait_all();
+    if (pl == 0) bulk_store_wait_all();
 }
 
 // ------------------------------------------------------------------------------------------------
