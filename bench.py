@@ -36,8 +36,8 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of each kernel of the step on the default C2 workload, from one
 # `ncu --set full` capture of this program (profiles/tensor_core_plan_kernels_C2.md); reported as `roofline.traffic`
 NCU_DRAM_BYTES_C2 = {
-    "tc_gate_up_gemm": 176.2e6, "tc_select_mask": 257.3e6, "tc_down_gemm": 75.0e6, "tc_bwd_sample": 234.3e6,
-    "tc_dz_gemm": 42.9e6, "tc_wgrad_gemm": 255.2e6, "tc_dx_gemm": 158.9e6,
+    "tc_gate_up_gemm": 173.5e6, "tc_select_mask": 255.1e6, "tc_down_gemm": 75.0e6, "tc_bwd_sample": 235.6e6,
+    "tc_dz_gemm": 43.4e6, "tc_wgrad_gemm": 256.7e6, "tc_dx_gemm": 158.6e6,
 }
 
 
