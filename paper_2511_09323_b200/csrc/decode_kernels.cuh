@@ -11,12 +11,13 @@
 //                    more issue slots than one (one FMA per loaded weight and token would be ALU-bound).
 //   2. select      : one 1024-thread CTA per token, exact Top-K by a radix select whose digits are taken
 //                    relative to the range the candidates lie in (see the kernel).  Decode needs the set,
-//                    not the order: the token's bit is set in a per-channel mask.
-//   3. up          : the same GEMV over the listed rows of W_up; z = SiLU(g) u for the tokens in each
-//                    channel's mask (zero for the others), stored as bf16 in MMA-ready blocks.
+//                    not the order: each token's selection is a bitmap written word by word from warp
+//                    ballots; the last CTA to finish lists the union of the bitmaps (ascending channels).
+//   3. up          : the same GEMV over the listed rows of W_up; z = SiLU(g) u for the tokens whose bitmap
+//                    holds the channel (zero for the others), stored as bf16 in MMA-ready blocks.
 //   4. down        : CTA = (512-column slice, part of the list).  Stages of 16 rows x 1 KiB; the rows are
 //                    the contraction index, so the B fragments are read transposed with ldmatrix.
-//                    Per-slice partial sums are added to an fp32 accumulator with atomics and the last
+//                    Per-slice partial sums are added to an fp32 accumulator with vector reductions and the last
 //                    CTA of a slice writes the bf16 output (the summation order across CTAs is not
 //                    fixed, so the last bit of `out` may vary from run to run).
 #pragma once
@@ -73,7 +74,7 @@ __device__ __forceinline__ void consumer_bar_sync() { asm volatile("bar.sync 1, 
 // ---------------------------------------------------------------------------------------------- 1 + 3. GEMV
 // R[t, r] = sum_i x[t,i] W[row(r), i] for the CTA's share of the rows, all tokens at once.
 //   GATHER == false: rows are the channels 0..F-1 of W_gate; result -> G          (Eq. (Moc-1))
-//   GATHER == true : rows are the listed channels of W_up;   result -> z = SiLU(g) u on the masks
+//   GATHER == true : rows are the listed channels of W_up;   result -> z = SiLU(g) u on the selection bitmaps
 // CTA b owns row slots [b n / grid, (b+1) n / grid).  Each lane reads 16 contiguous bytes (8 contraction
 // elements) of a weight row per fragment; the same permutation of the contraction index is applied to the
 // x fragment, so the MMA operands need no data movement.
@@ -273,8 +274,10 @@ __global__ void __launch_bounds__(kGemvThreads, 2) gemv_rows_kernel(const __nv_b
 // that the range maps onto at most 2048 bins.  The first level uses the row's minimum and maximum key;
 // the bin that holds the K-th largest then holds a handful of keys, which are copied to a short list and
 // ranked directly.  Further levels (only for very uneven data) repeat the step on the list.
-// Decode needs the set, not the order: the token's bit is set in a per-channel mask with plain
-// reductions; only when ties at the threshold must be cut does the ordered emission run.
+// Decode needs the set, not the order: consecutive lanes hold consecutive channels, so a warp ballot of
+// "key >= threshold" is one word of the token's selection bitmap; only when ties at the threshold must be
+// cut does the ordered emission run.  The kernels are chained with programmatic dependent launch: each
+// calls pdl_wait before it touches what an earlier kernel wrote.
 struct SelectLevel {
     uint32_t lo, hi;  // candidates lie in [lo, hi]
     uint32_t m;       // the m-th largest of them is wanted
