@@ -1,9 +1,11 @@
 // bf16 tensor-core GEMM for sm_100a: tcgen05.mma with TMEM accumulators, TMA-fed operands.
 //
 // One persistent CTA per SM (192 threads): warp 0 issues TMA loads, warp 1 issues tcgen05.mma and
-// owns the TMEM allocation, warps 2..5 run the epilogue.  Output tile 128 x 256, K step 64, four
-// shared-memory stages (48 KiB each), two accumulator stages in TMEM (2 x 256 columns) so that the
-// epilogue of tile i overlaps the main loop of tile i+1.
+// owns the TMEM allocation, warps 2..5 run the epilogue (TMEM -> swizzled shared-memory boxes -> bulk
+// tensor stores).  Two forms: gemm_kernel, one CTA per 128 x 256 output tile (K step 64, four 48 KiB
+// shared-memory stages), and gemm_pair_kernel, clusters of two CTAs sharing one cta_group::2 MMA on a
+// 256 x 256 tile (six 32 KiB stages per CTA).  Both keep two accumulator stages in TMEM (2 x 256
+// columns) so that the epilogue of tile i overlaps the main loop of tile i+1.
 //
 // Operands may be K-major (rows of 64 contraction elements = one 128-byte swizzle row) or MN-major
 // (the tensor's contiguous dimension is M or N; loaded as 64-wide boxes of 64 contraction rows).

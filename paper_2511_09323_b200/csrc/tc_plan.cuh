@@ -2,9 +2,11 @@
 // At 12.5 % unstructured density the tensor cores finish the dense contraction several times faster
 // than the ALUs finish the sparse one, so every contraction runs as a dense GEMM over the full
 // channel range and the Top-K structure is applied around it: the forward selects from the fp32
-// gate tile and turns the dense up projection into the masked Z' in place; the backward samples
-// dD Wd^T at the saved indices in the GEMM epilogue.  Only idx / g / u in compact [T,K] form leave
-// the forward; all dense [T,F] arrays are transient workspace.
+// gate rows and turns the dense up projection into the masked Z' in place; the backward samples the
+// dense dD Wd^T at the saved indices in a per-token kernel that also writes the masked dU' and dG' rows
+// the gradient GEMMs contract.  Only idx / g / u in compact [T,K] form leave the forward; all dense
+// [T,F] arrays are transient workspace.  The per-token kernels stage a token's rows in shared memory
+// with bulk async copies and give each token a warp or a team of two or four warps.
 #pragma once
 
 #include <cuda.h>
