@@ -322,25 +322,20 @@ int forward_tc(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat1
     const int nv = ceil_div(F, 128);  // 128-channel groups of a row
     // each warp stages its token's rows in its own slice of shared memory: as many warps per SM as fit, in one
     // or two CTAs
-    // (rows too long for that with separate gate and up buffers let the two rows share one buffer).  Two warps
-    // work on a token (MOC_FFN_SELECT=warp in the environment: one warp per token, kept for comparison).
-    static const bool sel_pairs = !(getenv("MOC_FFN_SELECT") && strcmp(getenv("MOC_FFN_SELECT"), "warp") == 0);
-    // teams of four warps for long rows (few tokens fit an SM there), pairs otherwise
-    // (measured: LLaMA-1B width 0.59 -> 0.50 ms and LLaMA-7B width 0.56 -> 0.41 ms with four; 2048 channels 0.080 ->
-    // 0.124 ms, so short rows keep pairs)
+    // (rows too long for that with separate gate and up buffers let the two rows share one buffer).  Teams of four
+    // warps for long rows (few tokens fit an SM there), pairs otherwise (measured: LLaMA-1B width 0.59 -> 0.50 ms and
+    // LLaMA-7B width 0.56 -> 0.41 ms with four; 2048 channels 0.080 -> 0.124 ms, so short rows keep pairs)
     const int sel_team = nv >= 40 ? 4 : 2;
     const auto units_fit = [&](bool shared) {  // tokens in flight per SM
-        const size_t words = sel_pairs ? pair_select_words(nv, K, shared, sel_team) : warp_select_words(nv, K, shared);
-        return (int)std::min<size_t>((size_t)220 * 1024 / (words * sizeof(uint32_t)), 16);
+        return (int)std::min<size_t>(
+            (size_t)220 * 1024 / (pair_select_words(nv, K, shared, sel_team) * sizeof(uint32_t)), 16);
     };
-    const bool parks = sel_pairs ? pair_select_parks_gates(nv, K, sel_team) : warp_select_parks_gates(nv, K);
-    const int min_units = sel_pairs ? 2 : 4;  // at least four warps per SM
+    const bool parks = pair_select_parks_gates(nv, K, sel_team);
+    const int min_units = 2;  // at least two tokens in flight per SM
     const bool sel_shared_u = units_fit(false) < min_units && parks && units_fit(true) >= min_units;
-    const size_t warp_bytes =
-        (sel_pairs ? pair_select_words(nv, K, sel_shared_u, sel_team) : warp_select_words(nv, K, sel_shared_u)) *
-        sizeof(uint32_t);
-    const int warps_per_sm = units_fit(sel_shared_u);  // tokens in flight per SM (a warp or a pair of warps each)
-    const int sel_units_per_cta = sel_pairs ? kPairSelMaxWarps / sel_team : kWarpSelMaxWarps;
+    const size_t warp_bytes = pair_select_words(nv, K, sel_shared_u, sel_team) * sizeof(uint32_t);
+    const int warps_per_sm = units_fit(sel_shared_u);  // tokens in flight per SM (one team each)
+    const int sel_units_per_cta = kPairSelMaxWarps / sel_team;
     const int sel_ctas_per_sm = warps_per_sm > sel_units_per_cta ? 2 : 1;
     const int sel_wpc = std::min(warps_per_sm / sel_ctas_per_sm, sel_units_per_cta);  // tokens per CTA
     const size_t warp_smem = (size_t)sel_wpc * warp_bytes;
@@ -349,7 +344,7 @@ int forward_tc(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat1
     float *hint = reinterpret_cast<float *>(ws + L.off_hint);
     int rc = MOC_OK;
     if (warp_select) {
-        if (sel_pairs && sel_team == 4) {
+        if (sel_team == 4) {
             if (sel_shared_u) {
                 rc = set_smem(select_mask_rows_pair_kernel<0, true, 4>, warp_smem, 2048);
             } else if (nv == 43) {
@@ -357,26 +352,14 @@ int forward_tc(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat1
             } else {
                 rc = set_smem(select_mask_rows_pair_kernel<0, false, 4>, warp_smem, 2048);
             }
-        } else if (sel_pairs) {
-            if (sel_shared_u) {
-                rc = set_smem(select_mask_rows_pair_kernel<0, true, 2>, warp_smem, 2048);
-            } else {
-                switch (nv) {
-                    case 8: rc = set_smem(select_mask_rows_pair_kernel<8, false, 2>, warp_smem, 2048); break;
-                    case 16: rc = set_smem(select_mask_rows_pair_kernel<16, false, 2>, warp_smem, 2048); break;
-                    case 32: rc = set_smem(select_mask_rows_pair_kernel<32, false, 2>, warp_smem, 2048); break;
-                    default: rc = set_smem(select_mask_rows_pair_kernel<0, false, 2>, warp_smem, 2048); break;
-                }
-            }
         } else if (sel_shared_u) {
-            rc = set_smem(select_mask_rows_warp_kernel<0, true>, warp_smem, 2048);
+            rc = set_smem(select_mask_rows_pair_kernel<0, true, 2>, warp_smem, 2048);
         } else {
             switch (nv) {
-                case 8: rc = set_smem(select_mask_rows_warp_kernel<8, false>, warp_smem, 2048); break;
-                case 16: rc = set_smem(select_mask_rows_warp_kernel<16, false>, warp_smem, 2048); break;
-                case 32: rc = set_smem(select_mask_rows_warp_kernel<32, false>, warp_smem, 2048); break;
-                case 43: rc = set_smem(select_mask_rows_warp_kernel<43, false>, warp_smem, 2048); break;
-                default: rc = set_smem(select_mask_rows_warp_kernel<0, false>, warp_smem, 2048); break;
+                case 8: rc = set_smem(select_mask_rows_pair_kernel<8, false, 2>, warp_smem, 2048); break;
+                case 16: rc = set_smem(select_mask_rows_pair_kernel<16, false, 2>, warp_smem, 2048); break;
+                case 32: rc = set_smem(select_mask_rows_pair_kernel<32, false, 2>, warp_smem, 2048); break;
+                default: rc = set_smem(select_mask_rows_pair_kernel<0, false, 2>, warp_smem, 2048); break;
             }
         }
     } else {
@@ -434,23 +417,16 @@ int forward_tc(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat1
                (__VA_ARGS__<<<grid, sel_wpc * THREADS_PER_TOKEN, warp_smem, st>>>(                          \
                    G, L.ldf, Uc, L.ldf, n, F, nv, K, o_idx, o_g, o_u, meta, status)))
             // the usual row lengths get their loops unrolled
-            if (sel_pairs && sel_team == 4) {
+            if (sel_team == 4) {
                 if (sel_shared_u) MOC_SELECT_LAUNCH(128, select_mask_rows_pair_kernel<0, true, 4>);
                 else if (nv == 43) MOC_SELECT_LAUNCH(128, select_mask_rows_pair_kernel<43, false, 4>);
                 else MOC_SELECT_LAUNCH(128, select_mask_rows_pair_kernel<0, false, 4>);
-            } else if (sel_pairs) {
+            } else {
                 if (sel_shared_u) MOC_SELECT_LAUNCH(64, select_mask_rows_pair_kernel<0, true, 2>);
                 else if (nv == 8) MOC_SELECT_LAUNCH(64, select_mask_rows_pair_kernel<8, false, 2>);
                 else if (nv == 16) MOC_SELECT_LAUNCH(64, select_mask_rows_pair_kernel<16, false, 2>);
                 else if (nv == 32) MOC_SELECT_LAUNCH(64, select_mask_rows_pair_kernel<32, false, 2>);
                 else MOC_SELECT_LAUNCH(64, select_mask_rows_pair_kernel<0, false, 2>);
-            } else {
-                if (sel_shared_u) MOC_SELECT_LAUNCH(32, select_mask_rows_warp_kernel<0, true>);
-                else if (nv == 8) MOC_SELECT_LAUNCH(32, select_mask_rows_warp_kernel<8, false>);
-                else if (nv == 16) MOC_SELECT_LAUNCH(32, select_mask_rows_warp_kernel<16, false>);
-                else if (nv == 32) MOC_SELECT_LAUNCH(32, select_mask_rows_warp_kernel<32, false>);
-                else if (nv == 43) MOC_SELECT_LAUNCH(32, select_mask_rows_warp_kernel<43, false>);
-                else MOC_SELECT_LAUNCH(32, select_mask_rows_warp_kernel<0, false>);
             }
 #undef MOC_SELECT_LAUNCH
         } else {

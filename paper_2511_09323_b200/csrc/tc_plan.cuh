@@ -191,12 +191,12 @@ __global__ void __launch_bounds__(kSelectThreads) select_hint_kernel(const float
 }
 
 // ------------------------------------------------------------------------------------------------
-// Forward selector for rows that fit a warp's slice of shared memory: ONE WARP per token, no block barriers.
-// nv = number of 128-channel groups of a row.
+// Forward selector for rows that fit a slice of shared memory: a TEAM of two or four warps per token, no block
+// barriers (the warps of a team meet at a named barrier of their own).  nv = number of 128-channel groups of a row.
 // Same outputs as the CTA-per-token kernel below.
 //
-// Every warp owns a slice of shared memory into which lane 0 bulk-copies the token's gate row (fp32) and up
-// row (bf16); the warp works on those copies, turns the up row into the masked Z' row in place and
+// Every team owns a slice of shared memory into which its first thread bulk-copies the token's gate row (fp32)
+// and up row (bf16); the team works on those copies, turns the up row into the masked Z' row in place and
 // bulk-stores it back.  All global traffic of a row is therefore three asynchronous, fully coalesced
 // copies plus the compact outputs, and the scattered accesses of the method (K values per token) stay in
 // shared memory.
@@ -204,7 +204,7 @@ __global__ void __launch_bounds__(kSelectThreads) select_hint_kernel(const float
 // The launch starts from one bracket [center - width, center + width] that is expected to contain every
 // row's threshold; it comes from the thresholds of the previous launch (kept in the workspace).  A row whose
 // threshold lies outside moves the bracket (tripling its reach on that side) and tries again; without a
-// bracket from an earlier launch a warp derives one from the first threshold it finds.  Per row:
+// bracket from an earlier launch a team derives one from the first threshold it finds.  Per row:
 //   1. the gate values are classified with plain float compares: values above the bracket are counted,
 //      values inside it are parked (raw bits) in the lane's column of shared memory;
 //   2. if the counts prove that the K-th largest value is a parked one, a 64-bin histogram over the
@@ -227,21 +227,9 @@ __host__ __device__ constexpr int warp_select_cand_words(int nv) {
 }
 constexpr int kWarpSelWords = 128;                       // bitmap words, at least (also scratch of the search)
 constexpr float kBracketTag = 20251109.0f;
-constexpr int kWarpSelMaxWarps = 8;                      // warps per CTA, at most
 
 // Words of shared memory one warp needs: gate row, up row, parked keys, bitmap, kept list, mbarrier.
 __host__ __device__ constexpr int warp_select_bitmap_words(int nv) { return nv * 4 > kWarpSelWords ? nv * 4 : kWarpSelWords; }
-// shared_u: the up row is copied into the gate row's buffer once the gate values are no longer needed there
-// (less shared memory per warp, so longer rows still get several warps per SM; no prefetch of the next gate row)
-__host__ __device__ constexpr size_t warp_select_words(int nv, int K, bool shared_u = false) {
-    return (size_t)nv * 128 + (shared_u ? 0 : (size_t)nv * 64) + warp_select_cand_words(nv) +
-           warp_select_bitmap_words(nv) + (size_t)((K + 3) & ~3) + 4;
-}
-// whether the kept channels' gate values fit the search scratch (see the kernel); shared_u needs it
-__host__ __device__ constexpr bool warp_select_parks_gates(int nv, int K) {
-    return K <= warp_select_cand_words(nv) + warp_select_bitmap_words(nv);
-}
-
 struct SelectMeta {
     float *bracket;      // {center, half width, tag}; rewritten by the last CTA of the launch
     float *acc;          // {sum of thresholds, sum of |threshold - center|, rows}: this launch's statistics
@@ -313,330 +301,15 @@ __device__ __noinline__ uint32_t warp_select_row_general(const float *g, int F, 
     return res;
 }
 
-// NV: number of 128-channel groups when known at compile time, 0: taken from nv_runtime
-// shared_u: one buffer for the gate row and, after step 3, the up row (see warp_select_words)
-template <int NV, bool shared_u>
-__global__ void __launch_bounds__(kWarpSelMaxWarps * 32) select_mask_rows_warp_kernel(
-    const float *__restrict__ G, int ldg, __nv_bfloat16 *__restrict__ U, int ldu, int64_t rows, int F, int nv_runtime, int K,
-    int16_t *__restrict__ idx_out, __nv_bfloat16 *__restrict__ g_out, __nv_bfloat16 *__restrict__ u_out,
-    SelectMeta meta, int *status) {
-    extern __shared__ __align__(128) uint32_t warp_sel_smem[];
-    __shared__ float s_stat[kWarpSelMaxWarps][3];
-    __shared__ int s_abort;
-    const int nv = NV > 0 ? NV : nv_runtime;
-    const int slots = warp_select_slots(nv);
-    const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5, wpc = blockDim.x >> 5;
-    uint32_t *base = warp_sel_smem + (size_t)wib * warp_select_words(nv, K, shared_u);
-    float *sg = reinterpret_cast<float *>(base);                                // [nv * 128] gate row
-    __nv_bfloat16 *su = reinterpret_cast<__nv_bfloat16 *>(shared_u ? base : base + nv * 128);  // up row -> Z' row
-    uint32_t *cand = base + nv * 128 + (shared_u ? 0 : nv * 64);                                 // [slot][lane] parked values
-    uint32_t *bitmap = cand + warp_select_cand_words(nv);                                     // kept-channel bitmap
-    uint32_t *kept = bitmap + warp_select_bitmap_words(nv);                                    // [K] channel | z bits << 16
-    uint64_t *bar_mem = reinterpret_cast<uint64_t *>(kept + ((K + 3) & ~3));
-    const uint32_t bar_g = smem_u32(bar_mem), bar_u = smem_u32(bar_mem + 1);  // gate row / up row arrived
-    // the kept channels' gate values are parked in the search scratch (free by then) when it is large enough: the
-    // gate buffer can then take the next token's row while this token's values are still being worked on
-    float *gkept = reinterpret_cast<float *>(cand);
-    const bool early_gate = warp_select_parks_gates(nv, K);  // (the host only asks for shared_u when this holds)
-    const int64_t gw = (int64_t)blockIdx.x * wpc + wib, nw = (int64_t)gridDim.x * wpc;
-    const float b_center = meta.bracket[0], b_width = meta.bracket[1];
-    const bool have_bracket = meta.bracket[2] == kBracketTag && b_width > 0.f && fabsf(b_center) <= 3.0e38f;
-    float cen = b_center, wid = b_width;  // this warp's bracket
-    bool have = have_bracket;
-    float st_sum = 0.f, st_abs = 0.f, st_n = 0.f;
-    const int words = (F + 31) >> 5;
-    const uint32_t g_bytes = (uint32_t)ldg * 4u, u_bytes = (uint32_t)ldu * 2u;  // multiples of 16: ld % 8 == 0
-
-    if (threadIdx.x == 0) s_abort = 0;
-    if (lane == 0) {
-        mbar_init(bar_g, 1);
-        mbar_init(bar_u, 1);
-    }
-    // channels the copies never write read as -inf for good
-    for (int c = ldg + lane; c < nv * 128; c += 32) sg[c] = -INFINITY;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    __syncthreads();
-    uint32_t phase = 0;  // both barriers complete once per token
-    bool dead = false;
-    if (lane == 0 && gw < rows && !shared_u) {
-        mbar_expect_tx(bar_g, g_bytes);
-        bulk_copy_g2s(smem_u32(sg), G + gw * (int64_t)ldg, g_bytes, bar_g);
-    }
-
-    for (int64_t r = gw; r < rows && !dead; r += nw) {
-        __nv_bfloat16 *u = U + r * (int64_t)ldu;
-        // ---- the up row is needed only in step 4: its copy starts now (once the previous token's store has read
-        //      the buffer) and lands while steps 1-3 run; the gate row was requested during the previous token
-        //      (one buffer for both rows: the gate row is requested here and the up row after step 3)
-        if (lane == 0) {
-            bulk_store_wait_read<0>();
-            fence_async_smem();
-            if (shared_u) {
-                mbar_expect_tx(bar_g, g_bytes);
-                bulk_copy_g2s(smem_u32(sg), G + r * (int64_t)ldg, g_bytes, bar_g);
-            } else {
-                mbar_expect_tx(bar_u, u_bytes);
-                bulk_copy_g2s(smem_u32(su), u, u_bytes, bar_u);
-            }
-        }
-        if (!__all_sync(0xffffffffu, mbar_wait(bar_g, phase, &s_abort, status))) {
-            dead = true;
-            break;
-        }
-        for (int c = F + lane; c < ldg; c += 32) sg[c] = -INFINITY;  // padding columns of this row
-        __syncwarp();
-
-        uint32_t tau = 0, res = 0;
-        bool fast = false, settled = false, no_cut = false;
-        float lo_f = cen - wid, hi_f = cen + wid;
-        for (int attempt = 0; have && attempt < 8; ++attempt) {
-            // ---- 1. classify: lane reads channels (v*32 + lane)*4 .. +3 of every 128-channel group v
-            uint32_t n_above = 0, n_mine = 0;
-#pragma unroll 4
-            for (int v = 0; v < nv; ++v) {
-                const float4 q = *reinterpret_cast<const float4 *>(sg + (v * 32 + lane) * 4);
-                const float e4[4] = {q.x, q.y, q.z, q.w};
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const float x = e4[e];
-                    n_above += x > hi_f ? 1u : 0u;
-                    const bool inside = x >= lo_f && x <= hi_f;
-                    if (inside) cand[min(n_mine, (uint32_t)slots) * 32 + lane] = __float_as_uint(x);
-                    n_mine += inside ? 1u : 0u;
-                }
-            }
-            const uint32_t c_hi = __reduce_add_sync(0xffffffffu, n_above);
-            const uint32_t n_band = __reduce_add_sync(0xffffffffu, n_mine);
-            const uint32_t max_mine = __reduce_max_sync(0xffffffffu, n_mine);
-            if (max_mine > (uint32_t)slots) {  // too many values inside: halve the bracket
-                const float c = 0.5f * (lo_f + hi_f), w = 0.25f * (hi_f - lo_f);
-                lo_f = c - w;
-                hi_f = c + w;
-                continue;
-            }
-            if (c_hi >= (uint32_t)K) {  // the threshold is above the bracket
-                const float w = hi_f - lo_f;
-                lo_f = hi_f;
-                hi_f += 2.f * w;
-                continue;
-            }
-            if (c_hi + n_band < (uint32_t)K) {  // ... below it
-                const float w = hi_f - lo_f;
-                hi_f = lo_f;
-                lo_f -= 2.f * w;
-                continue;
-            }
-            // ---- 2. the m-th largest parked key: a 64-bin histogram over the bracket's key range finds its
-            //         bin, the (few) keys of that bin are ranked against each other
-            const uint32_t lo_k = gate_key(lo_f), hi_k = gate_key(hi_f);
-            const uint32_t m = (uint32_t)K - c_hi;
-            uint32_t *hist = bitmap, *list = bitmap + 64, *list_n = bitmap + 96;
-            const uint32_t span = hi_k - lo_k;
-            const int shift = max(0, 26 - __clz(span | 1u));  // (span >> shift) < 64
-            hist[lane] = 0u;
-            hist[lane + 32] = 0u;
-            if (lane == 0) *list_n = 0u;
-            __syncwarp();
-            for (uint32_t s = 0; s < n_mine; ++s) {
-                const uint32_t key = gate_key(__uint_as_float(cand[s * 32 + lane]));
-                atomicAdd(&hist[(key - lo_k) >> shift], 1u);
-            }
-            __syncwarp();
-            const uint32_t h0 = hist[2 * lane], h1 = hist[2 * lane + 1], tot = h0 + h1;
-            uint32_t suf = tot;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const uint32_t nb = __shfl_down_sync(0xffffffffu, suf, o);
-                if (lane + o < 32) suf += nb;
-            }
-            const uint32_t above = suf - tot;  // keys in bins above 2 lane + 1
-            const bool f1 = above < m && m <= above + h1, f0 = above + h1 < m && m <= above + tot;
-            const int src = __ffs(__ballot_sync(0xffffffffu, f0 || f1)) - 1;  // one lane: 1 <= m <= n_band
-            const uint32_t tbin = __shfl_sync(0xffffffffu, (uint32_t)(2 * lane + (f1 ? 1 : 0)), src);
-            const uint32_t m2 = m - __shfl_sync(0xffffffffu, f1 ? above : above + h1, src);
-            const uint32_t nbin = __shfl_sync(0xffffffffu, f1 ? h1 : h0, src);
-            if (nbin <= 32u) {
-                for (uint32_t s = 0; s < n_mine; ++s) {
-                    const uint32_t key = gate_key(__uint_as_float(cand[s * 32 + lane]));
-                    if (((key - lo_k) >> shift) == tbin) list[atomicAdd(list_n, 1u)] = key;
-                }
-                __syncwarp();
-                const uint32_t mykey = (uint32_t)lane < nbin ? list[lane] : 0u;
-                uint32_t n_gt = 0, n_eq = 0;
-                for (uint32_t i = 0; i < nbin; ++i) {
-                    const uint32_t o = list[i];
-                    n_gt += o > mykey ? 1u : 0u;
-                    n_eq += o == mykey ? 1u : 0u;
-                }
-                const bool is_tau = (uint32_t)lane < nbin && n_gt < m2 && m2 <= n_gt + n_eq;
-                const int tl = __ffs(__ballot_sync(0xffffffffu, is_tau)) - 1;
-                res = __shfl_sync(0xffffffffu, mykey, tl);
-                // no tie to cut iff every key equal to the threshold is kept
-                no_cut = __shfl_sync(0xffffffffu, n_gt + n_eq, tl) == m2;
-                settled = true;
-            }
-            break;
-        }
-        __syncwarp();
-        const float tau_f = key_to_float(res);
-        if (settled && no_cut && fabsf(tau_f) <= 3.0e38f) {
-            // ---- 3. kept set = {g >= tau}.  Four flags per group go to the shared bitmap (channel
-            //         (v*32 + lane)*4 + e is bit (lane & 7) * 4 + e of word v*4 + lane / 8)
-            for (int w = lane; w < words; w += 32) bitmap[w] = 0u;
-            __syncwarp();
-#pragma unroll 4
-            for (int v = 0; v < nv; ++v) {
-                const float4 q = *reinterpret_cast<const float4 *>(sg + (v * 32 + lane) * 4);
-                const uint32_t nib = (q.x >= tau_f ? 1u : 0u) | (q.y >= tau_f ? 2u : 0u) |
-                                     (q.z >= tau_f ? 4u : 0u) | (q.w >= tau_f ? 8u : 0u);
-                if (nib) atomicOr(&bitmap[v * 4 + (lane >> 3)], nib << ((lane & 7) * 4));
-            }
-            __syncwarp();
-            // enumerate in ascending channel order: lane l owns words [l*wpl, (l+1)*wpl)
-            const int wpl = (words + 31) >> 5;
-            uint32_t mine = 0;
-            for (int i = 0; i < wpl; ++i) {
-                const int w = lane * wpl + i;
-                mine += w < words ? (uint32_t)__popc(bitmap[w]) : 0u;
-            }
-            uint32_t pre = mine;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const uint32_t nb = __shfl_up_sync(0xffffffffu, pre, o);
-                if (lane >= o) pre += nb;
-            }
-            if (__shfl_sync(0xffffffffu, pre, 31) == (uint32_t)K) {  // counts and compares agree
-                uint32_t pos = pre - mine;
-                for (int i = 0; i < wpl; ++i) {
-                    const int w = lane * wpl + i;
-                    uint32_t bits = w < words ? bitmap[w] : 0u;
-                    while (bits) {
-                        const int b = __ffs(bits) - 1;
-                        bits &= bits - 1u;
-                        kept[pos++] = (uint32_t)(w * 32 + b);
-                    }
-                }
-                tau = res;
-                fast = true;
-            }
-        }
-        __syncwarp();
-        if (!fast) tau = warp_select_row_general(sg, F, K, cand, kept);
-        __syncwarp();
-        // ---- 4. values of the kept channels (shared-memory gathers).  Gate values first, so that the gate buffer
-        //         can be handed to the next token's copy
-        auto request_next_gate = [&]() {
-            if (lane == 0 && r + nw < rows) {
-                fence_async_smem();
-                mbar_expect_tx(bar_g, g_bytes);
-                bulk_copy_g2s(smem_u32(sg), G + (r + nw) * (int64_t)ldg, g_bytes, bar_g);
-            }
-        };
-        if (early_gate) {
-            for (int i = lane; i < K; i += 32) gkept[i] = sg[kept[i]];
-            __syncwarp();
-            if (!shared_u) {
-                request_next_gate();
-            } else if (lane == 0) {
-                fence_async_smem();
-                mbar_expect_tx(bar_u, u_bytes);
-                bulk_copy_g2s(smem_u32(su), u, u_bytes, bar_u);
-            }
-        }
-        if (!__all_sync(0xffffffffu, mbar_wait(bar_u, phase, &s_abort, status))) {
-            dead = true;
-            break;
-        }
-        phase ^= 1u;
-        //         the compact outputs are written with consecutive lanes on consecutive slots
-        for (int i = lane; i < K; i += 32) {
-            const uint32_t j = kept[i];
-            const float gval = early_gate ? gkept[i] : sg[j];
-            const __nv_bfloat16 ub = su[j];
-            const __nv_bfloat16 zb = __float2bfloat16_rn(silu_f(gval) * __bfloat162float(ub));
-            kept[i] = j | ((uint32_t)(*reinterpret_cast<const uint16_t *>(&zb)) << 16);
-            if (idx_out) {
-                idx_out[r * K + i] = (int16_t)j;
-                g_out[r * K + i] = __float2bfloat16_rn(gval);
-                u_out[r * K + i] = ub;
-            }
-        }
-        __syncwarp();
-        if (!early_gate) request_next_gate();
-        // ---- up row -> masked Z' row, in shared memory, then one bulk store
-        uint4 *row16 = reinterpret_cast<uint4 *>(su);
-        for (int i = lane; i < (ldu >> 3); i += 32) row16[i] = make_uint4(0, 0, 0, 0);
-        __syncwarp();
-        for (int i = lane; i < K; i += 32) {
-            const uint32_t e = kept[i];
-            const uint16_t zb = (uint16_t)(e >> 16);
-            su[e & 0xffffu] = *reinterpret_cast<const __nv_bfloat16 *>(&zb);
-        }
-        fence_async_smem();
-        __syncwarp();
-        if (lane == 0) bulk_copy_s2g(u, smem_u32(su), u_bytes);
-        // ---- statistics for the next launch's bracket
-        const float t = key_to_float(tau);
-        if (fabsf(t) <= 3.0e38f) {
-            st_sum += t;
-            st_abs += have_bracket ? fabsf(t - b_center) : 0.f;
-            st_n += 1.f;
-            if (!have) {  // no bracket from an earlier launch: the warp makes its own from its first threshold
-                cen = t;
-                wid = 0.15f * fabsf(t) + 1e-30f;
-                have = true;
-            }
-        }
-    }
-    if (lane == 0) bulk_store_wait_all();
-    // ---- publish: per CTA one set of atomics; the last CTA turns the launch's statistics into the next bracket
-    if (lane == 0) {
-        s_stat[wib][0] = st_sum;
-        s_stat[wib][1] = st_abs;
-        s_stat[wib][2] = st_n;
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        float a = 0.f, b = 0.f, c = 0.f;
-        for (int w = 0; w < wpc; ++w) {
-            a += s_stat[w][0];
-            b += s_stat[w][1];
-            c += s_stat[w][2];
-        }
-        if (c > 0.f) {
-            atomicAdd(&meta.acc[0], a);
-            atomicAdd(&meta.acc[1], b);
-            atomicAdd(&meta.acc[2], c);
-        }
-        __threadfence();
-        // wrapping counter: back at zero after the last CTA, whatever it held when the workspace was new
-        if (atomicInc(meta.done, gridDim.x - 1) == gridDim.x - 1) {
-            __threadfence();
-            const float sum = atomicAdd(&meta.acc[0], 0.f), dev = atomicAdd(&meta.acc[1], 0.f),
-                        n = atomicAdd(&meta.acc[2], 0.f);
-            if (n > 0.f) {
-                const float center = sum / n;
-                // five mean absolute deviations (about four standard deviations) once a center existed to
-                // measure them against; 15 % of the center otherwise; never narrower than 2 %
-                float width = have_bracket ? 5.0f * dev / n : 0.15f * fabsf(center);
-                width = fmaxf(width, 0.02f * fabsf(center) + 1e-30f);
-                meta.bracket[0] = center;
-                meta.bracket[1] = width;
-                meta.bracket[2] = kBracketTag;
-            } else {
-                meta.bracket[2] = 0.f;
-            }
-            meta.acc[0] = meta.acc[1] = meta.acc[2] = 0.f;
-        }
-    }
-}
-
 // ------------------------------------------------------------------------------------------------
-// The same selector with a TEAM of W = 2 or 4 warps per token (same staging, same steps, same exactness): the
-// team shares one slice of shared memory, warp w takes the 128-channel groups w, w + W, ... in steps 1 and 3 and
-// every W-th batch of kept channels in step 4, and the warps meet at a named barrier of their own between the
-// steps.  A token's rows occupy the slice for a fraction of the time, so the shared memory of an SM (which
-// bounds the tokens in flight) feeds W times as many warps.
+// The kernel.  Warp w of a team of W takes the 128-channel groups w, w + W, ... in steps 1 and 3 and every W-th
+// batch of kept channels in step 4; the warps meet at the team's named barrier between the steps.  The shared
+// memory of an SM bounds the tokens in flight, so W warps per token make it feed W times as many warps (measured
+// against one warp per token: 2048 channels 0.086 -> 0.080 ms with pairs; 5504 channels 0.85 -> 0.50 ms and 11008
+// channels 0.68 -> 0.41 ms with teams of four).
+// shared_u: the up row is copied into the gate row's buffer once the gate values are no longer needed there
+// (less shared memory per token, so longer rows still fit; no prefetch of the next gate row).  It is a template
+// parameter: as a run-time flag it slowed the common path by a quarter.
 __host__ __device__ constexpr size_t pair_select_words(int nv, int K, bool shared_u, int W = 2) {
     return (size_t)nv * 128 + (shared_u ? 0 : (size_t)nv * 64) + (size_t)W * warp_select_cand_words(nv) +
            warp_select_bitmap_words(nv) + (size_t)((K + 3) & ~3) + 32 /* exchange */ + 4 /* two mbarriers */;

@@ -447,17 +447,3 @@ def test_full_size_sweep_workload_sampled_against_oracle(K):
     """C5 at its full 65536 tokens with the smallest and the largest K of the sweep (d_ff / 16 and d_ff / 4)."""
     import dataclasses
     _full_size_sampled(dataclasses.replace(syn.C5, k=K, name=f"C5-k{K}"), 32, 8)
-
-
-def test_one_warp_per_token_selector_selected_by_environment():
-    """MOC_FFN_SELECT=warp (read once per process) routes the tensor-core forward to the one-warp-per-token selector
-    instead of the default two: run the shape, tie and chunking cases again in a child process with it set."""
-    import os
-    import subprocess
-    import sys
-    env = dict(os.environ, MOC_FFN_SELECT="warp")
-    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
-    r = subprocess.run([sys.executable, "-m", "pytest", os.path.join(root, "tests", "test_gpu_parity.py"), "-q", "-x",
-                        "-m", "gpu", "-k", "tc_plan_shapes or ties_go or several_token_chunks or llama1b_padded_slice or degenerate"],
-                       cwd=root, env=env, capture_output=True, text=True, timeout=900)
-    assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
