@@ -312,7 +312,7 @@ __device__ __noinline__ uint32_t warp_select_row_general(const float *g, int F, 
 // parameter: as a run-time flag it slowed the common path by a quarter.
 __host__ __device__ constexpr size_t pair_select_words(int nv, int K, bool shared_u, int W = 2) {
     return (size_t)nv * 128 + (shared_u ? 0 : (size_t)nv * 64) + (size_t)W * warp_select_cand_words(nv) +
-           warp_select_bitmap_words(nv) + (size_t)((K + 3) & ~3) + 32 /* exchange */ + 4 /* two mbarriers */;
+           warp_select_bitmap_words(nv) + (size_t)((K + 3) & ~3) + 40 /* exchange */ + 4 /* two mbarriers */;
 }
 __host__ __device__ constexpr bool pair_select_parks_gates(int nv, int K, int W = 2) {
     return K <= W * warp_select_cand_words(nv) + warp_select_bitmap_words(nv);
@@ -341,7 +341,7 @@ __global__ void __launch_bounds__(kPairSelMaxWarps * 32, 2) select_mask_rows_pai
     uint32_t *bitmap = cand0 + W * cw;
     uint32_t *kept = bitmap + warp_select_bitmap_words(nv);
     uint32_t *xch = kept + ((K + 3) & ~3);  // [2 parities][W warps][4] counts exchanged between the warps
-    uint64_t *bar_mem = reinterpret_cast<uint64_t *>(xch + 32);
+    uint64_t *bar_mem = reinterpret_cast<uint64_t *>(xch + 40);  // (xch[32..35]: the warps' wait verdicts)
     const uint32_t bar_g = smem_u32(bar_mem), bar_u = smem_u32(bar_mem + 1);
     float *gkept = reinterpret_cast<float *>(cand0);
     const bool early_gate = pair_select_parks_gates(nv, K, W);
@@ -385,13 +385,23 @@ __global__ void __launch_bounds__(kPairSelMaxWarps * 32, 2) select_mask_rows_pai
                 bulk_copy_g2s(smem_u32(su), u, u_bytes, bar_u);
             }
         }
-        if (!__all_sync(0xffffffffu, mbar_wait(bar_g, phase, &s_abort, status))) dead = true;
-        if (!dead)
+        // a wait that gave up ends the team: the warps exchange their verdicts so that all of them leave together
+        // (another team's time-out can make one warp's wait return early and not its partner's)
+        const auto team_agrees = [&](bool ok) {
+            if (lane == 0) xch[32 + w] = ok ? 1u : 0u;
+            pair_sync();
+            bool all_ok = true;
+#pragma unroll
+            for (int i = 0; i < W; ++i) all_ok = all_ok && xch[32 + i] != 0u;
+            return all_ok;
+        };
+        const bool g_ok = __all_sync(0xffffffffu, mbar_wait(bar_g, phase, &s_abort, status));
+        if (g_ok)
             for (int c = F + pl; c < ldg; c += TT) sg[c] = -INFINITY;
-        // the partner must see the same verdict: a failed wait ends the pair (s_abort is set block-wide)
-        pair_sync();
-        if (s_abort) dead = true;
-        if (dead) break;
+        if (!team_agrees(g_ok)) {
+            dead = true;
+            break;
+        }
 
         uint32_t tau = 0, res = 0;
         bool fast = false, settled = false, no_cut = false;
@@ -581,10 +591,10 @@ __global__ void __launch_bounds__(kPairSelMaxWarps * 32, 2) select_mask_rows_pai
                 bulk_copy_g2s(smem_u32(su), u, u_bytes, bar_u);
             }
         }
-        if (!__all_sync(0xffffffffu, mbar_wait(bar_u, phase, &s_abort, status))) dead = true;
-        pair_sync();
-        if (s_abort) dead = true;
-        if (dead) break;
+        if (!team_agrees(__all_sync(0xffffffffu, mbar_wait(bar_u, phase, &s_abort, status)))) {
+            dead = true;
+            break;
+        }
         phase ^= 1u;
         for (int i = pl; i < K; i += TT) {
             const uint32_t j = kept[i];
@@ -777,7 +787,7 @@ __global__ void __launch_bounds__(256) backward_sample_rows_kernel(
 // coalesced and the scattered accesses stay on chip.  Used when the four rows of a token fit a slice.
 __host__ __device__ constexpr size_t sample_warp_words(int ld, int K) {
     return (size_t)2 * ld /* four bf16 rows */ + (size_t)2 * ((K + 1) & ~1) /* entries */ +
-           (size_t)3 * ((K + 7) & ~7) /* saved idx, g, u of two tokens */ + 4 /* two mbarriers */;
+           (size_t)3 * ((K + 7) & ~7) /* saved idx, g, u of two tokens */ + 4 /* two mbarriers */ + 4 /* verdicts */;
 }
 constexpr int kSampleMaxWarps = 10;
 
@@ -835,9 +845,19 @@ __global__ void __launch_bounds__(kSampleMaxWarps * 32) backward_sample_rows_war
     if (pl == 0 && gw < T) request(gw, 0);
     int b = 0;
     for (int64_t t = gw; t < T; t += nw, b ^= 1) {
-        mbar_wait(bar0 + 8u * (uint32_t)b, (phases >> b) & 1u, &s_abort, status);  // a failed wait sets s_abort
-        team_sync();
-        if (s_abort) break;  // the whole team sees the same flag after the barrier
+        // a wait that gave up ends the team: the warps exchange their verdicts so that all of them leave together
+        const bool ok = __all_sync(0xffffffffu, mbar_wait(bar0 + 8u * (uint32_t)b, (phases >> b) & 1u, &s_abort, status));
+        if (W > 1) {
+            uint32_t *verdict = reinterpret_cast<uint32_t *>(bar_mem + 2);
+            if (lane == 0) verdict[wib % W] = ok ? 1u : 0u;
+            team_sync();
+            bool all_ok = true;
+#pragma unroll
+            for (int i = 0; i < W; ++i) all_ok = all_ok && verdict[i] != 0u;
+            if (!all_ok) break;
+        } else if (!ok) {
+            break;
+        }
         phases ^= 1u << b;
         __nv_bfloat16 *zr = zbuf0 + (size_t)b * ld;
         const uint16_t *sv = saved0 + (size_t)b * 3 * K8;
