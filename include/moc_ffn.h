@@ -173,6 +173,15 @@ MOC_API int moc_tc_gemm_bf16(int64_t m, int64_t n, int64_t k, const void *a, int
                              void *cuda_stream);
 
 /*
+ * Test hook for the time-out path every kernel of the library shares: launches one warp that waits, with the
+ * library's bounded wait, on a barrier nothing completes.  After `limit_cycles` SM clock cycles (1 .. 4e9) the wait
+ * gives up, the kernel raises MOC_ERR_TIMEOUT in the device status word and returns normally; nothing traps or
+ * faults, and the context stays usable.  Returns MOC_OK when the launch was enqueued.  (The paper has no
+ * counterpart: it is how the error behaviour stated above is checked.)
+ */
+MOC_API int moc_test_bounded_wait(int64_t limit_cycles, void *cuda_stream);
+
+/*
  * Synchronises `cuda_stream`, then returns and clears the current device's sticky status word:
  * MOC_OK, MOC_ERR_TIMEOUT or MOC_ERR_BAD_INDEX (MOC_ERR_CUDA if the synchronisation itself failed).
  */

@@ -79,6 +79,8 @@ def load() -> ctypes.CDLL:
         lib.moc_topk_select.restype = ctypes.c_int
         lib.moc_topk_select.argtypes = [ctypes.c_int64, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, vp, vp, vp]
         lib.moc_last_device_status.restype = ctypes.c_int
+        lib.moc_test_bounded_wait.argtypes = [ctypes.c_int64, vp]
+        lib.moc_test_bounded_wait.restype = ctypes.c_int
         lib.moc_last_device_status.argtypes = [vp]
         lib.moc_status_string.restype = ctypes.c_char_p
         lib.moc_status_string.argtypes = [ctypes.c_int]
@@ -255,6 +257,14 @@ def moc_topk_select(gate: torch.Tensor, k: int, n: int | None = None, stream=Non
 
 def moc_last_device_status(stream=None) -> int:
     return int(load().moc_last_device_status(_stream_ptr(stream)))
+
+
+def moc_test_bounded_wait(limit_cycles: int, stream=None) -> None:
+    """Launches the probe whose bounded wait runs out after `limit_cycles` SM cycles (the status word then reads
+    MOC_ERR_TIMEOUT)."""
+    rc = load().moc_test_bounded_wait(int(limit_cycles), _stream_ptr(stream))
+    if rc != MOC_OK:
+        raise MocError(rc, "moc_test_bounded_wait")
 
 
 def moc_launch_count() -> int:

@@ -865,6 +865,15 @@ int moc_tc_gemm_bf16(int64_t m, int64_t n, int64_t k, const void *a, int a_mn_ma
     return rc;
 }
 
+int moc_test_bounded_wait(int64_t limit_cycles, void *cuda_stream) {
+    if (limit_cycles < 1 || limit_cycles > tc::kWaitLimitCycles) return MOC_ERR_INVALID_ARG;
+    int *status = device_status_ptr();
+    if (!status) return MOC_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    tc::bounded_wait_probe_kernel<<<1, 32, 0, st>>>((long long)limit_cycles, status, nullptr);
+    return launch_ok();
+}
+
 int moc_last_device_status(void *cuda_stream) {
     if (cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return MOC_ERR_CUDA;
     int *p = device_status_ptr();

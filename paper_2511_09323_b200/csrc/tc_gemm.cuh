@@ -88,15 +88,18 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-// Bounded wait (about two seconds of SM clock).  Returns false when it gave up or another role already did.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status) {
+// Bounded wait (by default about two seconds of SM clock).  Returns false when it gave up or another role already
+// did; giving up raises MOC_ERR_TIMEOUT in the device status word and sets *abort_flag.
+constexpr long long kWaitLimitCycles = 4000000000LL;
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status,
+                                          long long limit_cycles = kWaitLimitCycles) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     uint32_t spins = 0;
     while (!mbar_try_wait(bar, parity)) {
         if ((++spins & 0x3ff) == 0) {
             if (*abort_flag) return false;
-            if (clock64() - t0 > 4000000000LL) {
+            if (clock64() - t0 > limit_cycles) {
                 *abort_flag = 1;
                 raise_status(status, MOC_ERR_TIMEOUT);
                 return false;
@@ -766,6 +769,23 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_pair_kernel(const __grid_cons
         tc_fence_after();
         tmem_dealloc_pair(tmem_base, TMEM_COLS);
     }
+}
+
+// ---------------------------------------------------------------------------------------------- wait probe
+// One warp waits, with the bounded wait every kernel here uses, on an mbarrier that nothing ever completes.  The
+// wait runs out after `limit_cycles`, raises MOC_ERR_TIMEOUT and the kernel returns normally: the test of the
+// time-out path (nothing traps, faults or spins without end).
+__global__ void bounded_wait_probe_kernel(long long limit_cycles, int *status, int *gave_up) {
+    __shared__ uint64_t bar;
+    __shared__ int s_abort;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        s_abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    const bool ok = mbar_wait(smem_u32(&bar), 0, &s_abort, status, limit_cycles);
+    if (threadIdx.x == 0 && gave_up) *gave_up = ok ? 0 : 1;
 }
 
 }  // namespace tc

@@ -447,3 +447,20 @@ def test_full_size_sweep_workload_sampled_against_oracle(K):
     """C5 at its full 65536 tokens with the smallest and the largest K of the sweep (d_ff / 16 and d_ff / 4)."""
     import dataclasses
     _full_size_sampled(dataclasses.replace(syn.C5, k=K, name=f"C5-k{K}"), 32, 8)
+
+
+def test_bounded_wait_runs_out_reports_timeout_and_leaves_the_context_usable():
+    """The time-out path all kernels share: a wait on a barrier nothing completes gives up after its limit (here
+    50 M cycles, about 25 ms), the kernel returns normally, the status word reads MOC_ERR_TIMEOUT once, and the
+    next call works."""
+    import time
+    assert B.moc_last_device_status() == B.MOC_OK
+    t0 = time.perf_counter()
+    B.moc_test_bounded_wait(50_000_000)
+    assert B.moc_last_device_status() == B.MOC_ERR_TIMEOUT          # synchronises, reports, clears
+    assert time.perf_counter() - t0 < 2.0
+    assert B.moc_last_device_status() == B.MOC_OK
+    with pytest.raises(B.MocError):
+        B.moc_test_bounded_wait(0)                                   # limit out of range: nothing launched
+    _run_forward_backward(syn.Workload("after-timeout", "bf16", 300, 128, 512, 512, 64, seed=9))
+    assert B.moc_last_device_status() == B.MOC_OK
