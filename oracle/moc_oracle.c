@@ -159,6 +159,46 @@ int moc_oracle_topk_f32(int64_t rows, int32_t F, int64_t ld, int32_t K, const fl
     return err ? MOC_ORACLE_NOMEM : MOC_ORACLE_OK;
 }
 
+/* Grouped selection, the a:b form (Section 4, "MoC with structured 2:8 sparsity"; Appendix, Theorem 1): the row is
+ * cut into consecutive groups of `group` channels and in every group the `keep` channels with the largest signed
+ * pre-SiLU gate values are kept (the input-based key of Section 3.2; equal values: the lower channel; NaN as -inf).
+ * F must be a multiple of `group`.  idx_out [rows, keep * F / group], ascending.
+ * Brute force: every group is sorted on its own with the comparator of the global rule. */
+int moc_oracle_topk_grouped(int64_t rows, int32_t F, int64_t ld, int32_t group, int32_t keep, const double *gate,
+                            int32_t *idx_out)
+{
+    if (rows < 0 || F < 1 || group < 1 || keep < 1 || keep > group || F % group != 0 || ld < F || !gate || !idx_out)
+        return MOC_ORACLE_BAD_ARG;
+    const int32_t groups = F / group;
+    const int64_t K = (int64_t)groups * keep;
+    int err = 0;
+#pragma omp parallel
+    {
+        keyed_t *scratch = (keyed_t *)malloc((size_t)group * sizeof(keyed_t));
+        if (!scratch) {
+#pragma omp atomic write
+            err = 1;
+        }
+#pragma omp for schedule(static)
+        for (int64_t t = 0; t < rows; ++t) {
+            if (!scratch) continue;
+            for (int32_t q = 0; q < groups; ++q) {
+                for (int32_t e = 0; e < group; ++e) {
+                    double v = gate[t * ld + (int64_t)q * group + e];
+                    scratch[e].key = isnan(v) ? -INFINITY : v;
+                    scratch[e].j = q * group + e;
+                }
+                qsort(scratch, (size_t)group, sizeof(keyed_t), cmp_keyed);
+                int32_t *dst = idx_out + t * K + (int64_t)q * keep;
+                for (int32_t k = 0; k < keep; ++k) dst[k] = scratch[k].j;
+                qsort(dst, (size_t)keep, sizeof(int32_t), cmp_i32);
+            }
+        }
+        free(scratch);
+    }
+    return err ? MOC_ORACLE_NOMEM : MOC_ORACLE_OK;
+}
+
 /* ---------------------------------------------------------------- forward */
 
 static double dot(const double *a, const double *b, int32_t n)

@@ -133,6 +133,40 @@ def topk(gate, K: int, F: int | None = None):
     return idx
 
 
+def topk_grouped(gate, group: int = 8, keep: int = 2, F: int | None = None):
+    """Grouped selection (the a:b form, keep of every `group` consecutive channels; Section 4 and Theorem 1):
+    [rows, keep * F / group] channel indices, ascending."""
+    gate = _f64(np.ascontiguousarray(gate))
+    if gate.ndim != 2:
+        raise ValueError("gate must be 2-D")
+    rows, ld = gate.shape
+    F = ld if F is None else F
+    if F % group:
+        raise ValueError("F must be a multiple of the group size")
+    idx = np.empty((rows, F // group * keep), dtype=np.int32)
+    rc = _load().moc_oracle_topk_grouped(ctypes.c_int64(rows), ctypes.c_int32(F), ctypes.c_int64(ld),
+                                         ctypes.c_int32(group), ctypes.c_int32(keep), _p(gate), _p(idx))
+    _check(rc, "moc_oracle_topk_grouped")
+    return idx
+
+
+def gate_projection(x, w_gate, F: int | None = None):
+    """G = X W_gate (Eq. (Moc-1)) for the first F channels, [T, F] float64."""
+    x, w_gate = _f64(x), _f64(w_gate)
+    F = w_gate.shape[0] if F is None else F
+    return x @ w_gate[:F].T
+
+
+def forward_grouped(x, w_gate, w_up, w_down, group: int = 8, keep: int = 2, F: int | None = None):
+    """The layer with the grouped mask: gate projection, grouped selection, then the steps of the layer on the
+    selected channels.  Returns dict(out, idx, gval, uval, g)."""
+    g = gate_projection(x, w_gate, F)
+    idx = topk_grouped(g, group, keep)
+    res = forward_given_idx(x, w_gate, w_up, w_down, idx, F=F)
+    res["idx"], res["g"] = idx, g
+    return res
+
+
 def forward(x, w_gate, w_up, w_down, K: int, F: int | None = None, want_g: bool = False):
     """Returns dict(out, idx, gval, uval[, g]); weights are [>=F, d] channel-major."""
     x = _f64(x)

@@ -419,3 +419,87 @@ def test_bad_arguments_are_rejected():
         orc.forward(x, wg, wu, wd, K=5)
     with pytest.raises(RuntimeError):
         orc.forward_given_idx(x, wg, wu, wd, np.array([[0, 4], [1, 2]], dtype=np.int32))
+
+
+# ------------------------------------------------------------------ grouped selection (MoC 2:8, Section 4; Theorem 1)
+
+
+def _np_grouped_sets(g, group, keep):
+    """Brute force by counting: a channel is kept when fewer than `keep` channels of its group precede it in
+    (value descending, channel ascending) order.  No sort involved."""
+    g = np.where(np.isnan(g), -np.inf, g) + 0.0
+    rows, F = g.shape
+    out = []
+    for t in range(rows):
+        kept = []
+        for q in range(F // group):
+            for e in range(group):
+                j = q * group + e
+                before = sum(1 for f in range(group)
+                             if g[t, q * group + f] > g[t, j] or (g[t, q * group + f] == g[t, j] and f < e))
+                if before < keep:
+                    kept.append(j)
+        out.append(kept)
+    return np.asarray(out, dtype=np.int32)
+
+
+@pytest.mark.parametrize("group,keep", [(8, 2), (4, 1), (8, 8), (2, 1)])
+def test_grouped_selection_brute_force(group, keep):
+    rng = np.random.default_rng(group * 10 + keep)
+    g = rng.standard_normal((7, 8 * group))
+    g[1, :] = 0.5                                   # all equal: the first `keep` channels of every group
+    g[2, ::2] = g[2, 1::2]                          # pairs of equal values
+    g[3, 3] = np.nan
+    g[3, 4] = np.inf
+    g[4, :group] = [-0.0, 0.0] * (group // 2) if group % 2 == 0 else 0.0
+    g[5] = np.round(g[5] * 2) / 2                   # many ties
+    got = orc.topk_grouped(g, group, keep)
+    assert np.array_equal(got, _np_grouped_sets(g, group, keep))
+    assert np.array_equal(got[1], np.concatenate([np.arange(q * group, q * group + keep) for q in range(8)]))
+    # exactly `keep` per group, ascending
+    assert np.all(np.diff(got, axis=1) > 0)
+    assert np.all((got // group) == np.repeat(np.arange(8), keep)[None, :])
+
+
+def test_grouped_selection_with_one_group_is_the_global_rule():
+    rng = np.random.default_rng(5)
+    g = rng.standard_normal((9, 24))
+    g[0, 5] = g[0, 17]
+    assert np.array_equal(orc.topk_grouped(g, group=24, keep=7), orc.topk(g, 7))
+    assert np.array_equal(orc.topk_grouped(g, group=24, keep=7), _np_topk_sets(g, 7))
+
+
+def test_grouped_forward_keep_all_is_dense_swiglu_and_matches_dense_masked_form():
+    x, wg, wu, wd = _rand_problem(21, T=6, d=10, F=32)
+    full = orc.forward_grouped(x, wg, wu, wd, group=8, keep=8)
+    dense = (_np_silu(x @ wg.T) * (x @ wu.T)) @ wd
+    np.testing.assert_allclose(full["out"], dense, rtol=1e-12, atol=1e-13)
+    # 2 of 8: Eqs. (Moc-1), mask, (MoC-2) written as dense matrices with the grouped mask
+    res = orc.forward_grouped(x, wg, wu, wd, group=8, keep=2)
+    G, U = x @ wg.T, x @ wu.T
+    M = np.zeros_like(G)
+    np.put_along_axis(M, _np_grouped_sets(G, 8, 2).astype(np.int64), 1.0, axis=1)
+    np.testing.assert_allclose(res["out"], (_np_silu(G) * M * U) @ wd, rtol=1e-12, atol=1e-13)
+    np.testing.assert_allclose(res["gval"], np.take_along_axis(G, res["idx"].astype(np.int64), axis=1), rtol=1e-13)
+
+
+def test_theorem_1_embedding_dense_ffn_into_2_of_8():
+    """Theorem 1 with a:b = 2:8: a dense SwiGLU FFN of width d_ffn is reproduced exactly by MoC 2:8 of width
+    8 * ceil(d_ffn / 2) whose groups hold two real channels and six zero channels.  With the input-based key the
+    zero channels must not beat the real ones, so the inputs are chosen with all real gate values positive."""
+    rng = np.random.default_rng(8)
+    d, d_ffn = 6, 7
+    x = rng.uniform(0.1, 1.0, (5, d))
+    wg = rng.uniform(0.05, 0.5, (d_ffn, d))          # x, wg > 0: every real gate value exceeds the padded channels' 0
+    wu = rng.standard_normal((d_ffn, d))
+    wd = rng.standard_normal((d_ffn, d))
+    groups = -(-d_ffn // 2)
+    wg2, wu2, wd2 = (np.zeros((8 * groups, d)) for _ in range(3))
+    for j in range(d_ffn):
+        q, r = divmod(j, 2)
+        wg2[q * 8 + r], wu2[q * 8 + r], wd2[q * 8 + r] = wg[j], wu[j], wd[j]
+    dense = (_np_silu(x @ wg.T) * (x @ wu.T)) @ wd
+    moc = orc.forward_grouped(x, wg2, wu2, wd2, group=8, keep=2)
+    np.testing.assert_allclose(moc["out"], dense, rtol=1e-12, atol=1e-13)
+    # a group whose second real slot is padding keeps a zero channel, which contributes nothing
+    assert moc["idx"].shape == (5, 2 * groups)
