@@ -67,6 +67,13 @@ typedef enum { MOC_OP_FORWARD = 0, MOC_OP_BACKWARD = 1, MOC_OP_DECODE = 2 } moc_
 
 /* bit 0 of moc_ffn_desc.flags: add into grad_w_* instead of overwriting them */
 #define MOC_FLAG_ACCUMULATE_WGRAD 1u
+/* bit 1: grouped mask, MoC 2:8 (Section 4, "MoC with structured 2:8 sparsity"; Theorem 1 states the a:b form):
+ * instead of the K largest gate values of the whole row, the 2 largest of every group of 8 consecutive channels are
+ * kept (signed pre-SiLU values, equal values: the lower channel, NaN as -inf).  Requires d_ff % 8 == 0 and
+ * k == d_ff / 4; the kept channels of group q occupy slots 2q and 2q + 1 of topk_idx / topk_gate / topk_up.
+ * Honoured by moc_ffn_forward, moc_ffn_decode and moc_ffn_decode_static; moc_ffn_backward takes the saved
+ * indices as they are (the flag changes nothing there). */
+#define MOC_FLAG_SELECT_2_OF_8 2u
 
 typedef struct moc_ffn_desc {
     int64_t tokens;   /* T = batch * seq, >= 0 (0 is a no-op)                                   */

@@ -20,6 +20,8 @@
  *   moc_oracle_topk               the mask definition of Section 3.2: exactly K ones per row,
  *                                 the K largest SIGNED pre-SiLU values.
  *   moc_oracle_forward_given_idx  Eq. (MoC-2) with the mask M supplied by the caller.
+ *   moc_oracle_topk_grouped       the a:b mask of Section 4 ("MoC with structured 2:8 sparsity") and Theorem 1:
+ *                                 the `keep` largest signed pre-SiLU values of every `group` consecutive channels.
  *   moc_oracle_backward           Section 4, Eqs. (bp-1)..(bp-5), with S' and Z' recomputed from the
  *                                 saved G.M and U.M ("MoC + GCP", Table 1).
  *   moc_oracle_silu / dsilu       Eq. (silu) and its derivative.

@@ -108,3 +108,34 @@ def check_backward(dev: dict, x, w_gate, w_up, w_down, idx, gval, uval, grad_out
             got = got[:F]
         rep["grad_" + n] = assert_close(got, ref["grad_" + n], dtype, "grad_" + n)
     return rep
+
+
+def check_picks_grouped(idx_dev: np.ndarray, g_oracle: np.ndarray, group: int = 8, keep: int = 2,
+                        band: float = PICK_BAND):
+    """Rule 1 for the grouped (a:b) mask: per token and group, the device's channels may differ from the oracle's
+    only by channels whose oracle gate value lies within ``band`` of that group's keep-th largest value.
+    Returns the number of groups whose set differs."""
+    idx_ref = orc.topk_grouped(g_oracle, group, keep)
+    idx_dev = np.asarray(idx_dev).astype(np.int64)
+    T, F = g_oracle.shape
+    check_index_sets(idx_dev, F)
+    groups = F // group
+    if idx_dev.shape != (T, groups * keep):
+        raise AssertionError(f"grouped index shape {idx_dev.shape}")
+    if not np.array_equal(idx_dev // group, np.repeat(np.arange(groups), keep)[None, :].repeat(T, axis=0)):
+        raise AssertionError("not exactly `keep` channels in every group")
+    key = np.where(np.isnan(g_oracle), -np.inf, g_oracle)
+    differing = 0
+    diff_rows, diff_cols = np.nonzero(idx_dev != idx_ref)
+    for t, c in zip(diff_rows.tolist(), diff_cols.tolist()):
+        q = c // keep
+        vals = np.sort(key[t, q * group:(q + 1) * group])[::-1]
+        tau = vals[keep - 1]
+        a = set(idx_dev[t, q * keep:(q + 1) * keep].tolist())
+        b = set(idx_ref[t, q * keep:(q + 1) * keep].tolist())
+        for j in a ^ b:
+            if abs(key[t, j] - tau) > band:
+                raise AssertionError(f"token {t} group {q}: channel {j} (g={key[t, j]:.6g}) differs outside the band "
+                                     f"around {tau:.6g}")
+        differing += 1
+    return differing

@@ -26,6 +26,7 @@ MOC_STATIC_MAX_TOKENS, MOC_STATIC_MAX_DFF = 16, 16384
 MOC_F32, MOC_BF16 = 0, 1
 MOC_OP_FORWARD, MOC_OP_BACKWARD, MOC_OP_DECODE = 0, 1, 2
 MOC_FLAG_ACCUMULATE_WGRAD = 1
+MOC_FLAG_SELECT_2_OF_8 = 2
 
 EXPORTED = (
     "moc_ffn_workspace_bytes", "moc_ffn_forward", "moc_ffn_backward", "moc_ffn_decode", "moc_topk_select",
@@ -151,13 +152,26 @@ def alloc_workspace(desc: MocFfnDesc, op: int, device=None) -> torch.Tensor:
     return torch.empty(max(n, 16), dtype=torch.uint8, device=device or torch.device("cuda"))
 
 
+def _grouped_k(k, d_ff):
+    """k of the 2-of-8 mask (d_ff / 4); a caller may pass it or leave it None."""
+    if d_ff % 8:
+        raise ValueError("the 2-of-8 mask needs d_ff to be a multiple of 8")
+    if k is not None and int(k) != d_ff // 4:
+        raise ValueError("the 2-of-8 mask keeps d_ff / 4 channels")
+    return d_ff // 4
+
+
 def moc_ffn_forward(x, w_gate, w_up, w_down, k, d_ff=None, save=True, out=None, saved=None, workspace=None,
-                    stream=None):
-    """Returns (out, topk_idx, topk_gate, topk_up); the last three are None when save=False."""
+                    stream=None, grouped=False):
+    """Returns (out, topk_idx, topk_gate, topk_up); the last three are None when save=False.
+    grouped=True: the 2-of-8 mask (MOC_FLAG_SELECT_2_OF_8) instead of the row Top-K; k is then d_ff / 4."""
     _check_dev(x, w_gate, w_up, w_down, out, workspace)
     T, d = x.shape
     F_ld = w_gate.shape[0]
-    desc = make_desc(T, d, F_ld if d_ff is None else d_ff, k, x.dtype, d_ff_ld=F_ld)
+    if grouped:
+        k = _grouped_k(k, F_ld if d_ff is None else d_ff)
+    desc = make_desc(T, d, F_ld if d_ff is None else d_ff, k, x.dtype, d_ff_ld=F_ld,
+                     flags=MOC_FLAG_SELECT_2_OF_8 if grouped else 0)
     if out is None:
         out = torch.empty_like(x)
     if save:
@@ -210,11 +224,14 @@ def moc_ffn_backward(x, w_gate, w_up, w_down, topk_idx, topk_gate, topk_up, grad
     return res
 
 
-def moc_ffn_decode(x, w_gate, w_up, w_down, k, d_ff=None, out=None, workspace=None, stream=None):
+def moc_ffn_decode(x, w_gate, w_up, w_down, k, d_ff=None, out=None, workspace=None, stream=None, grouped=False):
     _check_dev(x, w_gate, w_up, w_down, out, workspace)
     T, d = x.shape
     F_ld = w_gate.shape[0]
-    desc = make_desc(T, d, F_ld if d_ff is None else d_ff, k, x.dtype, d_ff_ld=F_ld)
+    if grouped:
+        k = _grouped_k(k, F_ld if d_ff is None else d_ff)
+    desc = make_desc(T, d, F_ld if d_ff is None else d_ff, k, x.dtype, d_ff_ld=F_ld,
+                     flags=MOC_FLAG_SELECT_2_OF_8 if grouped else 0)
     if out is None:
         out = torch.empty_like(x)
     if workspace is None:
@@ -226,14 +243,17 @@ def moc_ffn_decode(x, w_gate, w_up, w_down, k, d_ff=None, out=None, workspace=No
     return out
 
 
-def moc_ffn_decode_static(x, w_gate, w_up, w_down, k, out, d_ff=None, stream=None):
+def moc_ffn_decode_static(x, w_gate, w_up, w_down, k, out, d_ff=None, stream=None, grouped=False):
     """Decode for callers that cannot allocate: no workspace argument, and `out` must be supplied, so that
     nothing on this call path asks any allocator (torch's included) for memory.  The transient buffers
     live in an array inside the library; see the limits and the sharing rules in include/moc_ffn.h."""
     _check_dev(x, w_gate, w_up, w_down, out)
     T, d = x.shape
     F_ld = w_gate.shape[0]
-    desc = make_desc(T, d, F_ld if d_ff is None else d_ff, k, x.dtype, d_ff_ld=F_ld)
+    if grouped:
+        k = _grouped_k(k, F_ld if d_ff is None else d_ff)
+    desc = make_desc(T, d, F_ld if d_ff is None else d_ff, k, x.dtype, d_ff_ld=F_ld,
+                     flags=MOC_FLAG_SELECT_2_OF_8 if grouped else 0)
     rc = load().moc_ffn_decode_static(ctypes.byref(desc), _ptr(x), _ptr(w_gate), _ptr(w_up), _ptr(w_down),
                                       _ptr(out), _stream_ptr(stream))
     if rc != MOC_OK:

@@ -12,6 +12,7 @@
 
 #include "decode_kernels.cuh"
 #include "gather_kernels.cuh"
+#include "grouped_select.cuh"
 #include "moc_common.cuh"
 #include "tc_gemm.cuh"
 #include "tc_plan.cuh"
@@ -121,7 +122,8 @@ int check_desc(const moc_ffn_desc *d) {
     if (d->tokens < 0 || d->d_model < 1 || d->d_ff < 1 || d->d_ff_ld < d->d_ff || d->k < 1 || d->k > d->d_ff)
         return MOC_ERR_INVALID_ARG;
     if (d->dtype != MOC_F32 && d->dtype != MOC_BF16) return MOC_ERR_UNSUPPORTED;
-    if (d->flags & ~MOC_FLAG_ACCUMULATE_WGRAD) return MOC_ERR_INVALID_ARG;
+    if (d->flags & ~(MOC_FLAG_ACCUMULATE_WGRAD | MOC_FLAG_SELECT_2_OF_8)) return MOC_ERR_INVALID_ARG;
+    if ((d->flags & MOC_FLAG_SELECT_2_OF_8) && (d->d_ff % 8 != 0 || d->k != d->d_ff / 4)) return MOC_ERR_INVALID_ARG;
     if (d->d_ff > 32768) return MOC_ERR_UNSUPPORTED;     // int16 channel indices
     if (d->d_model % 8 != 0) return MOC_ERR_UNSUPPORTED;  // 16-byte row vectors
     if ((double)d->tokens * (double)d->k >= 4294967296.0) return MOC_ERR_UNSUPPORTED;  // 32-bit pair ids
@@ -233,10 +235,17 @@ int forward_gather(const moc_ffn_desc &d, const T *x, const T *wg, const T *wu, 
         dim3 grid((F + 63) / 64, (unsigned)((n + 63) / 64));
         MOC_LAUNCH(KID_GATE_GEMM_ALU, st, (gemm_nt_alu_kernel<T><<<grid, 256, 0, st>>>(x + t0 * dm, wg, G, (int)n, F, dm, F)));
         if ((rc = launch_ok()) != MOC_OK) return rc;
-        const unsigned sel_grid = (unsigned)std::min<int64_t>(n, 148 * 32);
-        MOC_LAUNCH(KID_SELECT_ROWS, st,
-                   (select_rows_kernel<T><<<sel_grid, kSelectThreads, sel_smem, st>>>(
-                       G, n, F, F, K, idx + t0 * K, tg ? tg + t0 * K : nullptr)));
+        if (d.flags & MOC_FLAG_SELECT_2_OF_8) {
+            const unsigned grp_grid = (unsigned)std::min<int64_t>((n * (F / 8) + 255) / 256, 148 * 32);
+            MOC_LAUNCH(KID_SELECT_ROWS, st,
+                       (select_grouped_idx_kernel<T><<<grp_grid, 256, 0, st>>>(G, n, F, F, idx + t0 * K,
+                                                                                tg ? tg + t0 * K : nullptr)));
+        } else {
+            const unsigned sel_grid = (unsigned)std::min<int64_t>(n, 148 * 32);
+            MOC_LAUNCH(KID_SELECT_ROWS, st,
+                       (select_rows_kernel<T><<<sel_grid, kSelectThreads, sel_smem, st>>>(
+                           G, n, F, F, K, idx + t0 * K, tg ? tg + t0 * K : nullptr)));
+        }
         if ((rc = launch_ok()) != MOC_OK) return rc;
         MOC_LAUNCH(KID_FORWARD_TOKEN, st,
                    (forward_token_kernel<T><<<(unsigned)n, kTokenThreads, tok_smem, st>>>(
@@ -409,7 +418,12 @@ int forward_tc(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat1
         int16_t *o_idx = idx ? idx + t0 * K : nullptr;
         __nv_bfloat16 *o_g = idx ? tg + t0 * K : nullptr, *o_u = idx ? tu + t0 * K : nullptr;
         __nv_bfloat16 *Uc = U + t0 * L.ldf;
-        if (warp_select) {
+        if (d.flags & MOC_FLAG_SELECT_2_OF_8) {
+            // local mask: one thread per group of eight channels, no search
+            const unsigned grid = (unsigned)std::min<int64_t>((n * (F / 8) + 255) / 256, (int64_t)sm_count() * 64);
+            MOC_LAUNCH(KID_TC_SELECT_MASK, st,
+                       (select_grouped_mask_kernel<<<grid, 256, 0, st>>>(G, L.ldf, Uc, L.ldf, n, F, o_idx, o_g, o_u)));
+        } else if (warp_select) {
             const unsigned grid =
                 (unsigned)std::min<int64_t>((n + sel_wpc - 1) / sel_wpc, (int64_t)sm_count() * sel_ctas_per_sm);
 #define MOC_SELECT_LAUNCH(THREADS_PER_TOKEN, ...)                                                          \
@@ -632,6 +646,7 @@ int decode_bf16(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat
     int rc;
     const size_t sel_smem = ((size_t)F + 2 * dec::kSelListCap) * sizeof(uint32_t);
     if ((rc = set_smem(dec::select_mask_kernel, sel_smem)) != MOC_OK) return rc;
+    if ((rc = set_smem(dec::select_grouped_bits_kernel, sel_smem)) != MOC_OK) return rc;
     if ((rc = set_smem(dec::down_rows_kernel, dec::kDownSmem)) != MOC_OK) return rc;
     if ((rc = set_smem(dec::gemv_rows_kernel<false>, dec::kGemvSmem)) != MOC_OK) return rc;
     if ((rc = set_smem(dec::gemv_rows_kernel<true>, dec::kGemvSmem)) != MOC_OK) return rc;
@@ -640,9 +655,15 @@ int decode_bf16(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat
                launch_pdl(dec::gemv_rows_kernel<false>, dim3(L.gemv_grid), dec::kGemvThreads, dec::kGemvSmem, st, x, wg, T,
                           dm, F, ws, L.slices, status));
     if ((rc = launch_ok()) != MOC_OK) return rc;
-    MOC_LAUNCH(KID_DEC_SELECT, st,
-               launch_pdl(dec::select_mask_kernel, dim3(T), dec::kSelThreads, sel_smem, st, ws, F, K,
-                          ws.counters + L.slices));
+    if (d.flags & MOC_FLAG_SELECT_2_OF_8) {
+        MOC_LAUNCH(KID_DEC_SELECT, st,
+                   launch_pdl(dec::select_grouped_bits_kernel, dim3(T), dec::kSelThreads, sel_smem, st, ws, F,
+                              ws.counters + L.slices));
+    } else {
+        MOC_LAUNCH(KID_DEC_SELECT, st,
+                   launch_pdl(dec::select_mask_kernel, dim3(T), dec::kSelThreads, sel_smem, st, ws, F, K,
+                              ws.counters + L.slices));
+    }
     if ((rc = launch_ok()) != MOC_OK) return rc;
     MOC_LAUNCH(KID_DEC_UP, st,
                launch_pdl(dec::gemv_rows_kernel<true>, dim3(L.gemv_grid), dec::kGemvThreads, dec::kGemvSmem, st, x, wu, T,

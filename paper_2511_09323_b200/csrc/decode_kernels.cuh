@@ -263,6 +263,93 @@ __global__ void __launch_bounds__(kGemvThreads, 2) gemv_rows_kernel(const __nv_b
     }
 }
 
+// Last step of both select kernels: the last CTA to get here (one CTA per token) lists the used channels (ascending)
+// for the up and down kernels.  dyn: the CTA's dynamic shared memory (free by now, at least d_ff / 2 + 1 words).
+__device__ __forceinline__ void list_used_channels(const Workspace &ws, int F, int *arrivals, uint32_t *dyn) {
+    constexpr int NW = kSelThreads / 32;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    __shared__ int s_is_last, s_warp_cnt[NW];
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        s_is_last = atomicAdd(arrivals, 1) == (int)gridDim.x - 1;
+    }
+    __syncthreads();
+    if (!s_is_last) return;
+    __threadfence();
+    // union of the tokens' bitmaps, one word per thread (at most 1024 words), block-wide exclusive scan of the
+    // popcounts, then every thread writes the channels of its word
+    uint32_t word = 0;
+    if (tid < ws.sel_words) {
+        uint32_t part[16];  // at most 16 tokens: all loads in flight together
+#pragma unroll
+        for (int tt = 0; tt < 16; ++tt)
+            part[tt] = tt < (int)gridDim.x ? __ldcg(&ws.sel_bits[(int64_t)tt * ws.sel_words + tid]) : 0u;
+#pragma unroll
+        for (int tt = 0; tt < 16; ++tt) word |= part[tt];
+    }
+    const int v = __popc(word);
+    int inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int u = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += u;
+    }
+    if (lane == 31) s_warp_cnt[warp] = inc;
+    __syncthreads();
+    int wt = s_warp_cnt[lane], winc = wt;  // NW == 32: one warp total per lane
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int u = __shfl_up_sync(0xffffffffu, winc, o);
+        if (lane >= o) winc += u;
+    }
+    const int before_warp = __shfl_sync(0xffffffffu, winc - wt, warp), total = __shfl_sync(0xffffffffu, winc, 31);
+    // the list is put together in shared memory (the keys' memory, free by now) and leaves in whole words:
+    // consecutive 2-byte stores of one thread to global memory serialise on their sector
+    uint16_t *slist = reinterpret_cast<uint16_t *>(dyn);
+    __syncthreads();  // all threads are done with the keys
+    int pos = before_warp + inc - v;
+    while (word) {
+        const int bpos = __ffs(word) - 1;
+        word &= word - 1u;
+        slist[pos++] = (uint16_t)(tid * 32 + bpos);
+    }
+    __syncthreads();
+    for (int i = tid; i < (total + 1) / 2; i += kSelThreads)  // the list array holds F (rounded up to even) entries
+        reinterpret_cast<uint32_t *>(ws.list)[i] = reinterpret_cast<const uint32_t *>(slist)[i];
+    if (tid == 0) *ws.list_count = total;
+}
+
+// ---------------------------------------------------------------------------------------------- 2'. grouped select
+// MoC 2:8 (Section 4): the 2 largest of every 8 consecutive channels.  One CTA per token as above, but the mask is
+// local: the eight lanes that hold a group rank their keys against each other with shuffles, and the ballot of
+// "rank < 2" is a word of the token's selection bitmap.
+__global__ void __launch_bounds__(kSelThreads) select_grouped_bits_kernel(Workspace ws, int F, int *arrivals) {
+    extern __shared__ __align__(16) uint32_t dyn[];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    constexpr int NW = kSelThreads / 32;
+    const int t = blockIdx.x;
+    tc::pdl_launch_dependents();
+    tc::pdl_wait();
+    const float *g = ws.G + (int64_t)t * ws.ldf;
+    uint32_t *my_bits = ws.sel_bits + (int64_t)t * ws.sel_words;
+    const int nch = (F + kSelThreads - 1) / kSelThreads;
+    for (int c = 0; c < nch; ++c) {
+        const int j = c * kSelThreads + tid;  // d_ff is a multiple of 8: a group never straddles the end
+        const uint32_t key = j < F ? gate_key(g[j]) : 0u;
+        const int first = lane & ~7, me = lane & 7;
+        int before = 0;
+#pragma unroll
+        for (int f = 0; f < 8; ++f) {
+            const uint32_t o = __shfl_sync(0xffffffffu, key, first + f);
+            before += (o > key || (o == key && f < me)) ? 1 : 0;
+        }
+        const uint32_t b = __ballot_sync(0xffffffffu, j < F && before < 2);
+        if (lane == 0 && c * kSelThreads + warp * 32 < F) my_bits[c * NW + warp] = b;
+    }
+    list_used_channels(ws, F, arrivals, dyn);
+}
+
 // ---------------------------------------------------------------------------------------------- 2. select
 // One CTA per token: exact Top-K set of G[t, 0..F).
 //
@@ -449,57 +536,7 @@ __global__ void __launch_bounds__(kSelThreads) select_mask_kernel(Workspace ws, 
         block_ordered_emit<kSelThreads>(keys, F, tau, need, sm,
                                         [&](int, int j) { atomicOr(&my_bits[j >> 5], 1u << (j & 31)); });
     }
-    // ---- the last CTA to get here lists the used channels (ascending) for the up and down kernels
-    __shared__ int s_is_last, s_warp_cnt[NW];
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) {
-        s_is_last = atomicAdd(arrivals, 1) == (int)gridDim.x - 1;
-    }
-    __syncthreads();
-    if (!s_is_last) return;
-    __threadfence();
-    // union of the tokens' bitmaps, one word per thread (at most 1024 words), block-wide exclusive scan of the
-    // popcounts, then every thread writes the channels of its word
-    uint32_t word = 0;
-    if (tid < ws.sel_words) {
-        uint32_t part[16];  // at most 16 tokens: all loads in flight together
-#pragma unroll
-        for (int tt = 0; tt < 16; ++tt)
-            part[tt] = tt < (int)gridDim.x ? __ldcg(&ws.sel_bits[(int64_t)tt * ws.sel_words + tid]) : 0u;
-#pragma unroll
-        for (int tt = 0; tt < 16; ++tt) word |= part[tt];
-    }
-    const int v = __popc(word);
-    int inc = v;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const int u = __shfl_up_sync(0xffffffffu, inc, o);
-        if (lane >= o) inc += u;
-    }
-    if (lane == 31) s_warp_cnt[warp] = inc;
-    __syncthreads();
-    int wt = s_warp_cnt[lane], winc = wt;  // NW == 32: one warp total per lane
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const int u = __shfl_up_sync(0xffffffffu, winc, o);
-        if (lane >= o) winc += u;
-    }
-    const int before_warp = __shfl_sync(0xffffffffu, winc - wt, warp), total = __shfl_sync(0xffffffffu, winc, 31);
-    // the list is put together in shared memory (the keys' memory, free by now) and leaves in whole words:
-    // consecutive 2-byte stores of one thread to global memory serialise on their sector
-    uint16_t *slist = reinterpret_cast<uint16_t *>(dyn);
-    __syncthreads();  // all threads are done with the keys
-    int pos = before_warp + inc - v;
-    while (word) {
-        const int bpos = __ffs(word) - 1;
-        word &= word - 1u;
-        slist[pos++] = (uint16_t)(tid * 32 + bpos);
-    }
-    __syncthreads();
-    for (int i = tid; i < (total + 1) / 2; i += kSelThreads)  // the list array holds F (rounded up to even) entries
-        reinterpret_cast<uint32_t *>(ws.list)[i] = reinterpret_cast<const uint32_t *>(slist)[i];
-    if (tid == 0) *ws.list_count = total;
+    list_used_channels(ws, F, arrivals, dyn);
 }
 
 // ---------------------------------------------------------------------------------------------- 4. down

@@ -1,0 +1,102 @@
+"""MoC 2:8 (the grouped mask of Section 4: the 2 largest of every 8 consecutive channels) through the C ABI, against
+the oracle's grouped selection; everything after the mask is the operator the other GPU tests cover."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import moc_oracle as orc
+from oracle import parity
+from paper_2511_09323_b200 import binding as B
+from paper_2511_09323_b200 import build as moc_build
+from paper_2511_09323_b200 import synthetic as syn
+from paper_2511_09323_b200.autograd import MoCFFN
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    moc_build.build()
+    B.load()
+    yield
+    assert B.moc_last_device_status() == B.MOC_OK
+
+
+def _forward_backward(w: syn.Workload):
+    wg, wu, wd = syn.make_weights(w)
+    x, dD = syn.make_x(w), syn.make_grad_out(w)
+    xd, wgd, wud, wdd, dDd = (t.cuda() for t in (x, wg, wu, wd, dD))
+    out, idx, tg, tu = B.moc_ffn_forward(xd, wgd, wud, wdd, None, grouped=True)
+    grads = B.moc_ffn_backward(xd, wgd, wud, wdd, idx, tg, tu, dDd)
+    torch.cuda.synchronize()
+    assert B.moc_last_device_status() == B.MOC_OK
+    x64, wg64, wu64, wd64, dD64 = map(syn.to_f64, (x, wg, wu, wd, dD))
+    idx_np = idx.cpu().numpy()
+    assert idx_np.shape == (w.tokens, w.d_ff // 4)
+    parity.check_picks_grouped(idx_np, orc.gate_projection(x64, wg64))
+    ref = orc.forward_given_idx(x64, wg64, wu64, wd64, idx_np.astype(np.int32))
+    parity.assert_close(syn.to_f64(out), ref["out"], w.dtype, "out")
+    parity.assert_close(syn.to_f64(tg), ref["gval"], w.dtype, "topk_gate")
+    parity.assert_close(syn.to_f64(tu), ref["uval"], w.dtype, "topk_up")
+    gdev = {k: syn.to_f64(v) for k, v in grads.items()}
+    parity.check_backward(gdev, x64, wg64, wu64, wd64, idx_np, syn.to_f64(tg), syn.to_f64(tu), dD64, w.d_ff, w.dtype)
+    return (xd, wgd, wud, wdd), out
+
+
+@pytest.mark.parametrize("dtype,T,d,F", [
+    ("bf16", 300, 128, 1024),    # tensor-core plan
+    ("bf16", 5, 64, 256),        # tensor-core plan, a handful of tokens
+    ("f32", 40, 64, 256),        # gathered plan
+])
+def test_grouped_forward_backward(dtype, T, d, F):
+    _forward_backward(syn.Workload(f"g28-{dtype}-{T}", dtype, T, d, F, F, F // 4, seed=2800 + T))
+
+
+def test_grouped_ties_keep_the_lower_channels_exactly():
+    """Channels 8q+1, 8q+3 copy the gate rows of 8q, 8q+2: bit-identical gate values; the kept pair of a group is
+    then decided by the tie rule and must equal the oracle's choice on the device's own fp32 gate values."""
+    w = syn.Workload("g28-ties", "bf16", 300, 64, 512, 512, 128, seed=31)
+    wg, wu, wd = syn.make_weights(w)
+    wg[1::8], wg[3::8] = wg[0::8].clone(), wg[2::8].clone()
+    x = syn.make_x(w)
+    _, idx, tg, _ = B.moc_ffn_forward(x.cuda(), wg.cuda(), wu.cuda(), wd.cuda(), None, grouped=True)
+    idx = idx.cpu().numpy().astype(np.int64)
+    for t in range(w.tokens):
+        sel = set(idx[t].tolist())
+        for j in idx[t]:
+            if j % 8 in (1, 3):
+                assert j - 1 in sel, f"token {t}: channel {j} kept without its equal lower twin"
+
+
+@pytest.mark.parametrize("T", [1, 3, 16])
+def test_grouped_decode_matches_forward_and_oracle(T):
+    w = syn.Workload(f"g28-dec-{T}", "bf16", T, 512, 2048, 2048, 512, seed=77 + T)
+    wg, wu, wd = syn.make_weights(w)
+    x = syn.make_x(w)
+    xd, wgd, wud, wdd = (t.cuda() for t in (x, wg, wu, wd))
+    out = B.moc_ffn_decode(xd, wgd, wud, wdd, None, grouped=True)
+    out_s = torch.empty_like(xd)
+    B.moc_ffn_decode_static(xd, wgd, wud, wdd, None, out_s, grouped=True)
+    out_f, idx, _, _ = B.moc_ffn_forward(xd, wgd, wud, wdd, None, grouped=True)
+    torch.cuda.synchronize()
+    x64, wg64, wu64, wd64 = map(syn.to_f64, (x, wg, wu, wd))
+    idx_np = idx.cpu().numpy()
+    parity.check_picks_grouped(idx_np, orc.gate_projection(x64, wg64))
+    ref = orc.forward_given_idx(x64, wg64, wu64, wd64, idx_np.astype(np.int32))["out"]
+    for name, o in (("decode", out), ("decode_static", out_s), ("forward", out_f)):
+        parity.assert_close(syn.to_f64(o), ref, "bf16", name)
+
+
+def test_grouped_argument_rules_and_module():
+    x = torch.zeros(4, 64, dtype=torch.bfloat16, device="cuda")
+    wbad = torch.zeros(100, 64, dtype=torch.bfloat16, device="cuda")     # d_ff not a multiple of 8
+    with pytest.raises(ValueError):
+        B.moc_ffn_forward(x, wbad, wbad, wbad, None, grouped=True)
+    w = torch.zeros(128, 64, dtype=torch.bfloat16, device="cuda")
+    desc = B.make_desc(4, 64, 128, 16, torch.bfloat16, flags=B.MOC_FLAG_SELECT_2_OF_8)   # k must be d_ff / 4 = 32
+    assert B.moc_ffn_workspace_bytes(desc, B.MOC_OP_FORWARD) == 0
+    m = MoCFFN(64, 128, None, grouped=True)
+    assert m.k == 32
+    y = m(torch.randn(2, 7, 64, device="cuda", dtype=torch.bfloat16))
+    y.float().sum().backward()
+    assert m.w_down.grad is not None and torch.isfinite(m.w_down.grad.float()).all()
