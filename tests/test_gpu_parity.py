@@ -261,6 +261,21 @@ def test_decode_llama7b_shape(T):
     _check_decode(syn.to_f64(out), x64, wg64, wu64, wd64, w.k, "bf16", f"decode T={T}")
 
 
+def test_decode_with_padded_weight_arrays():
+    """d_ff = 1000 in arrays of 1024 rows whose tail holds junk: the padding rows must never be selected or read as
+    channels by the decode path (bf16 decode plan and the fp32 gathered plan)."""
+    for dtype, T in (("bf16", 3), ("bf16", 16), ("f32", 2)):
+        w = syn.Workload(f"dec-pad-{dtype}-{T}", dtype, T, 128, 1000, 1024, 125, seed=640 + T)
+        wg, wu, wd = syn.make_weights(w)
+        for m in (wg, wu, wd):
+            m[w.d_ff:] = 3.0      # junk, larger than any real gate value
+        x = syn.make_x(w)
+        out = B.moc_ffn_decode(_dev(x), _dev(wg), _dev(wu), _dev(wd), w.k, d_ff=w.d_ff)
+        torch.cuda.synchronize()
+        x64, wg64, wu64, wd64 = map(syn.to_f64, (x, wg[:w.d_ff], wu[:w.d_ff], wd[:w.d_ff]))
+        _check_decode(syn.to_f64(out), x64, wg64, wu64, wd64, w.k, dtype, f"padded decode {dtype} T={T}")
+
+
 @pytest.mark.parametrize("dtype,T,d,F,K", [("f32", 3, 64, 200, 25), ("bf16", 16, 256, 1000, 125), ("bf16", 7, 520, 777, 97)])
 def test_decode_small_shapes(dtype, T, d, F, K):
     w = syn.Workload("dec", dtype, T, d, F, F, K, seed=77, decode=True)
@@ -280,6 +295,8 @@ def test_decode_small_shapes(dtype, T, d, F, K):
     (513, 264, 1100, 1104, 137),   # d not a multiple of 64, F not a multiple of 256, ragged token tile
     (256, 128, 96, 96, 96),        # K = F: dense SwiGLU through the tensor-core plan
     (384, 512, 4500, 4504, 563),   # more than 4096 channels: few warps per SM in the warp-per-token selector
+    (257, 8, 64, 64, 1),           # smallest contraction, a single kept channel
+    (300, 64, 200, 200, 199),      # all but one channel kept
     (300, 128, 9000, 9000, 700),   # long rows: teams of four warps, two tokens in flight per SM
     (260, 64, 16000, 16000, 1200), # rows too long for separate gate and up buffers: both rows share one buffer
     (260, 64, 24000, 24000, 1500), # rows too long for any shared-memory slice: CTA-per-token selector
