@@ -297,6 +297,7 @@ def test_decode_small_shapes(dtype, T, d, F, K):
     (384, 512, 4500, 4504, 563),   # more than 4096 channels: few warps per SM in the warp-per-token selector
     (257, 8, 64, 64, 1),           # smallest contraction, a single kept channel
     (300, 64, 200, 200, 199),      # all but one channel kept
+    (270, 64, 2048, 2048, 1500),   # more kept channels than the search scratch can park: gate row freed late
     (300, 128, 9000, 9000, 700),   # long rows: teams of four warps, two tokens in flight per SM
     (260, 64, 16000, 16000, 1200), # rows too long for separate gate and up buffers: both rows share one buffer
     (260, 64, 24000, 24000, 1500), # rows too long for any shared-memory slice: CTA-per-token selector
