@@ -14,6 +14,7 @@
 #include "gather_kernels.cuh"
 #include "grouped_select.cuh"
 #include "moc_common.cuh"
+#include "small_batch.cuh"
 #include "tc_gemm.cuh"
 #include "tc_plan.cuh"
 #include "topk_select.cuh"
@@ -64,6 +65,9 @@ enum KernelId {
     KID_DEC_SELECT,
     KID_DEC_UP,
     KID_DEC_DOWN,
+    KID_SB_GATE_UP,
+    KID_SB_SELECT,
+    KID_SB_DOWN,
     KID_COUNT
 };
 static const char *const kKernelNames[KID_COUNT] = {
@@ -71,7 +75,8 @@ static const char *const kKernelNames[KID_COUNT] = {
     "csr_scan_blocks", "csr_scan_channels", "csr_fill",      "wgrad_rows",     "topk_select",
     "tc_gate_up_gemm", "tc_select_mask",  "tc_down_gemm",  "tc_bwd_sample",  "tc_dz_gemm",
     "tc_wgrad_gemm",   "tc_dx_gemm",      "tc_test_gemm",  "tc_select_hint", "dec_gate_gemv",
-    "dec_select",      "dec_up",          "dec_down",
+    "dec_select",      "dec_up",          "dec_down",      "sb_gate_up",     "sb_select",
+    "sb_down",
 };
 
 struct Profiler {
@@ -675,6 +680,109 @@ int decode_bf16(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat
     return launch_ok();
 }
 
+// ---- small-batch plan (bf16, 17..128 tokens): three weight-streaming tcgen05 kernels ----------------------
+struct SmallBatchLayout {
+    int ldf, ldz, m_tiles, splits, k_blocks_down;
+    size_t off_g, off_u, off_z, off_acc, off_cnt, total;
+};
+
+SmallBatchLayout small_batch_layout(const moc_ffn_desc &d) {
+    SmallBatchLayout L{};
+    L.ldf = (d.d_ff + 7) & ~7;
+    L.ldz = (d.d_ff + 7) & ~7;
+    L.m_tiles = (d.d_model + sb::kTile - 1) / sb::kTile;
+    L.k_blocks_down = (d.d_ff + sb::kBK - 1) / sb::kBK;
+    // about two CTAs per SM in the down kernel, every CTA at least one channel block
+    L.splits = std::max(1, std::min(2 * tc::sm_count() / L.m_tiles, L.k_blocks_down));
+    Carver c;
+    L.off_g = c.take((size_t)d.tokens * L.ldf * sizeof(float));
+    L.off_u = c.take((size_t)d.tokens * L.ldf * sizeof(float));
+    L.off_z = c.take((size_t)d.tokens * L.ldz * sizeof(__nv_bfloat16));
+    L.off_acc = c.take((size_t)d.tokens * d.d_model * sizeof(float));
+    L.off_cnt = c.take((size_t)L.m_tiles * sizeof(int));
+    L.total = c.off;
+    return L;
+}
+
+bool use_small_batch_plan(const moc_ffn_desc &d) {
+    return d.dtype == MOC_BF16 && d.tokens > 16 && d.tokens <= sb::kMaxTokens &&
+           ((size_t)d.d_ff + 2 * dec::kSelListCap) * sizeof(uint32_t) + 48 * 1024 <= (size_t)kMaxDynSmem;
+}
+
+int forward_small_batch(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat16 *wg,
+                        const __nv_bfloat16 *wu, const __nv_bfloat16 *wd, __nv_bfloat16 *out, int16_t *idx,
+                        __nv_bfloat16 *tg, __nv_bfloat16 *tu, char *wsp, cudaStream_t st) {
+    const SmallBatchLayout L = small_batch_layout(d);
+    const int T = (int)d.tokens, F = d.d_ff, dm = d.d_model;
+    int *status = device_status_ptr();
+    if (!status) return MOC_ERR_CUDA;
+    const sb::GemmShape shape = sb::gemm_shape(T);
+    float *G = reinterpret_cast<float *>(wsp + L.off_g), *U = reinterpret_cast<float *>(wsp + L.off_u);
+    __nv_bfloat16 *Z = reinterpret_cast<__nv_bfloat16 *>(wsp + L.off_z);
+    float *acc = reinterpret_cast<float *>(wsp + L.off_acc);
+    int *counters = reinterpret_cast<int *>(wsp + L.off_cnt);
+    int rc;
+    const size_t sel_smem = ((size_t)F + 2 * dec::kSelListCap) * sizeof(uint32_t);
+    if ((rc = set_smem(sb::sb_gate_up_kernel, shape.smem, 1024)) != MOC_OK) return rc;
+    if ((rc = set_smem(sb::sb_down_kernel, shape.smem, 1024)) != MOC_OK) return rc;
+    if ((rc = set_smem(sb::sb_select_kernel, sel_smem)) != MOC_OK) return rc;
+
+    sb::GateUpParams gp;
+    memset(&gp, 0, sizeof(gp));
+    if (!tc::make_map(&gp.w_map[0], wg, F, dm, dm, sb::kBK, sb::kTile) ||
+        !tc::make_map(&gp.w_map[1], wu, F, dm, dm, sb::kBK, sb::kTile) ||
+        !tc::make_map(&gp.x_map, x, T, dm, dm, sb::kBK, shape.tn))
+        return MOC_ERR_CUDA;
+    gp.T = T;
+    gp.tn = shape.tn;
+    gp.tmem_cols = shape.tmem_cols;
+    gp.stages = shape.stages;
+    gp.stage_bytes = shape.stage_bytes;
+    gp.F = F;
+    gp.k_blocks = (dm + sb::kBK - 1) / sb::kBK;
+    gp.tiles = (F + sb::kTile - 1) / sb::kTile;
+    gp.G = G;
+    gp.U = U;
+    gp.ldf = L.ldf;
+    gp.counters = counters;
+    gp.n_counters = L.m_tiles;
+    gp.status = status;
+    MOC_LAUNCH(KID_SB_GATE_UP, st,
+               launch_pdl(sb::sb_gate_up_kernel, dim3(2 * gp.tiles), sb::kThreads, shape.smem, st, gp));
+    if ((rc = launch_ok()) != MOC_OK) return rc;
+
+    sb::SelectParams sp{G, U, L.ldf, F, d.k, dm, Z, L.ldz, acc, idx, tg, tu};
+    if (d.flags & MOC_FLAG_SELECT_2_OF_8) {
+        MOC_LAUNCH(KID_SB_SELECT, st,
+                   launch_pdl(sb::sb_select_grouped_kernel, dim3(T), dec::kSelThreads, 0, st, sp));
+    } else {
+        MOC_LAUNCH(KID_SB_SELECT, st, launch_pdl(sb::sb_select_kernel, dim3(T), dec::kSelThreads, sel_smem, st, sp));
+    }
+    if ((rc = launch_ok()) != MOC_OK) return rc;
+
+    sb::DownParams dp;
+    memset(&dp, 0, sizeof(dp));
+    if (!tc::make_map(&dp.wd_map, wd, F, dm, dm, 64, sb::kBK) ||
+        !tc::make_map(&dp.z_map, Z, T, F, L.ldz, sb::kBK, shape.tn))
+        return MOC_ERR_CUDA;
+    dp.T = T;
+    dp.tn = shape.tn;
+    dp.tmem_cols = shape.tmem_cols;
+    dp.stages = shape.stages;
+    dp.stage_bytes = shape.stage_bytes;
+    dp.d = dm;
+    dp.k_blocks = L.k_blocks_down;
+    dp.m_tiles = L.m_tiles;
+    dp.splits = L.splits;
+    dp.acc = acc;
+    dp.out = out;
+    dp.counters = counters;
+    dp.status = status;
+    MOC_LAUNCH(KID_SB_DOWN, st,
+               launch_pdl(sb::sb_down_kernel, dim3(L.m_tiles * L.splits), sb::kThreads, shape.smem, st, dp));
+    return launch_ok();
+}
+
 }  // namespace
 }  // namespace moc
 
@@ -687,11 +795,13 @@ size_t moc_ffn_workspace_bytes(const moc_ffn_desc *desc, int op) {
     if (check_desc(desc) != MOC_OK) return 0;
     if (desc->tokens == 0) return 0;
     switch (op) {
-        case MOC_OP_FORWARD:
-            return use_tc_plan(*desc) ? tc::tc_forward_layout(*desc).total : plan_forward(*desc).total;
         case MOC_OP_DECODE:
-            if (desc->tokens > 16) return 0;
-            return use_decode_plan(*desc) ? decode_layout(*desc).total : plan_forward(*desc).total;
+            if (desc->tokens > sb::kMaxTokens) return 0;
+            if (use_decode_plan(*desc)) return decode_layout(*desc).total;
+            // fall through: the forward with nothing saved
+        case MOC_OP_FORWARD:
+            if (use_small_batch_plan(*desc)) return small_batch_layout(*desc).total;
+            return use_tc_plan(*desc) ? tc::tc_forward_layout(*desc).total : plan_forward(*desc).total;
         case MOC_OP_BACKWARD:
             return use_tc_plan(*desc) ? tc::tc_backward_layout(*desc).total : plan_backward(*desc).total;
         default:
@@ -723,6 +833,9 @@ int moc_ffn_forward(const moc_ffn_desc *desc, const void *x, const void *w_gate,
     char *ws = static_cast<char *>(workspace);
     if (desc->dtype == MOC_BF16) {
         using T = __nv_bfloat16;
+        if (use_small_batch_plan(*desc))
+            return forward_small_batch(*desc, (const T *)x, (const T *)w_gate, (const T *)w_up, (const T *)w_down,
+                                       (T *)out, topk_idx, (T *)topk_gate, (T *)topk_up, ws, st);
         if (use_tc_plan(*desc))
             return forward_tc(*desc, (const T *)x, (const T *)w_gate, (const T *)w_up, (const T *)w_down, (T *)out,
                               topk_idx, (T *)topk_gate, (T *)topk_up, ws, st);
@@ -784,8 +897,8 @@ int moc_ffn_decode(const moc_ffn_desc *desc, const void *x, const void *w_gate, 
                    const void *w_down, void *out, void *workspace, size_t workspace_bytes, void *cuda_stream) {
     int rc = check_desc(desc);
     if (rc != MOC_OK) return rc;
-    if (desc->tokens > 16) return MOC_ERR_UNSUPPORTED;
-    if (!use_decode_plan(*desc))  // fp32 storage: the gathered forward with nothing saved
+    if (desc->tokens > sb::kMaxTokens) return MOC_ERR_UNSUPPORTED;
+    if (!use_decode_plan(*desc))  // more than 16 tokens, or fp32 storage: the forward with nothing saved
         return moc_ffn_forward(desc, x, w_gate, w_up, w_down, out, nullptr, nullptr, nullptr, workspace,
                                workspace_bytes, cuda_stream);
     if (!good_ptr(x) || !good_ptr(w_gate) || !good_ptr(w_up) || !good_ptr(w_down) || !good_ptr(out))

@@ -371,20 +371,19 @@ struct SelectLevel {
     uint32_t count;   // number of candidates
 };
 
-__global__ void __launch_bounds__(kSelThreads) select_mask_kernel(Workspace ws, int F, int K, int *arrivals) {
-    static_assert(kSelThreads == 1024, "the listing step scans one count per lane");
-    extern __shared__ __align__(16) uint32_t dyn[];  // keys [F] | candidate lists 2 x [kSelListCap]
-    __shared__ SelectSmemT<kSelThreads / 32> sm;      // full radix select (fallback); its arrays double as scratch
+// The threshold search of one CTA (kSelThreads threads) over the row g[0..F): fills keys = dyn[0..F) and returns the
+// K-th largest key `tau`, how many keys equal to tau belong to the set (`need`), and whether some keys equal to
+// tau must be left out (`ties_cut`; false: the set is exactly "key >= tau").
+// dyn: keys [F] | candidate lists 2 x [kSelListCap]; sm: the full radix select's state (its arrays double as scratch).
+__device__ __forceinline__ void cta_select_threshold(const float *__restrict__ g, int F, int K, uint32_t *dyn,
+                                                     SelectSmemT<kSelThreads / 32> &sm, uint32_t &tau_out,
+                                                     int &need_out, bool &ties_cut_out) {
     __shared__ uint32_t s_min[32], s_max[32], s_pick, s_above, s_inbin, s_n;
     uint32_t *keys = dyn;
     uint32_t *lists[2] = {dyn + F, dyn + F + kSelListCap};
     uint32_t *hist = sm.priv;  // 2048 entries
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     constexpr int NW = kSelThreads / 32;
-    const int t = blockIdx.x;
-    tc::pdl_launch_dependents();
-    tc::pdl_wait();
-    const float *g = ws.G + (int64_t)t * ws.ldf;
 
     // ---- keys, minimum and maximum
     uint32_t kmin = 0xffffffffu, kmax = 0u;
@@ -520,6 +519,25 @@ __global__ void __launch_bounds__(kSelThreads) select_mask_kernel(Workspace ws, 
         block_radix_threshold<kSelThreads>(keys, F, K, sm, tau, need);
     else
         ties_cut = in_bin != (uint32_t)need;
+    tau_out = tau;
+    need_out = need;
+    ties_cut_out = ties_cut;
+}
+
+__global__ void __launch_bounds__(kSelThreads) select_mask_kernel(Workspace ws, int F, int K, int *arrivals) {
+    static_assert(kSelThreads == 1024, "the listing step scans one count per lane");
+    extern __shared__ __align__(16) uint32_t dyn[];  // keys [F] | candidate lists 2 x [kSelListCap]
+    __shared__ SelectSmemT<kSelThreads / 32> sm;
+    const uint32_t *keys = dyn;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    constexpr int NW = kSelThreads / 32;
+    const int t = blockIdx.x;
+    tc::pdl_launch_dependents();
+    tc::pdl_wait();
+    uint32_t tau;
+    int need;
+    bool ties_cut;
+    cta_select_threshold(ws.G + (int64_t)t * ws.ldf, F, K, dyn, sm, tau, need, ties_cut);
     uint32_t *my_bits = ws.sel_bits + (int64_t)t * ws.sel_words;
     const int nch = (F + kSelThreads - 1) / kSelThreads;
     if (!ties_cut) {

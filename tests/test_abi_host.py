@@ -95,7 +95,7 @@ def test_null_pointers_and_small_workspace_are_rejected_before_launch(lib):
                                None) == B.MOC_ERR_WORKSPACE
     assert lib.moc_ffn_backward(ctypes.byref(d), *([fake] * 12), None, 0, None) == B.MOC_ERR_WORKSPACE
     # decode batch limit
-    big = B.make_desc(17, 16, 32, 4, B.MOC_BF16)
+    big = B.make_desc(129, 16, 32, 4, B.MOC_BF16)
     assert lib.moc_ffn_decode(ctypes.byref(big), fake, fake, fake, fake, fake, None, 0, None) == B.MOC_ERR_UNSUPPORTED
     # zero tokens is a no-op that needs no buffers
     zero = B.make_desc(0, 16, 32, 4, B.MOC_BF16)

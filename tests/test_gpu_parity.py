@@ -149,7 +149,7 @@ def test_k_equals_dff_matches_dense_swiglu_formula():
 
 
 def test_inference_forward_saves_nothing_and_matches_training_forward():
-    w = syn.Workload("inf", "bf16", 50, 128, 256, 256, 32, seed=9)
+    w = syn.Workload("inf", "bf16", 200, 128, 256, 256, 32, seed=9)
     x, wg, wu, wd, _ = map(_dev, _problem(w))
     out_a, *_ = B.moc_ffn_forward(x, wg, wu, wd, w.k, save=True)
     out_b, idx, tg, tu = B.moc_ffn_forward(x, wg, wu, wd, w.k, save=False)
@@ -215,7 +215,7 @@ def test_host_errors_raise_before_launch():
         B.moc_ffn_forward(x, wg, wu, wd, 8, workspace=torch.empty(16, dtype=torch.uint8, device="cuda"))
     assert e.value.status == B.MOC_ERR_WORKSPACE
     with pytest.raises(B.MocError) as e:
-        B.moc_ffn_decode(_dev(syn.make_x(w, tokens=17)), wg, wu, wd, 8)
+        B.moc_ffn_decode(_dev(syn.make_x(w, tokens=129)), wg, wu, wd, 8)
     assert e.value.status == B.MOC_ERR_UNSUPPORTED
     assert B.moc_last_device_status() == B.MOC_OK
 
