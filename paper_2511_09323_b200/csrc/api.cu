@@ -649,7 +649,7 @@ int decode_bf16(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat
     ws.counters = reinterpret_cast<int *>(wsp + L.off_cnt);
     ws.ldf = L.ldf;
     int rc;
-    const size_t sel_smem = ((size_t)F + 2 * dec::kSelListCap) * sizeof(uint32_t);
+    const size_t sel_smem = ((size_t)((F + 3) & ~3) + 2 * dec::kSelListCap) * sizeof(uint32_t);
     if ((rc = set_smem(dec::select_mask_kernel, sel_smem)) != MOC_OK) return rc;
     if ((rc = set_smem(dec::select_grouped_bits_kernel, sel_smem)) != MOC_OK) return rc;
     if ((rc = set_smem(dec::down_rows_kernel, dec::kDownSmem)) != MOC_OK) return rc;
@@ -667,7 +667,7 @@ int decode_bf16(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat
     } else {
         MOC_LAUNCH(KID_DEC_SELECT, st,
                    launch_pdl(dec::select_mask_kernel, dim3(T), dec::kSelThreads, sel_smem, st, ws, F, K,
-                              ws.counters + L.slices));
+                              ws.counters + L.slices, status));
     }
     if ((rc = launch_ok()) != MOC_OK) return rc;
     MOC_LAUNCH(KID_DEC_UP, st,
@@ -682,18 +682,36 @@ int decode_bf16(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat
 
 // ---- small-batch plan (bf16, 17..128 tokens): three weight-streaming tcgen05 kernels ----------------------
 struct SmallBatchLayout {
-    int ldf, ldz, m_tiles, splits, k_blocks_down;
+    int ldf, ldz;
+    int rows, ctas_per_matrix;                   // gate + up: channels per CTA, CTAs per weight matrix
+    int accs, m_tiles, splits, k_blocks_down;    // down: 128 * accs columns per CTA, CTAs = m_tiles * splits
+    bool stage_u;                                // the selector holds the token's up row in shared memory
     size_t off_g, off_u, off_z, off_acc, off_cnt, total;
 };
 
 SmallBatchLayout small_batch_layout(const moc_ffn_desc &d) {
     SmallBatchLayout L{};
+    const int sms = tc::sm_count();
     L.ldf = (d.d_ff + 7) & ~7;
     L.ldz = (d.d_ff + 7) & ~7;
-    L.m_tiles = (d.d_model + sb::kTile - 1) / sb::kTile;
+    // gate + up: one CTA per SM, half of them per matrix
+    const int per = std::max(1, sms / 2);
+    L.rows = std::min(sb::kMaxRows, std::max(8, (((d.d_ff + per - 1) / per) + 7) & ~7));
+    L.ctas_per_matrix = (d.d_ff + L.rows - 1) / L.rows;
+    // down: about one CTA per SM, every CTA at least one channel block; wide column blocks when they still fill the GPU
     L.k_blocks_down = (d.d_ff + sb::kBK - 1) / sb::kBK;
-    // about two CTAs per SM in the down kernel, every CTA at least one channel block
-    L.splits = std::max(1, std::min(2 * tc::sm_count() / L.m_tiles, L.k_blocks_down));
+    auto ctas = [&](int accs, int &m_tiles, int &splits) {
+        m_tiles = (d.d_model + sb::kTile * accs - 1) / (sb::kTile * accs);
+        splits = std::max(1, std::min(sms / m_tiles, L.k_blocks_down));
+        return m_tiles * splits;
+    };
+    int m1, s1, m2, s2;
+    const int c1 = ctas(1, m1, s1), c2 = ctas(2, m2, s2);
+    const bool wide = d.d_model > sb::kTile && (c2 >= c1 || 20 * c2 >= 17 * sms);
+    L.accs = wide ? 2 : 1;
+    L.m_tiles = wide ? m2 : m1;
+    L.splits = wide ? s2 : s1;
+    L.stage_u = sb::select_smem(d.d_ff, true) + 48 * 1024 <= (size_t)kMaxDynSmem;
     Carver c;
     L.off_g = c.take((size_t)d.tokens * L.ldf * sizeof(float));
     L.off_u = c.take((size_t)d.tokens * L.ldf * sizeof(float));
@@ -706,7 +724,7 @@ SmallBatchLayout small_batch_layout(const moc_ffn_desc &d) {
 
 bool use_small_batch_plan(const moc_ffn_desc &d) {
     return d.dtype == MOC_BF16 && d.tokens > 16 && d.tokens <= sb::kMaxTokens &&
-           ((size_t)d.d_ff + 2 * dec::kSelListCap) * sizeof(uint32_t) + 48 * 1024 <= (size_t)kMaxDynSmem;
+           sb::select_smem(d.d_ff, false) + 48 * 1024 <= (size_t)kMaxDynSmem;
 }
 
 int forward_small_batch(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat16 *wg,
@@ -716,31 +734,34 @@ int forward_small_batch(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __n
     const int T = (int)d.tokens, F = d.d_ff, dm = d.d_model;
     int *status = device_status_ptr();
     if (!status) return MOC_ERR_CUDA;
-    const sb::GemmShape shape = sb::gemm_shape(T);
+    const sb::GemmShape gs = sb::gemm_shape(T, L.rows), ds = sb::gemm_shape(T, sb::kTile * L.accs);
+    if (gs.stages < 2 || ds.stages < 2) return MOC_ERR_UNSUPPORTED;
     float *G = reinterpret_cast<float *>(wsp + L.off_g), *U = reinterpret_cast<float *>(wsp + L.off_u);
     __nv_bfloat16 *Z = reinterpret_cast<__nv_bfloat16 *>(wsp + L.off_z);
     float *acc = reinterpret_cast<float *>(wsp + L.off_acc);
     int *counters = reinterpret_cast<int *>(wsp + L.off_cnt);
     int rc;
-    const size_t sel_smem = ((size_t)F + 2 * dec::kSelListCap) * sizeof(uint32_t);
-    if ((rc = set_smem(sb::sb_gate_up_kernel, shape.smem, 1024)) != MOC_OK) return rc;
-    if ((rc = set_smem(sb::sb_down_kernel, shape.smem, 1024)) != MOC_OK) return rc;
+    const size_t sel_smem = sb::select_smem(F, L.stage_u);
+    if ((rc = set_smem(sb::sb_gate_up_kernel, gs.smem, 1024)) != MOC_OK) return rc;
+    if ((rc = set_smem(sb::sb_down_kernel, ds.smem, 1024)) != MOC_OK) return rc;
     if ((rc = set_smem(sb::sb_select_kernel, sel_smem)) != MOC_OK) return rc;
 
     sb::GateUpParams gp;
     memset(&gp, 0, sizeof(gp));
-    if (!tc::make_map(&gp.w_map[0], wg, F, dm, dm, sb::kBK, sb::kTile) ||
-        !tc::make_map(&gp.w_map[1], wu, F, dm, dm, sb::kBK, sb::kTile) ||
-        !tc::make_map(&gp.x_map, x, T, dm, dm, sb::kBK, shape.tn))
+    if (!tc::make_map(&gp.w_map[0], wg, F, dm, dm, sb::kBK, L.rows) ||
+        !tc::make_map(&gp.w_map[1], wu, F, dm, dm, sb::kBK, L.rows) ||
+        !tc::make_map(&gp.x_map, x, T, dm, dm, sb::kBK, gs.tn))
         return MOC_ERR_CUDA;
     gp.T = T;
-    gp.tn = shape.tn;
-    gp.tmem_cols = shape.tmem_cols;
-    gp.stages = shape.stages;
-    gp.stage_bytes = shape.stage_bytes;
+    gp.tn = gs.tn;
+    gp.tmem_cols = gs.tmem_cols;
+    gp.stages = gs.stages;
+    gp.w_bytes = gs.w_bytes;
+    gp.stage_bytes = gs.stage_bytes;
     gp.F = F;
     gp.k_blocks = (dm + sb::kBK - 1) / sb::kBK;
-    gp.tiles = (F + sb::kTile - 1) / sb::kTile;
+    gp.rows = L.rows;
+    gp.ctas_per_matrix = L.ctas_per_matrix;
     gp.G = G;
     gp.U = U;
     gp.ldf = L.ldf;
@@ -748,10 +769,19 @@ int forward_small_batch(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __n
     gp.n_counters = L.m_tiles;
     gp.status = status;
     MOC_LAUNCH(KID_SB_GATE_UP, st,
-               launch_pdl(sb::sb_gate_up_kernel, dim3(2 * gp.tiles), sb::kThreads, shape.smem, st, gp));
+               launch_pdl(sb::sb_gate_up_kernel, dim3(2 * L.ctas_per_matrix), sb::kThreads, gs.smem, st, gp));
     if ((rc = launch_ok()) != MOC_OK) return rc;
 
-    sb::SelectParams sp{G, U, L.ldf, F, d.k, dm, Z, L.ldz, acc, idx, tg, tu};
+    // W_down fits into L2 next to the workspace on this part when it is below ~100 MB; it is asked for while the
+    // selection runs.  MOC_FFN_SB_PREFETCH=0 in the environment turns that off (for measurements).
+    static const bool prefetch_on = [] {
+        const char *e = getenv("MOC_FFN_SB_PREFETCH");
+        return !(e && e[0] == '0');
+    }();
+    const uint64_t wd_bytes = (uint64_t)F * dm * sizeof(__nv_bfloat16);
+    const bool prefetch = prefetch_on && wd_bytes <= ((uint64_t)100 << 20);
+    sb::SelectParams sp{G,  U,  L.ldf, F, d.k, dm, Z, L.ldz, acc, idx, tg, tu, L.stage_u ? 1 : 0, status,
+                        prefetch ? reinterpret_cast<const uint8_t *>(wd) : nullptr, wd_bytes};
     if (d.flags & MOC_FLAG_SELECT_2_OF_8) {
         MOC_LAUNCH(KID_SB_SELECT, st,
                    launch_pdl(sb::sb_select_grouped_kernel, dim3(T), dec::kSelThreads, 0, st, sp));
@@ -763,23 +793,25 @@ int forward_small_batch(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __n
     sb::DownParams dp;
     memset(&dp, 0, sizeof(dp));
     if (!tc::make_map(&dp.wd_map, wd, F, dm, dm, 64, sb::kBK) ||
-        !tc::make_map(&dp.z_map, Z, T, F, L.ldz, sb::kBK, shape.tn))
+        !tc::make_map(&dp.z_map, Z, T, F, L.ldz, sb::kBK, ds.tn))
         return MOC_ERR_CUDA;
     dp.T = T;
-    dp.tn = shape.tn;
-    dp.tmem_cols = shape.tmem_cols;
-    dp.stages = shape.stages;
-    dp.stage_bytes = shape.stage_bytes;
+    dp.tn = ds.tn;
+    dp.tmem_cols = ds.tmem_cols;
+    dp.stages = ds.stages;
+    dp.w_bytes = ds.w_bytes;
+    dp.stage_bytes = ds.stage_bytes;
     dp.d = dm;
     dp.k_blocks = L.k_blocks_down;
     dp.m_tiles = L.m_tiles;
     dp.splits = L.splits;
+    dp.accs = L.accs;
     dp.acc = acc;
     dp.out = out;
     dp.counters = counters;
     dp.status = status;
     MOC_LAUNCH(KID_SB_DOWN, st,
-               launch_pdl(sb::sb_down_kernel, dim3(L.m_tiles * L.splits), sb::kThreads, shape.smem, st, dp));
+               launch_pdl(sb::sb_down_kernel, dim3(L.m_tiles * L.splits), sb::kThreads, ds.smem, st, dp));
     return launch_ok();
 }
 
@@ -1083,5 +1115,8 @@ const char *moc_status_string(int status) {
 
 }  // extern "C"
 
-
-
+#ifdef MOC_SB_TIMELINE
+extern "C" __attribute__((visibility("default"))) int moc_debug_sb_read(void *host) {
+    return cudaMemcpyFromSymbol(host, moc::sb::g_tl, sizeof(moc::sb::g_tl)) == cudaSuccess ? 0 : -1;
+}
+#endif

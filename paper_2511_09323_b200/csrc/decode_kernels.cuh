@@ -371,16 +371,43 @@ struct SelectLevel {
     uint32_t count;   // number of candidates
 };
 
-// The threshold search of one CTA (kSelThreads threads) over the row g[0..F): fills keys = dyn[0..F) and returns the
+// One bulk copy of `bytes` (a multiple of 16) from global `src` to shared `dst` (both 16-byte aligned), or two when
+// src2 is given (begin), and a bounded wait for them (wait).  Every thread of the CTA calls both; the result is the
+// same for all (false: the wait ran out and MOC_ERR_TIMEOUT was raised).  `bar` / `abort_flag`: shared scratch.
+__device__ __forceinline__ void cta_stage_rows_begin(uint64_t *bar, int *abort_flag, void *dst, const void *src,
+                                                     uint32_t bytes, void *dst2 = nullptr,
+                                                     const void *src2 = nullptr) {
+    const uint32_t b = tc::smem_u32(bar);
+    if (threadIdx.x == 0) {
+        tc::mbar_init(b, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        tc::mbar_expect_tx(b, src2 ? 2 * bytes : bytes);
+        tc::bulk_copy_g2s(tc::smem_u32(dst), src, bytes, b);
+        if (src2) tc::bulk_copy_g2s(tc::smem_u32(dst2), src2, bytes, b);
+    }
+    __syncthreads();  // the barrier is initialised before anyone polls it
+}
+__device__ __forceinline__ bool cta_stage_rows_wait(uint64_t *bar, int *abort_flag, int *status) {
+    const bool ok = tc::mbar_wait(tc::smem_u32(bar), 0u, abort_flag, status);
+    return __syncthreads_or(ok ? 0 : 1) == 0;
+}
+__device__ __forceinline__ bool cta_stage_rows(uint64_t *bar, int *abort_flag, int *status, void *dst, const void *src,
+                                               uint32_t bytes) {
+    cta_stage_rows_begin(bar, abort_flag, dst, src, bytes);
+    return cta_stage_rows_wait(bar, abort_flag, status);
+}
+
+// The threshold search of one CTA (kSelThreads threads) over the row g[0..F): fills keys[0..F) and returns the
 // K-th largest key `tau`, how many keys equal to tau belong to the set (`need`), and whether some keys equal to
 // tau must be left out (`ties_cut`; false: the set is exactly "key >= tau").
-// dyn: keys [F] | candidate lists 2 x [kSelListCap]; sm: the full radix select's state (its arrays double as scratch).
-__device__ __forceinline__ void cta_select_threshold(const float *__restrict__ g, int F, int K, uint32_t *dyn,
-                                                     SelectSmemT<kSelThreads / 32> &sm, uint32_t &tau_out,
-                                                     int &need_out, bool &ties_cut_out) {
+// g == nullptr: keys[] already holds the row's fp32 values (staged by a bulk copy) and is converted in place.
+// lists0: two candidate lists of kSelListCap entries; sm: the full radix select's state (its arrays double as scratch).
+__device__ __forceinline__ void cta_select_threshold(const float *__restrict__ g, int F, int K, uint32_t *keys,
+                                                     uint32_t *lists0, SelectSmemT<kSelThreads / 32> &sm,
+                                                     uint32_t &tau_out, int &need_out, bool &ties_cut_out) {
     __shared__ uint32_t s_min[32], s_max[32], s_pick, s_above, s_inbin, s_n;
-    uint32_t *keys = dyn;
-    uint32_t *lists[2] = {dyn + F, dyn + F + kSelListCap};
+    uint32_t *lists[2] = {lists0, lists0 + kSelListCap};
     uint32_t *hist = sm.priv;  // 2048 entries
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     constexpr int NW = kSelThreads / 32;
@@ -388,7 +415,7 @@ __device__ __forceinline__ void cta_select_threshold(const float *__restrict__ g
     // ---- keys, minimum and maximum
     uint32_t kmin = 0xffffffffu, kmax = 0u;
     for (int j = tid; j < F; j += kSelThreads) {
-        const uint32_t key = gate_key(g[j]);
+        const uint32_t key = gate_key(g ? g[j] : __uint_as_float(keys[j]));
         keys[j] = key;
         kmin = min(kmin, key);
         kmax = max(kmax, key);
@@ -524,20 +551,26 @@ __device__ __forceinline__ void cta_select_threshold(const float *__restrict__ g
     ties_cut_out = ties_cut;
 }
 
-__global__ void __launch_bounds__(kSelThreads) select_mask_kernel(Workspace ws, int F, int K, int *arrivals) {
+__global__ void __launch_bounds__(kSelThreads) select_mask_kernel(Workspace ws, int F, int K, int *arrivals,
+                                                                  int *__restrict__ status) {
     static_assert(kSelThreads == 1024, "the listing step scans one count per lane");
-    extern __shared__ __align__(16) uint32_t dyn[];  // keys [F] | candidate lists 2 x [kSelListCap]
+    extern __shared__ __align__(16) uint32_t dyn[];  // keys [F rounded up to 4] | candidate lists 2 x [kSelListCap]
     __shared__ SelectSmemT<kSelThreads / 32> sm;
+    __shared__ uint64_t s_bar;
+    __shared__ int s_abort;
     const uint32_t *keys = dyn;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     constexpr int NW = kSelThreads / 32;
     const int t = blockIdx.x;
+    const int Fp = (F + 3) & ~3;
     tc::pdl_launch_dependents();
     tc::pdl_wait();
+    // the token's gate row arrives with one bulk copy instead of a chain of dependent loads
+    if (!cta_stage_rows(&s_bar, &s_abort, status, dyn, ws.G + (int64_t)t * ws.ldf, (uint32_t)Fp * 4u)) return;
     uint32_t tau;
     int need;
     bool ties_cut;
-    cta_select_threshold(ws.G + (int64_t)t * ws.ldf, F, K, dyn, sm, tau, need, ties_cut);
+    cta_select_threshold(nullptr, F, K, dyn, dyn + Fp, sm, tau, need, ties_cut);
     uint32_t *my_bits = ws.sel_bits + (int64_t)t * ws.sel_words;
     const int nch = (F + kSelThreads - 1) / kSelThreads;
     if (!ties_cut) {

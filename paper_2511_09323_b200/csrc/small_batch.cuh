@@ -3,21 +3,22 @@
 // With a few dozen tokens the union of the tokens' Top-K sets covers nearly every channel
 // (1 - (1 - K/F)^T), so the row gathers of the decode plan (Section 5) no longer save bytes: the whole
 // of W_gate, W_up and W_down is read once, and the job is to keep HBM busy.  The token count is far
-// below a 128-row MMA tile, so the operands are swapped: the WEIGHTS are the M side of the MMA
-// (128 channels, or 128 output columns, per CTA) and the tokens are its N side (T rounded up to 32).
+// below a 128-row MMA tile, so the operands are swapped: the WEIGHTS are the M side of the MMA and the
+// tokens are its N side (T rounded up to 32).
 //
 //   1. sb_gate_up_kernel   G^T | U^T [channel, token] = [Wg ; Wu] x^T          (Eq. (Moc-1) and U = X W_up)
-//                          one CTA per (matrix, 128 channels); fp32 G and U [T, ldf] in the workspace
+//                          every CTA owns `rows` consecutive channels of one matrix, rows chosen so that the
+//                          grid is one CTA per SM; fp32 G and U [T, ldf] go to the workspace
 //   2. sb_select_kernel    per token: exact Top-K of G (or 2 of every 8), Z' = SiLU(G) . M . U  (mask, Eq. (MoC-2))
 //                          as a dense bf16 row; optionally the compact saved triple; zeroes the output accumulator
-//   3. sb_down_kernel      D^T [column, token] = Wd^T Z'^T, the channels split over several CTAs per 128 columns;
-//                          partial sums meet in an fp32 accumulator (vector-free red.add), the last CTA of a
+//   3. sb_down_kernel      D^T [column, token] = Wd^T Z'^T; a CTA owns 128 or 256 output columns and a share of
+//                          the channels; partial sums meet in an fp32 accumulator (16-byte red.add), the last CTA of a
 //                          column block rounds to bf16
 //
-// Every CTA owns one tile and two CTAs share an SM, so that all tiles are resident at once and the
-// bytes in flight, not a tile schedule, set the pace.  The kernels are chained with programmatic
-// dependent launch: weights stream before the dependency wait, activations and the workspace are
-// touched after it.  Waits are bounded as everywhere else in the library.
+// One CTA per SM with the deepest ring of stages shared memory allows: the bytes in flight set the pace.
+// The kernels are chained with programmatic dependent launch: weights stream before the dependency
+// wait, activations and the workspace are touched after it.  Waits are bounded as everywhere else in
+// the library.
 #pragma once
 
 #include "decode_kernels.cuh"
@@ -28,41 +29,60 @@
 namespace moc {
 namespace sb {
 
-constexpr int kTile = 128;      // MMA M: weight rows (channels / output columns) per CTA
+#ifdef MOC_SB_TIMELINE
+__device__ unsigned long long g_tl[4][512][8];
+__device__ __forceinline__ void tl_stamp(int k, int slot) {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    if (blockIdx.x < 512) g_tl[k][blockIdx.x][slot] = t;
+}
+#define SB_TL(k, slot) tl_stamp(k, slot)
+#else
+#define SB_TL(k, slot)
+#endif
+
+constexpr int kTile = 128;      // MMA M
 constexpr int kBK = 64;         // contraction elements per stage: one 128-byte swizzle row
-constexpr int kThreads = 192;   // warp 0 TMA, warp 1 MMA + TMEM, warps 2..5 epilogue
-constexpr int kMaxStages = 8;
+constexpr int kThreads = 320;   // warp 0 TMA, warp 1 MMA + TMEM, warps 2..9 epilogue (two per TMEM lane quarter)
+constexpr int kEpiThreads = kThreads - 64;
+constexpr int kMaxStages = 10;
 constexpr int kMaxTokens = 128;
-constexpr uint32_t kWeightStageBytes = kTile * kBK * 2;  // 16 KiB
+constexpr int kMaxRows = 256;   // weight rows per CTA: two MMA tiles
 constexpr uint32_t kBarRegion = 256;
-constexpr size_t kSmemBudget = 108 * 1024;  // per CTA, two CTAs per SM
+constexpr size_t kSmemBudget = 224 * 1024;
+constexpr size_t kSmemSlack = 1024 /*alignment*/ + kTile * kBK * 2 /*an MMA over a short tile reads 128 rows*/;
 
 struct GemmShape {
-    int tn;        // tokens rounded up to a multiple of 32 (MMA N, rows of the activation box)
-    int tmem_cols; // power of two >= tn
+    int tn;            // tokens rounded up to a multiple of 32 (MMA N, rows of the activation box)
+    int tmem_cols;     // power of two >= accumulators * tn
     int stages;
+    uint32_t w_bytes;  // weight bytes per stage
     uint32_t stage_bytes;
     size_t smem;
 };
 
-inline GemmShape gemm_shape(int tokens) {
+// weight_rows: rows (gate/up: channels; down: output columns) per CTA, at most kMaxRows
+inline GemmShape gemm_shape(int tokens, int weight_rows) {
     GemmShape s{};
     s.tn = (tokens + 31) & ~31;
-    s.tmem_cols = s.tn <= 32 ? 32 : s.tn <= 64 ? 64 : 128;
-    s.stage_bytes = kWeightStageBytes + (uint32_t)s.tn * kBK * 2;
-    const size_t room = kSmemBudget - 1024 - kBarRegion;
+    const int cols = s.tn * (weight_rows > kTile ? 2 : 1);
+    s.tmem_cols = cols <= 32 ? 32 : cols <= 64 ? 64 : cols <= 128 ? 128 : 256;
+    s.w_bytes = (uint32_t)weight_rows * kBK * 2;
+    s.stage_bytes = s.w_bytes + (uint32_t)s.tn * kBK * 2;
+    const size_t room = kSmemBudget - kSmemSlack - kBarRegion;
     s.stages = (int)std::min<size_t>(kMaxStages, room / s.stage_bytes);
-    s.smem = 1024 + (size_t)s.stages * s.stage_bytes + kBarRegion;
+    s.smem = kSmemSlack + (size_t)s.stages * s.stage_bytes + kBarRegion;
     return s;
 }
 
 struct GateUpParams {
-    CUtensorMap w_map[2];  // W_gate, W_up: [F, d] rows of d contiguous elements, boxes of 128 rows x 64
+    CUtensorMap w_map[2];  // W_gate, W_up: [F, d] rows of d contiguous elements, boxes of `rows` rows x 64
     CUtensorMap x_map;     // x [T, d], boxes of tn rows x 64 (rows >= T read as zero)
     int T, tn, tmem_cols, stages;
-    uint32_t stage_bytes;
-    int F, k_blocks, tiles;  // tiles = ceil(F / 128) per matrix
-    float *G, *U;            // [T, ldf]
+    uint32_t w_bytes, stage_bytes;
+    int F, k_blocks;
+    int rows, ctas_per_matrix;  // channels per CTA (multiple of 8, <= 256); grid = 2 * ctas_per_matrix
+    float *G, *U;               // [T, ldf]
     int ldf;
     int *counters, n_counters;  // zeroed here for the down kernel
     int *status;
@@ -72,8 +92,9 @@ struct DownParams {
     CUtensorMap wd_map;  // W_down [F, d] read as the M-major operand: boxes of 64 channels x 64 columns
     CUtensorMap z_map;   // Z' [T, F], boxes of tn rows x 64 channels
     int T, tn, tmem_cols, stages;
-    uint32_t stage_bytes;
+    uint32_t w_bytes, stage_bytes;
     int d, k_blocks, m_tiles, splits;
+    int accs;            // 1 or 2: the CTA owns 128 * accs output columns
     float *acc;          // [T, d] fp32, zero on entry
     __nv_bfloat16 *out;  // [T, d]
     int *counters;       // [m_tiles], zero on entry, left zero
@@ -93,21 +114,30 @@ struct Ring {
     __device__ __forceinline__ uint32_t full(int s) const { return bar_base + 8u * s; }
     __device__ __forceinline__ uint32_t empty(int s) const { return bar_base + 8u * (kMaxStages + s); }
     __device__ __forceinline__ uint32_t tfull() const { return bar_base + 8u * (2 * kMaxStages); }
+    __device__ __forceinline__ uint32_t extra() const { return bar_base + 8u * (2 * kMaxStages + 2); }  // after the TMEM address and the abort flag
 };
 
 // ---------------------------------------------------------------------------------------------- 1. gate + up
-__global__ void __launch_bounds__(kThreads, 2) sb_gate_up_kernel(const __grid_constant__ GateUpParams p) {
+// A CTA's `rows` channels are covered by one MMA tile (rows <= 128; the rows of the tile beyond `rows` are whatever
+// follows in shared memory and land in accumulator lanes nobody reads) or by two overlapping ones: tile 0 = rows
+// 0..127, tile 1 = rows (rows - 128)..(rows - 1), of which only the last rows - 128 lanes are new.
+__global__ void __launch_bounds__(kThreads, 1) sb_gate_up_kernel(const __grid_constant__ GateUpParams p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = tc::smem_u32(smem_raw);
     Ring ring;
     ring.base = (raw + 1023u) & ~1023u;
     ring.stage_bytes = p.stage_bytes;
-    ring.bar_base = ring.base + (uint32_t)p.stages * p.stage_bytes;
+    ring.bar_base = ring.base + (uint32_t)p.stages * p.stage_bytes + kTile * kBK * 2;
     uint8_t *bar_ptr = smem_raw + (ring.bar_base - raw);
     volatile uint32_t *tmem_holder = reinterpret_cast<volatile uint32_t *>(bar_ptr + 8 * (2 * kMaxStages + 1));
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_holder + 1);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     tc::pdl_launch_dependents();
+    if (threadIdx.x == 0) SB_TL(0, 0);
+
+    const int prob = (int)blockIdx.x / p.ctas_per_matrix;
+    const int ch0 = ((int)blockIdx.x - prob * p.ctas_per_matrix) * p.rows;
+    const int ahead = min(p.stages, p.k_blocks);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
@@ -118,6 +148,12 @@ __global__ void __launch_bounds__(kThreads, 2) sb_gate_up_kernel(const __grid_co
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        // the weights depend on nothing earlier in the stream: the first stages' weight boxes leave at once,
+        // their activation boxes after the dependency wait
+        for (int kb = 0; kb < ahead; ++kb) {
+            tc::mbar_expect_tx(ring.full(kb), p.stage_bytes);
+            tc::tma_load_2d(ring.stage(kb), &p.w_map[prob], ring.full(kb), kb * kBK, ch0);
+        }
     }
     if (warp == 1) {
         tc::tmem_alloc(tc::smem_u32(const_cast<uint32_t *>(tmem_holder)), (uint32_t)p.tmem_cols);
@@ -127,31 +163,22 @@ __global__ void __launch_bounds__(kThreads, 2) sb_gate_up_kernel(const __grid_co
     __syncthreads();
     tc::tc_fence_after();
     const uint32_t tmem_base = *tmem_holder;
-
-    const int prob = (int)blockIdx.x / p.tiles;
-    const int ch0 = ((int)blockIdx.x - prob * p.tiles) * kTile;
+    if (threadIdx.x == 0) SB_TL(0, 1);
+    const int extra = p.rows > kTile ? p.rows - kTile : 0;  // rows of the second tile that are new
 
     if (warp == 0) {
         if (lane == 0) {
-            tc::prefetch_tmap(&p.w_map[prob]);
-            tc::prefetch_tmap(&p.x_map);
-            // the weights depend on nothing earlier in the stream: the first stages' weight boxes leave at once,
-            // their activation boxes after the dependency wait
-            const int ahead = min(p.stages, p.k_blocks);
-            for (int kb = 0; kb < ahead; ++kb) {
-                tc::mbar_expect_tx(ring.full(kb), p.stage_bytes);
-                tc::tma_load_2d(ring.stage(kb), &p.w_map[prob], ring.full(kb), kb * kBK, ch0);
-            }
             tc::pdl_wait();
+            SB_TL(0, 2);
             for (int kb = 0; kb < ahead; ++kb)
-                tc::tma_load_2d(ring.stage(kb) + kWeightStageBytes, &p.x_map, ring.full(kb), kb * kBK, 0);
+                tc::tma_load_2d(ring.stage(kb) + p.w_bytes, &p.x_map, ring.full(kb), kb * kBK, 0);
             int stage = 0;
             uint32_t phase = 1;  // the ring has gone round once
             for (int kb = ahead; kb < p.k_blocks; ++kb) {
                 if (!tc::mbar_wait(ring.empty(stage), phase ^ 1u, abort_flag, p.status)) break;
                 tc::mbar_expect_tx(ring.full(stage), p.stage_bytes);
                 tc::tma_load_2d(ring.stage(stage), &p.w_map[prob], ring.full(stage), kb * kBK, ch0);
-                tc::tma_load_2d(ring.stage(stage) + kWeightStageBytes, &p.x_map, ring.full(stage), kb * kBK, 0);
+                tc::tma_load_2d(ring.stage(stage) + p.w_bytes, &p.x_map, ring.full(stage), kb * kBK, 0);
                 if (++stage == p.stages) {
                     stage = 0;
                     phase ^= 1u;
@@ -170,11 +197,18 @@ __global__ void __launch_bounds__(kThreads, 2) sb_gate_up_kernel(const __grid_co
                     break;
                 }
                 tc::tc_fence_after();
-                const uint32_t sa = ring.stage(stage), sb = sa + kWeightStageBytes;
+                if (kb == 0) SB_TL(0, 3);
+                const uint32_t sa = ring.stage(stage), sb = sa + p.w_bytes;
 #pragma unroll
-                for (int k = 0; k < kBK / 16; ++k)
-                    tc::umma_bf16(tmem_base, tc::make_smem_desc(sa + k * 32, 16, 1024),
-                                  tc::make_smem_desc(sb + k * 32, 16, 1024), idesc, (kb | k) != 0 ? 1u : 0u);
+                for (int k = 0; k < kBK / 16; ++k) {
+                    const uint64_t bd = tc::make_smem_desc(sb + k * 32, 16, 1024);
+                    tc::umma_bf16(tmem_base, tc::make_smem_desc(sa + k * 32, 16, 1024), bd, idesc,
+                                  (kb | k) != 0 ? 1u : 0u);
+                    if (extra)
+                        tc::umma_bf16(tmem_base + (uint32_t)p.tn,
+                                      tc::make_smem_desc(sa + (uint32_t)extra * 128u + k * 32, 16, 1024), bd, idesc,
+                                      (kb | k) != 0 ? 1u : 0u);
+                }
                 tc::umma_commit(ring.empty(stage));
                 if (++stage == p.stages) {
                     stage = 0;
@@ -182,32 +216,66 @@ __global__ void __launch_bounds__(kThreads, 2) sb_gate_up_kernel(const __grid_co
                 }
             }
             if (ok) tc::umma_commit(ring.tfull());
+            SB_TL(0, 4);
         }
     } else {
         // ---- epilogue: lane = channel, columns = tokens; a warp's store of one token is 128 contiguous bytes
         const int quarter = warp & 3;
         tc::pdl_wait();  // the workspace may still be read by the previous call's kernels
         if (blockIdx.x == 0)
-            for (int i = (int)threadIdx.x - 64; i < p.n_counters; i += 128) p.counters[i] = 0;
+            for (int i = (int)threadIdx.x - 64; i < p.n_counters; i += kEpiThreads) p.counters[i] = 0;
         if (__all_sync(0xffffffffu, tc::mbar_wait(ring.tfull(), 0u, abort_flag, p.status))) {
             tc::tc_fence_after();
-            const int ch = ch0 + quarter * 32 + lane;
-            float *dst = (prob == 0 ? p.G : p.U) + ch;
-            for (int c0 = 0; c0 < p.tn; c0 += 32) {
+            if (threadIdx.x == 64) SB_TL(0, 5);
+            float *base = prob == 0 ? p.G : p.U;
+            const int trow = quarter * 32 + lane;  // row of the MMA tile this thread reads
+            const int valid = min(p.rows, p.F - ch0);  // channels of this CTA inside the matrix
+            // The tile goes through the (now idle) stage ring, transposed to [token][channel], and leaves as one
+            // bulk store per token: 128 scalar stores per thread would add microseconds to the end of the kernel.
+            // A channel count that is not a multiple of 4 (a ragged last CTA) cannot be a bulk copy: direct stores.
+            const bool bulk = (valid & 3) == 0;
+            const uint32_t pitch = (uint32_t)p.rows * 4u;
+            float *stage_f = reinterpret_cast<float *>(smem_raw + (ring.base - raw));
+            // work items = (tile, 32-token chunk); the two warps of a lane quarter take alternate items
+            const int chunks = p.tn >> 5, half = (warp - 2) >> 2;
+            for (int item = half; item < (extra ? 2 : 1) * chunks; item += 2) {
+                const int tile = item / chunks, c0 = (item - tile * chunks) << 5;
+                const int row = tile == 0 ? trow : extra + trow;  // row within the CTA's channels
+                const bool mine = (tile == 0 ? trow < p.rows : trow >= kTile - extra) && row < valid;
+                if (tile == 1 && quarter * 32 + 31 < kTile - extra) continue;  // warp-uniform: nothing new in this quarter
                 uint32_t r[32];
                 __syncwarp();
-                tc::tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0, r);
+                tc::tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(tile * p.tn + c0), r);
                 tc::tmem_ld_wait();
-                if (ch < p.F) {
+                if (!mine) {
+                    // (no early exit: the TMEM load above is warp-collective)
+                } else if (bulk) {
+                    float *dst = stage_f + (size_t)c0 * p.rows + row;
 #pragma unroll
                     for (int i = 0; i < 32; ++i)
-                        if (c0 + i < p.T) dst[(int64_t)(c0 + i) * p.ldf] = __uint_as_float(r[i]);
+                        if (c0 + i < p.T) dst[i * p.rows] = __uint_as_float(r[i]);
+                } else {
+                    float *dst = base + ch0 + row + (int64_t)c0 * p.ldf;
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        if (c0 + i < p.T) dst[(int64_t)i * p.ldf] = __uint_as_float(r[i]);
+                }
+            }
+            if (bulk) {
+                tc::fence_async_smem();
+                asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
+                const int etid = (int)threadIdx.x - 64;
+                if (etid < p.T) {
+                    tc::bulk_copy_s2g(base + (int64_t)etid * p.ldf + ch0, ring.base + (uint32_t)etid * pitch,
+                                      (uint32_t)valid * 4u);
+                    tc::bulk_store_wait_read<0>();  // shared memory must outlive the copy's reads
                 }
             }
         }
     }
 
     __syncwarp();
+    if (threadIdx.x == 64) SB_TL(0, 6);
     if (*abort_flag) {
         const long long t0 = clock64();
         while (clock64() - t0 < 2000000LL) __nanosleep(1000);
@@ -229,26 +297,64 @@ struct SelectParams {
     float *acc;          // [T, d], zeroed here
     int16_t *idx_out;    // compact saved activations [T, K] (all three or none)
     __nv_bfloat16 *g_out, *u_out;
+    int stage_u;         // 1: shared memory has room for the token's up row as well
+    int *status;
+    const uint8_t *next_weights;  // W_down: pulled into L2 while the selection runs (HBM is idle then), or null
+    uint64_t next_bytes;
 };
 
-// One CTA per token.  The threshold search is the decode plan's; the set then leaves as the token's dense
-// masked row Z' (and, when asked for, as the compact triple in ascending channel order).
+constexpr uint32_t kPrefetchChunk = 16 * 1024;
+
+// CTA `part` of `parts` asks for its share of [ptr, ptr + bytes) to be brought into L2.
+__device__ __forceinline__ void prefetch_share(const uint8_t *ptr, uint64_t bytes, int part, int parts) {
+    if (!ptr) return;
+    const int64_t chunks = (int64_t)((bytes + kPrefetchChunk - 1) / kPrefetchChunk);
+    const int64_t c0 = chunks * part / parts, c1 = chunks * (part + 1) / parts;
+    for (int64_t c = c0 + threadIdx.x; c < c1; c += blockDim.x) {
+        const uint64_t off = (uint64_t)c * kPrefetchChunk;
+        tc::bulk_prefetch_l2(ptr + off, (uint32_t)min((uint64_t)kPrefetchChunk, bytes - off));
+    }
+}
+
+// dynamic shared memory of sb_select_kernel: keys [Fp] | 2 candidate lists | up row [Fp] (when staged)
+inline size_t select_smem(int F, bool stage_u) {
+    const size_t Fp = (size_t)((F + 3) & ~3);
+    return (Fp * (stage_u ? 2 : 1) + 2 * dec::kSelListCap) * sizeof(uint32_t);
+}
+
+// One CTA per token.  The token's gate row (and up row) arrive with bulk copies; the threshold search is the decode
+// plan's; the set then leaves as the token's dense masked row Z' (and, when asked for, as the compact triple in
+// ascending channel order).  Gate values are recovered from their keys, so a NaN gate value acts as -inf in the
+// product as well as in the selection.
 __global__ void __launch_bounds__(dec::kSelThreads) sb_select_kernel(const SelectParams p) {
-    extern __shared__ __align__(16) uint32_t dyn[];  // keys [F] | 2 candidate lists (the first doubles as the bitmap)
+    extern __shared__ __align__(16) uint32_t dyn[];
     __shared__ SelectSmemT<dec::kSelThreads / 32> sm;
+    __shared__ uint64_t s_bar;
+    __shared__ int s_abort;
     const int tid = threadIdx.x;
     const int t = blockIdx.x;
+    const int Fp = (p.F + 3) & ~3;
+    uint32_t *keys = dyn, *lists = dyn + Fp;
+    uint32_t *bits = lists;  // bitmap of the kept channels once the search is over
+    const float *u_row = p.stage_u ? reinterpret_cast<const float *>(lists + 2 * dec::kSelListCap)
+                                   : p.U + (int64_t)t * p.ldf;
     tc::pdl_launch_dependents();
+    if (tid == 0) SB_TL(2, 0);
     tc::pdl_wait();
-    const float *g = p.G + (int64_t)t * p.ldf, *u = p.U + (int64_t)t * p.ldf;
-    for (int i = tid; i < p.d / 4; i += dec::kSelThreads)
+    if (tid == 0) SB_TL(2, 1);
+    prefetch_share(p.next_weights, p.next_bytes, t, (int)gridDim.x);
+    dec::cta_stage_rows_begin(&s_bar, &s_abort, keys, p.G + (int64_t)t * p.ldf, (uint32_t)Fp * 4u,
+                              p.stage_u ? lists + 2 * dec::kSelListCap : nullptr,
+                              p.stage_u ? p.U + (int64_t)t * p.ldf : nullptr);
+    for (int i = tid; i < p.d / 4; i += dec::kSelThreads)  // while the rows travel
         reinterpret_cast<float4 *>(p.acc + (int64_t)t * p.d)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (!dec::cta_stage_rows_wait(&s_bar, &s_abort, p.status)) return;
+    if (tid == 0) SB_TL(2, 2);
     uint32_t tau;
     int need;
     bool ties_cut;
-    dec::cta_select_threshold(g, p.F, p.K, dyn, sm, tau, need, ties_cut);
-    const uint32_t *keys = dyn;
-    uint32_t *bits = dyn + p.F;  // bitmap of the kept channels, only when ties are cut or the triple is wanted
+    dec::cta_select_threshold(nullptr, p.F, p.K, keys, lists, sm, tau, need, ties_cut);
+    if (tid == 0) SB_TL(2, 3);
     const bool save = p.idx_out != nullptr;
     const bool by_bitmap = ties_cut || save;
     if (by_bitmap) {
@@ -262,31 +368,41 @@ __global__ void __launch_bounds__(dec::kSelThreads) sb_select_kernel(const Selec
             atomicOr(&bits[j >> 5], 1u << (j & 31));
             if (save) {
                 io[pos] = (int16_t)j;
-                go[pos] = __float2bfloat16_rn(g[j]);
-                uo[pos] = __float2bfloat16_rn(u[j]);
+                go[pos] = __float2bfloat16_rn(key_to_float(keys[j]));
+                uo[pos] = __float2bfloat16_rn(u_row[j]);
             }
         });
     }
-    // Z' row, two channels per thread.  The saved up value is rounded to bf16 before it is used, so that the
-    // backward pass, which recomputes z from the saved pair, sees the same product.
+    if (tid == 0) SB_TL(2, 4);
+    // Z' row, eight channels (one 16-byte store) per thread and step.  When the triple is saved the up value is
+    // rounded to bf16 before it is used, so that the backward pass, which recomputes z from the saved pair, sees the
+    // same product.  The last group may reach into the row's padding (ldz is a multiple of 8): zeros go there.
     __nv_bfloat16 *z = p.Z + (int64_t)t * p.ldz;
-    for (int j = 2 * tid; j < p.F; j += 2 * dec::kSelThreads) {
-        float v[2] = {0.f, 0.f};
+    for (int q = tid; q * 8 < p.F; q += dec::kSelThreads) {
+        const int j0 = q * 8;
+        // (16-byte reads: the keys' array is followed by the lists, so a group that straddles F reads valid memory)
+        const uint4 ka = *reinterpret_cast<const uint4 *>(keys + j0), kb = *reinterpret_cast<const uint4 *>(keys + j0 + 4);
+        const uint32_t kk[8] = {ka.x, ka.y, ka.z, ka.w, kb.x, kb.y, kb.z, kb.w};
+        uint32_t kept = 0;
+        if (by_bitmap) {
+            kept = (bits[j0 >> 5] >> (j0 & 31)) & 0xffu;
+        } else {
 #pragma unroll
-        for (int e = 0; e < 2; ++e) {
-            const int jj = j + e;
-            if (jj >= p.F) continue;
-            const bool kept = by_bitmap ? ((bits[jj >> 5] >> (jj & 31)) & 1u) != 0u : keys[jj] >= tau;
-            if (kept) {
-                const float uv = save ? __bfloat162float(__float2bfloat16_rn(u[jj])) : u[jj];
-                v[e] = silu_f(g[jj]) * uv;
+            for (int e = 0; e < 8; ++e)
+                if (j0 + e < p.F && kk[e] >= tau) kept |= 1u << e;
+        }
+        float v[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            if ((kept >> e) & 1u) {
+                const float uv = save ? __bfloat162float(__float2bfloat16_rn(u_row[j0 + e])) : u_row[j0 + e];
+                v[e] = silu_f(key_to_float(kk[e])) * uv;
             }
         }
-        if (j + 1 < p.ldz)
-            *reinterpret_cast<__nv_bfloat162 *>(z + j) = __floats2bfloat162_rn(v[0], v[1]);
-        else
-            z[j] = __float2bfloat16_rn(v[0]);
+        *reinterpret_cast<uint4 *>(z + j0) = make_uint4(tc::pack_bf16(v[0], v[1]), tc::pack_bf16(v[2], v[3]),
+                                                        tc::pack_bf16(v[4], v[5]), tc::pack_bf16(v[6], v[7]));
     }
+    if (tid == 0) SB_TL(2, 5);
 }
 
 // MoC 2:8 (Section 4): the mask is local, one thread per group of 8 channels.
@@ -295,6 +411,7 @@ __global__ void __launch_bounds__(dec::kSelThreads) sb_select_grouped_kernel(con
     const int t = blockIdx.x;
     tc::pdl_launch_dependents();
     tc::pdl_wait();
+    prefetch_share(p.next_weights, p.next_bytes, t, (int)gridDim.x);
     const float *g = p.G + (int64_t)t * p.ldf, *u = p.U + (int64_t)t * p.ldf;
     for (int i = tid; i < p.d / 4; i += dec::kSelThreads)
         reinterpret_cast<float4 *>(p.acc + (int64_t)t * p.d)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -303,7 +420,10 @@ __global__ void __launch_bounds__(dec::kSelThreads) sb_select_grouped_kernel(con
     for (int q = tid; q < p.F / kGroup; q += dec::kSelThreads) {
         const float4 g0 = reinterpret_cast<const float4 *>(g + q * kGroup)[0];
         const float4 g1 = reinterpret_cast<const float4 *>(g + q * kGroup)[1];
+        const float4 u0 = reinterpret_cast<const float4 *>(u + q * kGroup)[0];
+        const float4 u1 = reinterpret_cast<const float4 *>(u + q * kGroup)[1];
         const float gv[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+        const float uv[8] = {u0.x, u0.y, u0.z, u0.w, u1.x, u1.y, u1.z, u1.w};
         uint32_t key[8];
 #pragma unroll
         for (int e = 0; e < 8; ++e) key[e] = gate_key(gv[e]);
@@ -313,11 +433,13 @@ __global__ void __launch_bounds__(dec::kSelThreads) sb_select_grouped_kernel(con
         const int sel[2] = {lo, hi};
 #pragma unroll
         for (int s = 0; s < 2; ++s) {
-            float gs = 0.f;
+            float gs = 0.f, us = 0.f;
 #pragma unroll
             for (int e = 0; e < 8; ++e)
-                if (e == sel[s]) gs = gv[e];
-            float us = u[q * kGroup + sel[s]];
+                if (e == sel[s]) {
+                    gs = gv[e];
+                    us = uv[e];
+                }
             if (save) {
                 const int64_t o = (int64_t)t * p.K + 2 * q + s;
                 p.idx_out[o] = (int16_t)(q * kGroup + sel[s]);
@@ -337,20 +459,35 @@ __global__ void __launch_bounds__(dec::kSelThreads) sb_select_grouped_kernel(con
 }
 
 // ---------------------------------------------------------------------------------------------- 3. down
-// grid = m_tiles * splits; CTA (m, s) contracts its share of the channel blocks for output columns 128 m ..
-__global__ void __launch_bounds__(kThreads, 2) sb_down_kernel(const __grid_constant__ DownParams p) {
+// grid = m_tiles * splits; CTA (m, s) contracts its share of the channel blocks for output columns
+// 128 * accs * m ..; with accs == 2 the activation box of a stage feeds two MMA tiles.
+__global__ void __launch_bounds__(kThreads, 1) sb_down_kernel(const __grid_constant__ DownParams p) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ int s_last;
     const uint32_t raw = tc::smem_u32(smem_raw);
     Ring ring;
     ring.base = (raw + 1023u) & ~1023u;
     ring.stage_bytes = p.stage_bytes;
-    ring.bar_base = ring.base + (uint32_t)p.stages * p.stage_bytes;
+    ring.bar_base = ring.base + (uint32_t)p.stages * p.stage_bytes + kTile * kBK * 2;
     uint8_t *bar_ptr = smem_raw + (ring.bar_base - raw);
     volatile uint32_t *tmem_holder = reinterpret_cast<volatile uint32_t *>(bar_ptr + 8 * (2 * kMaxStages + 1));
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_holder + 1);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     tc::pdl_launch_dependents();
+    if (threadIdx.x == 0) SB_TL(1, 0);
+
+    const int m_blk = (int)blockIdx.x / p.splits, split = (int)blockIdx.x - m_blk * p.splits;
+    const int kb0 = (int)(((int64_t)split * p.k_blocks) / p.splits);
+    const int kb1 = (int)(((int64_t)(split + 1) * p.k_blocks) / p.splits);
+    const int nkb = kb1 - kb0;  // >= 1: the host keeps splits <= k_blocks
+    const int col0 = m_blk * kTile * p.accs;
+    const int ahead = min(p.stages, nkb);
+    auto load_w = [&](int stage, int kb) {
+        // boxes of 64 columns x 64 channels, 8 KiB each: the M-major operand layout, two boxes per MMA tile
+        for (int b = 0; b < 2 * p.accs; ++b)
+            tc::tma_load_2d(ring.stage(stage) + (uint32_t)b * (64 * kBK * 2), &p.wd_map, ring.full(stage), col0 + 64 * b,
+                            kb * kBK);
+    };
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
@@ -358,9 +495,14 @@ __global__ void __launch_bounds__(kThreads, 2) sb_down_kernel(const __grid_const
             tc::mbar_init(ring.empty(s), 1);
         }
         tc::mbar_init(ring.tfull(), 1);
+        tc::mbar_init(ring.extra(), 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        for (int i = 0; i < ahead; ++i) {  // weights first: they depend on nothing earlier in the stream
+            tc::mbar_expect_tx(ring.full(i), p.stage_bytes);
+            load_w(i, kb0 + i);
+        }
     }
     if (warp == 1) {
         tc::tmem_alloc(tc::smem_u32(const_cast<uint32_t *>(tmem_holder)), (uint32_t)p.tmem_cols);
@@ -370,37 +512,20 @@ __global__ void __launch_bounds__(kThreads, 2) sb_down_kernel(const __grid_const
     __syncthreads();
     tc::tc_fence_after();
     const uint32_t tmem_base = *tmem_holder;
-
-    const int m_blk = (int)blockIdx.x / p.splits, split = (int)blockIdx.x - m_blk * p.splits;
-    const int kb0 = (int)(((int64_t)split * p.k_blocks) / p.splits);
-    const int kb1 = (int)(((int64_t)(split + 1) * p.k_blocks) / p.splits);
-    const int nkb = kb1 - kb0;  // >= 1: the host keeps splits <= k_blocks
-    const int col0 = m_blk * kTile;
+    if (threadIdx.x == 0) SB_TL(1, 1);
 
     if (warp == 0) {
         if (lane == 0) {
-            tc::prefetch_tmap(&p.wd_map);
-            tc::prefetch_tmap(&p.z_map);
-            auto load_w = [&](int stage, int kb) {
-                // two boxes of 64 columns x 64 channels: the M-major operand layout
-                tc::tma_load_2d(ring.stage(stage), &p.wd_map, ring.full(stage), col0, kb * kBK);
-                tc::tma_load_2d(ring.stage(stage) + 64 * kBK * 2, &p.wd_map, ring.full(stage), col0 + 64, kb * kBK);
-            };
-            const int ahead = min(p.stages, nkb);
-            for (int i = 0; i < ahead; ++i) {
-                tc::mbar_expect_tx(ring.full(i), p.stage_bytes);
-                load_w(i, kb0 + i);
-            }
             tc::pdl_wait();  // Z' comes from the select kernel
             for (int i = 0; i < ahead; ++i)
-                tc::tma_load_2d(ring.stage(i) + kWeightStageBytes, &p.z_map, ring.full(i), (kb0 + i) * kBK, 0);
+                tc::tma_load_2d(ring.stage(i) + p.w_bytes, &p.z_map, ring.full(i), (kb0 + i) * kBK, 0);
             int stage = 0;
             uint32_t phase = 1;
             for (int i = ahead; i < nkb; ++i) {
                 if (!tc::mbar_wait(ring.empty(stage), phase ^ 1u, abort_flag, p.status)) break;
                 tc::mbar_expect_tx(ring.full(stage), p.stage_bytes);
                 load_w(stage, kb0 + i);
-                tc::tma_load_2d(ring.stage(stage) + kWeightStageBytes, &p.z_map, ring.full(stage), (kb0 + i) * kBK, 0);
+                tc::tma_load_2d(ring.stage(stage) + p.w_bytes, &p.z_map, ring.full(stage), (kb0 + i) * kBK, 0);
                 if (++stage == p.stages) {
                     stage = 0;
                     phase ^= 1u;
@@ -419,11 +544,16 @@ __global__ void __launch_bounds__(kThreads, 2) sb_down_kernel(const __grid_const
                     break;
                 }
                 tc::tc_fence_after();
-                const uint32_t sa = ring.stage(stage), sb = sa + kWeightStageBytes;
+                if (i == 0) SB_TL(1, 3);
+                const uint32_t sa = ring.stage(stage), sb = sa + p.w_bytes;
 #pragma unroll
-                for (int k = 0; k < kBK / 16; ++k)
-                    tc::umma_bf16(tmem_base, tc::make_smem_desc(sa + k * 2048, kBK * 128, 1024),
-                                  tc::make_smem_desc(sb + k * 32, 16, 1024), idesc, (i | k) != 0 ? 1u : 0u);
+                for (int k = 0; k < kBK / 16; ++k) {
+                    const uint64_t bd = tc::make_smem_desc(sb + k * 32, 16, 1024);
+                    for (int a = 0; a < p.accs; ++a)
+                        tc::umma_bf16(tmem_base + (uint32_t)(a * p.tn),
+                                      tc::make_smem_desc(sa + (uint32_t)a * (2 * 64 * kBK * 2) + k * 2048, kBK * 128, 1024),
+                                      bd, idesc, (i | k) != 0 ? 1u : 0u);
+                }
                 tc::umma_commit(ring.empty(stage));
                 if (++stage == p.stages) {
                     stage = 0;
@@ -431,6 +561,7 @@ __global__ void __launch_bounds__(kThreads, 2) sb_down_kernel(const __grid_const
                 }
             }
             if (ok) tc::umma_commit(ring.tfull());
+            SB_TL(1, 4);
         }
     } else {
         // ---- epilogue: lane = output column, TMEM columns = tokens
@@ -438,41 +569,87 @@ __global__ void __launch_bounds__(kThreads, 2) sb_down_kernel(const __grid_const
         const int etid = (int)threadIdx.x - 64;
         tc::pdl_wait();
         const bool done = __all_sync(0xffffffffu, tc::mbar_wait(ring.tfull(), 0u, abort_flag, p.status));
+        if (etid == 0) SB_TL(1, 5);
         if (done) {
             tc::tc_fence_after();
-            const int col = col0 + quarter * 32 + lane;
-            float *dst = p.acc + col;
-            for (int c0 = 0; c0 < p.tn; c0 += 32) {
+            const int chunks = p.tn >> 5, half = (warp - 2) >> 2;
+            for (int item = half; item < p.accs * chunks; item += 2) {
+                const int a = item / chunks, c0 = (item - a * chunks) << 5;
+                const int col = col0 + a * kTile + quarter * 32 + lane;
                 uint32_t r[32];
                 __syncwarp();
-                tc::tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0, r);
+                tc::tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(a * p.tn + c0), r);
                 tc::tmem_ld_wait();
-                if (col < p.d) {
+                // 4 x 4 transposes among the four lanes that hold four adjacent columns: lane l of the group ends up
+                // with the four columns of token 4 g + l, which leave as one 16-byte vector reduction (d is a
+                // multiple of 8, so a group of four columns is inside the row or outside it as a whole)
+                const int l4 = lane & 3;
+                const bool odd = (l4 & 1) != 0, hi = (l4 & 2) != 0;
 #pragma unroll
-                    for (int i = 0; i < 32; ++i)
-                        if (c0 + i < p.T) atomicAdd(dst + (int64_t)(c0 + i) * p.d, __uint_as_float(r[i]));
+                for (int g4 = 0; g4 < 8; ++g4) {
+                    float v0 = __uint_as_float(r[4 * g4]), v1 = __uint_as_float(r[4 * g4 + 1]);
+                    float v2 = __uint_as_float(r[4 * g4 + 2]), v3 = __uint_as_float(r[4 * g4 + 3]);
+                    float x0 = __shfl_xor_sync(0xffffffffu, odd ? v0 : v1, 1);
+                    float x1 = __shfl_xor_sync(0xffffffffu, odd ? v2 : v3, 1);
+                    if (odd) {
+                        v0 = x0;
+                        v2 = x1;
+                    } else {
+                        v1 = x0;
+                        v3 = x1;
+                    }
+                    x0 = __shfl_xor_sync(0xffffffffu, hi ? v0 : v2, 2);
+                    x1 = __shfl_xor_sync(0xffffffffu, hi ? v1 : v3, 2);
+                    if (hi) {
+                        v0 = x0;
+                        v1 = x1;
+                    } else {
+                        v2 = x0;
+                        v3 = x1;
+                    }
+                    const int tok = c0 + 4 * g4 + l4;
+                    if (tok < p.T && col < p.d)
+                        asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(
+                                         p.acc + (int64_t)tok * p.d + (col - l4)),
+                                     "f"(v0), "f"(v1), "f"(v2), "f"(v3)
+                                     : "memory");
                 }
             }
         }
         // the last CTA of this column block to get here rounds the sums to bf16
+        if (etid == 0) SB_TL(1, 6);
         __threadfence();
-        asm volatile("bar.sync 1, 128;" ::: "memory");
+        asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
         if (etid == 0) s_last = atomicAdd(&p.counters[m_blk], 1) == p.splits - 1;
-        asm volatile("bar.sync 1, 128;" ::: "memory");
+        asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
         if (s_last) {
             __threadfence();
-            const int cols = min(kTile, p.d - col0);  // even: d is a multiple of 8
-            const int half = cols / 2;
-            for (int i = etid; i < p.T * half; i += 128) {
-                const int t = i / half, c = (i - t * half) * 2;
-                const float2 v = __ldcg(reinterpret_cast<const float2 *>(p.acc + (int64_t)t * p.d + col0 + c));
-                *reinterpret_cast<__nv_bfloat162 *>(p.out + (int64_t)t * p.d + col0 + c) = __floats2bfloat162_rn(v.x, v.y);
+            // The sums of this column block come back with one bulk copy per token into the (now idle) stage ring
+            // -- a handful of plain loads per thread would take longer than the whole main loop -- and leave as bf16.
+            asm volatile("fence.proxy.async;" ::: "memory");
+            const int cols = min(kTile * p.accs, p.d - col0);  // a multiple of 8
+            const uint32_t row_bytes = (uint32_t)cols * 4u;
+            if (etid == 0) tc::mbar_expect_tx(ring.extra(), row_bytes * (uint32_t)p.T);
+            asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
+            for (int t = etid; t < p.T; t += kEpiThreads)
+                tc::bulk_copy_g2s(ring.base + (uint32_t)t * row_bytes, p.acc + (int64_t)t * p.d + col0, row_bytes,
+                                  ring.extra());
+            if (__all_sync(0xffffffffu, tc::mbar_wait(ring.extra(), 0u, abort_flag, p.status))) {
+                const uint8_t *stage_ptr = smem_raw + (ring.base - raw);
+                const int vecs = cols / 4, total = p.T * vecs;
+                for (int i = etid; i < total; i += kEpiThreads) {
+                    const int t = i / vecs, c = (i - t * vecs) * 4;
+                    const float4 v = *reinterpret_cast<const float4 *>(stage_ptr + (size_t)t * row_bytes + (size_t)c * 4);
+                    *reinterpret_cast<uint2 *>(p.out + (int64_t)t * p.d + col0 + c) =
+                        make_uint2(tc::pack_bf16(v.x, v.y), tc::pack_bf16(v.z, v.w));
+                }
             }
             if (etid == 0) p.counters[m_blk] = 0;
         }
     }
 
     __syncwarp();
+    if (threadIdx.x == 64) SB_TL(1, 7);
     if (*abort_flag) {
         const long long t0 = clock64();
         while (clock64() - t0 < 2000000LL) __nanosleep(1000);
