@@ -53,7 +53,7 @@ extern "C" {
 typedef enum {
     MOC_OK = 0,
     MOC_ERR_INVALID_ARG = -1, /* NULL/misaligned pointer, k outside [1, d_ff], negative sizes ...   */
-    MOC_ERR_UNSUPPORTED = -2, /* d_ff > 32768 (int16 indices), d_model % 8 != 0, decode tokens > 16 */
+    MOC_ERR_UNSUPPORTED = -2, /* d_ff > 32768 (int16 indices), d_model % 8 != 0, decode tokens > 128 */
     MOC_ERR_WORKSPACE = -3,   /* workspace pointer NULL or smaller than moc_ffn_workspace_bytes()    */
     MOC_ERR_CUDA = -4,        /* a CUDA runtime call or a launch failed                             */
     MOC_ERR_TIMEOUT = -5,     /* device status: a bounded wait inside a kernel expired              */
@@ -119,9 +119,14 @@ MOC_API int moc_ffn_backward(const moc_ffn_desc *desc, const void *x, const void
                              void *cuda_stream);
 
 /*
- * Small-batch inference (Section 5): the same forward for tokens <= 16, organised so that only the
- * gate matrix and the selected rows of w_up / w_down are read from HBM
- * (d d_ffn + 2 K d weight elements per token instead of 3 d d_ffn).  Nothing is saved.
+ * Small-batch inference (Section 5): the same forward with nothing saved, for tokens <= 128
+ * (more: MOC_ERR_UNSUPPORTED; use moc_ffn_forward).  Up to 16 tokens it is organised so that only the
+ * gate matrix and the selected rows of w_up / w_down are read from HBM (d d_ffn + 2 K d weight
+ * elements per token instead of 3 d d_ffn).  From 17 tokens on the union of the tokens' channel sets
+ * covers nearly every channel, and all three matrices are streamed once through tensor-core kernels
+ * whose tiles are shaped for a few dozen tokens; moc_ffn_forward takes the same path for such batches.
+ * In both forms the partial sums of the down projection meet in an fp32 accumulator in an order that
+ * is not fixed, so the last bit of `out` can differ from run to run.
  */
 MOC_API int moc_ffn_decode(const moc_ffn_desc *desc, const void *x, const void *w_gate, const void *w_up,
                            const void *w_down, void *out, void *workspace, size_t workspace_bytes,
@@ -162,7 +167,9 @@ MOC_API int moc_ffn_decode_static(const moc_ffn_desc *desc, const void *x, const
 /*
  * The Top-K selector alone (the mask definition of Section 3.2), exposed so that it can be checked
  * bit-exactly: gate [rows, n_ld] fp32 on the device, only the first n columns of a row are channels;
- * idx_out [rows, k] int16 ascending.  Needs no workspace.
+ * idx_out [rows, k] int16 ascending.  Needs no workspace.  As in the plans, up to 128 rows are handled by
+ * the selector that gives a whole CTA to each row (decode and small-batch plans), more rows by the
+ * selector of the gathered plan; both are exact.
  */
 MOC_API int moc_topk_select(int64_t rows, int32_t n, int32_t n_ld, int32_t k, const float *gate,
                             int16_t *idx_out, void *cuda_stream);

@@ -3,6 +3,7 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <cmath>
 #include <atomic>
 #include <cstdint>
 #include <cstring>
@@ -611,8 +612,11 @@ DecodeLayout decode_layout(const moc_ffn_desc &d) {
     return L;
 }
 
+bool use_small_batch_plan(const moc_ffn_desc &d);
+
 bool use_decode_plan(const moc_ffn_desc &d) {
-    return d.dtype == MOC_BF16 && d.tokens >= 1 && d.tokens <= 16 && d.d_model <= 256 * dec::kSliceCols;
+    return d.dtype == MOC_BF16 && d.tokens >= 1 && d.tokens <= 16 && d.d_model <= 256 * dec::kSliceCols &&
+           !use_small_batch_plan(d);
 }
 
 // Launch with programmatic stream serialization allowed: the kernel may become resident while its predecessor in
@@ -722,8 +726,24 @@ SmallBatchLayout small_batch_layout(const moc_ffn_desc &d) {
     return L;
 }
 
+// Which of the two small-batch forms reads fewer bytes: the decode plan reads W_gate and the rows of W_up / W_down
+// that some token selected, (1 + 2 u) F d elements with u = 1 - (1 - K/F)^T the expected share of used channels; the
+// small-batch plan reads all 3 F d but has one kernel less and no gathers.  Measured on the LLaMA-7B shape the two
+// cross where u reaches one half (6 tokens at K = F/8); from 17 tokens on only the small-batch plan exists.
+// MOC_FFN_SB_MIN_TOKENS=n in the environment moves the boundary to n tokens (measurements only).
+bool small_batch_preferred(const moc_ffn_desc &d) {
+    static const int forced = [] {
+        const char *e = getenv("MOC_FFN_SB_MIN_TOKENS");
+        return e ? atoi(e) : 0;
+    }();
+    if (forced >= 1) return d.tokens >= forced;
+    if (d.tokens > 16) return true;
+    const double unused = std::pow(1.0 - (double)d.k / (double)d.d_ff, (double)d.tokens);
+    return 1.0 - unused >= 0.5;
+}
+
 bool use_small_batch_plan(const moc_ffn_desc &d) {
-    return d.dtype == MOC_BF16 && d.tokens > 16 && d.tokens <= sb::kMaxTokens &&
+    return d.dtype == MOC_BF16 && d.tokens >= 1 && d.tokens <= sb::kMaxTokens && small_batch_preferred(d) &&
            sb::select_smem(d.d_ff, false) + 48 * 1024 <= (size_t)kMaxDynSmem;
 }
 
@@ -772,16 +792,7 @@ int forward_small_batch(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __n
                launch_pdl(sb::sb_gate_up_kernel, dim3(2 * L.ctas_per_matrix), sb::kThreads, gs.smem, st, gp));
     if ((rc = launch_ok()) != MOC_OK) return rc;
 
-    // W_down fits into L2 next to the workspace on this part when it is below ~100 MB; it is asked for while the
-    // selection runs.  MOC_FFN_SB_PREFETCH=0 in the environment turns that off (for measurements).
-    static const bool prefetch_on = [] {
-        const char *e = getenv("MOC_FFN_SB_PREFETCH");
-        return !(e && e[0] == '0');
-    }();
-    const uint64_t wd_bytes = (uint64_t)F * dm * sizeof(__nv_bfloat16);
-    const bool prefetch = prefetch_on && wd_bytes <= ((uint64_t)100 << 20);
-    sb::SelectParams sp{G,  U,  L.ldf, F, d.k, dm, Z, L.ldz, acc, idx, tg, tu, L.stage_u ? 1 : 0, status,
-                        prefetch ? reinterpret_cast<const uint8_t *>(wd) : nullptr, wd_bytes};
+    sb::SelectParams sp{G, U, L.ldf, F, d.k, dm, Z, L.ldz, acc, idx, tg, tu, L.stage_u ? 1 : 0, status};
     if (d.flags & MOC_FLAG_SELECT_2_OF_8) {
         MOC_LAUNCH(KID_SB_SELECT, st,
                    launch_pdl(sb::sb_select_grouped_kernel, dim3(T), dec::kSelThreads, 0, st, sp));
@@ -948,11 +959,23 @@ int moc_topk_select(int64_t rows, int32_t n, int32_t n_ld, int32_t k, const floa
     if (n > 32768) return MOC_ERR_UNSUPPORTED;
     if (rows == 0) return MOC_OK;
     if (!good_ptr(gate) || !idx_out || (reinterpret_cast<uintptr_t>(idx_out) & 1u)) return MOC_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (rows <= sb::kMaxTokens) {
+        // as in the plans: a small batch of rows goes to the selector that gives a whole CTA to each row
+        const size_t smem1 = ((size_t)((n + 3) & ~3) + 2 * dec::kSelListCap) * sizeof(uint32_t);
+        int *status = device_status_ptr();
+        if (!status) return MOC_ERR_CUDA;
+        int rc1 = set_smem(dec::cta_select_idx_kernel, smem1);
+        if (rc1 != MOC_OK) return rc1;
+        MOC_LAUNCH(KID_TOPK_SELECT, st,
+                   (dec::cta_select_idx_kernel<<<(unsigned)rows, dec::kSelThreads, smem1, st>>>(gate, n, n_ld, k, idx_out,
+                                                                                                  status)));
+        return launch_ok();
+    }
     const size_t smem = (size_t)n * sizeof(uint32_t);
     int rc = set_smem(topk_select_kernel<kSelectThreads>, smem);
     if (rc != MOC_OK) return rc;
     const unsigned grid = (unsigned)std::min<int64_t>(rows, 148 * 32);
-    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     MOC_LAUNCH(KID_TOPK_SELECT, st,
                (topk_select_kernel<kSelectThreads><<<grid, kSelectThreads, smem, st>>>(gate, rows, n, n_ld, k,
                                                                                         idx_out)));
@@ -1115,8 +1138,3 @@ const char *moc_status_string(int status) {
 
 }  // extern "C"
 
-#ifdef MOC_SB_TIMELINE
-extern "C" __attribute__((visibility("default"))) int moc_debug_sb_read(void *host) {
-    return cudaMemcpyFromSymbol(host, moc::sb::g_tl, sizeof(moc::sb::g_tl)) == cudaSuccess ? 0 : -1;
-}
-#endif

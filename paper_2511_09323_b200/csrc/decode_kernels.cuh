@@ -29,8 +29,11 @@
 namespace moc {
 namespace dec {
 
+
+
 constexpr int kSelThreads = 1024;
 constexpr int kSelListCap = 4096;   // candidate list entries (two lists)
+constexpr int kSelCached = 12;      // keys per thread held in registers by the CTA selector (rows up to 12288 channels)
 constexpr int kSliceCols = 512;     // down projection: columns per CTA (1 KiB of a bf16 row)
 constexpr int kMaxPart = 512;       // list entries per down CTA (bound of its shared arrays)
 
@@ -412,13 +415,31 @@ __device__ __forceinline__ void cta_select_threshold(const float *__restrict__ g
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     constexpr int NW = kSelThreads / 32;
 
-    // ---- keys, minimum and maximum
+    // ---- keys, minimum and maximum.  Rows of up to kSelCached * kSelThreads channels also stay in registers (element
+    // i of a thread is channel tid + i * kSelThreads): the first level's passes then run without loads.
     uint32_t kmin = 0xffffffffu, kmax = 0u;
-    for (int j = tid; j < F; j += kSelThreads) {
-        const uint32_t key = gate_key(g ? g[j] : __uint_as_float(keys[j]));
-        keys[j] = key;
-        kmin = min(kmin, key);
-        kmax = max(kmax, key);
+    uint32_t kreg[kSelCached];
+    const bool cached = F <= kSelCached * kSelThreads;
+    if (cached) {
+#pragma unroll
+        for (int i = 0; i < kSelCached; ++i) {
+            const int j = tid + i * kSelThreads;
+            kreg[i] = 0u;
+            if (j < F) {
+                const uint32_t key = gate_key(g ? g[j] : __uint_as_float(keys[j]));
+                keys[j] = key;
+                kreg[i] = key;
+                kmin = min(kmin, key);
+                kmax = max(kmax, key);
+            }
+        }
+    } else {
+        for (int j = tid; j < F; j += kSelThreads) {
+            const uint32_t key = gate_key(g ? g[j] : __uint_as_float(keys[j]));
+            keys[j] = key;
+            kmin = min(kmin, key);
+            kmax = max(kmax, key);
+        }
     }
     kmin = __reduce_min_sync(0xffffffffu, kmin);
     kmax = __reduce_max_sync(0xffffffffu, kmax);
@@ -437,10 +458,10 @@ __device__ __forceinline__ void cta_select_threshold(const float *__restrict__ g
     SelectLevel lv{kmin, kmax, (uint32_t)K, (uint32_t)F};
     const uint32_t *src = keys;
     int which = 0;
-    bool failed = false;
+    bool failed = false, by_value = true;
     uint32_t tau = 0, in_bin = 0;
-    int need = 0;
-    // ---- range-relative radix levels
+    int need = 0, level = 0;
+    // ---- levels: histogram the candidates over their own range, keep the bin that holds the m-th largest
     while (true) {
         const uint32_t span = lv.hi - lv.lo;
         if (span == 0) {  // all candidates equal
@@ -449,24 +470,32 @@ __device__ __forceinline__ void cta_select_threshold(const float *__restrict__ g
             in_bin = lv.count;
             break;
         }
-        if (lv.count <= 64 && src != keys) {
-            // rank the few candidates directly: candidate i is the answer when exactly m-1 others precede it
-            // in (value descending, position ascending) order
-            if (tid < (int)lv.count) {
-                const uint32_t mine = src[tid];
-                uint32_t before = 0, equal = 0, gt = 0;
-#pragma unroll 8
-                for (uint32_t i = 0; i < lv.count; ++i) {  // independent broadcast loads, eight in flight
-                    const uint32_t o = src[i];
+        if (lv.count <= 128u && src != keys) {
+            // The usual end of the search: a handful of candidates, ranked by the whole CTA at once.  Eight threads
+            // share a candidate and split the others between them; candidate i is the answer when exactly m-1
+            // others precede it in (value descending, list position ascending) order.
+            const uint32_t cand = (uint32_t)tid >> 3, sub = (uint32_t)tid & 7u;
+            const bool act = cand < lv.count;
+            const uint32_t mine = act ? src[cand] : 0u;
+            uint32_t before = 0, equal = 0, gt = 0;
+            if (act) {
+                for (uint32_t j = sub; j < lv.count; j += 8) {
+                    const uint32_t o = src[j];
                     gt += o > mine ? 1u : 0u;
-                    before += (o > mine || (o == mine && i < (uint32_t)tid)) ? 1u : 0u;
+                    before += (o > mine || (o == mine && j < cand)) ? 1u : 0u;
                     equal += o == mine ? 1u : 0u;
                 }
-                if (before == lv.m - 1) {
-                    s_pick = mine;
-                    s_above = lv.m - gt;  // how many keys equal to tau are wanted
-                    s_inbin = equal;
-                }
+            }
+#pragma unroll
+            for (int o = 1; o < 8; o <<= 1) {
+                before += __shfl_xor_sync(0xffffffffu, before, o);
+                equal += __shfl_xor_sync(0xffffffffu, equal, o);
+                gt += __shfl_xor_sync(0xffffffffu, gt, o);
+            }
+            if (act && sub == 0 && before == lv.m - 1) {
+                s_pick = mine;
+                s_above = lv.m - gt;  // how many keys equal to tau are wanted
+                s_inbin = equal;
             }
             __syncthreads();
             tau = s_pick;
@@ -474,12 +503,30 @@ __device__ __forceinline__ void cta_select_threshold(const float *__restrict__ g
             in_bin = s_inbin;
             break;
         }
+        // Bins are taken over the candidates' VALUE range where that is possible: the keys of one row share sign and
+        // exponent, so equal steps of the key put a quarter of an octave into one bin (hundreds of candidates around
+        // the threshold), while equal steps of the value leave a handful.  The map value -> bin is monotone, which is
+        // all the search needs; ranks inside the kept bin are decided on the exact keys.  Where the value range is
+        // not finite, or a level made no progress, the bins are equal steps of the key (which always narrow).
+        const float lo_f = key_to_float(lv.lo), hi_f = key_to_float(lv.hi);
+        const float inv = 2048.0f / (hi_f - lo_f);
+        const bool lin = by_value && isfinite(lo_f) && isfinite(hi_f) && isfinite(inv) && inv > 0.f;
         const int bits = 32 - __clz(span);
         const int shift = bits > 11 ? bits - 11 : 0;
-        // histogram of (key - lo) >> shift over the candidates (hist is zero on entry)
-        for (uint32_t i = tid; i < lv.count; i += kSelThreads) {
-            const uint32_t key = src[i];
-            if (key >= lv.lo && key <= lv.hi) atomicAdd(&hist[(key - lv.lo) >> shift], 1u);
+        auto bin_of = [&](uint32_t key) -> uint32_t {
+            if (lin) return (uint32_t)min(2047, max(0, __float2int_rd((key_to_float(key) - lo_f) * inv)));
+            return (key - lv.lo) >> shift;
+        };
+        // histogram over the candidates (hist is zero on entry)
+        if (src == keys && cached) {
+#pragma unroll
+            for (int i = 0; i < kSelCached; ++i)
+                if (tid + i * kSelThreads < F) atomicAdd(&hist[bin_of(kreg[i])], 1u);
+        } else {
+            for (uint32_t i = tid; i < lv.count; i += kSelThreads) {
+                const uint32_t key = src[i];
+                if (key >= lv.lo && key <= lv.hi) atomicAdd(&hist[bin_of(key)], 1u);
+            }
         }
         __syncthreads();
         // suffix sums: thread i owns bins 2i, 2i+1
@@ -512,13 +559,15 @@ __device__ __forceinline__ void cta_select_threshold(const float *__restrict__ g
             s_above = s - h0;
             s_inbin = h0;
         }
+        if (tid == 0) {
+            s_min[0] = 0xffffffffu;  // range of the kept bin's keys, for the next level
+            s_max[0] = 0u;
+        }
         __syncthreads();
         const uint32_t bin = s_pick;
-        const uint32_t new_lo = lv.lo + (bin << shift);
-        const uint32_t new_hi = shift ? min(lv.hi, new_lo + ((1u << shift) - 1u)) : new_lo;
         const uint32_t new_m = lv.m - s_above, new_count = s_inbin;
-        if (shift == 0) {  // the bin is a single key value
-            tau = new_lo;
+        if (!lin && shift == 0) {  // the bin is a single key value
+            tau = lv.lo + bin;
             need = (int)new_m;
             in_bin = new_count;
             break;
@@ -527,19 +576,30 @@ __device__ __forceinline__ void cta_select_threshold(const float *__restrict__ g
             failed = true;
             break;
         }
-        // copy the bin's keys to the other list and clear the histogram for the next level
+        // copy the bin's keys to the other list (with their range) and clear the histogram for the next level
         uint32_t *dst = lists[which];
-        for (uint32_t i = tid; i < lv.count; i += kSelThreads) {
-            const uint32_t key = src[i];
-            if (key >= new_lo && key <= new_hi) dst[atomicAdd(&s_n, 1u)] = key;
+        auto keep = [&](uint32_t key) {
+            if (key >= lv.lo && key <= lv.hi && bin_of(key) == bin) {
+                dst[atomicAdd(&s_n, 1u)] = key;
+                atomicMin(&s_min[0], key);
+                atomicMax(&s_max[0], key);
+            }
+        };
+        if (src == keys && cached) {
+#pragma unroll
+            for (int i = 0; i < kSelCached; ++i)
+                if (tid + i * kSelThreads < F) keep(kreg[i]);
+        } else {
+            for (uint32_t i = tid; i < lv.count; i += kSelThreads) keep(src[i]);
         }
         for (int i = tid; i < 2048; i += kSelThreads) hist[i] = 0;
         __syncthreads();
-        if (tid == 0) s_n = 0;
-        lv = SelectLevel{new_lo, new_hi, new_m, new_count};
+        if (++level >= 6) by_value = false;  // rows whose values thin out over many octaves: key steps end in three levels
+        lv = SelectLevel{s_min[0], s_max[0], new_m, new_count};
         src = dst;
         which ^= 1;
         __syncthreads();
+        if (tid == 0) s_n = 0;
     }
     bool ties_cut = true;  // true: some keys equal to tau must be left out -> ordered emission
     if (failed)
@@ -588,6 +648,28 @@ __global__ void __launch_bounds__(kSelThreads) select_mask_kernel(Workspace ws, 
                                         [&](int, int j) { atomicOr(&my_bits[j >> 5], 1u << (j & 31)); });
     }
     list_used_channels(ws, F, arrivals, dyn);
+}
+
+
+// Stand-alone form of the CTA-per-row selector (test hook): gate [rows, n_ld] fp32 -> idx_out [rows, k] int16 ascending.
+__global__ void __launch_bounds__(kSelThreads) cta_select_idx_kernel(const float *__restrict__ gate, int n, int n_ld,
+                                                                      int k, int16_t *__restrict__ idx_out,
+                                                                      int *__restrict__ status) {
+    extern __shared__ __align__(16) uint32_t dyn[];
+    __shared__ SelectSmemT<kSelThreads / 32> sm;
+    __shared__ uint64_t s_bar;
+    __shared__ int s_abort;
+    const int np = (n + 3) & ~3;
+    const float *g = gate + (int64_t)blockIdx.x * n_ld;
+    // rows that start on a 16-byte boundary and can be read four values at a time arrive with a bulk copy
+    const bool staged = (n_ld & 3) == 0 && np <= n_ld && (reinterpret_cast<uintptr_t>(gate) & 15u) == 0;
+    if (staged && !cta_stage_rows(&s_bar, &s_abort, status, dyn, g, (uint32_t)np * 4u)) return;
+    uint32_t tau;
+    int need;
+    bool ties_cut;
+    cta_select_threshold(staged ? nullptr : g, n, k, dyn, dyn + np, sm, tau, need, ties_cut);
+    int16_t *out = idx_out + (int64_t)blockIdx.x * k;
+    block_ordered_emit<kSelThreads>(dyn, n, tau, need, sm, [&](int pos, int j) { out[pos] = (int16_t)j; });
 }
 
 // ---------------------------------------------------------------------------------------------- 4. down

@@ -29,18 +29,6 @@
 namespace moc {
 namespace sb {
 
-#ifdef MOC_SB_TIMELINE
-__device__ unsigned long long g_tl[4][512][8];
-__device__ __forceinline__ void tl_stamp(int k, int slot) {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    if (blockIdx.x < 512) g_tl[k][blockIdx.x][slot] = t;
-}
-#define SB_TL(k, slot) tl_stamp(k, slot)
-#else
-#define SB_TL(k, slot)
-#endif
-
 constexpr int kTile = 128;      // MMA M
 constexpr int kBK = 64;         // contraction elements per stage: one 128-byte swizzle row
 constexpr int kThreads = 320;   // warp 0 TMA, warp 1 MMA + TMEM, warps 2..9 epilogue (two per TMEM lane quarter)
@@ -133,7 +121,6 @@ __global__ void __launch_bounds__(kThreads, 1) sb_gate_up_kernel(const __grid_co
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_holder + 1);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     tc::pdl_launch_dependents();
-    if (threadIdx.x == 0) SB_TL(0, 0);
 
     const int prob = (int)blockIdx.x / p.ctas_per_matrix;
     const int ch0 = ((int)blockIdx.x - prob * p.ctas_per_matrix) * p.rows;
@@ -163,13 +150,11 @@ __global__ void __launch_bounds__(kThreads, 1) sb_gate_up_kernel(const __grid_co
     __syncthreads();
     tc::tc_fence_after();
     const uint32_t tmem_base = *tmem_holder;
-    if (threadIdx.x == 0) SB_TL(0, 1);
     const int extra = p.rows > kTile ? p.rows - kTile : 0;  // rows of the second tile that are new
 
     if (warp == 0) {
         if (lane == 0) {
             tc::pdl_wait();
-            SB_TL(0, 2);
             for (int kb = 0; kb < ahead; ++kb)
                 tc::tma_load_2d(ring.stage(kb) + p.w_bytes, &p.x_map, ring.full(kb), kb * kBK, 0);
             int stage = 0;
@@ -197,7 +182,6 @@ __global__ void __launch_bounds__(kThreads, 1) sb_gate_up_kernel(const __grid_co
                     break;
                 }
                 tc::tc_fence_after();
-                if (kb == 0) SB_TL(0, 3);
                 const uint32_t sa = ring.stage(stage), sb = sa + p.w_bytes;
 #pragma unroll
                 for (int k = 0; k < kBK / 16; ++k) {
@@ -216,7 +200,6 @@ __global__ void __launch_bounds__(kThreads, 1) sb_gate_up_kernel(const __grid_co
                 }
             }
             if (ok) tc::umma_commit(ring.tfull());
-            SB_TL(0, 4);
         }
     } else {
         // ---- epilogue: lane = channel, columns = tokens; a warp's store of one token is 128 contiguous bytes
@@ -226,7 +209,6 @@ __global__ void __launch_bounds__(kThreads, 1) sb_gate_up_kernel(const __grid_co
             for (int i = (int)threadIdx.x - 64; i < p.n_counters; i += kEpiThreads) p.counters[i] = 0;
         if (__all_sync(0xffffffffu, tc::mbar_wait(ring.tfull(), 0u, abort_flag, p.status))) {
             tc::tc_fence_after();
-            if (threadIdx.x == 64) SB_TL(0, 5);
             float *base = prob == 0 ? p.G : p.U;
             const int trow = quarter * 32 + lane;  // row of the MMA tile this thread reads
             const int valid = min(p.rows, p.F - ch0);  // channels of this CTA inside the matrix
@@ -275,7 +257,6 @@ __global__ void __launch_bounds__(kThreads, 1) sb_gate_up_kernel(const __grid_co
     }
 
     __syncwarp();
-    if (threadIdx.x == 64) SB_TL(0, 6);
     if (*abort_flag) {
         const long long t0 = clock64();
         while (clock64() - t0 < 2000000LL) __nanosleep(1000);
@@ -299,22 +280,7 @@ struct SelectParams {
     __nv_bfloat16 *g_out, *u_out;
     int stage_u;         // 1: shared memory has room for the token's up row as well
     int *status;
-    const uint8_t *next_weights;  // W_down: pulled into L2 while the selection runs (HBM is idle then), or null
-    uint64_t next_bytes;
 };
-
-constexpr uint32_t kPrefetchChunk = 16 * 1024;
-
-// CTA `part` of `parts` asks for its share of [ptr, ptr + bytes) to be brought into L2.
-__device__ __forceinline__ void prefetch_share(const uint8_t *ptr, uint64_t bytes, int part, int parts) {
-    if (!ptr) return;
-    const int64_t chunks = (int64_t)((bytes + kPrefetchChunk - 1) / kPrefetchChunk);
-    const int64_t c0 = chunks * part / parts, c1 = chunks * (part + 1) / parts;
-    for (int64_t c = c0 + threadIdx.x; c < c1; c += blockDim.x) {
-        const uint64_t off = (uint64_t)c * kPrefetchChunk;
-        tc::bulk_prefetch_l2(ptr + off, (uint32_t)min((uint64_t)kPrefetchChunk, bytes - off));
-    }
-}
 
 // dynamic shared memory of sb_select_kernel: keys [Fp] | 2 candidate lists | up row [Fp] (when staged)
 inline size_t select_smem(int F, bool stage_u) {
@@ -339,22 +305,17 @@ __global__ void __launch_bounds__(dec::kSelThreads) sb_select_kernel(const Selec
     const float *u_row = p.stage_u ? reinterpret_cast<const float *>(lists + 2 * dec::kSelListCap)
                                    : p.U + (int64_t)t * p.ldf;
     tc::pdl_launch_dependents();
-    if (tid == 0) SB_TL(2, 0);
     tc::pdl_wait();
-    if (tid == 0) SB_TL(2, 1);
-    prefetch_share(p.next_weights, p.next_bytes, t, (int)gridDim.x);
     dec::cta_stage_rows_begin(&s_bar, &s_abort, keys, p.G + (int64_t)t * p.ldf, (uint32_t)Fp * 4u,
                               p.stage_u ? lists + 2 * dec::kSelListCap : nullptr,
                               p.stage_u ? p.U + (int64_t)t * p.ldf : nullptr);
     for (int i = tid; i < p.d / 4; i += dec::kSelThreads)  // while the rows travel
         reinterpret_cast<float4 *>(p.acc + (int64_t)t * p.d)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     if (!dec::cta_stage_rows_wait(&s_bar, &s_abort, p.status)) return;
-    if (tid == 0) SB_TL(2, 2);
     uint32_t tau;
     int need;
     bool ties_cut;
     dec::cta_select_threshold(nullptr, p.F, p.K, keys, lists, sm, tau, need, ties_cut);
-    if (tid == 0) SB_TL(2, 3);
     const bool save = p.idx_out != nullptr;
     const bool by_bitmap = ties_cut || save;
     if (by_bitmap) {
@@ -373,7 +334,6 @@ __global__ void __launch_bounds__(dec::kSelThreads) sb_select_kernel(const Selec
             }
         });
     }
-    if (tid == 0) SB_TL(2, 4);
     // Z' row, eight channels (one 16-byte store) per thread and step.  When the triple is saved the up value is
     // rounded to bf16 before it is used, so that the backward pass, which recomputes z from the saved pair, sees the
     // same product.  The last group may reach into the row's padding (ldz is a multiple of 8): zeros go there.
@@ -391,18 +351,20 @@ __global__ void __launch_bounds__(dec::kSelThreads) sb_select_kernel(const Selec
             for (int e = 0; e < 8; ++e)
                 if (j0 + e < p.F && kk[e] >= tau) kept |= 1u << e;
         }
-        float v[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        // only the kept channels (one in eight on average) pay for the SiLU; their bf16 values are OR-ed into place
+        uint32_t w[4] = {0u, 0u, 0u, 0u};
+        while (kept) {
+            const int e = __ffs(kept) - 1;
+            kept &= kept - 1u;
+            const float uv = save ? __bfloat162float(__float2bfloat16_rn(u_row[j0 + e])) : u_row[j0 + e];
+            const float zz = silu_f(key_to_float(keys[j0 + e])) * uv;
+            const uint32_t hbits = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(zz)) << (16 * (e & 1));
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            if ((kept >> e) & 1u) {
-                const float uv = save ? __bfloat162float(__float2bfloat16_rn(u_row[j0 + e])) : u_row[j0 + e];
-                v[e] = silu_f(key_to_float(kk[e])) * uv;
-            }
+            for (int q2 = 0; q2 < 4; ++q2)
+                if ((e >> 1) == q2) w[q2] |= hbits;
         }
-        *reinterpret_cast<uint4 *>(z + j0) = make_uint4(tc::pack_bf16(v[0], v[1]), tc::pack_bf16(v[2], v[3]),
-                                                        tc::pack_bf16(v[4], v[5]), tc::pack_bf16(v[6], v[7]));
+        *reinterpret_cast<uint4 *>(z + j0) = make_uint4(w[0], w[1], w[2], w[3]);
     }
-    if (tid == 0) SB_TL(2, 5);
 }
 
 // MoC 2:8 (Section 4): the mask is local, one thread per group of 8 channels.
@@ -411,7 +373,6 @@ __global__ void __launch_bounds__(dec::kSelThreads) sb_select_grouped_kernel(con
     const int t = blockIdx.x;
     tc::pdl_launch_dependents();
     tc::pdl_wait();
-    prefetch_share(p.next_weights, p.next_bytes, t, (int)gridDim.x);
     const float *g = p.G + (int64_t)t * p.ldf, *u = p.U + (int64_t)t * p.ldf;
     for (int i = tid; i < p.d / 4; i += dec::kSelThreads)
         reinterpret_cast<float4 *>(p.acc + (int64_t)t * p.d)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -474,7 +435,6 @@ __global__ void __launch_bounds__(kThreads, 1) sb_down_kernel(const __grid_const
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_holder + 1);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     tc::pdl_launch_dependents();
-    if (threadIdx.x == 0) SB_TL(1, 0);
 
     const int m_blk = (int)blockIdx.x / p.splits, split = (int)blockIdx.x - m_blk * p.splits;
     const int kb0 = (int)(((int64_t)split * p.k_blocks) / p.splits);
@@ -512,7 +472,6 @@ __global__ void __launch_bounds__(kThreads, 1) sb_down_kernel(const __grid_const
     __syncthreads();
     tc::tc_fence_after();
     const uint32_t tmem_base = *tmem_holder;
-    if (threadIdx.x == 0) SB_TL(1, 1);
 
     if (warp == 0) {
         if (lane == 0) {
@@ -544,7 +503,6 @@ __global__ void __launch_bounds__(kThreads, 1) sb_down_kernel(const __grid_const
                     break;
                 }
                 tc::tc_fence_after();
-                if (i == 0) SB_TL(1, 3);
                 const uint32_t sa = ring.stage(stage), sb = sa + p.w_bytes;
 #pragma unroll
                 for (int k = 0; k < kBK / 16; ++k) {
@@ -561,7 +519,6 @@ __global__ void __launch_bounds__(kThreads, 1) sb_down_kernel(const __grid_const
                 }
             }
             if (ok) tc::umma_commit(ring.tfull());
-            SB_TL(1, 4);
         }
     } else {
         // ---- epilogue: lane = output column, TMEM columns = tokens
@@ -569,7 +526,6 @@ __global__ void __launch_bounds__(kThreads, 1) sb_down_kernel(const __grid_const
         const int etid = (int)threadIdx.x - 64;
         tc::pdl_wait();
         const bool done = __all_sync(0xffffffffu, tc::mbar_wait(ring.tfull(), 0u, abort_flag, p.status));
-        if (etid == 0) SB_TL(1, 5);
         if (done) {
             tc::tc_fence_after();
             const int chunks = p.tn >> 5, half = (warp - 2) >> 2;
@@ -617,7 +573,6 @@ __global__ void __launch_bounds__(kThreads, 1) sb_down_kernel(const __grid_const
             }
         }
         // the last CTA of this column block to get here rounds the sums to bf16
-        if (etid == 0) SB_TL(1, 6);
         __threadfence();
         asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
         if (etid == 0) s_last = atomicAdd(&p.counters[m_blk], 1) == p.splits - 1;
@@ -649,7 +604,6 @@ __global__ void __launch_bounds__(kThreads, 1) sb_down_kernel(const __grid_const
     }
 
     __syncwarp();
-    if (threadIdx.x == 64) SB_TL(1, 7);
     if (*abort_flag) {
         const long long t0 = clock64();
         while (clock64() - t0 < 2000000LL) __nanosleep(1000);

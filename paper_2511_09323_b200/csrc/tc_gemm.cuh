@@ -132,10 +132,6 @@ __device__ __forceinline__ void bulk_copy_s2g(void *dst, uint32_t src, uint32_t 
                  : "memory");
     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
 }
-// asks for `bytes` (a multiple of 16) at `src` to be brought into L2; nothing waits for it
-__device__ __forceinline__ void bulk_prefetch_l2(const void *src, uint32_t bytes) {
-    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
-}
 // the issuing thread's bulk stores: all but the newest `Keep` groups have read their shared-memory source
 template <int Keep>
 __device__ __forceinline__ void bulk_store_wait_read() {

@@ -68,7 +68,7 @@ def test_grouped_ties_keep_the_lower_channels_exactly():
                 assert j - 1 in sel, f"token {t}: channel {j} kept without its equal lower twin"
 
 
-@pytest.mark.parametrize("T", [1, 3, 16])
+@pytest.mark.parametrize("T", [1, 2, 3, 16])   # 1, 2: decode plan; 3, 16: small-batch plan (half the channels in use)
 def test_grouped_decode_matches_forward_and_oracle(T):
     w = syn.Workload(f"g28-dec-{T}", "bf16", T, 512, 2048, 2048, 512, seed=77 + T)
     wg, wu, wd = syn.make_weights(w)

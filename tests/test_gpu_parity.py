@@ -65,13 +65,21 @@ def _adversarial_rows(n):
         (np.round(np.random.default_rng(1).standard_normal(n) * 16) / 16).astype(np.float32),  # many duplicates
         np.random.default_rng(2).standard_normal(n).astype(np.float32) * 1e-30,               # tiny magnitudes
         np.float32(1e30) * np.random.default_rng(3).standard_normal(n).astype(np.float32),
+        (np.float32(2.0) ** (-(r % 140))).astype(np.float32),                                  # thinning out over 140 octaves
+        (np.float32(1.0) + (r % 97) * np.float32(1.2e-7)).astype(np.float32),                  # a few ulps apart
+        np.where(r == 0, 1e30, np.where(r == 1, -1e30,                                          # two outliers stretch
+                 np.random.default_rng(4).standard_normal(n) * 1e-3)).astype(np.float32),      # the range of a cluster
+        (np.random.default_rng(5).standard_normal(n) * 1e-42).astype(np.float32),              # denormals
     ]
     return np.stack(rows)
 
 
-@pytest.mark.parametrize("n,n_ld", [(1, 4), (37, 40), (256, 256), (257, 264), (2048, 2048), (5461, 5504), (32768, 32768)])
-def test_selector_bit_exact_adversarial(n, n_ld):
+@pytest.mark.parametrize("repeat", [1, 12])   # 11 rows: a CTA per row; 132 rows: the gathered plan's selector
+@pytest.mark.parametrize("n,n_ld", [(1, 4), (37, 40), (37, 37), (256, 256), (257, 264), (2048, 2048), (5461, 5504),
+                                    (11008, 11008), (32768, 32768)])
+def test_selector_bit_exact_adversarial(n, n_ld, repeat):
     rows = _adversarial_rows(max(n, 3))[:, :n] if n >= 3 else np.zeros((3, n), np.float32)
+    rows = np.tile(rows, (repeat, 1))
     g = np.full((rows.shape[0], n_ld), 1e9, np.float32)  # padding columns hold large values: must be ignored
     g[:, :n] = rows
     gd = torch.from_numpy(g).cuda()
@@ -250,7 +258,7 @@ def _check_decode(out64, x64, wg64, wu64, wd64, K, dtype, what):
         assert np.abs(out64[t] - ref).max() <= tol, f"{what}: token {t} matches neither pick"
 
 
-@pytest.mark.parametrize("T", [1, 4, 16])
+@pytest.mark.parametrize("T", [1, 4, 5, 6, 16])   # up to 5 tokens: row gathers; from 6: all weights streamed once
 def test_decode_llama7b_shape(T):
     w = syn.C4.with_tokens(T)
     wg, wu, wd = syn.make_weights(w)
@@ -263,9 +271,10 @@ def test_decode_llama7b_shape(T):
 
 def test_decode_with_padded_weight_arrays():
     """d_ff = 1000 in arrays of 1024 rows whose tail holds junk: the padding rows must never be selected or read as
-    channels by the decode path (bf16 decode plan and the fp32 gathered plan)."""
-    for dtype, T in (("bf16", 3), ("bf16", 16), ("f32", 2)):
-        w = syn.Workload(f"dec-pad-{dtype}-{T}", dtype, T, 128, 1000, 1024, 125, seed=640 + T)
+    channels by the decode path (bf16 decode plan at few tokens or few kept channels, the small-batch plan where most
+    channels are used, and the fp32 gathered plan)."""
+    for dtype, T, K in (("bf16", 3, 125), ("bf16", 16, 20), ("bf16", 16, 125), ("f32", 2, 125)):
+        w = syn.Workload(f"dec-pad-{dtype}-{T}-{K}", dtype, T, 128, 1000, 1024, K, seed=640 + T)
         wg, wu, wd = syn.make_weights(w)
         for m in (wg, wu, wd):
             m[w.d_ff:] = 3.0      # junk, larger than any real gate value
@@ -273,10 +282,16 @@ def test_decode_with_padded_weight_arrays():
         out = B.moc_ffn_decode(_dev(x), _dev(wg), _dev(wu), _dev(wd), w.k, d_ff=w.d_ff)
         torch.cuda.synchronize()
         x64, wg64, wu64, wd64 = map(syn.to_f64, (x, wg[:w.d_ff], wu[:w.d_ff], wd[:w.d_ff]))
-        _check_decode(syn.to_f64(out), x64, wg64, wu64, wd64, w.k, dtype, f"padded decode {dtype} T={T}")
+        _check_decode(syn.to_f64(out), x64, wg64, wu64, wd64, w.k, dtype, f"padded decode {dtype} T={T} K={K}")
 
 
-@pytest.mark.parametrize("dtype,T,d,F,K", [("f32", 3, 64, 200, 25), ("bf16", 16, 256, 1000, 125), ("bf16", 7, 520, 777, 97)])
+@pytest.mark.parametrize("dtype,T,d,F,K", [
+    ("f32", 3, 64, 200, 25),
+    ("bf16", 16, 256, 1000, 125),   # most channels used by some token: small-batch plan
+    ("bf16", 16, 512, 4096, 64),    # sixteen tokens, few kept channels: decode plan with its full batch
+    ("bf16", 5, 520, 777, 97),      # decode plan, ragged everything
+    ("bf16", 7, 520, 777, 97),      # small-batch plan below 17 tokens
+])
 def test_decode_small_shapes(dtype, T, d, F, K):
     w = syn.Workload("dec", dtype, T, d, F, F, K, seed=77, decode=True)
     wg, wu, wd = syn.make_weights(w)
