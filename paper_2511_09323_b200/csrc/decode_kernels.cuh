@@ -406,9 +406,12 @@ __device__ __forceinline__ bool cta_stage_rows(uint64_t *bar, int *abort_flag, i
 // tau must be left out (`ties_cut`; false: the set is exactly "key >= tau").
 // g == nullptr: keys[] already holds the row's fp32 values (staged by a bulk copy) and is converted in place.
 // lists0: two candidate lists of kSelListCap entries; sm: the full radix select's state (its arrays double as scratch).
+// kreg: the calling thread's keys when the row is short enough to be held in registers (F <= kSelCached * kSelThreads;
+// element i = channel tid + i * kSelThreads, 0 beyond the row), for callers that go over the row once more.
 __device__ __forceinline__ void cta_select_threshold(const float *__restrict__ g, int F, int K, uint32_t *keys,
                                                      uint32_t *lists0, SelectSmemT<kSelThreads / 32> &sm,
-                                                     uint32_t &tau_out, int &need_out, bool &ties_cut_out) {
+                                                     uint32_t &tau_out, int &need_out, bool &ties_cut_out,
+                                                     uint32_t (&kreg)[kSelCached]) {
     __shared__ uint32_t s_min[32], s_max[32], s_pick, s_above, s_inbin, s_n;
     uint32_t *lists[2] = {lists0, lists0 + kSelListCap};
     uint32_t *hist = sm.priv;  // 2048 entries
@@ -418,7 +421,6 @@ __device__ __forceinline__ void cta_select_threshold(const float *__restrict__ g
     // ---- keys, minimum and maximum.  Rows of up to kSelCached * kSelThreads channels also stay in registers (element
     // i of a thread is channel tid + i * kSelThreads): the first level's passes then run without loads.
     uint32_t kmin = 0xffffffffu, kmax = 0u;
-    uint32_t kreg[kSelCached];
     const bool cached = F <= kSelCached * kSelThreads;
     if (cached) {
 #pragma unroll
@@ -630,7 +632,8 @@ __global__ void __launch_bounds__(kSelThreads) select_mask_kernel(Workspace ws, 
     uint32_t tau;
     int need;
     bool ties_cut;
-    cta_select_threshold(nullptr, F, K, dyn, dyn + Fp, sm, tau, need, ties_cut);
+    uint32_t kreg[kSelCached];
+    cta_select_threshold(nullptr, F, K, dyn, dyn + Fp, sm, tau, need, ties_cut, kreg);
     uint32_t *my_bits = ws.sel_bits + (int64_t)t * ws.sel_words;
     const int nch = (F + kSelThreads - 1) / kSelThreads;
     if (!ties_cut) {
@@ -667,7 +670,8 @@ __global__ void __launch_bounds__(kSelThreads) cta_select_idx_kernel(const float
     uint32_t tau;
     int need;
     bool ties_cut;
-    cta_select_threshold(staged ? nullptr : g, n, k, dyn, dyn + np, sm, tau, need, ties_cut);
+    uint32_t kreg[kSelCached];
+    cta_select_threshold(staged ? nullptr : g, n, k, dyn, dyn + np, sm, tau, need, ties_cut, kreg);
     int16_t *out = idx_out + (int64_t)blockIdx.x * k;
     block_ordered_emit<kSelThreads>(dyn, n, tau, need, sm, [&](int pos, int j) { out[pos] = (int16_t)j; });
 }

@@ -315,7 +315,8 @@ __global__ void __launch_bounds__(dec::kSelThreads) sb_select_kernel(const Selec
     uint32_t tau;
     int need;
     bool ties_cut;
-    dec::cta_select_threshold(nullptr, p.F, p.K, keys, lists, sm, tau, need, ties_cut);
+    uint32_t kreg[dec::kSelCached];
+    dec::cta_select_threshold(nullptr, p.F, p.K, keys, lists, sm, tau, need, ties_cut, kreg);
     const bool save = p.idx_out != nullptr;
     const bool by_bitmap = ties_cut || save;
     if (by_bitmap) {
@@ -334,36 +335,49 @@ __global__ void __launch_bounds__(dec::kSelThreads) sb_select_kernel(const Selec
             }
         });
     }
-    // Z' row, eight channels (one 16-byte store) per thread and step.  When the triple is saved the up value is
-    // rounded to bf16 before it is used, so that the backward pass, which recomputes z from the saved pair, sees the
-    // same product.  The last group may reach into the row's padding (ldz is a multiple of 8): zeros go there.
+    // Z' row.  When the triple is saved the up value is rounded to bf16 before it is used, so that the backward pass,
+    // which recomputes z from the saved pair, sees the same product.
     __nv_bfloat16 *z = p.Z + (int64_t)t * p.ldz;
-    for (int q = tid; q * 8 < p.F; q += dec::kSelThreads) {
-        const int j0 = q * 8;
-        // (16-byte reads: the keys' array is followed by the lists, so a group that straddles F reads valid memory)
-        const uint4 ka = *reinterpret_cast<const uint4 *>(keys + j0), kb = *reinterpret_cast<const uint4 *>(keys + j0 + 4);
-        const uint32_t kk[8] = {ka.x, ka.y, ka.z, ka.w, kb.x, kb.y, kb.z, kb.w};
-        uint32_t kept = 0;
-        if (by_bitmap) {
-            kept = (bits[j0 >> 5] >> (j0 & 31)) & 0xffu;
-        } else {
+    auto z_of = [&](uint32_t key, int j) {
+        const float uv = save ? __bfloat162float(__float2bfloat16_rn(u_row[j])) : u_row[j];
+        return __float2bfloat16_rn(silu_f(key_to_float(key)) * uv);
+    };
+    if (p.F <= dec::kSelCached * dec::kSelThreads) {
+        // The thread's keys are still in registers: the row is zero-filled with 16-byte stores (into the padding up
+        // to ldz as well), then every thread drops the values of its own kept channels (one in eight) into place.
+        for (int q = tid; q * 8 < p.F; q += dec::kSelThreads) *reinterpret_cast<uint4 *>(z + q * 8) = make_uint4(0u, 0u, 0u, 0u);
+        __syncthreads();
 #pragma unroll
-            for (int e = 0; e < 8; ++e)
-                if (j0 + e < p.F && kk[e] >= tau) kept |= 1u << e;
+        for (int i = 0; i < dec::kSelCached; ++i) {
+            const int j = tid + i * dec::kSelThreads;
+            if (j < p.F) {
+                const bool kept = by_bitmap ? ((bits[j >> 5] >> (j & 31)) & 1u) != 0u : kreg[i] >= tau;
+                if (kept) z[j] = z_of(kreg[i], j);
+            }
         }
-        // only the kept channels (one in eight on average) pay for the SiLU; their bf16 values are OR-ed into place
-        uint32_t w[4] = {0u, 0u, 0u, 0u};
-        while (kept) {
-            const int e = __ffs(kept) - 1;
-            kept &= kept - 1u;
-            const float uv = save ? __bfloat162float(__float2bfloat16_rn(u_row[j0 + e])) : u_row[j0 + e];
-            const float zz = silu_f(key_to_float(keys[j0 + e])) * uv;
-            const uint32_t hbits = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(zz)) << (16 * (e & 1));
+    } else {
+        // long rows: eight channels (one 16-byte store) per thread and step
+        for (int q = tid; q * 8 < p.F; q += dec::kSelThreads) {
+            const int j0 = q * 8;
+            uint32_t kept = 0;
+            if (by_bitmap) {
+                kept = (bits[j0 >> 5] >> (j0 & 31)) & 0xffu;
+            } else {
 #pragma unroll
-            for (int q2 = 0; q2 < 4; ++q2)
-                if ((e >> 1) == q2) w[q2] |= hbits;
+                for (int e = 0; e < 8; ++e)
+                    if (j0 + e < p.F && keys[j0 + e] >= tau) kept |= 1u << e;
+            }
+            uint32_t w[4] = {0u, 0u, 0u, 0u};
+            while (kept) {
+                const int e = __ffs(kept) - 1;
+                kept &= kept - 1u;
+                const uint32_t hbits = (uint32_t)__bfloat16_as_ushort(z_of(keys[j0 + e], j0 + e)) << (16 * (e & 1));
+#pragma unroll
+                for (int q2 = 0; q2 < 4; ++q2)
+                    if ((e >> 1) == q2) w[q2] |= hbits;
+            }
+            *reinterpret_cast<uint4 *>(z + j0) = make_uint4(w[0], w[1], w[2], w[3]);
         }
-        *reinterpret_cast<uint4 *>(z + j0) = make_uint4(w[0], w[1], w[2], w[3]);
     }
 }
 

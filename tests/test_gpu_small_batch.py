@@ -72,6 +72,9 @@ def _check_against_oracle_picks(out64, x64, wg64, wu64, wd64, K, what):
     (128, 256, 520, 520, 1),       # the largest batch, a single kept channel
     (128, 136, 264, 264, 264),     # K = F: dense SwiGLU
     (40, 64, 200, 200, 199),       # all but one channel kept
+    (24, 64, 16000, 16000, 1200),  # rows longer than the selector keeps in registers
+    (20, 64, 24000, 24000, 1500),  # rows so long that the up row stays in global memory
+    (6, 64, 96, 96, 12),           # below 17 tokens the plan runs where at least half of the channels are in use
 ])
 def test_small_batch_forward_backward(T, d, F, F_ld, K):
     w = syn.Workload(f"sb-{T}-{d}-{F}-{K}", "bf16", T, d, F, F_ld, K, seed=900 + T)
