@@ -119,6 +119,20 @@ MOC_API int moc_ffn_backward(const moc_ffn_desc *desc, const void *x, const void
                              void *cuda_stream);
 
 /*
+ * The up values of the kept channels again: topk_up[t, k] = x[t, :] . w_up[topk_idx[t, k], :], rounded to the
+ * storage dtype.  For callers that keep only (topk_idx, topk_gate) between forward and backward -- the
+ * recomputation idea of Section 4 (Table 1, the "+GCP" columns) taken one step further: 2 K + K e instead of
+ * 2 K + 2 K e bytes per token are held, and the backward pass pays one more up projection (2 T d d_ffn flops on
+ * the tensor-core plan, 2 T K d on the gathered plan).  The result feeds moc_ffn_backward as topk_up.
+ *   in : x [T,d], w_up [d_ff_ld, d], topk_idx [T,k] as written by moc_ffn_forward
+ *   out: topk_up [T,k]
+ * workspace: moc_ffn_workspace_bytes(desc, MOC_OP_BACKWARD) bytes (the same buffer moc_ffn_backward takes next).
+ * A saved index outside [0, d_ff) yields 0 and is reported through moc_last_device_status().
+ */
+MOC_API int moc_ffn_recompute_up(const moc_ffn_desc *desc, const void *x, const void *w_up, const int16_t *topk_idx,
+                                 void *topk_up, void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
  * Small-batch inference (Section 5): the same forward with nothing saved, for tokens <= 128
  * (more: MOC_ERR_UNSUPPORTED; use moc_ffn_forward).  Up to 16 tokens it is organised so that only the
  * gate matrix and the selected rows of w_up / w_down are read from HBM (d d_ffn + 2 K d weight

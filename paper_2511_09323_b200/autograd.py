@@ -17,50 +17,55 @@ from . import binding as B
 
 class _MoCFFNFunction(torch.autograd.Function):
     @staticmethod
-    def forward(ctx, x, w_gate, w_up, w_down, k, d_ff, grouped):
+    def forward(ctx, x, w_gate, w_up, w_down, k, d_ff, grouped, recompute_up):
         shape = x.shape
         x2 = x.reshape(-1, shape[-1]).contiguous()
         save = any(ctx.needs_input_grad[:4])
         out, idx, tg, tu = B.moc_ffn_forward(x2, w_gate, w_up, w_down, None if k is None else int(k), d_ff=d_ff,
                                              save=save, grouped=bool(grouped))
         if save:
-            ctx.save_for_backward(x2, w_gate, w_up, w_down, idx, tg, tu)
+            # recompute_up: the up values are dropped here and formed again in backward from x, w_up and the indices
+            ctx.save_for_backward(x2, w_gate, w_up, w_down, idx, tg, *(() if recompute_up else (tu,)))
             ctx.d_ff = d_ff
             ctx.x_shape = shape
         return out.reshape(shape)
 
     @staticmethod
     def backward(ctx, grad_out):
-        x2, w_gate, w_up, w_down, idx, tg, tu = ctx.saved_tensors
+        x2, w_gate, w_up, w_down, idx, tg, *rest = ctx.saved_tensors
         names = ("x", "w_gate", "w_up", "w_down")
         want = tuple(n for n, need in zip(names, ctx.needs_input_grad[:4]) if need)
         go = grad_out.reshape(-1, grad_out.shape[-1]).contiguous()
+        tu = rest[0] if rest else B.moc_ffn_recompute_up(x2, w_up, idx, d_ff=ctx.d_ff)
         res = B.moc_ffn_backward(x2, w_gate, w_up, w_down, idx, tg, tu, go, d_ff=ctx.d_ff, want=want)
         gx = res["grad_x"]
         return (None if gx is None else gx.reshape(ctx.x_shape), res["grad_w_gate"], res["grad_w_up"],
-                res["grad_w_down"], None, None, None)
+                res["grad_w_down"], None, None, None, None)
 
 
 def moc_ffn(x: torch.Tensor, w_gate: torch.Tensor, w_up: torch.Tensor, w_down: torch.Tensor, k: int | None,
-            d_ff: int | None = None, grouped: bool = False) -> torch.Tensor:
+            d_ff: int | None = None, grouped: bool = False, recompute_up: bool = False) -> torch.Tensor:
     """out[..., :] = sum over the k channels j with the largest pre-SiLU gate value x.w_gate[j] of
     SiLU(x.w_gate[j]) * (x.w_up[j]) * w_down[j, :].  `x` is `[..., d_model]`, the weights `[d_ff_ld, d_model]` (rows at and
     past `d_ff`, when given, are padding and never selected).  grouped=True: the 2-of-8 mask of MoC 2:8 (Section 4)
-    instead of the row Top-K: the 2 largest of every 8 consecutive channels, k = d_ff / 4."""
-    return _MoCFFNFunction.apply(x, w_gate, w_up, w_down, k, d_ff, grouped)
+    instead of the row Top-K: the 2 largest of every 8 consecutive channels, k = d_ff / 4.  recompute_up=True keeps only
+    the indices and the gate values between forward and backward (k * (2 + e) instead of k * (2 + 2 e) bytes per token)
+    and pays one more up projection in backward."""
+    return _MoCFFNFunction.apply(x, w_gate, w_up, w_down, k, d_ff, grouped, recompute_up)
 
 
 class MoCFFN(torch.nn.Module):
     """SwiGLU feed-forward block with Top-K channel selection on the gate (Section 3.2)."""
 
     def __init__(self, d_model: int, d_ff: int, k: int | None, dtype=torch.bfloat16, device="cuda", init_std: float = 0.02,
-                 grouped: bool = False):
+                 grouped: bool = False, recompute_up: bool = False):
         super().__init__()
         if grouped:
             k = B._grouped_k(k, d_ff)
         if not 1 <= k <= d_ff:
             raise ValueError("k must be in [1, d_ff]")
         self.d_model, self.d_ff, self.k, self.grouped = int(d_model), int(d_ff), int(k), bool(grouped)
+        self.recompute_up = bool(recompute_up)
         mk = lambda: torch.nn.Parameter(torch.empty(d_ff, d_model, dtype=dtype, device=device))
         self.w_gate, self.w_up, self.w_down = mk(), mk(), mk()
         self.reset_parameters(init_std)
@@ -70,12 +75,13 @@ class MoCFFN(torch.nn.Module):
             torch.nn.init.normal_(p, mean=0.0, std=std)
 
     def forward(self, x: torch.Tensor) -> torch.Tensor:
-        return moc_ffn(x, self.w_gate, self.w_up, self.w_down, self.k, grouped=self.grouped)
+        return moc_ffn(x, self.w_gate, self.w_up, self.w_down, self.k, grouped=self.grouped,
+                       recompute_up=self.recompute_up)
 
     def saved_bytes_per_token(self) -> int:
         """Bytes of activations alive between forward and backward per token, besides x and the output."""
         e = torch.empty((), dtype=self.w_gate.dtype).element_size()
-        return self.k * (2 + 2 * e)
+        return self.k * (2 + (1 if self.recompute_up else 2) * e)
 
     def extra_repr(self) -> str:
         rule = "2 of every 8" if self.grouped else "row Top-K"

@@ -32,7 +32,7 @@ EXPORTED = (
     "moc_ffn_workspace_bytes", "moc_ffn_forward", "moc_ffn_backward", "moc_ffn_decode", "moc_topk_select",
     "moc_last_device_status", "moc_ffn_saved_bytes_per_token", "moc_status_string", "moc_launch_count",
     "moc_profile_enable", "moc_profile_collect", "moc_profile_kernel_count", "moc_profile_kernel_name",
-    "moc_profile_read", "moc_ffn_decode_static", "moc_tc_gemm_bf16",
+    "moc_profile_read", "moc_ffn_decode_static", "moc_tc_gemm_bf16", "moc_ffn_recompute_up",
 )
 
 
@@ -72,6 +72,8 @@ def load() -> ctypes.CDLL:
         lib.moc_ffn_backward.argtypes = [dp] + [vp] * 13 + [sz, vp]
         lib.moc_ffn_decode.restype = ctypes.c_int
         lib.moc_ffn_decode.argtypes = [dp] + [vp] * 6 + [sz, vp]
+        lib.moc_ffn_recompute_up.restype = ctypes.c_int
+        lib.moc_ffn_recompute_up.argtypes = [dp] + [vp] * 5 + [sz, vp]
         lib.moc_ffn_decode_static.restype = ctypes.c_int
         lib.moc_ffn_decode_static.argtypes = [dp] + [vp] * 5 + [vp]
         lib.moc_tc_gemm_bf16.restype = ctypes.c_int
@@ -222,6 +224,25 @@ def moc_ffn_backward(x, w_gate, w_up, w_down, topk_idx, topk_gate, topk_up, grad
     if rc != MOC_OK:
         raise MocError(rc, "moc_ffn_backward")
     return res
+
+
+def moc_ffn_recompute_up(x, w_up, topk_idx, d_ff=None, out=None, workspace=None, stream=None):
+    """topk_up [T, k] again from x, w_up and the saved indices (for callers that kept only indices and gate values).
+    `workspace`: a MOC_OP_BACKWARD workspace (the one the backward call takes next can be passed to both)."""
+    _check_dev(x, w_up, topk_idx, out, workspace)
+    T, d = x.shape
+    F_ld = w_up.shape[0]
+    k = topk_idx.shape[1]
+    desc = make_desc(T, d, F_ld if d_ff is None else d_ff, k, x.dtype, d_ff_ld=F_ld)
+    if out is None:
+        out = torch.empty((T, k), dtype=x.dtype, device=x.device)
+    if workspace is None:
+        workspace = alloc_workspace(desc, MOC_OP_BACKWARD, x.device)
+    rc = load().moc_ffn_recompute_up(ctypes.byref(desc), _ptr(x), _ptr(w_up), _ptr(topk_idx), _ptr(out),
+                                     _ptr(workspace), workspace.numel(), _stream_ptr(stream))
+    if rc != MOC_OK:
+        raise MocError(rc, "moc_ffn_recompute_up")
+    return out
 
 
 def moc_ffn_decode(x, w_gate, w_up, w_down, k, d_ff=None, out=None, workspace=None, stream=None, grouped=False):

@@ -69,6 +69,7 @@ enum KernelId {
     KID_SB_GATE_UP,
     KID_SB_SELECT,
     KID_SB_DOWN,
+    KID_RECOMPUTE_UP,
     KID_COUNT
 };
 static const char *const kKernelNames[KID_COUNT] = {
@@ -77,7 +78,7 @@ static const char *const kKernelNames[KID_COUNT] = {
     "tc_gate_up_gemm", "tc_select_mask",  "tc_down_gemm",  "tc_bwd_sample",  "tc_dz_gemm",
     "tc_wgrad_gemm",   "tc_dx_gemm",      "tc_test_gemm",  "tc_select_hint", "dec_gate_gemv",
     "dec_select",      "dec_up",          "dec_down",      "sb_gate_up",     "sb_select",
-    "sb_down",
+    "sb_down",         "recompute_up",
 };
 
 struct Profiler {
@@ -951,6 +952,60 @@ int moc_ffn_decode(const moc_ffn_desc *desc, const void *x, const void *w_gate, 
     using T = __nv_bfloat16;
     return decode_bf16(*desc, (const T *)x, (const T *)w_gate, (const T *)w_up, (const T *)w_down, (T *)out,
                        static_cast<char *>(workspace), static_cast<cudaStream_t>(cuda_stream));
+}
+
+int moc_ffn_recompute_up(const moc_ffn_desc *desc, const void *x, const void *w_up, const int16_t *topk_idx,
+                         void *topk_up, void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    int rc = check_desc(desc);
+    if (rc != MOC_OK) return rc;
+    if (desc->tokens == 0) return MOC_OK;
+    if (!good_ptr(x) || !good_ptr(w_up) || !good_ptr(topk_idx) || !good_ptr(topk_up)) return MOC_ERR_INVALID_ARG;
+    const size_t need = moc_ffn_workspace_bytes(desc, MOC_OP_BACKWARD);
+    if (need && (!good_ptr(workspace) || workspace_bytes < need)) return MOC_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    int *status = device_status_ptr();
+    if (!status) return MOC_ERR_CUDA;
+    const int64_t T = desc->tokens;
+    const int F = desc->d_ff, K = desc->k, dm = desc->d_model;
+    const int64_t total = T * K;
+    if (desc->dtype == MOC_BF16 && use_tc_plan(*desc)) {
+        // dense U = x Wu^T with the GEMM of the forward pass (same contraction order: the same bf16 values), then a gather
+        using namespace tc;
+        using B16 = __nv_bfloat16;
+        const TcBackwardLayout L = tc_backward_layout(*desc);
+        B16 *U = reinterpret_cast<B16 *>(static_cast<char *>(workspace) + L.off_z);
+        Params p;
+        init_params(p);
+        if (!map_k_major(&p.a_map[0], x, T, dm, dm, BM) || !map_k_major(&p.b_map[0], w_up, F, dm, dm, b_box_rows()))
+            return MOC_ERR_CUDA;
+        p.k_blocks = ceil_div(dm, BK);
+        p.M = (int)T;
+        p.N = F;
+        p.m_tiles = ceil_div(T, BM);
+        p.n_tiles = ceil_div(F, BN);
+        p.c[0] = U;
+        p.ldc[0] = L.ldf;
+        p.status = status;
+        MOC_LAUNCH(KID_RECOMPUTE_UP, st, (rc = launch_gemm<false, false, EPI_BF16>(p, st)));
+        if (rc != MOC_OK) return rc;
+        const unsigned grid = (unsigned)std::min<int64_t>((total + 255) / 256, 148 * 16);
+        MOC_LAUNCH(KID_RECOMPUTE_UP, st,
+                   (recompute_up_kernel<B16><<<grid, 256, 0, st>>>((const B16 *)x, (const B16 *)w_up, U, L.ldf, topk_idx, T,
+                                                                    K, F, dm, (B16 *)topk_up, status)));
+        return launch_ok();
+    }
+    const unsigned grid = (unsigned)std::min<int64_t>((total + 7) / 8, 148 * 32);
+    if (desc->dtype == MOC_BF16) {
+        using B16 = __nv_bfloat16;
+        MOC_LAUNCH(KID_RECOMPUTE_UP, st,
+                   (recompute_up_kernel<B16><<<grid, 256, 0, st>>>((const B16 *)x, (const B16 *)w_up, nullptr, 0, topk_idx,
+                                                                    T, K, F, dm, (B16 *)topk_up, status)));
+    } else {
+        MOC_LAUNCH(KID_RECOMPUTE_UP, st,
+                   (recompute_up_kernel<float><<<grid, 256, 0, st>>>((const float *)x, (const float *)w_up, nullptr, 0,
+                                                                      topk_idx, T, K, F, dm, (float *)topk_up, status)));
+    }
+    return launch_ok();
 }
 
 int moc_topk_select(int64_t rows, int32_t n, int32_t n_ld, int32_t k, const float *gate, int16_t *idx_out,

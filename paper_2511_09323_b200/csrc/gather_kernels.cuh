@@ -453,4 +453,53 @@ __global__ void __launch_bounds__(kTokenThreads) wgrad_rows_kernel(
     }
 }
 
+// ---------------------------------------------------------------------------------------------- up values again
+// topk_up[t, k] = U[t, idx[t, k]] from a dense U [T, ldu] (the tensor-core plan recomputes U with its GEMM), or, with
+// U == nullptr, the dot product x[t, :] . w_up[idx[t, k], :] itself in fp32 (one warp per kept channel).
+// An index outside [0, F) is skipped (its output is set to zero) and reported.
+template <typename T>
+__global__ void __launch_bounds__(256) recompute_up_kernel(const T *__restrict__ x, const T *__restrict__ w_up,
+                                                           const __nv_bfloat16 *__restrict__ U, int ldu,
+                                                           const int16_t *__restrict__ idx, int64_t tokens, int K, int F,
+                                                           int d, T *__restrict__ up_out, int *__restrict__ status) {
+    const int lane = threadIdx.x & 31;
+    const int64_t total = tokens * K;
+    if (U) {
+        for (int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x; i < total; i += (int64_t)gridDim.x * 256) {
+            const int64_t t = i / K;
+            const int j = idx[i];
+            if (j < 0 || j >= F) {
+                raise_status(status, MOC_ERR_BAD_INDEX);
+                up_out[i] = from_f32<T>(0.f);
+            } else {
+                up_out[i] = from_f32<T>(__bfloat162float(U[t * ldu + j]));
+            }
+        }
+        return;
+    }
+    const int64_t warps = (int64_t)gridDim.x * 8;
+    for (int64_t i = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5); i < total; i += warps) {
+        const int64_t t = i / K;
+        const int j = idx[i];
+        if (j < 0 || j >= F) {
+            if (lane == 0) {
+                raise_status(status, MOC_ERR_BAD_INDEX);
+                up_out[i] = from_f32<T>(0.f);
+            }
+            continue;
+        }
+        const T *xr = x + t * d, *wr = w_up + (int64_t)j * d;
+        float sum = 0.f;
+        for (int c = lane * 8; c < d; c += 256) {
+            float a[8], b[8];
+            Vec8<T>::load(xr + c, a);
+            Vec8<T>::load(wr + c, b);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) sum = fmaf(a[e], b[e], sum);
+        }
+        sum = warp_sum(sum);
+        if (lane == 0) up_out[i] = from_f32<T>(sum);
+    }
+}
+
 }  // namespace moc

@@ -70,3 +70,65 @@ def test_module_trains_a_step_and_skips_unneeded_gradients():
     unused = torch.ones(512, dtype=torch.bool, device="cuda")
     unused[idx.long().unique()] = False
     assert torch.all(m.w_down.grad[unused] == 0) and torch.all(m.w_up.grad[unused] == 0)
+
+
+@pytest.mark.parametrize("dtype,T,d,F,F_ld,K", [
+    ("bf16", 320, 256, 1000, 1024, 125),   # tensor-core plan: dense U with the forward's GEMM, then a gather
+    ("bf16", 40, 128, 520, 520, 65),       # a small batch: forward on the small-batch plan, up values again on the tensor cores
+    ("bf16", 5, 64, 32768, 32768, 11008),  # rows too long for the tensor-core selector: gathered plan
+    ("f32", 33, 64, 160, 160, 20),         # fp32: gathered plan
+])
+def test_recompute_up_reproduces_the_saved_up_values(dtype, T, d, F, F_ld, K):
+    """topk_up formed again from x, w_up and the saved indices: against the oracle's u on the same indices, against what
+    the forward pass saved (the same contraction on the same inputs: at most one rounding step apart), and as the
+    input of a backward pass whose gradients are checked with the recomputed values as the saved ones."""
+    w = syn.Workload(f"reup-{dtype}-{T}", dtype, T, d, F, F_ld, K, seed=4300 + T)
+    wg, wu, wd = syn.make_weights(w)
+    x, dD = syn.make_x(w), syn.make_grad_out(w)
+    xd, wgd, wud, wdd, dDd = (t.cuda() for t in (x, wg, wu, wd, dD))
+    out, idx, tg, tu = B.moc_ffn_forward(xd, wgd, wud, wdd, K, d_ff=F)
+    tu2 = B.moc_ffn_recompute_up(xd, wud, idx, d_ff=F)
+    torch.cuda.synchronize()
+    x64, wg64, wu64, wd64, dD64 = map(syn.to_f64, (x, wg[:F], wu[:F], wd[:F], dD))
+    idx_np = idx.cpu().numpy()
+    u_ref = np.einsum("td,tkd->tk", x64, wu64[idx_np.astype(np.int64)])
+    parity.assert_close(syn.to_f64(tu2), u_ref, dtype, "recomputed topk_up")
+    ulp = 2.0 ** -7 if dtype == "bf16" else 2.0 ** -20
+    a, b = syn.to_f64(tu2), syn.to_f64(tu)
+    assert np.all(np.abs(a - b) <= ulp * np.maximum(np.abs(b), 1e-3)), "recomputed and saved up values differ by more than a rounding step"
+    grads = B.moc_ffn_backward(xd, wgd, wud, wdd, idx, tg, tu2, dDd, d_ff=F)
+    gdev = {k: syn.to_f64(v) for k, v in grads.items()}
+    parity.check_backward(gdev, x64, wg64, wu64, wd64, idx_np, syn.to_f64(tg), syn.to_f64(tu2), dD64, F, dtype)
+
+
+def test_recompute_up_option_of_the_module_and_bad_indices():
+    torch.manual_seed(5)
+    m = MoCFFN(128, 512, 64, dtype=torch.bfloat16, recompute_up=True)
+    ref = MoCFFN(128, 512, 64, dtype=torch.bfloat16)
+    ref.load_state_dict(m.state_dict())
+    assert m.saved_bytes_per_token() == 64 * 4 and ref.saved_bytes_per_token() == 64 * 6
+    x = torch.randn(3, 100, 128, device="cuda", dtype=torch.bfloat16)
+    xa, xb = x.clone().requires_grad_(True), x.clone().requires_grad_(True)
+    ya, yb = m(xa), ref(xb)
+    assert torch.equal(ya, yb)
+    ya.float().pow(2).mean().backward()
+    yb.float().pow(2).mean().backward()
+    torch.testing.assert_close(xa.grad.float(), xb.grad.float(), rtol=2e-2, atol=1e-5)
+    for pa, pb in zip(m.parameters(), ref.parameters()):
+        torch.testing.assert_close(pa.grad.float(), pb.grad.float(), rtol=2e-2, atol=1e-5)
+    # an index outside [0, d_ff) yields 0 and raises the device status; the others are unaffected
+    w = syn.Workload("reup-bad", "bf16", 300, 64, 96, 96, 8, seed=12)
+    wg, wu, wd = (t.cuda() for t in syn.make_weights(w))
+    xd = syn.make_x(w).cuda()
+    _, idx, _, tu = B.moc_ffn_forward(xd, wg, wu, wd, w.k)
+    good = B.moc_ffn_recompute_up(xd, wu, idx)
+    bad = idx.clone()
+    bad[3, 2] = 96
+    bad[7, 0] = -5
+    assert B.moc_last_device_status() == B.MOC_OK
+    got = B.moc_ffn_recompute_up(xd, wu, bad)
+    assert B.moc_last_device_status() == B.MOC_ERR_BAD_INDEX
+    assert got[3, 2] == 0 and got[7, 0] == 0
+    mask = torch.ones_like(got, dtype=torch.bool)
+    mask[3, 2] = mask[7, 0] = False
+    assert torch.equal(got[mask], good[mask])
