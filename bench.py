@@ -543,7 +543,7 @@ def act_bytes_report(w, T, e, saved, B, desc):
 
 
 def decode_report(torch, B, syn, dev, peaks, calls=32, sets=4, replays=5):
-    """moc_ffn_decode on the LLaMA-7B shape for 1/4/16 tokens (the paper's decode table) and for 32/64/128 tokens
+    """moc_ffn_decode on the LLaMA-7B shape for 1/4/16 tokens (the paper's decode table) and for 32/64/128/256 tokens
     (the batch range beyond it).  One CUDA graph holds `calls` back-to-back calls that rotate through `sets`
     distinct weight sets (4 x 270 MB > L2), so every call streams its weights from HBM and launch overhead is what
     a served model would see; the graph is replayed `replays` times.  `frac` is always against the ALGORITHMIC
@@ -554,7 +554,7 @@ def decode_report(torch, B, syn, dev, peaks, calls=32, sets=4, replays=5):
     rep = {"weight_sets": sets, "calls_per_graph": calls, "replays": replays, "timing": "CUDA graph replay"}
     e = 2
     stream = torch.cuda.Stream(device=dev)
-    for T in tuple(syn.C4_BATCHES) + (32, 64, 128):
+    for T in tuple(syn.C4_BATCHES) + (32, 64, 128, 256):
         x = syn.make_x(w, tokens=T).to(dev)
         out = torch.empty_like(x)
         desc = B.make_desc(T, w.d_model, w.d_ff, w.k, x.dtype, d_ff_ld=w.d_ff_ld)

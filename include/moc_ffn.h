@@ -53,7 +53,7 @@ extern "C" {
 typedef enum {
     MOC_OK = 0,
     MOC_ERR_INVALID_ARG = -1, /* NULL/misaligned pointer, k outside [1, d_ff], negative sizes ...   */
-    MOC_ERR_UNSUPPORTED = -2, /* d_ff > 32768 (int16 indices), d_model % 8 != 0, decode tokens > 128 */
+    MOC_ERR_UNSUPPORTED = -2, /* d_ff > 32768 (int16 indices), d_model % 8 != 0, decode tokens > 256 */
     MOC_ERR_WORKSPACE = -3,   /* workspace pointer NULL or smaller than moc_ffn_workspace_bytes()    */
     MOC_ERR_CUDA = -4,        /* a CUDA runtime call or a launch failed                             */
     MOC_ERR_TIMEOUT = -5,     /* device status: a bounded wait inside a kernel expired              */
@@ -133,7 +133,7 @@ MOC_API int moc_ffn_recompute_up(const moc_ffn_desc *desc, const void *x, const 
                                  void *topk_up, void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
- * Small-batch inference (Section 5): the same forward with nothing saved, for tokens <= 128
+ * Small-batch inference (Section 5): the same forward with nothing saved, for tokens <= 256
  * (more: MOC_ERR_UNSUPPORTED; use moc_ffn_forward).  Up to 16 tokens it is organised so that only the
  * gate matrix and the selected rows of w_up / w_down are read from HBM (d d_ffn + 2 K d weight
  * elements per token instead of 3 d d_ffn).  From 17 tokens on the union of the tokens' channel sets
@@ -181,7 +181,7 @@ MOC_API int moc_ffn_decode_static(const moc_ffn_desc *desc, const void *x, const
 /*
  * The Top-K selector alone (the mask definition of Section 3.2), exposed so that it can be checked
  * bit-exactly: gate [rows, n_ld] fp32 on the device, only the first n columns of a row are channels;
- * idx_out [rows, k] int16 ascending.  Needs no workspace.  As in the plans, up to 128 rows are handled by
+ * idx_out [rows, k] int16 ascending.  Needs no workspace.  As in the plans, up to 256 rows are handled by
  * the selector that gives a whole CTA to each row (decode and small-batch plans), more rows by the
  * selector of the gathered plan; both are exact.
  */

@@ -1,4 +1,4 @@
-// Small-batch plan (bf16, 17..128 tokens): the forward as three weight-streaming kernels on tcgen05.
+// Small-batch plan (bf16, up to 256 tokens): the forward as three weight-streaming kernels on tcgen05.
 //
 // With a few dozen tokens the union of the tokens' Top-K sets covers nearly every channel
 // (1 - (1 - K/F)^T), so the row gathers of the decode plan (Section 5) no longer save bytes: the whole
@@ -34,7 +34,7 @@ constexpr int kBK = 64;         // contraction elements per stage: one 128-byte 
 constexpr int kThreads = 320;   // warp 0 TMA, warp 1 MMA + TMEM, warps 2..9 epilogue (two per TMEM lane quarter)
 constexpr int kEpiThreads = kThreads - 64;
 constexpr int kMaxStages = 10;
-constexpr int kMaxTokens = 128;
+constexpr int kMaxTokens = 256;
 constexpr int kMaxRows = 256;   // weight rows per CTA: two MMA tiles
 constexpr uint32_t kBarRegion = 256;
 constexpr size_t kSmemBudget = 224 * 1024;
@@ -54,7 +54,7 @@ inline GemmShape gemm_shape(int tokens, int weight_rows) {
     GemmShape s{};
     s.tn = (tokens + 31) & ~31;
     const int cols = s.tn * (weight_rows > kTile ? 2 : 1);
-    s.tmem_cols = cols <= 32 ? 32 : cols <= 64 ? 64 : cols <= 128 ? 128 : 256;
+    s.tmem_cols = cols <= 32 ? 32 : cols <= 64 ? 64 : cols <= 128 ? 128 : cols <= 256 ? 256 : 512;
     s.w_bytes = (uint32_t)weight_rows * kBK * 2;
     s.stage_bytes = s.w_bytes + (uint32_t)s.tn * kBK * 2;
     const size_t room = kSmemBudget - kSmemSlack - kBarRegion;
@@ -214,8 +214,9 @@ __global__ void __launch_bounds__(kThreads, 1) sb_gate_up_kernel(const __grid_co
             const int valid = min(p.rows, p.F - ch0);  // channels of this CTA inside the matrix
             // The tile goes through the (now idle) stage ring, transposed to [token][channel], and leaves as one
             // bulk store per token: 128 scalar stores per thread would add microseconds to the end of the kernel.
-            // A channel count that is not a multiple of 4 (a ragged last CTA) cannot be a bulk copy: direct stores.
-            const bool bulk = (valid & 3) == 0;
+            // A channel count that is not a multiple of 4 (a ragged last CTA) cannot be a bulk copy, and the tile of a
+            // large batch of long rows may not fit the ring: direct stores.
+            const bool bulk = (valid & 3) == 0 && (uint32_t)p.T * (uint32_t)p.rows * 4u <= (uint32_t)p.stages * p.stage_bytes;
             const uint32_t pitch = (uint32_t)p.rows * 4u;
             float *stage_f = reinterpret_cast<float *>(smem_raw + (ring.base - raw));
             // work items = (tile, 32-token chunk); the two warps of a lane quarter take alternate items
@@ -598,18 +599,25 @@ __global__ void __launch_bounds__(kThreads, 1) sb_down_kernel(const __grid_const
             asm volatile("fence.proxy.async;" ::: "memory");
             const int cols = min(kTile * p.accs, p.d - col0);  // a multiple of 8
             const uint32_t row_bytes = (uint32_t)cols * 4u;
-            if (etid == 0) tc::mbar_expect_tx(ring.extra(), row_bytes * (uint32_t)p.T);
-            asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
-            for (int t = etid; t < p.T; t += kEpiThreads)
-                tc::bulk_copy_g2s(ring.base + (uint32_t)t * row_bytes, p.acc + (int64_t)t * p.d + col0, row_bytes,
-                                  ring.extra());
-            if (__all_sync(0xffffffffu, tc::mbar_wait(ring.extra(), 0u, abort_flag, p.status))) {
-                const uint8_t *stage_ptr = smem_raw + (ring.base - raw);
-                const int vecs = cols / 4, total = p.T * vecs;
-                for (int i = etid; i < total; i += kEpiThreads) {
+            const int per_round = (int)min((uint32_t)p.T, ((uint32_t)p.stages * p.stage_bytes) / row_bytes);  // tokens the ring holds
+            const uint8_t *stage_ptr = smem_raw + (ring.base - raw);
+            const int vecs = cols / 4;
+            uint32_t parity = 0;
+            for (int t0 = 0; t0 < p.T; t0 += per_round, parity ^= 1u) {
+                const int nt = min(per_round, p.T - t0);
+                asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");  // the ring is free again
+                if (etid == 0) tc::mbar_expect_tx(ring.extra(), row_bytes * (uint32_t)nt);
+                asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
+                for (int t = etid; t < nt; t += kEpiThreads)
+                    tc::bulk_copy_g2s(ring.base + (uint32_t)t * row_bytes, p.acc + (int64_t)(t0 + t) * p.d + col0, row_bytes,
+                                      ring.extra());
+                // (after a failed wait the rounds go on, so that every warp meets the barriers above; their waits
+                //  return at once because the abort flag is set)
+                const bool landed = __all_sync(0xffffffffu, tc::mbar_wait(ring.extra(), parity, abort_flag, p.status));
+                for (int i = etid; landed && i < nt * vecs; i += kEpiThreads) {
                     const int t = i / vecs, c = (i - t * vecs) * 4;
                     const float4 v = *reinterpret_cast<const float4 *>(stage_ptr + (size_t)t * row_bytes + (size_t)c * 4);
-                    *reinterpret_cast<uint2 *>(p.out + (int64_t)t * p.d + col0 + c) =
+                    *reinterpret_cast<uint2 *>(p.out + (int64_t)(t0 + t) * p.d + col0 + c) =
                         make_uint2(tc::pack_bf16(v.x, v.y), tc::pack_bf16(v.z, v.w));
                 }
             }

@@ -50,7 +50,8 @@ def test_descriptor_validation_is_host_side(lib):
     ok = B.make_desc(256, 128, 512, 64, B.MOC_F32)
     assert B.moc_ffn_workspace_bytes(ok, B.MOC_OP_FORWARD) > 0
     assert B.moc_ffn_workspace_bytes(ok, B.MOC_OP_BACKWARD) > 0
-    assert B.moc_ffn_workspace_bytes(ok, B.MOC_OP_DECODE) == 0  # 256 tokens is not a decode batch
+    assert B.moc_ffn_workspace_bytes(ok, B.MOC_OP_DECODE) > 0   # 256 tokens: the largest decode batch
+    assert B.moc_ffn_workspace_bytes(B.make_desc(257, 128, 512, 64, B.MOC_F32), B.MOC_OP_DECODE) == 0
     assert B.moc_ffn_saved_bytes_per_token(ok) == 64 * (2 + 2 * 4)
     assert B.moc_ffn_saved_bytes_per_token(B.make_desc(1, 2048, 5504, 688, B.MOC_BF16)) == 4128
     bad = [
@@ -95,7 +96,7 @@ def test_null_pointers_and_small_workspace_are_rejected_before_launch(lib):
                                None) == B.MOC_ERR_WORKSPACE
     assert lib.moc_ffn_backward(ctypes.byref(d), *([fake] * 12), None, 0, None) == B.MOC_ERR_WORKSPACE
     # decode batch limit
-    big = B.make_desc(129, 16, 32, 4, B.MOC_BF16)
+    big = B.make_desc(257, 16, 32, 4, B.MOC_BF16)
     assert lib.moc_ffn_decode(ctypes.byref(big), fake, fake, fake, fake, fake, None, 0, None) == B.MOC_ERR_UNSUPPORTED
     # zero tokens is a no-op that needs no buffers
     zero = B.make_desc(0, 16, 32, 4, B.MOC_BF16)

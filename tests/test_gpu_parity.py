@@ -74,7 +74,7 @@ def _adversarial_rows(n):
     return np.stack(rows)
 
 
-@pytest.mark.parametrize("repeat", [1, 12])   # 11 rows: a CTA per row; 132 rows: the gathered plan's selector
+@pytest.mark.parametrize("repeat", [1, 20])   # 15 rows: a CTA per row; 300 rows: the gathered plan's selector
 @pytest.mark.parametrize("n,n_ld", [(1, 4), (37, 40), (37, 37), (256, 256), (257, 264), (2048, 2048), (5461, 5504),
                                     (11008, 11008), (32768, 32768)])
 def test_selector_bit_exact_adversarial(n, n_ld, repeat):
@@ -157,7 +157,7 @@ def test_k_equals_dff_matches_dense_swiglu_formula():
 
 
 def test_inference_forward_saves_nothing_and_matches_training_forward():
-    w = syn.Workload("inf", "bf16", 200, 128, 256, 256, 32, seed=9)
+    w = syn.Workload("inf", "bf16", 300, 128, 256, 256, 32, seed=9)
     x, wg, wu, wd, _ = map(_dev, _problem(w))
     out_a, *_ = B.moc_ffn_forward(x, wg, wu, wd, w.k, save=True)
     out_b, idx, tg, tu = B.moc_ffn_forward(x, wg, wu, wd, w.k, save=False)
@@ -223,7 +223,7 @@ def test_host_errors_raise_before_launch():
         B.moc_ffn_forward(x, wg, wu, wd, 8, workspace=torch.empty(16, dtype=torch.uint8, device="cuda"))
     assert e.value.status == B.MOC_ERR_WORKSPACE
     with pytest.raises(B.MocError) as e:
-        B.moc_ffn_decode(_dev(syn.make_x(w, tokens=129)), wg, wu, wd, 8)
+        B.moc_ffn_decode(_dev(syn.make_x(w, tokens=257)), wg, wu, wd, 8)
     assert e.value.status == B.MOC_ERR_UNSUPPORTED
     assert B.moc_last_device_status() == B.MOC_OK
 

@@ -1,4 +1,4 @@
-"""The small-batch plan (bf16, 17..128 tokens: three weight-streaming tensor-core kernels) against the oracle, through
+"""The small-batch plan (bf16, up to 256 tokens: three weight-streaming tensor-core kernels) against the oracle, through
 `moc_ffn_forward` (with and without the saved triple) and `moc_ffn_decode`."""
 import numpy as np
 import pytest
@@ -69,12 +69,16 @@ def _check_against_oracle_picks(out64, x64, wg64, wu64, wd64, K, what):
     (33, 128, 1000, 1024, 125),    # 64-token MMA with 31 empty columns
     (64, 768, 2048, 2048, 256),    # the 130M layer
     (100, 520, 777, 784, 97),      # 128-token MMA, five column blocks in the down projection, the last 8 wide
-    (128, 256, 520, 520, 1),       # the largest batch, a single kept channel
+    (128, 256, 520, 520, 1),       # a single kept channel
     (128, 136, 264, 264, 264),     # K = F: dense SwiGLU
     (40, 64, 200, 200, 199),       # all but one channel kept
     (24, 64, 16000, 16000, 1200),  # rows longer than the selector keeps in registers
     (20, 64, 24000, 24000, 1500),  # rows so long that the up row stays in global memory
     (6, 64, 96, 96, 12),           # below 17 tokens the plan runs where at least half of the channels are in use
+    (20, 8, 8, 8, 1),              # the smallest width of everything
+    (200, 264, 333, 336, 41),      # 224-token MMA
+    (256, 768, 2048, 2048, 256),   # the largest batch: 256-token MMA, all of the tensor memory
+    (256, 64, 20000, 20000, 300),  # 256 tokens x 256-channel tiles: the gate+up tile does not fit the ring (direct stores)
 ])
 def test_small_batch_forward_backward(T, d, F, F_ld, K):
     w = syn.Workload(f"sb-{T}-{d}-{F}-{K}", "bf16", T, d, F, F_ld, K, seed=900 + T)
@@ -85,7 +89,7 @@ def test_small_batch_llama1b_padded_shape_with_junk_in_the_padding_rows():
     _forward_backward(syn.C3.with_tokens(48), junk_padding=True)
 
 
-@pytest.mark.parametrize("T", [17, 64, 128])
+@pytest.mark.parametrize("T", [17, 64, 128, 256])
 def test_small_batch_decode_llama7b_shape(T):
     w = syn.C4.with_tokens(T)
     wg, wu, wd = syn.make_weights(w)
