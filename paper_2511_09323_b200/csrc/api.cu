@@ -685,7 +685,7 @@ int decode_bf16(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat
     return launch_ok();
 }
 
-// ---- small-batch plan (bf16, 17..128 tokens): three weight-streaming tcgen05 kernels ----------------------
+// ---- small-batch plan (bf16, up to 256 tokens): three weight-streaming tcgen05 kernels ----------------------
 struct SmallBatchLayout {
     int ldf, ldz;
     int rows, ctas_per_matrix;                   // gate + up: channels per CTA, CTAs per weight matrix
