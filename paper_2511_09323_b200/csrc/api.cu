@@ -614,10 +614,11 @@ DecodeLayout decode_layout(const moc_ffn_desc &d) {
 }
 
 bool use_small_batch_plan(const moc_ffn_desc &d);
+bool small_batch_preferred(const moc_ffn_desc &d);
 
 bool use_decode_plan(const moc_ffn_desc &d) {
     return d.dtype == MOC_BF16 && d.tokens >= 1 && d.tokens <= 16 && d.d_model <= 256 * dec::kSliceCols &&
-           !use_small_batch_plan(d);
+           !(use_small_batch_plan(d) && small_batch_preferred(d));
 }
 
 // Launch with programmatic stream serialization allowed: the kernel may become resident while its predecessor in
@@ -743,8 +744,10 @@ bool small_batch_preferred(const moc_ffn_desc &d) {
     return 1.0 - unused >= 0.5;
 }
 
+// moc_ffn_forward takes the small-batch plan for every bf16 batch it can serve (the tensor-core plan's tiles need
+// thousands of tokens); moc_ffn_decode takes it where small_batch_preferred says so, else the decode plan.
 bool use_small_batch_plan(const moc_ffn_desc &d) {
-    return d.dtype == MOC_BF16 && d.tokens >= 1 && d.tokens <= sb::kMaxTokens && small_batch_preferred(d) &&
+    return d.dtype == MOC_BF16 && d.tokens >= 1 && d.tokens <= sb::kMaxTokens &&
            sb::select_smem(d.d_ff, false) + 48 * 1024 <= (size_t)kMaxDynSmem;
 }
 

@@ -308,7 +308,7 @@ def test_decode_small_shapes(dtype, T, d, F, K):
 
 @pytest.mark.parametrize("T,d,F,F_ld,K", [
     (513, 264, 1100, 1104, 137),   # d not a multiple of 64, F not a multiple of 256, ragged token tile
-    (256, 128, 96, 96, 96),        # K = F: dense SwiGLU through the tensor-core plan
+    (320, 128, 96, 96, 96),        # K = F: dense SwiGLU through the tensor-core plan
     (384, 512, 4500, 4504, 563),   # more than 4096 channels: few warps per SM in the warp-per-token selector
     (257, 8, 64, 64, 1),           # smallest contraction, a single kept channel
     (300, 64, 200, 200, 199),      # all but one channel kept
