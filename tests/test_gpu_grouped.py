@@ -45,7 +45,7 @@ def _forward_backward(w: syn.Workload):
 
 @pytest.mark.parametrize("dtype,T,d,F", [
     ("bf16", 300, 128, 1024),    # tensor-core plan
-    ("bf16", 5, 64, 256),        # tensor-core plan, a handful of tokens
+    ("bf16", 5, 64, 256),        # a handful of tokens: small-batch forward, tensor-core backward
     ("f32", 40, 64, 256),        # gathered plan
 ])
 def test_grouped_forward_backward(dtype, T, d, F):
