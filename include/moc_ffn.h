@@ -31,6 +31,11 @@
  *            (a saved index outside [0, d_ff), a bounded wait that expired) make the kernel skip the
  *            offending work without touching out-of-range memory and raise a sticky per-device status
  *            word that moc_last_device_status() reports.
+ * Weights    The kernels of moc_ffn_decode, and of moc_ffn_forward for batches of up to 256 tokens, are chained with
+ *            programmatic dependent launch and start fetching WEIGHTS before they synchronise with earlier work of
+ *            the stream (activations and the workspace are touched only after that synchronisation).  Weights are
+ *            therefore expected to be settled when the call is enqueued: a kernel that writes them and itself
+ *            releases its dependents early must be followed by an event or stream synchronisation first.
  * Threads    Entry points may be called from several host threads on different streams as long as
  *            their buffers (workspace included) do not overlap.
  */
