@@ -323,6 +323,28 @@ bool use_tc_plan(const moc_ffn_desc &d) {
 
 inline int ceil_div(int64_t a, int64_t b) { return (int)((a + b - 1) / b); }
 
+// D = Z' W_down over all tokens: A = Z' [T, F] (K-major), B = Wd [F, d] (its contiguous dimension is N)
+int forward_tc_down(const moc_ffn_desc &d, const __nv_bfloat16 *Z, int ldz, const __nv_bfloat16 *wd, __nv_bfloat16 *out,
+                    int *status, cudaStream_t st) {
+    using namespace tc;
+    const int F = d.d_ff, dm = d.d_model;
+    const int64_t T = d.tokens;
+    int rc = MOC_OK;
+    Params q;
+    init_params(q);
+    if (!map_k_major(&q.a_map[0], Z, T, F, ldz, BM) || !map_mn_major(&q.b_map[0], wd, F, dm, dm)) return MOC_ERR_CUDA;
+    q.k_blocks = ceil_div(F, BK);
+    q.M = (int)T;
+    q.N = dm;
+    q.m_tiles = ceil_div(T, BM);
+    q.n_tiles = ceil_div(dm, BN);
+    q.c[0] = out;
+    q.ldc[0] = dm;
+    q.status = status;
+    MOC_LAUNCH(KID_TC_DOWN_GEMM, st, (rc = launch_gemm<false, true, EPI_BF16>(q, st)));
+    return rc;
+}
+
 int forward_tc(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat16 *wg, const __nv_bfloat16 *wu,
                const __nv_bfloat16 *wd, __nv_bfloat16 *out, int16_t *idx, __nv_bfloat16 *tg, __nv_bfloat16 *tu,
                char *ws, cudaStream_t st) {
@@ -397,6 +419,30 @@ int forward_tc(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat1
 
     int *status = device_status_ptr();
     if (!status) return MOC_ERR_CUDA;
+    if ((d.flags & MOC_FLAG_SELECT_2_OF_8) && pair_mode()) {
+        // MoC 2:8: the mask is local to groups of eight channels, so it is applied in the epilogue of one GEMM whose
+        // tiles hold the gate and the up projection of the same 128 channels side by side: Z' and the saved triple
+        // are all that reaches memory, and no selector kernel runs
+        Params q;
+        init_params(q);
+        if (!map_k_major(&q.a_map[0], x, T, dm, dm, BM) || !map_k_major(&q.b_map[0], wg, F, dm, dm, BN / 2) ||
+            !map_k_major(&q.b_map[1], wu, F, dm, dm, BN / 2))
+            return MOC_ERR_CUDA;
+        q.status = status;
+        q.k_blocks = ceil_div(dm, BK);
+        q.M = (int)T;
+        q.N = F;
+        q.m_tiles = ceil_div(T, BM);
+        q.n_tiles = ceil_div(F, BN / 2);
+        q.c[0] = U;
+        q.ldc[0] = L.ldf;
+        q.sv_idx = idx;
+        q.sv_g = idx ? tg : nullptr;
+        q.sv_u = idx ? tu : nullptr;
+        MOC_LAUNCH(KID_TC_GATE_UP_GEMM, st, (rc = launch_gemm<false, false, EPI_GATE_UP_2OF8>(q, st)));
+        if (rc != MOC_OK) return rc;
+        return forward_tc_down(d, U, L.ldf, wd, out, status, st);
+    }
     Params p;
     init_params(p);
     if (!map_k_major(&p.b_map[0], wg, F, dm, dm, b_box_rows()) || !map_k_major(&p.b_map[1], wu, F, dm, dm, b_box_rows()))
@@ -458,21 +504,7 @@ int forward_tc(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat1
         }
         if ((rc = launch_ok()) != MOC_OK) return rc;
     }
-    // D = Z' W_down over all tokens: A = Z' [T, F] (K-major), B = Wd [F, d] (its contiguous dimension is N)
-    Params q;
-    init_params(q);
-    if (!map_k_major(&q.a_map[0], U, T, F, L.ldf, BM) || !map_mn_major(&q.b_map[0], wd, F, dm, dm))
-        return MOC_ERR_CUDA;
-    q.k_blocks = ceil_div(F, BK);
-    q.M = (int)T;
-    q.N = dm;
-    q.m_tiles = ceil_div(T, BM);
-    q.n_tiles = ceil_div(dm, BN);
-    q.c[0] = out;
-    q.ldc[0] = dm;
-    q.status = status;
-    MOC_LAUNCH(KID_TC_DOWN_GEMM, st, (rc = launch_gemm<false, true, EPI_BF16>(q, st)));
-    return rc;
+    return forward_tc_down(d, U, L.ldf, wd, out, status, st);
 }
 
 int backward_tc(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat16 *wg, const __nv_bfloat16 *wu,

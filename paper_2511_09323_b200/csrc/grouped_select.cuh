@@ -13,14 +13,21 @@ constexpr int kGroup = 8, kGroupKeep = 2;
 
 // the two kept offsets of a group, ascending
 __device__ __forceinline__ void top2_of_8(const uint32_t (&key)[8], int &lo, int &hi) {
-    int i1 = 0;
+    // (the running best keys are carried in registers: indexing key[] with a run-time index would put it in local memory)
+    uint32_t k1 = key[0], k2 = 0u;
+    int i1 = 0, i2 = -1;
 #pragma unroll
     for (int e = 1; e < 8; ++e)
-        if (key[e] > key[i1]) i1 = e;  // strict: among equal keys the lowest channel stays
-    int i2 = i1 == 0 ? 1 : 0;
+        if (key[e] > k1) {  // strict: among equal keys the lowest channel stays
+            k1 = key[e];
+            i1 = e;
+        }
 #pragma unroll
     for (int e = 0; e < 8; ++e)
-        if (e != i1 && key[e] > key[i2]) i2 = e;
+        if (e != i1 && (i2 < 0 || key[e] > k2)) {
+            k2 = key[e];
+            i2 = e;
+        }
     lo = min(i1, i2);
     hi = max(i1, i2);
 }

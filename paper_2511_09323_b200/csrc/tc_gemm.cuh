@@ -24,6 +24,7 @@
 
 #include <cuda.h>
 
+#include "grouped_select.cuh"
 #include "moc_common.cuh"
 
 namespace moc {
@@ -31,6 +32,8 @@ namespace tc {
 
 constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4, ACC_STAGES = 2;
 constexpr int THREADS = 192;
+// the fused 2-of-8 epilogue is arithmetic-heavy: two epilogue warps per TMEM lane quarter there
+constexpr int pair_threads(int epi) { return epi == 3 ? 320 : THREADS; }
 constexpr uint32_t A_STAGE_BYTES = BM * BK * 2, B_STAGE_BYTES = BN * BK * 2;
 constexpr uint32_t STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
 constexpr uint32_t TMEM_COLS = ACC_STAGES * BN;  // 512
@@ -42,7 +45,13 @@ constexpr size_t SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)STAGES * STAGE_
 enum Epilogue : int {
     EPI_F32 = 0,       // C fp32 [M, ldc]
     EPI_GATE_UP = 1,   // problem 0 -> fp32 G [M, ldg]; problem 1 -> bf16 U [M, ldu]
-    EPI_BF16 = 2       // C bf16 [M, ldc]  (optionally accumulating into C)
+    EPI_BF16 = 2,      // C bf16 [M, ldc]  (optionally accumulating into C)
+    // CTA pairs only.  A tile is 256 rows x 128 CHANNELS: the pair's first CTA stages the channels' rows of b_map[0]
+    // (W_gate), the second those of b_map[1] (W_up), so the accumulator holds G in columns 0..127 and U in columns
+    // 128..255 of the same rows.  The epilogue applies the 2-of-8 mask of MoC 2:8 (Section 4) on the spot and writes
+    // the masked hidden state Z' = SiLU(G) . M . U (bf16 [M, ldc], c[0]) and the compact saved triple: no gate or up
+    // array ever reaches memory and no selector kernel runs.
+    EPI_GATE_UP_2OF8 = 3
 };
 
 struct Params {
@@ -62,6 +71,9 @@ struct Params {
     CUtensorMap c_map[3];  // per problem: [M, N] with 32-row boxes of 128 bytes (32 fp32 or 64 bf16 columns)
     int direct_store;      // 1: the output cannot be described by a tensor map; threads store their rows
     int single_cta;        // 1: one CTA per tile even where CTA pairs are available (set by the caller)
+    // EPI_GATE_UP_2OF8: compact saved activations [M, N / 4] (all three or none)
+    int16_t *sv_idx;
+    __nv_bfloat16 *sv_g, *sv_u;
     int *status;
 };
 
@@ -396,6 +408,131 @@ __device__ __forceinline__ void epilogue_tile(const Params &p, int prob, int row
     }
 }
 
+// Group G8 (channels 8 G8 .. 8 G8 + 7) of a 32-channel chunk: r = gate accumulators, q = up accumulators of one row.
+// Writes the group's four words of Z' and its two saved entries (index pair, gate pair, up pair).
+template <int G8>
+__device__ __forceinline__ void mask_group_2of8(const uint32_t (&r)[32], const uint32_t (&q)[32], uint32_t chunk_channel,
+                                                uint32_t (&zw)[16], uint32_t (&iw)[4], uint32_t (&gw)[4],
+                                                uint32_t (&uw)[4]) {
+    // the two largest gate values by plain float comparison: -0 equals +0 there as in the keys, and NaN is mapped to
+    // -inf first; strict comparisons in ascending channel order leave equal values to the lower channel
+    float g[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+        const float v = __uint_as_float(r[8 * G8 + e]);
+        g[e] = v != v ? __int_as_float(0xff800000) : v;
+    }
+    float g1 = g[0], u1 = __uint_as_float(q[8 * G8]);
+    int i1 = 0;
+#pragma unroll
+    for (int e = 1; e < 8; ++e)
+        if (g[e] > g1) {
+            g1 = g[e];
+            u1 = __uint_as_float(q[8 * G8 + e]);
+            i1 = e;
+        }
+    float g2 = 0.f, u2 = 0.f;
+    int i2 = -1;
+#pragma unroll
+    for (int e = 0; e < 8; ++e)
+        if (e != i1 && (i2 < 0 || g[e] > g2)) {
+            g2 = g[e];
+            u2 = __uint_as_float(q[8 * G8 + e]);
+            i2 = e;
+        }
+    const bool swap = i2 < i1;  // saved in ascending channel order
+    const int lo = swap ? i2 : i1, hi = swap ? i1 : i2;
+    const float glo = swap ? g2 : g1, ghi = swap ? g1 : g2, ulo = swap ? u2 : u1, uhi = swap ? u1 : u2;
+    // SiLU(g) = g / (1 + exp(-g)) with the fast exponential and reciprocal (the result is rounded to bf16 anyway);
+    // u is rounded to bf16 before the product, as it is where U goes through memory
+    const __nv_bfloat16 ub_lo = __float2bfloat16_rn(ulo), ub_hi = __float2bfloat16_rn(uhi);
+    const float z_lo = glo * __frcp_rn(1.0f + __expf(-glo)) * __bfloat162float(ub_lo);
+    const float z_hi = ghi * __frcp_rn(1.0f + __expf(-ghi)) * __bfloat162float(ub_hi);
+    const uint32_t zb_lo = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(z_lo)) << ((lo & 1) * 16);
+    const uint32_t zb_hi = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(z_hi)) << ((hi & 1) * 16);
+#pragma unroll
+    for (int wd = 0; wd < 4; ++wd)
+        zw[4 * G8 + wd] = ((lo >> 1) == wd ? zb_lo : 0u) | ((hi >> 1) == wd ? zb_hi : 0u);
+    const uint32_t chan = chunk_channel + 8u * G8;
+    iw[G8] = (chan + (uint32_t)lo) | ((chan + (uint32_t)hi) << 16);
+    gw[G8] = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(glo)) |
+             ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(ghi)) << 16);
+    uw[G8] = (uint32_t)__bfloat16_as_ushort(ub_lo) | ((uint32_t)__bfloat16_as_ushort(ub_hi) << 16);
+}
+
+// EPI_GATE_UP_2OF8: one warp's 32 rows x 128 channels of a finished accumulator (G at taddr, U 128 columns further).
+// Per group of 8 channels the 2 largest gate values are kept (ties: the lower channel; NaN as -inf); u is rounded to
+// bf16 before the product, as it is where U goes through memory, so both forms of the forward agree bit for bit.
+__device__ __forceinline__ void epilogue_tile_2of8(const Params &p, int row0, int ch0, int half, uint32_t taddr,
+                                                   uint32_t box) {
+    // `half`: which 64 channels of the tile this warp takes (two warps share a TMEM lane quarter); box: its staging box
+    const int lane = threadIdx.x & 31;
+    const int row = row0 + lane;
+    const bool row_ok = row < p.M;
+    const bool direct = p.direct_store != 0;
+    const int K = p.N >> 2;                       // kept channels per row
+    const bool vec_saves = (K & 7) == 0;          // 16-byte stores of eight saved entries need 16-byte aligned rows
+    const uint32_t my_row = (uint32_t)lane * 128u, sw = (uint32_t)(lane & 7);
+    if (row0 >= p.M || ch0 + 64 * half >= p.N) return;
+    if (!direct) {
+        if (lane == 0) bulk_store_wait_read<0>();  // the previous tile's store has read the box
+        __syncwarp();
+    }
+#pragma unroll 1
+    for (int c0 = 64 * half; c0 < 64 * half + 64 && ch0 + c0 < p.N; c0 += 32) {
+        uint32_t r[32], q[32];
+        __syncwarp();
+        tmem_ld32(taddr + (uint32_t)c0, r);
+        tmem_ld32(taddr + (uint32_t)(BN / 2 + c0), q);
+        tmem_ld_wait();
+        uint32_t zw[16];                          // 32 bf16 values of Z'
+        uint32_t iw[4], gw[4], uw[4];             // 8 saved entries each
+        mask_group_2of8<0>(r, q, (uint32_t)(ch0 + c0), zw, iw, gw, uw);
+        mask_group_2of8<1>(r, q, (uint32_t)(ch0 + c0), zw, iw, gw, uw);
+        mask_group_2of8<2>(r, q, (uint32_t)(ch0 + c0), zw, iw, gw, uw);
+        mask_group_2of8<3>(r, q, (uint32_t)(ch0 + c0), zw, iw, gw, uw);
+        const int col = ch0 + c0;
+        const int valid = p.N - col;              // channels of this chunk inside the row (a multiple of 8)
+        // ---- saved triple: slots (col / 4) .. of the row
+        if (p.sv_idx && row_ok) {
+            const int64_t o = (int64_t)row * K + (col >> 2);
+            if (vec_saves && valid >= 32) {
+                *reinterpret_cast<uint4 *>(p.sv_idx + o) = make_uint4(iw[0], iw[1], iw[2], iw[3]);
+                *reinterpret_cast<uint4 *>(p.sv_g + o) = make_uint4(gw[0], gw[1], gw[2], gw[3]);
+                *reinterpret_cast<uint4 *>(p.sv_u + o) = make_uint4(uw[0], uw[1], uw[2], uw[3]);
+            } else {
+#pragma unroll
+                for (int g8 = 0; g8 < 4; ++g8)
+                    if (8 * g8 < valid) {
+                        reinterpret_cast<uint32_t *>(p.sv_idx + o)[g8] = iw[g8];
+                        reinterpret_cast<uint32_t *>(p.sv_g + o)[g8] = gw[g8];
+                        reinterpret_cast<uint32_t *>(p.sv_u + o)[g8] = uw[g8];
+                    }
+            }
+        }
+        // ---- Z': the warp's two chunks share one 32-row x 128-byte box
+        if (direct) {
+            if (row_ok) {
+                uint32_t *dst = reinterpret_cast<uint32_t *>(static_cast<__nv_bfloat16 *>(p.c[0]) + (int64_t)row * p.ldc[0] + col);
+#pragma unroll
+                for (int i = 0; i < 16; ++i)
+                    if (2 * i < valid) dst[i] = zw[i];
+            }
+        } else {
+            const int part = (c0 >> 5) & 1;
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                st_shared_v4(box + my_row + (((uint32_t)(4 * part + i) ^ sw) << 4), zw[4 * i], zw[4 * i + 1], zw[4 * i + 2],
+                             zw[4 * i + 3]);
+            if (part == 1 || ch0 + c0 + 32 >= p.N) {  // (a lone first part at the end of the row: the rest is clipped away)
+                fence_async_smem();
+                __syncwarp();
+                if (lane == 0) tma_store_2d(&p.c_map[0], box, ch0 + 64 * half, row0);
+            }
+        }
+    }
+}
+
 // ---------------------------------------------------------------------------------------------- kernel
 template <bool A_MN, bool B_MN, int EPI>
 __global__ void __launch_bounds__(THREADS, 1) gemm_kernel(const __grid_constant__ Params p) {
@@ -592,7 +729,7 @@ constexpr uint32_t PAIR_B_STAGE_BYTES = (BN / 2) * BK * 2, PAIR_STAGE_BYTES = A_
 static_assert(PAIR_STAGES * PAIR_STAGE_BYTES == STAGES * STAGE_BYTES, "both kernels use the same shared-memory layout");
 
 template <bool A_MN, bool B_MN, int EPI>
-__global__ void __launch_bounds__(THREADS, 1) gemm_pair_kernel(const __grid_constant__ Params p) {
+__global__ void __launch_bounds__(pair_threads(EPI), 1) gemm_pair_kernel(const __grid_constant__ Params p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;  // 128-byte swizzle atoms need 1024-byte alignment
@@ -621,7 +758,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_pair_kernel(const __grid_cons
         }
         for (int a = 0; a < ACC_STAGES; ++a) {
             mbar_init(tfull_bar(a), 1);
-            mbar_init(tempty_bar(a), 8);  // one arrival per epilogue warp of the pair
+            mbar_init(tempty_bar(a), 2 * (pair_threads(EPI) / 32 - 2));  // one arrival per epilogue warp of the pair
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -659,7 +796,8 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_pair_kernel(const __grid_cons
                 int m_blk, prob, n_blk;
                 decode_tile(tile, m_blk, prob, n_blk);
                 const int m0 = m_blk * (2 * BM) + (int)rank * BM;          // this CTA's rows of A
-                const int nb0 = n_blk * BN + (int)rank * (BN / 2);         // this CTA's half of the B tile
+                // this CTA's half of the B tile (EPI_GATE_UP_2OF8: the same channels of its own weight matrix)
+                const int nb0 = EPI == EPI_GATE_UP_2OF8 ? n_blk * (BN / 2) : n_blk * BN + (int)rank * (BN / 2);
                 for (int kb = 0; kb < kb_total; ++kb) {
                     if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status)) {
                         ok = false;
@@ -667,7 +805,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_pair_kernel(const __grid_cons
                     }
                     const int seg = kb / p.k_blocks, kk = (kb - seg * p.k_blocks) * BK;
                     const CUtensorMap *am = &p.a_map[p.a_idx[prob][seg]];
-                    const CUtensorMap *bm = &p.b_map[p.b_idx[prob][seg]];
+                    const CUtensorMap *bm = &p.b_map[EPI == EPI_GATE_UP_2OF8 ? (int)rank : p.b_idx[prob][seg]];
                     const uint32_t sa = base + stage * PAIR_STAGE_BYTES, sb = sa + A_STAGE_BYTES;
                     const uint32_t lead_full = map_to_cta(full_bar(stage), 0);
                     if (rank == 0) mbar_expect_tx(full_bar(stage), 2 * PAIR_STAGE_BYTES);
@@ -742,9 +880,14 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_pair_kernel(const __grid_cons
             decode_tile(tile, m_blk, prob, n_blk);
             if (!__all_sync(0xffffffffu, mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.status))) break;
             tc_fence_after();
-            epilogue_tile<EPI>(p, prob, m_blk * (2 * BM) + (int)rank * BM + quarter * 32, n_blk * BN,
-                               tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)acc * BN,
-                               epi_base + (uint32_t)quarter * EPI_BUFS * EPI_BOX_BYTES, ebuf);
+            if (EPI == EPI_GATE_UP_2OF8)
+                epilogue_tile_2of8(p, m_blk * (2 * BM) + (int)rank * BM + quarter * 32, n_blk * (BN / 2), (warp - 2) >> 2,
+                                   tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)acc * BN,
+                                   epi_base + (uint32_t)(warp - 2) * EPI_BOX_BYTES);
+            else
+                epilogue_tile<EPI>(p, prob, m_blk * (2 * BM) + (int)rank * BM + quarter * 32, n_blk * BN,
+                                   tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)acc * BN,
+                                   epi_base + (uint32_t)quarter * EPI_BUFS * EPI_BOX_BYTES, ebuf);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(map_to_cta(tempty_bar(acc), 0));

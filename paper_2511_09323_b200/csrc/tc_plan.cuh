@@ -122,7 +122,7 @@ inline int launch_gemm(const Params &p_in, cudaStream_t st) {
         attr[0].val.clusterDim.x = 2;
         attr[0].val.clusterDim.y = 1;
         attr[0].val.clusterDim.z = 1;
-        cfg.blockDim = dim3(THREADS);
+        cfg.blockDim = dim3(pair_threads(EPI));
         cfg.dynamicSmemBytes = SMEM_BYTES;
         cfg.stream = st;
         cfg.attrs = attr;

@@ -44,7 +44,8 @@ def _forward_backward(w: syn.Workload):
 
 
 @pytest.mark.parametrize("dtype,T,d,F", [
-    ("bf16", 300, 128, 1024),    # tensor-core plan
+    ("bf16", 300, 128, 1024),    # tensor-core plan: the mask fused into the gate+up GEMM's epilogue
+    ("bf16", 700, 264, 1000),    # the same with ragged tiles: 125 groups, the last channel tile 104 wide, K = 250
     ("bf16", 5, 64, 256),        # a handful of tokens: small-batch forward, tensor-core backward
     ("f32", 40, 64, 256),        # gathered plan
 ])
@@ -100,3 +101,18 @@ def test_grouped_argument_rules_and_module():
     y = m(torch.randn(2, 7, 64, device="cuda", dtype=torch.bfloat16))
     y.float().sum().backward()
     assert m.w_down.grad is not None and torch.isfinite(m.w_down.grad.float()).all()
+
+
+def test_grouped_forward_without_cta_pairs():
+    """MOC_FFN_GEMM=single (read once per process): without CTA pairs the 2-of-8 mask is not fused into the gate+up
+    GEMM's epilogue; the GEMM writes G and U and a kernel with one thread per group applies the mask.  Run the
+    tensor-core cases again in a child process with it set."""
+    import os
+    import subprocess
+    import sys
+    env = dict(os.environ, MOC_FFN_GEMM="single")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    r = subprocess.run([sys.executable, "-m", "pytest", os.path.join(root, "tests", "test_gpu_grouped.py"), "-q", "-x",
+                        "-m", "gpu", "-k", "grouped_forward_backward or ties_keep"],
+                       cwd=root, env=env, capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
