@@ -460,6 +460,12 @@ def run_ours(args):
             "act_bytes": act_bytes_report(w, T, e, saved, B, desc),
             "strict_roofline": strict_roofline(w, T, e, worst_ms / args.steps, peaks),
         }
+    # ---- the MoC 2:8 variant on the same layer (rank 0; extra information, not the headline) ---------
+    if rank == 0 and not args.no_decode and w.dtype == "bf16" and w.d_ff % 8 == 0:
+        try:
+            line["moc_2of8"] = grouped_report(torch, B, x, dD, wg, wu, wd, flush, args.steps)
+        except Exception as exc:
+            line["moc_2of8"] = {"error": repr(exc)}
     # ---- decode (rank 0, after the training timing) ----------------------------------------------
     if rank == 0 and not args.no_decode:
         del flush, ws_f, ws_b
@@ -540,6 +546,28 @@ def act_bytes_report(w, T, e, saved, B, desc):
     return {"moc_saved_per_token": B.moc_ffn_saved_bytes_per_token(desc), "measured_saved_total": measured,
             "measured_saved_per_token": measured / T, "dense_swiglu_per_token": 4 * w.d_ff * e,
             "dense_gcp_per_token": 2 * w.d_ff * e, "x_and_out_per_token_each": w.d_model * e}
+
+
+def grouped_report(torch, B, x, dD, wg, wu, wd, flush, steps):
+    """Forward + backward with the 2-of-8 mask (MoC 2:8: K = d_ff / 4, the mask applied in the gate+up GEMM's
+    epilogue) on the bench workload's tensors; same timing rules as the headline (L2 flushed between steps, CUDA
+    events around each step)."""
+    T, F = x.shape[0], wg.shape[0]
+    for _ in range(3):
+        out, idx, tg, tu = B.moc_ffn_forward(x, wg, wu, wd, None, grouped=True)
+        B.moc_ffn_backward(x, wg, wu, wd, idx, tg, tu, dD)
+    torch.cuda.synchronize()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    grads = None
+    for s, t in ev:
+        flush.zero_()
+        s.record()
+        out, idx, tg, tu = B.moc_ffn_forward(x, wg, wu, wd, None, grouped=True)
+        grads = B.moc_ffn_backward(x, wg, wu, wd, idx, tg, tu, dD, grads=grads)
+        t.record()
+    torch.cuda.synchronize()
+    ms = sum(s.elapsed_time(t) for s, t in ev) / steps
+    return {"k": F // 4, "ms_per_step": ms, "tokens_per_s": T / (ms / 1e3), "launch": "direct calls"}
 
 
 def decode_report(torch, B, syn, dev, peaks, calls=32, sets=4, replays=5):
