@@ -116,3 +116,40 @@ def test_grouped_forward_without_cta_pairs():
                         "-m", "gpu", "-k", "grouped_forward_backward or ties_keep"],
                        cwd=root, env=env, capture_output=True, text=True, timeout=600)
     assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
+
+
+def test_grouped_full_size_bench_layer_sampled_against_oracle():
+    """The 2-of-8 mask on C2's layer at its full 16384 tokens (the configuration bench.py's `moc_2of8` line times): picks of
+    sampled tokens per group, their out / saved values / grad_x and sampled rows of the weight gradients against the
+    oracle; the slot layout of every token."""
+    import dataclasses
+    w = dataclasses.replace(syn.C2, k=syn.C2.d_ff // 4, name="C2-2of8")
+    wg, wu, wd = syn.make_weights(w)
+    x, dD = syn.make_x(w), syn.make_grad_out(w)
+    xd, wgd, wud, wdd, dDd = (t.cuda() for t in (x, wg, wu, wd, dD))
+    out, idx, tg, tu = B.moc_ffn_forward(xd, wgd, wud, wdd, None, grouped=True)
+    grads = B.moc_ffn_backward(xd, wgd, wud, wdd, idx, tg, tu, dDd)
+    torch.cuda.synchronize()
+    assert B.moc_last_device_status() == B.MOC_OK
+    idx_np = idx.cpu().numpy().astype(np.int64)
+    slots = np.arange(w.k)
+    assert np.all(idx_np // 8 == slots // 2), "slot 2q, 2q+1 must hold channels of group q"
+    assert np.all(idx_np[:, 0::2] < idx_np[:, 1::2])
+    rng = np.random.default_rng(0)
+    toks = np.sort(rng.choice(w.tokens, 96, replace=False))
+    wg64, wu64, wd64 = map(syn.to_f64, (wg, wu, wd))
+    x64s, dD64s = syn.to_f64(x[toks]), syn.to_f64(dD[toks])
+    parity.check_picks_grouped(idx_np[toks], orc.gate_projection(x64s, wg64))
+    ref = orc.forward_given_idx(x64s, wg64, wu64, wd64, idx_np[toks].astype(np.int32))
+    parity.assert_close(syn.to_f64(out[toks]), ref["out"], "bf16", "out")
+    parity.assert_close(syn.to_f64(tg[toks]), ref["gval"], "bf16", "topk_gate")
+    parity.assert_close(syn.to_f64(tu[toks]), ref["uval"], "bf16", "topk_up")
+    rb = orc.backward(x64s, wg64, wu64, wd64, idx_np[toks].astype(np.int32), syn.to_f64(tg[toks]), syn.to_f64(tu[toks]),
+                      dD64s, F=w.d_ff, want=("x",))
+    parity.assert_close(syn.to_f64(grads["grad_x"][toks]), rb["grad_x"], "bf16", "grad_x (sampled tokens)")
+    rows = np.sort(rng.choice(w.d_ff, 16, replace=False)).astype(np.int32)
+    wrows = orc.backward_weight_rows(syn.to_f64(x), wd64, idx_np.astype(np.int32), syn.to_f64(tg), syn.to_f64(tu),
+                                     syn.to_f64(dD), rows, w.d_ff)
+    for name in ("grad_w_gate", "grad_w_up", "grad_w_down"):
+        got = syn.to_f64(grads[name][torch.from_numpy(rows.astype(np.int64)).cuda()])
+        parity.assert_close(got, wrows[name], "bf16", name + " (sampled rows)")
