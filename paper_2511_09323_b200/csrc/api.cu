@@ -507,6 +507,9 @@ int forward_tc(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat1
     return forward_tc_down(d, U, L.ldf, wd, out, status, st);
 }
 
+int small_batch_dx(const moc_ffn_desc &d, const __nv_bfloat16 *dG, const __nv_bfloat16 *dU, int ldf,
+                   const __nv_bfloat16 *wg, const __nv_bfloat16 *wu, __nv_bfloat16 *gx, char *small, cudaStream_t st);
+
 int backward_tc(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat16 *wg, const __nv_bfloat16 *wu,
                 const __nv_bfloat16 *wd, const int16_t *idx, const __nv_bfloat16 *tg, const __nv_bfloat16 *tu,
                 const __nv_bfloat16 *dout, __nv_bfloat16 *gx, __nv_bfloat16 *gwg, __nv_bfloat16 *gwu,
@@ -595,7 +598,11 @@ int backward_tc(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat
         if (rc != MOC_OK) return rc;
     }
     // dX = dG' Wg + dU' Wu   (Eq. (bp-5)): one accumulator, two contraction segments
-    if (gx) {
+    if (gx && L.small_bytes) {
+        // a small batch: the weight-streaming kernel of the small-batch plan (a 256-row tile of tokens would leave
+        // most SMs without work: d_model / 256 tiles in all)
+        if ((rc = small_batch_dx(d, dGp, dUp, L.ldf, wg, wu, gx, ws + L.off_small, st)) != MOC_OK) return rc;
+    } else if (gx) {
         Params p;
         init_params(p);
         if (!map_k_major(&p.a_map[0], dGp, T, F, L.ldf, BM) || !map_k_major(&p.a_map[1], dUp, T, F, L.ldf, BM) ||
@@ -727,6 +734,23 @@ struct SmallBatchLayout {
     size_t off_g, off_u, off_z, off_acc, off_cnt, total;
 };
 
+// Grid of sb_down_kernel for `d_model` output columns and `k_blocks` channel blocks in all: about one CTA per SM,
+// every CTA at least one channel block; 256-column blocks (accs = 2) when they still fill the GPU, else 128.
+void down_geometry(int d_model, int k_blocks, int &accs, int &m_tiles, int &splits) {
+    const int sms = tc::sm_count();
+    auto ctas = [&](int a, int &mt, int &sp) {
+        mt = (d_model + sb::kTile * a - 1) / (sb::kTile * a);
+        sp = std::max(1, std::min(sms / mt, k_blocks));
+        return mt * sp;
+    };
+    int m1, s1, m2, s2;
+    const int c1 = ctas(1, m1, s1), c2 = ctas(2, m2, s2);
+    const bool wide = d_model > sb::kTile && (c2 >= c1 || 20 * c2 >= 17 * sms);
+    accs = wide ? 2 : 1;
+    m_tiles = wide ? m2 : m1;
+    splits = wide ? s2 : s1;
+}
+
 SmallBatchLayout small_batch_layout(const moc_ffn_desc &d) {
     SmallBatchLayout L{};
     const int sms = tc::sm_count();
@@ -736,19 +760,8 @@ SmallBatchLayout small_batch_layout(const moc_ffn_desc &d) {
     const int per = std::max(1, sms / 2);
     L.rows = std::min(sb::kMaxRows, std::max(8, (((d.d_ff + per - 1) / per) + 7) & ~7));
     L.ctas_per_matrix = (d.d_ff + L.rows - 1) / L.rows;
-    // down: about one CTA per SM, every CTA at least one channel block; wide column blocks when they still fill the GPU
     L.k_blocks_down = (d.d_ff + sb::kBK - 1) / sb::kBK;
-    auto ctas = [&](int accs, int &m_tiles, int &splits) {
-        m_tiles = (d.d_model + sb::kTile * accs - 1) / (sb::kTile * accs);
-        splits = std::max(1, std::min(sms / m_tiles, L.k_blocks_down));
-        return m_tiles * splits;
-    };
-    int m1, s1, m2, s2;
-    const int c1 = ctas(1, m1, s1), c2 = ctas(2, m2, s2);
-    const bool wide = d.d_model > sb::kTile && (c2 >= c1 || 20 * c2 >= 17 * sms);
-    L.accs = wide ? 2 : 1;
-    L.m_tiles = wide ? m2 : m1;
-    L.splits = wide ? s2 : s1;
+    down_geometry(d.d_model, L.k_blocks_down, L.accs, L.m_tiles, L.splits);
     L.stage_u = sb::select_smem(d.d_ff, true) + 48 * 1024 <= (size_t)kMaxDynSmem;
     Carver c;
     L.off_g = c.take((size_t)d.tokens * L.ldf * sizeof(float));
@@ -839,9 +852,10 @@ int forward_small_batch(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __n
 
     sb::DownParams dp;
     memset(&dp, 0, sizeof(dp));
-    if (!tc::make_map(&dp.wd_map, wd, F, dm, dm, 64, sb::kBK) ||
-        !tc::make_map(&dp.z_map, Z, T, F, L.ldz, sb::kBK, ds.tn))
+    if (!tc::make_map(&dp.wd_map[0], wd, F, dm, dm, 64, sb::kBK) ||
+        !tc::make_map(&dp.z_map[0], Z, T, F, L.ldz, sb::kBK, ds.tn))
         return MOC_ERR_CUDA;
+    dp.segments = 1;
     dp.T = T;
     dp.tn = ds.tn;
     dp.tmem_cols = ds.tmem_cols;
@@ -859,6 +873,50 @@ int forward_small_batch(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __n
     dp.status = status;
     MOC_LAUNCH(KID_SB_DOWN, st,
                launch_pdl(sb::sb_down_kernel, dim3(L.m_tiles * L.splits), sb::kThreads, ds.smem, st, dp));
+    return launch_ok();
+}
+
+// dX = dG' Wg + dU' Wu for a small batch with sb_down_kernel: two contraction segments into one accumulator.
+// `small`: T * d floats (the accumulator) followed by the column blocks' counters; both are cleared here.
+int small_batch_dx(const moc_ffn_desc &d, const __nv_bfloat16 *dG, const __nv_bfloat16 *dU, int ldf,
+                   const __nv_bfloat16 *wg, const __nv_bfloat16 *wu, __nv_bfloat16 *gx, char *small, cudaStream_t st) {
+    const int T = (int)d.tokens, F = d.d_ff, dm = d.d_model;
+    int *status = device_status_ptr();
+    if (!status) return MOC_ERR_CUDA;
+    const size_t acc_bytes = (size_t)T * dm * sizeof(float);
+    float *acc = reinterpret_cast<float *>(small);
+    int *counters = reinterpret_cast<int *>(small + acc_bytes);
+    const int k_blocks = (F + sb::kBK - 1) / sb::kBK;
+    int accs, m_tiles, splits;
+    down_geometry(dm, 2 * k_blocks, accs, m_tiles, splits);
+    if ((size_t)m_tiles * sizeof(int) > 1024) return MOC_ERR_UNSUPPORTED;
+    const sb::GemmShape ds = sb::gemm_shape(T, sb::kTile * accs);
+    if (ds.stages < 2) return MOC_ERR_UNSUPPORTED;
+    int rc;
+    if ((rc = set_smem(sb::sb_down_kernel, ds.smem, 1024)) != MOC_OK) return rc;
+    if (cudaMemsetAsync(small, 0, acc_bytes + (size_t)m_tiles * sizeof(int), st) != cudaSuccess) return MOC_ERR_CUDA;
+    sb::DownParams dp;
+    memset(&dp, 0, sizeof(dp));
+    if (!tc::make_map(&dp.wd_map[0], wg, F, dm, dm, 64, sb::kBK) || !tc::make_map(&dp.wd_map[1], wu, F, dm, dm, 64, sb::kBK) ||
+        !tc::make_map(&dp.z_map[0], dG, T, F, ldf, sb::kBK, ds.tn) || !tc::make_map(&dp.z_map[1], dU, T, F, ldf, sb::kBK, ds.tn))
+        return MOC_ERR_CUDA;
+    dp.segments = 2;
+    dp.T = T;
+    dp.tn = ds.tn;
+    dp.tmem_cols = ds.tmem_cols;
+    dp.stages = ds.stages;
+    dp.w_bytes = ds.w_bytes;
+    dp.stage_bytes = ds.stage_bytes;
+    dp.d = dm;
+    dp.k_blocks = k_blocks;
+    dp.m_tiles = m_tiles;
+    dp.splits = splits;
+    dp.accs = accs;
+    dp.acc = acc;
+    dp.out = gx;
+    dp.counters = counters;
+    dp.status = status;
+    MOC_LAUNCH(KID_TC_DX_GEMM, st, (sb::sb_down_kernel<<<m_tiles * splits, sb::kThreads, ds.smem, st>>>(dp)));
     return launch_ok();
 }
 

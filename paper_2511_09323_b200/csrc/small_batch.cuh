@@ -77,11 +77,15 @@ struct GateUpParams {
 };
 
 struct DownParams {
-    CUtensorMap wd_map;  // W_down [F, d] read as the M-major operand: boxes of 64 channels x 64 columns
-    CUtensorMap z_map;   // Z' [T, F], boxes of tn rows x 64 channels
+    // One or two contraction segments, each a weight matrix [F, d] read as the M-major operand (boxes of 64 channels x
+    // 64 columns) and an activation array [T, F] (boxes of tn rows x 64 channels): the forward's D = Z' Wd has one,
+    // the backward's dX = dG' Wg + dU' Wu (Eq. (bp-5)) two that add into the same accumulator.
+    CUtensorMap wd_map[2];
+    CUtensorMap z_map[2];
+    int segments;
     int T, tn, tmem_cols, stages;
     uint32_t w_bytes, stage_bytes;
-    int d, k_blocks, m_tiles, splits;
+    int d, k_blocks, m_tiles, splits;  // k_blocks: channel blocks of ONE segment; the splits share segments * k_blocks
     int accs;            // 1 or 2: the CTA owns 128 * accs output columns
     float *acc;          // [T, d] fp32, zero on entry
     __nv_bfloat16 *out;  // [T, d]
@@ -452,16 +456,22 @@ __global__ void __launch_bounds__(kThreads, 1) sb_down_kernel(const __grid_const
     tc::pdl_launch_dependents();
 
     const int m_blk = (int)blockIdx.x / p.splits, split = (int)blockIdx.x - m_blk * p.splits;
-    const int kb0 = (int)(((int64_t)split * p.k_blocks) / p.splits);
-    const int kb1 = (int)(((int64_t)(split + 1) * p.k_blocks) / p.splits);
+    const int kb_all = p.k_blocks * p.segments;
+    const int kb0 = (int)(((int64_t)split * kb_all) / p.splits);
+    const int kb1 = (int)(((int64_t)(split + 1) * kb_all) / p.splits);
     const int nkb = kb1 - kb0;  // >= 1: the host keeps splits <= k_blocks
     const int col0 = m_blk * kTile * p.accs;
     const int ahead = min(p.stages, nkb);
     auto load_w = [&](int stage, int kb) {
         // boxes of 64 columns x 64 channels, 8 KiB each: the M-major operand layout, two boxes per MMA tile
+        const int sg = kb >= p.k_blocks ? 1 : 0;
         for (int b = 0; b < 2 * p.accs; ++b)
-            tc::tma_load_2d(ring.stage(stage) + (uint32_t)b * (64 * kBK * 2), &p.wd_map, ring.full(stage), col0 + 64 * b,
-                            kb * kBK);
+            tc::tma_load_2d(ring.stage(stage) + (uint32_t)b * (64 * kBK * 2), &p.wd_map[sg], ring.full(stage), col0 + 64 * b,
+                            (kb - sg * p.k_blocks) * kBK);
+    };
+    auto load_z = [&](int stage, int kb) {
+        const int sg = kb >= p.k_blocks ? 1 : 0;
+        tc::tma_load_2d(ring.stage(stage) + p.w_bytes, &p.z_map[sg], ring.full(stage), (kb - sg * p.k_blocks) * kBK, 0);
     };
 
     if (threadIdx.x == 0) {
@@ -491,15 +501,14 @@ __global__ void __launch_bounds__(kThreads, 1) sb_down_kernel(const __grid_const
     if (warp == 0) {
         if (lane == 0) {
             tc::pdl_wait();  // Z' comes from the select kernel
-            for (int i = 0; i < ahead; ++i)
-                tc::tma_load_2d(ring.stage(i) + p.w_bytes, &p.z_map, ring.full(i), (kb0 + i) * kBK, 0);
+            for (int i = 0; i < ahead; ++i) load_z(i, kb0 + i);
             int stage = 0;
             uint32_t phase = 1;
             for (int i = ahead; i < nkb; ++i) {
                 if (!tc::mbar_wait(ring.empty(stage), phase ^ 1u, abort_flag, p.status)) break;
                 tc::mbar_expect_tx(ring.full(stage), p.stage_bytes);
                 load_w(stage, kb0 + i);
-                tc::tma_load_2d(ring.stage(stage) + p.w_bytes, &p.z_map, ring.full(stage), (kb0 + i) * kBK, 0);
+                load_z(stage, kb0 + i);
                 if (++stage == p.stages) {
                     stage = 0;
                     phase ^= 1u;

@@ -954,6 +954,7 @@ struct TcForwardLayout {
 struct TcBackwardLayout {
     int ldf;
     size_t off_z, off_du, off_dg, total;  // three dense bf16 [T, ldf] arrays
+    size_t off_small, small_bytes;        // batches of up to 256 tokens: fp32 accumulator [T, d] + counters of the dX kernel
 };
 
 inline int round_up8(int v) { return (v + 7) & ~7; }
@@ -999,6 +1000,9 @@ inline TcBackwardLayout tc_backward_layout(const moc_ffn_desc &d) {
     off += dense;
     L.off_dg = off;
     off += dense;
+    L.off_small = off;
+    L.small_bytes = d.tokens <= 256 ? align_up((size_t)d.tokens * d.d_model * sizeof(float) + 1024, 256) : 0;
+    off += L.small_bytes;
     L.total = off;
     return L;
 }
