@@ -164,6 +164,9 @@ MOC_API int moc_ffn_decode(const moc_ffn_desc *desc, const void *x, const void *
  * library image, MOC_STATIC_SCRATCH_BYTES long.  Every GPU that loads the library holds that array
  * from load until the process exits, whether or not this entry point is ever called.
  *
+ * Kernels bf16 problems whose decode-plan buffers fit the array (the LLaMA-7B layer at 16 tokens does) run the
+ *         same HBM-streaming kernels as moc_ffn_decode with its decode plan; everything else the limits admit
+ *         runs the exact gathered kernels (correct, but milliseconds rather than tens of microseconds).
  * Limits  tokens <= MOC_STATIC_MAX_TOKENS and d_ff <= MOC_STATIC_MAX_DFF; anything larger returns
  *         MOC_ERR_STATIC_LIMIT and launches nothing (use moc_ffn_decode with a workspace instead).
  *         All other argument rules are those of moc_ffn_decode.

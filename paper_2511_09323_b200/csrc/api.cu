@@ -1155,11 +1155,19 @@ int moc_ffn_decode_static(const moc_ffn_desc *desc, const void *x, const void *w
     if (desc->tokens == 0) return MOC_OK;
     if (!good_ptr(x) || !good_ptr(w_gate) || !good_ptr(w_up) || !good_ptr(w_down) || !good_ptr(out))
         return MOC_ERR_INVALID_ARG;
-    // same carving as the workspace variant; the limits above bound it by the array's size
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    // bf16: the decode plan's kernels whenever their workspace fits the array (the LLaMA-7B layer does at 16 tokens)
+    if (desc->dtype == MOC_BF16 && desc->d_model <= 256 * dec::kSliceCols &&
+        decode_layout(*desc).total <= MOC_STATIC_SCRATCH_BYTES) {
+        char *wsd = static_scratch_ptr();
+        if (!wsd) return MOC_ERR_CUDA;
+        using T = __nv_bfloat16;
+        return decode_bf16(*desc, (const T *)x, (const T *)w_gate, (const T *)w_up, (const T *)w_down, (T *)out, wsd, st);
+    }
+    // otherwise the gathered kernels: same carving as the workspace variant; the limits above bound it by the array's size
     if (plan_forward(*desc).total > MOC_STATIC_SCRATCH_BYTES) return MOC_ERR_STATIC_LIMIT;
     char *ws = static_scratch_ptr();
     if (!ws) return MOC_ERR_CUDA;
-    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     if (desc->dtype == MOC_BF16) {
         using T = __nv_bfloat16;
         return forward_gather<T>(*desc, (const T *)x, (const T *)w_gate, (const T *)w_up, (const T *)w_down,

@@ -55,11 +55,19 @@ def test_static_decode_matches_workspace_decode_twice_in_a_row(dtype):
     assert B.moc_last_device_status() == B.MOC_OK
 
 
-def test_static_decode_llama7b_shape():
-    w = syn.C4.with_tokens(4)
+@pytest.mark.parametrize("T", [4, 16])
+def test_static_decode_llama7b_shape(T):
+    """The LLaMA-7B layer: the decode plan's transient buffers fit the built-in array at every batch up to 16, so the
+    call runs the decode plan's kernels (also where moc_ffn_decode itself prefers the small-batch plan)."""
+    w = syn.C4.with_tokens(T)
     wg, wu, wd = (t.cuda() for t in syn.make_weights(w))
     x = syn.make_x(w).cuda()
     _compare(w, x, wg, wu, wd)
+
+
+def test_static_decode_falls_back_to_the_gathered_kernels_when_the_decode_plan_does_not_fit():
+    """16 tokens on a 16384-channel layer: the decode plan's buffers exceed the built-in array, the gathered plan's do not."""
+    _compare(*_case("bf16", 16, 2048, 16384, 16384, 2048, seed=33))
 
 
 def test_static_decode_rejects_what_does_not_fit():
