@@ -13,7 +13,8 @@
 //                          as a dense bf16 row; optionally the compact saved triple; zeroes the output accumulator
 //   3. sb_down_kernel      D^T [column, token] = Wd^T Z'^T; a CTA owns 128 or 256 output columns and a share of
 //                          the channels; partial sums meet in an fp32 accumulator (16-byte red.add), the last CTA of a
-//                          column block rounds to bf16
+//                          column block rounds to bf16.  The backward of a small batch uses the same kernel for
+//                          grad_x = dG' Wg + dU' Wu (Eq. (bp-5)): two contraction segments into one accumulator
 //
 // One CTA per SM with the deepest ring of stages shared memory allows: the bytes in flight set the pace.
 // The kernels are chained with programmatic dependent launch: weights stream before the dependency
