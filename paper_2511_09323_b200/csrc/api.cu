@@ -11,6 +11,7 @@
 #include <unordered_map>
 #include <vector>
 
+#include "decode_coop.cuh"
 #include "decode_kernels.cuh"
 #include "gather_kernels.cuh"
 #include "grouped_select.cuh"
@@ -70,6 +71,7 @@ enum KernelId {
     KID_SB_SELECT,
     KID_SB_DOWN,
     KID_RECOMPUTE_UP,
+    KID_DEC_COOP,
     KID_COUNT
 };
 static const char *const kKernelNames[KID_COUNT] = {
@@ -78,7 +80,7 @@ static const char *const kKernelNames[KID_COUNT] = {
     "tc_gate_up_gemm", "tc_select_mask",  "tc_down_gemm",  "tc_bwd_sample",  "tc_dz_gemm",
     "tc_wgrad_gemm",   "tc_dx_gemm",      "tc_test_gemm",  "tc_select_hint", "dec_gate_gemv",
     "dec_select",      "dec_up",          "dec_down",      "sb_gate_up",     "sb_select",
-    "sb_down",         "recompute_up",
+    "sb_down",         "recompute_up",    "dec_coop",
 };
 
 struct Profiler {
@@ -677,6 +679,106 @@ cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, unsigned block, size_t
     return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
 }
 
+// ---- cooperative decode (bf16, one or two tokens, d_model <= 4096): one kernel, every SM keeps its channels ----
+struct CoopLayout {
+    int grid, unit, stages;
+    size_t smem, off_hist, off_n, off_cand, off_acc, total;
+};
+
+// ok == false: the problem or the device does not admit the cooperative kernel (the four-kernel plan runs then)
+CoopLayout coop_layout(const moc_ffn_desc &d, bool &ok) {
+    CoopLayout L{};
+    ok = false;
+    static const bool off = [] {
+        const char *e = getenv("MOC_FFN_DECODE");  // "chain": the four-kernel decode plan (comparisons, tests)
+        return e && strcmp(e, "chain") == 0;
+    }();
+    if (off || d.dtype != MOC_BF16 || d.tokens < 1 || d.tokens > dc::kMaxTokens || d.d_model > dc::kMaxD) return L;
+    static const int coop_ok = [] {
+        int dev = 0, v = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess) return 0;
+        return v;
+    }();
+    if (!coop_ok) return L;
+    const int T = (int)d.tokens, dm = d.d_model, F = d.d_ff;
+    L.unit = (F % 8 == 0) ? 8 : 1;
+    if ((d.flags & MOC_FLAG_SELECT_2_OF_8) && L.unit != 8) return L;
+    const int units = (F + L.unit - 1) / L.unit;
+    L.grid = std::min(tc::sm_count(), units);
+    if (((units + L.grid - 1) / L.grid) * L.unit > dc::kMaxRows) return L;
+    const size_t fixed = (size_t)T * dm * 2 + (size_t)2 * T * dc::kMaxRows * 4;
+    const size_t budget = (size_t)216 * 1024;
+    if (fixed + (size_t)4 * dm * 2 > budget) return L;
+    L.stages = (int)std::min<size_t>(dc::kMaxStages, (budget - fixed) / ((size_t)dm * 2));
+    L.smem = dc::smem_bytes(T, dm, L.stages);
+    Carver c;
+    L.off_hist = c.take((size_t)T * dc::kBins * sizeof(uint32_t));
+    L.off_n = c.take((size_t)T * sizeof(uint32_t));
+    L.off_cand = c.take((size_t)T * F * sizeof(uint2));
+    L.off_acc = c.take((size_t)T * dm * sizeof(float));
+    L.total = c.off;
+    ok = true;
+    return L;
+}
+
+template <int T>
+int launch_coop(const dc::Params &prm, const CoopLayout &L, cudaStream_t st) {
+    auto kern = dc::decode_coop_kernel<T>;
+    int rc;
+    if ((rc = set_smem(kern, L.smem, 8 * 1024)) != MOC_OK) return rc;
+    // all CTAs must be resident at once (the launch would be refused otherwise); asked once per shared-memory size
+    static std::mutex mu;
+    static std::unordered_map<size_t, int> per_sm_of;
+    int per_sm = 0;
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        auto it = per_sm_of.find(L.smem);
+        if (it == per_sm_of.end()) {
+            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, dc::kThreads, L.smem) != cudaSuccess)
+                return MOC_ERR_CUDA;
+            per_sm_of[L.smem] = per_sm;
+        } else {
+            per_sm = it->second;
+        }
+    }
+    if (per_sm < 1 || L.grid > per_sm * tc::sm_count()) return MOC_ERR_UNSUPPORTED;
+    dc::Params local = prm;
+    void *args[] = {&local};
+    MOC_LAUNCH(KID_DEC_COOP, st,
+               cudaLaunchCooperativeKernel(reinterpret_cast<void *>(kern), dim3(L.grid), dim3(dc::kThreads), args, L.smem, st));
+    return launch_ok();
+}
+
+int decode_coop(const moc_ffn_desc &d, const CoopLayout &L, const __nv_bfloat16 *x, const __nv_bfloat16 *wg,
+                const __nv_bfloat16 *wu, const __nv_bfloat16 *wd, __nv_bfloat16 *out, char *wsp, cudaStream_t st) {
+    int *status = device_status_ptr();
+    if (!status) return MOC_ERR_CUDA;
+    dc::Params prm{};
+    prm.x = x;
+    prm.wg = wg;
+    prm.wu = wu;
+    prm.wd = wd;
+    prm.out = out;
+    prm.T = (int)d.tokens;
+    prm.d = d.d_model;
+    prm.F = d.d_ff;
+    prm.K = d.k;
+    prm.grouped = (d.flags & MOC_FLAG_SELECT_2_OF_8) ? 1 : 0;
+    prm.unit = L.unit;
+    prm.stages = L.stages;
+    prm.hist = reinterpret_cast<uint32_t *>(wsp + L.off_hist);
+    prm.cand_n = reinterpret_cast<uint32_t *>(wsp + L.off_n);
+    prm.cand = reinterpret_cast<uint2 *>(wsp + L.off_cand);
+    prm.acc = reinterpret_cast<float *>(wsp + L.off_acc);
+    prm.status = status;
+    switch (prm.T) {
+        case 1: return launch_coop<1>(prm, L, st);
+        case 2: return launch_coop<2>(prm, L, st);
+        default: return MOC_ERR_UNSUPPORTED;
+    }
+}
+
 int decode_bf16(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat16 *wg, const __nv_bfloat16 *wu,
                 const __nv_bfloat16 *wd, __nv_bfloat16 *out, char *wsp, cudaStream_t st) {
     const DecodeLayout L = decode_layout(d);
@@ -934,7 +1036,11 @@ size_t moc_ffn_workspace_bytes(const moc_ffn_desc *desc, int op) {
     switch (op) {
         case MOC_OP_DECODE:
             if (desc->tokens > sb::kMaxTokens) return 0;
-            if (use_decode_plan(*desc)) return decode_layout(*desc).total;
+            if (use_decode_plan(*desc)) {
+                bool coop = false;
+                const CoopLayout C = coop_layout(*desc, coop);
+                return std::max(decode_layout(*desc).total, coop ? C.total : (size_t)0);
+            }
             // fall through: the forward with nothing saved
         case MOC_OP_FORWARD:
             if (use_small_batch_plan(*desc)) return small_batch_layout(*desc).total;
@@ -1040,9 +1146,20 @@ int moc_ffn_decode(const moc_ffn_desc *desc, const void *x, const void *w_gate, 
                                workspace_bytes, cuda_stream);
     if (!good_ptr(x) || !good_ptr(w_gate) || !good_ptr(w_up) || !good_ptr(w_down) || !good_ptr(out))
         return MOC_ERR_INVALID_ARG;
-    const size_t need = decode_layout(*desc).total;
+    const size_t need = moc_ffn_workspace_bytes(desc, MOC_OP_DECODE);
     if (!good_ptr(workspace) || workspace_bytes < need) return MOC_ERR_WORKSPACE;
     using T = __nv_bfloat16;
+    {
+        // a handful of tokens: one cooperative kernel; where the device or the problem does not admit it, or its
+        // launch is refused, the four-kernel plan
+        bool coop = false;
+        const CoopLayout C = coop_layout(*desc, coop);
+        if (coop) {
+            const int rc2 = decode_coop(*desc, C, (const T *)x, (const T *)w_gate, (const T *)w_up, (const T *)w_down,
+                                        (T *)out, static_cast<char *>(workspace), static_cast<cudaStream_t>(cuda_stream));
+            if (rc2 != MOC_ERR_UNSUPPORTED) return rc2;
+        }
+    }
     return decode_bf16(*desc, (const T *)x, (const T *)w_gate, (const T *)w_up, (const T *)w_down, (T *)out,
                        static_cast<char *>(workspace), static_cast<cudaStream_t>(cuda_stream));
 }

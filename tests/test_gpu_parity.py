@@ -258,7 +258,7 @@ def _check_decode(out64, x64, wg64, wu64, wd64, K, dtype, what):
         assert np.abs(out64[t] - ref).max() <= tol, f"{what}: token {t} matches neither pick"
 
 
-@pytest.mark.parametrize("T", [1, 4, 5, 6, 16])   # up to 5 tokens: row gathers; from 6: all weights streamed once
+@pytest.mark.parametrize("T", [1, 2, 4, 5, 6, 16])   # 1, 2: cooperative kernel; to 5: four-kernel plan; from 6: small-batch plan
 def test_decode_llama7b_shape(T):
     w = syn.C4.with_tokens(T)
     wg, wu, wd = syn.make_weights(w)
@@ -497,3 +497,36 @@ def test_bounded_wait_runs_out_reports_timeout_and_leaves_the_context_usable():
         B.moc_test_bounded_wait(0)                                   # limit out of range: nothing launched
     _run_forward_backward(syn.Workload("after-timeout", "bf16", 300, 128, 512, 512, 64, seed=9))
     assert B.moc_last_device_status() == B.MOC_OK
+
+
+def test_decode_four_kernel_plan_selected_by_environment():
+    """MOC_FFN_DECODE=chain (read once per process) keeps one- and two-token batches on the four-kernel decode plan
+    instead of the cooperative kernel: run the decode cases again in a child process with it set."""
+    import os
+    import subprocess
+    import sys
+    env = dict(os.environ, MOC_FFN_DECODE="chain")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    r = subprocess.run([sys.executable, "-m", "pytest", os.path.join(root, "tests", "test_gpu_parity.py"),
+                        os.path.join(root, "tests", "test_gpu_grouped.py"), "-q", "-x", "-m", "gpu", "-k",
+                        "decode_llama7b_shape or decode_small_shapes or decode_with_padded or grouped_decode or decode_ties"],
+                       cwd=root, env=env, capture_output=True, text=True, timeout=900)
+    assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
+
+
+@pytest.mark.parametrize("T", [1, 2, 4, 8])
+def test_decode_ties_and_degenerate_tokens(T):
+    """Duplicated gate rows (bit-identical gate values; K odd, so exactly one pair is split and the lower channel must
+    win), an all-zero token (every value ties: channels 0..K-1) -- through every decode form (cooperative kernel,
+    four-kernel plan, small-batch plan)."""
+    w = syn.Workload("dec-ties", "bf16", T, 128, 512, 512, 65, seed=77 + T, decode=True)
+    wg, wu, wd = syn.make_weights(w)
+    wg[1::2] = wg[0::2]
+    x = syn.make_x(w)
+    x[T - 1] = 0
+    out = B.moc_ffn_decode(_dev(x), _dev(wg), _dev(wu), _dev(wd), w.k)
+    torch.cuda.synchronize()
+    assert torch.all(out[T - 1] == 0)
+    x64, wg64, wu64, wd64 = map(syn.to_f64, (x, wg, wu, wd))
+    ref = orc.forward(x64, wg64, wu64, wd64, w.k)["out"]     # the oracle's tie rule: the lower channel
+    parity.assert_close(syn.to_f64(out), ref, "bf16", f"decode with ties T={T}")
