@@ -621,8 +621,8 @@ def decode_report(torch, B, syn, dev, peaks, calls=32, sets=4, replays=5):
             rep[f"T{T}"].update(plan="small-batch (all weights streamed once, tcgen05)", executed_bytes=executed,
                                 executed_frac=executed / (peaks["hbm_gbs"] * 1e9) * 1e6 / us)
         else:
-            rep[f"T{T}"].update(plan="decode (gate matrix + gathered rows)", executed_bytes=algo,
-                                executed_frac=roof_us / us)
+            rep[f"T{T}"].update(plan=("decode, one cooperative kernel" if launches == 1 else "decode, four kernels") +
+                                " (gate matrix + gathered rows)", executed_bytes=algo, executed_frac=roof_us / us)
         del ws, graph
     if B.moc_last_device_status() != B.MOC_OK:
         raise RuntimeError("device status raised during decode")
