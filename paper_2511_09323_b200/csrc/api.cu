@@ -710,7 +710,9 @@ CoopLayout coop_layout(const moc_ffn_desc &d, bool &ok) {
     const size_t fixed = (size_t)T * dm * 2 + (size_t)2 * T * dc::kMaxRows * 4;
     const size_t budget = (size_t)216 * 1024;
     if (fixed + (size_t)4 * dm * 2 > budget) return L;
-    L.stages = (int)std::min<size_t>(dc::kMaxStages, (budget - fixed) / ((size_t)dm * 2));
+    // a multiple of the consumer warps: every stage is then always consumed by the same warp (see the kernel)
+    L.stages = (int)std::min<size_t>(dc::kMaxStages, (budget - fixed) / ((size_t)dm * 2)) / dc::kConsumerWarps * dc::kConsumerWarps;
+    if (L.stages < dc::kConsumerWarps) return L;
     L.smem = dc::smem_bytes(T, dm, L.stages);
     Carver c;
     L.off_hist = c.take((size_t)T * dc::kBins * sizeof(uint32_t));

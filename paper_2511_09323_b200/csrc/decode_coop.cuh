@@ -36,7 +36,7 @@ constexpr int kConsumerWarps = 16;
 constexpr int kThreads = (kConsumerWarps + 1) * 32;  // + one producer warp
 constexpr int kMaxRows = 256;        // channels per CTA
 constexpr int kBins = 2048;          // top 11 bits of the key
-constexpr int kMaxStages = 24;
+constexpr int kMaxStages = 32;         // a multiple of kConsumerWarps
 
 struct Params {
     const __nv_bfloat16 *x, *wg, *wu, *wd;
@@ -122,6 +122,11 @@ __global__ void __launch_bounds__(kThreads, 1) decode_coop_kernel(const Params p
     auto release = [&](uint32_t count) {  // the calling lane frees the current stage on behalf of `count` warps
         asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0], %1;" ::"r"(empty_bar(c_stage)), "r"(count) : "memory");
     };
+    // A parity test only tells an odd from an even number of completed rounds of a stage, so a warp must see every round
+    // of the stages it waits on (a stage two rounds behind would pass the test for the current round at once).  The
+    // number of stages is therefore a multiple of the number of consumer warps: row r goes to stage r mod stages and to
+    // warp r mod 16, so a stage is always consumed by the same warp.  (In the last phase every warp sees every row.)
+    auto wait_row = [&](int) -> bool { return tc::mbar_wait(full_bar(c_stage), c_phase, &s_abort, p.status); };
     // dot products of one staged row with the T tokens, by one warp (every lane gets the sums)
     auto row_dots = [&](const uint8_t *row, float (&sum)[T]) {
 #pragma unroll
@@ -167,7 +172,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_coop_kernel(const Params p
     } else {
         for (int r = 0; r < rows; ++r) {
             if (r % kConsumerWarps == warp) {
-                const bool ok = __all_sync(0xffffffffu, tc::mbar_wait(full_bar(c_stage), c_phase, &s_abort, p.status));
+                const bool ok = __all_sync(0xffffffffu, wait_row(r));
                 float sum[T];
                 if (ok) row_dots(ring + (size_t)c_stage * row_bytes, sum);
                 __syncwarp();
@@ -318,7 +323,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_coop_kernel(const Params p
     } else {
         for (int i = 0; i < nsel; ++i) {
             if (i % kConsumerWarps == warp) {
-                const bool ok = __all_sync(0xffffffffu, tc::mbar_wait(full_bar(c_stage), c_phase, &s_abort, p.status));
+                const bool ok = __all_sync(0xffffffffu, wait_row(rows + i));
                 float sum[T];
                 if (ok) row_dots(ring + (size_t)c_stage * row_bytes, sum);
                 __syncwarp();
