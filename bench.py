@@ -517,6 +517,7 @@ def roofline_report(prof, steps, T, w, e, peaks):
         else:
             roof.update(bound="alu", achieved=rate / 1e12, peak=ALU_FP32_PEAK_TFLOPS, unit="TFLOP/s")
         roof["frac"] = roof["achieved"] / roof["peak"]
+        roof["executed_frac"] = roof["executed_rate"] / roof["peak"]   # the dense work the kernel really does
         roof["peak_source"] = peaks["source"] if bound != "alu" else "derived: 148 SM x 128 lanes x 2 x 1.965 GHz"
         roof["algorithmic_per_launch"] = per_launch
     # measured DRAM bytes per launch exist for the default workload only (one launch of each kernel per step there)
