@@ -24,6 +24,8 @@
  *                                 the `keep` largest signed pre-SiLU values of every `group` consecutive channels.
  *   moc_oracle_backward           Section 4, Eqs. (bp-1)..(bp-5), with S' and Z' recomputed from the
  *                                 saved G.M and U.M ("MoC + GCP", Table 1).
+ *   moc_oracle_rmsnorm            Section 2, item "RMSNorm": y = x / RMS(x) . g, RMS(x) = sqrt(mean(x^2) + eps).
+ *   moc_oracle_residual           Section 2, item "Residual connections": Z = X + Y.
  *   moc_oracle_silu / dsilu       Eq. (silu) and its derivative.
  *   moc_oracle_macs_*             Section 5: 3 d d_ffn versus d d_ffn + 2 K d.
  *   moc_oracle_saved_elems_*      Table 1: 4 d_ffn (FFN), 2 d_ffn (FFN+GCP), d_ffn-equivalent 5K (MoC),
@@ -441,6 +443,30 @@ int moc_oracle_backward_weight_rows(int64_t T, int32_t d, int32_t F, int32_t K, 
     }
     free(slot);
     return MOC_ORACLE_OK;
+}
+
+/* ---------------------------------------------------------------- the block around the layer */
+
+/* Section 2, "RMSNorm": for each row x of X [T, d], y = x / RMS(x) . g with RMS(x) = sqrt((1/d) sum x_i^2 + eps). */
+int moc_oracle_rmsnorm(int64_t T, int32_t d, const double *x, const double *weight, double eps, double *y)
+{
+    if (T < 0 || d <= 0 || !x || !weight || !y || !(eps >= 0.0)) return -1;
+    for (int64_t t = 0; t < T; ++t) {
+        const double *xt = x + t * (int64_t)d;
+        double ss = 0.0;
+        for (int32_t i = 0; i < d; ++i) ss += xt[i] * xt[i];
+        const double rms = sqrt(ss / (double)d + eps);
+        for (int32_t i = 0; i < d; ++i) y[t * (int64_t)d + i] = xt[i] / rms * weight[i];
+    }
+    return 0;
+}
+
+/* Section 2, "Residual connections": Z = X + Y, element by element. */
+int moc_oracle_residual(int64_t n, const double *x, const double *y, double *z)
+{
+    if (n < 0 || !x || !y || !z) return -1;
+    for (int64_t i = 0; i < n; ++i) z[i] = x[i] + y[i];
+    return 0;
 }
 
 /* ---------------------------------------------------------------- counting formulas */

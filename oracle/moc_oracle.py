@@ -157,6 +157,40 @@ def gate_projection(x, w_gate, F: int | None = None):
     return x @ w_gate[:F].T
 
 
+def rmsnorm(x, weight, eps: float):
+    """y = x / RMS(x) . g per row, RMS(x) = sqrt(mean(x^2) + eps) (Section 2, item "RMSNorm"); [T, d] float64."""
+    x, weight = _f64(x), _f64(weight)
+    T, d = x.shape
+    assert weight.shape == (d,)
+    y = np.empty_like(x)
+    _check(_load().moc_oracle_rmsnorm(ctypes.c_int64(T), ctypes.c_int32(d), _p(x), _p(weight), ctypes.c_double(eps),
+                                      _p(y)), "moc_oracle_rmsnorm")
+    return y
+
+
+def residual(x, y):
+    """Z = X + Y (Section 2, item "Residual connections")."""
+    x, y = _f64(x), _f64(y)
+    assert x.shape == y.shape
+    z = np.empty_like(x)
+    _check(_load().moc_oracle_residual(ctypes.c_int64(x.size), _p(x), _p(y), _p(z)), "moc_oracle_residual")
+    return z
+
+
+def decode_block(h, rms_weight, eps: float, w_gate, w_up, w_down, K: int, F: int | None = None, store=None):
+    """The FFN half of a pre-norm Transformer layer (Section 2, "LLM structure"): out = h + MoC_FFN(RMSNorm(h)).
+
+    `store`: what writing the normalised activations in the storage type does to them (the paper runs in BF16:
+    the rounding to bf16), a callable on float64 arrays; None keeps them in float64.  Returns (out, x, picks) with x
+    the activations the layer saw and picks the layer's forward dictionary.
+    """
+    x = rmsnorm(h, rms_weight, eps)
+    if store is not None:
+        x = _f64(store(x))
+    f = forward(x, w_gate, w_up, w_down, K, F, want_g=True)
+    return residual(h, f["out"]), x, f
+
+
 def forward_grouped(x, w_gate, w_up, w_down, group: int = 8, keep: int = 2, F: int | None = None):
     """The layer with the grouped mask: gate projection, grouped selection, then the steps of the layer on the
     selected channels.  Returns dict(out, idx, gval, uval, g)."""

@@ -503,3 +503,62 @@ def test_theorem_1_embedding_dense_ffn_into_2_of_8():
     np.testing.assert_allclose(moc["out"], dense, rtol=1e-12, atol=1e-13)
     # a group whose second real slot is padding keeps a zero channel, which contributes nothing
     assert moc["idx"].shape == (5, 2 * groups)
+
+
+# --------------------------------------------------------------------------- the block around the layer (Section 2)
+
+def test_rmsnorm_worked_example_and_closed_forms():
+    """Section 2, item "RMSNorm": y = x / sqrt(mean(x^2) + eps) . g."""
+    # x = (3, 4): mean square 12.5, RMS 3.5355339059..., so y = (0.848528137.., 1.131370849..) before the weight
+    y = orc.rmsnorm(np.array([[3.0, 4.0]]), np.array([1.0, 2.0]), 0.0)
+    np.testing.assert_allclose(y, [[0.8485281374238570, 2.2627416997969520]], rtol=1e-15)
+    # eps enters under the root: x = (1, 1, 1, 1), eps = 3 gives RMS 2
+    y = orc.rmsnorm(np.ones((1, 4)), np.array([1.0, -2.0, 4.0, 0.5]), 3.0)
+    np.testing.assert_allclose(y, [[0.5, -1.0, 2.0, 0.25]], rtol=1e-15)
+    # a zero row stays zero (eps keeps the division finite)
+    assert np.all(orc.rmsnorm(np.zeros((2, 8)), np.ones(8), 1e-6) == 0.0)
+    rng = np.random.default_rng(21)
+    x = rng.standard_normal((7, 96)) * rng.uniform(0.01, 100.0, (7, 1))
+    g = rng.standard_normal(96)
+    # unit weight, eps = 0: every row has mean square exactly 1; rows are invariant to their scale
+    y1 = orc.rmsnorm(x, np.ones(96), 0.0)
+    np.testing.assert_allclose((y1 * y1).mean(axis=1), 1.0, rtol=1e-13)
+    np.testing.assert_allclose(orc.rmsnorm(-3.5 * x, np.ones(96), 0.0), -y1, rtol=1e-13)
+    # the weight multiplies element by element
+    np.testing.assert_allclose(orc.rmsnorm(x, g, 0.0), y1 * g, rtol=1e-13)
+
+
+def test_rmsnorm_matches_the_library_routine():
+    torch = pytest.importorskip("torch")
+    rng = np.random.default_rng(22)
+    x = rng.standard_normal((5, 160))
+    g = rng.standard_normal(160)
+    for eps in (0.0, 1e-6, 0.3):
+        ref = torch.nn.functional.rms_norm(torch.from_numpy(x), (160,), torch.from_numpy(g), eps).numpy()
+        np.testing.assert_allclose(orc.rmsnorm(x, g, eps), ref, rtol=1e-13, atol=1e-15)
+
+
+def test_residual_and_block_composition():
+    """Section 2, item "Residual connections" (Z = X + Y) and "LLM structure": out = h + FFN(RMSNorm(h))."""
+    np.testing.assert_array_equal(orc.residual(np.array([[1.0, -2.0], [0.5, 4.0]]), np.array([[10.0, 20.0], [30.0, 40.0]])),
+                                  [[11.0, 18.0], [30.5, 44.0]])
+    rng = np.random.default_rng(23)
+    T, d, F, K = 4, 24, 40, 7
+    h = rng.standard_normal((T, d)) * 3.0
+    g = rng.uniform(0.5, 1.5, d)
+    wg, wu, wd = (rng.standard_normal((F, d)) * 0.2 for _ in range(3))
+    # a zero down projection leaves the residual stream untouched
+    out, x, _ = orc.decode_block(h, g, 1e-5, wg, wu, np.zeros_like(wd), K)
+    np.testing.assert_array_equal(out, h)
+    # the layer sees the normalised rows: unit-ish mean square whatever the scale of h
+    np.testing.assert_allclose(((x / g) ** 2).mean(axis=1), 1.0, rtol=1e-4)
+    # scaling h by a positive constant changes only the residual term (eps = 0: the norm removes the scale)
+    out1, _, f1 = orc.decode_block(h, g, 0.0, wg, wu, wd, K)
+    out2, _, f2 = orc.decode_block(7.0 * h, g, 0.0, wg, wu, wd, K)
+    np.testing.assert_array_equal(f1["idx"], f2["idx"])
+    np.testing.assert_allclose(out2 - 7.0 * h, out1 - h, rtol=1e-10, atol=1e-12)
+    # `store` is applied to what the layer reads: a coarse rounding changes the layer's input and nothing else
+    coarse = lambda a: np.round(a * 8.0) / 8.0
+    out3, x3, f3 = orc.decode_block(h, g, 1e-5, wg, wu, wd, K, store=coarse)
+    np.testing.assert_array_equal(x3, coarse(orc.rmsnorm(h, g, 1e-5)))
+    np.testing.assert_allclose(out3, h + orc.forward(x3, wg, wu, wd, K)["out"], rtol=1e-13, atol=1e-14)
