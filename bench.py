@@ -588,26 +588,31 @@ def decode_report(torch, B, syn, dev, peaks, calls=32, sets=4, replays=5):
         out = torch.empty_like(x)
         desc = B.make_desc(T, w.d_model, w.d_ff, w.k, x.dtype, d_ff_ld=w.d_ff_ld)
         ws = B.alloc_workspace(desc, B.MOC_OP_DECODE, dev)
-        for i in range(sets):   # warm-up; also performs every one-time set-up outside the capture
-            B.moc_ffn_decode(x, *weights[i], w.k, out=out, workspace=ws)
-        torch.cuda.synchronize()
-        launches0 = B.moc_launch_count()
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.stream(stream):
-            with torch.cuda.graph(graph, stream=stream):
-                for i in range(calls):
-                    B.moc_ffn_decode(x, *weights[i % sets], w.k, out=out, workspace=ws, stream=stream)
-        launches = (B.moc_launch_count() - launches0) // calls
-        torch.cuda.synchronize()
-        graph.replay()
-        torch.cuda.synchronize()
-        s, t = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        s.record()
-        for _ in range(replays):
+        def timed(call):
+            """us per call and library kernels per call of `call(i, stream)` captured `calls` times in one graph."""
+            for i in range(sets):   # warm-up; also performs every one-time set-up outside the capture
+                call(i, None)
+            torch.cuda.synchronize()
+            launches0 = B.moc_launch_count()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.stream(stream):
+                with torch.cuda.graph(graph, stream=stream):
+                    for i in range(calls):
+                        call(i, stream)
+            n_launch = (B.moc_launch_count() - launches0) // calls
+            torch.cuda.synchronize()
             graph.replay()
-        t.record()
-        torch.cuda.synchronize()
-        us = s.elapsed_time(t) * 1e3 / (calls * replays)
+            torch.cuda.synchronize()
+            s, t = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            s.record()
+            for _ in range(replays):
+                graph.replay()
+            t.record()
+            torch.cuda.synchronize()
+            del graph
+            return s.elapsed_time(t) * 1e3 / (calls * replays), n_launch
+
+        us, launches = timed(lambda i, st: B.moc_ffn_decode(x, *weights[i % sets], w.k, out=out, workspace=ws, stream=st))
         # union of selected channels from a saved forward on set 0 (same selection rule)
         _, idx, _, _ = B.moc_ffn_forward(x, *weights[0], w.k)
         union = int(torch.unique(idx.long()).numel())
@@ -624,7 +629,24 @@ def decode_report(torch, B, syn, dev, peaks, calls=32, sets=4, replays=5):
         else:
             rep[f"T{T}"].update(plan=("decode, one cooperative kernel" if launches == 1 else "decode, four kernels") +
                                 " (gate matrix + gathered rows)", executed_bytes=algo, executed_frac=roof_us / us)
-        del ws, graph
+        if T in syn.C4_BATCHES:
+            # the FFN half of a pre-norm layer, out = h + FFN(RMSNorm(h)): one library call against the same steps as
+            # separate launches (torch's RMSNorm and addition around moc_ffn_decode)
+            gamma = torch.ones(w.d_model, dtype=x.dtype, device=dev)
+            wsb = B.alloc_workspace(desc, B.MOC_OP_DECODE_BLOCK, dev)
+            us_b, n_b = timed(lambda i, st: B.moc_ffn_decode_block(x, gamma, 1e-6, *weights[i % sets], w.k, out=out,
+                                                                   workspace=wsb, stream=st))
+
+            def unfused(i, st):
+                xn = torch.nn.functional.rms_norm(x, (w.d_model,), gamma, 1e-6)
+                B.moc_ffn_decode(xn, *weights[i % sets], w.k, out=out, workspace=ws, stream=st)
+                torch.add(x, out, out=out)
+
+            us_u, _ = timed(unfused)
+            rep[f"T{T}"]["block"] = {"us_per_step": us_b, "kernels_per_call": n_b,
+                                     "unfused_us_per_step": us_u, "what": "out = h + FFN(RMSNorm(h))"}
+            del wsb
+        del ws
     if B.moc_last_device_status() != B.MOC_OK:
         raise RuntimeError("device status raised during decode")
     return rep

@@ -68,7 +68,7 @@ typedef enum {
 
 typedef enum { MOC_F32 = 0, MOC_BF16 = 1 } moc_dtype;
 
-typedef enum { MOC_OP_FORWARD = 0, MOC_OP_BACKWARD = 1, MOC_OP_DECODE = 2 } moc_op;
+typedef enum { MOC_OP_FORWARD = 0, MOC_OP_BACKWARD = 1, MOC_OP_DECODE = 2, MOC_OP_DECODE_BLOCK = 3 } moc_op;
 
 /* bit 0 of moc_ffn_desc.flags: add into grad_w_* instead of overwriting them */
 #define MOC_FLAG_ACCUMULATE_WGRAD 1u
@@ -150,6 +150,28 @@ MOC_API int moc_ffn_recompute_up(const moc_ffn_desc *desc, const void *x, const 
 MOC_API int moc_ffn_decode(const moc_ffn_desc *desc, const void *x, const void *w_gate, const void *w_up,
                            const void *w_down, void *out, void *workspace, size_t workspace_bytes,
                            void *cuda_stream);
+
+/*
+ * The FFN half of a pre-norm Transformer layer for small batches (Section 2, "LLM structure", with the items
+ * "RMSNorm" and "Residual connections" of its activation list): out = h + MoC_FFN(RMSNorm(h)), where
+ * RMSNorm(h) = h / sqrt(mean(h^2) + rms_eps) . rms_weight per token, rounded to bf16 as the layer's input, and the
+ * sum h + D is formed in fp32 from the layer's unrounded output and rounded once.  The normalisation and the
+ * residual addition ride on the decode kernels instead of being two more launches around them: with one or two
+ * tokens both happen inside the one cooperative kernel; otherwise a one-CTA-per-token kernel chained in front writes
+ * the normalised rows and the last step of the down projection adds h.
+ *
+ *   h           [tokens, d_model] bf16, device: the residual stream
+ *   rms_weight  [d_model] bf16, device
+ *   rms_eps     >= 0
+ *   out         [tokens, d_model] bf16, device; may be h itself (update in place)
+ *   workspace   moc_ffn_workspace_bytes(desc, MOC_OP_DECODE_BLOCK) bytes
+ * bf16 only, tokens <= 256, d_model a multiple of 8, and a d_ff that the small-batch selector holds in shared
+ * memory (moc_ffn_workspace_bytes returns 0 otherwise and the call MOC_ERR_UNSUPPORTED).  Weights, stream,
+ * ownership and the status word as for moc_ffn_decode.
+ */
+MOC_API int moc_ffn_decode_block(const moc_ffn_desc *desc, const void *h, const void *rms_weight, float rms_eps,
+                                 const void *w_gate, const void *w_up, const void *w_down, void *out,
+                                 void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
  * moc_ffn_decode for callers that must not allocate.  (The paper has no counterpart: this is a

@@ -24,7 +24,7 @@ MOC_ERR_BAD_INDEX = -6
 MOC_ERR_STATIC_LIMIT = -7
 MOC_STATIC_MAX_TOKENS, MOC_STATIC_MAX_DFF = 16, 16384
 MOC_F32, MOC_BF16 = 0, 1
-MOC_OP_FORWARD, MOC_OP_BACKWARD, MOC_OP_DECODE = 0, 1, 2
+MOC_OP_FORWARD, MOC_OP_BACKWARD, MOC_OP_DECODE, MOC_OP_DECODE_BLOCK = 0, 1, 2, 3
 MOC_FLAG_ACCUMULATE_WGRAD = 1
 MOC_FLAG_SELECT_2_OF_8 = 2
 
@@ -72,6 +72,8 @@ def load() -> ctypes.CDLL:
         lib.moc_ffn_backward.argtypes = [dp] + [vp] * 13 + [sz, vp]
         lib.moc_ffn_decode.restype = ctypes.c_int
         lib.moc_ffn_decode.argtypes = [dp] + [vp] * 6 + [sz, vp]
+        lib.moc_ffn_decode_block.restype = ctypes.c_int
+        lib.moc_ffn_decode_block.argtypes = [dp, vp, vp, ctypes.c_float] + [vp] * 5 + [sz, vp]
         lib.moc_ffn_recompute_up.restype = ctypes.c_int
         lib.moc_ffn_recompute_up.argtypes = [dp] + [vp] * 5 + [sz, vp]
         lib.moc_ffn_decode_static.restype = ctypes.c_int
@@ -261,6 +263,30 @@ def moc_ffn_decode(x, w_gate, w_up, w_down, k, d_ff=None, out=None, workspace=No
                                _ptr(workspace), workspace.numel(), _stream_ptr(stream))
     if rc != MOC_OK:
         raise MocError(rc, "moc_ffn_decode")
+    return out
+
+
+def moc_ffn_decode_block(h, rms_weight, rms_eps, w_gate, w_up, w_down, k, d_ff=None, out=None, workspace=None,
+                         stream=None, grouped=False):
+    """out = h + MoC_FFN(RMSNorm(h; rms_weight, rms_eps)) for up to 256 bf16 tokens; `out` may be `h`."""
+    _check_dev(h, rms_weight, w_gate, w_up, w_down, out, workspace)
+    T, d = h.shape
+    if rms_weight.dtype != h.dtype or tuple(rms_weight.shape) != (d,):
+        raise TypeError("rms_weight must be a [d_model] tensor of the activations' dtype")
+    F_ld = w_gate.shape[0]
+    if grouped:
+        k = _grouped_k(k, F_ld if d_ff is None else d_ff)
+    desc = make_desc(T, d, F_ld if d_ff is None else d_ff, k, h.dtype, d_ff_ld=F_ld,
+                     flags=MOC_FLAG_SELECT_2_OF_8 if grouped else 0)
+    if out is None:
+        out = torch.empty_like(h)
+    if workspace is None:
+        workspace = alloc_workspace(desc, MOC_OP_DECODE_BLOCK, h.device)
+    rc = load().moc_ffn_decode_block(ctypes.byref(desc), _ptr(h), _ptr(rms_weight), float(rms_eps), _ptr(w_gate),
+                                     _ptr(w_up), _ptr(w_down), _ptr(out), _ptr(workspace), workspace.numel(),
+                                     _stream_ptr(stream))
+    if rc != MOC_OK:
+        raise MocError(rc, "moc_ffn_decode_block")
     return out
 
 

@@ -72,6 +72,7 @@ enum KernelId {
     KID_SB_DOWN,
     KID_RECOMPUTE_UP,
     KID_DEC_COOP,
+    KID_DEC_RMSNORM,
     KID_COUNT
 };
 static const char *const kKernelNames[KID_COUNT] = {
@@ -80,7 +81,7 @@ static const char *const kKernelNames[KID_COUNT] = {
     "tc_gate_up_gemm", "tc_select_mask",  "tc_down_gemm",  "tc_bwd_sample",  "tc_dz_gemm",
     "tc_wgrad_gemm",   "tc_dx_gemm",      "tc_test_gemm",  "tc_select_hint", "dec_gate_gemv",
     "dec_select",      "dec_up",          "dec_down",      "sb_gate_up",     "sb_select",
-    "sb_down",         "recompute_up",    "dec_coop",
+    "sb_down",         "recompute_up",    "dec_coop",      "dec_rmsnorm",
 };
 
 struct Profiler {
@@ -752,8 +753,10 @@ int launch_coop(const dc::Params &prm, const CoopLayout &L, cudaStream_t st) {
     return launch_ok();
 }
 
+// rms_w != nullptr: the block form (x is the residual stream h: RMSNorm in front, h added behind)
 int decode_coop(const moc_ffn_desc &d, const CoopLayout &L, const __nv_bfloat16 *x, const __nv_bfloat16 *wg,
-                const __nv_bfloat16 *wu, const __nv_bfloat16 *wd, __nv_bfloat16 *out, char *wsp, cudaStream_t st) {
+                const __nv_bfloat16 *wu, const __nv_bfloat16 *wd, __nv_bfloat16 *out, char *wsp, cudaStream_t st,
+                const __nv_bfloat16 *rms_w = nullptr, float rms_eps = 0.f) {
     int *status = device_status_ptr();
     if (!status) return MOC_ERR_CUDA;
     dc::Params prm{};
@@ -769,6 +772,8 @@ int decode_coop(const moc_ffn_desc &d, const CoopLayout &L, const __nv_bfloat16 
     prm.grouped = (d.flags & MOC_FLAG_SELECT_2_OF_8) ? 1 : 0;
     prm.unit = L.unit;
     prm.stages = L.stages;
+    prm.rms_w = rms_w;
+    prm.rms_eps = rms_eps;
     prm.hist = reinterpret_cast<uint32_t *>(wsp + L.off_hist);
     prm.cand_n = reinterpret_cast<uint32_t *>(wsp + L.off_n);
     prm.cand = reinterpret_cast<uint2 *>(wsp + L.off_cand);
@@ -781,8 +786,10 @@ int decode_coop(const moc_ffn_desc &d, const CoopLayout &L, const __nv_bfloat16 
     }
 }
 
+// resid != nullptr: added to the layer's output before the rounding (the block form)
 int decode_bf16(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat16 *wg, const __nv_bfloat16 *wu,
-                const __nv_bfloat16 *wd, __nv_bfloat16 *out, char *wsp, cudaStream_t st) {
+                const __nv_bfloat16 *wd, __nv_bfloat16 *out, char *wsp, cudaStream_t st,
+                const __nv_bfloat16 *resid = nullptr) {
     const DecodeLayout L = decode_layout(d);
     const int T = (int)d.tokens, F = d.d_ff, K = d.k, dm = d.d_model;
     int *status = device_status_ptr();
@@ -825,7 +832,7 @@ int decode_bf16(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat
     if ((rc = launch_ok()) != MOC_OK) return rc;
     MOC_LAUNCH(KID_DEC_DOWN, st,
                launch_pdl(dec::down_rows_kernel, dim3(L.slices, L.parts), dec::kGemvThreads, dec::kDownSmem, st, wd, T, dm,
-                          F, ws, out, status));
+                          F, ws, out, resid, status));
     return launch_ok();
 }
 
@@ -902,7 +909,8 @@ bool use_small_batch_plan(const moc_ffn_desc &d) {
 
 int forward_small_batch(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat16 *wg,
                         const __nv_bfloat16 *wu, const __nv_bfloat16 *wd, __nv_bfloat16 *out, int16_t *idx,
-                        __nv_bfloat16 *tg, __nv_bfloat16 *tu, char *wsp, cudaStream_t st) {
+                        __nv_bfloat16 *tg, __nv_bfloat16 *tu, char *wsp, cudaStream_t st,
+                        const __nv_bfloat16 *resid = nullptr) {
     const SmallBatchLayout L = small_batch_layout(d);
     const int T = (int)d.tokens, F = d.d_ff, dm = d.d_model;
     int *status = device_status_ptr();
@@ -973,6 +981,7 @@ int forward_small_batch(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __n
     dp.accs = L.accs;
     dp.acc = acc;
     dp.out = out;
+    dp.resid = resid;
     dp.counters = counters;
     dp.status = status;
     MOC_LAUNCH(KID_SB_DOWN, st,
@@ -1032,6 +1041,12 @@ using namespace moc;
 // =====================================================================================================
 extern "C" {
 
+// The block form runs on the three weight-streaming plans for small bf16 batches.
+static bool block_form_supported(const moc_ffn_desc &d) {
+    return d.dtype == MOC_BF16 && d.tokens >= 1 && d.tokens <= sb::kMaxTokens && d.d_model % 8 == 0 &&
+           (use_decode_plan(d) || use_small_batch_plan(d));
+}
+
 size_t moc_ffn_workspace_bytes(const moc_ffn_desc *desc, int op) {
     if (check_desc(desc) != MOC_OK) return 0;
     if (desc->tokens == 0) return 0;
@@ -1049,6 +1064,12 @@ size_t moc_ffn_workspace_bytes(const moc_ffn_desc *desc, int op) {
             return use_tc_plan(*desc) ? tc::tc_forward_layout(*desc).total : plan_forward(*desc).total;
         case MOC_OP_BACKWARD:
             return use_tc_plan(*desc) ? tc::tc_backward_layout(*desc).total : plan_backward(*desc).total;
+        case MOC_OP_DECODE_BLOCK: {
+            // the decode workspace followed by the normalised activations [tokens, d_model]
+            if (!block_form_supported(*desc)) return 0;
+            return align_up(moc_ffn_workspace_bytes(desc, MOC_OP_DECODE), 256) +
+                   align_up((size_t)desc->tokens * desc->d_model * sizeof(__nv_bfloat16), 256);
+        }
         default:
             return 0;
     }
@@ -1164,6 +1185,45 @@ int moc_ffn_decode(const moc_ffn_desc *desc, const void *x, const void *w_gate, 
     }
     return decode_bf16(*desc, (const T *)x, (const T *)w_gate, (const T *)w_up, (const T *)w_down, (T *)out,
                        static_cast<char *>(workspace), static_cast<cudaStream_t>(cuda_stream));
+}
+
+int moc_ffn_decode_block(const moc_ffn_desc *desc, const void *h, const void *rms_weight, float rms_eps,
+                         const void *w_gate, const void *w_up, const void *w_down, void *out, void *workspace,
+                         size_t workspace_bytes, void *cuda_stream) {
+    int rc = check_desc(desc);
+    if (rc != MOC_OK) return rc;
+    if (desc->tokens == 0) return MOC_OK;
+    if (!block_form_supported(*desc)) return MOC_ERR_UNSUPPORTED;
+    if (!good_ptr(h) || !good_ptr(rms_weight) || !good_ptr(w_gate) || !good_ptr(w_up) || !good_ptr(w_down) ||
+        !good_ptr(out) || !(rms_eps >= 0.f))
+        return MOC_ERR_INVALID_ARG;
+    const size_t need = moc_ffn_workspace_bytes(desc, MOC_OP_DECODE_BLOCK);
+    if (!good_ptr(workspace) || workspace_bytes < need) return MOC_ERR_WORKSPACE;
+    using T = __nv_bfloat16;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    char *wsp = static_cast<char *>(workspace);
+    if (use_decode_plan(*desc)) {
+        // one or two tokens: the cooperative kernel normalises its staged rows and adds h itself
+        bool coop = false;
+        const CoopLayout C = coop_layout(*desc, coop);
+        if (coop) {
+            const int rc2 = decode_coop(*desc, C, (const T *)h, (const T *)w_gate, (const T *)w_up, (const T *)w_down,
+                                        (T *)out, wsp, st, (const T *)rms_weight, rms_eps);
+            if (rc2 != MOC_ERR_UNSUPPORTED) return rc2;
+        }
+    }
+    // otherwise a small kernel writes RMSNorm(h) behind the decode workspace, the plan's first kernel reads it as
+    // its x, and the plan's last step adds h before it rounds
+    T *xn = reinterpret_cast<T *>(wsp + align_up(moc_ffn_workspace_bytes(desc, MOC_OP_DECODE), 256));
+    MOC_LAUNCH(KID_DEC_RMSNORM, st,
+               launch_pdl(dec::rmsnorm_rows_kernel, dim3((unsigned)desc->tokens), 256, 0, st, (const T *)h,
+                          (const T *)rms_weight, rms_eps, desc->d_model, xn));
+    if ((rc = launch_ok()) != MOC_OK) return rc;
+    if (use_decode_plan(*desc))
+        return decode_bf16(*desc, xn, (const T *)w_gate, (const T *)w_up, (const T *)w_down, (T *)out, wsp, st,
+                           (const T *)h);
+    return forward_small_batch(*desc, xn, (const T *)w_gate, (const T *)w_up, (const T *)w_down, (T *)out, nullptr,
+                               nullptr, nullptr, wsp, st, (const T *)h);
 }
 
 int moc_ffn_recompute_up(const moc_ffn_desc *desc, const void *x, const void *w_up, const int16_t *topk_idx,

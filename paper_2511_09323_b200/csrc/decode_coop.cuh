@@ -50,6 +50,10 @@ struct Params {
     uint2 *cand;         // [T][F]  (key, channel)
     float *acc;          // [T][d]
     int *status;
+    // the block form (Section 2, "LLM structure"): x holds the residual stream h, the layer reads RMSNorm(h) with
+    // weight rms_w and adds h to its output; rms_w == nullptr: the plain layer on x
+    const __nv_bfloat16 *rms_w;
+    float rms_eps;
 };
 
 inline size_t smem_bytes(int T, int d, int stages) {
@@ -154,6 +158,33 @@ __global__ void __launch_bounds__(kThreads, 1) decode_coop_kernel(const Params p
     {
         for (int i = tid * 8; i < T * d; i += kThreads * 8)
             *reinterpret_cast<uint4 *>(sx + i) = *reinterpret_cast<const uint4 *>(p.x + i);
+        if (p.rms_w) {
+            // RMSNorm of the staged rows, in place: y = h / sqrt(mean(h^2) + eps) . weight, rounded to bf16 as the
+            // layer's input (every CTA normalises all T rows: 2 d values)
+            __syncthreads();
+            float ss[T];
+#pragma unroll
+            for (int t = 0; t < T; ++t) {
+                ss[t] = 0.f;
+                for (int i = tid; i < d; i += kThreads) {
+                    const float v = __bfloat162float(sx[t * d + i]);
+                    ss[t] = fmaf(v, v, ss[t]);
+                }
+                ss[t] = warp_sum(ss[t]);
+            }
+            if (lane == 0)
+#pragma unroll
+                for (int t = 0; t < T; ++t) sz[t * kMaxRows + warp] = ss[t];  // (z is not in use yet)
+            __syncthreads();
+#pragma unroll
+            for (int t = 0; t < T; ++t) {
+                float tot = 0.f;
+                for (int w = 0; w < kThreads / 32; ++w) tot += sz[t * kMaxRows + w];
+                const float scale = rsqrtf(tot / (float)d + p.rms_eps);
+                for (int i = tid; i < d; i += kThreads)
+                    sx[t * d + i] = __float2bfloat16_rn(__bfloat162float(sx[t * d + i]) * scale * __bfloat162float(p.rms_w[i]));
+            }
+        }
         for (int i = tid; i < kMaxRows; i += kThreads) s_mask[i] = 0;
         const int nthr = (int)gridDim.x * kThreads, gtid = (int)blockIdx.x * kThreads + tid;
         for (int i = gtid; i < T * kBins; i += nthr) p.hist[i] = 0u;
@@ -375,8 +406,14 @@ __global__ void __launch_bounds__(kThreads, 1) decode_coop_kernel(const Params p
     {
         const int vecs = T * d / 8;
         for (int v = (int)blockIdx.x * kThreads + tid; v < vecs; v += (int)gridDim.x * kThreads) {
-            const float4 a = __ldcg(reinterpret_cast<const float4 *>(p.acc) + 2 * v);
-            const float4 b = __ldcg(reinterpret_cast<const float4 *>(p.acc) + 2 * v + 1);
+            float4 a = __ldcg(reinterpret_cast<const float4 *>(p.acc) + 2 * v);
+            float4 b = __ldcg(reinterpret_cast<const float4 *>(p.acc) + 2 * v + 1);
+            if (p.rms_w) {  // the residual connection: out = h + D
+                float h8[8];
+                Vec8<__nv_bfloat16>::load(p.x + (size_t)v * 8, h8);
+                a.x += h8[0], a.y += h8[1], a.z += h8[2], a.w += h8[3];
+                b.x += h8[4], b.y += h8[5], b.z += h8[6], b.w += h8[7];
+            }
             reinterpret_cast<uint4 *>(p.out)[v] =
                 make_uint4(tc::pack_bf16(a.x, a.y), tc::pack_bf16(a.z, a.w), tc::pack_bf16(b.x, b.y), tc::pack_bf16(b.z, b.w));
         }

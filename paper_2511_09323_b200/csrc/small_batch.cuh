@@ -90,6 +90,7 @@ struct DownParams {
     int accs;            // 1 or 2: the CTA owns 128 * accs output columns
     float *acc;          // [T, d] fp32, zero on entry
     __nv_bfloat16 *out;  // [T, d]
+    const __nv_bfloat16 *resid;  // [T, d] added to the sums before rounding (the block form's residual), or nullptr
     int *counters;       // [m_tiles], zero on entry, left zero
     int *status;
 };
@@ -626,7 +627,14 @@ __global__ void __launch_bounds__(kThreads, 1) sb_down_kernel(const __grid_const
                 const bool landed = __all_sync(0xffffffffu, tc::mbar_wait(ring.extra(), parity, abort_flag, p.status));
                 for (int i = etid; landed && i < nt * vecs; i += kEpiThreads) {
                     const int t = i / vecs, c = (i - t * vecs) * 4;
-                    const float4 v = *reinterpret_cast<const float4 *>(stage_ptr + (size_t)t * row_bytes + (size_t)c * 4);
+                    float4 v = *reinterpret_cast<const float4 *>(stage_ptr + (size_t)t * row_bytes + (size_t)c * 4);
+                    if (p.resid) {  // out = h + D (out may be h itself: the same thread reads and writes an element)
+                        const uint2 hb = *reinterpret_cast<const uint2 *>(p.resid + (int64_t)(t0 + t) * p.d + col0 + c);
+                        v.x += __uint_as_float(hb.x << 16);
+                        v.y += __uint_as_float(hb.x & 0xffff0000u);
+                        v.z += __uint_as_float(hb.y << 16);
+                        v.w += __uint_as_float(hb.y & 0xffff0000u);
+                    }
                     *reinterpret_cast<uint2 *>(p.out + (int64_t)(t0 + t) * p.d + col0 + c) =
                         make_uint2(tc::pack_bf16(v.x, v.y), tc::pack_bf16(v.z, v.w));
                 }
