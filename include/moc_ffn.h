@@ -79,6 +79,15 @@ typedef enum { MOC_OP_FORWARD = 0, MOC_OP_BACKWARD = 1, MOC_OP_DECODE = 2, MOC_O
  * Honoured by moc_ffn_forward, moc_ffn_decode and moc_ffn_decode_static; moc_ffn_backward takes the saved
  * indices as they are (the flag changes nothing there). */
 #define MOC_FLAG_SELECT_2_OF_8 2u
+/* bit 2: the Top-K operator placed AFTER the activation (Section 6.5, "Effect of top-K position": the ablation whose
+ * other arm is the default): the K channels with the largest SiLU(g) are kept instead of those with the largest g.
+ * The two agree whenever a token has at least K positive gate values (SiLU is increasing there and negative below
+ * zero); they differ on tokens with fewer, where SiLU's minimum near g = -1.28 reorders the negative values.  Keys
+ * are SiLU(g) evaluated in fp32; equal keys: the lower channel; a NaN key (a NaN or -inf gate value) orders as -inf.
+ * What is saved and what the backward pass computes do not change (the mask is taken as saved).  Not combinable with
+ * MOC_FLAG_SELECT_2_OF_8.  This variant runs the exact gathered kernels for every dtype and batch size (it exists
+ * for ablations, not for speed); moc_ffn_decode_block does not take it. */
+#define MOC_FLAG_SELECT_POST_SILU 4u
 
 typedef struct moc_ffn_desc {
     int64_t tokens;   /* T = batch * seq, >= 0 (0 is a no-op)                                   */

@@ -24,6 +24,8 @@
  *                                 the `keep` largest signed pre-SiLU values of every `group` consecutive channels.
  *   moc_oracle_backward           Section 4, Eqs. (bp-1)..(bp-5), with S' and Z' recomputed from the
  *                                 saved G.M and U.M ("MoC + GCP", Table 1).
+ *   moc_oracle_silu_rows          Eq. (silu) element by element: the selection key of the ablation that places the
+ *                                 Top-K operator after the activation (Section 6.5, "Effect of top-K position").
  *   moc_oracle_rmsnorm            Section 2, item "RMSNorm": y = x / RMS(x) . g, RMS(x) = sqrt(mean(x^2) + eps).
  *   moc_oracle_residual           Section 2, item "Residual connections": Z = X + Y.
  *   moc_oracle_silu / dsilu       Eq. (silu) and its derivative.
@@ -443,6 +445,14 @@ int moc_oracle_backward_weight_rows(int64_t T, int32_t d, int32_t F, int32_t K, 
     }
     free(slot);
     return MOC_ORACLE_OK;
+}
+
+/* Eq. (silu) on an array. */
+int moc_oracle_silu_rows(int64_t n, const double *g, double *s)
+{
+    if (n < 0 || !g || !s) return -1;
+    for (int64_t i = 0; i < n; ++i) s[i] = moc_oracle_silu(g[i]);
+    return 0;
 }
 
 /* ---------------------------------------------------------------- the block around the layer */

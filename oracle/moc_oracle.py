@@ -157,6 +157,26 @@ def gate_projection(x, w_gate, F: int | None = None):
     return x @ w_gate[:F].T
 
 
+def silu_rows(g):
+    """SiLU (Eq. (silu)) of every element, float64."""
+    g = _f64(g)
+    s = np.empty_like(g)
+    _check(_load().moc_oracle_silu_rows(ctypes.c_int64(g.size), _p(g), _p(s)), "moc_oracle_silu_rows")
+    return s
+
+
+def forward_post_silu(x, w_gate, w_up, w_down, K: int, F: int | None = None):
+    """The layer with the Top-K operator placed after the activation (Section 6.5, "Effect of top-K position"): the
+    mask keeps the K largest SiLU(g) of a token (equal values: the lower channel); everything else as in `forward`.
+    Returns forward_given_idx's dictionary plus idx, g (gate values) and s (their SiLU: the selection keys)."""
+    G = gate_projection(x, w_gate, F)
+    S = silu_rows(G)
+    idx = topk(S, K)
+    res = forward_given_idx(x, w_gate, w_up, w_down, idx, F)
+    res.update(idx=idx, g=G, s=S)
+    return res
+
+
 def rmsnorm(x, weight, eps: float):
     """y = x / RMS(x) . g per row, RMS(x) = sqrt(mean(x^2) + eps) (Section 2, item "RMSNorm"); [T, d] float64."""
     x, weight = _f64(x), _f64(weight)

@@ -17,12 +17,12 @@ from . import binding as B
 
 class _MoCFFNFunction(torch.autograd.Function):
     @staticmethod
-    def forward(ctx, x, w_gate, w_up, w_down, k, d_ff, grouped, recompute_up):
+    def forward(ctx, x, w_gate, w_up, w_down, k, d_ff, grouped, recompute_up, post_silu=False):
         shape = x.shape
         x2 = x.reshape(-1, shape[-1]).contiguous()
         save = any(ctx.needs_input_grad[:4])
         out, idx, tg, tu = B.moc_ffn_forward(x2, w_gate, w_up, w_down, None if k is None else int(k), d_ff=d_ff,
-                                             save=save, grouped=bool(grouped))
+                                             save=save, grouped=bool(grouped), post_silu=bool(post_silu))
         if save:
             # recompute_up: the up values are dropped here and formed again in backward from x, w_up and the indices
             ctx.save_for_backward(x2, w_gate, w_up, w_down, idx, tg, *(() if recompute_up else (tu,)))
@@ -40,25 +40,27 @@ class _MoCFFNFunction(torch.autograd.Function):
         res = B.moc_ffn_backward(x2, w_gate, w_up, w_down, idx, tg, tu, go, d_ff=ctx.d_ff, want=want)
         gx = res["grad_x"]
         return (None if gx is None else gx.reshape(ctx.x_shape), res["grad_w_gate"], res["grad_w_up"],
-                res["grad_w_down"], None, None, None, None)
+                res["grad_w_down"], None, None, None, None, None)
 
 
 def moc_ffn(x: torch.Tensor, w_gate: torch.Tensor, w_up: torch.Tensor, w_down: torch.Tensor, k: int | None,
-            d_ff: int | None = None, grouped: bool = False, recompute_up: bool = False) -> torch.Tensor:
+            d_ff: int | None = None, grouped: bool = False, recompute_up: bool = False,
+            post_silu: bool = False) -> torch.Tensor:
     """out[..., :] = sum over the k channels j with the largest pre-SiLU gate value x.w_gate[j] of
     SiLU(x.w_gate[j]) * (x.w_up[j]) * w_down[j, :].  `x` is `[..., d_model]`, the weights `[d_ff_ld, d_model]` (rows at and
     past `d_ff`, when given, are padding and never selected).  grouped=True: the 2-of-8 mask of MoC 2:8 (Section 4)
     instead of the row Top-K: the 2 largest of every 8 consecutive channels, k = d_ff / 4.  recompute_up=True keeps only
     the indices and the gate values between forward and backward (k * (2 + e) instead of k * (2 + 2 e) bytes per token)
-    and pays one more up projection in backward."""
-    return _MoCFFNFunction.apply(x, w_gate, w_up, w_down, k, d_ff, grouped, recompute_up)
+    and pays one more up projection in backward.  post_silu=True ranks the channels by SiLU(gate value) instead of the
+    gate value (the paper's ablation of the Top-K position, Section 6.5; exact but slow kernels)."""
+    return _MoCFFNFunction.apply(x, w_gate, w_up, w_down, k, d_ff, grouped, recompute_up, post_silu)
 
 
 class MoCFFN(torch.nn.Module):
     """SwiGLU feed-forward block with Top-K channel selection on the gate (Section 3.2)."""
 
     def __init__(self, d_model: int, d_ff: int, k: int | None, dtype=torch.bfloat16, device="cuda", init_std: float = 0.02,
-                 grouped: bool = False, recompute_up: bool = False):
+                 grouped: bool = False, recompute_up: bool = False, post_silu: bool = False):
         super().__init__()
         if grouped:
             k = B._grouped_k(k, d_ff)
@@ -66,6 +68,7 @@ class MoCFFN(torch.nn.Module):
             raise ValueError("k must be in [1, d_ff]")
         self.d_model, self.d_ff, self.k, self.grouped = int(d_model), int(d_ff), int(k), bool(grouped)
         self.recompute_up = bool(recompute_up)
+        self.post_silu = bool(post_silu)
         mk = lambda: torch.nn.Parameter(torch.empty(d_ff, d_model, dtype=dtype, device=device))
         self.w_gate, self.w_up, self.w_down = mk(), mk(), mk()
         self.reset_parameters(init_std)
@@ -76,7 +79,7 @@ class MoCFFN(torch.nn.Module):
 
     def forward(self, x: torch.Tensor) -> torch.Tensor:
         return moc_ffn(x, self.w_gate, self.w_up, self.w_down, self.k, grouped=self.grouped,
-                       recompute_up=self.recompute_up)
+                       recompute_up=self.recompute_up, post_silu=self.post_silu)
 
     def saved_bytes_per_token(self) -> int:
         """Bytes of activations alive between forward and backward per token, besides x and the output."""
@@ -84,7 +87,7 @@ class MoCFFN(torch.nn.Module):
         return self.k * (2 + (1 if self.recompute_up else 2) * e)
 
     def extra_repr(self) -> str:
-        rule = "2 of every 8" if self.grouped else "row Top-K"
+        rule = "2 of every 8" if self.grouped else "row Top-K after SiLU" if self.post_silu else "row Top-K"
         return f"d_model={self.d_model}, d_ff={self.d_ff}, k={self.k} ({100.0 * self.k / self.d_ff:.1f} % of channels, {rule})"
 
 

@@ -27,6 +27,7 @@ MOC_F32, MOC_BF16 = 0, 1
 MOC_OP_FORWARD, MOC_OP_BACKWARD, MOC_OP_DECODE, MOC_OP_DECODE_BLOCK = 0, 1, 2, 3
 MOC_FLAG_ACCUMULATE_WGRAD = 1
 MOC_FLAG_SELECT_2_OF_8 = 2
+MOC_FLAG_SELECT_POST_SILU = 4
 
 EXPORTED = (
     "moc_ffn_workspace_bytes", "moc_ffn_forward", "moc_ffn_backward", "moc_ffn_decode", "moc_topk_select",
@@ -166,16 +167,17 @@ def _grouped_k(k, d_ff):
 
 
 def moc_ffn_forward(x, w_gate, w_up, w_down, k, d_ff=None, save=True, out=None, saved=None, workspace=None,
-                    stream=None, grouped=False):
+                    stream=None, grouped=False, post_silu=False):
     """Returns (out, topk_idx, topk_gate, topk_up); the last three are None when save=False.
-    grouped=True: the 2-of-8 mask (MOC_FLAG_SELECT_2_OF_8) instead of the row Top-K; k is then d_ff / 4."""
+    grouped=True: the 2-of-8 mask (MOC_FLAG_SELECT_2_OF_8) instead of the row Top-K; k is then d_ff / 4.
+    post_silu=True: the Top-K on SiLU(g) instead of g (MOC_FLAG_SELECT_POST_SILU, the ablation variant)."""
     _check_dev(x, w_gate, w_up, w_down, out, workspace)
     T, d = x.shape
     F_ld = w_gate.shape[0]
     if grouped:
         k = _grouped_k(k, F_ld if d_ff is None else d_ff)
     desc = make_desc(T, d, F_ld if d_ff is None else d_ff, k, x.dtype, d_ff_ld=F_ld,
-                     flags=MOC_FLAG_SELECT_2_OF_8 if grouped else 0)
+                     flags=(MOC_FLAG_SELECT_2_OF_8 if grouped else 0) | (MOC_FLAG_SELECT_POST_SILU if post_silu else 0))
     if out is None:
         out = torch.empty_like(x)
     if save:
@@ -247,14 +249,15 @@ def moc_ffn_recompute_up(x, w_up, topk_idx, d_ff=None, out=None, workspace=None,
     return out
 
 
-def moc_ffn_decode(x, w_gate, w_up, w_down, k, d_ff=None, out=None, workspace=None, stream=None, grouped=False):
+def moc_ffn_decode(x, w_gate, w_up, w_down, k, d_ff=None, out=None, workspace=None, stream=None, grouped=False,
+                   post_silu=False):
     _check_dev(x, w_gate, w_up, w_down, out, workspace)
     T, d = x.shape
     F_ld = w_gate.shape[0]
     if grouped:
         k = _grouped_k(k, F_ld if d_ff is None else d_ff)
     desc = make_desc(T, d, F_ld if d_ff is None else d_ff, k, x.dtype, d_ff_ld=F_ld,
-                     flags=MOC_FLAG_SELECT_2_OF_8 if grouped else 0)
+                     flags=(MOC_FLAG_SELECT_2_OF_8 if grouped else 0) | (MOC_FLAG_SELECT_POST_SILU if post_silu else 0))
     if out is None:
         out = torch.empty_like(x)
     if workspace is None:

@@ -132,7 +132,9 @@ int check_desc(const moc_ffn_desc *d) {
     if (d->tokens < 0 || d->d_model < 1 || d->d_ff < 1 || d->d_ff_ld < d->d_ff || d->k < 1 || d->k > d->d_ff)
         return MOC_ERR_INVALID_ARG;
     if (d->dtype != MOC_F32 && d->dtype != MOC_BF16) return MOC_ERR_UNSUPPORTED;
-    if (d->flags & ~(MOC_FLAG_ACCUMULATE_WGRAD | MOC_FLAG_SELECT_2_OF_8)) return MOC_ERR_INVALID_ARG;
+    if (d->flags & ~(MOC_FLAG_ACCUMULATE_WGRAD | MOC_FLAG_SELECT_2_OF_8 | MOC_FLAG_SELECT_POST_SILU))
+        return MOC_ERR_INVALID_ARG;
+    if ((d->flags & MOC_FLAG_SELECT_2_OF_8) && (d->flags & MOC_FLAG_SELECT_POST_SILU)) return MOC_ERR_INVALID_ARG;
     if ((d->flags & MOC_FLAG_SELECT_2_OF_8) && (d->d_ff % 8 != 0 || d->k != d->d_ff / 4)) return MOC_ERR_INVALID_ARG;
     if (d->d_ff > 32768) return MOC_ERR_UNSUPPORTED;     // int16 channel indices
     if (d->d_model % 8 != 0) return MOC_ERR_UNSUPPORTED;  // 16-byte row vectors
@@ -254,7 +256,8 @@ int forward_gather(const moc_ffn_desc &d, const T *x, const T *wg, const T *wu, 
             const unsigned sel_grid = (unsigned)std::min<int64_t>(n, 148 * 32);
             MOC_LAUNCH(KID_SELECT_ROWS, st,
                        (select_rows_kernel<T><<<sel_grid, kSelectThreads, sel_smem, st>>>(
-                           G, n, F, F, K, idx + t0 * K, tg ? tg + t0 * K : nullptr)));
+                           G, n, F, F, K, idx + t0 * K, tg ? tg + t0 * K : nullptr,
+                           (d.flags & MOC_FLAG_SELECT_POST_SILU) ? 1 : 0)));
         }
         if ((rc = launch_ok()) != MOC_OK) return rc;
         MOC_LAUNCH(KID_FORWARD_TOKEN, st,
@@ -323,6 +326,10 @@ bool use_tc_plan(const moc_ffn_desc &d) {
     // the forward selector keeps F keys and K packed entries in shared memory
     return ((size_t)d.d_ff + (size_t)d.k) * 4 <= 170 * 1024;
 }
+
+// The forward pass of the tensor-core plan selects on the gate values themselves: the post-SiLU ablation variant
+// takes the gathered kernels (the backward pass does not select and keeps its plan).
+bool use_tc_forward(const moc_ffn_desc &d) { return use_tc_plan(d) && !(d.flags & MOC_FLAG_SELECT_POST_SILU); }
 
 inline int ceil_div(int64_t a, int64_t b) { return (int)((a + b - 1) / b); }
 
@@ -659,7 +666,7 @@ bool use_small_batch_plan(const moc_ffn_desc &d);
 bool small_batch_preferred(const moc_ffn_desc &d);
 
 bool use_decode_plan(const moc_ffn_desc &d) {
-    return d.dtype == MOC_BF16 && d.tokens >= 1 && d.tokens <= 16 && d.d_model <= 256 * dec::kSliceCols &&
+    return !(d.flags & MOC_FLAG_SELECT_POST_SILU) && d.dtype == MOC_BF16 && d.tokens >= 1 && d.tokens <= 16 && d.d_model <= 256 * dec::kSliceCols &&
            !(use_small_batch_plan(d) && small_batch_preferred(d));
 }
 
@@ -903,7 +910,7 @@ bool small_batch_preferred(const moc_ffn_desc &d) {
 // moc_ffn_forward takes the small-batch plan for every bf16 batch it can serve (the tensor-core plan's tiles need
 // thousands of tokens); moc_ffn_decode takes it where small_batch_preferred says so, else the decode plan.
 bool use_small_batch_plan(const moc_ffn_desc &d) {
-    return d.dtype == MOC_BF16 && d.tokens >= 1 && d.tokens <= sb::kMaxTokens &&
+    return !(d.flags & MOC_FLAG_SELECT_POST_SILU) && d.dtype == MOC_BF16 && d.tokens >= 1 && d.tokens <= sb::kMaxTokens &&
            sb::select_smem(d.d_ff, false) + 48 * 1024 <= (size_t)kMaxDynSmem;
 }
 
@@ -1061,7 +1068,7 @@ size_t moc_ffn_workspace_bytes(const moc_ffn_desc *desc, int op) {
             // fall through: the forward with nothing saved
         case MOC_OP_FORWARD:
             if (use_small_batch_plan(*desc)) return small_batch_layout(*desc).total;
-            return use_tc_plan(*desc) ? tc::tc_forward_layout(*desc).total : plan_forward(*desc).total;
+            return use_tc_forward(*desc) ? tc::tc_forward_layout(*desc).total : plan_forward(*desc).total;
         case MOC_OP_BACKWARD:
             return use_tc_plan(*desc) ? tc::tc_backward_layout(*desc).total : plan_backward(*desc).total;
         case MOC_OP_DECODE_BLOCK: {
@@ -1102,7 +1109,7 @@ int moc_ffn_forward(const moc_ffn_desc *desc, const void *x, const void *w_gate,
         if (use_small_batch_plan(*desc))
             return forward_small_batch(*desc, (const T *)x, (const T *)w_gate, (const T *)w_up, (const T *)w_down,
                                        (T *)out, topk_idx, (T *)topk_gate, (T *)topk_up, ws, st);
-        if (use_tc_plan(*desc))
+        if (use_tc_forward(*desc))
             return forward_tc(*desc, (const T *)x, (const T *)w_gate, (const T *)w_up, (const T *)w_down, (T *)out,
                               topk_idx, (T *)topk_gate, (T *)topk_up, ws, st);
         return forward_gather<T>(*desc, (const T *)x, (const T *)w_gate, (const T *)w_up, (const T *)w_down,

@@ -77,7 +77,7 @@ template <typename T>
 __global__ void __launch_bounds__(kSelectThreads) select_rows_kernel(const float *__restrict__ G, int64_t rows,
                                                                       int F, int ldg, int K,
                                                                       int16_t *__restrict__ idx_out,
-                                                                      T *__restrict__ topk_gate) {
+                                                                      T *__restrict__ topk_gate, int post_silu) {
     extern __shared__ __align__(16) uint32_t select_keys[];
     __shared__ SelectSmem sm;
     SelectGuess guess;
@@ -85,14 +85,15 @@ __global__ void __launch_bounds__(kSelectThreads) select_rows_kernel(const float
         const float *g = G + r * (int64_t)ldg;
         uint32_t tau;
         int need;
-        block_select_row<kSelectThreads>(g, F, K, select_keys, sm, guess, tau, need);
+        block_select_row<kSelectThreads>(g, F, K, select_keys, sm, guess, tau, need, post_silu != 0);
         int16_t *o = idx_out + r * (int64_t)K;
         T *og = topk_gate ? topk_gate + r * (int64_t)K : nullptr;
         block_ordered_emit<kSelectThreads>(select_keys, F, tau, need, sm, [&](int pos, int j) {
             o[pos] = (int16_t)j;
             // the value comes back from the key in shared memory: a global load inside the ordered walk
             // would cost a memory round trip per chunk
-            if (og) og[pos] = from_f32<T>(key_to_float(select_keys[j]));
+            // (keys of SiLU(g) do not give g back: the post-SiLU variant reads it)
+            if (og) og[pos] = from_f32<T>(post_silu ? g[j] : key_to_float(select_keys[j]));
         });
         __syncthreads();
     }

@@ -162,7 +162,7 @@ __device__ __forceinline__ float key_to_float(uint32_t key) {
 template <int THREADS>
 __device__ __forceinline__ void block_select_row(const float *__restrict__ g, int n, int k, uint32_t *keys,
                                                  SelectSmemT<THREADS / 32> &sm, SelectGuess &guess, uint32_t &tau,
-                                                 int &need) {
+                                                 int &need, bool post_silu = false) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     uint32_t lo = 1u, hi = 0u;  // empty bracket
     if (guess.valid) {
@@ -176,7 +176,7 @@ __device__ __forceinline__ void block_select_row(const float *__restrict__ g, in
         const int j = base + tid;
         uint32_t key = 0u;
         if (j < n) {
-            key = gate_key(g[j]);
+            key = gate_key(post_silu ? silu_f(g[j]) : g[j]);  // the key the ranking uses: g, or SiLU(g)
             keys[j] = key;
         }
         if (guess.valid) {

@@ -132,3 +132,20 @@ def test_recompute_up_option_of_the_module_and_bad_indices():
     mask = torch.ones_like(got, dtype=torch.bool)
     mask[3, 2] = mask[7, 0] = False
     assert torch.equal(got[mask], good[mask])
+
+
+def test_module_post_silu_option_matches_direct_calls():
+    """post_silu=True reaches the library (MOC_FLAG_SELECT_POST_SILU) through the module, forward and backward."""
+    torch.manual_seed(7)
+    m = MoCFFN(64, 256, 32, dtype=torch.float32, post_silu=True)
+    with torch.no_grad():
+        m.w_gate -= 0.05   # with x > 0 below most gate values are negative: the two rules differ
+    x = (torch.rand(24, 64, device="cuda") + 0.5).requires_grad_(True)
+    y = m(x)
+    y.sum().backward()
+    out, idx, tg, tu = B.moc_ffn_forward(x.detach(), m.w_gate.detach(), m.w_up.detach(), m.w_down.detach(), 32, post_silu=True)
+    default = B.moc_ffn_forward(x.detach(), m.w_gate.detach(), m.w_up.detach(), m.w_down.detach(), 32)
+    assert torch.equal(y.detach(), out)
+    assert not torch.equal(idx, default[1])
+    g = B.moc_ffn_backward(x.detach(), m.w_gate.detach(), m.w_up.detach(), m.w_down.detach(), idx, tg, tu, torch.ones_like(out))
+    assert torch.equal(x.grad, g["grad_x"]) and torch.equal(m.w_down.grad, g["grad_w_down"])

@@ -562,3 +562,46 @@ def test_residual_and_block_composition():
     out3, x3, f3 = orc.decode_block(h, g, 1e-5, wg, wu, wd, K, store=coarse)
     np.testing.assert_array_equal(x3, coarse(orc.rmsnorm(h, g, 1e-5)))
     np.testing.assert_allclose(out3, h + orc.forward(x3, wg, wu, wd, K)["out"], rtol=1e-13, atol=1e-14)
+
+
+# --------------------------------------------------------------------------- Top-K after the activation (Section 6.5)
+
+def test_post_silu_selection_equals_pre_silu_when_enough_gates_are_positive():
+    """SiLU is increasing and positive on g > 0 and negative on g < 0, so with at least K positive gate values the
+    K largest SiLU(g) are the K largest g."""
+    rng = np.random.default_rng(31)
+    T, d, F, K = 6, 16, 48, 9
+    x = rng.standard_normal((T, d))
+    wg, wu, wd = (rng.standard_normal((F, d)) * 0.3 for _ in range(3))
+    G = x @ wg.T
+    assert (G > 0).sum(axis=1).min() >= K
+    post, pre = orc.forward_post_silu(x, wg, wu, wd, K), orc.forward(x, wg, wu, wd, K)
+    np.testing.assert_array_equal(post["idx"], pre["idx"])
+    np.testing.assert_allclose(post["out"], pre["out"], rtol=1e-13, atol=1e-14)
+    np.testing.assert_allclose(post["s"], G * expit(G), rtol=1e-13, atol=1e-300)
+
+
+def test_post_silu_selection_differs_where_it_must():
+    """One token, hand-made gate values through an identity gate matrix.  Only two are positive; with K = 4 the other
+    two picks are the negative values whose SiLU is closest to zero: g = -0.01 (SiLU -0.00497..) and g = -12
+    (SiLU -7.4e-5), not g = -0.5 (-0.189) or g = -1.3 (-0.279), while the pre-SiLU rule takes -0.01 and -0.5."""
+    g = np.array([[2.0, -0.5, -12.0, 0.3, -1.3, -0.01, -3.0, -0.8]])
+    F = g.shape[1]
+    eye = np.eye(F)
+    wu, wd = np.ones((F, F)), np.eye(F)
+    post = orc.forward_post_silu(g, eye, wu, wd, 4)
+    pre = orc.forward(g, eye, wu, wd, 4)
+    np.testing.assert_array_equal(post["idx"], [[0, 2, 3, 5]])
+    np.testing.assert_array_equal(pre["idx"], [[0, 1, 3, 5]])
+    # brute force over all subsets of size 4: the kept set maximises the sum of SiLU(g)
+    import itertools
+    s = g[0] * expit(g[0])
+    best = max(itertools.combinations(range(F), 4), key=lambda c: s[list(c)].sum())
+    assert list(best) == post["idx"][0].tolist()
+    # the output is Eq. (MoC-2) on that mask: u = sum(g) for every channel, W_down = I
+    expect = np.zeros(F)
+    expect[list(best)] = s[list(best)] * g.sum()
+    np.testing.assert_allclose(post["out"][0], expect, rtol=1e-13, atol=1e-15)
+    # equal keys: the lower channel (two channels with the same gate value on the threshold)
+    tie = orc.forward_post_silu(np.array([[1.0, -2.0, -2.0, -0.1]]), np.eye(4), np.ones((4, 4)), np.eye(4), 3)
+    np.testing.assert_array_equal(tie["idx"], [[0, 1, 3]])
