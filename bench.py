@@ -458,6 +458,10 @@ def run_ours(args):
                              "forward_ms_min_median": [min(fwd_ms), statistics.median(fwd_ms)],
                              "backward_ms_min_median": [min(bwd_ms), statistics.median(bwd_ms)]},
             "act_bytes": act_bytes_report(w, T, e, saved, B, desc),
+            # tokens whose K-th largest gate value is positive: for those the Top-K before SiLU (what runs) and after
+            # SiLU (the paper's ablation arm) keep the same channels
+            "selection": {"tokens": T, "tokens_with_positive_threshold":
+                          int((saved[1].float().min(dim=1).values > 0).sum().item())},
             "strict_roofline": strict_roofline(w, T, e, worst_ms / args.steps, peaks),
         }
     # ---- the MoC 2:8 variant on the same layer (rank 0; extra information, not the headline) ---------
