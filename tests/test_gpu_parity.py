@@ -435,12 +435,34 @@ def test_tc_plan_corrupted_saved_index_is_skipped_and_reported():
         assert torch.isfinite(g[k].float()).all()
 
 
-def _full_size_sampled(w, n_tokens, n_rows):
+def _full_size_sampled(w, n_tokens, n_rows, graph=False):
     x, wg, wu, wd, dD = _problem(w)
     xd, wgd, wud, wdd, dDd = map(_dev, (x, wg, wu, wd, dD))
     out, idx, tg, tu = B.moc_ffn_forward(xd, wgd, wud, wdd, w.k, d_ff=w.d_ff)
     grads = B.moc_ffn_backward(xd, wgd, wud, wdd, idx, tg, tu, dDd, d_ff=w.d_ff)
     torch.cuda.synchronize()
+    if graph:
+        # the launch configuration bench.py times: both calls captured once into a CUDA graph (preallocated outputs
+        # and workspaces, a side stream) and replayed; the buffers are cleared first so that what is checked below
+        # was written by the replays
+        names = ("grad_x", "grad_w_gate", "grad_w_up", "grad_w_down")
+        desc = B.make_desc(w.tokens, w.d_model, w.d_ff, w.k, xd.dtype, d_ff_ld=w.d_ff_ld)
+        ws_f = B.alloc_workspace(desc, B.MOC_OP_FORWARD, xd.device)
+        ws_b = B.alloc_workspace(desc, B.MOC_OP_BACKWARD, xd.device)
+        stream = torch.cuda.Stream()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(stream):
+            with torch.cuda.graph(g, stream=stream):
+                B.moc_ffn_forward(xd, wgd, wud, wdd, w.k, d_ff=w.d_ff, out=out, saved=(idx, tg, tu), workspace=ws_f,
+                                  stream=stream)
+                B.moc_ffn_backward(xd, wgd, wud, wdd, idx, tg, tu, dDd, d_ff=w.d_ff, grads=grads, workspace=ws_b,
+                                   stream=stream)
+        torch.cuda.synchronize()
+        for t in (out, idx, tg, tu, *(grads[n] for n in names)):
+            t.zero_()
+        g.replay()
+        g.replay()
+        torch.cuda.synchronize()
     assert B.moc_last_device_status() == B.MOC_OK
     rng = np.random.default_rng(0)
     toks = np.sort(rng.choice(w.tokens, n_tokens, replace=False))
@@ -468,6 +490,40 @@ def test_full_size_bench_workload_sampled_against_oracle():
     """C2 at its full 16384 tokens, in the configuration bench.py times: sampled tokens of out / saved values /
     grad_x and sampled rows of the weight gradients are recomputed one by one by the oracle."""
     _full_size_sampled(syn.C2, 96, 24)
+
+
+def test_full_size_bench_workload_replayed_from_a_cuda_graph():
+    """The same comparison on the outputs of a CUDA graph replay of forward + backward (how bench.py launches them)."""
+    _full_size_sampled(syn.C2, 48, 12, graph=True)
+
+
+@pytest.mark.parametrize("T", [1, 2, 4, 16, 64])
+def test_decode_replayed_from_a_cuda_graph_with_rotating_weights(T):
+    """bench.py's decode timing replays a CUDA graph of calls that rotate weight sets: every plan (the cooperative
+    kernel, the four-kernel chain, the small-batch kernels) must give under replay what its direct call gives."""
+    w = syn.C4.with_tokens(T)
+    sets = [tuple(t.cuda() for t in syn.make_weights(w, seed_offset=s)) for s in range(2)]
+    x = syn.make_x(w).cuda()
+    desc = B.make_desc(T, w.d_model, w.d_ff, w.k, x.dtype)
+    ws = B.alloc_workspace(desc, B.MOC_OP_DECODE, x.device)
+    direct = [B.moc_ffn_decode(x, *sets[i], w.k, workspace=ws).clone() for i in range(2)]
+    torch.cuda.synchronize()
+    outs = [torch.zeros_like(x) for _ in range(4)]
+    stream = torch.cuda.Stream()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        with torch.cuda.graph(g, stream=stream):
+            for i in range(4):
+                B.moc_ffn_decode(x, *sets[i % 2], w.k, out=outs[i], workspace=ws, stream=stream)
+    torch.cuda.synchronize()
+    for o in outs:
+        o.zero_()
+    g.replay()
+    g.replay()
+    torch.cuda.synchronize()
+    assert B.moc_last_device_status() == B.MOC_OK
+    for i in range(4):   # the partial sums meet in an order that is not fixed: last-bit differences only
+        torch.testing.assert_close(outs[i].float(), direct[i % 2].float(), rtol=2e-2, atol=2e-3)
 
 
 def test_full_size_llama1b_padded_sampled_against_oracle():
