@@ -108,6 +108,35 @@ def test_null_pointers_and_small_workspace_are_rejected_before_launch(lib):
     assert lib.moc_topk_select(0, 8, 8, 2, None, None, None) == B.MOC_OK
 
 
+def test_block_form_and_selection_flags_are_validated_on_the_host(lib):
+    fake = ctypes.c_void_p(0x1000)
+    eps = ctypes.c_float(1e-6)
+    block = lambda d, *ptrs, ws=None, n=0, e=eps: lib.moc_ffn_decode_block(ctypes.byref(d), ptrs[0], ptrs[1], e, *ptrs[2:],
+                                                                         ws, n, None)
+    zero = B.make_desc(0, 16, 32, 8, B.MOC_BF16)
+    assert block(zero, *([None] * 6)) == B.MOC_OK                       # no tokens: a no-op that needs no buffers
+    f32 = B.make_desc(4, 16, 32, 8, B.MOC_F32)
+    assert B.moc_ffn_workspace_bytes(f32, B.MOC_OP_DECODE_BLOCK) == 0   # bf16 only
+    assert block(f32, *([fake] * 6)) == B.MOC_ERR_UNSUPPORTED
+    big = B.make_desc(257, 16, 32, 8, B.MOC_BF16)
+    assert block(big, *([fake] * 6)) == B.MOC_ERR_UNSUPPORTED           # at most 256 tokens
+    d = B.make_desc(4, 16, 32, 8, B.MOC_BF16)
+    need = B.moc_ffn_workspace_bytes(d, B.MOC_OP_DECODE_BLOCK)
+    assert need > B.moc_ffn_workspace_bytes(d, B.MOC_OP_DECODE) > 0     # the normalised rows live behind the decode workspace
+    assert block(d, *([None] * 6)) == B.MOC_ERR_INVALID_ARG
+    assert block(d, *([fake] * 6), e=ctypes.c_float(-1.0)) == B.MOC_ERR_INVALID_ARG
+    assert block(d, *([fake] * 6)) == B.MOC_ERR_WORKSPACE
+    assert block(d, *([fake] * 6), ws=fake, n=need - 1) == B.MOC_ERR_WORKSPACE
+    # selection flags: the two rules exclude each other; the post-SiLU variant has no block form
+    both = B.make_desc(4, 16, 32, 8, B.MOC_BF16, flags=B.MOC_FLAG_SELECT_2_OF_8 | B.MOC_FLAG_SELECT_POST_SILU)
+    assert lib.moc_ffn_forward(ctypes.byref(both), *([None] * 9), 0, None) == B.MOC_ERR_INVALID_ARG
+    post = B.make_desc(4, 16, 32, 8, B.MOC_BF16, flags=B.MOC_FLAG_SELECT_POST_SILU)
+    assert B.moc_ffn_workspace_bytes(post, B.MOC_OP_FORWARD) > 0
+    assert B.moc_ffn_workspace_bytes(post, B.MOC_OP_DECODE) > 0
+    assert B.moc_ffn_workspace_bytes(post, B.MOC_OP_DECODE_BLOCK) == 0
+    assert block(post, *([fake] * 6)) == B.MOC_ERR_UNSUPPORTED
+
+
 def test_binding_fails_loudly_without_library(monkeypatch, tmp_path):
     monkeypatch.setattr(B, "_lib", None)
     monkeypatch.setattr(B, "LIB_PATH", str(tmp_path / "missing.so"))
