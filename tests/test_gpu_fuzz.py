@@ -1,0 +1,92 @@
+"""Seeded random shapes through every entry point: forward + backward, decode and the block form against the oracle.
+The fixed cases of the other files pin known corners; this sweep walks the plan boundaries (1 ... 300 tokens, ragged
+widths, padded weight rows, K from 1 to d_ff) with shapes nobody chose by hand."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import moc_oracle as orc
+from oracle import parity
+from paper_2511_09323_b200 import binding as B
+from paper_2511_09323_b200 import build as moc_build
+from paper_2511_09323_b200 import synthetic as syn
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    moc_build.build()
+    B.load()
+    assert B.moc_last_device_status() == B.MOC_OK
+    yield
+    assert B.moc_last_device_status() == B.MOC_OK
+
+
+def _random_workloads(n, seed):
+    rng = np.random.default_rng(seed)
+    out = []
+    for i in range(n):
+        dtype = "bf16" if rng.random() < 0.75 else "f32"
+        T = int(rng.choice([1, 2, 3, 5, 6, 16, 17, 31, 64, 100, 129, 256, 257, 300]))
+        d = 8 * int(rng.integers(1, 66))
+        F = int(rng.integers(8, 1500 if dtype == "f32" else 3000))
+        F_ld = F + 8 * int(rng.integers(0, 3)) if rng.random() < 0.4 else F
+        F_ld = (F_ld + 7) // 8 * 8 if F_ld > F else F_ld
+        K = int(rng.integers(1, F + 1)) if rng.random() < 0.3 else max(1, int(F * rng.uniform(0.03, 0.3)))
+        out.append(syn.Workload(f"fuzz-{seed}-{i}", dtype, T, d, F, F_ld, K, seed=7000 + 31 * seed + i))
+    return out
+
+
+def _band_check(out64, full, x64, wg64, wu64, wd64, K, F, dtype, what, base=None):
+    """Rows of `out64` against the oracle's; a token whose K-th and (K+1)-th gate values nearly tie may have taken the
+    swapped pick.  `base`: what is added to the layer's output (the residual stream of the block form)."""
+    ref = full["out"] if base is None else base + full["out"]
+    tol = parity.REL_TOL[dtype] * max(np.abs(ref).max(), 1e-30)
+    for t in range(out64.shape[0]):
+        err = np.abs(out64[t] - ref[t]).max()
+        if err <= tol:
+            continue
+        g = full["g"][t]
+        order = np.lexsort((np.arange(F), -g))
+        assert K < F and g[order[K - 1]] - g[order[K]] <= 1e-3, f"{what}: token {t} error {err:.3e} > {tol:.3e}"
+        alt = np.sort(np.concatenate([order[: K - 1], order[K: K + 1]])).astype(np.int32)[None]
+        alt_out = orc.forward_given_idx(x64[t: t + 1], wg64, wu64, wd64, alt)["out"][0]
+        if base is not None:
+            alt_out = base[t] + alt_out
+        assert np.abs(out64[t] - alt_out).max() <= tol, f"{what}: token {t} matches neither pick"
+
+
+@pytest.mark.parametrize("w", _random_workloads(28, 1), ids=lambda w: f"{w.dtype}-T{w.tokens}-d{w.d_model}-F{w.d_ff}of{w.d_ff_ld}-K{w.k}")
+def test_random_shape_forward_backward_decode(w):
+    wg, wu, wd = syn.make_weights(w)
+    x, dD = syn.make_x(w), syn.make_grad_out(w)
+    xd, wgd, wud, wdd, dDd = (t.cuda() for t in (x, wg, wu, wd, dD))
+    F, K = w.d_ff, w.k
+    out, idx, tg, tu = B.moc_ffn_forward(xd, wgd, wud, wdd, K, d_ff=F)
+    grads = B.moc_ffn_backward(xd, wgd, wud, wdd, idx, tg, tu, dDd, d_ff=F)
+    torch.cuda.synchronize()
+    x64, wg64, wu64, wd64, dD64 = map(syn.to_f64, (x, wg[:F], wu[:F], wd[:F], dD))
+    dev = dict(out=syn.to_f64(out), idx=idx.cpu().numpy(), gval=syn.to_f64(tg), uval=syn.to_f64(tu))
+    parity.check_forward(dev, x64, wg64, wu64, wd64, K, F, w.dtype)
+    gdev = {k: syn.to_f64(v) for k, v in grads.items()}
+    parity.check_backward(gdev, x64, wg64, wu64, wd64, dev["idx"], dev["gval"], dev["uval"], dD64, F, w.dtype)
+    if w.d_ff_ld > F:
+        for name in ("grad_w_gate", "grad_w_up", "grad_w_down"):
+            assert torch.all(grads[name][F:] == 0), name
+    if w.tokens <= 256:
+        full = orc.forward(x64, wg64, wu64, wd64, K, want_g=True)
+        out_d = B.moc_ffn_decode(xd, wgd, wud, wdd, K, d_ff=F)
+        torch.cuda.synchronize()
+        _band_check(syn.to_f64(out_d), full, x64, wg64, wu64, wd64, K, F, w.dtype, "decode")
+        desc = B.make_desc(w.tokens, w.d_model, F, K, xd.dtype, d_ff_ld=w.d_ff_ld)
+        if B.moc_ffn_workspace_bytes(desc, B.MOC_OP_DECODE_BLOCK) > 0:
+            gen = torch.Generator().manual_seed(w.seed + 5)
+            h = (torch.randn(w.tokens, w.d_model, generator=gen) * 2.0).to(torch.bfloat16)
+            gamma = (0.5 + torch.rand(w.d_model, generator=gen)).to(torch.bfloat16)
+            out_b = B.moc_ffn_decode_block(h.cuda(), gamma.cuda(), 1e-5, wgd, wud, wdd, K, d_ff=F)
+            torch.cuda.synchronize()
+            h64 = syn.to_f64(h)
+            store = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(torch.bfloat16).double().numpy()
+            _, xn, fb = orc.decode_block(h64, syn.to_f64(gamma), 1e-5, wg64, wu64, wd64, K, store=store)
+            _band_check(syn.to_f64(out_b), fb, xn, wg64, wu64, wd64, K, F, "bf16", "block", base=h64)
