@@ -90,3 +90,34 @@ def test_random_shape_forward_backward_decode(w):
             store = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(torch.bfloat16).double().numpy()
             _, xn, fb = orc.decode_block(h64, syn.to_f64(gamma), 1e-5, wg64, wu64, wd64, K, store=store)
             _band_check(syn.to_f64(out_b), fb, xn, wg64, wu64, wd64, K, F, "bf16", "block", base=h64)
+
+
+def test_random_rows_through_the_selector_hook_are_bit_exact():
+    """`moc_topk_select` on 48 seeded random problems (row counts either side of the 256-row switch between the two
+    selectors, widths up to the int16 limit, duplicates, all-equal rows, tiny values, NaN / +-inf / -0): the indices
+    must equal the oracle's on the same fp32 array."""
+    rng = np.random.default_rng(11)
+    for i in range(48):
+        rows = int(rng.choice([1, 3, 17, 200, 256, 257, 700]))
+        n = int(rng.integers(1, 12000)) if rng.random() < 0.8 else int(rng.integers(12000, 32768))
+        n_ld = n + int(rng.integers(0, 9))
+        k = int(rng.integers(1, n + 1)) if rng.random() < 0.3 else max(1, int(n * rng.uniform(0.01, 0.3)))
+        mode = int(rng.integers(0, 6))
+        g = rng.standard_normal((rows, n_ld)).astype(np.float32)
+        if mode == 1:
+            g = np.round(g * 4) / 4            # heavy duplicates
+        elif mode == 2:
+            g = np.round(g * 64) / 64
+        elif mode == 3:
+            g[:] = g[:, :1]                    # every row a constant
+        elif mode == 4:
+            g = np.abs(g) * 1e-30              # tiny values
+        elif mode == 5:
+            g[rng.random(g.shape) < 0.01] = np.nan
+            g[rng.random(g.shape) < 0.01] = -np.inf
+            g[rng.random(g.shape) < 0.005] = np.inf
+            g[rng.random(g.shape) < 0.02] = -0.0
+        g = np.ascontiguousarray(g.astype(np.float32))
+        ref = orc.topk(g, k, F=n)
+        got = B.moc_topk_select(torch.from_numpy(g).cuda(), k, n=n).cpu().numpy().astype(np.int32)
+        assert np.array_equal(ref, got), f"problem {i}: rows={rows} n={n} n_ld={n_ld} k={k} mode={mode}"
