@@ -121,3 +121,27 @@ def test_random_rows_through_the_selector_hook_are_bit_exact():
         ref = orc.topk(g, k, F=n)
         got = B.moc_topk_select(torch.from_numpy(g).cuda(), k, n=n).cpu().numpy().astype(np.int32)
         assert np.array_equal(ref, got), f"problem {i}: rows={rows} n={n} n_ld={n_ld} k={k} mode={mode}"
+
+
+@pytest.mark.parametrize("dtype,T,d,F,F_ld,K", [
+    ("bf16", 1, 8192, 512, 512, 64),        # d_model beyond the cooperative kernel's 4096 columns: four-kernel plan
+    ("bf16", 2, 8192, 520, 520, 65),
+    ("bf16", 4, 8192, 512, 512, 64),
+    ("bf16", 20, 8192, 512, 512, 64),       # small-batch plan, 128 contraction blocks
+    ("bf16", 300, 8192, 512, 512, 64),      # tensor-core plan
+    ("bf16", 1, 16384, 256, 256, 32),
+    ("bf16", 5, 12288, 256, 256, 32),
+    ("bf16", 40, 16384, 264, 264, 33),
+    ("f32", 3, 8192, 256, 256, 32),
+    ("bf16", 1, 8, 8, 8, 1),                # the smallest of everything
+    ("bf16", 1, 8, 16, 16, 16),             # K = d_ff on the decode path
+    ("bf16", 256, 8, 8, 8, 8),
+    ("bf16", 3, 4104, 300, 304, 7),         # one 8-column step past 4096, padded weight rows
+    ("bf16", 2, 4096, 32768, 32768, 4096),  # the int16 limit of d_ff on the cooperative kernel
+    ("bf16", 1, 64, 32768, 32768, 1),
+    ("bf16", 16, 64, 32760, 32768, 4000),
+    ("bf16", 200, 64, 30000, 30000, 3000),
+])
+def test_extreme_shapes(dtype, T, d, F, F_ld, K):
+    test_random_shape_forward_backward_decode(
+        syn.Workload(f"extreme-{T}-{d}-{F}", dtype, T, d, F, F_ld, K, seed=9500 + T + d + F))
