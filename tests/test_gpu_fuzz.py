@@ -145,3 +145,49 @@ def test_random_rows_through_the_selector_hook_are_bit_exact():
 def test_extreme_shapes(dtype, T, d, F, F_ld, K):
     test_random_shape_forward_backward_decode(
         syn.Workload(f"extreme-{T}-{d}-{F}", dtype, T, d, F, F_ld, K, seed=9500 + T + d + F))
+
+
+@pytest.mark.parametrize("T,d,F,K", [(1, 520, 776, 97), (2, 520, 776, 97), (4, 264, 333, 41), (16, 768, 2048, 256),
+                                     (40, 768, 2048, 256), (300, 768, 2048, 256)])
+def test_results_do_not_depend_on_what_the_workspace_held(T, d, F, K):
+    """Every operation with a workspace of zeros, of 0xff bytes and of random bytes: the same results (up to the
+    order in which partial sums meet); decode twice in a row on the same workspace as well."""
+    w = syn.Workload("ws", "bf16", T, d, F, (F + 7) // 8 * 8, K, seed=321 + T)
+    wg, wu, wd = (t.cuda() for t in syn.make_weights(w))
+    x, dD = syn.make_x(w).cuda(), syn.make_grad_out(w).cuda()
+    desc = B.make_desc(T, d, F, K, x.dtype, d_ff_ld=w.d_ff_ld)
+    saved = B.moc_ffn_forward(x, wg, wu, wd, K, d_ff=F)
+    gamma = torch.ones(d, dtype=x.dtype, device="cuda")
+
+    def run(op, ws):
+        if op == B.MOC_OP_FORWARD:
+            o = B.moc_ffn_forward(x, wg, wu, wd, K, d_ff=F, workspace=ws)
+            return [o[0].clone(), o[1].float(), o[2].clone(), o[3].clone()]
+        if op == B.MOC_OP_BACKWARD:
+            g = B.moc_ffn_backward(x, wg, wu, wd, saved[1], saved[2], saved[3], dD, d_ff=F, workspace=ws)
+            return [g[k].clone() for k in sorted(g)]
+        if op == B.MOC_OP_DECODE:
+            return [B.moc_ffn_decode(x, wg, wu, wd, K, d_ff=F, workspace=ws).clone(),
+                    B.moc_ffn_decode(x, wg, wu, wd, K, d_ff=F, workspace=ws).clone()]
+        return [B.moc_ffn_decode_block(x, gamma, 1e-5, wg, wu, wd, K, d_ff=F, workspace=ws).clone()]
+
+    gen = torch.Generator(device="cuda").manual_seed(5)
+    for op in (B.MOC_OP_FORWARD, B.MOC_OP_BACKWARD, B.MOC_OP_DECODE, B.MOC_OP_DECODE_BLOCK):
+        n = B.moc_ffn_workspace_bytes(desc, op)
+        if n == 0:
+            continue
+        results = []
+        for fill in ("zero", "ff", "random"):
+            ws = torch.empty(n, dtype=torch.uint8, device="cuda")
+            if fill == "zero":
+                ws.zero_()
+            elif fill == "ff":
+                ws.fill_(0xff)
+            else:
+                ws.copy_(torch.randint(0, 256, (n,), dtype=torch.uint8, device="cuda", generator=gen))
+            results.append(run(op, ws))
+        torch.cuda.synchronize()
+        for other in results[1:]:
+            for a, b in zip(other, results[0]):
+                torch.testing.assert_close(a.float(), b.float(), rtol=2e-2, atol=2e-3 * max(1.0, b.float().abs().max().item()))
+    assert B.moc_last_device_status() == B.MOC_OK
