@@ -20,6 +20,8 @@
  *   moc_oracle_topk               the mask definition of Section 3.2: exactly K ones per row,
  *                                 the K largest SIGNED pre-SiLU values.
  *   moc_oracle_forward_given_idx  Eq. (MoC-2) with the mask M supplied by the caller.
+ *   moc_oracle_gate_projection    Eq. (Moc-1), G = X W_gate, on its own (the variants that select with another rule
+ *                                 start from it).
  *   moc_oracle_topk_grouped       the a:b mask of Section 4 ("MoC with structured 2:8 sparsity") and Theorem 1:
  *                                 the `keep` largest signed pre-SiLU values of every `group` consecutive channels.
  *   moc_oracle_backward           Section 4, Eqs. (bp-1)..(bp-5), with S' and Z' recomputed from the
@@ -33,7 +35,7 @@
  *   moc_oracle_saved_elems_*      Table 1: 4 d_ffn (FFN), 2 d_ffn (FFN+GCP), d_ffn-equivalent 5K (MoC),
  *                                 3K (MoC+GCP) stored elements per token, each plus d for D.
  *
- * Readings where the paper is silent (all also listed in the design notes):
+ * Readings where the paper is silent:
  *   - ties at the K-th value go to the lower channel index; -0.0 equals +0.0;
  *   - NaN gate values are ordered as -infinity (lowest), so selection never depends on NaN compares;
  *   - indices of a token are reported in ascending channel order;
@@ -231,6 +233,16 @@ static void token_given_idx(const double *xt, const double *w_gate, const double
         if (gval_t) gval_t[k] = g;
         if (uval_t) uval_t[k] = u;
     }
+}
+
+/* G = X W_gate (Eq. (Moc-1)) for the first F channels: g [T,F], the same sequential dot products the forward uses. */
+int moc_oracle_gate_projection(int64_t T, int32_t d, int32_t F, const double *x, const double *w_gate, double *g)
+{
+    if (T < 0 || d < 1 || F < 1 || !x || !w_gate || !g) return MOC_ORACLE_BAD_ARG;
+#pragma omp parallel for schedule(static)
+    for (int64_t t = 0; t < T; ++t)
+        for (int32_t j = 0; j < F; ++j) g[t * (int64_t)F + j] = dot(x + t * d, w_gate + (int64_t)j * d, d);
+    return MOC_ORACLE_OK;
 }
 
 /*

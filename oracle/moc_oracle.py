@@ -2,7 +2,8 @@
 
 Only the tests, the smoke check and the benchmark's CPU-baseline leg import this
 module.  It compiles ``moc_oracle.c`` with gcc on first use and marshals numpy
-float64 arrays; every piece of arithmetic lives in the C file.
+float64 arrays; every piece of arithmetic lives in the C file (the functions here only compose
+the C routines: a selection rule applied to the gate projection, then the layer's remaining steps).
 """
 from __future__ import annotations
 
@@ -154,7 +155,13 @@ def gate_projection(x, w_gate, F: int | None = None):
     """G = X W_gate (Eq. (Moc-1)) for the first F channels, [T, F] float64."""
     x, w_gate = _f64(x), _f64(w_gate)
     F = w_gate.shape[0] if F is None else F
-    return x @ w_gate[:F].T
+    T, d = x.shape
+    if w_gate.ndim != 2 or w_gate.shape[1] != d or w_gate.shape[0] < F:
+        raise ValueError("weight shape")
+    g = np.empty((T, F))
+    _check(_load().moc_oracle_gate_projection(ctypes.c_int64(T), ctypes.c_int32(d), ctypes.c_int32(F), _p(x),
+                                              _p(w_gate), _p(g)), "moc_oracle_gate_projection")
+    return g
 
 
 def silu_rows(g):

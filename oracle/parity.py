@@ -139,3 +139,25 @@ def check_picks_grouped(idx_dev: np.ndarray, g_oracle: np.ndarray, group: int = 
                                      f"around {tau:.6g}")
         differing += 1
     return differing
+
+
+def check_decode(out, x, w_gate, w_up, w_down, K: int, dtype: str, what: str = "decode"):
+    """A decode result (no indices come back) against the oracle's own picks.  Where a token's margin between its K-th
+    and (K+1)-th gate value is below 1e-4 (inside the exclusion band) the swapped pick is accepted as well; every other
+    token must match within the tolerance.  Arrays are float64; weights hold the logical channels only."""
+    full = orc.forward(x, w_gate, w_up, w_down, K, want_g=True)
+    F = w_gate.shape[0]
+    scale = np.abs(full["out"]).max()
+    tol = REL_TOL[dtype] * scale
+    for t in range(x.shape[0]):
+        err = np.abs(out[t] - full["out"][t]).max()
+        if err <= tol:
+            continue
+        g = full["g"][t]
+        order = np.lexsort((np.arange(F), -g))
+        if not (K < F and g[order[K - 1]] - g[order[K]] <= 1e-4):
+            raise AssertionError(f"{what}: token {t} error {err:.3e} > {tol:.3e}")
+        alt = np.sort(np.concatenate([order[: K - 1], order[K: K + 1]])).astype(np.int32)[None]
+        ref = orc.forward_given_idx(x[t: t + 1], w_gate, w_up, w_down, alt)["out"][0]
+        if not np.abs(out[t] - ref).max() <= tol:
+            raise AssertionError(f"{what}: token {t} matches neither pick")

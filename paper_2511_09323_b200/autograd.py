@@ -1,8 +1,9 @@
 """`torch.autograd` front end of the MoC FFN operator: marshalling only, every step runs in the CUDA library.
 
-`moc_ffn(x, w_gate, w_up, w_down, k)` is the layer of Section 3.2 (Eqs. (Moc-1)..(Moc-3)) with the backward of Section 3.3
-(Eqs. (bp-1)..(bp-5)); between forward and backward only the compact Top-K activations are kept alive (int16 channel
-indices and the gate / up values of the K selected channels per token, Section 3.4), plus `x` for the weight gradients.
+`moc_ffn(x, w_gate, w_up, w_down, k)` is the layer of Section 3.2 (Eq. (Moc-1), the Top-K mask, Eq. (MoC-2)) with the
+backward of Section 4 (Eqs. (bp-1)..(bp-5)); between forward and backward only the compact Top-K activations are kept alive
+(int16 channel indices and the gate / up values of the K selected channels per token: Section 4, Table 1, column "MoC+GCP"),
+plus `x` for the weight gradients.
 `MoCFFN` is a drop-in module holding the three weight matrices channel-major (`[d_ff, d_model]` each, the layout of
 `nn.Linear.weight` for gate / up and of its transpose for down).
 

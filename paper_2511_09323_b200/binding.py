@@ -293,7 +293,7 @@ def moc_ffn_decode_block(h, rms_weight, rms_eps, w_gate, w_up, w_down, k, d_ff=N
     return out
 
 
-def moc_ffn_decode_static(x, w_gate, w_up, w_down, k, out, d_ff=None, stream=None, grouped=False):
+def moc_ffn_decode_static(x, w_gate, w_up, w_down, k, out, d_ff=None, stream=None, grouped=False, post_silu=False):
     """Decode for callers that cannot allocate: no workspace argument, and `out` must be supplied, so that
     nothing on this call path asks any allocator (torch's included) for memory.  The transient buffers
     live in an array inside the library; see the limits and the sharing rules in include/moc_ffn.h."""
@@ -303,7 +303,7 @@ def moc_ffn_decode_static(x, w_gate, w_up, w_down, k, out, d_ff=None, stream=Non
     if grouped:
         k = _grouped_k(k, F_ld if d_ff is None else d_ff)
     desc = make_desc(T, d, F_ld if d_ff is None else d_ff, k, x.dtype, d_ff_ld=F_ld,
-                     flags=MOC_FLAG_SELECT_2_OF_8 if grouped else 0)
+                     flags=(MOC_FLAG_SELECT_2_OF_8 if grouped else 0) | (MOC_FLAG_SELECT_POST_SILU if post_silu else 0))
     rc = load().moc_ffn_decode_static(ctypes.byref(desc), _ptr(x), _ptr(w_gate), _ptr(w_up), _ptr(w_down),
                                       _ptr(out), _stream_ptr(stream))
     if rc != MOC_OK:

@@ -27,16 +27,19 @@ namespace moc {
 __device__ int g_status_word = 0;
 
 int *device_status_ptr() {
-    // the symbol has one instance per device; its address is looked up once per device
-    static int *cache[64] = {};
+    // the symbol has one instance per device; its address is looked up once per device (several host threads may
+    // race to look it up: they store the same value)
+    static std::atomic<int *> cache[64] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
-    if (!cache[dev]) {
+    int *have = cache[dev].load(std::memory_order_relaxed);
+    if (!have) {
         void *p = nullptr;
         if (cudaGetSymbolAddress(&p, g_status_word) != cudaSuccess) return nullptr;
-        cache[dev] = static_cast<int *>(p);
+        have = static_cast<int *>(p);
+        cache[dev].store(have, std::memory_order_relaxed);
     }
-    return cache[dev];
+    return have;
 }
 
 // ---- launch bookkeeping --------------------------------------------------------------------------
@@ -1322,15 +1325,17 @@ int moc_topk_select(int64_t rows, int32_t n, int32_t n_ld, int32_t k, const floa
 static __device__ __align__(256) unsigned char g_static_scratch[MOC_STATIC_SCRATCH_BYTES];
 
 static char *static_scratch_ptr() {
-    static char *cache[64] = {};
+    static std::atomic<char *> cache[64] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
-    if (!cache[dev]) {
+    char *have = cache[dev].load(std::memory_order_relaxed);
+    if (!have) {
         void *p = nullptr;
         if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return nullptr;
-        cache[dev] = static_cast<char *>(p);
+        have = static_cast<char *>(p);
+        cache[dev].store(have, std::memory_order_relaxed);
     }
-    return cache[dev];
+    return have;
 }
 
 int moc_ffn_decode_static(const moc_ffn_desc *desc, const void *x, const void *w_gate, const void *w_up,
@@ -1343,7 +1348,8 @@ int moc_ffn_decode_static(const moc_ffn_desc *desc, const void *x, const void *w
         return MOC_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     // bf16: the decode plan's kernels whenever their workspace fits the array (the LLaMA-7B layer does at 16 tokens)
-    if (desc->dtype == MOC_BF16 && desc->d_model <= 256 * dec::kSliceCols &&
+    // (the post-SiLU selection key exists on the gathered kernels only, as for moc_ffn_decode)
+    if (desc->dtype == MOC_BF16 && !(desc->flags & MOC_FLAG_SELECT_POST_SILU) && desc->d_model <= 256 * dec::kSliceCols &&
         decode_layout(*desc).total <= MOC_STATIC_SCRATCH_BYTES) {
         char *wsd = static_scratch_ptr();
         if (!wsd) return MOC_ERR_CUDA;

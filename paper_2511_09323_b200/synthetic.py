@@ -38,8 +38,9 @@ class Workload:
         return replace(self, tokens=tokens, batch=0, seq=0)
 
 
-# The five benchmark configurations.  C1 is the tiny fp32 case the oracle finishes at once;
-# C2 is the one the headline metric is quoted on.
+# The five benchmark configurations.  C1 is the tiny fp32 case the oracle finishes at once; C2 and C3 are the
+# LLaMA-130M and LLaMA-1B training shapes; C4 is the LLaMA-7B decode shape; C5 (65536 tokens on the 1B shape, three K)
+# is the largest single-GPU training case and the one the benchmark's headline line runs.
 C1 = Workload("C1-tiny-f32", "f32", 256, 128, 512, 512, 64, seed=0)
 C2 = Workload("C2-llama130m-bf16", "bf16", 64 * 256, 768, 2048, 2048, 256, seed=2, rms_norm_x=True,
               batch=64, seq=256)

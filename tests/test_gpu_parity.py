@@ -239,23 +239,7 @@ def test_zero_tokens_is_a_noop():
 
 
 def _check_decode(out64, x64, wg64, wu64, wd64, K, dtype, what):
-    """Decode returns no indices, so the comparison is with the oracle's own picks.  Where a token's margin
-    between its K-th and (K+1)-th gate value is below 1e-4 (inside the 1e-3 exclusion band) the swapped pick
-    is accepted as well; every other token must match within the tolerance."""
-    full = orc.forward(x64, wg64, wu64, wd64, K, want_g=True)
-    F = wg64.shape[0]
-    scale = np.abs(full["out"]).max()
-    tol = parity.REL_TOL[dtype] * scale
-    for t in range(x64.shape[0]):
-        err = np.abs(out64[t] - full["out"][t]).max()
-        if err <= tol:
-            continue
-        g = full["g"][t]
-        order = np.lexsort((np.arange(F), -g))
-        assert K < F and g[order[K - 1]] - g[order[K]] <= 1e-4, f"{what}: token {t} error {err:.3e} > {tol:.3e}"
-        alt = np.sort(np.concatenate([order[: K - 1], order[K: K + 1]])).astype(np.int32)[None]
-        ref = orc.forward_given_idx(x64[t: t + 1], wg64, wu64, wd64, alt)["out"][0]
-        assert np.abs(out64[t] - ref).max() <= tol, f"{what}: token {t} matches neither pick"
+    parity.check_decode(out64, x64, wg64, wu64, wd64, K, dtype, what)
 
 
 @pytest.mark.parametrize("T", [1, 2, 4, 5, 6, 16])   # 1, 2: cooperative kernel; to 5: four-kernel plan; from 6: small-batch plan

@@ -224,6 +224,23 @@ def test_forward_one_hot_input_hand_computed():
     np.testing.assert_allclose(r["out"][0], np.full(d, z0 * 1 + z3 * 4), rtol=1e-14)
 
 
+def test_gate_projection_one_hot_rows_and_library_matmul():
+    # x = e_i picks column i of every channel's weight row: G[t, j] = Wg[j, i] exactly; a padded tail is not projected
+    d, F = 6, 9
+    rng = np.random.default_rng(17)
+    wg = rng.standard_normal((F + 3, d))
+    x = np.eye(d)
+    np.testing.assert_array_equal(orc.gate_projection(x, wg, F), wg[:F].T)
+    # general rows against the library routine (numpy matmul), and against the dense g the full forward reports
+    x, wg, wu, wd = _rand_problem(23, 7, 11, 20)
+    g = orc.gate_projection(x, wg)
+    assert g.shape == (7, 20)
+    np.testing.assert_allclose(g, x @ wg.T, rtol=1e-13, atol=1e-14)
+    np.testing.assert_array_equal(g, orc.forward(x, wg, wu, wd, K=5, want_g=True)["g"])
+    with pytest.raises(ValueError):
+        orc.gate_projection(x, wg[:, :5])
+
+
 def test_forward_structure_token_independence_permutation_linearity():
     T, d, F, K = 12, 10, 30, 7
     x, wg, wu, wd = _rand_problem(5, T, d, F)
@@ -578,7 +595,10 @@ def test_post_silu_selection_equals_pre_silu_when_enough_gates_are_positive():
     post, pre = orc.forward_post_silu(x, wg, wu, wd, K), orc.forward(x, wg, wu, wd, K)
     np.testing.assert_array_equal(post["idx"], pre["idx"])
     np.testing.assert_allclose(post["out"], pre["out"], rtol=1e-13, atol=1e-14)
-    np.testing.assert_allclose(post["s"], G * expit(G), rtol=1e-13, atol=1e-300)
+    # the keys are SiLU of the gate values the oracle itself formed (sequential dot products; numpy's matmul sums in
+    # another order, which shows as ~1e-17 absolute on values that cancel to nearly zero)
+    np.testing.assert_allclose(post["g"], G, rtol=1e-13, atol=1e-15)
+    np.testing.assert_allclose(post["s"], post["g"] * expit(post["g"]), rtol=1e-13, atol=1e-300)
 
 
 def test_post_silu_selection_differs_where_it_must():

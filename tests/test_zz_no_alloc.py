@@ -5,17 +5,21 @@ free byte of HBM to its KV-cache pool, a latency-critical loop that cannot take 
 synchronisation cudaMalloc/cudaFree imply, a plug-in that receives tensors but no allocator.  They
 call this entry point with inputs and an output buffer only; its transient buffers are an array
 built into the library.  The checks below call it through the C ABI and compare it with
-moc_ffn_decode (caller-provided workspace) on two calls in a row, the second smaller than the
-first, so that anything left in the shared array by the first call would show up.
+moc_ffn_decode (caller-provided workspace) and with the CPU oracle on two calls in a row, the
+second smaller than the first, so that anything left in the shared array by the first call would
+show up; one more check watches the device's free memory across a series of calls.
 
 The file name sorts last on purpose: a run that stops at the first failure has then already run
 every other test.
 """
 import ctypes
 
+import numpy as np
 import pytest
 import torch
 
+from oracle import moc_oracle as orc
+from oracle import parity
 from paper_2511_09323_b200 import binding as B
 from paper_2511_09323_b200 import build as moc_build
 from paper_2511_09323_b200 import synthetic as syn
@@ -43,6 +47,10 @@ def _compare(w, x, wg, wu, wd):
     err = (out.double() - ref.double()).abs().max().item()
     scale = ref.double().abs().max().item()
     assert err <= REL[w.dtype] * scale, f"{err:.3e} vs {REL[w.dtype] * scale:.3e}"
+    # and against the definition itself: the two entry points may share kernels, the oracle shares nothing with them
+    F = w.d_ff
+    x64, wg64, wu64, wd64 = (syn.to_f64(t) for t in (x, wg[:F], wu[:F], wd[:F]))
+    parity.check_decode(syn.to_f64(out), x64, wg64, wu64, wd64, w.k, w.dtype, "static decode")
 
 
 @pytest.mark.parametrize("dtype", ["bf16", "f32"])
@@ -68,6 +76,60 @@ def test_static_decode_llama7b_shape(T):
 def test_static_decode_falls_back_to_the_gathered_kernels_when_the_decode_plan_does_not_fit():
     """16 tokens on a 16384-channel layer: the decode plan's buffers exceed the built-in array, the gathered plan's do not."""
     _compare(*_case("bf16", 16, 2048, 16384, 16384, 2048, seed=33))
+
+
+@pytest.mark.parametrize("dtype,T,d,F,F_ld,K", [("bf16", 12, 128, 1000, 1024, 125), ("f32", 5, 72, 333, 336, 41)])
+def test_static_decode_honours_the_post_silu_key(dtype, T, d, F, F_ld, K):
+    """MOC_FLAG_SELECT_POST_SILU (the Top-K placed after the activation) on inputs with fewer positive gate values than
+    K, where the two selection rules keep different channels: the entry point must give the post-SiLU result of the
+    oracle, as moc_ffn_decode does, whichever of its kernel plans the problem size would otherwise pick."""
+    w = syn.Workload("static-ps", dtype, T, d, F, F_ld, K, seed=35)
+    wg, wu, wd = syn.make_weights(w)
+    x = (syn.make_x(w).float() + 1.0).to(wg.dtype)
+    wg = (wg.float() - 0.05 / np.sqrt(d / 128)).to(wg.dtype)
+    wg[F:] = 0
+    xd, wgd, wud, wdd = (t.cuda() for t in (x, wg, wu, wd))
+    out = torch.full_like(xd, float("nan"))
+    B.moc_ffn_decode_static(xd, wgd, wud, wdd, K, out, d_ff=F, post_silu=True)
+    ref_dev = B.moc_ffn_decode(xd, wgd, wud, wdd, K, d_ff=F, post_silu=True)
+    torch.cuda.synchronize()
+    x64, wg64, wu64, wd64 = (syn.to_f64(t) for t in (x, wg[:F], wu[:F], wd[:F]))
+    ref = orc.forward_post_silu(x64, wg64, wu64, wd64, K)
+    assert np.median((ref["g"] > 0).sum(axis=1)) < K, "the inputs must make the two rules differ"
+    pre = orc.forward(x64, wg64, wu64, wd64, K)
+    assert not np.array_equal(ref["idx"], pre["idx"])
+    got = syn.to_f64(out)
+    scale = np.abs(ref["out"]).max()
+    # tokens whose post-SiLU threshold is not a near-tie must match the oracle's post-SiLU output (and not the default rule's)
+    s_sorted = np.sort(ref["s"], axis=1)[:, ::-1]
+    clear = (s_sorted[:, K - 1] - s_sorted[:, K]) > 1e-3
+    assert clear.sum() >= T // 2
+    err = np.abs(got - ref["out"]).max(axis=1)
+    assert np.all(err[clear] <= REL[dtype] * scale), f"{err[clear].max():.3e} vs {REL[dtype] * scale:.3e}"
+    differs = np.abs(pre["out"] - ref["out"]).max(axis=1) > 10 * REL[dtype] * scale
+    assert np.all(np.abs(got - pre["out"]).max(axis=1)[clear & differs] > REL[dtype] * scale)
+    assert (out.double() - ref_dev.double()).abs().max().item() <= REL[dtype] * scale
+
+
+def test_static_decode_leaves_device_memory_alone():
+    """What the entry point is for: after the first call on the device (which looks up the built-in array's address),
+    further calls change neither the device's free memory nor what torch's allocator holds -- on the decode plan's
+    kernels and on the gathered kernels alike."""
+    cases = [_case("bf16", 16, 256, 1000, 1024, 125, seed=36), _case("f32", 3, 128, 333, 336, 41, seed=37)]
+    outs = [torch.empty_like(c[1]) for c in cases]
+    for (w, x, wg, wu, wd), out in zip(cases, outs):     # first calls: one-time set-up happens here
+        B.moc_ffn_decode_static(x, wg, wu, wd, w.k, out, d_ff=w.d_ff)
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    held0, reserved0 = torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
+    for _ in range(5):
+        for (w, x, wg, wu, wd), out in zip(cases, outs):
+            B.moc_ffn_decode_static(x, wg, wu, wd, w.k, out, d_ff=w.d_ff)
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert (torch.cuda.memory_allocated(), torch.cuda.memory_reserved()) == (held0, reserved0)
+    assert free1 == free0, f"free device memory changed by {free0 - free1} bytes"
+    assert B.moc_last_device_status() == B.MOC_OK
 
 
 def test_static_decode_rejects_what_does_not_fit():
