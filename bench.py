@@ -1,18 +1,20 @@
 #!/usr/bin/env python
 """Benchmark of the MoC FFN hot path on B200.
 
-One "step" is one pass of the training hot path -- moc_ffn_forward followed by moc_ffn_backward
-(all four gradients) -- over one batch of the LLaMA-130M-shaped workload (16384 tokens, d_model 768,
-d_ff 2048, K 256, bf16 storage with fp32 accumulation), called through the C ABI.  The line printed
-by rank 0 also carries: the end-to-end number with host buffers (``e2e``), the roofline of the
-dominant kernel measured with CUDA events inside the timed region (``roofline``), the CPU oracle
-timed on this machine's host cores (``cpu_baseline``), small-batch decode latencies on the LLaMA-7B
-shape (``decode``) and the saved-activation bytes (``act_bytes``).
+One "step" is one pass of the training hot path -- moc_ffn_forward followed by moc_ffn_backward (all four
+gradients) -- over one batch of the largest single-GPU training workload: 65536 tokens on the LLaMA-1B FFN shape
+(d_model 2048, d_ff 5504, K 688, bf16 storage with fp32 accumulation), called through the C ABI.  The line printed by
+rank 0 also carries: the end-to-end number with host buffers (``e2e``), the roofline of the dominant kernel measured
+with CUDA events (``roofline``), the whole step against the strict roofline (``strict_roofline``), the K sweep of the
+same shape with the saved-activation bytes (``sweep``, ``act_bytes``), small-batch decode latencies on the LLaMA-7B
+shape (``decode``) and the CPU oracle timed on this machine's host cores (``cpu_baseline``).
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload C2|C3|C5]
 
-With N > 1 it is launched by torchrun, one rank per GPU; every rank runs the same per-GPU batch
-(weak scaling, tokens are independent, no data-path collective).
+With N > 1 it is launched by torchrun, one rank per GPU.  Tokens are independent, so every rank owns its own shard of
+the batch (weak scaling: the per-GPU shard is fixed) with the weights replicated; the one exchange is the sum of the
+weight gradients over ranks, Eqs. (bp-1) and (bp-4) being sums over tokens: one NCCL all-reduce of 3 d_ff d elements
+per step on a side stream, started when the weight-gradient kernel is done so that it overlaps the grad_x kernel.
 """
 from __future__ import annotations
 
@@ -33,8 +35,13 @@ METRIC = "moc_ffn_fwd_bwd_tokens_per_s"
 UNIT = "tokens/s"
 ALU_FP32_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12   # 148 SMs x 128 FMA lanes x 2 flop x max SM clock
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of each kernel of the step on the default C2 workload, from one
-# `ncu --set full` capture of this program (profiles/tensor_core_plan_kernels_C2.md); reported as `roofline.traffic`
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of a kernel of the step, from `ncu` captures of this library's
+# kernels: (workload, kernel) -> (bytes that do not depend on the token count, bytes per token).  A capture holds a few
+# thousand tokens on the device (the full batch is too large to capture); two token counts give the two coefficients,
+# and `roofline.traffic` is their value at the benchmarked token count.
+NCU_DRAM_BYTES = {
+}
+# the same for the LLaMA-130M workload, measured at its full size (one launch of each kernel per step)
 NCU_DRAM_BYTES_C2 = {
     "tc_gate_up_gemm": 173.5e6, "tc_select_mask": 255.1e6, "tc_down_gemm": 75.0e6, "tc_bwd_sample": 235.6e6,
     "tc_dz_gemm": 43.4e6, "tc_wgrad_gemm": 256.7e6, "tc_dx_gemm": 158.6e6,
@@ -47,9 +54,10 @@ def parse_args():
     p.add_argument("--steps", type=int, default=20)
     p.add_argument("--warmup", type=int, default=5)
     p.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    p.add_argument("--workload", default="C2", choices=["C1", "C2", "C3", "C5"])
+    p.add_argument("--workload", default="C5", choices=["C1", "C2", "C3", "C5"])
     p.add_argument("--tokens", type=int, default=0, help="override the workload's token count (debugging)")
     p.add_argument("--no-decode", action="store_true")
+    p.add_argument("--no-sweep", action="store_true", help="skip the K / (batch, seq) sweep of the 1B shape")
     p.add_argument("--no-graph", action="store_true", help="time direct calls instead of a CUDA graph replay of the step")
     p.add_argument("--no-cpu-baseline", action="store_true")
     p.add_argument("--cpu-seconds", type=float, default=15.0, help="target seconds of oracle work")
@@ -199,6 +207,7 @@ def calibrate_oracle_tokens(w, target_s, cap):
     """Token count whose oracle forward+backward takes about target_s on this host."""
     probe = min(cap, 64)
     run, threads = oracle_step_fn(w, probe)
+    run()      # the first call pays for thread start-up and first-touch page faults
     t0 = time.perf_counter()
     run()
     dt = max(time.perf_counter() - t0, 1e-4)
@@ -248,6 +257,62 @@ def workload_config(w, tokens, extra=None):
 
 
 # ------------------------------------------------------------------------------------------------ our arm
+# The pieces of the multi-rank path that need no GPU are functions of their own, so that two gloo ranks on CPU run
+# exactly what the NCCL ranks run.
+
+
+def init_distributed(backend: str, device=None):
+    """Joins the process group described by the environment (RANK, WORLD_SIZE, MASTER_ADDR, MASTER_PORT).
+    Returns (torch.distributed or None when WORLD_SIZE is 1, world, rank)."""
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    if world <= 1:
+        return None, 1, 0
+    import torch.distributed as dist
+    if backend == "nccl":
+        dist.init_process_group("nccl", device_id=device)
+    else:
+        dist.init_process_group(backend, rank=rank, world_size=world)
+    return dist, world, rank
+
+
+def max_over_ranks(dist, values, device=None):
+    """Element-wise maximum over ranks of a list of floats (the job's time is its slowest rank's)."""
+    import torch
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def flat_weight_grads(torch, like, device=None):
+    """The three weight gradients as views of ONE buffer [3, d_ff_ld, d] (gate, up, down), so that the job's only
+    exchange is a single all-reduce.  Returns (flat, dict of views keyed like moc_ffn_backward's result)."""
+    flat = torch.empty((3,) + tuple(like.shape), dtype=like.dtype, device=like.device if device is None else device)
+    return flat, {"grad_w_gate": flat[0], "grad_w_up": flat[1], "grad_w_down": flat[2]}
+
+
+def allreduce_weight_grads(dist, flat):
+    """Sum of the weight gradients over the token shards (Eqs. (bp-1), (bp-4) are sums over tokens): one all-reduce
+    of 3 d_ff d elements.  Returns the bytes one rank contributes."""
+    if dist is not None:
+        dist.all_reduce(flat, op=dist.ReduceOp.SUM)
+    return flat.numel() * flat.element_size()
+
+
+def job_throughput(world, tokens_per_rank, steps, worst_ms):
+    """Whole-job tokens/s: every rank processed `tokens_per_rank` tokens per step; the job took the slowest rank's time."""
+    return aggregate([worst_ms] * world, [tokens_per_rank] * world, steps)[0]
+
+
+def choose_tensor_peak(peaks, clocks):
+    """Which measured bf16 figure a kernel timed in this run is held against: the burst figure when the SM clock
+    sampled during the measurement sat at (within 3 % of) its maximum, the sustained (power-capped, seconds-long)
+    figure when it sagged.  Returns (TFLOP/s, "burst" | "sustained")."""
+    sm, smax = clocks.get("sm_mhz"), clocks.get("sm_max_mhz")
+    if sm and smax and sm < 0.97 * smax:
+        return peaks["bf16_tflops_sustained"], "sustained"
+    return peaks["bf16_tflops"], "burst"
 
 
 def run_ours(args):
@@ -256,18 +321,12 @@ def run_ours(args):
     from paper_2511_09323_b200 import build as moc_build
     from paper_2511_09323_b200 import synthetic as syn
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device (there is no CPU path)")
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist_mod
-        dist = dist_mod
-        dist.init_process_group("nccl", device_id=dev)
+    dist, world, rank = init_distributed("nccl", dev)
     if rank == 0:
         moc_build.build()
     if dist:
@@ -275,29 +334,39 @@ def run_ours(args):
     B.load()
 
     w = syn.WORKLOADS[args.workload]
-    T = args.tokens or w.tokens
-    _, T = shard_plan(world, rank, T)
+    shard_offset, T = shard_plan(world, rank, args.tokens or w.tokens)
     e = 2 if w.dtype == "bf16" else 4
     wg, wu, wd = (t.to(dev) for t in syn.make_weights(w))
-    x_h = syn.make_x(w, tokens=T).pin_memory()
-    dD_h = syn.make_grad_out(w, tokens=T).pin_memory()
+    # this rank's shard of the job's batch: tokens [shard_offset, shard_offset + T)
+    x_h = syn.make_x(w, tokens=T, shard=rank).pin_memory()
+    dD_h = syn.make_grad_out(w, tokens=T, shard=rank).pin_memory()
     x, dD = x_h.to(dev), dD_h.to(dev)
     out = torch.empty_like(x)
     saved = (torch.empty((T, w.k), dtype=torch.int16, device=dev), torch.empty((T, w.k), dtype=x.dtype, device=dev),
              torch.empty((T, w.k), dtype=x.dtype, device=dev))
-    grads = {"grad_x": torch.empty_like(x), "grad_w_gate": torch.empty_like(wg),
-             "grad_w_up": torch.empty_like(wu), "grad_w_down": torch.empty_like(wd)}
+    wgrad_flat, grads = flat_weight_grads(torch, wg)
+    grads["grad_x"] = torch.empty_like(x)
     desc = B.make_desc(T, w.d_model, w.d_ff, w.k, x.dtype, d_ff_ld=w.d_ff_ld)
     ws_f = B.alloc_workspace(desc, B.MOC_OP_FORWARD, dev)
     ws_b = B.alloc_workspace(desc, B.MOC_OP_BACKWARD, dev)
     out_h = torch.empty_like(x_h).pin_memory()
     gx_h = torch.empty_like(x_h).pin_memory()
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)   # 2 x L2
+    side = torch.cuda.Stream(dev) if dist else None                 # carries the weight-gradient all-reduce
+    wgrad_ev = torch.cuda.Event() if dist else None
 
-    def step(xd, dd):
-        B.moc_ffn_forward(xd, wg, wu, wd, w.k, d_ff=w.d_ff, out=out, saved=saved, workspace=ws_f)
-        B.moc_ffn_backward(xd, wg, wu, wd, saved[0], saved[1], saved[2], dd, d_ff=w.d_ff, grads=grads,
-                           workspace=ws_b)
+    def step(xd, dd, out_t=out, grads_t=grads):
+        B.moc_ffn_forward(xd, wg, wu, wd, w.k, d_ff=w.d_ff, out=out_t, saved=saved, workspace=ws_f)
+        B.moc_ffn_backward(xd, wg, wu, wd, saved[0], saved[1], saved[2], dd, d_ff=w.d_ff, grads=grads_t,
+                           workspace=ws_b, wgrad_event=wgrad_ev)
+        if dist:
+            # the all-reduce starts when the weight-gradient kernel is done and runs beside the grad_x kernel;
+            # the step ends when both have finished
+            main = torch.cuda.current_stream(dev)
+            side.wait_event(wgrad_ev)
+            with torch.cuda.stream(side):
+                allreduce_weight_grads(dist, wgrad_flat)
+            main.wait_stream(side)
 
     def barrier():
         torch.cuda.synchronize()
@@ -318,16 +387,16 @@ def run_ours(args):
         uuid = "GPU-" + str(torch.cuda.get_device_properties(dev).uuid)
     except Exception:
         pass
-    sampler = ClockSampler(uuid)
-    # The step is replayed from a CUDA graph when the two calls capture (they enqueue kernels only: no allocation,
-    # no synchronisation), otherwise called directly; the per-kernel CUDA events of the library would sit between
-    # the kernels and stretch the step, so they are recorded in a second pass of the same K steps (`profile_pass`),
-    # which feeds the roofline and the per-kernel table.
+    # At one GPU the step is replayed from a CUDA graph when the two calls capture (they enqueue kernels only: no
+    # allocation, no synchronisation), otherwise called directly; with several ranks the step holds a collective on a
+    # second stream and is called directly.  The per-kernel CUDA events of the library would sit between the kernels
+    # and stretch the step, so they are recorded in a second pass of the same K steps (`profile_pass`), which feeds
+    # the roofline and the per-kernel table.
     launches0 = B.moc_launch_count()
     step(x, dD)
     launches_per_step = B.moc_launch_count() - launches0
     run_step, launch_mode = (lambda: step(x, dD)), "direct calls"
-    if not args.no_graph:
+    if not args.no_graph and not dist:
         try:
             graph = torch.cuda.CUDAGraph()
             with torch.cuda.graph(graph):
@@ -340,6 +409,7 @@ def run_ours(args):
             torch.cuda.synchronize()
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
     barrier()
+    sampler = ClockSampler(uuid)
     sampler.start()
     for s, t in ev:
         flush.zero_()
@@ -357,6 +427,8 @@ def run_ours(args):
     B.moc_profile_enable(True)
     barrier()
     evm = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]   # between forward and backward
+    sampler_p = ClockSampler(uuid)
+    sampler_p.start()
     for (s, t), m in zip(evp, evm):
         flush.zero_()
         s.record()
@@ -365,6 +437,7 @@ def run_ours(args):
         B.moc_ffn_backward(x, wg, wu, wd, saved[0], saved[1], saved[2], dD, d_ff=w.d_ff, grads=grads, workspace=ws_b)
         t.record()
     barrier()
+    clocks_p = sampler_p.stop()
     prof = B.moc_profile_collect()
     B.moc_profile_enable(False)
     profile_ms_per_step = sum(s.elapsed_time(t) for s, t in evp) / args.steps
@@ -376,7 +449,7 @@ def run_ours(args):
     # device buffers, so step i+1's inputs travel while step i computes and step i-1's results travel back.
     # Every step still moves its own x and grad_out from pinned host memory and its own out and grad_x back;
     # the region runs from the first host->device copy to the last device->host copy.  (No L2 flush here: a step
-    # touches about 1 GB of inputs, outputs and workspace, far more than the L2 holds.)
+    # touches gigabytes of inputs, outputs and workspace, far more than the L2 holds.)
     s_in, s_comp, s_out = torch.cuda.Stream(dev), torch.cuda.current_stream(dev), torch.cuda.Stream(dev)
     xb = [torch.empty_like(x) for _ in range(2)]
     db = [torch.empty_like(dD) for _ in range(2)]
@@ -398,9 +471,7 @@ def run_ours(args):
             s_comp.wait_event(ev_in[b])
             if i >= 2:
                 s_comp.wait_event(ev_out[b])         # step i-2's results have left these output buffers
-            B.moc_ffn_forward(xb[b], wg, wu, wd, w.k, d_ff=w.d_ff, out=ob[b], saved=saved, workspace=ws_f)
-            B.moc_ffn_backward(xb[b], wg, wu, wd, saved[0], saved[1], saved[2], db[b], d_ff=w.d_ff, grads=gb[b],
-                               workspace=ws_b)
+            step(xb[b], db[b], ob[b], gb[b])
             ev_comp[b].record(s_comp)
             with torch.cuda.stream(s_out):
                 s_out.wait_event(ev_comp[b])
@@ -423,12 +494,9 @@ def run_ours(args):
     d2h = out_h.numel() * e * 2
 
     # ---- aggregate over ranks (max time, sum tokens) ---------------------------------------------
-    tot = torch.tensor([total_ms, e2e_total_ms], dtype=torch.float64, device=dev)
-    if dist:
-        dist.all_reduce(tot, op=dist.ReduceOp.MAX)
-    worst_ms, worst_e2e_ms = tot.tolist()
-    value = world * T * args.steps / (worst_ms / 1e3)
-    e2e_value = world * T * args.steps / (worst_e2e_ms / 1e3)
+    worst_ms, worst_e2e_ms = max_over_ranks(dist, [total_ms, e2e_total_ms], dev)
+    value = job_throughput(world, T, args.steps, worst_ms)
+    e2e_value = job_throughput(world, T, args.steps, worst_e2e_ms)
 
     status = B.moc_last_device_status()
     if status != B.MOC_OK:
@@ -437,45 +505,59 @@ def run_ours(args):
     line = None
     if rank == 0:
         peaks = load_peaks()
-        roof, kernels = roofline_report(prof, args.steps, T, w, e, peaks)
+        roof, kernels = roofline_report(prof, args.steps, T, w, e, peaks, clocks_p)
+        exchange = ("one NCCL all-reduce (sum) of the weight gradients per step, "
+                    f"{wgrad_flat.numel() * wgrad_flat.element_size()} B per rank, on a side stream beside the grad_x kernel"
+                    if dist else "none (one GPU)")
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": worst_ms / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32",
             "data": "synthetic",
-            "config": workload_config(w, T, {"l2": "flushed between steps by a 256 MiB write outside the timed events",
-                                             "parallelism": f"token-sharded x{world}, no collective",
-                                             "launch": launch_mode}),
+            "config": workload_config(w, T, {"l2": "flushed between steps by a 256 MiB write outside the timed events "
+                                                   "(the step's inputs alone are larger than the L2)",
+                                             "parallelism": f"token-sharded x{world}, weights replicated",
+                                             "exchange": exchange, "launch": launch_mode}),
             "clocks": {k: clocks[k] for k in ("sm_mhz", "sm_max_mhz", "reasons")},
-            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                    "ms_per_step": worst_e2e_ms / args.steps},
             "gpu_launches": launches,
-            "roofline": roof,
             "kernels": kernels,
             "step_ms_min_median": [min(step_ms), statistics.median(step_ms)],
+            "ms_x_sm_mhz": (worst_ms / args.steps) * clocks["sm_mhz"] if clocks.get("sm_mhz") else None,
             "profile_pass": {"ms_per_step": profile_ms_per_step, "launch": "direct calls, a CUDA event pair around "
                              "every kernel (source of `roofline` and `kernels`)",
                              "forward_ms_min_median": [min(fwd_ms), statistics.median(fwd_ms)],
-                             "backward_ms_min_median": [min(bwd_ms), statistics.median(bwd_ms)]},
+                             "backward_ms_min_median": [min(bwd_ms), statistics.median(bwd_ms)],
+                             "clocks": {k: clocks_p[k] for k in ("sm_mhz", "sm_max_mhz", "reasons")}},
             "act_bytes": act_bytes_report(w, T, e, saved, B, desc),
             # tokens whose K-th largest gate value is positive: for those the Top-K before SiLU (what runs) and after
             # SiLU (the paper's ablation arm) keep the same channels
             "selection": {"tokens": T, "tokens_with_positive_threshold":
                           int((saved[1].float().min(dim=1).values > 0).sum().item())},
-            "strict_roofline": strict_roofline(w, T, e, worst_ms / args.steps, peaks),
         }
-    # ---- the MoC 2:8 variant on the same layer (rank 0; extra information, not the headline) ---------
+    # ---- K x (batch, seq) sweep of the 1B shape and the MoC 2:8 variant (rank 0; extra information) ---------
+    if rank == 0 and not args.no_sweep and w.name.startswith("C5"):
+        try:
+            line["sweep"] = sweep_report(torch, B, syn, w, x, dD, wg, wu, wd, out, grads, flush, e)
+        except Exception as exc:
+            line["sweep"] = {"error": repr(exc)}
     if rank == 0 and not args.no_decode and w.dtype == "bf16" and w.d_ff % 8 == 0:
         try:
-            line["moc_2of8"] = grouped_report(torch, B, x, dD, wg, wu, wd, flush, args.steps)
+            line["moc_2of8"] = grouped_report(torch, B, x, dD, wg, wu, wd, flush, min(args.steps, 5))
         except Exception as exc:
             line["moc_2of8"] = {"error": repr(exc)}
+    if rank == 0:
+        line["strict_roofline"] = strict_roofline(w, T, e, worst_ms / args.steps, peaks, clocks)
+        line["e2e"] = {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                       "ms_per_step": worst_e2e_ms / args.steps}
+        line["roofline"] = roof
     # ---- decode (rank 0, after the training timing) ----------------------------------------------
     if rank == 0 and not args.no_decode:
-        del flush, ws_f, ws_b
+        del flush, ws_f, ws_b, xb, db, ob, gb
         torch.cuda.empty_cache()
         try:
-            line["decode"] = decode_report(torch, B, syn, dev, load_peaks())
+            more, main = decode_report(torch, B, syn, dev, load_peaks())
+            line["decode_more"] = more
+            line["decode"] = main
         except Exception as exc:  # the training number stands on its own
             line["decode"] = {"error": repr(exc)}
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -494,8 +576,56 @@ def run_ours(args):
     return 0
 
 
-def roofline_report(prof, steps, T, w, e, peaks):
-    """Roofline of the kernel with the largest share of the timed region + a per-kernel table."""
+def sweep_report(torch, B, syn, w, x, dD, wg, wu, wd, out, grads, flush, e, steps=3):
+    """Forward + backward on the 65536-token LLaMA-1B-shaped batch for K = d_ff/16, d_ff/8, d_ff/4 and for the five
+    (batch, seq) splits of the same tokens, with the bytes kept between forward and backward against dense SwiGLU
+    (Table 1: 4 d_ffn elements per token, 2 d_ffn with recomputation; MoC keeps int16 + 2 values for K channels).
+    The FFN acts on tokens, so the five splits are one [T, d] problem: each is run and timed in its own right.
+    Direct calls, L2 flushed between steps, CUDA events around each step."""
+    T, dev = x.shape[0], x.device
+    rep = {"tokens": T, "steps_per_point": steps, "launch": "direct calls",
+           "dense_swiglu_bytes_per_token": 4 * w.d_ff * e, "dense_gcp_bytes_per_token": 2 * w.d_ff * e, "points": []}
+    for k in syn.C5_K:
+        desc = B.make_desc(T, w.d_model, w.d_ff, k, x.dtype, d_ff_ld=w.d_ff_ld)
+        saved = (torch.empty((T, k), dtype=torch.int16, device=dev), torch.empty((T, k), dtype=x.dtype, device=dev),
+                 torch.empty((T, k), dtype=x.dtype, device=dev))
+        ws_f = B.alloc_workspace(desc, B.MOC_OP_FORWARD, dev)
+        ws_b = B.alloc_workspace(desc, B.MOC_OP_BACKWARD, dev)
+
+        def one():
+            B.moc_ffn_forward(x, wg, wu, wd, k, d_ff=w.d_ff, out=out, saved=saved, workspace=ws_f)
+            B.moc_ffn_backward(x, wg, wu, wd, saved[0], saved[1], saved[2], dD, d_ff=w.d_ff, grads=grads, workspace=ws_b)
+
+        for _ in range(2):
+            one()
+        torch.cuda.synchronize()
+        by_label = {}
+        for batch, seq in syn.C5_BATCH_SEQ:
+            if batch * seq != T:
+                continue
+            ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+            for s, t in ev:
+                flush.zero_()
+                s.record()
+                one()
+                t.record()
+            torch.cuda.synchronize()
+            by_label[f"{batch}x{seq}"] = round(sum(s.elapsed_time(t) for s, t in ev) / steps, 4)
+        ms = statistics.median(by_label.values()) if by_label else None
+        kept = sum(t.numel() * t.element_size() for t in saved)
+        rep["points"].append({
+            "k": k, "ms_per_step_by_batch_x_seq": by_label, "ms_per_step": ms,
+            "tokens_per_s": T / (ms / 1e3) if ms else None,
+            "saved_bytes_per_token": kept / T, "saved_bytes_total": kept,
+            "vs_dense_swiglu": 4 * w.d_ff * e / (kept / T), "vs_dense_gcp": 2 * w.d_ff * e / (kept / T),
+            "workspace_bytes": {"forward": ws_f.numel(), "backward": ws_b.numel()}})
+        del saved, ws_f, ws_b
+    return rep
+
+
+def roofline_report(prof, steps, T, w, e, peaks, clocks=None):
+    """Roofline of the kernel with the largest share of the timed region + a per-kernel table.  `clocks`: what
+    nvidia-smi showed while the kernels were timed (picks the burst or the sustained tensor peak)."""
     kernels = {}
     total = sum(ms for k, (n, ms) in prof.items() if not k.startswith("_")) or 1.0
     for name, (n, ms) in prof.items():
@@ -516,41 +646,68 @@ def roofline_report(prof, steps, T, w, e, peaks):
         roof["executed_rate"] = executed * steps / n / (ms / n / 1e3) / (1e9 if bound == "hbm" else 1e12)
         if bound == "hbm":
             roof.update(bound="hbm", achieved=rate / 1e9, peak=peaks["hbm_gbs"], unit="GB/s")
+            roof["peak_source"] = peaks["source"]
         elif bound == "tensor":
-            roof.update(bound="tensor", achieved=rate / 1e12, peak=peaks["bf16_tflops_sustained"], unit="TFLOP/s")
+            peak, kind = choose_tensor_peak(peaks, clocks or {})
+            roof.update(bound="tensor", achieved=rate / 1e12, peak=peak, unit="TFLOP/s")
+            roof["peak_source"] = f"{peaks['source']}, {kind} bf16 figure (SM clock while timed: " \
+                                  f"{(clocks or {}).get('sm_mhz')} of {(clocks or {}).get('sm_max_mhz')} MHz)"
         else:
             roof.update(bound="alu", achieved=rate / 1e12, peak=ALU_FP32_PEAK_TFLOPS, unit="TFLOP/s")
+            roof["peak_source"] = "derived: 148 SM x 128 lanes x 2 x 1.965 GHz"
         roof["frac"] = roof["achieved"] / roof["peak"]
         roof["executed_frac"] = roof["executed_rate"] / roof["peak"]   # the dense work the kernel really does
-        roof["peak_source"] = peaks["source"] if bound != "alu" else "derived: 148 SM x 128 lanes x 2 x 1.965 GHz"
         roof["algorithmic_per_launch"] = per_launch
-    # measured DRAM bytes per launch exist for the default workload only (one launch of each kernel per step there)
-    at_default = w.name.startswith("C2-") and T == 64 * 256 and n == steps
-    roof["traffic"] = NCU_DRAM_BYTES_C2.get(top) if at_default else None
+        if (clocks or {}).get("sm_mhz"):
+            roof["avg_ms_x_sm_mhz"] = ms / n * clocks["sm_mhz"]
+    roof["traffic"], roof["traffic_source"] = measured_traffic(w, T, top, n, steps)
     return roof, kernels
 
 
-def strict_roofline(w, T, e, ms_per_step, peaks):
+def measured_traffic(w, T, kernel, launches, steps):
+    """ncu DRAM bytes per launch of `kernel` on this workload, or (None, why)."""
+    name = w.name.split("-")[0]
+    if name == "C2" and T == 64 * 256 and launches == steps and kernel in NCU_DRAM_BYTES_C2:
+        return NCU_DRAM_BYTES_C2[kernel], "ncu dram__bytes_read.sum + dram__bytes_write.sum, one launch at the full size"
+    if (name, kernel) in NCU_DRAM_BYTES and launches == steps:
+        fixed, per_token = NCU_DRAM_BYTES[(name, kernel)]
+        return fixed + per_token * T, ("ncu dram__bytes_read.sum + dram__bytes_write.sum captured at two smaller token "
+                                       "counts of the same shape, linear in the token count, evaluated at this one")
+    return None, "no capture for this workload / token count"
+
+
+def strict_roofline(w, T, e, ms_per_step, peaks, clocks=None):
     """Whole-step figures: strict roofline = max(gate GEMM at tensor peak, compulsory bytes at HBM rate)."""
     d, F, K = w.d_model, w.d_ff, w.k
     gate = 2.0 * T * d * F
     sparse = 16.0 * T * K * d
     comp_bytes = (T * d * e * 2 + 3 * F * d * e + T * K * (2 + 2 * e)) + \
                  (2 * T * d * e + 3 * F * d * e + T * K * (2 + 2 * e) + T * d * e + 3 * F * d * e)
-    r_gate = gate / (peaks["bf16_tflops"] * 1e12) * 1e3
+    peak, kind = choose_tensor_peak(peaks, clocks or {})
+    r_gate = gate / (peak * 1e12) * 1e3
     r_bytes = comp_bytes / (peaks["hbm_gbs"] * 1e9) * 1e3
     r_strict = max(r_gate, r_bytes)
-    return {"r_gate_ms": r_gate, "r_bytes_ms": r_bytes, "strict_frac": r_strict / ms_per_step,
+    dense_equiv = 18.0 * T * d * F / (ms_per_step / 1e3) / 1e12
+    return {"r_gate_ms": r_gate, "r_bytes_ms": r_bytes, "compulsory_bytes": comp_bytes,
+            "strict_frac": r_strict / ms_per_step,
             "algorithmic_tflops": (gate + sparse) / (ms_per_step / 1e3) / 1e12,
-            "dense_equiv_tflops": 18.0 * T * d * F / (ms_per_step / 1e3) / 1e12,
-            "peak_source": peaks["source"]}
+            "algorithmic_frac": (gate + sparse) / (ms_per_step / 1e3) / 1e12 / peak,
+            "dense_equiv_tflops": dense_equiv, "dense_equiv_frac": dense_equiv / peak,
+            "tensor_peak": peak, "peak_source": f"{peaks['source']}, {kind} bf16 figure"}
 
 
 def act_bytes_report(w, T, e, saved, B, desc):
+    """Bytes alive between forward and backward (Table 1) and, separately, the transient workspace of each call: the
+    workspace is scratch that a model reuses across layers, so it counts once per model, the saved bytes once per layer."""
     measured = sum(t.numel() * t.element_size() for t in saved)
+    ws_f = B.moc_ffn_workspace_bytes(desc, B.MOC_OP_FORWARD)
+    ws_b = B.moc_ffn_workspace_bytes(desc, B.MOC_OP_BACKWARD)
     return {"moc_saved_per_token": B.moc_ffn_saved_bytes_per_token(desc), "measured_saved_total": measured,
             "measured_saved_per_token": measured / T, "dense_swiglu_per_token": 4 * w.d_ff * e,
-            "dense_gcp_per_token": 2 * w.d_ff * e, "x_and_out_per_token_each": w.d_model * e}
+            "dense_gcp_per_token": 2 * w.d_ff * e, "x_and_out_per_token_each": w.d_model * e,
+            "transient_workspace": {"forward_bytes": ws_f, "backward_bytes": ws_b,
+                                    "forward_per_token": ws_f / T, "backward_per_token": ws_b / T,
+                                    "note": "scratch, reused by every layer; not kept between forward and backward"}}
 
 
 def grouped_report(torch, B, x, dD, wg, wu, wd, flush, steps):
@@ -581,10 +738,13 @@ def decode_report(torch, B, syn, dev, peaks, calls=32, sets=4, replays=5):
     distinct weight sets (4 x 270 MB > L2), so every call streams its weights from HBM and launch overhead is what
     a served model would see; the graph is replayed `replays` times.  `frac` is always against the ALGORITHMIC
     bytes (gate matrix + each used row of the other two once); a call that takes the small-batch plan reads all
-    three matrices, which `executed_bytes` / `executed_frac` report."""
+    three matrices, which `executed_bytes` / `executed_frac` report.
+    Returns (more, main): `main` holds the three batch sizes of the paper's table, `more` everything else."""
     w = syn.C4
     weights = [tuple(t.to(dev) for t in syn.make_weights(w, seed_offset=s)) for s in range(sets)]
-    rep = {"weight_sets": sets, "calls_per_graph": calls, "replays": replays, "timing": "CUDA graph replay"}
+    note = {"weight_sets": sets, "calls_per_graph": calls, "replays": replays, "timing": "CUDA graph replay",
+            "roofline": "algorithmic bytes / measured HBM copy bandwidth"}
+    main, more = dict(note), {}
     e = 2
     stream = torch.cuda.Stream(device=dev)
     for T in tuple(syn.C4_BATCHES) + (32, 64, 128, 256):
@@ -622,18 +782,18 @@ def decode_report(torch, B, syn, dev, peaks, calls=32, sets=4, replays=5):
         union = int(torch.unique(idx.long()).numel())
         algo = w.d_ff * w.d_model * e + 2 * union * w.d_model * e + 2 * T * w.d_model * e
         roof_us = algo / (peaks["hbm_gbs"] * 1e9) * 1e6
-        rep[f"T{T}"] = {"us_per_step": us, "us_per_token": us / T, "union_channels": union,
-                        "algorithmic_bytes": algo, "roofline_us": roof_us, "frac": roof_us / us,
-                        "achieved_gbs": algo / (us * 1e-6) / 1e9, "kernels_per_call": launches,
-                        "dense_ffn_bytes": 3 * w.d_ff * w.d_model * e}
+        entry = {"us_per_step": round(us, 3), "us_per_token": round(us / T, 3), "frac": round(roof_us / us, 4),
+                 "roofline_us": round(roof_us, 3), "algorithmic_bytes": algo, "union_channels": union,
+                 "achieved_gbs": round(algo / (us * 1e-6) / 1e9, 1), "kernels_per_call": launches}
         if launches == 3:   # gate+up, select, down: every weight matrix streamed once
             executed = 3 * w.d_ff * w.d_model * e + 2 * T * w.d_model * e
-            rep[f"T{T}"].update(plan="small-batch (all weights streamed once, tcgen05)", executed_bytes=executed,
-                                executed_frac=executed / (peaks["hbm_gbs"] * 1e9) * 1e6 / us)
+            entry.update(plan="small-batch: all weights streamed once (tcgen05)", executed_bytes=executed,
+                         executed_frac=round(executed / (peaks["hbm_gbs"] * 1e9) * 1e6 / us, 4))
         else:
-            rep[f"T{T}"].update(plan=("decode, one cooperative kernel" if launches == 1 else "decode, four kernels") +
-                                " (gate matrix + gathered rows)", executed_bytes=algo, executed_frac=roof_us / us)
+            entry.update(plan=("one cooperative kernel" if launches == 1 else f"{launches} kernels") +
+                         ": gate matrix + gathered rows")
         if T in syn.C4_BATCHES:
+            main[f"T{T}"] = entry
             # the FFN half of a pre-norm layer, out = h + FFN(RMSNorm(h)): one library call against the same steps as
             # separate launches (torch's RMSNorm and addition around moc_ffn_decode)
             gamma = torch.ones(w.d_model, dtype=x.dtype, device=dev)
@@ -647,13 +807,16 @@ def decode_report(torch, B, syn, dev, peaks, calls=32, sets=4, replays=5):
                 torch.add(x, out, out=out)
 
             us_u, _ = timed(unfused)
-            rep[f"T{T}"]["block"] = {"us_per_step": us_b, "kernels_per_call": n_b,
-                                     "unfused_us_per_step": us_u, "what": "out = h + FFN(RMSNorm(h))"}
+            more[f"T{T}_block"] = {"us_per_step": round(us_b, 3), "kernels_per_call": n_b,
+                                   "unfused_us_per_step": round(us_u, 3), "what": "out = h + FFN(RMSNorm(h))"}
             del wsb
+        else:
+            more[f"T{T}"] = entry
         del ws
+    main["dense_ffn_bytes"] = 3 * w.d_ff * w.d_model * e
     if B.moc_last_device_status() != B.MOC_OK:
         raise RuntimeError("device status raised during decode")
-    return rep
+    return more, main
 
 
 def main():

@@ -133,6 +133,23 @@ MOC_API int moc_ffn_backward(const moc_ffn_desc *desc, const void *x, const void
                              void *cuda_stream);
 
 /*
+ * moc_ffn_backward for data-parallel training: Eqs. (bp-1) and (bp-4) are sums over tokens, so when a batch is
+ * sharded by tokens over several GPUs (weights replicated) each GPU's grad_w_* is a partial sum and the job adds
+ * them with one all-reduce of 3 d_ffn d elements, while Eq. (bp-5), grad_x, stays local.  This variant lets that
+ * all-reduce overlap the grad_x kernel: `wgrad_done_event` (a cudaEvent_t passed as void*, created by the caller;
+ * NULL = plain moc_ffn_backward) is recorded on `cuda_stream` at the point where every kernel that writes
+ * grad_w_gate / grad_w_up / grad_w_down has been enqueued and before the grad_x kernel where the plan orders them
+ * that way (the tensor-core plan; on the gathered plan the weight gradients come last, so the event marks the end of
+ * the call).  A second stream that waits on the event may read the weight gradients at once.  It is recorded on
+ * every successful return, also when no weight gradient was asked for.  Everything else as moc_ffn_backward.
+ */
+MOC_API int moc_ffn_backward_overlap(const moc_ffn_desc *desc, const void *x, const void *w_gate, const void *w_up,
+                                     const void *w_down, const int16_t *topk_idx, const void *topk_gate,
+                                     const void *topk_up, const void *grad_out, void *grad_x, void *grad_w_gate,
+                                     void *grad_w_up, void *grad_w_down, void *workspace, size_t workspace_bytes,
+                                     void *cuda_stream, void *wgrad_done_event);
+
+/*
  * The up values of the kept channels again: topk_up[t, k] = x[t, :] . w_up[topk_idx[t, k], :], rounded to the
  * storage dtype.  For callers that keep only (topk_idx, topk_gate) between forward and backward -- the
  * recomputation idea of Section 4 (Table 1, the "+GCP" columns) taken one step further: 2 K + K e instead of

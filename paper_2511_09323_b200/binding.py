@@ -34,6 +34,7 @@ EXPORTED = (
     "moc_last_device_status", "moc_ffn_saved_bytes_per_token", "moc_status_string", "moc_launch_count",
     "moc_profile_enable", "moc_profile_collect", "moc_profile_kernel_count", "moc_profile_kernel_name",
     "moc_profile_read", "moc_ffn_decode_static", "moc_tc_gemm_bf16", "moc_ffn_recompute_up",
+    "moc_ffn_backward_overlap",
 )
 
 
@@ -71,6 +72,8 @@ def load() -> ctypes.CDLL:
         lib.moc_ffn_forward.argtypes = [dp] + [vp] * 9 + [sz, vp]
         lib.moc_ffn_backward.restype = ctypes.c_int
         lib.moc_ffn_backward.argtypes = [dp] + [vp] * 13 + [sz, vp]
+        lib.moc_ffn_backward_overlap.restype = ctypes.c_int
+        lib.moc_ffn_backward_overlap.argtypes = [dp] + [vp] * 13 + [sz, vp, vp]
         lib.moc_ffn_decode.restype = ctypes.c_int
         lib.moc_ffn_decode.argtypes = [dp] + [vp] * 6 + [sz, vp]
         lib.moc_ffn_decode_block.restype = ctypes.c_int
@@ -200,8 +203,11 @@ def moc_ffn_forward(x, w_gate, w_up, w_down, k, d_ff=None, save=True, out=None, 
 
 def moc_ffn_backward(x, w_gate, w_up, w_down, topk_idx, topk_gate, topk_up, grad_out, d_ff=None,
                      want=("x", "w_gate", "w_up", "w_down"), grads=None, accumulate=False, workspace=None,
-                     stream=None):
-    """Returns dict(grad_x, grad_w_gate, grad_w_up, grad_w_down) (None for entries not in `want`)."""
+                     stream=None, wgrad_event=None):
+    """Returns dict(grad_x, grad_w_gate, grad_w_up, grad_w_down) (None for entries not in `want`).
+    `wgrad_event`: a torch.cuda.Event that the library records once the weight gradients are complete in stream
+    order and before the grad_x kernel (moc_ffn_backward_overlap): a side stream that waits on it can all-reduce the
+    weight gradients of a token-sharded batch while grad_x is still being computed."""
     _check_dev(x, w_gate, w_up, w_down, topk_idx, topk_gate, topk_up, grad_out, workspace)
     T, d = x.shape
     F_ld = w_gate.shape[0]
@@ -221,10 +227,15 @@ def moc_ffn_backward(x, w_gate, w_up, w_down, topk_idx, topk_gate, topk_up, grad
     _check_dev(*res.values())
     if workspace is None:
         workspace = alloc_workspace(desc, MOC_OP_BACKWARD, x.device)
-    rc = load().moc_ffn_backward(ctypes.byref(desc), _ptr(x), _ptr(w_gate), _ptr(w_up), _ptr(w_down),
-                                 _ptr(topk_idx), _ptr(topk_gate), _ptr(topk_up), _ptr(grad_out),
-                                 _ptr(res["grad_x"]), _ptr(res["grad_w_gate"]), _ptr(res["grad_w_up"]),
-                                 _ptr(res["grad_w_down"]), _ptr(workspace), workspace.numel(), _stream_ptr(stream))
+    args = (ctypes.byref(desc), _ptr(x), _ptr(w_gate), _ptr(w_up), _ptr(w_down), _ptr(topk_idx), _ptr(topk_gate),
+            _ptr(topk_up), _ptr(grad_out), _ptr(res["grad_x"]), _ptr(res["grad_w_gate"]), _ptr(res["grad_w_up"]),
+            _ptr(res["grad_w_down"]), _ptr(workspace), workspace.numel(), _stream_ptr(stream))
+    if wgrad_event is None:
+        rc = load().moc_ffn_backward(*args)
+    else:
+        if not wgrad_event.cuda_event:       # torch creates the underlying cudaEvent_t lazily: force it with a record
+            wgrad_event.record(torch.cuda.current_stream(x.device) if stream is None else stream)
+        rc = load().moc_ffn_backward_overlap(*args, ctypes.c_void_p(wgrad_event.cuda_event))
     if rc != MOC_OK:
         raise MocError(rc, "moc_ffn_backward")
     return res

@@ -276,7 +276,7 @@ int forward_gather(const moc_ffn_desc &d, const T *x, const T *wg, const T *wu, 
 template <typename T>
 int backward_gather(const moc_ffn_desc &d, const T *x, const T *wg, const T *wu, const T *wd,
                     const int16_t *idx, const T *tg, const T *tu, const T *dout, T *gx, T *gwg, T *gwu, T *gwd,
-                    char *ws, cudaStream_t st) {
+                    char *ws, cudaStream_t st, cudaEvent_t wgrad_done) {
     const BackwardPlan p = plan_backward(d);
     const int F = d.d_ff, K = d.k, dm = d.d_model;
     const int64_t TK = d.tokens * (int64_t)K;
@@ -292,7 +292,10 @@ int backward_gather(const moc_ffn_desc &d, const T *x, const T *wg, const T *wu,
                (backward_token_kernel<T><<<(unsigned)d.tokens, kTokenThreads, tok_smem, st>>>(
                    wg, wu, wd, idx, tg, tu, dout, dm, F, K, TK, gx, want_w ? coef : nullptr, status)));
     if ((rc = launch_ok()) != MOC_OK) return rc;
-    if (!want_w) return MOC_OK;
+    if (!want_w) {
+        if (wgrad_done && cudaEventRecord(wgrad_done, st) != cudaSuccess) return MOC_ERR_CUDA;
+        return MOC_OK;
+    }
 
     uint32_t *counts = reinterpret_cast<uint32_t *>(ws + p.off_counts);
     uint32_t *totals = reinterpret_cast<uint32_t *>(ws + p.off_totals);
@@ -318,7 +321,9 @@ int backward_gather(const moc_ffn_desc &d, const T *x, const T *wg, const T *wu,
                (wgrad_rows_kernel<T><<<d.d_ff_ld, kTokenThreads, red, st>>>(
                    x, dout, coef, TK, row_start, pairs, dm, F, K, gwg, gwu, gwd,
                    (d.flags & MOC_FLAG_ACCUMULATE_WGRAD) ? 1 : 0)));
-    return launch_ok();
+    if ((rc = launch_ok()) != MOC_OK) return rc;
+    if (wgrad_done && cudaEventRecord(wgrad_done, st) != cudaSuccess) return MOC_ERR_CUDA;
+    return MOC_OK;
 }
 
 // ---- tensor-core plan (bf16 training shapes) ---------------------------------------------------------
@@ -526,7 +531,7 @@ int small_batch_dx(const moc_ffn_desc &d, const __nv_bfloat16 *dG, const __nv_bf
 int backward_tc(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat16 *wg, const __nv_bfloat16 *wu,
                 const __nv_bfloat16 *wd, const int16_t *idx, const __nv_bfloat16 *tg, const __nv_bfloat16 *tu,
                 const __nv_bfloat16 *dout, __nv_bfloat16 *gx, __nv_bfloat16 *gwg, __nv_bfloat16 *gwu,
-                __nv_bfloat16 *gwd, char *ws, cudaStream_t st) {
+                __nv_bfloat16 *gwd, char *ws, cudaStream_t st, cudaEvent_t wgrad_done) {
     using namespace tc;
     const TcBackwardLayout L = tc_backward_layout(d);
     __nv_bfloat16 *Zp = reinterpret_cast<__nv_bfloat16 *>(ws + L.off_z);
@@ -610,6 +615,8 @@ int backward_tc(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat
         MOC_LAUNCH(KID_TC_WGRAD_GEMM, st, (rc = launch_gemm<true, true, EPI_BF16>(p, st)));
         if (rc != MOC_OK) return rc;
     }
+    // the weight gradients are complete in stream order here; the grad_x kernel that follows does not touch them
+    if (wgrad_done && cudaEventRecord(wgrad_done, st) != cudaSuccess) return MOC_ERR_CUDA;
     // dX = dG' Wg + dU' Wu   (Eq. (bp-5)): one accumulator, two contraction segments
     if (gx && L.small_bytes) {
         // a small batch: the weight-streaming kernel of the small-batch plan (a 256-row tile of tokens would leave
@@ -1127,6 +1134,16 @@ int moc_ffn_backward(const moc_ffn_desc *desc, const void *x, const void *w_gate
                      const void *w_down, const int16_t *topk_idx, const void *topk_gate, const void *topk_up,
                      const void *grad_out, void *grad_x, void *grad_w_gate, void *grad_w_up, void *grad_w_down,
                      void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    return moc_ffn_backward_overlap(desc, x, w_gate, w_up, w_down, topk_idx, topk_gate, topk_up, grad_out, grad_x,
+                                    grad_w_gate, grad_w_up, grad_w_down, workspace, workspace_bytes, cuda_stream, nullptr);
+}
+
+int moc_ffn_backward_overlap(const moc_ffn_desc *desc, const void *x, const void *w_gate, const void *w_up,
+                             const void *w_down, const int16_t *topk_idx, const void *topk_gate, const void *topk_up,
+                             const void *grad_out, void *grad_x, void *grad_w_gate, void *grad_w_up,
+                             void *grad_w_down, void *workspace, size_t workspace_bytes, void *cuda_stream,
+                             void *wgrad_done_event) {
+    cudaEvent_t wgrad_done = static_cast<cudaEvent_t>(wgrad_done_event);
     int rc = check_desc(desc);
     if (rc != MOC_OK) return rc;
     if (desc->tokens == 0) {
@@ -1141,6 +1158,7 @@ int moc_ffn_backward(const moc_ffn_desc *desc, const void *x, const void *w_gate
         for (void *g : gw) {
             if (g && cudaMemsetAsync(g, 0, wbytes, st0) != cudaSuccess) return MOC_ERR_CUDA;
         }
+        if (wgrad_done && cudaEventRecord(wgrad_done, st0) != cudaSuccess) return MOC_ERR_CUDA;
         return MOC_OK;
     }
     if (!good_ptr(x) || !good_ptr(w_gate) || !good_ptr(w_up) || !good_ptr(w_down) || !good_ptr(topk_idx) ||
@@ -1148,7 +1166,11 @@ int moc_ffn_backward(const moc_ffn_desc *desc, const void *x, const void *w_gate
         return MOC_ERR_INVALID_ARG;
     if (!aligned16(grad_x) || !aligned16(grad_w_gate) || !aligned16(grad_w_up) || !aligned16(grad_w_down))
         return MOC_ERR_INVALID_ARG;
-    if (!grad_x && !grad_w_gate && !grad_w_up && !grad_w_down) return MOC_OK;
+    if (!grad_x && !grad_w_gate && !grad_w_up && !grad_w_down) {
+        if (wgrad_done && cudaEventRecord(wgrad_done, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+            return MOC_ERR_CUDA;
+        return MOC_OK;
+    }
     const size_t need = moc_ffn_workspace_bytes(desc, MOC_OP_BACKWARD);
     if (need && (!good_ptr(workspace) || workspace_bytes < need)) return MOC_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
@@ -1158,15 +1180,15 @@ int moc_ffn_backward(const moc_ffn_desc *desc, const void *x, const void *w_gate
         if (use_tc_plan(*desc))
             return backward_tc(*desc, (const T *)x, (const T *)w_gate, (const T *)w_up, (const T *)w_down, topk_idx,
                                (const T *)topk_gate, (const T *)topk_up, (const T *)grad_out, (T *)grad_x,
-                               (T *)grad_w_gate, (T *)grad_w_up, (T *)grad_w_down, ws, st);
+                               (T *)grad_w_gate, (T *)grad_w_up, (T *)grad_w_down, ws, st, wgrad_done);
         return backward_gather<T>(*desc, (const T *)x, (const T *)w_gate, (const T *)w_up, (const T *)w_down,
                                   topk_idx, (const T *)topk_gate, (const T *)topk_up, (const T *)grad_out,
-                                  (T *)grad_x, (T *)grad_w_gate, (T *)grad_w_up, (T *)grad_w_down, ws, st);
+                                  (T *)grad_x, (T *)grad_w_gate, (T *)grad_w_up, (T *)grad_w_down, ws, st, wgrad_done);
     }
     using T = float;
     return backward_gather<T>(*desc, (const T *)x, (const T *)w_gate, (const T *)w_up, (const T *)w_down,
                               topk_idx, (const T *)topk_gate, (const T *)topk_up, (const T *)grad_out,
-                              (T *)grad_x, (T *)grad_w_gate, (T *)grad_w_up, (T *)grad_w_down, ws, st);
+                              (T *)grad_x, (T *)grad_w_gate, (T *)grad_w_up, (T *)grad_w_down, ws, st, wgrad_done);
 }
 
 int moc_ffn_decode(const moc_ffn_desc *desc, const void *x, const void *w_gate, const void *w_up,

@@ -76,20 +76,23 @@ def make_weights(w: Workload, seed_offset: int = 0):
     return tuple(out)
 
 
-def make_x(w: Workload, tokens: int | None = None):
-    """x [T, d] ~ N(0,1), optionally RMS-normalised per token, rounded to the storage dtype."""
+def make_x(w: Workload, tokens: int | None = None, shard: int = 0):
+    """x [T, d] ~ N(0,1), optionally RMS-normalised per token, rounded to the storage dtype.
+
+    `shard`: a batch sharded by tokens over several GPUs is the concatenation of its shards, each drawn from its own
+    seed (shard 0 is the single-GPU batch), so no rank has to draw the other ranks' tokens."""
     T = w.tokens if tokens is None else tokens
-    g = _gen(1000003 * (w.seed + 1) + 1)
+    g = _gen(1000003 * (w.seed + 1) + 1 + 104729 * shard)
     x = torch.randn(T, w.d_model, generator=g, dtype=torch.float32)
     if w.rms_norm_x:
         x = x / torch.sqrt(x.pow(2).mean(dim=1, keepdim=True) + 1e-6)
     return x.to(torch_dtype(w.dtype)).contiguous()
 
 
-def make_grad_out(w: Workload, tokens: int | None = None):
-    """Upstream gradient [T, d] ~ N(0,1), rounded to the storage dtype."""
+def make_grad_out(w: Workload, tokens: int | None = None, shard: int = 0):
+    """Upstream gradient [T, d] ~ N(0,1), rounded to the storage dtype; `shard` as in make_x."""
     T = w.tokens if tokens is None else tokens
-    g = _gen(1000003 * (w.seed + 1) + 2)
+    g = _gen(1000003 * (w.seed + 1) + 2 + 104729 * shard)
     return torch.randn(T, w.d_model, generator=g, dtype=torch.float32).to(torch_dtype(w.dtype)).contiguous()
 
 
