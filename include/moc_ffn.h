@@ -245,6 +245,41 @@ MOC_API int moc_topk_select(int64_t rows, int32_t n, int32_t n_ld, int32_t k, co
                             int16_t *idx_out, void *cuda_stream);
 
 /*
+ * The row Top-K selector of the tensor-core plan (the one moc_ffn_forward runs on training-sized bf16 batches) alone,
+ * on caller-supplied fp32 gate rows, so that the mask definition of Section 3.2 can be checked bit-exactly on it too.
+ * Which kernel form runs depends on the row length and k exactly as in moc_ffn_forward: teams of two or four warps per
+ * row with the row staged in shared memory, the same with one buffer for the gate and the up row (long rows), or one
+ * CTA per row (rows too long for a team's slice); `*variant` (host, may be NULL) receives which:
+ * 0 CTA per row, 1 teams of two, 2 teams of four, 3 teams of four with a shared buffer.
+ *   gate     [rows, n_ld] fp32, device; n_ld a multiple of 8 with n <= n_ld <= n rounded up to 128
+ *   idx_out  [rows, k] int16, device, ascending
+ *   bracket  host pointer to {center, half width} of the threshold bracket the launch starts from (what the previous
+ *            launch of a forward pass would have left in the workspace), or NULL for the state of a first call; the
+ *            bracket is a hint only: any value, however wrong, must give the same exact result
+ *   workspace  moc_topk_select_tc_workspace_bytes(rows, n, n_ld, k) bytes (0 = shape not served by this selector:
+ *            (n + k) * 4 bytes must fit 170 KiB)
+ */
+MOC_API size_t moc_topk_select_tc_workspace_bytes(int64_t rows, int32_t n, int32_t n_ld, int32_t k);
+MOC_API int moc_topk_select_tc(int64_t rows, int32_t n, int32_t n_ld, int32_t k, const float *gate, int16_t *idx_out,
+                               const float *bracket, int *variant, void *workspace, size_t workspace_bytes,
+                               void *cuda_stream);
+
+/*
+ * The one-kernel form of moc_ffn_decode for one or two bf16 tokens (MOC_ERR_UNSUPPORTED where the problem or the
+ * device does not admit that kernel; it runs here for every k, also where moc_ffn_decode would prefer another form),
+ * which additionally reports the mask it applied: kept [tokens, d_ff] bytes on the device,
+ * 1 for a kept channel.  In that kernel no SM ever holds a token's whole gate row (the K-th largest value is found
+ * through a histogram and a candidate list shared by all SMs), so this is the only way to see its selection directly.
+ * A test that makes x a one-hot row e_i reads G[t, j] = w_gate[j, i] exactly and can so put any bf16 gate row in front
+ * of the selection.  workspace: moc_ffn_decode_probe_workspace_bytes(desc) bytes.  Arguments otherwise as
+ * moc_ffn_decode.
+ */
+MOC_API size_t moc_ffn_decode_probe_workspace_bytes(const moc_ffn_desc *desc);
+MOC_API int moc_ffn_decode_probe(const moc_ffn_desc *desc, const void *x, const void *w_gate, const void *w_up,
+                                 const void *w_down, void *out, uint8_t *kept, void *workspace, size_t workspace_bytes,
+                                 void *cuda_stream);
+
+/*
  * The dense bf16 contraction used for the gate projection G = X W_gate of Eq. (Moc-1) and for every
  * other contraction of the tensor-core plan, exposed so that it can be checked on its own:
  *     C[m, n] (fp32, row-major, leading dimension ldc) = sum_k A(m, k) * B(n, k),  fp32 accumulation.

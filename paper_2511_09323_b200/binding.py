@@ -34,7 +34,8 @@ EXPORTED = (
     "moc_last_device_status", "moc_ffn_saved_bytes_per_token", "moc_status_string", "moc_launch_count",
     "moc_profile_enable", "moc_profile_collect", "moc_profile_kernel_count", "moc_profile_kernel_name",
     "moc_profile_read", "moc_ffn_decode_static", "moc_tc_gemm_bf16", "moc_ffn_recompute_up",
-    "moc_ffn_backward_overlap",
+    "moc_ffn_backward_overlap", "moc_topk_select_tc", "moc_topk_select_tc_workspace_bytes", "moc_ffn_decode_probe",
+    "moc_ffn_decode_probe_workspace_bytes",
 )
 
 
@@ -87,6 +88,15 @@ def load() -> ctypes.CDLL:
                                                                 ctypes.c_int64, vp, ctypes.c_int64, vp]
         lib.moc_topk_select.restype = ctypes.c_int
         lib.moc_topk_select.argtypes = [ctypes.c_int64, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, vp, vp, vp]
+        lib.moc_topk_select_tc_workspace_bytes.restype = sz
+        lib.moc_topk_select_tc_workspace_bytes.argtypes = [ctypes.c_int64] + [ctypes.c_int32] * 3
+        lib.moc_topk_select_tc.restype = ctypes.c_int
+        lib.moc_topk_select_tc.argtypes = [ctypes.c_int64] + [ctypes.c_int32] * 3 + [vp, vp, ctypes.POINTER(ctypes.c_float),
+                                                                                  ctypes.POINTER(ctypes.c_int), vp, sz, vp]
+        lib.moc_ffn_decode_probe_workspace_bytes.restype = sz
+        lib.moc_ffn_decode_probe_workspace_bytes.argtypes = [dp]
+        lib.moc_ffn_decode_probe.restype = ctypes.c_int
+        lib.moc_ffn_decode_probe.argtypes = [dp] + [vp] * 7 + [sz, vp]
         lib.moc_last_device_status.restype = ctypes.c_int
         lib.moc_test_bounded_wait.argtypes = [ctypes.c_int64, vp]
         lib.moc_test_bounded_wait.restype = ctypes.c_int
@@ -334,6 +344,54 @@ def moc_topk_select(gate: torch.Tensor, k: int, n: int | None = None, stream=Non
     if rc != MOC_OK:
         raise MocError(rc, "moc_topk_select")
     return idx
+
+
+SELECT_VARIANTS = ("cta_per_row", "team2", "team4", "team4_shared")
+
+
+def moc_topk_select_tc(gate: torch.Tensor, k: int, n: int | None = None, bracket=None, stream=None):
+    """The tensor-core plan's selector alone: gate [rows, n_ld] fp32 -> (idx [rows, k] int16, variant name).
+    `bracket`: (center, half width) the launch starts from, None = the state of a first call."""
+    _check_dev(gate)
+    if gate.dtype != torch.float32 or gate.dim() != 2:
+        raise TypeError("gate must be a 2-D fp32 tensor")
+    rows, n_ld = gate.shape
+    n = n_ld if n is None else n
+    lib = load()
+    need = lib.moc_topk_select_tc_workspace_bytes(rows, n, n_ld, k)
+    if need == 0:
+        raise MocError(MOC_ERR_UNSUPPORTED, "moc_topk_select_tc")
+    ws = torch.empty(need, dtype=torch.uint8, device=gate.device)
+    idx = torch.empty((rows, k), dtype=torch.int16, device=gate.device)
+    variant = ctypes.c_int(-1)
+    br = None if bracket is None else (ctypes.c_float * 2)(float(bracket[0]), float(bracket[1]))
+    rc = lib.moc_topk_select_tc(rows, n, n_ld, k, _ptr(gate), _ptr(idx), br, ctypes.byref(variant), _ptr(ws), need,
+                                _stream_ptr(stream))
+    if rc != MOC_OK:
+        raise MocError(rc, "moc_topk_select_tc")
+    return idx, SELECT_VARIANTS[variant.value]
+
+
+def moc_ffn_decode_probe(x, w_gate, w_up, w_down, k, d_ff=None, stream=None, grouped=False):
+    """The one-kernel decode form for one or two tokens with its mask: (out [T, d], kept [T, d_ff] uint8)."""
+    _check_dev(x, w_gate, w_up, w_down)
+    T, d = x.shape
+    F_ld = w_gate.shape[0]
+    F = F_ld if d_ff is None else d_ff
+    if grouped:
+        k = _grouped_k(k, F)
+    desc = make_desc(T, d, F, k, x.dtype, d_ff_ld=F_ld, flags=MOC_FLAG_SELECT_2_OF_8 if grouped else 0)
+    out = torch.empty_like(x)
+    kept = torch.full((T, F), 255, dtype=torch.uint8, device=x.device)
+    need = load().moc_ffn_decode_probe_workspace_bytes(ctypes.byref(desc))
+    if need == 0:
+        raise MocError(MOC_ERR_UNSUPPORTED, "moc_ffn_decode_probe")
+    ws = torch.empty(need, dtype=torch.uint8, device=x.device)
+    rc = load().moc_ffn_decode_probe(ctypes.byref(desc), _ptr(x), _ptr(w_gate), _ptr(w_up), _ptr(w_down), _ptr(out),
+                                     _ptr(kept), _ptr(ws), ws.numel(), _stream_ptr(stream))
+    if rc != MOC_OK:
+        raise MocError(rc, "moc_ffn_decode_probe")
+    return out, kept
 
 
 def moc_last_device_status(stream=None) -> int:

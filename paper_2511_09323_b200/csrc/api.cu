@@ -341,6 +341,118 @@ bool use_tc_forward(const moc_ffn_desc &d) { return use_tc_plan(d) && !(d.flags 
 
 inline int ceil_div(int64_t a, int64_t b) { return (int)((a + b - 1) / b); }
 
+// ---- the row Top-K selector of the tensor-core plan: which kernel form serves a row of F channels with K kept ----
+// A team of warps per token while at least two tokens' rows fit an SM's shared memory (each team stages its token's
+// rows in its own slice: as many teams per SM as fit, in one or two CTAs; rows too long for that with separate gate
+// and up buffers let the two rows share one buffer), else one CTA per token.  Teams of four warps for long rows (few
+// tokens fit an SM there), pairs otherwise (measured: LLaMA-1B width 0.59 -> 0.50 ms and LLaMA-7B width 0.56 -> 0.41 ms
+// with four; 2048 channels 0.080 -> 0.124 ms, so short rows keep pairs).
+struct TcSelect {
+    int nv;             // 128-channel groups of a row
+    int team;           // warps per token (2 or 4)
+    bool team_select;   // false: one CTA per token (select_mask_rows_kernel)
+    bool shared_u;      // gate and up row share one buffer
+    int tokens_per_cta, ctas_per_sm;
+    size_t smem;        // dynamic shared memory of the launch
+    int variant;        // MOC_SELECT_VARIANT_* (what a test hook reports)
+};
+
+enum {
+    MOC_SELECT_VARIANT_CTA_PER_ROW = 0,   // select_mask_rows_kernel
+    MOC_SELECT_VARIANT_TEAM2 = 1,         // teams of two warps, separate gate / up buffers
+    MOC_SELECT_VARIANT_TEAM4 = 2,         // teams of four warps, separate buffers
+    MOC_SELECT_VARIANT_TEAM4_SHARED = 3,  // teams of four, one buffer for both rows
+};
+
+TcSelect tc_select_config(int F, int K) {
+    using namespace tc;
+    TcSelect c{};
+    c.nv = ceil_div(F, 128);
+    c.team = c.nv >= 40 ? 4 : 2;
+    const auto units_fit = [&](bool shared) {  // tokens in flight per SM
+        return (int)std::min<size_t>(
+            (size_t)220 * 1024 / (pair_select_words(c.nv, K, shared, c.team) * sizeof(uint32_t)), 16);
+    };
+    const bool parks = pair_select_parks_gates(c.nv, K, c.team);
+    const int min_units = 2;  // at least two tokens in flight per SM
+    // (rows short enough for teams of two always fit with separate buffers: the shared form exists for teams of four)
+    c.shared_u = c.team == 4 && units_fit(false) < min_units && parks && units_fit(true) >= min_units;
+    const size_t team_bytes = pair_select_words(c.nv, K, c.shared_u, c.team) * sizeof(uint32_t);
+    const int per_sm = units_fit(c.shared_u);
+    const int units_per_cta = kPairSelMaxWarps / c.team;
+    c.team_select = per_sm >= min_units;
+    if (c.team_select) {
+        c.ctas_per_sm = per_sm > units_per_cta ? 2 : 1;
+        c.tokens_per_cta = std::min(per_sm / c.ctas_per_sm, units_per_cta);
+        c.smem = (size_t)c.tokens_per_cta * team_bytes;
+        c.variant = c.team == 4 ? (c.shared_u ? MOC_SELECT_VARIANT_TEAM4_SHARED : MOC_SELECT_VARIANT_TEAM4)
+                                : MOC_SELECT_VARIANT_TEAM2;
+    } else {
+        c.ctas_per_sm = 6;
+        c.tokens_per_cta = 1;
+        c.smem = ((size_t)F + K) * sizeof(uint32_t);
+        c.variant = MOC_SELECT_VARIANT_CTA_PER_ROW;
+    }
+    return c;
+}
+
+// the usual row lengths get their loops unrolled (the template's first parameter)
+#define MOC_TC_SELECT_DISPATCH(c, DO)                                                   \
+    do {                                                                                \
+        if ((c).team == 4) {                                                            \
+            if ((c).shared_u) DO((tc::select_mask_rows_pair_kernel<0, true, 4>), 128);  \
+            else if ((c).nv == 43) DO((tc::select_mask_rows_pair_kernel<43, false, 4>), 128); \
+            else DO((tc::select_mask_rows_pair_kernel<0, false, 4>), 128);              \
+        } else {                                                                        \
+            if ((c).nv == 8) DO((tc::select_mask_rows_pair_kernel<8, false, 2>), 64);   \
+            else if ((c).nv == 16) DO((tc::select_mask_rows_pair_kernel<16, false, 2>), 64); \
+            else if ((c).nv == 32) DO((tc::select_mask_rows_pair_kernel<32, false, 2>), 64); \
+            else DO((tc::select_mask_rows_pair_kernel<0, false, 2>), 64);               \
+        }                                                                               \
+    } while (0)
+
+int tc_select_prepare(const TcSelect &c, int F, int K) {
+    int rc = MOC_OK;
+    if (c.team_select) {
+#define MOC_DO_SET(KERN, TPT) rc = set_smem(KERN, c.smem, 2048)
+        MOC_TC_SELECT_DISPATCH(c, MOC_DO_SET);
+#undef MOC_DO_SET
+    } else {
+        rc = set_smem(tc::select_mask_rows_kernel, c.smem);
+    }
+    if (rc != MOC_OK) return rc;
+    return set_smem(tc::select_hint_kernel, (size_t)F * sizeof(uint32_t));
+}
+
+// Team selector: every launch works with one bracket kept in the workspace ({center, width, tag} at hint[0..2]); it
+// gathers the statistics of its thresholds (hint[4..6], CTA counter at hint[8]) and its last CTA rewrites the bracket
+// for the next launch.  The bracket is only a hint: a stale or garbage one costs time (rows take the general exact
+// path), never correctness; the statistics and the counter reset themselves at the end of every launch.
+// CTA-per-token selector: hint[0..1] is the guess select_hint_kernel left.
+void tc_select_launch(const TcSelect &c, const float *G, int ldg, __nv_bfloat16 *U, int ldu, int64_t n, int F, int K,
+                      int16_t *o_idx, __nv_bfloat16 *o_g, __nv_bfloat16 *o_u, float *hint, int *status, cudaStream_t st) {
+    using namespace tc;
+    if (c.team_select) {
+        SelectMeta meta{};
+        meta.bracket = hint;
+        meta.acc = hint + 4;
+        meta.done = reinterpret_cast<unsigned int *>(hint + 8);
+        const unsigned grid = (unsigned)std::min<int64_t>((n + c.tokens_per_cta - 1) / c.tokens_per_cta,
+                                                          (int64_t)sm_count() * c.ctas_per_sm);
+#define MOC_DO_LAUNCH(KERN, TPT)                                                                     \
+    MOC_LAUNCH(KID_TC_SELECT_MASK, st,                                                               \
+               (KERN<<<grid, c.tokens_per_cta * TPT, c.smem, st>>>(G, ldg, U, ldu, n, F, c.nv, K, o_idx, o_g, o_u, \
+                                                                    meta, status)))
+        MOC_TC_SELECT_DISPATCH(c, MOC_DO_LAUNCH);
+#undef MOC_DO_LAUNCH
+    } else {
+        const unsigned grid = (unsigned)std::min<int64_t>(n, (int64_t)sm_count() * 6);
+        MOC_LAUNCH(KID_TC_SELECT_MASK, st,
+                   (select_mask_rows_kernel<<<grid, kSelectThreads, c.smem, st>>>(G, ldg, U, ldu, n, F, K, o_idx, o_g,
+                                                                                   o_u, hint)));
+    }
+}
+
 // D = Z' W_down over all tokens: A = Z' [T, F] (K-major), B = Wd [F, d] (its contiguous dimension is N)
 int forward_tc_down(const moc_ffn_desc &d, const __nv_bfloat16 *Z, int ldz, const __nv_bfloat16 *wd, __nv_bfloat16 *out,
                     int *status, cudaStream_t st) {
@@ -374,66 +486,10 @@ int forward_tc(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat1
     const int64_t T = d.tokens;
     const int f_tiles = ceil_div(F, BN);
 
-    // selector: one warp per token while at least four warps' rows fit an SM's shared memory, else one CTA per token
-    const int nv = ceil_div(F, 128);  // 128-channel groups of a row
-    // each warp stages its token's rows in its own slice of shared memory: as many warps per SM as fit, in one
-    // or two CTAs
-    // (rows too long for that with separate gate and up buffers let the two rows share one buffer).  Teams of four
-    // warps for long rows (few tokens fit an SM there), pairs otherwise (measured: LLaMA-1B width 0.59 -> 0.50 ms and
-    // LLaMA-7B width 0.56 -> 0.41 ms with four; 2048 channels 0.080 -> 0.124 ms, so short rows keep pairs)
-    const int sel_team = nv >= 40 ? 4 : 2;
-    const auto units_fit = [&](bool shared) {  // tokens in flight per SM
-        return (int)std::min<size_t>(
-            (size_t)220 * 1024 / (pair_select_words(nv, K, shared, sel_team) * sizeof(uint32_t)), 16);
-    };
-    const bool parks = pair_select_parks_gates(nv, K, sel_team);
-    const int min_units = 2;  // at least two tokens in flight per SM
-    const bool sel_shared_u = units_fit(false) < min_units && parks && units_fit(true) >= min_units;
-    const size_t warp_bytes = pair_select_words(nv, K, sel_shared_u, sel_team) * sizeof(uint32_t);
-    const int warps_per_sm = units_fit(sel_shared_u);  // tokens in flight per SM (one team each)
-    const int sel_units_per_cta = kPairSelMaxWarps / sel_team;
-    const int sel_ctas_per_sm = warps_per_sm > sel_units_per_cta ? 2 : 1;
-    const int sel_wpc = std::min(warps_per_sm / sel_ctas_per_sm, sel_units_per_cta);  // tokens per CTA
-    const size_t warp_smem = (size_t)sel_wpc * warp_bytes;
-    const size_t cta_smem = ((size_t)F + K) * sizeof(uint32_t);
-    const bool warp_select = warps_per_sm >= min_units;
+    const TcSelect sel = tc_select_config(F, K);
     float *hint = reinterpret_cast<float *>(ws + L.off_hint);
-    int rc = MOC_OK;
-    if (warp_select) {
-        if (sel_team == 4) {
-            if (sel_shared_u) {
-                rc = set_smem(select_mask_rows_pair_kernel<0, true, 4>, warp_smem, 2048);
-            } else if (nv == 43) {
-                rc = set_smem(select_mask_rows_pair_kernel<43, false, 4>, warp_smem, 2048);
-            } else {
-                rc = set_smem(select_mask_rows_pair_kernel<0, false, 4>, warp_smem, 2048);
-            }
-        } else if (sel_shared_u) {
-            rc = set_smem(select_mask_rows_pair_kernel<0, true, 2>, warp_smem, 2048);
-        } else {
-            switch (nv) {
-                case 8: rc = set_smem(select_mask_rows_pair_kernel<8, false, 2>, warp_smem, 2048); break;
-                case 16: rc = set_smem(select_mask_rows_pair_kernel<16, false, 2>, warp_smem, 2048); break;
-                case 32: rc = set_smem(select_mask_rows_pair_kernel<32, false, 2>, warp_smem, 2048); break;
-                default: rc = set_smem(select_mask_rows_pair_kernel<0, false, 2>, warp_smem, 2048); break;
-            }
-        }
-    } else {
-        rc = set_smem(select_mask_rows_kernel, cta_smem);
-    }
+    int rc = tc_select_prepare(sel, F, K);
     if (rc != MOC_OK) return rc;
-    if ((rc = set_smem(select_hint_kernel, (size_t)F * sizeof(uint32_t))) != MOC_OK) return rc;
-    // Warp selector: every launch works with one bracket kept in the workspace ({center, width, tag} at
-    // hint[0..2]); it gathers the statistics of its thresholds (hint[4..6], CTA counter at hint[8]) and its last
-    // CTA rewrites the bracket for the next launch.  The bracket is only a hint: a stale or garbage one costs
-    // time (rows take the general exact path), never correctness; the statistics and the counter reset themselves
-    // at the end of every launch.
-    SelectMeta meta{};
-    if (warp_select) {
-        meta.bracket = hint;
-        meta.acc = hint + 4;
-        meta.done = reinterpret_cast<unsigned int *>(hint + 8);
-    }
 
     int *status = device_status_ptr();
     if (!status) return MOC_ERR_CUDA;
@@ -481,7 +537,7 @@ int forward_tc(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat1
         p.c[1] = U + t0 * L.ldf;
         MOC_LAUNCH(KID_TC_GATE_UP_GEMM, st, (rc = launch_gemm<false, false, EPI_GATE_UP>(p, st)));
         if (rc != MOC_OK) return rc;
-        if (t0 == 0 && !warp_select) {
+        if (t0 == 0 && !sel.team_select) {
             MOC_LAUNCH(KID_TC_SELECT_HINT, st,
                        (select_hint_kernel<<<1, kSelectThreads, (size_t)F * sizeof(uint32_t), st>>>(G, F, K, hint)));
             if ((rc = launch_ok()) != MOC_OK) return rc;
@@ -494,31 +550,8 @@ int forward_tc(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat1
             const unsigned grid = (unsigned)std::min<int64_t>((n * (F / 8) + 255) / 256, (int64_t)sm_count() * 64);
             MOC_LAUNCH(KID_TC_SELECT_MASK, st,
                        (select_grouped_mask_kernel<<<grid, 256, 0, st>>>(G, L.ldf, Uc, L.ldf, n, F, o_idx, o_g, o_u)));
-        } else if (warp_select) {
-            const unsigned grid =
-                (unsigned)std::min<int64_t>((n + sel_wpc - 1) / sel_wpc, (int64_t)sm_count() * sel_ctas_per_sm);
-#define MOC_SELECT_LAUNCH(THREADS_PER_TOKEN, ...)                                                          \
-    MOC_LAUNCH(KID_TC_SELECT_MASK, st,                                                                     \
-               (__VA_ARGS__<<<grid, sel_wpc * THREADS_PER_TOKEN, warp_smem, st>>>(                          \
-                   G, L.ldf, Uc, L.ldf, n, F, nv, K, o_idx, o_g, o_u, meta, status)))
-            // the usual row lengths get their loops unrolled
-            if (sel_team == 4) {
-                if (sel_shared_u) MOC_SELECT_LAUNCH(128, select_mask_rows_pair_kernel<0, true, 4>);
-                else if (nv == 43) MOC_SELECT_LAUNCH(128, select_mask_rows_pair_kernel<43, false, 4>);
-                else MOC_SELECT_LAUNCH(128, select_mask_rows_pair_kernel<0, false, 4>);
-            } else {
-                if (sel_shared_u) MOC_SELECT_LAUNCH(64, select_mask_rows_pair_kernel<0, true, 2>);
-                else if (nv == 8) MOC_SELECT_LAUNCH(64, select_mask_rows_pair_kernel<8, false, 2>);
-                else if (nv == 16) MOC_SELECT_LAUNCH(64, select_mask_rows_pair_kernel<16, false, 2>);
-                else if (nv == 32) MOC_SELECT_LAUNCH(64, select_mask_rows_pair_kernel<32, false, 2>);
-                else MOC_SELECT_LAUNCH(64, select_mask_rows_pair_kernel<0, false, 2>);
-            }
-#undef MOC_SELECT_LAUNCH
         } else {
-            const unsigned grid = (unsigned)std::min<int64_t>(n, (int64_t)sm_count() * 6);
-            MOC_LAUNCH(KID_TC_SELECT_MASK, st,
-                       (select_mask_rows_kernel<<<grid, kSelectThreads, cta_smem, st>>>(G, L.ldf, Uc, L.ldf, n, F, K,
-                                                                                         o_idx, o_g, o_u, hint)));
+            tc_select_launch(sel, G, L.ldf, Uc, L.ldf, n, F, K, o_idx, o_g, o_u, hint, status, st);
         }
         if ((rc = launch_ok()) != MOC_OK) return rc;
     }
@@ -773,7 +806,7 @@ int launch_coop(const dc::Params &prm, const CoopLayout &L, cudaStream_t st) {
 // rms_w != nullptr: the block form (x is the residual stream h: RMSNorm in front, h added behind)
 int decode_coop(const moc_ffn_desc &d, const CoopLayout &L, const __nv_bfloat16 *x, const __nv_bfloat16 *wg,
                 const __nv_bfloat16 *wu, const __nv_bfloat16 *wd, __nv_bfloat16 *out, char *wsp, cudaStream_t st,
-                const __nv_bfloat16 *rms_w = nullptr, float rms_eps = 0.f) {
+                const __nv_bfloat16 *rms_w = nullptr, float rms_eps = 0.f, uint8_t *kept_out = nullptr) {
     int *status = device_status_ptr();
     if (!status) return MOC_ERR_CUDA;
     dc::Params prm{};
@@ -791,6 +824,7 @@ int decode_coop(const moc_ffn_desc &d, const CoopLayout &L, const __nv_bfloat16 
     prm.stages = L.stages;
     prm.rms_w = rms_w;
     prm.rms_eps = rms_eps;
+    prm.kept_out = kept_out;
     prm.hist = reinterpret_cast<uint32_t *>(wsp + L.off_hist);
     prm.cand_n = reinterpret_cast<uint32_t *>(wsp + L.off_n);
     prm.cand = reinterpret_cast<uint2 *>(wsp + L.off_cand);
@@ -924,6 +958,103 @@ bool use_small_batch_plan(const moc_ffn_desc &d) {
            sb::select_smem(d.d_ff, false) + 48 * 1024 <= (size_t)kMaxDynSmem;
 }
 
+int small_batch_down(const moc_ffn_desc &d, const SmallBatchLayout &L, const sb::GemmShape &ds, const __nv_bfloat16 *wd,
+                     const __nv_bfloat16 *Z, float *acc, int *counters, __nv_bfloat16 *out, const __nv_bfloat16 *resid,
+                     int *status, cudaStream_t st);
+
+// The overlapped form of the small-batch plan, for calls that keep nothing: the gate matrix is streamed by ALL SMs
+// first, and the selection (one CTA per token, a dozen microseconds during which HBM would idle) then runs beside the
+// kernel that streams the up matrix on the remaining SMs; that kernel's epilogue waits for the selection and forms the
+// masked hidden state Z' from its accumulators, the gate values and the selection bitmaps.  Four kernels:
+//   gate (all SMs) -> select (T CTAs, bitmaps only) || up + mask (SMs - ceil(T/2) CTAs) -> down.
+// MOC_FFN_SB_OVERLAP=0 in the environment keeps the three-kernel form everywhere (comparisons); =n: up to n tokens.
+bool small_batch_overlapped(const moc_ffn_desc &d, bool saving) {
+    static const int limit = [] {
+        const char *e = getenv("MOC_FFN_SB_OVERLAP");
+        return e ? atoi(e) : 32;  // measured on the LLaMA-7B shape: 67 / 70 us against 70 / 72 us at 16 / 32 tokens, but 86 against 76 us at 64
+    }();
+    return !saving && !(d.flags & MOC_FLAG_SELECT_2_OF_8) && d.tokens <= limit && tc::sm_count() >= 32;
+}
+
+// channels per CTA when `ctas` CTAs share the F channels of one matrix: a multiple of 8, at most sb::kMaxRows
+int sb_rows_for(int F, int ctas) {
+    return std::min(sb::kMaxRows, std::max(8, (((F + ctas - 1) / ctas) + 7) & ~7));
+}
+
+int forward_small_batch_overlapped(const moc_ffn_desc &d, const SmallBatchLayout &L, const __nv_bfloat16 *x,
+                                   const __nv_bfloat16 *wg, const __nv_bfloat16 *wu, const __nv_bfloat16 *wd,
+                                   __nv_bfloat16 *out, char *wsp, cudaStream_t st, const __nv_bfloat16 *resid) {
+    const int T = (int)d.tokens, F = d.d_ff, dm = d.d_model;
+    int *status = device_status_ptr();
+    if (!status) return MOC_ERR_CUDA;
+    const int sms = tc::sm_count();
+    // a selector CTA per SM (asking for more than half an SM's shared memory keeps a second one away: two of them on
+    // one SM would halve each other's pace); the up kernel gets the other SMs
+    const int sel_sms = std::min(T, sms / 2);
+    const int rows_g = sb_rows_for(F, sms), rows_u = sb_rows_for(F, sms - sel_sms);
+    const int ctas_g = (F + rows_g - 1) / rows_g, ctas_u = (F + rows_u - 1) / rows_u;
+    const int boxes = 2;  // two 64-element blocks per stage: the CTAs' row counts are small here
+    const sb::GemmShape gg = sb::gemm_shape(T, rows_g, boxes), gu = sb::gemm_shape(T, rows_u, boxes),
+                        ds = sb::gemm_shape(T, sb::kTile * L.accs);
+    if (gg.stages < 2 || gu.stages < 2 || ds.stages < 2) return MOC_ERR_UNSUPPORTED;
+    float *G = reinterpret_cast<float *>(wsp + L.off_g);
+    uint32_t *kept = reinterpret_cast<uint32_t *>(wsp + L.off_u);  // the bitmaps live where the three-kernel form keeps U
+    const int kept_words = (F + 31) / 32;
+    __nv_bfloat16 *Z = reinterpret_cast<__nv_bfloat16 *>(wsp + L.off_z);
+    float *acc = reinterpret_cast<float *>(wsp + L.off_acc);
+    int *counters = reinterpret_cast<int *>(wsp + L.off_cnt);
+    int rc;
+    const size_t sel_smem = std::max(sb::select_smem(F, false), (size_t)116 * 1024);
+    if ((rc = set_smem(sb::sb_gate_up_kernel, std::max(gg.smem, gu.smem), 1024)) != MOC_OK) return rc;
+    if ((rc = set_smem(sb::sb_down_kernel, ds.smem, 1024)) != MOC_OK) return rc;
+    if ((rc = set_smem(sb::sb_select_kernel, sel_smem)) != MOC_OK) return rc;
+
+    auto gate_up_params = [&](sb::GateUpParams &gp, const sb::GemmShape &gs, int rows, int ctas) {
+        memset(&gp, 0, sizeof(gp));
+        if (!tc::make_map(&gp.w_map[0], wg, F, dm, dm, sb::kBK, rows) ||
+            !tc::make_map(&gp.w_map[1], wu, F, dm, dm, sb::kBK, rows) ||
+            !tc::make_map(&gp.x_map, x, T, dm, dm, sb::kBK, gs.tn))
+            return false;
+        gp.T = T;
+        gp.tn = gs.tn;
+        gp.tmem_cols = gs.tmem_cols;
+        gp.stages = gs.stages;
+        gp.w_bytes = gs.w_bytes;
+        gp.stage_bytes = gs.stage_bytes;
+        gp.F = F;
+        gp.boxes = boxes;
+        gp.k_blocks = (dm + sb::kBK * boxes - 1) / (sb::kBK * boxes);
+        gp.rows = rows;
+        gp.ctas_per_matrix = ctas;
+        gp.G = G;
+        gp.ldf = L.ldf;
+        gp.status = status;
+        return true;
+    };
+    sb::GateUpParams gp;
+    if (!gate_up_params(gp, gg, rows_g, ctas_g)) return MOC_ERR_CUDA;
+    gp.counters = counters;
+    gp.n_counters = L.m_tiles;
+    MOC_LAUNCH(KID_SB_GATE_UP, st, launch_pdl(sb::sb_gate_up_kernel, dim3(ctas_g), sb::kThreads, gg.smem, st, gp));
+    if ((rc = launch_ok()) != MOC_OK) return rc;
+
+    sb::SelectParams sp{G, nullptr, L.ldf, F, d.k, dm, Z, L.ldz, acc, nullptr, nullptr, nullptr, 0, status, kept, kept_words};
+    MOC_LAUNCH(KID_SB_SELECT, st, launch_pdl(sb::sb_select_kernel, dim3(T), dec::kSelThreads, sel_smem, st, sp));
+    if ((rc = launch_ok()) != MOC_OK) return rc;
+
+    sb::GateUpParams up;
+    if (!gate_up_params(up, gu, rows_u, ctas_u)) return MOC_ERR_CUDA;
+    up.prob0 = 1;
+    up.mask_mode = 1;
+    up.kept_bits = kept;
+    up.kept_words = kept_words;
+    up.Z = Z;
+    up.ldz = L.ldz;
+    MOC_LAUNCH(KID_SB_GATE_UP, st, launch_pdl(sb::sb_gate_up_kernel, dim3(ctas_u), sb::kThreads, gu.smem, st, up));
+    if ((rc = launch_ok()) != MOC_OK) return rc;
+    return small_batch_down(d, L, ds, wd, Z, acc, counters, out, resid, status, st);
+}
+
 int forward_small_batch(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat16 *wg,
                         const __nv_bfloat16 *wu, const __nv_bfloat16 *wd, __nv_bfloat16 *out, int16_t *idx,
                         __nv_bfloat16 *tg, __nv_bfloat16 *tu, char *wsp, cudaStream_t st,
@@ -944,6 +1075,9 @@ int forward_small_batch(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __n
     if ((rc = set_smem(sb::sb_down_kernel, ds.smem, 1024)) != MOC_OK) return rc;
     if ((rc = set_smem(sb::sb_select_kernel, sel_smem)) != MOC_OK) return rc;
 
+    if (small_batch_overlapped(d, idx != nullptr))
+        return forward_small_batch_overlapped(d, L, x, wg, wu, wd, out, wsp, st, resid);
+
     sb::GateUpParams gp;
     memset(&gp, 0, sizeof(gp));
     if (!tc::make_map(&gp.w_map[0], wg, F, dm, dm, sb::kBK, L.rows) ||
@@ -959,6 +1093,7 @@ int forward_small_batch(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __n
     gp.F = F;
     gp.k_blocks = (dm + sb::kBK - 1) / sb::kBK;
     gp.rows = L.rows;
+    gp.boxes = 1;
     gp.ctas_per_matrix = L.ctas_per_matrix;
     gp.G = G;
     gp.U = U;
@@ -970,7 +1105,7 @@ int forward_small_batch(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __n
                launch_pdl(sb::sb_gate_up_kernel, dim3(2 * L.ctas_per_matrix), sb::kThreads, gs.smem, st, gp));
     if ((rc = launch_ok()) != MOC_OK) return rc;
 
-    sb::SelectParams sp{G, U, L.ldf, F, d.k, dm, Z, L.ldz, acc, idx, tg, tu, L.stage_u ? 1 : 0, status};
+    sb::SelectParams sp{G, U, L.ldf, F, d.k, dm, Z, L.ldz, acc, idx, tg, tu, L.stage_u ? 1 : 0, status, nullptr, 0};
     if (d.flags & MOC_FLAG_SELECT_2_OF_8) {
         MOC_LAUNCH(KID_SB_SELECT, st,
                    launch_pdl(sb::sb_select_grouped_kernel, dim3(T), dec::kSelThreads, 0, st, sp));
@@ -979,6 +1114,14 @@ int forward_small_batch(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __n
     }
     if ((rc = launch_ok()) != MOC_OK) return rc;
 
+    return small_batch_down(d, L, ds, wd, Z, acc, counters, out, resid, status, st);
+}
+
+// D = Z' W_down of the small-batch plan (both forms end with it)
+int small_batch_down(const moc_ffn_desc &d, const SmallBatchLayout &L, const sb::GemmShape &ds, const __nv_bfloat16 *wd,
+                     const __nv_bfloat16 *Z, float *acc, int *counters, __nv_bfloat16 *out, const __nv_bfloat16 *resid,
+                     int *status, cudaStream_t st) {
+    const int T = (int)d.tokens, F = d.d_ff, dm = d.d_model;
     sb::DownParams dp;
     memset(&dp, 0, sizeof(dp));
     if (!tc::make_map(&dp.wd_map[0], wd, F, dm, dm, 64, sb::kBK) ||
@@ -1341,6 +1484,98 @@ int moc_topk_select(int64_t rows, int32_t n, int32_t n_ld, int32_t k, const floa
     return launch_ok();
 }
 
+// ---- test hooks: the selectors of the tensor-core plan and of the cooperative decode kernel on their own ----------
+namespace moc {
+namespace {
+__global__ void set_hint_kernel(float *hint, float center, float width, float tag) {
+    hint[0] = center;
+    hint[1] = width;
+    hint[2] = tag;
+}
+
+struct SelectTcLayout {
+    size_t off_u, off_g, off_v, off_hint, total;
+};
+SelectTcLayout select_tc_layout(int64_t rows, int n_ld, int k) {
+    SelectTcLayout L{};
+    Carver c;
+    L.off_u = c.take((size_t)rows * n_ld * sizeof(__nv_bfloat16));
+    L.off_g = c.take((size_t)rows * k * sizeof(__nv_bfloat16));
+    L.off_v = c.take((size_t)rows * k * sizeof(__nv_bfloat16));
+    L.off_hint = c.take(256);
+    L.total = c.off;
+    return L;
+}
+bool select_tc_shape_ok(int64_t rows, int n, int n_ld, int k) {
+    return rows >= 0 && n >= 1 && k >= 1 && k <= n && n <= 32768 && n_ld >= n && n_ld % 8 == 0 &&
+           n_ld <= ((n + 127) / 128) * 128 && ((size_t)n + (size_t)k) * 4 <= 170 * 1024;
+}
+}  // namespace
+}  // namespace moc
+
+size_t moc_topk_select_tc_workspace_bytes(int64_t rows, int32_t n, int32_t n_ld, int32_t k) {
+    if (!select_tc_shape_ok(rows, n, n_ld, k)) return 0;
+    return select_tc_layout(rows, n_ld, k).total;
+}
+
+int moc_topk_select_tc(int64_t rows, int32_t n, int32_t n_ld, int32_t k, const float *gate, int16_t *idx_out,
+                       const float *bracket, int *variant, void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    if (!select_tc_shape_ok(rows, n, n_ld, k)) return MOC_ERR_INVALID_ARG;
+    const TcSelect sel = tc_select_config(n, k);
+    if (variant) *variant = sel.variant;
+    if (rows == 0) return MOC_OK;
+    if (!good_ptr(gate) || !good_ptr(idx_out)) return MOC_ERR_INVALID_ARG;
+    const SelectTcLayout L = select_tc_layout(rows, n_ld, k);
+    if (!good_ptr(workspace) || workspace_bytes < L.total) return MOC_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    char *ws = static_cast<char *>(workspace);
+    int *status = device_status_ptr();
+    if (!status) return MOC_ERR_CUDA;
+    int rc = tc_select_prepare(sel, n, k);
+    if (rc != MOC_OK) return rc;
+    using B16 = __nv_bfloat16;
+    B16 *U = reinterpret_cast<B16 *>(ws + L.off_u);
+    float *hint = reinterpret_cast<float *>(ws + L.off_hint);
+    // a zero up row: the selector forms SiLU(g) * 0 for its masked row, which nobody reads here
+    if (cudaMemsetAsync(U, 0, (size_t)rows * n_ld * sizeof(B16), st) != cudaSuccess) return MOC_ERR_CUDA;
+    if (cudaMemsetAsync(hint, 0, 256, st) != cudaSuccess) return MOC_ERR_CUDA;
+    if (bracket) {
+        set_hint_kernel<<<1, 1, 0, st>>>(hint, bracket[0], bracket[1], tc::kBracketTag);
+    } else if (!sel.team_select) {
+        // as in the forward pass: the CTA-per-row form starts from the exact threshold of the first row
+        tc::select_hint_kernel<<<1, kSelectThreads, (size_t)n * sizeof(uint32_t), st>>>(gate, n, k, hint);
+    }
+    if ((rc = launch_ok()) != MOC_OK) return rc;
+    tc_select_launch(sel, gate, n_ld, U, n_ld, rows, n, k, idx_out, reinterpret_cast<B16 *>(ws + L.off_g),
+                     reinterpret_cast<B16 *>(ws + L.off_v), hint, status, st);
+    return launch_ok();
+}
+
+size_t moc_ffn_decode_probe_workspace_bytes(const moc_ffn_desc *desc) {
+    if (check_desc(desc) != MOC_OK || desc->tokens < 1) return 0;
+    bool coop = false;
+    const CoopLayout C = coop_layout(*desc, coop);
+    return coop ? C.total : 0;
+}
+
+int moc_ffn_decode_probe(const moc_ffn_desc *desc, const void *x, const void *w_gate, const void *w_up,
+                         const void *w_down, void *out, uint8_t *kept, void *workspace, size_t workspace_bytes,
+                         void *cuda_stream) {
+    int rc = check_desc(desc);
+    if (rc != MOC_OK) return rc;
+    // (whatever form moc_ffn_decode would prefer for this K: the probe exists to look at this kernel's selection)
+    bool coop = false;
+    const bool plain = desc->tokens >= 1 && desc->dtype == MOC_BF16 && !(desc->flags & MOC_FLAG_SELECT_POST_SILU);
+    const CoopLayout C = plain ? coop_layout(*desc, coop) : CoopLayout{};
+    if (!coop) return MOC_ERR_UNSUPPORTED;
+    if (!good_ptr(x) || !good_ptr(w_gate) || !good_ptr(w_up) || !good_ptr(w_down) || !good_ptr(out) || !kept)
+        return MOC_ERR_INVALID_ARG;
+    if (!good_ptr(workspace) || workspace_bytes < C.total) return MOC_ERR_WORKSPACE;
+    using T = __nv_bfloat16;
+    return decode_coop(*desc, C, (const T *)x, (const T *)w_gate, (const T *)w_up, (const T *)w_down, (T *)out,
+                       static_cast<char *>(workspace), static_cast<cudaStream_t>(cuda_stream), nullptr, 0.f, kept);
+}
+
 // ---- decode without a caller workspace --------------------------------------------------------------
 // Scratch for moc_ffn_decode_static.  In host code the name below is only a handle for the runtime,
 // not a device address: the address is asked for once per device and that pointer goes to the kernels.
@@ -1444,6 +1679,14 @@ int moc_last_device_status(void *cuda_stream) {
     }
     return v;
 }
+
+#ifdef MOC_TIMELINE
+extern "C" __attribute__((visibility("default"))) int moc_debug_timeline(unsigned long long *out, int n) {
+    if (cudaDeviceSynchronize() != cudaSuccess) return MOC_ERR_CUDA;
+    return cudaMemcpyFromSymbol(out, g_timeline, sizeof(unsigned long long) * (size_t)std::min(n, 4096)) == cudaSuccess
+               ? MOC_OK : MOC_ERR_CUDA;
+}
+#endif
 
 int64_t moc_launch_count(void) { return g_prof.launches.load(std::memory_order_relaxed); }
 

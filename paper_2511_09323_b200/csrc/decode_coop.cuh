@@ -54,6 +54,8 @@ struct Params {
     // weight rms_w and adds h to its output; rms_w == nullptr: the plain layer on x
     const __nv_bfloat16 *rms_w;
     float rms_eps;
+    // test hook: when not null, [T][F] bytes that receive 1 for every channel a token keeps and 0 for the others
+    uint8_t *kept_out;
 };
 
 inline size_t smem_bytes(int T, int d, int stages) {
@@ -325,6 +327,11 @@ __global__ void __launch_bounds__(kThreads, 1) decode_coop_kernel(const Params p
         }
     }
     __syncthreads();
+    if (p.kept_out)
+        for (int i = tid; i < T * rows; i += kThreads) {
+            const int t = i / rows, r = i - t * rows;
+            p.kept_out[(int64_t)t * F + c0 + r] = (uint8_t)((s_mask[r] >> t) & 1);
+        }
     if (warp == 0) {  // the kept channels in ascending order
         int n = 0;
         for (int base = 0; base < rows; base += 32) {

@@ -102,4 +102,27 @@ __device__ __forceinline__ uint32_t gate_key(float g) {
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// ---- development aid: device-clock stamps (only in builds with -DMOC_TIMELINE) ---------------------------------
+// MOC_TL(slot) lets the first thread of the first CTA of a kernel note the GPU's nanosecond timer in g_timeline[slot].
+#ifdef MOC_TIMELINE
+__device__ unsigned long long g_timeline[4096];
+__device__ __forceinline__ void timeline_stamp(int slot, bool who) {
+    if (who) {
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+        g_timeline[slot] = t;
+    }
+}
+// MOC_TL_CTA(base): every CTA's first thread notes the timer in g_timeline[base + blockIdx.x]
+#define MOC_TL_CTA(base) ::moc::timeline_stamp((base) + (int)blockIdx.x, threadIdx.x == 0)
+#define MOC_TL_CTA_ANY(base) ::moc::timeline_stamp((base) + (int)blockIdx.x, true)
+#define MOC_TL(slot) ::moc::timeline_stamp(slot, blockIdx.x == 0 && threadIdx.x == 0)
+#define MOC_TL_IF(slot, cond) ::moc::timeline_stamp(slot, cond)
+#else
+#define MOC_TL(slot) ((void)0)
+#define MOC_TL_CTA(base) ((void)0)
+#define MOC_TL_CTA_ANY(base) ((void)0)
+#define MOC_TL_IF(slot, cond) ((void)0)
+#endif
+
 }  // namespace moc

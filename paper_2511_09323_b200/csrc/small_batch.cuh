@@ -34,10 +34,10 @@ constexpr int kTile = 128;      // MMA M
 constexpr int kBK = 64;         // contraction elements per stage: one 128-byte swizzle row
 constexpr int kThreads = 320;   // warp 0 TMA, warp 1 MMA + TMEM, warps 2..9 epilogue (two per TMEM lane quarter)
 constexpr int kEpiThreads = kThreads - 64;
-constexpr int kMaxStages = 10;
+constexpr int kMaxStages = 16;  // narrow stages (few rows per CTA) need many of them to keep enough bytes in flight
 constexpr int kMaxTokens = 256;
 constexpr int kMaxRows = 256;   // weight rows per CTA: two MMA tiles
-constexpr uint32_t kBarRegion = 256;
+constexpr uint32_t kBarRegion = 512;
 constexpr size_t kSmemBudget = 224 * 1024;
 constexpr size_t kSmemSlack = 1024 /*alignment*/ + kTile * kBK * 2 /*an MMA over a short tile reads 128 rows*/;
 
@@ -51,13 +51,15 @@ struct GemmShape {
 };
 
 // weight_rows: rows (gate/up: channels; down: output columns) per CTA, at most kMaxRows
-inline GemmShape gemm_shape(int tokens, int weight_rows) {
+// boxes: 64-element contraction blocks per stage (gate/up kernel only: with few rows per CTA a stage of one block is
+// so small that the per-stage hand-overs, not HBM, set the pace; two blocks per stage halve their number)
+inline GemmShape gemm_shape(int tokens, int weight_rows, int boxes = 1) {
     GemmShape s{};
     s.tn = (tokens + 31) & ~31;
     const int cols = s.tn * (weight_rows > kTile ? 2 : 1);
     s.tmem_cols = cols <= 32 ? 32 : cols <= 64 ? 64 : cols <= 128 ? 128 : cols <= 256 ? 256 : 512;
-    s.w_bytes = (uint32_t)weight_rows * kBK * 2;
-    s.stage_bytes = s.w_bytes + (uint32_t)s.tn * kBK * 2;
+    s.w_bytes = (uint32_t)weight_rows * kBK * 2 * (uint32_t)boxes;
+    s.stage_bytes = s.w_bytes + (uint32_t)s.tn * kBK * 2 * (uint32_t)boxes;
     const size_t room = kSmemBudget - kSmemSlack - kBarRegion;
     s.stages = (int)std::min<size_t>(kMaxStages, room / s.stage_bytes);
     s.smem = kSmemSlack + (size_t)s.stages * s.stage_bytes + kBarRegion;
@@ -75,6 +77,19 @@ struct GateUpParams {
     int ldf;
     int *counters, n_counters;  // zeroed here for the down kernel
     int *status;
+    int boxes;  // 64-element contraction blocks per stage (1 or 2); k_blocks counts stages
+    // Which matrices the grid covers: CTA b works on matrix prob0 + b / ctas_per_matrix (prob0 = 0 and a grid of
+    // 2 * ctas_per_matrix: both, as one launch; the overlapped form launches the kernel once per matrix).
+    int prob0;
+    // mask_mode (the up projection of the overlapped form): instead of storing U, the epilogue forms the masked hidden
+    // state Z' = SiLU(G) . M . U (Eq. (MoC-2)) for its channels from the gate values in G and the selection bitmaps
+    // that the select kernel left, and stores it as bf16 [T, ldz].  The kernel then reads x without waiting for the
+    // kernels before it: it is only launched once the kernel that wrote G has completed, which itself read x.
+    int mask_mode;
+    const uint32_t *kept_bits;  // [T, kept_words]: bit j of a token's words = channel j is kept
+    int kept_words;
+    __nv_bfloat16 *Z;           // [T, ldz]
+    int ldz;
 };
 
 struct DownParams {
@@ -127,10 +142,13 @@ __global__ void __launch_bounds__(kThreads, 1) sb_gate_up_kernel(const __grid_co
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_holder + 1);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     tc::pdl_launch_dependents();
+    MOC_TL(p.mask_mode ? 32 : 0);
+    MOC_TL_CTA(p.mask_mode ? 1536 : 256);
 
-    const int prob = (int)blockIdx.x / p.ctas_per_matrix;
-    const int ch0 = ((int)blockIdx.x - prob * p.ctas_per_matrix) * p.rows;
+    const int prob = p.prob0 + (int)blockIdx.x / p.ctas_per_matrix;
+    const int ch0 = ((int)blockIdx.x % p.ctas_per_matrix) * p.rows;
     const int ahead = min(p.stages, p.k_blocks);
+    const uint32_t w_box = (uint32_t)p.rows * kBK * 2, x_box = (uint32_t)p.tn * kBK * 2;  // one 64-element block of each
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
@@ -145,7 +163,8 @@ __global__ void __launch_bounds__(kThreads, 1) sb_gate_up_kernel(const __grid_co
         // their activation boxes after the dependency wait
         for (int kb = 0; kb < ahead; ++kb) {
             tc::mbar_expect_tx(ring.full(kb), p.stage_bytes);
-            tc::tma_load_2d(ring.stage(kb), &p.w_map[prob], ring.full(kb), kb * kBK, ch0);
+            for (int b = 0; b < p.boxes; ++b)
+                tc::tma_load_2d(ring.stage(kb) + (uint32_t)b * w_box, &p.w_map[prob], ring.full(kb), (kb * p.boxes + b) * kBK, ch0);
         }
     }
     if (warp == 1) {
@@ -160,16 +179,22 @@ __global__ void __launch_bounds__(kThreads, 1) sb_gate_up_kernel(const __grid_co
 
     if (warp == 0) {
         if (lane == 0) {
-            tc::pdl_wait();
+            if (!p.mask_mode) tc::pdl_wait();
             for (int kb = 0; kb < ahead; ++kb)
-                tc::tma_load_2d(ring.stage(kb) + p.w_bytes, &p.x_map, ring.full(kb), kb * kBK, 0);
+                for (int b = 0; b < p.boxes; ++b)
+                    tc::tma_load_2d(ring.stage(kb) + p.w_bytes + (uint32_t)b * x_box, &p.x_map, ring.full(kb),
+                                    (kb * p.boxes + b) * kBK, 0);
             int stage = 0;
             uint32_t phase = 1;  // the ring has gone round once
             for (int kb = ahead; kb < p.k_blocks; ++kb) {
                 if (!tc::mbar_wait(ring.empty(stage), phase ^ 1u, abort_flag, p.status)) break;
                 tc::mbar_expect_tx(ring.full(stage), p.stage_bytes);
-                tc::tma_load_2d(ring.stage(stage), &p.w_map[prob], ring.full(stage), kb * kBK, ch0);
-                tc::tma_load_2d(ring.stage(stage) + p.w_bytes, &p.x_map, ring.full(stage), kb * kBK, 0);
+                for (int b = 0; b < p.boxes; ++b) {
+                    tc::tma_load_2d(ring.stage(stage) + (uint32_t)b * w_box, &p.w_map[prob], ring.full(stage),
+                                    (kb * p.boxes + b) * kBK, ch0);
+                    tc::tma_load_2d(ring.stage(stage) + p.w_bytes + (uint32_t)b * x_box, &p.x_map, ring.full(stage),
+                                    (kb * p.boxes + b) * kBK, 0);
+                }
                 if (++stage == p.stages) {
                     stage = 0;
                     phase ^= 1u;
@@ -188,16 +213,18 @@ __global__ void __launch_bounds__(kThreads, 1) sb_gate_up_kernel(const __grid_co
                     break;
                 }
                 tc::tc_fence_after();
-                const uint32_t sa = ring.stage(stage), sb = sa + p.w_bytes;
+                for (int b = 0; b < p.boxes; ++b) {
+                    const uint32_t sa = ring.stage(stage) + (uint32_t)b * w_box, sb = ring.stage(stage) + p.w_bytes + (uint32_t)b * x_box;
 #pragma unroll
-                for (int k = 0; k < kBK / 16; ++k) {
-                    const uint64_t bd = tc::make_smem_desc(sb + k * 32, 16, 1024);
-                    tc::umma_bf16(tmem_base, tc::make_smem_desc(sa + k * 32, 16, 1024), bd, idesc,
-                                  (kb | k) != 0 ? 1u : 0u);
-                    if (extra)
-                        tc::umma_bf16(tmem_base + (uint32_t)p.tn,
-                                      tc::make_smem_desc(sa + (uint32_t)extra * 128u + k * 32, 16, 1024), bd, idesc,
-                                      (kb | k) != 0 ? 1u : 0u);
+                    for (int k = 0; k < kBK / 16; ++k) {
+                        const uint64_t bd = tc::make_smem_desc(sb + k * 32, 16, 1024);
+                        tc::umma_bf16(tmem_base, tc::make_smem_desc(sa + k * 32, 16, 1024), bd, idesc,
+                                      (kb | b | k) != 0 ? 1u : 0u);
+                        if (extra)
+                            tc::umma_bf16(tmem_base + (uint32_t)p.tn,
+                                          tc::make_smem_desc(sa + (uint32_t)extra * 128u + k * 32, 16, 1024), bd, idesc,
+                                          (kb | b | k) != 0 ? 1u : 0u);
+                    }
                 }
                 tc::umma_commit(ring.empty(stage));
                 if (++stage == p.stages) {
@@ -206,23 +233,51 @@ __global__ void __launch_bounds__(kThreads, 1) sb_gate_up_kernel(const __grid_co
                 }
             }
             if (ok) tc::umma_commit(ring.tfull());
+            MOC_TL_IF(p.mask_mode ? 34 : 2, blockIdx.x == 0);
+            MOC_TL_CTA_ANY(p.mask_mode ? 1792 : 512);
         }
     } else {
         // ---- epilogue: lane = channel, columns = tokens; a warp's store of one token is 128 contiguous bytes
         const int quarter = warp & 3;
         tc::pdl_wait();  // the workspace may still be read by the previous call's kernels
+        MOC_TL_IF(p.mask_mode ? 35 : 3, blockIdx.x == 0 && threadIdx.x == 64);
         if (blockIdx.x == 0)
             for (int i = (int)threadIdx.x - 64; i < p.n_counters; i += kEpiThreads) p.counters[i] = 0;
+        const int valid = min(p.rows, p.F - ch0);  // channels of this CTA inside the matrix
+        // mask mode: the factors SiLU(g) . M of this thread's first items (four channels of one token each, as the loop
+        // after the accumulators' transposition deals them out) are fetched now, while the main loop still runs
+        constexpr int kPre = 4;
+        float4 sf[kPre];
+        const int quads_pre = valid >> 2;
+        if (p.mask_mode) {
+#pragma unroll
+            for (int q = 0; q < kPre; ++q) {
+                sf[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+                const int i = (int)threadIdx.x - 64 + q * kEpiThreads;
+                if ((valid & 3) == 0 && i < p.T * quads_pre) {
+                    const int t = i / quads_pre, ch = ch0 + ((i - t * quads_pre) << 2);
+                    const uint32_t nib = (p.kept_bits[(int64_t)t * p.kept_words + (ch >> 5)] >> (ch & 31)) & 0xfu;
+                    if (nib) {
+                        const float4 g4 = *reinterpret_cast<const float4 *>(p.G + (int64_t)t * p.ldf + ch);
+                        if (nib & 1u) sf[q].x = silu_f(key_to_float(gate_key(g4.x)));
+                        if (nib & 2u) sf[q].y = silu_f(key_to_float(gate_key(g4.y)));
+                        if (nib & 4u) sf[q].z = silu_f(key_to_float(gate_key(g4.z)));
+                        if (nib & 8u) sf[q].w = silu_f(key_to_float(gate_key(g4.w)));
+                    }
+                }
+            }
+        }
         if (__all_sync(0xffffffffu, tc::mbar_wait(ring.tfull(), 0u, abort_flag, p.status))) {
             tc::tc_fence_after();
             float *base = prob == 0 ? p.G : p.U;
+            if (p.mask_mode) base = nullptr;  // nothing of U is stored
             const int trow = quarter * 32 + lane;  // row of the MMA tile this thread reads
-            const int valid = min(p.rows, p.F - ch0);  // channels of this CTA inside the matrix
             // The tile goes through the (now idle) stage ring, transposed to [token][channel], and leaves as one
             // bulk store per token: 128 scalar stores per thread would add microseconds to the end of the kernel.
             // A channel count that is not a multiple of 4 (a ragged last CTA) cannot be a bulk copy, and the tile of a
             // large batch of long rows may not fit the ring: direct stores.
-            const bool bulk = (valid & 3) == 0 && (uint32_t)p.T * (uint32_t)p.rows * 4u <= (uint32_t)p.stages * p.stage_bytes;
+            const bool fits = (uint32_t)p.T * (uint32_t)p.rows * 4u <= (uint32_t)p.stages * p.stage_bytes;
+            const bool bulk = (valid & 3) == 0 && fits;
             const uint32_t pitch = (uint32_t)p.rows * 4u;
             float *stage_f = reinterpret_cast<float *>(smem_raw + (ring.base - raw));
             // work items = (tile, 32-token chunk); the two warps of a lane quarter take alternate items
@@ -238,6 +293,19 @@ __global__ void __launch_bounds__(kThreads, 1) sb_gate_up_kernel(const __grid_co
                 tc::tmem_ld_wait();
                 if (!mine) {
                     // (no early exit: the TMEM load above is warp-collective)
+                } else if (p.mask_mode && !bulk) {
+                    // ragged channel count or a tile too large for the ring: this thread's channel, token by token
+                    const int ch = ch0 + row;
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        const int t = c0 + i;
+                        if (t < p.T) {
+                            const bool kept = (p.kept_bits[(int64_t)t * p.kept_words + (ch >> 5)] >> (ch & 31)) & 1u;
+                            float z = 0.f;
+                            if (kept) z = silu_f(key_to_float(gate_key(p.G[(int64_t)t * p.ldf + ch]))) * __uint_as_float(r[i]);
+                            p.Z[(int64_t)t * p.ldz + ch] = __float2bfloat16_rn(z);
+                        }
+                    }
                 } else if (bulk) {
                     float *dst = stage_f + (size_t)c0 * p.rows + row;
 #pragma unroll
@@ -250,7 +318,37 @@ __global__ void __launch_bounds__(kThreads, 1) sb_gate_up_kernel(const __grid_co
                         if (c0 + i < p.T) dst[(int64_t)i * p.ldf] = __uint_as_float(r[i]);
                 }
             }
-            if (bulk) {
+            if (bulk && p.mask_mode) {
+                // the tile lies in shared memory as [token][channel]: four channels per step, kept ones multiplied by
+                // SiLU of their gate value (recovered from its key, so that a NaN acts as -inf here as in the selection)
+                asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
+                const int etid = (int)threadIdx.x - 64, quads = valid >> 2;
+#pragma unroll
+                for (int q = 0; q < kPre; ++q) {  // the items whose factors are in registers already
+                    const int i = etid + q * kEpiThreads;
+                    if (i < p.T * quads) {
+                        const int t = i / quads, c = (i - t * quads) << 2;
+                        const float4 u4 = *reinterpret_cast<const float4 *>(stage_f + (size_t)t * p.rows + c);
+                        *reinterpret_cast<uint2 *>(p.Z + (int64_t)t * p.ldz + ch0 + c) =
+                            make_uint2(tc::pack_bf16(sf[q].x * u4.x, sf[q].y * u4.y), tc::pack_bf16(sf[q].z * u4.z, sf[q].w * u4.w));
+                    }
+                }
+                for (int i = etid + kPre * kEpiThreads; i < p.T * quads; i += kEpiThreads) {
+                    const int t = i / quads, c = (i - t * quads) << 2, ch = ch0 + c;
+                    const float4 u4 = *reinterpret_cast<const float4 *>(stage_f + (size_t)t * p.rows + c);
+                    const uint32_t nib = (p.kept_bits[(int64_t)t * p.kept_words + (ch >> 5)] >> (ch & 31)) & 0xfu;
+                    float z[4] = {0.f, 0.f, 0.f, 0.f};
+                    if (nib) {
+                        const float4 g4 = *reinterpret_cast<const float4 *>(p.G + (int64_t)t * p.ldf + ch);
+                        const float gv[4] = {g4.x, g4.y, g4.z, g4.w}, uv[4] = {u4.x, u4.y, u4.z, u4.w};
+#pragma unroll
+                        for (int e = 0; e < 4; ++e)
+                            if ((nib >> e) & 1u) z[e] = silu_f(key_to_float(gate_key(gv[e]))) * uv[e];
+                    }
+                    *reinterpret_cast<uint2 *>(p.Z + (int64_t)t * p.ldz + ch) =
+                        make_uint2(tc::pack_bf16(z[0], z[1]), tc::pack_bf16(z[2], z[3]));
+                }
+            } else if (bulk) {
                 tc::fence_async_smem();
                 asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
                 const int etid = (int)threadIdx.x - 64;
@@ -270,6 +368,8 @@ __global__ void __launch_bounds__(kThreads, 1) sb_gate_up_kernel(const __grid_co
     }
     tc::tc_fence_before();
     __syncthreads();
+    MOC_TL(p.mask_mode ? 36 : 4);
+    MOC_TL_CTA(p.mask_mode ? 2048 : 768);
     if (warp == 1) {
         tc::tc_fence_after();
         tc::tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
@@ -287,6 +387,10 @@ struct SelectParams {
     __nv_bfloat16 *g_out, *u_out;
     int stage_u;         // 1: shared memory has room for the token's up row as well
     int *status;
+    // the overlapped form: when not null the kernel writes only the token's selection bitmap (kept_words words: bit j =
+    // channel j is kept) and zeroes the accumulator; U and Z are not touched (the up kernel's epilogue forms Z')
+    uint32_t *kept_bits;
+    int kept_words;
 };
 
 // dynamic shared memory of sb_select_kernel: keys [Fp] | 2 candidate lists | up row [Fp] (when staged)
@@ -311,8 +415,18 @@ __global__ void __launch_bounds__(dec::kSelThreads) sb_select_kernel(const Selec
     uint32_t *bits = lists;  // bitmap of the kept channels once the search is over
     const float *u_row = p.stage_u ? reinterpret_cast<const float *>(lists + 2 * dec::kSelListCap)
                                    : p.U + (int64_t)t * p.ldf;
-    tc::pdl_launch_dependents();
-    tc::pdl_wait();
+    MOC_TL(16);
+    if (p.kept_bits) {
+        // the up kernel behind this one streams its weights while the selection runs; it may start only now that the
+        // gate kernel has completed (it reads x without a wait of its own)
+        tc::pdl_wait();
+        tc::pdl_launch_dependents();
+        MOC_TL(17);
+        MOC_TL_CTA(1024);
+    } else {
+        tc::pdl_launch_dependents();
+        tc::pdl_wait();
+    }
     dec::cta_stage_rows_begin(&s_bar, &s_abort, keys, p.G + (int64_t)t * p.ldf, (uint32_t)Fp * 4u,
                               p.stage_u ? lists + 2 * dec::kSelListCap : nullptr,
                               p.stage_u ? p.U + (int64_t)t * p.ldf : nullptr);
@@ -324,6 +438,31 @@ __global__ void __launch_bounds__(dec::kSelThreads) sb_select_kernel(const Selec
     bool ties_cut;
     uint32_t kreg[dec::kSelCached];
     dec::cta_select_threshold(nullptr, p.F, p.K, keys, lists, sm, tau, need, ties_cut, kreg);
+    if (p.kept_bits) {
+        uint32_t *my_bits = p.kept_bits + (int64_t)t * p.kept_words;
+        const int lane = tid & 31, warp = tid >> 5;
+        constexpr int NW = dec::kSelThreads / 32;
+        if (!ties_cut) {
+            // consecutive lanes hold consecutive channels: a ballot is a word of the bitmap
+            const int nch = (p.F + dec::kSelThreads - 1) / dec::kSelThreads;
+            for (int c = 0; c < nch; ++c) {
+                const int j = c * dec::kSelThreads + tid;
+                const uint32_t b = __ballot_sync(0xffffffffu, j < p.F && keys[j] >= tau);
+                if (lane == 0 && c * dec::kSelThreads + warp * 32 < p.F) my_bits[c * NW + warp] = b;
+            }
+        } else {
+            __syncthreads();
+            for (int i = tid; i < p.kept_words; i += dec::kSelThreads) bits[i] = 0u;
+            __syncthreads();
+            block_ordered_emit<dec::kSelThreads>(keys, p.F, tau, need, sm,
+                                                 [&](int, int j) { atomicOr(&bits[j >> 5], 1u << (j & 31)); });
+            __syncthreads();
+            for (int i = tid; i < p.kept_words; i += dec::kSelThreads) my_bits[i] = bits[i];
+        }
+        MOC_TL(18);
+        MOC_TL_CTA(1280);
+        return;
+    }
     const bool save = p.idx_out != nullptr;
     const bool by_bitmap = ties_cut || save;
     if (by_bitmap) {
@@ -456,6 +595,8 @@ __global__ void __launch_bounds__(kThreads, 1) sb_down_kernel(const __grid_const
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_holder + 1);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     tc::pdl_launch_dependents();
+    MOC_TL(48);
+    MOC_TL_CTA(2304);
 
     const int m_blk = (int)blockIdx.x / p.splits, split = (int)blockIdx.x - m_blk * p.splits;
     const int kb_all = p.k_blocks * p.segments;
@@ -503,6 +644,8 @@ __global__ void __launch_bounds__(kThreads, 1) sb_down_kernel(const __grid_const
     if (warp == 0) {
         if (lane == 0) {
             tc::pdl_wait();  // Z' comes from the select kernel
+            MOC_TL_IF(49, blockIdx.x == 0);
+            MOC_TL_CTA_ANY(2560);
             for (int i = 0; i < ahead; ++i) load_z(i, kb0 + i);
             int stage = 0;
             uint32_t phase = 1;
@@ -545,6 +688,7 @@ __global__ void __launch_bounds__(kThreads, 1) sb_down_kernel(const __grid_const
                 }
             }
             if (ok) tc::umma_commit(ring.tfull());
+            MOC_TL_CTA_ANY(2816);
         }
     } else {
         // ---- epilogue: lane = output column, TMEM columns = tokens
@@ -614,6 +758,23 @@ __global__ void __launch_bounds__(kThreads, 1) sb_down_kernel(const __grid_const
             const uint8_t *stage_ptr = smem_raw + (ring.base - raw);
             const int vecs = cols / 4;
             uint32_t parity = 0;
+            if (p.T * vecs <= 4 * kEpiThreads) {
+                // a few vectors per thread: independent loads from L2 (where the reductions left the sums) cost one round
+                // trip, less than setting up and awaiting the bulk copies
+                for (int i = etid; i < p.T * vecs; i += kEpiThreads) {
+                    const int t = i / vecs, c = (i - t * vecs) * 4;
+                    float4 v = __ldcg(reinterpret_cast<const float4 *>(p.acc + (int64_t)t * p.d + col0 + c));
+                    if (p.resid) {
+                        const uint2 hb = *reinterpret_cast<const uint2 *>(p.resid + (int64_t)t * p.d + col0 + c);
+                        v.x += __uint_as_float(hb.x << 16);
+                        v.y += __uint_as_float(hb.x & 0xffff0000u);
+                        v.z += __uint_as_float(hb.y << 16);
+                        v.w += __uint_as_float(hb.y & 0xffff0000u);
+                    }
+                    *reinterpret_cast<uint2 *>(p.out + (int64_t)t * p.d + col0 + c) =
+                        make_uint2(tc::pack_bf16(v.x, v.y), tc::pack_bf16(v.z, v.w));
+                }
+            } else
             for (int t0 = 0; t0 < p.T; t0 += per_round, parity ^= 1u) {
                 const int nt = min(per_round, p.T - t0);
                 asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");  // the ring is free again
@@ -650,6 +811,8 @@ __global__ void __launch_bounds__(kThreads, 1) sb_down_kernel(const __grid_const
     }
     tc::tc_fence_before();
     __syncthreads();
+    MOC_TL(52);
+    MOC_TL_CTA(3072);
     if (warp == 1) {
         tc::tc_fence_after();
         tc::tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);

@@ -1,0 +1,66 @@
+"""Device-clock timeline of one moc_ffn_decode call on the LLaMA-7B shape (development aid).
+
+Needs a library built with the stamps compiled in:
+
+    MOC_FFN_NVCC_FLAGS=-DMOC_TIMELINE python -m paper_2511_09323_b200.build --force
+    python -m paper_2511_09323_b200.decode_timeline 16
+    python -m paper_2511_09323_b200.build --force          # back to the normal build
+
+Eight calls rotating four weight sets are replayed from one CUDA graph; every CTA of the small-batch kernels notes the
+GPU's nanosecond timer at a few points (the last call's stamps survive).  Printed: minimum / median / maximum over the
+CTAs of a kernel, relative to the moment the previous call had completed.
+"""
+import ctypes
+import sys
+
+import numpy as np
+import torch
+
+from . import binding as B
+from . import synthetic as syn
+
+REGIONS = [(256, "gate start"), (512, "gate mma done"), (768, "gate end"), (1024, "select after wait"),
+           (1280, "select end"), (1536, "up start"), (1792, "up mma done"), (2048, "up end"), (2304, "down start"),
+           (2560, "down after wait"), (2816, "down mma done"), (3072, "down end")]
+
+
+def main():
+    T = int(sys.argv[1]) if len(sys.argv) > 1 else 16
+    lib = B.load()
+    if not hasattr(lib, "moc_debug_timeline"):
+        raise SystemExit("this build has no stamps: rebuild with MOC_FFN_NVCC_FLAGS=-DMOC_TIMELINE")
+    w = syn.C4
+    sets = [tuple(t.cuda() for t in syn.make_weights(w, seed_offset=s)) for s in range(4)]
+    x = syn.make_x(w, tokens=T).cuda()
+    out = torch.empty_like(x)
+    desc = B.make_desc(T, w.d_model, w.d_ff, w.k, x.dtype)
+    ws = B.alloc_workspace(desc, B.MOC_OP_DECODE)
+    stream = torch.cuda.Stream()
+    for i in range(4):
+        B.moc_ffn_decode(x, *sets[i % 4], w.k, out=out, workspace=ws)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        with torch.cuda.graph(graph, stream=stream):
+            for i in range(8):
+                B.moc_ffn_decode(x, *sets[i % 4], w.k, out=out, workspace=ws, stream=stream)
+    for _ in range(3):
+        graph.replay()
+    torch.cuda.synchronize()
+    buf = (ctypes.c_ulonglong * 4096)()
+    lib.moc_debug_timeline.argtypes = [ctypes.c_void_p, ctypes.c_int]
+    if lib.moc_debug_timeline(buf, 4096) != 0:
+        raise SystemExit("reading the stamps failed")
+    a = np.array(buf, dtype=np.uint64).astype(np.int64)
+    ref = a[3] if a[3] else min(v for v in a[256:512] if v > 0)   # the first kernel's wait for the previous call returned
+    print(f"T = {T}: us after the previous call completed -- min / median / max over CTAs (n)")
+    for base, name in REGIONS:
+        v = a[base:base + 256]
+        v = v[v > 0]
+        if len(v):
+            r = (v - ref) / 1000.0
+            print(f"{name:18s} {r.min():8.2f} {np.median(r):8.2f} {r.max():8.2f}   ({len(v)})")
+
+
+if __name__ == "__main__":
+    main()

@@ -100,14 +100,14 @@ def test_static_decode_honours_the_post_silu_key(dtype, T, d, F, F_ld, K):
     assert not np.array_equal(ref["idx"], pre["idx"])
     got = syn.to_f64(out)
     scale = np.abs(ref["out"]).max()
-    # tokens whose post-SiLU threshold is not a near-tie must match the oracle's post-SiLU output (and not the default rule's)
-    s_sorted = np.sort(ref["s"], axis=1)[:, ::-1]
-    clear = (s_sorted[:, K - 1] - s_sorted[:, K]) > 1e-3
-    assert clear.sum() >= T // 2
+    # With every gate value negative the post-SiLU rule keeps the channels whose SiLU is closest to zero; the channels
+    # at its threshold carry SiLU values of a few 1e-3, so a near-tie there decided the other way moves the output by
+    # far less than the tolerance: every token must match the oracle's post-SiLU output, and none the default rule's.
     err = np.abs(got - ref["out"]).max(axis=1)
-    assert np.all(err[clear] <= REL[dtype] * scale), f"{err[clear].max():.3e} vs {REL[dtype] * scale:.3e}"
+    assert np.all(err <= REL[dtype] * scale), f"{err.max():.3e} vs {REL[dtype] * scale:.3e}"
     differs = np.abs(pre["out"] - ref["out"]).max(axis=1) > 10 * REL[dtype] * scale
-    assert np.all(np.abs(got - pre["out"]).max(axis=1)[clear & differs] > REL[dtype] * scale)
+    assert differs.sum() >= T // 2
+    assert np.all(np.abs(got - pre["out"]).max(axis=1)[differs] > REL[dtype] * scale)
     assert (out.double() - ref_dev.double()).abs().max().item() <= REL[dtype] * scale
 
 
