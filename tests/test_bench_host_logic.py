@@ -72,7 +72,8 @@ def test_measured_traffic_is_linear_in_tokens_where_two_captures_exist(monkeypat
     got, src = bench.measured_traffic(syn.C5, 1000, "tc_wgrad_gemm", 4, 4)
     assert got == 100.0 + 3.0 * 1000 and "linear" in src
     assert bench.measured_traffic(syn.C5, 1000, "tc_wgrad_gemm", 8, 4)[0] is None     # several launches per step
-    assert bench.measured_traffic(syn.C3, 1000, "tc_wgrad_gemm", 4, 4)[0] is None
+    assert bench.measured_traffic(syn.C2, 1000, "tc_wgrad_gemm", 4, 4)[0] is None     # another shape at another size
+    assert bench.measured_traffic(syn.C5, 1000, "tc_dz_gemm", 4, 4)[0] is None        # a kernel without a capture
 
 
 def test_strict_roofline_matches_the_hand_computed_figures():
