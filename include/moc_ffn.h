@@ -292,6 +292,37 @@ MOC_API int moc_tc_gemm_bf16(int64_t m, int64_t n, int64_t k, const void *a, int
                              void *cuda_stream);
 
 /*
+ * The 2:4-sparse bf16 contraction on the sparse tensor-core MMA (tcgen05.mma.sp), exposed so that it can be checked on
+ * its own.  Section 4 ("MoC with structured 2:8 sparsity") keeps 2 of every 8 consecutive channels, so every 4
+ * consecutive channels of the masked hidden state hold at most 2 non-zero values: a row is a valid 2:4-sparse operand.
+ *     C[m, n] (fp32, row-major, ldc) = sum_k A(m, k) * B(n, k)
+ *   a_compressed  [m, k / 2] bf16, device: of every 4 consecutive contraction elements of a row of A the 2 kept ones,
+ *                 in order (k a multiple of 16)
+ *   metadata      device, ceil(m / 128) * ceil(k / 128) * 128 * 4 32-bit words: for tile row block i and block j of 128
+ *                 contraction elements, lane l (0..127), column c (0..3) the word at ((i * kb + j) * 128 + l) * 4 + c
+ *                 holds, for the 32 contraction elements 32 c .. 32 c + 31 of the block, the nibbles (position of the
+ *                 first kept element | position of the second << 2, positions 0..3 inside their group of 4) of rows
+ *                 r = (l % 8) + 16 * (l / 16) (bits 0..15) and r + 8 (bits 16..31), groups 4 * ((l / 8) % 2) .. + 3 of
+ *                 the 8 groups, four bits each in ascending order -- the arrangement tensor memory wants
+ *   b             as in moc_tc_gemm_bf16: [n, k] (b_mn_major == 0) or [k, n]
+ */
+MOC_API int moc_tc_gemm_sp_bf16(int64_t m, int64_t n, int64_t k, const void *a_compressed, const void *metadata,
+                                const void *b, int b_mn_major, int64_t ldb, float *c, int64_t ldc, void *cuda_stream);
+
+/*
+ * The same contraction the way the operator uses it: A is given DENSE ([m, k] bf16 row-major, lda, at most 2 non-zero
+ * values in every 4 consecutive elements of a row); the library compresses it (values + metadata, into the workspace)
+ * and runs the sparse MMA on CTA pairs.  b is [k, n] with n contiguous (the layout of the weight matrices in the
+ * down projection), c is bf16 [m, ldc]; accumulate != 0 adds the previous content of c before rounding.
+ * Groups of 4 with more than 2 non-zero values keep their first 2; *overflow_count (host, may be NULL; asking for it
+ * synchronises the stream) receives how many values were left out.
+ */
+MOC_API size_t moc_tc_gemm_sp_dense_workspace_bytes(int64_t m, int64_t k);
+MOC_API int moc_tc_gemm_sp_dense_bf16(int64_t m, int64_t n, int64_t k, const void *a_dense, int64_t lda, const void *b,
+                                      int64_t ldb, void *c, int64_t ldc, int accumulate, int64_t *overflow_count,
+                                      void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
  * Test hook for the time-out path every kernel of the library shares: launches one warp that waits, with the
  * library's bounded wait, on a barrier nothing completes.  After `limit_cycles` SM clock cycles (1 .. 4e9) the wait
  * gives up, the kernel raises MOC_ERR_TIMEOUT in the device status word and returns normally; nothing traps or

@@ -18,6 +18,7 @@
 #include "moc_common.cuh"
 #include "small_batch.cuh"
 #include "tc_gemm.cuh"
+#include "tc_gemm_sp.cuh"
 #include "tc_plan.cuh"
 #include "topk_select.cuh"
 
@@ -76,6 +77,9 @@ enum KernelId {
     KID_RECOMPUTE_UP,
     KID_DEC_COOP,
     KID_DEC_RMSNORM,
+    KID_TC_COMPRESS,
+    KID_TC_SP_DOWN_GEMM,
+    KID_TC_SP_DX_GEMM,
     KID_COUNT
 };
 static const char *const kKernelNames[KID_COUNT] = {
@@ -84,7 +88,8 @@ static const char *const kKernelNames[KID_COUNT] = {
     "tc_gate_up_gemm", "tc_select_mask",  "tc_down_gemm",  "tc_bwd_sample",  "tc_dz_gemm",
     "tc_wgrad_gemm",   "tc_dx_gemm",      "tc_test_gemm",  "tc_select_hint", "dec_gate_gemv",
     "dec_select",      "dec_up",          "dec_down",      "sb_gate_up",     "sb_select",
-    "sb_down",         "recompute_up",    "dec_coop",      "dec_rmsnorm",
+    "sb_down",         "recompute_up",    "dec_coop",      "dec_rmsnorm",    "tc_compress_2of4",
+    "tc_sp_down_gemm", "tc_sp_dx_gemm",
 };
 
 struct Profiler {
@@ -453,6 +458,109 @@ void tc_select_launch(const TcSelect &c, const float *G, int ldg, __nv_bfloat16 
     }
 }
 
+// ---- 2:4-sparse contractions (tcgen05.mma.sp): compressed operand + metadata in the workspace -----------------
+struct SparseOperandLayout {
+    int kc_ld;          // leading dimension of the compressed rows (elements): K / 2 rounded up to 64
+    int k_stages;       // stages of 128 logical contraction elements
+    size_t comp_bytes, meta_bytes;
+};
+SparseOperandLayout sparse_operand_layout(int64_t rows, int K) {
+    SparseOperandLayout L{};
+    L.k_stages = ceil_div(K, tcsp::SBKL);
+    L.kc_ld = L.k_stages * (tcsp::SBKL / 2);
+    const int64_t blocks = (rows + 127) / 128;
+    L.comp_bytes = align_up((size_t)blocks * 128 * L.kc_ld * sizeof(__nv_bfloat16), kAlign);
+    L.meta_bytes = align_up((size_t)blocks * L.k_stages * 128 * 4 * sizeof(uint32_t), kAlign);
+    return L;
+}
+
+// MOC_FFN_SPARSE=0 in the environment keeps every contraction on the dense MMA (comparisons)
+bool sparse_mma_enabled() {
+    static const bool on = [] {
+        const char *e = getenv("MOC_FFN_SPARSE");
+        return !(e && strcmp(e, "0") == 0);
+    }();
+    return on && tc::pair_mode();
+}
+
+// dense [rows, ld] (at most 2 non-zero values per group of 4) -> compressed rows + metadata
+int sparse_compress(const __nv_bfloat16 *dense, int64_t rows, int K, int ld, const SparseOperandLayout &L,
+                    __nv_bfloat16 *comp, uint32_t *meta, tcsp::Overflow *overflow, int overflow_cap,
+                    unsigned int *overflow_n, cudaStream_t st) {
+    const int64_t jobs = ((rows + 127) / 128) * L.k_stages;
+    const unsigned grid = (unsigned)std::min<int64_t>(jobs, (int64_t)tc::sm_count() * 8);
+    MOC_LAUNCH(KID_TC_COMPRESS, st,
+               (tcsp::compress_2of4_kernel<<<grid, 512, 0, st>>>(dense, rows, K, ld, comp, L.kc_ld, meta, L.k_stages,
+                                                                  overflow, overflow_cap, overflow_n)));
+    return launch_ok();
+}
+
+// C [M, N] bf16 = sum over segments of A_seg (compressed, [M, K]) * B_seg ([K, N], N contiguous)
+int sparse_gemm_pair(int64_t M, int N, int K, int segments, const __nv_bfloat16 *const comp[2],
+                     const uint32_t *const meta[2], const SparseOperandLayout &L, const __nv_bfloat16 *const b[2],
+                     int ldb, __nv_bfloat16 *c, int ldc, bool accumulate, int kid, int *status, cudaStream_t st) {
+    using namespace tcsp;
+    using tc::EncodeTiledFn;
+    using tc::encode_fn;
+    SpPairParams p;
+    memset(&p, 0, sizeof(p));
+    for (int sgm = 0; sgm < segments; ++sgm) {
+        // (columns K / 2 .. kc_ld of the compressed rows are never written: the map ends at K / 2)
+        if (!tc::make_map(&p.a_map[sgm], comp[sgm], M, K / 2, L.kc_ld, 64, SBM) ||
+            !tc::make_map(&p.b_map[sgm], b[sgm], K, N, ldb, 64, 64))
+            return MOC_ERR_CUDA;
+        // the metadata as a matrix of 32-bit words, 4 per row: one stage of one 128-row block is a box of 4 x 128
+        EncodeTiledFn fn = encode_fn();
+        if (!fn) return MOC_ERR_CUDA;
+        const int64_t blocks = (M + 127) / 128;
+        cuuint64_t dims[2] = {4, (cuuint64_t)(blocks * L.k_stages * 128)};
+        cuuint64_t strides[1] = {16};
+        cuuint32_t box[2] = {4, 128};
+        cuuint32_t estr[2] = {1, 1};
+        if (fn(&p.e_map[sgm], CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<uint32_t *>(meta[sgm]), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return MOC_ERR_CUDA;
+    }
+    p.segments = segments;
+    p.k_stages = L.k_stages;
+    p.M = (int)M;
+    p.N = N;
+    p.m_pairs = ceil_div(M, 2 * SBM);
+    p.n_tiles = ceil_div(N, PBN);
+    p.c = c;
+    p.ldc = ldc;
+    p.accumulate = accumulate ? 1 : 0;
+    p.status = status;
+    static int max_pairs = 0;
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.blockDim = dim3(PTHREADS);
+    cfg.dynamicSmemBytes = PSMEM_BYTES;
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (!max_pairs) {
+        if (cudaFuncSetAttribute(gemm_sp_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PSMEM_BYTES) != cudaSuccess)
+            return MOC_ERR_CUDA;
+        cfg.gridDim = dim3(2 * (unsigned)tc::sm_count());
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, gemm_sp_pair_kernel, &cfg) != cudaSuccess || n <= 0) return MOC_ERR_CUDA;
+        max_pairs = n;
+    }
+    const int tiles = p.m_pairs * p.n_tiles;
+    const int pairs = std::min(tiles, max_pairs);
+    if (pairs <= 0) return MOC_OK;
+    cfg.gridDim = dim3(2 * (unsigned)pairs);
+    int rc = MOC_OK;
+    MOC_LAUNCH(kid, st, (rc = cudaLaunchKernelEx(&cfg, gemm_sp_pair_kernel, p) == cudaSuccess ? MOC_OK : MOC_ERR_CUDA));
+    return rc;
+}
+
 // D = Z' W_down over all tokens: A = Z' [T, F] (K-major), B = Wd [F, d] (its contiguous dimension is N)
 int forward_tc_down(const moc_ffn_desc &d, const __nv_bfloat16 *Z, int ldz, const __nv_bfloat16 *wd, __nv_bfloat16 *out,
                     int *status, cudaStream_t st) {
@@ -513,8 +621,27 @@ int forward_tc(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat1
         q.sv_idx = idx;
         q.sv_g = idx ? tg : nullptr;
         q.sv_u = idx ? tu : nullptr;
+        // Every 4 consecutive channels of a 2:8 row hold at most 2 kept values: the epilogue hands Z' over in the
+        // compressed form of the 2:4-sparse MMA, and the down projection contracts over twice the channels per instruction
+        const SparseOperandLayout SL = sparse_operand_layout(T, F);
+        // (the compressed rows live in U's buffer; with few output columns the GEMM is too short for its 1.5 x to pay
+        // for the slower epilogue of the gate + up GEMM: LLaMA-130M shape 0.170 -> 0.174 ms, LLaMA-1B shape 1.57 -> 1.43 ms)
+        const bool sparse_down = sparse_mma_enabled() && SL.kc_ld <= L.ldf && dm >= 1024;
+        uint32_t *zmeta = reinterpret_cast<uint32_t *>(ws + L.off_meta);
+        if (sparse_down) {
+            q.zc = U;
+            q.zc_ld = SL.kc_ld;
+            q.zmeta = zmeta;
+            q.zmeta_stages = SL.k_stages;
+        }
         MOC_LAUNCH(KID_TC_GATE_UP_GEMM, st, (rc = launch_gemm<false, false, EPI_GATE_UP_2OF8>(q, st)));
         if (rc != MOC_OK) return rc;
+        if (sparse_down) {
+            const __nv_bfloat16 *comps[2] = {U, nullptr};
+            const uint32_t *metas[2] = {zmeta, nullptr};
+            const __nv_bfloat16 *bs[2] = {wd, nullptr};
+            return sparse_gemm_pair(T, dm, F, 1, comps, metas, SL, bs, dm, out, dm, false, KID_TC_SP_DOWN_GEMM, status, st);
+        }
         return forward_tc_down(d, U, L.ldf, wd, out, status, st);
     }
     Params p;
@@ -1657,6 +1784,88 @@ int moc_tc_gemm_bf16(int64_t m, int64_t n, int64_t k, const void *a, int a_mn_ma
     else
         MOC_LAUNCH(KID_TC_TEST_GEMM, st, (rc = launch_gemm<true, false, EPI_F32>(p, st)));
     return rc;
+}
+
+int moc_tc_gemm_sp_bf16(int64_t m, int64_t n, int64_t k, const void *a_compressed, const void *metadata, const void *b,
+                        int b_mn_major, int64_t ldb, float *c, int64_t ldc, void *cuda_stream) {
+    using namespace tcsp;
+    if (m < 1 || n < 1 || k < 16 || k % 16 != 0 || m > INT32_MAX || n > INT32_MAX || k > INT32_MAX) return MOC_ERR_INVALID_ARG;
+    if (!good_ptr(a_compressed) || !good_ptr(metadata) || !good_ptr(b) || !good_ptr(c) || ldb % 8 || ldc < n)
+        return MOC_ERR_INVALID_ARG;
+    int *status = device_status_ptr();
+    if (!status) return MOC_ERR_CUDA;
+    SpParams p;
+    memset(&p, 0, sizeof(p));
+    if (!tc::make_map(&p.a_map, a_compressed, m, k / 2, k / 2, 64, SBM)) return MOC_ERR_CUDA;
+    const bool ok_b = b_mn_major ? tc::make_map(&p.b_map, b, k, n, ldb, 64, 64) : tc::make_map(&p.b_map, b, n, k, ldb, 64, SBN);
+    if (!ok_b) return MOC_ERR_CUDA;
+    p.e = static_cast<const uint4 *>(metadata);
+    p.k_stages = ceil_div(k, SBKL);
+    p.M = (int)m;
+    p.N = (int)n;
+    p.m_tiles = ceil_div(m, SBM);
+    p.n_tiles = ceil_div(n, SBN);
+    p.c = c;
+    p.ldc = (int)ldc;
+    p.out_bf16 = 0;
+    p.status = status;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const int grid = std::min(p.m_tiles * p.n_tiles, tc::sm_count());
+    if (b_mn_major) {
+        if (cudaFuncSetAttribute(gemm_sp_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SSMEM_BYTES) != cudaSuccess)
+            return MOC_ERR_CUDA;
+        MOC_LAUNCH(KID_TC_TEST_GEMM, st, (gemm_sp_kernel<true><<<grid, STHREADS, SSMEM_BYTES, st>>>(p)));
+    } else {
+        if (cudaFuncSetAttribute(gemm_sp_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SSMEM_BYTES) != cudaSuccess)
+            return MOC_ERR_CUDA;
+        MOC_LAUNCH(KID_TC_TEST_GEMM, st, (gemm_sp_kernel<false><<<grid, STHREADS, SSMEM_BYTES, st>>>(p)));
+    }
+    return launch_ok();
+}
+
+size_t moc_tc_gemm_sp_dense_workspace_bytes(int64_t m, int64_t k) {
+    if (m < 1 || k < 8 || k % 8 != 0 || k > INT32_MAX) return 0;
+    const SparseOperandLayout L = sparse_operand_layout(m, (int)k);
+    return L.comp_bytes + L.meta_bytes + 256 + 4096 * sizeof(tcsp::Overflow);
+}
+
+int moc_tc_gemm_sp_dense_bf16(int64_t m, int64_t n, int64_t k, const void *a_dense, int64_t lda, const void *b, int64_t ldb,
+                              void *c, int64_t ldc, int accumulate, int64_t *overflow_count, void *workspace,
+                              size_t workspace_bytes, void *cuda_stream) {
+    if (m < 1 || n < 1 || k < 8 || k % 8 != 0 || m > INT32_MAX || n > INT32_MAX || k > INT32_MAX) return MOC_ERR_INVALID_ARG;
+    if (!good_ptr(a_dense) || !good_ptr(b) || !c || lda % 8 || ldb % 8 || lda < k || ldb < n || ldc < n) return MOC_ERR_INVALID_ARG;
+    if (!tc::pair_mode()) return MOC_ERR_UNSUPPORTED;
+    const size_t need = moc_tc_gemm_sp_dense_workspace_bytes(m, k);
+    if (!good_ptr(workspace) || workspace_bytes < need) return MOC_ERR_WORKSPACE;
+    int *status = device_status_ptr();
+    if (!status) return MOC_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    using B16 = __nv_bfloat16;
+    const SparseOperandLayout L = sparse_operand_layout(m, (int)k);
+    char *ws = static_cast<char *>(workspace);
+    B16 *comp = reinterpret_cast<B16 *>(ws);
+    uint32_t *meta = reinterpret_cast<uint32_t *>(ws + L.comp_bytes);
+    unsigned int *ovf_n = reinterpret_cast<unsigned int *>(ws + L.comp_bytes + L.meta_bytes);
+    tcsp::Overflow *ovf = reinterpret_cast<tcsp::Overflow *>(ws + L.comp_bytes + L.meta_bytes + 256);
+    if (cudaMemsetAsync(ovf_n, 0, 256, st) != cudaSuccess) return MOC_ERR_CUDA;
+    // rows beyond m of the last 128-row block and columns beyond k / 2 are never read as values (the maps clip), but
+    // the metadata of clipped rows must be valid nibbles: the kernel writes fillers for them
+    int rc = sparse_compress(static_cast<const B16 *>(a_dense), m, (int)k, (int)lda, L, comp, meta, ovf, 4096, ovf_n, st);
+    if (rc != MOC_OK) return rc;
+    const B16 *comps[2] = {comp, nullptr};
+    const uint32_t *metas[2] = {meta, nullptr};
+    const B16 *bs[2] = {static_cast<const B16 *>(b), nullptr};
+    rc = sparse_gemm_pair(m, (int)n, (int)k, 1, comps, metas, L, bs, (int)ldb, static_cast<B16 *>(c), (int)ldc,
+                          accumulate != 0, KID_TC_TEST_GEMM, status, st);
+    if (rc != MOC_OK) return rc;
+    if (overflow_count) {
+        unsigned int h = 0;
+        if (cudaMemcpyAsync(&h, ovf_n, sizeof(h), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+            cudaStreamSynchronize(st) != cudaSuccess)
+            return MOC_ERR_CUDA;
+        *overflow_count = h;
+    }
+    return MOC_OK;
 }
 
 int moc_test_bounded_wait(int64_t limit_cycles, void *cuda_stream) {

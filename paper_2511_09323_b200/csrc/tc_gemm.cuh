@@ -74,6 +74,13 @@ struct Params {
     // EPI_GATE_UP_2OF8: compact saved activations [M, N / 4] (all three or none)
     int16_t *sv_idx;
     __nv_bfloat16 *sv_g, *sv_u;
+    // EPI_GATE_UP_2OF8, when zc != nullptr: Z' leaves in the 2:4-compressed form of the sparse MMA instead of as a
+    // dense array -- zc [M, zc_ld] holds the 2 kept (or filler) values of every 4 channels, zmeta the metadata words in
+    // the arrangement tensor memory wants ([128-row block][block of 128 channels][row of the block][4 words])
+    __nv_bfloat16 *zc;
+    int zc_ld;
+    uint32_t *zmeta;
+    int zmeta_stages;
     int *status;
 };
 
@@ -408,6 +415,35 @@ __device__ __forceinline__ void epilogue_tile(const Params &p, int prob, int row
     }
 }
 
+// Four consecutive bf16 values (w0 = elements 0, 1; w1 = elements 2, 3) with at most two non-zero ones -> the two
+// kept values (in order) and the metadata nibble of the sparse MMA: position of the first | position of the second
+// << 2, positions ascending; a group with fewer than two non-zero values points its fillers at zero elements.
+__device__ __forceinline__ void compress_group4(uint32_t w0, uint32_t w1, uint32_t &packed, uint32_t &nib) {
+    const uint32_t e[4] = {w0 & 0xffffu, w0 >> 16, w1 & 0xffffu, w1 >> 16};
+    int p0 = -1, p1 = -1;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const bool nz = (e[j] & 0x7fffu) != 0u;
+        if (nz && p0 < 0) p0 = j;
+        else if (nz && p1 < 0) p1 = j;
+    }
+    if (p0 < 0) {
+        p0 = 0;
+        p1 = 1;
+    } else if (p1 < 0) {
+        p1 = 3;
+        if (p0 == 3) p0 = 2;
+    }
+    uint32_t v0 = 0u, v1 = 0u;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        if (j == p0) v0 = e[j];
+        if (j == p1) v1 = e[j];
+    }
+    packed = v0 | (v1 << 16);
+    nib = (uint32_t)p0 | ((uint32_t)p1 << 2);
+}
+
 // Group G8 (channels 8 G8 .. 8 G8 + 7) of a 32-channel chunk: r = gate accumulators, q = up accumulators of one row.
 // Writes the group's four words of Z' and its two saved entries (index pair, gate pair, up pair).
 template <int G8>
@@ -474,7 +510,7 @@ __device__ __forceinline__ void epilogue_tile_2of8(const Params &p, int row0, in
     const bool vec_saves = (K & 7) == 0;          // 16-byte stores of eight saved entries need 16-byte aligned rows
     const uint32_t my_row = (uint32_t)lane * 128u, sw = (uint32_t)(lane & 7);
     if (row0 >= p.M || ch0 + 64 * half >= p.N) return;
-    if (!direct) {
+    if (!direct && !p.zc) {
         if (lane == 0) bulk_store_wait_read<0>();  // the previous tile's store has read the box
         __syncwarp();
     }
@@ -509,6 +545,29 @@ __device__ __forceinline__ void epilogue_tile_2of8(const Params &p, int row0, in
                         reinterpret_cast<uint32_t *>(p.sv_u + o)[g8] = uw[g8];
                     }
             }
+        }
+        if (p.zc) {
+            // ---- Z' in compressed form: 16 values and one metadata word for the chunk's 32 channels.  The word of a
+            // tensor-memory lane joins the 16 bits of two rows eight apart (lane ^ 8), for the chunk's first or second
+            // 16 channels: rows with bit 3 clear build the words of the first half, the others those of the second.
+            uint32_t pk[8], half16[2] = {0u, 0u};
+#pragma unroll
+            for (int g = 0; g < 8; ++g) {
+                uint32_t nib;
+                compress_group4(zw[2 * g], zw[2 * g + 1], pk[g], nib);
+                half16[g >> 2] |= nib << (4 * (g & 3));
+            }
+            const bool upper = (lane & 8) != 0;
+            const uint32_t got = __shfl_xor_sync(0xffffffffu, upper ? half16[0] : half16[1], 8);
+            const uint32_t word = upper ? (got | (half16[1] << 16)) : (half16[0] | (got << 16));
+            const int64_t blk = row0 >> 7;  // row0 is a multiple of 32 inside a 128-row block
+            p.zmeta[((blk * p.zmeta_stages + (col >> 7)) * 128 + ((row0 & 127) + lane)) * 4 + ((col >> 5) & 3)] = word;
+            if (row_ok) {
+                uint4 *dst = reinterpret_cast<uint4 *>(p.zc + (int64_t)row * p.zc_ld + (col >> 1));
+                dst[0] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                dst[1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+            }
+            continue;
         }
         // ---- Z': the warp's two chunks share one 32-row x 128-byte box
         if (direct) {

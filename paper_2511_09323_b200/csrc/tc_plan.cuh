@@ -949,6 +949,9 @@ struct TcForwardLayout {
     size_t off_g;   // fp32 G of one chunk [chunk, ldf]
     size_t off_u;   // bf16 U, rewritten in place into Z', for ALL tokens [T, ldf]
     size_t off_hint;  // bracket {center, width, tag}, statistics {sum, sum|dev|, rows}, CTA counter
+    // MoC 2:8 on the sparse MMA: Z' in compressed form lives where U would (it is half as large), its metadata here
+    size_t off_meta, meta_bytes;
+    int sp_k_stages;  // blocks of 128 channels
     size_t total;
 };
 struct TcBackwardLayout {
@@ -985,6 +988,10 @@ inline TcForwardLayout tc_forward_layout(const moc_ffn_desc &d) {
     off = align_up(off + (size_t)all_m * BM * L.ldf * 2, 256);
     L.off_hint = off;
     off += 256;
+    L.sp_k_stages = (d.d_ff + 127) / 128;
+    L.off_meta = off;
+    L.meta_bytes = (d.flags & MOC_FLAG_SELECT_2_OF_8) ? align_up((size_t)all_m * L.sp_k_stages * 128 * 16, 256) : 0;
+    off += L.meta_bytes;
     L.total = off;
     return L;
 }
