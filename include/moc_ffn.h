@@ -76,8 +76,13 @@ typedef enum { MOC_OP_FORWARD = 0, MOC_OP_BACKWARD = 1, MOC_OP_DECODE = 2, MOC_O
  * instead of the K largest gate values of the whole row, the 2 largest of every group of 8 consecutive channels are
  * kept (signed pre-SiLU values, equal values: the lower channel, NaN as -inf).  Requires d_ff % 8 == 0 and
  * k == d_ff / 4; the kept channels of group q occupy slots 2q and 2q + 1 of topk_idx / topk_gate / topk_up.
- * Honoured by moc_ffn_forward, moc_ffn_decode and moc_ffn_decode_static; moc_ffn_backward takes the saved
- * indices as they are (the flag changes nothing there). */
+ * Honoured by moc_ffn_forward, moc_ffn_decode and moc_ffn_decode_static.  For moc_ffn_backward the flag is a PROMISE
+ * about the saved indices (they came from a forward call with the flag: at most 2 kept channels in every 4 consecutive
+ * ones); the library may then form grad_x on the 2:4-sparse tensor-core MMA, as the forward call does for the down
+ * projection (bf16, d_model >= 1024; for grad_x only with MOC_FFN_SPARSE_DX=1 in the environment: compressing the two
+ * operands costs what the shorter contraction saves).  A saved row that breaks the promise raises MOC_ERR_BAD_INDEX in
+ * the device status word and its surplus channels are left out of grad_x; without the flag the backward pass takes the
+ * indices as they are. */
 #define MOC_FLAG_SELECT_2_OF_8 2u
 /* bit 2: the Top-K operator placed AFTER the activation (Section 6.5, "Effect of top-K position": the ablation whose
  * other arm is the default): the K channels with the largest SiLU(g) are kept instead of those with the largest g.

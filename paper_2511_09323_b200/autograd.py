@@ -28,6 +28,7 @@ class _MoCFFNFunction(torch.autograd.Function):
             # recompute_up: the up values are dropped here and formed again in backward from x, w_up and the indices
             ctx.save_for_backward(x2, w_gate, w_up, w_down, idx, tg, *(() if recompute_up else (tu,)))
             ctx.d_ff = d_ff
+            ctx.grouped = bool(grouped)
             ctx.x_shape = shape
         return out.reshape(shape)
 
@@ -38,7 +39,8 @@ class _MoCFFNFunction(torch.autograd.Function):
         want = tuple(n for n, need in zip(names, ctx.needs_input_grad[:4]) if need)
         go = grad_out.reshape(-1, grad_out.shape[-1]).contiguous()
         tu = rest[0] if rest else B.moc_ffn_recompute_up(x2, w_up, idx, d_ff=ctx.d_ff)
-        res = B.moc_ffn_backward(x2, w_gate, w_up, w_down, idx, tg, tu, go, d_ff=ctx.d_ff, want=want)
+        res = B.moc_ffn_backward(x2, w_gate, w_up, w_down, idx, tg, tu, go, d_ff=ctx.d_ff, want=want,
+                                 grouped=ctx.grouped)
         gx = res["grad_x"]
         return (None if gx is None else gx.reshape(ctx.x_shape), res["grad_w_gate"], res["grad_w_up"],
                 res["grad_w_down"], None, None, None, None, None)

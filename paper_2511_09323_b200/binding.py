@@ -35,7 +35,8 @@ EXPORTED = (
     "moc_profile_enable", "moc_profile_collect", "moc_profile_kernel_count", "moc_profile_kernel_name",
     "moc_profile_read", "moc_ffn_decode_static", "moc_tc_gemm_bf16", "moc_ffn_recompute_up",
     "moc_ffn_backward_overlap", "moc_topk_select_tc", "moc_topk_select_tc_workspace_bytes", "moc_ffn_decode_probe",
-    "moc_ffn_decode_probe_workspace_bytes",
+    "moc_ffn_decode_probe_workspace_bytes", "moc_tc_gemm_sp_bf16", "moc_tc_gemm_sp_dense_bf16",
+    "moc_tc_gemm_sp_dense_workspace_bytes",
 )
 
 
@@ -97,6 +98,15 @@ def load() -> ctypes.CDLL:
         lib.moc_ffn_decode_probe_workspace_bytes.argtypes = [dp]
         lib.moc_ffn_decode_probe.restype = ctypes.c_int
         lib.moc_ffn_decode_probe.argtypes = [dp] + [vp] * 7 + [sz, vp]
+        lib.moc_tc_gemm_sp_bf16.restype = ctypes.c_int
+        lib.moc_tc_gemm_sp_bf16.argtypes = [ctypes.c_int64] * 3 + [vp, vp, vp, ctypes.c_int, ctypes.c_int64, vp,
+                                                                  ctypes.c_int64, vp]
+        lib.moc_tc_gemm_sp_dense_workspace_bytes.restype = sz
+        lib.moc_tc_gemm_sp_dense_workspace_bytes.argtypes = [ctypes.c_int64] * 2
+        lib.moc_tc_gemm_sp_dense_bf16.restype = ctypes.c_int
+        lib.moc_tc_gemm_sp_dense_bf16.argtypes = [ctypes.c_int64] * 3 + [vp, ctypes.c_int64, vp, ctypes.c_int64, vp,
+                                                                        ctypes.c_int64, ctypes.c_int,
+                                                                        ctypes.POINTER(ctypes.c_int64), vp, sz, vp]
         lib.moc_last_device_status.restype = ctypes.c_int
         lib.moc_test_bounded_wait.argtypes = [ctypes.c_int64, vp]
         lib.moc_test_bounded_wait.restype = ctypes.c_int
@@ -213,7 +223,7 @@ def moc_ffn_forward(x, w_gate, w_up, w_down, k, d_ff=None, save=True, out=None, 
 
 def moc_ffn_backward(x, w_gate, w_up, w_down, topk_idx, topk_gate, topk_up, grad_out, d_ff=None,
                      want=("x", "w_gate", "w_up", "w_down"), grads=None, accumulate=False, workspace=None,
-                     stream=None, wgrad_event=None):
+                     stream=None, wgrad_event=None, grouped=False):
     """Returns dict(grad_x, grad_w_gate, grad_w_up, grad_w_down) (None for entries not in `want`).
     `wgrad_event`: a torch.cuda.Event that the library records once the weight gradients are complete in stream
     order and before the grad_x kernel (moc_ffn_backward_overlap): a side stream that waits on it can all-reduce the
@@ -222,8 +232,10 @@ def moc_ffn_backward(x, w_gate, w_up, w_down, topk_idx, topk_gate, topk_up, grad
     T, d = x.shape
     F_ld = w_gate.shape[0]
     k = topk_idx.shape[1]
+    # grouped=True tells the library that the saved indices come from the 2-of-8 mask (slots 2q, 2q + 1 hold channels of
+    # group q): grad_x may then run on the 2:4-sparse tensor-core MMA
     desc = make_desc(T, d, F_ld if d_ff is None else d_ff, k, x.dtype, d_ff_ld=F_ld,
-                     flags=MOC_FLAG_ACCUMULATE_WGRAD if accumulate else 0)
+                     flags=(MOC_FLAG_ACCUMULATE_WGRAD if accumulate else 0) | (MOC_FLAG_SELECT_2_OF_8 if grouped else 0))
     grads = dict(grads or {})
     res = {}
     for name, like in (("x", x), ("w_gate", w_gate), ("w_up", w_up), ("w_down", w_down)):
@@ -392,6 +404,42 @@ def moc_ffn_decode_probe(x, w_gate, w_up, w_down, k, d_ff=None, stream=None, gro
     if rc != MOC_OK:
         raise MocError(rc, "moc_ffn_decode_probe")
     return out, kept
+
+
+def moc_tc_gemm_sp_bf16(a_compressed: torch.Tensor, metadata: torch.Tensor, b: torch.Tensor, k: int,
+                        b_mn_major: bool = False, stream=None) -> torch.Tensor:
+    """The one-CTA sparse GEMM on caller-built operands: a_compressed [m, k/2] bf16, metadata int32 words in the
+    tensor-memory arrangement (include/moc_ffn.h), b [n, k] (or [k, n] when b_mn_major) -> C [m, n] fp32."""
+    _check_dev(a_compressed, metadata, b)
+    m = a_compressed.shape[0]
+    n = b.shape[1] if b_mn_major else b.shape[0]
+    c = torch.empty((m, n), dtype=torch.float32, device=b.device)
+    rc = load().moc_tc_gemm_sp_bf16(m, n, k, _ptr(a_compressed), _ptr(metadata), _ptr(b), int(b_mn_major), b.stride(0),
+                                    _ptr(c), n, _stream_ptr(stream))
+    if rc != MOC_OK:
+        raise MocError(rc, "moc_tc_gemm_sp_bf16")
+    return c
+
+
+def moc_tc_gemm_sp_dense_bf16(a: torch.Tensor, b: torch.Tensor, out=None, accumulate: bool = False, stream=None):
+    """a [m, k] bf16 with at most 2 non-zero values per 4 consecutive elements, b [k, n] bf16 -> (C [m, n] bf16, number
+    of values that did not fit the 2:4 pattern and were left out)."""
+    _check_dev(a, b, out)
+    m, k = a.shape
+    n = b.shape[1]
+    lib = load()
+    need = lib.moc_tc_gemm_sp_dense_workspace_bytes(m, k)
+    if need == 0:
+        raise MocError(MOC_ERR_INVALID_ARG, "moc_tc_gemm_sp_dense_bf16")
+    ws = torch.empty(need, dtype=torch.uint8, device=a.device)
+    if out is None:
+        out = torch.empty((m, n), dtype=torch.bfloat16, device=a.device)
+    left_out = ctypes.c_int64(-1)
+    rc = lib.moc_tc_gemm_sp_dense_bf16(m, n, k, _ptr(a), a.stride(0), _ptr(b), b.stride(0), _ptr(out), out.stride(0),
+                                       int(accumulate), ctypes.byref(left_out), _ptr(ws), need, _stream_ptr(stream))
+    if rc != MOC_OK:
+        raise MocError(rc, "moc_tc_gemm_sp_dense_bf16")
+    return out, int(left_out.value)
 
 
 def moc_last_device_status(stream=None) -> int:

@@ -486,12 +486,12 @@ bool sparse_mma_enabled() {
 // dense [rows, ld] (at most 2 non-zero values per group of 4) -> compressed rows + metadata
 int sparse_compress(const __nv_bfloat16 *dense, int64_t rows, int K, int ld, const SparseOperandLayout &L,
                     __nv_bfloat16 *comp, uint32_t *meta, tcsp::Overflow *overflow, int overflow_cap,
-                    unsigned int *overflow_n, cudaStream_t st) {
+                    unsigned int *overflow_n, cudaStream_t st, int *bad_status = nullptr) {
     const int64_t jobs = ((rows + 127) / 128) * L.k_stages;
     const unsigned grid = (unsigned)std::min<int64_t>(jobs, (int64_t)tc::sm_count() * 8);
     MOC_LAUNCH(KID_TC_COMPRESS, st,
                (tcsp::compress_2of4_kernel<<<grid, 512, 0, st>>>(dense, rows, K, ld, comp, L.kc_ld, meta, L.k_stages,
-                                                                  overflow, overflow_cap, overflow_n)));
+                                                                  overflow, overflow_cap, overflow_n, bad_status)));
     return launch_ok();
 }
 
@@ -702,6 +702,9 @@ int backward_tc(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat
     int *status = device_status_ptr();
     if (!status) return MOC_ERR_CUDA;
     int rc;
+    // MoC 2:8: dG' and dU' are 2:4-sparse rows; grad_x can contract them on the sparse MMA (the element-wise kernel then
+    // also writes them in compressed form).  With few output columns the shorter GEMM does not pay for that.
+    const bool sparse_dx = gx && L.sp_bytes != 0 && sparse_mma_enabled() && dm >= 1024;
 
     // dZ = dD Wd^T (dense, bf16), then the element-wise step at the saved indices -> masked Z', dU', dG'
     {
@@ -778,7 +781,20 @@ int backward_tc(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat
     // the weight gradients are complete in stream order here; the grad_x kernel that follows does not touch them
     if (wgrad_done && cudaEventRecord(wgrad_done, st) != cudaSuccess) return MOC_ERR_CUDA;
     // dX = dG' Wg + dU' Wu   (Eq. (bp-5)): one accumulator, two contraction segments
-    if (gx && L.small_bytes) {
+    if (sparse_dx) {
+        // dG' and dU' rows are 2:4-sparse (the caller's promise): compress both, then one sparse GEMM over two segments.
+        // Values a row holds beyond two per group of 4 are counted and reported as a broken promise.
+        const SparseOperandLayout SL = sparse_operand_layout(T, F);
+        __nv_bfloat16 *gc = reinterpret_cast<__nv_bfloat16 *>(ws + L.off_gc), *uc = reinterpret_cast<__nv_bfloat16 *>(ws + L.off_uc);
+        uint32_t *gmeta = reinterpret_cast<uint32_t *>(ws + L.off_gmeta), *umeta = reinterpret_cast<uint32_t *>(ws + L.off_umeta);
+        if ((rc = sparse_compress(dGp, T, F, L.ldf, SL, gc, gmeta, nullptr, 0, nullptr, st, status)) != MOC_OK) return rc;
+        if ((rc = sparse_compress(dUp, T, F, L.ldf, SL, uc, umeta, nullptr, 0, nullptr, st, status)) != MOC_OK) return rc;
+        const __nv_bfloat16 *comps[2] = {gc, uc};
+        const uint32_t *metas[2] = {gmeta, umeta};
+        const __nv_bfloat16 *bs[2] = {wg, wu};
+        if ((rc = sparse_gemm_pair(T, dm, F, 2, comps, metas, SL, bs, dm, gx, dm, false, KID_TC_SP_DX_GEMM, status, st)) != MOC_OK)
+            return rc;
+    } else if (gx && L.small_bytes) {
         // a small batch: the weight-streaming kernel of the small-batch plan (a 256-row tile of tokens would leave
         // most SMs without work: d_model / 256 tiles in all)
         if ((rc = small_batch_dx(d, dGp, dUp, L.ldf, wg, wu, gx, ws + L.off_small, st)) != MOC_OK) return rc;

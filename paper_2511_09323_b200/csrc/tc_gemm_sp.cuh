@@ -526,7 +526,8 @@ __global__ void __launch_bounds__(512) compress_2of4_kernel(const __nv_bfloat16 
                                                             int ld, __nv_bfloat16 *__restrict__ comp, int kc_ld,
                                                             uint32_t *__restrict__ meta, int k_stages,
                                                             Overflow *__restrict__ overflow, int overflow_cap,
-                                                            unsigned int *__restrict__ overflow_n) {
+                                                            unsigned int *__restrict__ overflow_n,
+                                                            int *__restrict__ bad_status) {
     __shared__ uint32_t s_half[128][4][2];  // [row][atom][k half]: the row's 16 metadata bits for 16 logical elements
     const int r = threadIdx.x & 127, atom = threadIdx.x >> 7;
     const int64_t blocks = (rows + 127) / 128;
@@ -558,7 +559,9 @@ __global__ void __launch_bounds__(512) compress_2of4_kernel(const __nv_bfloat16 
                     if (nz) {
                         if (p0 < 0) p0 = j;
                         else if (p1 < 0) p1 = j;
-                        else if (overflow) {
+                        else if (bad_status) {
+                            raise_status(bad_status, MOC_ERR_BAD_INDEX);  // the caller promised 2:4 rows
+                        } else if (overflow) {
                             const unsigned int at = atomicAdd(overflow_n, 1u);
                             if (at < (unsigned int)overflow_cap) {
                                 const uint32_t fb = (uint32_t)e[j] << 16;

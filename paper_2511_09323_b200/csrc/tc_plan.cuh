@@ -958,9 +958,23 @@ struct TcBackwardLayout {
     int ldf;
     size_t off_z, off_du, off_dg, total;  // three dense bf16 [T, ldf] arrays
     size_t off_small, small_bytes;        // batches of up to 256 tokens: fp32 accumulator [T, d] + counters of the dX kernel
+    // MoC 2:8 with grad_x on the sparse MMA: dG' and dU' in compressed form [T, F / 2] with their metadata (sp_bytes == 0:
+    // not used)
+    size_t off_gc, off_uc, off_gmeta, off_umeta, sp_bytes;
 };
 
 inline int round_up8(int v) { return (v + 7) & ~7; }
+
+// grad_x of the MoC 2:8 variant on the sparse MMA is built and checked but off by default: compressing dG' and dU' costs
+// what the shorter GEMM saves (LLaMA-1B shape, 65536 tokens: grad_x 2.14 -> 1.38 ms, two compression passes 0.8 ms).
+// MOC_FFN_SPARSE_DX=1 in the environment turns it on.
+inline bool sparse_dx_requested() {
+    static const bool on = [] {
+        const char *e = getenv("MOC_FFN_SPARSE_DX");
+        return e && strcmp(e, "1") == 0;
+    }();
+    return on;
+}
 
 inline TcForwardLayout tc_forward_layout(const moc_ffn_desc &d) {
     TcForwardLayout L{};
@@ -1010,6 +1024,18 @@ inline TcBackwardLayout tc_backward_layout(const moc_ffn_desc &d) {
     L.off_small = off;
     L.small_bytes = d.tokens <= 256 ? align_up((size_t)d.tokens * d.d_model * sizeof(float) + 1024, 256) : 0;
     off += L.small_bytes;
+    L.sp_bytes = 0;
+    if ((d.flags & MOC_FLAG_SELECT_2_OF_8) && sparse_dx_requested() && !L.small_bytes) {
+        const size_t rows = (size_t)((d.tokens + 127) / 128) * 128;
+        const size_t k_stages = (size_t)(d.d_ff + 127) / 128;
+        const size_t comp = align_up(rows * k_stages * 64 * 2, 256), meta = align_up(rows / 128 * k_stages * 2048, 256);
+        L.off_gc = off;
+        L.off_uc = off + comp;
+        L.off_gmeta = off + 2 * comp;
+        L.off_umeta = off + 2 * comp + meta;
+        L.sp_bytes = 2 * comp + 2 * meta;
+        off += L.sp_bytes;
+    }
     L.total = off;
     return L;
 }

@@ -22,12 +22,12 @@ def _lib():
     assert B.moc_last_device_status() == B.MOC_OK
 
 
-def _forward_backward(w: syn.Workload):
+def _forward_backward(w: syn.Workload, grouped_backward: bool = True):
     wg, wu, wd = syn.make_weights(w)
     x, dD = syn.make_x(w), syn.make_grad_out(w)
     xd, wgd, wud, wdd, dDd = (t.cuda() for t in (x, wg, wu, wd, dD))
     out, idx, tg, tu = B.moc_ffn_forward(xd, wgd, wud, wdd, None, grouped=True)
-    grads = B.moc_ffn_backward(xd, wgd, wud, wdd, idx, tg, tu, dDd)
+    grads = B.moc_ffn_backward(xd, wgd, wud, wdd, idx, tg, tu, dDd, grouped=grouped_backward)
     torch.cuda.synchronize()
     assert B.moc_last_device_status() == B.MOC_OK
     x64, wg64, wu64, wd64, dD64 = map(syn.to_f64, (x, wg, wu, wd, dD))
@@ -51,6 +51,85 @@ def _forward_backward(w: syn.Workload):
 ])
 def test_grouped_forward_backward(dtype, T, d, F):
     _forward_backward(syn.Workload(f"g28-{dtype}-{T}", dtype, T, d, F, F, F // 4, seed=2800 + T))
+
+
+@pytest.mark.parametrize("T,d,F,grouped_backward", [
+    (300, 1024, 1024, True),     # d_model >= 1024: down projection and grad_x on the 2:4-sparse MMA; one ragged tile pair
+    (300, 1024, 1024, False),    # the same saved tensors through the dense grad_x (no promise about the indices)
+    (700, 1288, 1280, True),     # ragged in every direction: 700 tokens, 1288 columns (5 tiles + 8), 10 blocks of 128 channels
+    (520, 1024, 1000, True),     # d_ff not a multiple of 128: compressed forward, dense grad_x
+])
+def test_grouped_forward_backward_on_the_sparse_mma(T, d, F, grouped_backward):
+    _forward_backward(syn.Workload(f"g28sp-{T}-{d}-{F}", "bf16", T, d, F, F, F // 4, seed=2900 + T), grouped_backward)
+
+
+def _run_isolated(code, env_extra):
+    """Runs `code` in a fresh interpreter (the library reads its environment switches once per process); the code saves a
+    dictionary of tensors to the path it gets as its argument."""
+    import os
+    import subprocess
+    import sys
+    import tempfile
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    with tempfile.NamedTemporaryFile(suffix=".pt") as fh:
+        subprocess.run([sys.executable, "-c", code, fh.name], check=True, cwd=root, env=dict(os.environ, **env_extra),
+                       timeout=600)
+        return torch.load(fh.name)
+
+
+_SPARSE_CASE = (
+    "import torch, sys; sys.path.insert(0, '.');"
+    "from paper_2511_09323_b200 import binding as B, synthetic as syn;"
+    "w = syn.Workload('g28cmp', 'bf16', 600, 1024, 2048, 2048, 512, seed=77);"
+    "wg, wu, wd = (t.cuda() for t in syn.make_weights(w)); x = syn.make_x(w).cuda(); dD = syn.make_grad_out(w).cuda();"
+    "out, idx, tg, tu = B.moc_ffn_forward(x, wg, wu, wd, None, grouped=True);"
+    "g = B.moc_ffn_backward(x, wg, wu, wd, idx, tg, tu, dD, grouped=True); torch.cuda.synchronize();"
+    "st = B.moc_last_device_status();"
+    "torch.save({'out': out.cpu(), 'idx': idx.cpu(), 'gx': g['grad_x'].cpu(), 'status': st}, sys.argv[1])")
+
+
+def test_grouped_sparse_paths_agree_with_the_dense_ones():
+    """The same layer with the sparse MMA switched off is a different set of kernels for the same arithmetic: down
+    projection and grad_x (the latter on the sparse MMA only when asked for) must agree within the bf16 tolerance, and the
+    sparse grad_x must match the oracle."""
+    sparse = _run_isolated(_SPARSE_CASE, {"MOC_FFN_SPARSE": "1", "MOC_FFN_SPARSE_DX": "1"})
+    dense = _run_isolated(_SPARSE_CASE, {"MOC_FFN_SPARSE": "0"})
+    assert sparse["status"] == B.MOC_OK and dense["status"] == B.MOC_OK
+    assert torch.equal(sparse["idx"], dense["idx"])
+    for key in ("out", "gx"):
+        a, b = sparse[key].double(), dense[key].double()
+        assert (a - b).abs().max().item() <= 1e-2 * b.abs().max().item(), key
+    w = syn.Workload("g28cmp", "bf16", 600, 1024, 2048, 2048, 512, seed=77)
+    wg, wu, wd = syn.make_weights(w)
+    x, dD = syn.make_x(w), syn.make_grad_out(w)
+    toks = np.arange(0, 600, 7)
+    x64, dD64 = syn.to_f64(x[toks]), syn.to_f64(dD[toks])
+    wg64, wu64, wd64 = map(syn.to_f64, (wg, wu, wd))
+    idx_np = sparse["idx"].numpy()[toks].astype(np.int32)
+    ref = orc.forward_given_idx(x64, wg64, wu64, wd64, idx_np)
+    parity.assert_close(syn.to_f64(sparse["out"][toks]), ref["out"], "bf16", "out (sparse down projection)")
+    rb = orc.backward(x64, wg64, wu64, wd64, idx_np, syn.round_to(ref["gval"], "bf16"), syn.round_to(ref["uval"], "bf16"),
+                      dD64, F=w.d_ff, want=("x",))
+    parity.assert_close(syn.to_f64(sparse["gx"][toks]), rb["grad_x"], "bf16", "grad_x (sparse MMA)")
+
+
+def test_backward_flag_on_rows_that_are_not_2_of_8_is_reported():
+    """Saved indices from the row Top-K (several kept channels in one group of 4) with the 2-of-8 promise set and grad_x
+    on the sparse MMA: the surplus channels are left out and the status word says so; nothing faults."""
+    code = (
+        "import torch, sys; sys.path.insert(0, '.');"
+        "from paper_2511_09323_b200 import binding as B, synthetic as syn;"
+        "w = syn.Workload('g28-bad', 'bf16', 300, 1024, 1024, 1024, 256, seed=41);"
+        "wg, wu, wd = (t.cuda() for t in syn.make_weights(w)); x = syn.make_x(w).cuda(); dD = syn.make_grad_out(w).cuda();"
+        "out, idx, tg, tu = B.moc_ffn_forward(x, wg, wu, wd, w.k);"
+        "B.moc_ffn_backward(x, wg, wu, wd, idx, tg, tu, dD, grouped=True);"
+        "st1 = B.moc_last_device_status(); st2 = B.moc_last_device_status();"
+        "ok = B.moc_ffn_backward(x, wg, wu, wd, idx, tg, tu, dD); torch.cuda.synchronize();"
+        "torch.save({'st1': st1, 'st2': st2, 'st3': B.moc_last_device_status(),"
+        " 'finite': bool(torch.isfinite(ok['grad_x'].float()).all())}, sys.argv[1])")
+    res = _run_isolated(code, {"MOC_FFN_SPARSE_DX": "1"})
+    assert res["st1"] == B.MOC_ERR_BAD_INDEX and res["st2"] == B.MOC_OK
+    assert res["st3"] == B.MOC_OK and res["finite"]
 
 
 def test_grouped_ties_keep_the_lower_channels_exactly():
