@@ -721,7 +721,7 @@ def grouped_report(torch, B, x, dD, wg, wu, wd, flush, steps):
     T, F = x.shape[0], wg.shape[0]
     for _ in range(3):
         out, idx, tg, tu = B.moc_ffn_forward(x, wg, wu, wd, None, grouped=True)
-        B.moc_ffn_backward(x, wg, wu, wd, idx, tg, tu, dD)
+        B.moc_ffn_backward(x, wg, wu, wd, idx, tg, tu, dD, grouped=True)
     torch.cuda.synchronize()
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
     grads = None
@@ -729,11 +729,17 @@ def grouped_report(torch, B, x, dD, wg, wu, wd, flush, steps):
         flush.zero_()
         s.record()
         out, idx, tg, tu = B.moc_ffn_forward(x, wg, wu, wd, None, grouped=True)
-        grads = B.moc_ffn_backward(x, wg, wu, wd, idx, tg, tu, dD, grads=grads)
+        grads = B.moc_ffn_backward(x, wg, wu, wd, idx, tg, tu, dD, grads=grads, grouped=True)
         t.record()
     torch.cuda.synchronize()
     ms = sum(s.elapsed_time(t) for s, t in ev) / steps
-    return {"k": F // 4, "ms_per_step": ms, "tokens_per_s": T / (ms / 1e3), "launch": "direct calls"}
+    names = set()
+    B.moc_profile_enable(True)
+    B.moc_ffn_forward(x, wg, wu, wd, None, grouped=True)
+    names = [k for k, (n, _) in B.moc_profile_collect().items() if n]
+    B.moc_profile_enable(False)
+    return {"k": F // 4, "ms_per_step": ms, "tokens_per_s": T / (ms / 1e3), "launch": "direct calls",
+            "down_projection": "2:4-sparse MMA (tcgen05.mma.sp)" if "tc_sp_down_gemm" in names else "dense MMA"}
 
 
 def decode_report(torch, B, syn, dev, peaks, calls=32, sets=4, replays=5):

@@ -774,6 +774,11 @@ int backward_tc(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat
         p.accumulate = (d.flags & MOC_FLAG_ACCUMULATE_WGRAD) ? 1 : 0;
         // long contraction, few tiles: the finer tile granularity of single CTAs fills the last wave better
         p.single_cta = 1;
+        static const bool problem_major = [] {
+            const char *e = getenv("MOC_FFN_WGRAD_ORDER");  // "m": the m-block-major order (comparisons)
+            return !(e && strcmp(e, "m") == 0);
+        }();
+        p.problem_major = problem_major ? 1 : 0;
         p.status = status;
         MOC_LAUNCH(KID_TC_WGRAD_GEMM, st, (rc = launch_gemm<true, true, EPI_BF16>(p, st)));
         if (rc != MOC_OK) return rc;

@@ -71,6 +71,10 @@ struct Params {
     CUtensorMap c_map[3];  // per problem: [M, N] with 32-row boxes of 128 bytes (32 fp32 or 64 bf16 columns)
     int direct_store;      // 1: the output cannot be described by a tensor map; threads store their rows
     int single_cta;        // 1: one CTA per tile even where CTA pairs are available (set by the caller)
+    // Tile order.  0: (m block, problem, n block) -- tiles of one m block are adjacent, right when the problems share A
+    // (gate | up).  1: (problem, m block, n block) -- a wave of CTAs works on ONE problem, right when the problems have
+    // different operands on both sides (the three weight gradients: a wave then streams one B matrix instead of two).
+    int problem_major;
     // EPI_GATE_UP_2OF8: compact saved activations [M, N / 4] (all three or none)
     int16_t *sv_idx;
     __nv_bfloat16 *sv_g, *sv_u;
@@ -639,6 +643,13 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_kernel(const __grid_constant_
     // tile id -> (m block, problem, n block): all tiles of one m block are adjacent, so CTAs running at
     // the same time share A rows and the (small) B operands stay in L2
     auto decode_tile = [&](int tile, int &m_blk, int &prob, int &n_blk) {
+        if (p.problem_major) {
+            prob = tile / tiles_per_problem;
+            const int r = tile - prob * tiles_per_problem;
+            m_blk = r / p.n_tiles;
+            n_blk = r - m_blk * p.n_tiles;
+            return;
+        }
         const int per_m = p.num_problems * p.n_tiles;
         m_blk = tile / per_m;
         const int r = tile - m_blk * per_m;
