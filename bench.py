@@ -40,9 +40,10 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # thousand tokens on the device (the full batch is too large to capture); two token counts give the two coefficients,
 # and `roofline.traffic` is their value at the benchmarked token count.
 NCU_DRAM_BYTES = {
-    # weight-gradient GEMM on the LLaMA-1B shape: 795.5 MB at 8192 tokens, 1555.5 MB at 16384 (read + write)
-    ("C5", "tc_wgrad_gemm"): (35.4e6, 92780.0),
-    ("C3", "tc_wgrad_gemm"): (35.4e6, 92780.0),
+    # weight-gradient GEMM on the LLaMA-1B shape: 524.4 MB at 8192 tokens, 1144.8 MB at 16384 (read + write); the L2
+    # holds a larger share of the operands at the smaller size, hence the negative constant
+    ("C5", "tc_wgrad_gemm"): (-96.1e6, 75735.0),
+    ("C3", "tc_wgrad_gemm"): (-96.1e6, 75735.0),
 }
 # the same for the LLaMA-130M workload, measured at its full size (one launch of each kernel per step)
 NCU_DRAM_BYTES_C2 = {
