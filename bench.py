@@ -755,7 +755,9 @@ def decode_report(torch, B, syn, dev, peaks, calls=32, sets=4, replays=5):
     weights = [tuple(t.to(dev) for t in syn.make_weights(w, seed_offset=s)) for s in range(sets)]
     note = {"weight_sets": sets, "calls_per_graph": calls, "replays": replays,
             "timing": "CUDA graph replay, 10 untimed replays first",
-            "roofline": "algorithmic bytes / measured HBM copy bandwidth"}
+            "roofline": "algorithmic bytes / measured HBM copy bandwidth",
+            "floor": "floor_us = a bare streaming read (bulk copies into shared memory, nothing computed) of the same bytes, "
+                     "timed with the same graph of rotating weight sets"}
     main, more = dict(note), {}
     e = 2
     stream = torch.cuda.Stream(device=dev)
@@ -818,6 +820,13 @@ def decode_report(torch, B, syn, dev, peaks, calls=32, sets=4, replays=5):
             entry.update(plan=("one cooperative kernel" if launches == 1 else f"{launches} kernels") +
                          ": gate matrix + gathered rows")
         if T in syn.C4_BATCHES:
+            # the floor: a bare streaming read of the same number of bytes (all of W_gate, as many bytes of W_up and W_down
+            # as the union of kept rows holds), same graph of rotating weight sets, nothing computed
+            rows_bytes = union * w.d_model * e
+            us_floor, _ = timed(lambda i, st: B.moc_profile_stream_read(
+                [(weights[i % sets][0], w.d_ff * w.d_model * e), (weights[i % sets][1], rows_bytes),
+                 (weights[i % sets][2], rows_bytes)], stream=st))
+            entry.update(floor_us=round(us_floor, 3), frac_of_floor=round(us_floor / us, 4))
             main[f"T{T}"] = entry
             # the FFN half of a pre-norm layer, out = h + FFN(RMSNorm(h)): one library call against the same steps as
             # separate launches (torch's RMSNorm and addition around moc_ffn_decode)

@@ -360,6 +360,13 @@ MOC_API size_t moc_ffn_saved_bytes_per_token(const moc_ffn_desc *desc);
  *   moc_profile_kernel_count / _name / _read   enumerate kernels and read launches + total ms.
  */
 MOC_API int64_t moc_launch_count(void);
+/*   moc_profile_stream_read   a bare streaming read of up to three device byte ranges (sizes multiples of 16, 0 = unused):
+ *                             every byte is brought into shared memory once by bulk copies, nothing is computed.  The time
+ *                             of this kernel for the bytes a decode call has to read (Section 5: the gate matrix and the
+ *                             selected rows of the other two) is the floor under any schedule for that call; a benchmark
+ *                             times it with the call's own protocol and reports the call against it. */
+MOC_API int moc_profile_stream_read(const void *a, size_t a_bytes, const void *b, size_t b_bytes, const void *c,
+                                    size_t c_bytes, void *cuda_stream);
 MOC_API int moc_profile_enable(int on);
 MOC_API int moc_profile_collect(void *cuda_stream);
 MOC_API int moc_profile_kernel_count(void);

@@ -36,7 +36,7 @@ EXPORTED = (
     "moc_profile_read", "moc_ffn_decode_static", "moc_tc_gemm_bf16", "moc_ffn_recompute_up",
     "moc_ffn_backward_overlap", "moc_topk_select_tc", "moc_topk_select_tc_workspace_bytes", "moc_ffn_decode_probe",
     "moc_ffn_decode_probe_workspace_bytes", "moc_tc_gemm_sp_bf16", "moc_tc_gemm_sp_dense_bf16",
-    "moc_tc_gemm_sp_dense_workspace_bytes",
+    "moc_tc_gemm_sp_dense_workspace_bytes", "moc_profile_stream_read",
 )
 
 
@@ -107,6 +107,8 @@ def load() -> ctypes.CDLL:
         lib.moc_tc_gemm_sp_dense_bf16.argtypes = [ctypes.c_int64] * 3 + [vp, ctypes.c_int64, vp, ctypes.c_int64, vp,
                                                                         ctypes.c_int64, ctypes.c_int,
                                                                         ctypes.POINTER(ctypes.c_int64), vp, sz, vp]
+        lib.moc_profile_stream_read.restype = ctypes.c_int
+        lib.moc_profile_stream_read.argtypes = [vp, sz, vp, sz, vp, sz, vp]
         lib.moc_last_device_status.restype = ctypes.c_int
         lib.moc_test_bounded_wait.argtypes = [ctypes.c_int64, vp]
         lib.moc_test_bounded_wait.restype = ctypes.c_int
@@ -462,6 +464,16 @@ def moc_profile_enable(on: bool) -> None:
     rc = load().moc_profile_enable(1 if on else 0)
     if rc != MOC_OK:
         raise MocError(rc, "moc_profile_enable")
+
+
+def moc_profile_stream_read(ranges, stream=None) -> None:
+    """A bare streaming read of up to three (tensor, bytes) ranges: the floor under any kernel that has to read them."""
+    flat = []
+    for t, n in list(ranges) + [(None, 0)] * (3 - len(ranges)):
+        flat += [_ptr(t) if t is not None else None, int(n) // 16 * 16]
+    rc = load().moc_profile_stream_read(*flat, _stream_ptr(stream))
+    if rc != MOC_OK:
+        raise MocError(rc, "moc_profile_stream_read")
 
 
 def moc_profile_collect(stream=None) -> dict:

@@ -80,6 +80,7 @@ enum KernelId {
     KID_TC_COMPRESS,
     KID_TC_SP_DOWN_GEMM,
     KID_TC_SP_DX_GEMM,
+    KID_STREAM_PROBE,
     KID_COUNT
 };
 static const char *const kKernelNames[KID_COUNT] = {
@@ -89,7 +90,7 @@ static const char *const kKernelNames[KID_COUNT] = {
     "tc_wgrad_gemm",   "tc_dx_gemm",      "tc_test_gemm",  "tc_select_hint", "dec_gate_gemv",
     "dec_select",      "dec_up",          "dec_down",      "sb_gate_up",     "sb_select",
     "sb_down",         "recompute_up",    "dec_coop",      "dec_rmsnorm",    "tc_compress_2of4",
-    "tc_sp_down_gemm", "tc_sp_dx_gemm",
+    "tc_sp_down_gemm", "tc_sp_dx_gemm", "stream_probe",
 };
 
 struct Profiler {
@@ -1917,6 +1918,27 @@ extern "C" __attribute__((visibility("default"))) int moc_debug_timeline(unsigne
                ? MOC_OK : MOC_ERR_CUDA;
 }
 #endif
+
+int moc_profile_stream_read(const void *a, size_t a_bytes, const void *b, size_t b_bytes, const void *c, size_t c_bytes,
+                            void *cuda_stream) {
+    const void *ptr[3] = {a, b, c};
+    const size_t n[3] = {a_bytes, b_bytes, c_bytes};
+    dec::ProbeRanges r{};
+    for (int i = 0; i < 3; ++i) {
+        if (n[i] && (!good_ptr(ptr[i]) || n[i] % 16 != 0)) return MOC_ERR_INVALID_ARG;
+        r.base[i] = static_cast<const uint8_t *>(ptr[i]);
+        r.bytes[i] = n[i];
+    }
+    int *status = device_status_ptr();
+    if (!status) return MOC_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const size_t smem = (size_t)dec::kProbeStages * dec::kProbeChunk;
+    int rc = set_smem(dec::stream_probe_kernel, smem, 1024);
+    if (rc != MOC_OK) return rc;
+    MOC_LAUNCH(KID_STREAM_PROBE, st,
+               launch_pdl(dec::stream_probe_kernel, dim3(2 * tc::sm_count()), dec::kProbeThreads, smem, st, r, status));
+    return launch_ok();
+}
 
 int64_t moc_launch_count(void) { return g_prof.launches.load(std::memory_order_relaxed); }
 

@@ -879,5 +879,69 @@ __global__ void __launch_bounds__(256) rmsnorm_rows_kernel(const __nv_bfloat16 *
     }
 }
 
+
+// ---------------------------------------------------------------------------------------------- stream probe
+// A bare streaming read (diagnostics): up to three byte ranges are read once, in 8 KiB bulk copies through a ring of
+// kProbeStages stages per CTA, two CTAs per SM, nothing computed: the time below which no schedule that has to read those
+// bytes from HBM can finish.  The ranges are split evenly over the CTAs.
+constexpr int kProbeStages = 11, kProbeChunk = 8192, kProbeThreads = 64;
+struct ProbeRanges {
+    const uint8_t *base[3];
+    unsigned long long bytes[3];  // multiples of 16
+};
+__global__ void __launch_bounds__(kProbeThreads, 2) stream_probe_kernel(const ProbeRanges r, int *__restrict__ status) {
+    extern __shared__ __align__(128) uint8_t dsm[];
+    __shared__ uint64_t bars[2 * kProbeStages];
+    __shared__ int s_abort;
+    const int tid = threadIdx.x;
+    auto full_bar = [&](int s) { return tc::smem_u32(&bars[s]); };
+    auto empty_bar = [&](int s) { return tc::smem_u32(&bars[kProbeStages + s]); };
+    if (tid == 0) {
+        for (int s = 0; s < kProbeStages; ++s) {
+            tc::mbar_init(full_bar(s), 1);
+            tc::mbar_init(empty_bar(s), 1);
+        }
+        s_abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    tc::pdl_launch_dependents();
+    // this CTA's share of every range, in chunks
+    if (tid == 0) {  // producer
+        int stage = 0;
+        uint32_t phase = 0;
+        for (int i = 0; i < 3; ++i) {
+            const unsigned long long chunks = (r.bytes[i] + kProbeChunk - 1) / kProbeChunk;
+            const unsigned long long c0 = chunks * blockIdx.x / gridDim.x, c1 = chunks * (blockIdx.x + 1) / gridDim.x;
+            for (unsigned long long c = c0; c < c1; ++c) {
+                if (!tc::mbar_wait(empty_bar(stage), phase ^ 1u, &s_abort, status)) return;
+                const unsigned long long off = c * kProbeChunk;
+                const uint32_t n = (uint32_t)min((unsigned long long)kProbeChunk, r.bytes[i] - off);
+                tc::mbar_expect_tx(full_bar(stage), n);
+                bulk_copy_g2s(tc::smem_u32(dsm + stage * kProbeChunk), r.base[i] + off, n, full_bar(stage));
+                if (++stage == kProbeStages) {
+                    stage = 0;
+                    phase ^= 1u;
+                }
+            }
+        }
+    } else if (tid == 32) {  // consumer: hands every stage straight back
+        int stage = 0;
+        uint32_t phase = 0;
+        for (int i = 0; i < 3; ++i) {
+            const unsigned long long chunks = (r.bytes[i] + kProbeChunk - 1) / kProbeChunk;
+            const unsigned long long c0 = chunks * blockIdx.x / gridDim.x, c1 = chunks * (blockIdx.x + 1) / gridDim.x;
+            for (unsigned long long c = c0; c < c1; ++c) {
+                if (!tc::mbar_wait(full_bar(stage), phase, &s_abort, status)) return;
+                tc::mbar_arrive(empty_bar(stage));
+                if (++stage == kProbeStages) {
+                    stage = 0;
+                    phase ^= 1u;
+                }
+            }
+        }
+    }
+}
+
 }  // namespace dec
 }  // namespace moc
