@@ -17,6 +17,7 @@
 #include "grouped_select.cuh"
 #include "moc_common.cuh"
 #include "small_batch.cuh"
+#include "small_batch_fused.cuh"
 #include "tc_gemm.cuh"
 #include "tc_gemm_sp.cuh"
 #include "tc_plan.cuh"
@@ -81,6 +82,7 @@ enum KernelId {
     KID_TC_SP_DOWN_GEMM,
     KID_TC_SP_DX_GEMM,
     KID_STREAM_PROBE,
+    KID_SB_FUSED,
     KID_COUNT
 };
 static const char *const kKernelNames[KID_COUNT] = {
@@ -90,7 +92,7 @@ static const char *const kKernelNames[KID_COUNT] = {
     "tc_wgrad_gemm",   "tc_dx_gemm",      "tc_test_gemm",  "tc_select_hint", "dec_gate_gemv",
     "dec_select",      "dec_up",          "dec_down",      "sb_gate_up",     "sb_select",
     "sb_down",         "recompute_up",    "dec_coop",      "dec_rmsnorm",    "tc_compress_2of4",
-    "tc_sp_down_gemm", "tc_sp_dx_gemm", "stream_probe",
+    "tc_sp_down_gemm", "tc_sp_dx_gemm", "stream_probe",    "sb_fused",
 };
 
 struct Profiler {
@@ -1047,8 +1049,8 @@ struct SmallBatchLayout {
 
 // Grid of sb_down_kernel for `d_model` output columns and `k_blocks` channel blocks in all: about one CTA per SM,
 // every CTA at least one channel block; 256-column blocks (accs = 2) when they still fill the GPU, else 128.
-void down_geometry(int d_model, int k_blocks, int &accs, int &m_tiles, int &splits) {
-    const int sms = tc::sm_count();
+void down_geometry(int d_model, int k_blocks, int &accs, int &m_tiles, int &splits, int sms = 0) {
+    if (sms <= 0) sms = tc::sm_count();
     auto ctas = [&](int a, int &mt, int &sp) {
         mt = (d_model + sb::kTile * a - 1) / (sb::kTile * a);
         sp = std::max(1, std::min(sms / mt, k_blocks));
@@ -1079,7 +1081,8 @@ SmallBatchLayout small_batch_layout(const moc_ffn_desc &d) {
     L.off_u = c.take((size_t)d.tokens * L.ldf * sizeof(float));
     L.off_z = c.take((size_t)d.tokens * L.ldz * sizeof(__nv_bfloat16));
     L.off_acc = c.take((size_t)d.tokens * d.d_model * sizeof(float));
-    L.off_cnt = c.take((size_t)L.m_tiles * sizeof(int));
+    // the column blocks' counters; the one-kernel form's geometry may have twice as many blocks and keeps its flags behind them
+    L.off_cnt = c.take(((size_t)2 * L.m_tiles + 8) * sizeof(int));
     L.total = c.off;
     return L;
 }
@@ -1204,6 +1207,134 @@ int forward_small_batch_overlapped(const moc_ffn_desc &d, const SmallBatchLayout
     return small_batch_down(d, L, ds, wd, Z, acc, counters, out, resid, status, st);
 }
 
+// The one-kernel form of the small-batch plan (small_batch_fused.cuh), for calls of up to 32 tokens that keep nothing:
+// T selector CTAs and SMs - T streamer CTAs in one cooperative launch.  ok == false: the problem or the device does not
+// admit it (the multi-kernel forms run then).  MOC_FFN_SB_FUSED=0 in the environment switches it off (comparisons).
+struct FusedLayout {
+    int tn, n_stream, n_gu, rows, gu_boxes, gu_stages, accs, m_tiles, splits, stages;
+    uint32_t w_pitch, slot_bytes, tail_off;
+    size_t smem;
+};
+
+FusedLayout fused_layout(const moc_ffn_desc &d, bool saving, bool &ok) {
+    FusedLayout L{};
+    ok = false;
+    static const bool off = [] {
+        const char *e = getenv("MOC_FFN_SB_FUSED");
+        return e && atoi(e) == 0;
+    }();
+    static const int coop_ok = [] {
+        int dev = 0, v = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess) return 0;
+        return v;
+    }();
+    const int T = (int)d.tokens, F = d.d_ff, dm = d.d_model, sms = tc::sm_count();
+    if (off || !coop_ok || saving || (d.flags & MOC_FLAG_SELECT_2_OF_8) || T < 1 || T > sbf::kMaxTokens || sms < 4 * T) return L;
+    L.n_stream = sms - T;
+    L.tn = T <= 16 ? 16 : 32;
+    const uint32_t xbox = (uint32_t)L.tn * sb::kBK * 2;
+    L.rows = (F + L.n_stream - 1) / L.n_stream;
+    if (L.rows > sb::kTile) L.rows = (L.rows + 7) & ~7;  // the second MMA tile starts at a whole swizzle group
+    if (L.rows > sb::kMaxRows) return L;
+    L.n_gu = (F + L.rows - 1) / L.rows;
+    L.w_pitch = ((uint32_t)L.rows * sb::kBK * 2 + 1023u) & ~1023u;
+    down_geometry(dm, (F + sb::kBK - 1) / sb::kBK, L.accs, L.m_tiles, L.splits, L.n_stream);
+    if (L.m_tiles > L.n_stream) return L;
+    // a stage of phases G and U holds as many 64-element blocks as make it about the size of a stage of phase D (the
+    // ring's slots have one size): few large stages keep more bytes in flight than many small ones that leave slots half used
+    const uint32_t d_slot = (uint32_t)L.accs * 16384u + xbox, gu_box = xbox + L.w_pitch;
+    static const int forced_boxes = [] {
+        const char *e = getenv("MOC_FFN_SB_FUSED_BOXES");
+        return e ? atoi(e) : 0;
+    }();
+    L.gu_boxes = forced_boxes > 0 ? forced_boxes : std::max(1, std::min(8, (int)((d_slot + gu_box / 2) / gu_box)));
+    L.gu_stages = (dm + L.gu_boxes * sb::kBK - 1) / (L.gu_boxes * sb::kBK);
+    const uint32_t gu_slot = (uint32_t)L.gu_boxes * gu_box;
+    L.slot_bytes = std::max(gu_slot, d_slot);
+    // behind the ring: the gate values and the barriers, and at least as many bytes as an MMA over a short weight box
+    // reads past the ring's end (it always reads 128 rows)
+    const uint32_t past = (uint32_t)L.gu_boxes * xbox + (uint32_t)(L.gu_boxes - 1) * L.w_pitch + (uint32_t)sb::kTile * sb::kBK * 2;
+    const uint32_t tail = std::max<uint32_t>((uint32_t)sbf::kTn * L.rows * 4 + 512, past > L.slot_bytes ? past - L.slot_bytes : 0);
+    const size_t budget = (size_t)kMaxDynSmem - 2048 /*static state of the selector role*/ - 1024 /*alignment*/;
+    if (tail + 2 * (size_t)L.slot_bytes > budget) return L;
+    L.stages = (int)std::min<size_t>(sbf::kStagesMax, (budget - tail) / L.slot_bytes);
+    L.tail_off = (uint32_t)L.stages * L.slot_bytes;
+    L.smem = std::max((size_t)1024 + L.tail_off + tail, sbf::selector_smem(F));
+    if (L.smem + 2048 > (size_t)kMaxDynSmem) return L;
+    ok = true;
+    return L;
+}
+
+int forward_small_batch_fused(const moc_ffn_desc &d, const SmallBatchLayout &L, const FusedLayout &FL, const __nv_bfloat16 *x,
+                              const __nv_bfloat16 *wg, const __nv_bfloat16 *wu, const __nv_bfloat16 *wd, __nv_bfloat16 *out,
+                              char *wsp, cudaStream_t st, const __nv_bfloat16 *resid) {
+    const int T = (int)d.tokens, F = d.d_ff, dm = d.d_model;
+    int *status = device_status_ptr();
+    if (!status) return MOC_ERR_CUDA;
+    int rc;
+    if ((rc = set_smem(sbf::sb_fused_kernel, FL.smem, 2048)) != MOC_OK) return rc;
+    // all CTAs must be resident at once (the launch would be refused otherwise); asked once per shared-memory size
+    static std::mutex mu;
+    static std::unordered_map<size_t, int> per_sm_of;
+    int per_sm = 0;
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        auto it = per_sm_of.find(FL.smem);
+        if (it == per_sm_of.end()) {
+            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, sbf::sb_fused_kernel, sbf::kBlock, FL.smem) != cudaSuccess)
+                return MOC_ERR_CUDA;
+            per_sm_of[FL.smem] = per_sm;
+        } else {
+            per_sm = it->second;
+        }
+    }
+    if (per_sm < 1) return MOC_ERR_UNSUPPORTED;
+    sbf::FusedParams fp;
+    memset(&fp, 0, sizeof(fp));
+    __nv_bfloat16 *Z = reinterpret_cast<__nv_bfloat16 *>(wsp + L.off_z);
+    if (!tc::make_map(&fp.wg_map, wg, F, dm, dm, sb::kBK, FL.rows) || !tc::make_map(&fp.wu_map, wu, F, dm, dm, sb::kBK, FL.rows) ||
+        !tc::make_map(&fp.x_map, x, T, dm, dm, sb::kBK, FL.tn) || !tc::make_map(&fp.wd_map, wd, F, dm, dm, 64, sb::kBK) ||
+        !tc::make_map(&fp.z_map, Z, T, F, L.ldz, sb::kBK, FL.tn))
+        return MOC_ERR_CUDA;
+    fp.T = T;
+    fp.F = F;
+    fp.K = d.k;
+    fp.d = dm;
+    fp.tn = FL.tn;
+    fp.n_stream = FL.n_stream;
+    fp.n_gu = FL.n_gu;
+    fp.rows = FL.rows;
+    fp.w_pitch = FL.w_pitch;
+    fp.gu_boxes = FL.gu_boxes;
+    fp.gu_stages = FL.gu_stages;
+    fp.accs = FL.accs;
+    fp.m_tiles = FL.m_tiles;
+    fp.splits = FL.splits;
+    fp.kb_down = (F + sb::kBK - 1) / sb::kBK;
+    fp.slot_bytes = FL.slot_bytes;
+    fp.stages = FL.stages;
+    fp.tail_off = FL.tail_off;
+    fp.G = reinterpret_cast<float *>(wsp + L.off_g);
+    fp.ldf = L.ldf;
+    fp.kept_bits = reinterpret_cast<uint32_t *>(wsp + L.off_u);  // the bitmaps live where the three-kernel form keeps U
+    fp.kept_words = (F + 31) / 32;
+    fp.Z = Z;
+    fp.ldz = L.ldz;
+    fp.acc = reinterpret_cast<float *>(wsp + L.off_acc);
+    fp.out = out;
+    fp.resid = resid;
+    fp.counters = reinterpret_cast<int *>(wsp + L.off_cnt);
+    fp.flags = reinterpret_cast<unsigned int *>(wsp + L.off_cnt) + 2 * L.m_tiles;
+    fp.status = status;
+    if (FL.m_tiles > 2 * L.m_tiles) return MOC_ERR_UNSUPPORTED;
+    void *args[] = {&fp};
+    MOC_LAUNCH(KID_SB_FUSED, st,
+               cudaLaunchCooperativeKernel(reinterpret_cast<void *>(sbf::sb_fused_kernel), dim3(FL.n_stream + T), dim3(sbf::kBlock),
+                                           args, FL.smem, st));
+    return launch_ok();
+}
+
 int forward_small_batch(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat16 *wg,
                         const __nv_bfloat16 *wu, const __nv_bfloat16 *wd, __nv_bfloat16 *out, int16_t *idx,
                         __nv_bfloat16 *tg, __nv_bfloat16 *tu, char *wsp, cudaStream_t st,
@@ -1224,6 +1355,14 @@ int forward_small_batch(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __n
     if ((rc = set_smem(sb::sb_down_kernel, ds.smem, 1024)) != MOC_OK) return rc;
     if ((rc = set_smem(sb::sb_select_kernel, sel_smem)) != MOC_OK) return rc;
 
+    {
+        bool fused_ok = false;
+        const FusedLayout FL = fused_layout(d, idx != nullptr, fused_ok);
+        if (fused_ok) {
+            rc = forward_small_batch_fused(d, L, FL, x, wg, wu, wd, out, wsp, st, resid);
+            if (rc != MOC_ERR_UNSUPPORTED) return rc;
+        }
+    }
     if (small_batch_overlapped(d, idx != nullptr))
         return forward_small_batch_overlapped(d, L, x, wg, wu, wd, out, wsp, st, resid);
 
@@ -1916,6 +2055,155 @@ extern "C" __attribute__((visibility("default"))) int moc_debug_timeline(unsigne
     if (cudaDeviceSynchronize() != cudaSuccess) return MOC_ERR_CUDA;
     return cudaMemcpyFromSymbol(out, g_timeline, sizeof(unsigned long long) * (size_t)std::min(n, 4096)) == cudaSuccess
                ? MOC_OK : MOC_ERR_CUDA;
+}
+
+// development probe: W [rows_total, cols] bf16 is read once in TMA boxes of rows_per_cta rows x 64 columns, `boxes`
+// adjacent boxes per stage through a ring of `stages` stages, nothing computed
+namespace moc { namespace {
+struct BoxProbe {
+    CUtensorMap map;
+    int rows, cols, boxes, stages;
+    uint32_t pitch;
+    int *status;
+};
+__global__ void __launch_bounds__(64, 1) box_probe_kernel(const __grid_constant__ BoxProbe p) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint64_t bars[64];
+    __shared__ int s_abort;
+    const uint32_t base = (tc::smem_u32(smem_raw) + 1023u) & ~1023u;
+    auto full_bar = [&](int s) { return tc::smem_u32(&bars[s]); };
+    auto empty_bar = [&](int s) { return tc::smem_u32(&bars[32 + s]); };
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < p.stages; ++s) {
+            tc::mbar_init(full_bar(s), 1);
+            tc::mbar_init(empty_bar(s), 1);
+        }
+        s_abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+    const int n = (p.cols / 64 + p.boxes - 1) / p.boxes;
+    const int row0 = (int)blockIdx.x * p.rows;
+    if (threadIdx.x == 0) {
+        int stage = 0;
+        uint32_t phase = 0;
+        for (int i = 0; i < n; ++i) {
+            if (!tc::mbar_wait(empty_bar(stage), phase ^ 1u, &s_abort, p.status)) return;
+            tc::mbar_expect_tx(full_bar(stage), (uint32_t)p.boxes * (uint32_t)p.rows * 128u);
+            for (int b = 0; b < p.boxes; ++b)
+                tc::tma_load_2d(base + (uint32_t)stage * p.boxes * p.pitch + (uint32_t)b * p.pitch, &p.map, full_bar(stage),
+                                (i * p.boxes + b) * 64, row0);
+            if (++stage == p.stages) {
+                stage = 0;
+                phase ^= 1u;
+            }
+        }
+    } else if (threadIdx.x == 32) {
+        int stage = 0;
+        uint32_t phase = 0;
+        for (int i = 0; i < n; ++i) {
+            if (!tc::mbar_wait(full_bar(stage), phase, &s_abort, p.status)) return;
+            tc::mbar_arrive(empty_bar(stage));
+            if (++stage == p.stages) {
+                stage = 0;
+                phase ^= 1u;
+            }
+        }
+    }
+}
+} }
+extern "C" MOC_API int moc_debug_stream_boxes(const void *w, int rows_total, int cols, int rows_per_cta, int boxes, int stages,
+                                              void *cuda_stream) {
+    BoxProbe p;
+    memset(&p, 0, sizeof(p));
+    if (stages > 32 || rows_per_cta > 256) return MOC_ERR_INVALID_ARG;
+    if (!tc::make_map(&p.map, static_cast<const __nv_bfloat16 *>(w), rows_total, cols, cols, 64, rows_per_cta)) return MOC_ERR_CUDA;
+    p.rows = rows_per_cta;
+    p.cols = cols;
+    p.boxes = boxes;
+    p.stages = stages;
+    p.pitch = ((uint32_t)rows_per_cta * 128u + 1023u) & ~1023u;
+    p.status = device_status_ptr();
+    const size_t smem = 1024 + (size_t)stages * boxes * p.pitch;
+    int rc = set_smem(box_probe_kernel, smem, 1024);
+    if (rc != MOC_OK) return rc;
+    box_probe_kernel<<<(rows_total + rows_per_cta - 1) / rows_per_cta, 64, smem, static_cast<cudaStream_t>(cuda_stream)>>>(p);
+    return launch_ok();
+}
+
+// development probe: cycles of `count` back-to-back MMAs of shape M x N x 16 (operands in shared memory, K-major)
+namespace moc { namespace {
+__global__ void __launch_bounds__(128, 1) mma_probe_kernel(int m, int n, int count, int per_commit, int naccs, long long *cycles, int *status) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint64_t bars4[4];
+    __shared__ uint32_t holder;
+    __shared__ int s_abort;
+    const uint32_t base = (tc::smem_u32(smem_raw) + 1023u) & ~1023u;
+    for (int i = threadIdx.x; i < 64 * 1024 / 4; i += 128) reinterpret_cast<uint32_t *>(smem_raw + (base - tc::smem_u32(smem_raw)))[i] = (naccs & 4) ? (uint32_t)(i * 2654435761u) & 0xbfffbfffu : ((naccs & 8) ? 0x3f803f80u : 0u);
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < 4; ++i) tc::mbar_init(tc::smem_u32(&bars4[i]), 1);
+        s_abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (threadIdx.x < 32) {
+        tc::tmem_alloc(tc::smem_u32(&holder), 512);
+        tc::tmem_relinquish();
+    }
+    tc::tc_fence_before();
+    __syncthreads();
+    tc::tc_fence_after();
+    const uint32_t who = threadIdx.x >> 5;
+    const uint32_t tmem = holder + who * 128;
+    uint64_t &bar = bars4[2 * (who & 1)], &bar2 = bars4[2 * (who & 1) + 1];
+    if (threadIdx.x == 0 || ((naccs & 32) && threadIdx.x == 32)) {
+        const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+        uint32_t parity = 0;
+        const long long t0 = clock64();
+        const uint64_t ad0 = tc::make_smem_desc(base, 16, 1024), bd0 = tc::make_smem_desc(base + 49152, 16, 1024);
+        uint64_t ad[8], bd[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            ad[e] = ad0 + (uint64_t)((e & 3) * 2 + (e >> 2) * 704);
+            bd[e] = bd0 + (uint64_t)((e & 3) * 2);
+        }
+        for (int i = 0; i < count; i += per_commit) {
+            for (int j = 0; j < per_commit; j += 8) {
+#pragma unroll
+                for (int e = 0; e < 8; ++e)
+                    asm volatile(
+                        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, 1, 0;\n\t"
+                        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem), "l"(ad[e]), "l"(bd[e]), "r"(idesc)
+                        : "memory");
+            }
+            if ((naccs & 16) && i + per_commit < count) {
+                tc::umma_commit(tc::smem_u32(&bar2));  // nobody waits for this one
+                continue;
+            }
+            tc::umma_commit(tc::smem_u32(&bar));
+            if (!tc::mbar_wait(tc::smem_u32(&bar), parity, &s_abort, status)) break;
+            parity ^= 1u;
+        }
+        if (blockIdx.x == 0 && threadIdx.x == 0) *cycles = clock64() - t0;
+    }
+    tc::tc_fence_before();
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        tc::tc_fence_after();
+        tc::tmem_dealloc(holder, 512);
+    }
+}
+} }
+extern "C" MOC_API long long moc_debug_mma_cycles(int m, int n, int count, int per_commit, int naccs) {
+    long long *dev = nullptr, host = -1;
+    if (cudaMalloc(&dev, sizeof(long long)) != cudaSuccess) return -1;
+    const size_t smem = 66 * 1024;
+    if (set_smem(mma_probe_kernel, smem, 1024) != MOC_OK) return -2;
+    mma_probe_kernel<<<tc::sm_count(), 128, smem>>>(m, n, count, per_commit, naccs, dev, device_status_ptr());
+    if (cudaMemcpy(&host, dev, sizeof(host), cudaMemcpyDeviceToHost) != cudaSuccess) host = -3;
+    cudaFree(dev);
+    return host;
 }
 #endif
 

@@ -22,6 +22,10 @@ from . import synthetic as syn
 REGIONS = [(256, "gate start"), (512, "gate mma done"), (768, "gate end"), (1024, "select after wait"),
            (1280, "select end"), (1536, "up start"), (1792, "up mma done"), (2048, "up end"), (2304, "down start"),
            (2560, "down after wait"), (2816, "down mma done"), (3072, "down end")]
+# the one-kernel form (streamer CTAs, then the selector CTAs, in one grid)
+REGIONS_FUSED = [(256, "start"), (512, "after grid barrier"), (768, "gate mma done"), (1024, "gate values stored"),
+                 (1280, "select: row wait over"), (1536, "select end"), (1792, "up mma done"), (2048, "Z' stored"),
+                 (2304, "down: Z' complete"), (2560, "down mma done"), (2816, "end")]
 
 
 def main():
@@ -53,8 +57,10 @@ def main():
         raise SystemExit("reading the stamps failed")
     a = np.array(buf, dtype=np.uint64).astype(np.int64)
     ref = a[3] if a[3] else min(v for v in a[256:512] if v > 0)   # the first kernel's wait for the previous call returned
+    if a[11]:
+        print(f"MMA thread, gate phase of CTA 5: wait {a[8]} clk, issue {a[9]} clk, all {a[10]} clk in {a[11]} ns")
     print(f"T = {T}: us after the previous call completed -- min / median / max over CTAs (n)")
-    for base, name in REGIONS:
+    for base, name in (REGIONS if a[3] else REGIONS_FUSED):
         v = a[base:base + 256]
         v = v[v > 0]
         if len(v):
