@@ -44,6 +44,34 @@ int *device_status_ptr() {
     return have;
 }
 
+// State that the one-kernel small-batch form keeps from one run to the next (the counters of its column blocks, the
+// flags its CTAs signal with and a mark that says both are zero): kept in the library's own device memory rather than
+// in the caller's workspace, whose contents between calls are the caller's.  One block of kFusedStateWords words per
+// workspace address -- a workspace serves one call at a time, so a block is never used by two runs at once.
+constexpr int kFusedStateWords = 128, kFusedStateSlots = 256;
+__device__ unsigned int g_fused_state[kFusedStateSlots * kFusedStateWords];
+
+unsigned int *fused_state_for(const void *workspace) {
+    static std::mutex mu;
+    static std::unordered_map<uint64_t, int> slot_of[64];
+    static unsigned int *base[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!base[dev]) {
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_fused_state) != cudaSuccess) return nullptr;
+        base[dev] = static_cast<unsigned int *>(p);
+    }
+    auto &m = slot_of[dev];
+    auto it = m.find(reinterpret_cast<uint64_t>(workspace));
+    if (it == m.end()) {
+        if ((int)m.size() >= kFusedStateSlots) return nullptr;  // (the multi-kernel forms serve further workspaces)
+        it = m.emplace(reinterpret_cast<uint64_t>(workspace), (int)m.size()).first;
+    }
+    return base[dev] + (size_t)it->second * kFusedStateWords;
+}
+
 // ---- launch bookkeeping --------------------------------------------------------------------------
 // Every kernel the library launches goes through MOC_LAUNCH: it counts the launch and, while a
 // profiling window is open, brackets it with a pair of CUDA events on the caller's stream so that
@@ -1081,8 +1109,7 @@ SmallBatchLayout small_batch_layout(const moc_ffn_desc &d) {
     L.off_u = c.take((size_t)d.tokens * L.ldf * sizeof(float));
     L.off_z = c.take((size_t)d.tokens * L.ldz * sizeof(__nv_bfloat16));
     L.off_acc = c.take((size_t)d.tokens * d.d_model * sizeof(float));
-    // the column blocks' counters; the one-kernel form's geometry may have twice as many blocks and keeps its flags behind them
-    L.off_cnt = c.take(((size_t)2 * L.m_tiles + 8) * sizeof(int));
+    L.off_cnt = c.take((size_t)L.m_tiles * sizeof(int));
     L.total = c.off;
     return L;
 }
@@ -1324,15 +1351,41 @@ int forward_small_batch_fused(const moc_ffn_desc &d, const SmallBatchLayout &L, 
     fp.acc = reinterpret_cast<float *>(wsp + L.off_acc);
     fp.out = out;
     fp.resid = resid;
-    fp.counters = reinterpret_cast<int *>(wsp + L.off_cnt);
-    fp.flags = reinterpret_cast<unsigned int *>(wsp + L.off_cnt) + 2 * L.m_tiles;
+    unsigned int *state = fused_state_for(wsp);
+    if (!state || FL.m_tiles > sbf::kStateCounters) return MOC_ERR_UNSUPPORTED;
+    fp.counters = reinterpret_cast<int *>(state);
+    fp.flags = state + sbf::kStateCounters;
     fp.status = status;
-    if (FL.m_tiles > 2 * L.m_tiles) return MOC_ERR_UNSUPPORTED;
+    // cooperative, and allowed to become resident while the previous kernel in the stream drains (the kernel waits for
+    // that kernel's completion before it touches anything but the weights); a driver that refuses the combination gets
+    // the plain cooperative launch from then on
+    static std::atomic<int> pdl_ok{1};
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(FL.n_stream + T);
+    cfg.blockDim = dim3(sbf::kBlock);
+    cfg.dynamicSmemBytes = FL.smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
     void *args[] = {&fp};
-    MOC_LAUNCH(KID_SB_FUSED, st,
-               cudaLaunchCooperativeKernel(reinterpret_cast<void *>(sbf::sb_fused_kernel), dim3(FL.n_stream + T), dim3(sbf::kBlock),
-                                           args, FL.smem, st));
-    return launch_ok();
+    cudaError_t err = cudaErrorUnknown;
+    if (pdl_ok.load(std::memory_order_relaxed)) {
+        cfg.numAttrs = 2;
+        MOC_LAUNCH(KID_SB_FUSED, st, err = cudaLaunchKernelExC(&cfg, reinterpret_cast<const void *>(sbf::sb_fused_kernel), args));
+        if (err != cudaSuccess) {
+            (void)cudaGetLastError();
+            pdl_ok.store(0, std::memory_order_relaxed);
+        }
+    }
+    if (err != cudaSuccess) {
+        cfg.numAttrs = 1;
+        MOC_LAUNCH(KID_SB_FUSED, st, err = cudaLaunchKernelExC(&cfg, reinterpret_cast<const void *>(sbf::sb_fused_kernel), args));
+    }
+    return err == cudaSuccess ? launch_ok() : MOC_ERR_CUDA;
 }
 
 int forward_small_batch(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat16 *wg,

@@ -21,9 +21,15 @@
 // as a whole stage's MMAs.  The stall is the thread's, not the tensor core's: a second issuer fills it.  Each issuer
 // accumulates into its own tensor-memory columns.
 //
-// CTAs wait on one another, so the launch is cooperative: all CTAs are resident, or the launch fails.  The flags live
-// in the workspace; CTA 0 zeroes them and a grid barrier at the start (behind the first ring of weight requests)
-// publishes that.  Every wait is bounded as everywhere else in the library.
+// CTAs wait on one another, so the launch is cooperative: all CTAs are resident, or the launch fails.  Every wait is
+// bounded as everywhere else in the library.
+//
+// The flags and the column blocks' counters live in a block of the library's own device memory (one per workspace
+// address; the caller's workspace is the caller's between calls).  A run that completes leaves them zero and writes a
+// 64-bit mark behind them; a run that finds the mark starts at once (and removes it as soon as every CTA has read it,
+// so that a run that does not complete leaves no mark).  A run that finds no mark -- the first one, or the one after a
+// run that gave up on a wait -- has CTA 0 zero the block and publishes that with a grid barrier, some 4 us during
+// which only the first ring of requests is in flight.
 #pragma once
 
 #include <cooperative_groups.h>
@@ -43,6 +49,8 @@ constexpr int kEpiThreads = kEpiWarps * 32;
 constexpr int kMaxTokens = 32;            // one 32-token accumulator chunk
 constexpr int kTn = 32;                   // columns of tensor memory per accumulator (MMA N is 16 or 32)
 constexpr int kStagesMax = 8;
+constexpr int kStateCounters = 112;        // counters of the column blocks; the flags follow them in the state block
+constexpr unsigned long long kCleanMark = 0x6d6f632d66757365ull;  // "the flags and counters of this workspace are zero"
 // Tensor memory: every MMA issuer has its own accumulators (the epilogue adds them).  32 columns per tile;
 // issuer w: gate tiles at 64 w (+32), up tiles at 128 + 64 w (+32), down accumulators at 256 + 64 w (+32).
 constexpr uint32_t kTmemCols = 512;
@@ -73,8 +81,9 @@ struct FusedParams {
     float *acc;                  // [T, d] fp32
     __nv_bfloat16 *out;
     const __nv_bfloat16 *resid;  // the block form's residual, or nullptr
-    int *counters;               // [m_tiles]
-    unsigned int *flags;         // [0] streamers done with G, [1] tokens selected, [2] streamers done with Z'
+    int *counters;               // [kStateCounters], of which m_tiles are used
+    unsigned int *flags;         // [0] streamers done with G, [1] tokens selected, [2] streamers done with Z', [3] CTAs that
+                                 // have read the mark, [4] CTAs that have finished, [6..7] the mark (8-byte aligned)
     int *status;
 };
 
@@ -141,6 +150,18 @@ __device__ __forceinline__ void umma_lohi(uint32_t tmem_d, uint32_t a_lo, uint32
         : "memory");
 }
 
+// One thread of a CTA that has used the flags for the last time: the last CTA of the grid to get here zeroes them for
+// the next run and leaves the mark.  (A CTA that gave up on a wait never gets here: no mark.)
+__device__ __forceinline__ void cta_finished(const FusedParams &p) {
+    __threadfence();
+    if (atomicAdd(p.flags + 4, 1u) == gridDim.x - 1) {
+#pragma unroll
+        for (int i = 0; i < 5; ++i) p.flags[i] = 0u;
+        __threadfence();
+        *reinterpret_cast<volatile unsigned long long *>(p.flags + 6) = kCleanMark;
+    }
+}
+
 // ------------------------------------------------------------------------------------------------ selector role
 __device__ __forceinline__ void selector_role(const FusedParams &p, uint32_t *dyn) {
     __shared__ uint64_t s_bar;
@@ -187,7 +208,10 @@ __device__ __forceinline__ void selector_role(const FusedParams &p, uint32_t *dy
     }
     __threadfence();
     __syncthreads();
-    if (tid == 0) atomicAdd(p.flags + 1, 1u);
+    if (tid == 0) {
+        atomicAdd(p.flags + 1, 1u);
+        cta_finished(p);
+    }
     MOC_TL_CTA(1536);
 }
 
@@ -195,10 +219,19 @@ __device__ __forceinline__ void selector_role(const FusedParams &p, uint32_t *dy
 __global__ void __launch_bounds__(kBlock, 1) sb_fused_kernel(const __grid_constant__ FusedParams p) {
     namespace cg = cooperative_groups;
     extern __shared__ __align__(16) uint8_t smem_raw[];
-    __shared__ int s_last;
+    __shared__ int s_last, s_clean;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const bool streamer = (int)blockIdx.x < p.n_stream;
+    tc::pdl_launch_dependents();  // the next kernel in the stream may become resident as this one's CTAs leave
     MOC_TL_CTA(256);
+#ifdef MOC_TIMELINE
+    if (blockIdx.x == 0 && threadIdx.x == 0) {  // the starts of the last 64 calls
+        const unsigned long long n = atomicAdd(&g_timeline[4095], 1ull);
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+        g_timeline[3584 + (int)(n & 63ull)] = t;
+    }
+#endif
 
     // ---- the streamer's shared memory and work (a selector CTA computes the same numbers and uses none of them)
     const uint32_t raw = tc::smem_u32(smem_raw);
@@ -239,20 +272,27 @@ __global__ void __launch_bounds__(kBlock, 1) sb_fused_kernel(const __grid_consta
             pr_phase ^= 1u;
         }
     };
-    // stage `pr_item` of phases G and U: activation boxes first (their size is fixed), then the weight boxes
-    auto issue_gu = [&]() {
-        const bool up = pr_item >= n_gu;
+    // stage `item` of phases G and U: activation boxes first (their size is fixed), then the weight boxes
+    auto gu_block0 = [&](int item) {
         // CTAs walk the contraction dimension from different starting points, so that at any moment they ask for
         // different lines of x
-        int s = (up ? pr_item - n_gu : pr_item) + k_shift;
+        int s = (item >= n_gu ? item - n_gu : item) + k_shift;
         if (s >= n_gu) s -= n_gu;
-        const CUtensorMap *wm = up ? &p.wu_map : &p.wg_map;
-        tc::mbar_expect_tx(full_bar(pr_stage), gu_bytes);
-        for (int b = 0; b < p.gu_boxes; ++b) {
-            tc::tma_load_2d(slot(pr_stage) + nb * kXBox + (uint32_t)b * p.w_pitch, wm, full_bar(pr_stage), (p.gu_boxes * s + b) * kBK, ch0);
-            tc::tma_load_2d(slot(pr_stage) + (uint32_t)b * kXBox, &p.x_map, full_bar(pr_stage), (p.gu_boxes * s + b) * kBK, 0);
-        }
+        return p.gu_boxes * s;
     };
+    auto issue_gu_w = [&](int item, int stage) {
+        const CUtensorMap *wm = item >= n_gu ? &p.wu_map : &p.wg_map;
+        const int kb = gu_block0(item);
+        tc::mbar_expect_tx(full_bar(stage), gu_bytes);
+        for (int b = 0; b < p.gu_boxes; ++b)
+            tc::tma_load_2d(slot(stage) + nb * kXBox + (uint32_t)b * p.w_pitch, wm, full_bar(stage), (kb + b) * kBK, ch0);
+    };
+    auto issue_gu_x = [&](int item, int stage) {
+        const int kb = gu_block0(item);
+        for (int b = 0; b < p.gu_boxes; ++b)
+            tc::tma_load_2d(slot(stage) + (uint32_t)b * kXBox, &p.x_map, full_bar(stage), (kb + b) * kBK, 0);
+    };
+    const int ahead = min(p.stages, 2 * n_gu);  // stages requested before the grid barrier
 
     if (streamer) {
         if (threadIdx.x == 0) {
@@ -266,24 +306,37 @@ __global__ void __launch_bounds__(kBlock, 1) sb_fused_kernel(const __grid_consta
             *abort_flag = 0;
             asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            // the first ring of weight and activation boxes leaves before the grid barrier
-            const int ahead = min(p.stages, 2 * n_gu);
-            while (pr_item < ahead) {
-                issue_gu();
-                pr_next();
-            }
+            // the first ring of weight boxes leaves at once: the weights depend on nothing earlier in the stream
+            for (int i = 0; i < ahead; ++i) issue_gu_w(i, i);
         }
         if (warp == 1) {
             tc::tmem_alloc(tc::smem_u32(const_cast<uint32_t *>(tmem_holder)), kTmemCols);
             tc::tmem_relinquish();
         }
-        if (blockIdx.x == 0) {
-            if (threadIdx.x < 4) p.flags[threadIdx.x] = 0u;
-            for (int i = (int)threadIdx.x; i < p.m_tiles; i += kBlock) p.counters[i] = 0;
+    }
+    // everything below touches what earlier kernels in the stream may still read or write (x, the workspace, out)
+    tc::pdl_wait();
+    if (streamer && threadIdx.x == 0) {
+        for (int i = 0; i < ahead; ++i) {
+            issue_gu_x(i, i);
+            pr_next();
         }
     }
+    if (threadIdx.x == 0) {
+        s_clean = __ldcg(reinterpret_cast<const unsigned long long *>(p.flags + 6)) == kCleanMark ? 1 : 0;
+        // the last CTA to have read the mark removes it: from here on a run that does not complete leaves none
+        if (atomicAdd(p.flags + 3, 1u) == gridDim.x - 1 && s_clean)
+            *reinterpret_cast<volatile unsigned long long *>(p.flags + 6) = 0ull;
+    }
     tc::tc_fence_before();
-    cg::this_grid().sync();  // the flags and counters are zero for everyone; this CTA's barriers and TMEM address are set
+    __syncthreads();  // this CTA's barriers and TMEM address are set
+    if (!s_clean) {   // (the same answer in every CTA: the mark changes only once all have read it)
+        if (blockIdx.x == 0) {
+            if (threadIdx.x < 6) p.flags[threadIdx.x] = 0u;
+            for (int i = (int)threadIdx.x; i < kStateCounters; i += kBlock) p.counters[i] = 0;
+        }
+        cg::this_grid().sync();  // the flags and counters are zero for everyone
+    }
     tc::tc_fence_after();
     MOC_TL_CTA(512);
 
@@ -302,7 +355,8 @@ __global__ void __launch_bounds__(kBlock, 1) sb_fused_kernel(const __grid_consta
                     ok = false;
                     break;
                 }
-                issue_gu();
+                issue_gu_w(pr_item, pr_stage);
+                issue_gu_x(pr_item, pr_stage);
                 pr_next();
             }
             // W_down: the weight boxes of as many stages as the ring gives leave before Z' is complete
@@ -556,6 +610,7 @@ __global__ void __launch_bounds__(kBlock, 1) sb_fused_kernel(const __grid_consta
                     *reinterpret_cast<uint2 *>(p.out + (int64_t)t * p.d + col0 + c) =
                         make_uint2(tc::pack_bf16(v.x, v.y), tc::pack_bf16(v.z, v.w));
                 }
+                if (etid == 0) p.counters[m_blk] = 0;  // ready for the next run
             }
         }
     }
@@ -568,6 +623,7 @@ __global__ void __launch_bounds__(kBlock, 1) sb_fused_kernel(const __grid_consta
     tc::tc_fence_before();
     __syncthreads();
     MOC_TL_CTA(2816);
+    if (threadIdx.x == 0 && !*abort_flag) cta_finished(p);
     if (warp == 1) {
         tc::tc_fence_after();
         tc::tmem_dealloc(tmem_base, kTmemCols);

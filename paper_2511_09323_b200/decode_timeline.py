@@ -57,8 +57,9 @@ def main():
         raise SystemExit("reading the stamps failed")
     a = np.array(buf, dtype=np.uint64).astype(np.int64)
     ref = a[3] if a[3] else min(v for v in a[256:512] if v > 0)   # the first kernel's wait for the previous call returned
-    if a[11]:
-        print(f"MMA thread, gate phase of CTA 5: wait {a[8]} clk, issue {a[9]} clk, all {a[10]} clk in {a[11]} ns")
+    if a[4095]:
+        starts = np.sort(a[3584:3648][a[3584:3648] > 0])
+        print("one-kernel form: us between the starts of successive calls:", np.round(np.diff(starts[-8:]) / 1000.0, 2))
     print(f"T = {T}: us after the previous call completed -- min / median / max over CTAs (n)")
     for base, name in (REGIONS if a[3] else REGIONS_FUSED):
         v = a[base:base + 256]
