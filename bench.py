@@ -811,9 +811,10 @@ def decode_report(torch, B, syn, dev, peaks, calls=32, sets=4, replays=5):
                  "roofline_us": round(roof_us, 3), "algorithmic_bytes": algo, "union_channels": union,
                  "achieved_gbs": round(algo / (us * 1e-6) / 1e9, 1), "kernels_per_call": launches}
         names = kernels_of(lambda: B.moc_ffn_decode(x, *weights[0], w.k, out=out, workspace=ws))
-        if "sb_down" in names:   # every weight matrix streamed once
+        if "sb_down" in names or "sb_fused" in names:   # every weight matrix streamed once
             executed = 3 * w.d_ff * w.d_model * e + 2 * T * w.d_model * e
-            form = "selection beside the up stream" if names.count("sb_gate_up") == 2 else "gate+up, select, down"
+            form = ("one cooperative kernel, selector CTAs beside the up stream" if "sb_fused" in names else
+                    "selection beside the up stream" if names.count("sb_gate_up") == 2 else "gate+up, select, down")
             entry.update(plan=f"small-batch: all weights streamed once (tcgen05; {form})", executed_bytes=executed,
                          executed_frac=round(executed / (peaks["hbm_gbs"] * 1e9) * 1e6 / us, 4))
         else:

@@ -223,6 +223,10 @@ __global__ void __launch_bounds__(kBlock, 1) sb_fused_kernel(const __grid_consta
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const bool streamer = (int)blockIdx.x < p.n_stream;
     tc::pdl_launch_dependents();  // the next kernel in the stream may become resident as this one's CTAs leave
+    if (streamer && warp == 2 && lane < 5) {  // the tensor maps' first use would otherwise wait for their fetch
+        const CUtensorMap *m = lane == 0 ? &p.wg_map : lane == 1 ? &p.x_map : lane == 2 ? &p.wu_map : lane == 3 ? &p.wd_map : &p.z_map;
+        asm volatile("prefetch.tensormap [%0];" ::"l"(m) : "memory");
+    }
     MOC_TL_CTA(256);
 #ifdef MOC_TIMELINE
     if (blockIdx.x == 0 && threadIdx.x == 0) {  // the starts of the last 64 calls
@@ -322,14 +326,13 @@ __global__ void __launch_bounds__(kBlock, 1) sb_fused_kernel(const __grid_consta
             pr_next();
         }
     }
-    if (threadIdx.x == 0) {
-        s_clean = __ldcg(reinterpret_cast<const unsigned long long *>(p.flags + 6)) == kCleanMark ? 1 : 0;
-        // the last CTA to have read the mark removes it: from here on a run that does not complete leaves none
-        if (atomicAdd(p.flags + 3, 1u) == gridDim.x - 1 && s_clean)
-            *reinterpret_cast<volatile unsigned long long *>(p.flags + 6) = 0ull;
-    }
+    // (a thread other than the one that is busy requesting the first ring reads the mark)
+    if (threadIdx.x == 96) s_clean = __ldcg(reinterpret_cast<const unsigned long long *>(p.flags + 6)) == kCleanMark ? 1 : 0;
     tc::tc_fence_before();
     __syncthreads();  // this CTA's barriers and TMEM address are set
+    // the last CTA to have read the mark removes it: from here on a run that does not complete leaves none
+    if (threadIdx.x == 96 && atomicAdd(p.flags + 3, 1u) == gridDim.x - 1 && s_clean)
+        *reinterpret_cast<volatile unsigned long long *>(p.flags + 6) = 0ull;
     if (!s_clean) {   // (the same answer in every CTA: the mark changes only once all have read it)
         if (blockIdx.x == 0) {
             if (threadIdx.x < 6) p.flags[threadIdx.x] = 0u;
@@ -501,8 +504,24 @@ __global__ void __launch_bounds__(kBlock, 1) sb_fused_kernel(const __grid_consta
             asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
             if (etid == 0) atomicAdd(p.flags, 1u);
             MOC_TL_IF(1024 + (int)blockIdx.x, etid == 0);
-            // ---- Z' = SiLU(g) u on the kept channels
+            // ---- Z' = SiLU(g) u on the kept channels.  The products are formed for every channel as soon as the up
+            // projection is complete; the bitmaps, which usually arrive last, then only decide which of them are stored.
             ok = ok && __all_sync(0xffffffffu, tc::mbar_wait(tfull_u, 0u, abort_flag, p.status));
+            // (the CTAs of a problem with at most 128 channels per CTA and at most 16 tokens have one item per warp)
+            const int item0 = half;
+            const int tile0 = item0 / chunks, t00 = (item0 - tile0 * chunks) << 4;
+            float z0[16];
+            const bool pre = ok && item0 < items && !(tile0 == 1 && quarter * 32 + 31 < kTile - extra);
+            if (pre) {
+                tc::tc_fence_after();
+                const int row = tile0 == 0 ? trow : extra + trow;
+                tmem_ld16_sum(lane_addr + (uint32_t)(128 + tile0 * kTn + t00), two, z0);
+                if (row < valid && (tile0 == 0 ? trow < p.rows : trow >= kTile - extra)) {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i)
+                        if (t00 + i < p.T) z0[i] *= silu_f(key_to_float(gate_key(sg[(t00 + i) * p.rows + row])));
+                }
+            }
             {
                 int fine = 1;
                 if (lane == 0) fine = ok && flag_wait(p.flags + 1, (unsigned int)p.T, abort_flag, p.status) ? 1 : 0;
@@ -515,8 +534,6 @@ __global__ void __launch_bounds__(kBlock, 1) sb_fused_kernel(const __grid_consta
                     if (tile == 1 && quarter * 32 + 31 < kTile - extra) continue;
                     const int row = tile == 0 ? trow : extra + trow;
                     const bool mine = (tile == 0 ? trow < p.rows : trow >= kTile - extra) && row < valid;
-                    float u[16];
-                    tmem_ld16_sum(lane_addr + (uint32_t)(128 + tile * kTn + t0), two, u);
                     // the warp's 32 channels lie in at most two words of a token's bitmap: lane i fetches those of token
                     // t0 + i (one trip to L2 for the whole warp), the loop below hands them round
                     const int ch_lo = ch0 + (tile == 0 ? quarter * 32 : extra + quarter * 32);  // lane 0's channel
@@ -526,6 +543,18 @@ __global__ void __launch_bounds__(kBlock, 1) sb_fused_kernel(const __grid_consta
                         w_lo = __ldcg(kb);
                         if ((ch_lo >> 5) + 1 < p.kept_words) w_hi = __ldcg(kb + 1);
                     }
+                    float z[16];
+                    if (item == item0) {
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) z[i] = z0[i];
+                    } else {  // (warp-uniform)
+                        tmem_ld16_sum(lane_addr + (uint32_t)(128 + tile * kTn + t0), two, z);
+                        if (mine) {
+#pragma unroll
+                            for (int i = 0; i < 16; ++i)
+                                if (t0 + i < p.T) z[i] *= silu_f(key_to_float(gate_key(sg[(t0 + i) * p.rows + row])));
+                        }
+                    }
                     const int bit = (ch_lo & 31) + lane;  // position in the 64-bit pair
                     __nv_bfloat16 *dst = p.Z + ch_lo + lane + (int64_t)t0 * p.ldz;
 #pragma unroll
@@ -533,10 +562,7 @@ __global__ void __launch_bounds__(kBlock, 1) sb_fused_kernel(const __grid_consta
                         const uint32_t lo = __shfl_sync(0xffffffffu, w_lo, i), hi = __shfl_sync(0xffffffffu, w_hi, i);
                         if (t0 + i < p.T && mine) {
                             const bool kept = ((bit < 32 ? lo >> bit : hi >> (bit - 32)) & 1u) != 0u;
-                            float z = 0.f;
-                            // the gate value is recovered from its key, so that a NaN acts as -inf here as in the selection
-                            if (kept) z = silu_f(key_to_float(gate_key(sg[(t0 + i) * p.rows + row]))) * u[i];
-                            dst[(int64_t)i * p.ldz] = __float2bfloat16_rn(z);
+                            dst[(int64_t)i * p.ldz] = __float2bfloat16_rn(kept ? z[i] : 0.f);
                         }
                     }
                 }
