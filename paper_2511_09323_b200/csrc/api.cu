@@ -2185,15 +2185,18 @@ extern "C" MOC_API int moc_debug_stream_boxes(const void *w, int rows_total, int
     return launch_ok();
 }
 
-// development probe: cycles of `count` back-to-back MMAs of shape M x N x 16 (operands in shared memory, K-major)
+// development probe: cycles per MMA, seen by the issuing thread, of `count` MMAs of shape M x N x 16 (bf16, operands in
+// shared memory, K-major, all zero) issued back to back with a tcgen05.commit after every `per_commit` of them.
+// mode bit 0: the thread waits for every commit's barrier (else only for the last); bit 1: a second thread issues the same
+// sequence at the same time into its own TMEM columns and barriers (the figure is still the first thread's).
 namespace moc { namespace {
-__global__ void __launch_bounds__(128, 1) mma_probe_kernel(int m, int n, int count, int per_commit, int naccs, long long *cycles, int *status) {
+__global__ void __launch_bounds__(128, 1) mma_probe_kernel(int m, int n, int count, int per_commit, int mode, long long *cycles, int *status) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t bars4[4];
     __shared__ uint32_t holder;
     __shared__ int s_abort;
     const uint32_t base = (tc::smem_u32(smem_raw) + 1023u) & ~1023u;
-    for (int i = threadIdx.x; i < 64 * 1024 / 4; i += 128) reinterpret_cast<uint32_t *>(smem_raw + (base - tc::smem_u32(smem_raw)))[i] = (naccs & 4) ? (uint32_t)(i * 2654435761u) & 0xbfffbfffu : ((naccs & 8) ? 0x3f803f80u : 0u);
+    for (int i = threadIdx.x; i < 96 * 1024 / 4; i += 128) reinterpret_cast<uint32_t *>(smem_raw + (base - tc::smem_u32(smem_raw)))[i] = 0u;
     if (threadIdx.x == 0) {
         for (int i = 0; i < 4; ++i) tc::mbar_init(tc::smem_u32(&bars4[i]), 1);
         s_abort = 0;
@@ -2208,12 +2211,12 @@ __global__ void __launch_bounds__(128, 1) mma_probe_kernel(int m, int n, int cou
     __syncthreads();
     tc::tc_fence_after();
     const uint32_t who = threadIdx.x >> 5;
-    const uint32_t tmem = holder + who * 128;
-    uint64_t &bar = bars4[2 * (who & 1)], &bar2 = bars4[2 * (who & 1) + 1];
-    if (threadIdx.x == 0 || ((naccs & 32) && threadIdx.x == 32)) {
+    const uint32_t tmem = holder + who * 256;
+    const uint32_t bar = tc::smem_u32(&bars4[2 * who]), bar_unwaited = tc::smem_u32(&bars4[2 * who + 1]);
+    if (threadIdx.x == 0 || ((mode & 2) && threadIdx.x == 32)) {
         const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
         uint32_t parity = 0;
-        const long long t0 = clock64();
+        // eight descriptor pairs held in registers: A walks over three 11 KiB regions, so that the loop is nothing but MMAs
         const uint64_t ad0 = tc::make_smem_desc(base, 16, 1024), bd0 = tc::make_smem_desc(base + 49152, 16, 1024);
         uint64_t ad[8], bd[8];
 #pragma unroll
@@ -2221,6 +2224,7 @@ __global__ void __launch_bounds__(128, 1) mma_probe_kernel(int m, int n, int cou
             ad[e] = ad0 + (uint64_t)((e & 3) * 2 + (e >> 2) * 704);
             bd[e] = bd0 + (uint64_t)((e & 3) * 2);
         }
+        const long long t0 = clock64();
         for (int i = 0; i < count; i += per_commit) {
             for (int j = 0; j < per_commit; j += 8) {
 #pragma unroll
@@ -2230,12 +2234,12 @@ __global__ void __launch_bounds__(128, 1) mma_probe_kernel(int m, int n, int cou
                         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem), "l"(ad[e]), "l"(bd[e]), "r"(idesc)
                         : "memory");
             }
-            if ((naccs & 16) && i + per_commit < count) {
-                tc::umma_commit(tc::smem_u32(&bar2));  // nobody waits for this one
+            if (!(mode & 1) && i + per_commit < count) {
+                tc::umma_commit(bar_unwaited);  // nobody waits for this one
                 continue;
             }
-            tc::umma_commit(tc::smem_u32(&bar));
-            if (!tc::mbar_wait(tc::smem_u32(&bar), parity, &s_abort, status)) break;
+            tc::umma_commit(bar);
+            if (!tc::mbar_wait(bar, parity, &s_abort, status)) break;
             parity ^= 1u;
         }
         if (blockIdx.x == 0 && threadIdx.x == 0) *cycles = clock64() - t0;
@@ -2248,12 +2252,14 @@ __global__ void __launch_bounds__(128, 1) mma_probe_kernel(int m, int n, int cou
     }
 }
 } }
-extern "C" MOC_API long long moc_debug_mma_cycles(int m, int n, int count, int per_commit, int naccs) {
+extern "C" MOC_API long long moc_debug_mma_cycles(int m, int n, int count, int per_commit, int mode) {
+    if (m != 64 && m != 128) return -4;
+    if (n < 16 || n > 256 || n % 16 || count < 8 || per_commit < 8 || per_commit % 8 || count % per_commit) return -4;
     long long *dev = nullptr, host = -1;
     if (cudaMalloc(&dev, sizeof(long long)) != cudaSuccess) return -1;
-    const size_t smem = 66 * 1024;
+    const size_t smem = 100 * 1024;  // A within the first 48 KiB, B (up to 256 rows of 128 bytes) behind it
     if (set_smem(mma_probe_kernel, smem, 1024) != MOC_OK) return -2;
-    mma_probe_kernel<<<tc::sm_count(), 128, smem>>>(m, n, count, per_commit, naccs, dev, device_status_ptr());
+    mma_probe_kernel<<<tc::sm_count(), 128, smem>>>(m, n, count, per_commit, mode, dev, device_status_ptr());
     if (cudaMemcpy(&host, dev, sizeof(host), cudaMemcpyDeviceToHost) != cudaSuccess) host = -3;
     cudaFree(dev);
     return host;
