@@ -37,6 +37,8 @@ constexpr int kThreads = (kConsumerWarps + 1) * 32;  // + one producer warp
 constexpr int kMaxRows = 256;        // channels per CTA
 constexpr int kBins = 2048;          // top 11 bits of the key
 constexpr int kMaxStages = 32;         // a multiple of kConsumerWarps
+constexpr int kFirstRows = 8;  // gate rows requested before x is staged and the shared arrays are cleared (16 or 32 of them
+                               // made that start-up 0.9 us longer and the call 1 us slower: they compete with it for the path from L2)
 
 struct Params {
     const __nv_bfloat16 *x, *wg, *wu, *wd;
@@ -77,6 +79,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_coop_kernel(const Params p
     __shared__ int s_nsel;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const bool producer = warp == kConsumerWarps;
+    MOC_TL_CTA(256);
     const int d = p.d, F = p.F;
     __nv_bfloat16 *sx = reinterpret_cast<__nv_bfloat16 *>(dsm);
     uint8_t *ring = dsm + (size_t)T * d * 2;
@@ -154,7 +157,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_coop_kernel(const Params p
 
     // ---- start: the first gate rows leave at once (the ring is empty: nothing to wait for); x is staged and the
     //      CTA clears its slices of the arrays all CTAs share
-    const int first = min(min(p.stages, 8), rows);  // a few rows at once; the producer must not be late for the barrier below
+    const int first = min(min(p.stages, kFirstRows), rows);  // (the producer lane joins the barrier below: it must not be late)
     if (producer && lane == 0)
         for (int i = 0; i < first; ++i) produce_row(p.wg, c0 + i);
     {
@@ -196,6 +199,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_coop_kernel(const Params p
     // #0, split: the CTA announces that its slices are clear now and waits for the others only when it is about to
     // touch the shared arrays, after phase 1 (the arrival is a block-wide barrier too: x is staged)
     auto clear_token = grid.barrier_arrive();
+    MOC_TL_CTA(512);
 
     // ---- phase 1: gate values of the CTA's channels (one warp per row), histogram of their keys
     if (producer) {
@@ -220,6 +224,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_coop_kernel(const Params p
     }
     __syncthreads();
     grid.barrier_wait(std::move(clear_token));  // every CTA's slices of the shared arrays are clear
+    MOC_TL_CTA(768);
 
     // ---- selection
     if (!p.grouped) {
@@ -228,6 +233,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_coop_kernel(const Params p
             atomicAdd(&p.hist[t * kBins + (gate_key(sg[t * kMaxRows + r]) >> 21)], 1u);
         }
         grid.sync();  // #1 (the barrier's release / acquire pair orders the CTAs' writes before the others' reads): every CTA's keys are in the histogram
+        MOC_TL_CTA(1024);
         // the bin of the K-th largest key and the number of keys above that bin, per token (suffix sums over 2048 bins:
         // four bins per consumer thread)
         for (int t = 0; t < T; ++t) {
@@ -270,6 +276,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_coop_kernel(const Params p
             }
         }
         grid.sync();  // #2: the candidate lists are complete
+        MOC_TL_CTA(1280);
         // rank the CTA's own candidates: one warp per candidate, the lanes share the list -- which is first copied to
         // shared memory (the ring is idle between the phases) when it fits, so that the ranking loops do not pay a
         // trip to L2 per step
@@ -345,6 +352,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_coop_kernel(const Params p
     }
     __syncthreads();
     const int nsel = s_nsel;
+    MOC_TL_CTA(1536);
 
     // ---- phase 3: up rows (one warp per row: u, z = SiLU(g) u), then down rows (every thread owns 8 columns)
     float acc[T][8];
@@ -407,7 +415,9 @@ __global__ void __launch_bounds__(kThreads, 1) decode_coop_kernel(const Params p
         }
     }
     __syncthreads();
+    MOC_TL_CTA(1792);
     grid.sync();  // #3: every CTA's partial output is in the accumulator
+    MOC_TL_CTA(2048);
 
     // ---- out = bf16(accumulator), a slice per CTA
     {
@@ -425,6 +435,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_coop_kernel(const Params p
                 make_uint4(tc::pack_bf16(a.x, a.y), tc::pack_bf16(a.z, a.w), tc::pack_bf16(b.x, b.y), tc::pack_bf16(b.z, b.w));
         }
     }
+    MOC_TL_CTA(2304);
     if (s_abort) {  // copies still in flight must land before shared memory goes away
         const long long t0 = clock64();
         while (clock64() - t0 < 2000000LL) __nanosleep(1000);

@@ -27,6 +27,10 @@ REGIONS = [(256, "gate start"), (512, "gate mma done"), (768, "gate end"), (1024
 REGIONS_FUSED = [(256, "start"), (512, "after grid barrier"), (768, "gate mma done"), (1024, "gate values stored"),
                  (1280, "select: row wait over"), (1536, "select end"), (1792, "up mma done"), (2048, "Z' stored"),
                  (2304, "down: Z' complete"), (2560, "down mma done"), (2816, "end")]
+# the one-kernel decode form for one or two tokens
+REGIONS_COOP = [(256, "start"), (512, "x staged, arrays cleared"), (768, "gate rows done, barrier 0"), (1024, "histogram complete (barrier 1)"),
+                (1280, "candidate lists complete (barrier 2)"), (1536, "kept channels ranked"), (1792, "rows of W_up, W_down done"),
+                (2048, "barrier 3"), (2304, "end")]
 
 
 def main():
@@ -66,12 +70,12 @@ def main():
         starts = np.sort(a[3584:3648][a[3584:3648] > 0])
         print("one-kernel form: us between the starts of successive calls:", np.round(np.diff(starts[-8:]) / 1000.0, 2))
     print(f"T = {T}: us after the previous call completed -- min / median / max over CTAs (n)")
-    for base, name in (REGIONS if a[3] else REGIONS_FUSED):
+    for base, name in (REGIONS if a[3] else REGIONS_COOP if T <= 2 else REGIONS_FUSED):
         v = a[base:base + 256]
         v = v[v > 0]
         if len(v):
             r = (v - ref) / 1000.0
-            print(f"{name:18s} {r.min():8.2f} {np.median(r):8.2f} {r.max():8.2f}   ({len(v)})")
+            print(f"{name:38s} {r.min():8.2f} {np.median(r):8.2f} {r.max():8.2f}   ({len(v)})")
 
 
 if __name__ == "__main__":
