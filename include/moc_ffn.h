@@ -38,6 +38,16 @@
  *            releases its dependents early must be followed by an event or stream synchronisation first.
  * Threads    Entry points may be called from several host threads on different streams as long as
  *            their buffers (workspace included) do not overlap.
+ * Workspace  A workspace serves one call at a time: the next call that names it may be enqueued on the same stream
+ *            behind the first, or anywhere once the first has completed.  Its contents between calls are the
+ *            caller's (nothing in it outlives a call).  For batches of up to 32 tokens the library keeps three
+ *            counters per workspace ADDRESS in its own statically allocated device memory (they are left zero by
+ *            every call that completes, so a call can start without clearing them); 256 addresses per device are
+ *            served that way, further ones by the kernels that need no such state.
+ * Co-op      Two kernels are launched cooperatively (cudaLaunchCooperativeKernel: their CTAs wait on one another, so
+ *            all must be resident): the one-kernel forms of moc_ffn_decode / moc_ffn_forward for one or two tokens
+ *            and for up to 32 tokens that keep nothing.  On a device or in a context that cannot launch them
+ *            (no cooperative launch, SMs partly reserved) the multi-kernel forms run instead.
  */
 #ifndef MOC_FFN_H_
 #define MOC_FFN_H_
@@ -173,8 +183,9 @@ MOC_API int moc_ffn_recompute_up(const moc_ffn_desc *desc, const void *x, const 
  * (more: MOC_ERR_UNSUPPORTED; use moc_ffn_forward).  Up to 16 tokens it is organised so that only the
  * gate matrix and the selected rows of w_up / w_down are read from HBM (d d_ffn + 2 K d weight
  * elements per token instead of 3 d d_ffn).  From 17 tokens on the union of the tokens' channel sets
- * covers nearly every channel, and all three matrices are streamed once through tensor-core kernels
- * whose tiles are shaped for a few dozen tokens; moc_ffn_forward takes the same path for such batches.
+ * covers nearly every channel (from 6 tokens on at least half of them), and all three matrices are
+ * streamed once through tensor-core kernels whose tiles are shaped for a few dozen tokens;
+ * moc_ffn_forward takes the same path for such batches.
  * In both forms the partial sums of the down projection meet in an fp32 accumulator in an order that
  * is not fixed, so the last bit of `out` can differ from run to run.
  */
