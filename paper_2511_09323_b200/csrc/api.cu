@@ -111,6 +111,7 @@ enum KernelId {
     KID_TC_SP_DX_GEMM,
     KID_STREAM_PROBE,
     KID_SB_FUSED,
+    KID_TC_SPLIT_SUM,
     KID_COUNT
 };
 static const char *const kKernelNames[KID_COUNT] = {
@@ -121,6 +122,7 @@ static const char *const kKernelNames[KID_COUNT] = {
     "dec_select",      "dec_up",          "dec_down",      "sb_gate_up",     "sb_select",
     "sb_down",         "recompute_up",    "dec_coop",      "dec_rmsnorm",    "tc_compress_2of4",
     "tc_sp_down_gemm", "tc_sp_dx_gemm", "stream_probe",    "sb_fused",
+    "tc_split_sum",
 };
 
 struct Profiler {
@@ -592,15 +594,69 @@ int sparse_gemm_pair(int64_t M, int N, int K, int segments, const __nv_bfloat16 
     return rc;
 }
 
-// D = Z' W_down over all tokens: A = Z' [T, F] (K-major), B = Wd [F, d] (its contiguous dimension is N)
+// out = bf16(a + b), 8 elements per thread (the two halves of a contraction that was split, see below)
+__global__ void __launch_bounds__(256) split_sum_kernel(const float *__restrict__ a, const float *__restrict__ b,
+                                                        __nv_bfloat16 *__restrict__ out, int64_t n8) {
+    for (int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x; i < n8; i += (int64_t)gridDim.x * 256) {
+        const float4 a0 = __ldcs(reinterpret_cast<const float4 *>(a) + 2 * i), a1 = __ldcs(reinterpret_cast<const float4 *>(a) + 2 * i + 1);
+        const float4 b0 = __ldcs(reinterpret_cast<const float4 *>(b) + 2 * i), b1 = __ldcs(reinterpret_cast<const float4 *>(b) + 2 * i + 1);
+        reinterpret_cast<uint4 *>(out)[i] = make_uint4(tc::pack_bf16(a0.x + b0.x, a0.y + b0.y), tc::pack_bf16(a0.z + b0.z, a0.w + b0.w),
+                                                      tc::pack_bf16(a1.x + b1.x, a1.y + b1.y), tc::pack_bf16(a1.z + b1.z, a1.w + b1.w));
+    }
+}
+
+// A GEMM whose output has so few tiles that half of the CTA pairs would idle (a few hundred tokens: 32 tiles of
+// 256 x 256 for 512 tokens and d_model = 4096, each with the whole d_ffn to contract) is split in two along its
+// contraction: the halves run as two problems of one launch into fp32 partial outputs, which split_sum_kernel adds.
+// MOC_FFN_SPLIT_K=0 in the environment switches the split off (comparisons).
+bool split_contraction(int64_t T, int n_cols, size_t scratch_floats) {
+    static const bool on = [] {
+        const char *e = getenv("MOC_FFN_SPLIT_K");
+        return !(e && atoi(e) == 0);
+    }();
+    if (!on || !tc::pair_mode() || (n_cols & 7)) return false;
+    const int tiles = (ceil_div(T, tc::BM) + 1) / 2 * ceil_div(n_cols, tc::BN);
+    return 2 * tiles <= tc::sm_count() / 2 && (size_t)2 * T * n_cols <= scratch_floats;
+}
+
+int launch_split_sum(const float *partial, int64_t T, int n_cols, __nv_bfloat16 *out, cudaStream_t st) {
+    const int64_t n8 = T * n_cols / 8;
+    const unsigned grid = (unsigned)std::min<int64_t>((n8 + 255) / 256, (int64_t)tc::sm_count() * 8);
+    MOC_LAUNCH(KID_TC_SPLIT_SUM, st, (split_sum_kernel<<<grid, 256, 0, st>>>(partial, partial + T * n_cols, out, n8)));
+    return launch_ok();
+}
+
+// D = Z' W_down over all tokens: A = Z' [T, F] (K-major), B = Wd [F, d] (its contiguous dimension is N).
+// scratch: fp32 words of dead workspace for the partial outputs of a split contraction (or none)
 int forward_tc_down(const moc_ffn_desc &d, const __nv_bfloat16 *Z, int ldz, const __nv_bfloat16 *wd, __nv_bfloat16 *out,
-                    int *status, cudaStream_t st) {
+                    int *status, cudaStream_t st, float *scratch = nullptr, size_t scratch_floats = 0) {
     using namespace tc;
     const int F = d.d_ff, dm = d.d_model;
     const int64_t T = d.tokens;
     int rc = MOC_OK;
     Params q;
     init_params(q);
+    if (scratch && F >= 4 * BK && split_contraction(T, dm, scratch_floats)) {
+        const int Kc = ceil_div(ceil_div(F, 2), BK) * BK;  // channels of the first half: whole 64-channel blocks
+        for (int h = 0; h < 2; ++h) {
+            const int k0 = h * Kc, kn = std::min(Kc, F - k0);
+            if (!map_k_major(&q.a_map[h], Z + k0, T, kn, ldz, BM) || !map_mn_major(&q.b_map[h], wd + (int64_t)k0 * dm, kn, dm, dm))
+                return MOC_ERR_CUDA;
+            q.a_idx[h][0] = q.b_idx[h][0] = (int8_t)h;
+            q.c[h] = scratch + (int64_t)h * T * dm;
+            q.ldc[h] = dm;
+        }
+        q.num_problems = 2;
+        q.k_blocks = Kc / BK;
+        q.M = (int)T;
+        q.N = dm;
+        q.m_tiles = ceil_div(T, BM);
+        q.n_tiles = ceil_div(dm, BN);
+        q.status = status;
+        MOC_LAUNCH(KID_TC_DOWN_GEMM, st, (rc = launch_gemm<false, true, EPI_F32>(q, st)));
+        if (rc != MOC_OK) return rc;
+        return launch_split_sum(scratch, T, dm, out, st);
+    }
     if (!map_k_major(&q.a_map[0], Z, T, F, ldz, BM) || !map_mn_major(&q.b_map[0], wd, F, dm, dm)) return MOC_ERR_CUDA;
     q.k_blocks = ceil_div(F, BK);
     q.M = (int)T;
@@ -713,7 +769,8 @@ int forward_tc(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat1
         }
         if ((rc = launch_ok()) != MOC_OK) return rc;
     }
-    return forward_tc_down(d, U, L.ldf, wd, out, status, st);
+    // (the fp32 gate values are dead by now: their buffer takes the partial outputs of a split contraction)
+    return forward_tc_down(d, U, L.ldf, wd, out, status, st, G, (size_t)std::min<int64_t>(L.chunk, T) * L.ldf);
 }
 
 int small_batch_dx(const moc_ffn_desc &d, const __nv_bfloat16 *dG, const __nv_bfloat16 *dU, int ldf,
