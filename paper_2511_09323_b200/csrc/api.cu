@@ -1314,12 +1314,13 @@ FusedLayout fused_layout(const moc_ffn_desc &d, bool saving, bool &ok) {
         return v;
     }();
     const int T = (int)d.tokens, F = d.d_ff, dm = d.d_model, sms = tc::sm_count();
-    if (off || !coop_ok || saving || (d.flags & MOC_FLAG_SELECT_2_OF_8) || T < 1 || T > sbf::kMaxTokens || sms < 4 * T) return L;
-    L.n_stream = sms - T;
+    const bool grouped = (d.flags & MOC_FLAG_SELECT_2_OF_8) != 0;  // local mask: no selector CTAs
+    if (off || !coop_ok || saving || T < 1 || T > sbf::kMaxTokens || sms < 4 * T || (grouped && F % 8 != 0)) return L;
+    L.n_stream = grouped ? sms : sms - T;
     L.tn = T <= 16 ? 16 : 32;
     const uint32_t xbox = (uint32_t)L.tn * sb::kBK * 2;
     L.rows = (F + L.n_stream - 1) / L.n_stream;
-    if (L.rows > sb::kTile) L.rows = (L.rows + 7) & ~7;  // the second MMA tile starts at a whole swizzle group
+    if (L.rows > sb::kTile || grouped) L.rows = (L.rows + 7) & ~7;  // the second MMA tile starts at a whole swizzle group; whole groups of 8
     if (L.rows > sb::kMaxRows) return L;
     L.n_gu = (F + L.rows - 1) / L.rows;
     L.w_pitch = ((uint32_t)L.rows * sb::kBK * 2 + 1023u) & ~1023u;
@@ -1386,6 +1387,7 @@ int forward_small_batch_fused(const moc_ffn_desc &d, const SmallBatchLayout &L, 
     fp.K = d.k;
     fp.d = dm;
     fp.tn = FL.tn;
+    fp.grouped = (d.flags & MOC_FLAG_SELECT_2_OF_8) ? 1 : 0;
     fp.n_stream = FL.n_stream;
     fp.n_gu = FL.n_gu;
     fp.rows = FL.rows;
@@ -1418,7 +1420,7 @@ int forward_small_batch_fused(const moc_ffn_desc &d, const SmallBatchLayout &L, 
     // the plain cooperative launch from then on
     static std::atomic<int> pdl_ok{1};
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(FL.n_stream + T);
+    cfg.gridDim = dim3(FL.n_stream + (fp.grouped ? 0 : T));
     cfg.blockDim = dim3(sbf::kBlock);
     cfg.dynamicSmemBytes = FL.smem;
     cfg.stream = st;

@@ -61,6 +61,8 @@ struct FusedParams {
     CUtensorMap wd_map;          // [F, d]: boxes of 64 columns x 64 channels (the M-major operand of the down projection)
     CUtensorMap z_map;           // Z' [T, F]: boxes of tn tokens x 64 channels
     int T, F, K, d;
+    int grouped;                 // MoC 2:8 (Section 4): the mask is local to groups of 8 channels -- no selector CTAs, the streamers'
+                                 // epilogue picks the two largest of every group itself (rows is then a multiple of 8)
     int tn;                      // MMA N and rows of an activation box: 16 (up to 16 tokens) or 32
     int n_stream;                // streamer CTAs: blocks [0, n_stream); block n_stream + t selects for token t
     int n_gu;                    // streamers that own channels: ceil(F / rows)
@@ -493,16 +495,24 @@ __global__ void __launch_bounds__(kBlock, 1) sb_fused_kernel(const __grid_consta
 #pragma unroll
                         for (int i = 0; i < 16; ++i) {
                             if (t0 + i < p.T) {
-                                dst[(int64_t)i * p.ldf] = g[i];  // a warp's store: 128 contiguous bytes
+                                if (!p.grouped) dst[(int64_t)i * p.ldf] = g[i];  // a warp's store: 128 contiguous bytes
                                 sg[(t0 + i) * p.rows + row] = g[i];
                             }
                         }
                     }
                 }
             }
-            __threadfence();
-            asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
-            if (etid == 0) atomicAdd(p.flags, 1u);
+            if (p.grouped) {
+                // no selector CTAs: the streamers clear the output accumulator, a slice each (ordered before every
+                // addition to it by the count of streamers whose Z' is written, which each joins only afterwards)
+                const int64_t vecs = (int64_t)p.T * p.d / 4;
+                const int64_t v0 = vecs * blockIdx.x / p.n_gu, v1 = vecs * (blockIdx.x + 1) / p.n_gu;
+                for (int64_t i = v0 + etid; i < v1; i += kEpiThreads) reinterpret_cast<float4 *>(p.acc)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+            } else {
+                __threadfence();
+                asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
+                if (etid == 0) atomicAdd(p.flags, 1u);
+            }
             MOC_TL_IF(1024 + (int)blockIdx.x, etid == 0);
             // ---- Z' = SiLU(g) u on the kept channels.  The products are formed for every channel as soon as the up
             // projection is complete; the bitmaps, which usually arrive last, then only decide which of them are stored.
@@ -522,7 +532,7 @@ __global__ void __launch_bounds__(kBlock, 1) sb_fused_kernel(const __grid_consta
                         if (t00 + i < p.T) z0[i] *= silu_f(key_to_float(gate_key(sg[(t00 + i) * p.rows + row])));
                 }
             }
-            {
+            if (!p.grouped) {
                 int fine = 1;
                 if (lane == 0) fine = ok && flag_wait(p.flags + 1, (unsigned int)p.T, abort_flag, p.status) ? 1 : 0;
                 ok = __shfl_sync(0xffffffffu, fine, 0) != 0;
@@ -538,7 +548,7 @@ __global__ void __launch_bounds__(kBlock, 1) sb_fused_kernel(const __grid_consta
                     // t0 + i (one trip to L2 for the whole warp), the loop below hands them round
                     const int ch_lo = ch0 + (tile == 0 ? quarter * 32 : extra + quarter * 32);  // lane 0's channel
                     uint32_t w_lo = 0u, w_hi = 0u;
-                    if (lane < 16 && t0 + lane < p.T && (ch_lo >> 5) < p.kept_words) {
+                    if (!p.grouped && lane < 16 && t0 + lane < p.T && (ch_lo >> 5) < p.kept_words) {
                         const uint32_t *kb = p.kept_bits + (int64_t)(t0 + lane) * p.kept_words + (ch_lo >> 5);
                         w_lo = __ldcg(kb);
                         if ((ch_lo >> 5) + 1 < p.kept_words) w_hi = __ldcg(kb + 1);
@@ -559,11 +569,23 @@ __global__ void __launch_bounds__(kBlock, 1) sb_fused_kernel(const __grid_consta
                     __nv_bfloat16 *dst = p.Z + ch_lo + lane + (int64_t)t0 * p.ldz;
 #pragma unroll
                     for (int i = 0; i < 16; ++i) {
-                        const uint32_t lo = __shfl_sync(0xffffffffu, w_lo, i), hi = __shfl_sync(0xffffffffu, w_hi, i);
-                        if (t0 + i < p.T && mine) {
-                            const bool kept = ((bit < 32 ? lo >> bit : hi >> (bit - 32)) & 1u) != 0u;
-                            dst[(int64_t)i * p.ldz] = __float2bfloat16_rn(kept ? z[i] : 0.f);
+                        bool kept;
+                        if (p.grouped) {
+                            // the 8 channels of a group sit in 8 adjacent lanes: a channel is kept when fewer than two of
+                            // its group come before it in (key descending, channel ascending) order
+                            const uint32_t key = (mine && t0 + i < p.T) ? gate_key(sg[(t0 + i) * p.rows + row]) : 0u;
+                            int before = 0;
+#pragma unroll
+                            for (int m = 1; m < 8; ++m) {
+                                const uint32_t other = __shfl_xor_sync(0xffffffffu, key, m);
+                                before += (other > key || (other == key && ((lane ^ m) & 7) < (lane & 7))) ? 1 : 0;
+                            }
+                            kept = before < kGroupKeep;
+                        } else {
+                            const uint32_t lo = __shfl_sync(0xffffffffu, w_lo, i), hi = __shfl_sync(0xffffffffu, w_hi, i);
+                            kept = ((bit < 32 ? lo >> bit : hi >> (bit - 32)) & 1u) != 0u;
                         }
+                        if (t0 + i < p.T && mine) dst[(int64_t)i * p.ldz] = __float2bfloat16_rn(kept ? z[i] : 0.f);
                     }
                 }
             }

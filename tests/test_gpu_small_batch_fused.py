@@ -158,3 +158,36 @@ def test_one_kernel_form_many_workspaces_and_batch_sizes_interleaved():
             continue   # (below 6 tokens moc_ffn_decode takes the gathering plans)
         bad = np.abs(syn.to_f64(out) - full[:T]).max(axis=1) > tol
         assert bad.sum() <= 1, f"T={T}: {bad.sum()} tokens off"   # (a near-tie may swap one pick)
+
+
+@pytest.mark.parametrize("T,d,F", [
+    (3, 512, 2048),       # three tokens (half of the channels are in use at K = F / 4)
+    (16, 512, 2048),      # the 16-column MMA
+    (32, 264, 1000),      # the largest batch; 125 groups, contraction 4 blocks + 8 elements
+    (9, 128, 20000),      # more than 128 channels per CTA: groups in the second MMA tile
+    (16, 2048, 5504),     # the LLaMA-1B layer (padded width) of the MoC 2:8 benchmark
+])
+def test_one_kernel_form_with_the_2_of_8_mask(T, d, F):
+    """MoC 2:8 (Section 4): the mask is local to groups of 8 channels, so the kernel runs without selector CTAs and its
+    streamers pick the two largest of every group themselves.  Picks (from the path that returns them) are checked
+    against the oracle's rule, the output against the oracle's forward on those picks; equal gate rows in pairs make
+    every group tie."""
+    w = syn.Workload(f"sbf-2of8-{T}-{d}-{F}", "bf16", T, d, F, F, F // 4, seed=2100 + T)
+    wg, wu, wd = syn.make_weights(w)
+    if T == 16 and d == 512:
+        wg[1::2] = wg[0::2]    # equal values inside every group: the lower channels win
+    x = syn.make_x(w)
+    xd, wgd, wud, wdd = (t.cuda() for t in (x, wg, wu, wd))
+    outs = []
+    for rep in range(2):
+        names = _kernels_of(lambda: outs.append(B.moc_ffn_decode(xd, wgd, wud, wdd, None, grouped=True).clone()))
+        assert "sb_fused" in names and "sb_select" not in names, names
+    _, idx, _, _ = B.moc_ffn_forward(xd, wgd, wud, wdd, None, grouped=True)
+    torch.cuda.synchronize()
+    assert B.moc_last_device_status() == B.MOC_OK
+    x64, wg64, wu64, wd64 = map(syn.to_f64, (x, wg, wu, wd))
+    idx_np = idx.cpu().numpy()
+    parity.check_picks_grouped(idx_np, orc.gate_projection(x64, wg64))
+    ref = orc.forward_given_idx(x64, wg64, wu64, wd64, idx_np.astype(np.int32))["out"]
+    for o in outs:
+        parity.assert_close(syn.to_f64(o), ref, "bf16", "decode, 2 of 8")
