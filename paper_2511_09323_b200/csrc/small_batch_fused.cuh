@@ -479,6 +479,7 @@ __global__ void __launch_bounds__(kBlock, 1) sb_fused_kernel(const __grid_consta
         if (has_gu) {
             const int items = (extra ? 2 : 1) * chunks;
             const bool two = n_gu >= 2;  // the second issuer had stages of its own
+            uint32_t kept0 = 0u;         // MoC 2:8: bit i = this lane's channel is kept by token i of the warp's first item
             // ---- gate values
             ok = __all_sync(0xffffffffu, tc::mbar_wait(tfull_g, 0u, abort_flag, p.status));
             if (ok) {
@@ -498,6 +499,22 @@ __global__ void __launch_bounds__(kBlock, 1) sb_fused_kernel(const __grid_consta
                                 if (!p.grouped) dst[(int64_t)i * p.ldf] = g[i];  // a warp's store: 128 contiguous bytes
                                 sg[(t0 + i) * p.rows + row] = g[i];
                             }
+                        }
+                    }
+                    if (p.grouped && item == half) {
+                        // The 2-of-8 mask needs the gate values only: it is worked out now, while the up projection
+                        // streams, not after it.  The 8 channels of a group sit in 8 adjacent lanes: a channel is kept
+                        // when fewer than two of its group come before it in (key descending, channel ascending) order.
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            const uint32_t key = (mine && t0 + i < p.T) ? gate_key(g[i]) : 0u;
+                            int before = 0;
+#pragma unroll
+                            for (int m = 1; m < 8; ++m) {
+                                const uint32_t other = __shfl_xor_sync(0xffffffffu, key, m);
+                                before += (other > key || (other == key && ((lane ^ m) & 7) < (lane & 7))) ? 1 : 0;
+                            }
+                            kept0 |= (before < kGroupKeep ? 1u : 0u) << i;
                         }
                     }
                 }
@@ -570,9 +587,9 @@ __global__ void __launch_bounds__(kBlock, 1) sb_fused_kernel(const __grid_consta
 #pragma unroll
                     for (int i = 0; i < 16; ++i) {
                         bool kept;
-                        if (p.grouped) {
-                            // the 8 channels of a group sit in 8 adjacent lanes: a channel is kept when fewer than two of
-                            // its group come before it in (key descending, channel ascending) order
+                        if (p.grouped && item == item0) {
+                            kept = ((kept0 >> i) & 1u) != 0u;
+                        } else if (p.grouped) {
                             const uint32_t key = (mine && t0 + i < p.T) ? gate_key(sg[(t0 + i) * p.rows + row]) : 0u;
                             int before = 0;
 #pragma unroll

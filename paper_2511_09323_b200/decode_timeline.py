@@ -4,7 +4,7 @@ The timeline needs a library built with the stamps compiled in (without them the
 target for a profiler):
 
     MOC_FFN_NVCC_FLAGS=-DMOC_TIMELINE python -m paper_2511_09323_b200.build --force
-    python -m paper_2511_09323_b200.decode_timeline 16
+    python -m paper_2511_09323_b200.decode_timeline 16            # (a second argument `grouped`: the MoC 2:8 mask)
     python -m paper_2511_09323_b200.build --force          # back to the normal build
 
 Eight calls rotating four weight sets are replayed from one CUDA graph; every CTA of the small-batch kernels notes the
@@ -35,23 +35,26 @@ REGIONS_COOP = [(256, "start"), (512, "x staged, arrays cleared"), (768, "gate r
 
 def main():
     T = int(sys.argv[1]) if len(sys.argv) > 1 else 16
+    grouped = len(sys.argv) > 2 and sys.argv[2] == "grouped"   # the MoC 2:8 mask (K = d_ff / 4)
     lib = B.load()
     stamps = hasattr(lib, "moc_debug_timeline")
     w = syn.C4
     sets = [tuple(t.cuda() for t in syn.make_weights(w, seed_offset=s)) for s in range(4)]
     x = syn.make_x(w, tokens=T).cuda()
     out = torch.empty_like(x)
-    desc = B.make_desc(T, w.d_model, w.d_ff, w.k, x.dtype)
+    k = None if grouped else w.k
+    desc = B.make_desc(T, w.d_model, w.d_ff, w.d_ff // 4 if grouped else w.k, x.dtype,
+                       flags=B.MOC_FLAG_SELECT_2_OF_8 if grouped else 0)
     ws = B.alloc_workspace(desc, B.MOC_OP_DECODE)
     stream = torch.cuda.Stream()
     for i in range(4):
-        B.moc_ffn_decode(x, *sets[i % 4], w.k, out=out, workspace=ws)
+        B.moc_ffn_decode(x, *sets[i % 4], k, out=out, workspace=ws, grouped=grouped)
     torch.cuda.synchronize()
     graph = torch.cuda.CUDAGraph()
     with torch.cuda.stream(stream):
         with torch.cuda.graph(graph, stream=stream):
             for i in range(8):
-                B.moc_ffn_decode(x, *sets[i % 4], w.k, out=out, workspace=ws, stream=stream)
+                B.moc_ffn_decode(x, *sets[i % 4], k, out=out, workspace=ws, stream=stream, grouped=grouped)
     for _ in range(3):
         graph.replay()
     torch.cuda.synchronize()
