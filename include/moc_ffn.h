@@ -348,6 +348,20 @@ MOC_API int moc_tc_gemm_sp_dense_bf16(int64_t m, int64_t n, int64_t k, const voi
 MOC_API int moc_test_bounded_wait(int64_t limit_cycles, void *cuda_stream);
 
 /*
+ * Test hook for the time-out path of the one kernel in which CTAs wait on one another through global memory (the
+ * cooperative small-batch forward for up to 32 tokens): the call is moc_ffn_decode's, except that the selector CTAs
+ * are told to wait for one streamer more than exists, and that every wait gives up after `limit_cycles` SM clock
+ * cycles (1 .. 4e9) instead of the library's two seconds.  Every CTA then runs into a wait that nothing completes,
+ * raises MOC_ERR_TIMEOUT and returns normally; `out` is not written; nothing traps or faults, the context stays usable,
+ * and the next call on the same workspace finds no "clean" mark and prepares its counters itself.  Arguments, layouts
+ * and host-side errors as moc_ffn_decode; MOC_ERR_UNSUPPORTED where that kernel would not run (more than 32 tokens,
+ * the 2-of-8 mask, no cooperative launch).  (The paper has no counterpart.)
+ */
+MOC_API int moc_test_small_batch_stall(const moc_ffn_desc *desc, const void *x, const void *w_gate, const void *w_up,
+                                       const void *w_down, void *out, void *workspace, size_t workspace_bytes,
+                                       int64_t limit_cycles, void *cuda_stream);
+
+/*
  * Synchronises `cuda_stream`, then returns and clears the current device's sticky status word:
  * MOC_OK, MOC_ERR_TIMEOUT or MOC_ERR_BAD_INDEX (MOC_ERR_CUDA if the synchronisation itself failed).
  */

@@ -36,7 +36,7 @@ EXPORTED = (
     "moc_profile_read", "moc_ffn_decode_static", "moc_tc_gemm_bf16", "moc_ffn_recompute_up",
     "moc_ffn_backward_overlap", "moc_topk_select_tc", "moc_topk_select_tc_workspace_bytes", "moc_ffn_decode_probe",
     "moc_ffn_decode_probe_workspace_bytes", "moc_tc_gemm_sp_bf16", "moc_tc_gemm_sp_dense_bf16",
-    "moc_tc_gemm_sp_dense_workspace_bytes", "moc_profile_stream_read",
+    "moc_tc_gemm_sp_dense_workspace_bytes", "moc_profile_stream_read", "moc_test_small_batch_stall",
 )
 
 
@@ -112,6 +112,8 @@ def load() -> ctypes.CDLL:
         lib.moc_last_device_status.restype = ctypes.c_int
         lib.moc_test_bounded_wait.argtypes = [ctypes.c_int64, vp]
         lib.moc_test_bounded_wait.restype = ctypes.c_int
+        lib.moc_test_small_batch_stall.argtypes = [dp] + [vp] * 6 + [sz, ctypes.c_int64, vp]
+        lib.moc_test_small_batch_stall.restype = ctypes.c_int
         lib.moc_last_device_status.argtypes = [vp]
         lib.moc_status_string.restype = ctypes.c_char_p
         lib.moc_status_string.argtypes = [ctypes.c_int]
@@ -454,6 +456,26 @@ def moc_test_bounded_wait(limit_cycles: int, stream=None) -> None:
     rc = load().moc_test_bounded_wait(int(limit_cycles), _stream_ptr(stream))
     if rc != MOC_OK:
         raise MocError(rc, "moc_test_bounded_wait")
+
+
+def moc_test_small_batch_stall(x, w_gate, w_up, w_down, k, limit_cycles: int, d_ff=None, out=None, workspace=None,
+                               stream=None):
+    """moc_ffn_decode's call for up to 32 tokens, run so that every CTA of its cooperative kernel meets a wait that nothing
+    completes and gives up after `limit_cycles` SM cycles (the status word then reads MOC_ERR_TIMEOUT; `out` is not
+    written).  Returns `out`."""
+    _check_dev(x, w_gate, w_up, w_down, out, workspace)
+    T, d = x.shape
+    F_ld = w_gate.shape[0]
+    desc = make_desc(T, d, F_ld if d_ff is None else d_ff, k, x.dtype, d_ff_ld=F_ld)
+    if out is None:
+        out = torch.empty_like(x)
+    if workspace is None:
+        workspace = alloc_workspace(desc, MOC_OP_DECODE, x.device)
+    rc = load().moc_test_small_batch_stall(ctypes.byref(desc), _ptr(x), _ptr(w_gate), _ptr(w_up), _ptr(w_down), _ptr(out),
+                                           _ptr(workspace), workspace.numel(), int(limit_cycles), _stream_ptr(stream))
+    if rc != MOC_OK:
+        raise MocError(rc, "moc_test_small_batch_stall")
+    return out
 
 
 def moc_launch_count() -> int:

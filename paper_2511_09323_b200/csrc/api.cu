@@ -1353,7 +1353,8 @@ FusedLayout fused_layout(const moc_ffn_desc &d, bool saving, bool &ok) {
 
 int forward_small_batch_fused(const moc_ffn_desc &d, const SmallBatchLayout &L, const FusedLayout &FL, const __nv_bfloat16 *x,
                               const __nv_bfloat16 *wg, const __nv_bfloat16 *wu, const __nv_bfloat16 *wd, __nv_bfloat16 *out,
-                              char *wsp, cudaStream_t st, const __nv_bfloat16 *resid) {
+                              char *wsp, cudaStream_t st, const __nv_bfloat16 *resid, long long wait_limit = tc::kWaitLimitCycles,
+                              int stall = 0) {
     const int T = (int)d.tokens, F = d.d_ff, dm = d.d_model;
     int *status = device_status_ptr();
     if (!status) return MOC_ERR_CUDA;
@@ -1415,6 +1416,8 @@ int forward_small_batch_fused(const moc_ffn_desc &d, const SmallBatchLayout &L, 
     fp.counters = reinterpret_cast<int *>(state);
     fp.flags = state + sbf::kStateCounters;
     fp.status = status;
+    fp.wait_limit = wait_limit;
+    fp.stall = stall;
     // cooperative, and allowed to become resident while the previous kernel in the stream drains (the kernel waits for
     // that kernel's completion before it touches anything but the weights); a driver that refuses the combination gets
     // the plain cooperative launch from then on
@@ -2139,6 +2142,26 @@ int moc_tc_gemm_sp_dense_bf16(int64_t m, int64_t n, int64_t k, const void *a_den
         *overflow_count = h;
     }
     return MOC_OK;
+}
+
+int moc_test_small_batch_stall(const moc_ffn_desc *desc, const void *x, const void *w_gate, const void *w_up,
+                               const void *w_down, void *out, void *workspace, size_t workspace_bytes, int64_t limit_cycles,
+                               void *cuda_stream) {
+    int rc = check_desc(desc);
+    if (rc != MOC_OK) return rc;
+    if (limit_cycles < 1 || limit_cycles > tc::kWaitLimitCycles) return MOC_ERR_INVALID_ARG;
+    if (!good_ptr(x) || !good_ptr(w_gate) || !good_ptr(w_up) || !good_ptr(w_down) || !good_ptr(out)) return MOC_ERR_INVALID_ARG;
+    if (!use_small_batch_plan(*desc) || (desc->flags & MOC_FLAG_SELECT_2_OF_8)) return MOC_ERR_UNSUPPORTED;
+    const size_t need = moc_ffn_workspace_bytes(desc, MOC_OP_DECODE);
+    if (!good_ptr(workspace) || workspace_bytes < need) return MOC_ERR_WORKSPACE;
+    bool ok = false;
+    const FusedLayout FL = fused_layout(*desc, false, ok);
+    if (!ok) return MOC_ERR_UNSUPPORTED;
+    using T = __nv_bfloat16;
+    const SmallBatchLayout L = small_batch_layout(*desc);
+    return forward_small_batch_fused(*desc, L, FL, (const T *)x, (const T *)w_gate, (const T *)w_up, (const T *)w_down, (T *)out,
+                                     static_cast<char *>(workspace), static_cast<cudaStream_t>(cuda_stream), nullptr,
+                                     (long long)limit_cycles, 1);
 }
 
 int moc_test_bounded_wait(int64_t limit_cycles, void *cuda_stream) {

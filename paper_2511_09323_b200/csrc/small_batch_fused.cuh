@@ -87,6 +87,8 @@ struct FusedParams {
     unsigned int *flags;         // [0] streamers done with G, [1] tokens selected, [2] streamers done with Z', [3] CTAs that
                                  // have read the mark, [4] CTAs that have finished, [6..7] the mark (8-byte aligned)
     int *status;
+    long long wait_limit;        // cycles after which a wait gives up (tc::kWaitLimitCycles; shorter in the time-out test)
+    int stall;                   // the time-out test: the selectors wait for this many streamers more than exist
 };
 
 // shared memory of the selector role: keys [Fp] | two candidate lists | the radix select's state
@@ -101,13 +103,14 @@ __device__ __forceinline__ unsigned int ld_acquire(const unsigned int *p) {
     return v;
 }
 // Bounded wait until *flag >= target.  False: it gave up (MOC_ERR_TIMEOUT raised) or another role already had.
-__device__ __forceinline__ bool flag_wait(const unsigned int *flag, unsigned int target, volatile int *abort_flag, int *status) {
+__device__ __forceinline__ bool flag_wait(const unsigned int *flag, unsigned int target, volatile int *abort_flag, int *status,
+                                          long long limit_cycles) {
     if (ld_acquire(flag) >= target) return true;
     const long long t0 = clock64();
     while (ld_acquire(flag) < target) {
         __nanosleep(40);
         if (*abort_flag) return false;
-        if (clock64() - t0 > tc::kWaitLimitCycles) {
+        if (clock64() - t0 > limit_cycles) {
             *abort_flag = 1;
             raise_status(status, MOC_ERR_TIMEOUT);
             return false;
@@ -178,7 +181,7 @@ __device__ __forceinline__ void selector_role(const FusedParams &p, uint32_t *dy
         reinterpret_cast<float4 *>(p.acc + (int64_t)t * p.d)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     if (tid == 0) {
         s_abort = 0;
-        flag_wait(p.flags, (unsigned int)p.n_gu, &s_abort, p.status);  // every streamer's gate values are in G
+        flag_wait(p.flags, (unsigned int)(p.n_gu + p.stall), &s_abort, p.status, p.wait_limit);  // every streamer's gate values are in G
         asm volatile("fence.proxy.async;" ::: "memory");               // ... written by ordinary stores; a bulk copy reads them
     }
     __syncthreads();
@@ -356,7 +359,7 @@ __global__ void __launch_bounds__(kBlock, 1) sb_fused_kernel(const __grid_consta
         if (lane == 0) {
             bool ok = true;
             while (ok && pr_item < 2 * n_gu) {  // W_gate, then W_up
-                if (!tc::mbar_wait(empty_bar(pr_stage), pr_phase ^ 1u, abort_flag, p.status)) {
+                if (!tc::mbar_wait(empty_bar(pr_stage), pr_phase ^ 1u, abort_flag, p.status, p.wait_limit)) {
                     ok = false;
                     break;
                 }
@@ -372,7 +375,7 @@ __global__ void __launch_bounds__(kBlock, 1) sb_fused_kernel(const __grid_consta
             const int first_stage = pr_stage;
             int issued = 0;
             for (; issued < n_d && issued < p.stages && ok; ++issued) {
-                if (!tc::mbar_wait(empty_bar(pr_stage), pr_phase ^ 1u, abort_flag, p.status)) {
+                if (!tc::mbar_wait(empty_bar(pr_stage), pr_phase ^ 1u, abort_flag, p.status, p.wait_limit)) {
                     ok = false;
                     break;
                 }
@@ -381,7 +384,7 @@ __global__ void __launch_bounds__(kBlock, 1) sb_fused_kernel(const __grid_consta
                 pr_next();
             }
             if (ok && n_d > 0) {
-                ok = flag_wait(p.flags + 2, (unsigned int)p.n_gu, abort_flag, p.status);  // every streamer's part of Z' is written
+                ok = flag_wait(p.flags + 2, (unsigned int)p.n_gu, abort_flag, p.status, p.wait_limit);  // every streamer's part of Z' is written
                 asm volatile("fence.proxy.async;" ::: "memory");                           // ... by ordinary stores; TMA reads it
                 MOC_TL_CTA_ANY(2304);
                 int st = first_stage;
@@ -391,7 +394,7 @@ __global__ void __launch_bounds__(kBlock, 1) sb_fused_kernel(const __grid_consta
                 }
             }
             for (int i = issued; i < n_d && ok; ++i) {
-                if (!tc::mbar_wait(empty_bar(pr_stage), pr_phase ^ 1u, abort_flag, p.status)) break;
+                if (!tc::mbar_wait(empty_bar(pr_stage), pr_phase ^ 1u, abort_flag, p.status, p.wait_limit)) break;
                 tc::mbar_expect_tx(full_bar(pr_stage), d_bytes);
                 load_wd(pr_stage, kb0 + i);
                 tc::tma_load_2d(slot(pr_stage) + d_w_bytes, &p.z_map, full_bar(pr_stage), (kb0 + i) * kBK, 0);
@@ -422,7 +425,7 @@ __global__ void __launch_bounds__(kBlock, 1) sb_fused_kernel(const __grid_consta
                 const uint32_t acc0 = tmem_base + (uint32_t)(128 * m) + 64u * w;
                 uint32_t accum = 0u;
                 for (int s = 0; s < n_gu; ++s) {
-                    if (!tc::mbar_wait(full_bar(stage), phase, abort_flag, p.status)) {
+                    if (!tc::mbar_wait(full_bar(stage), phase, abort_flag, p.status, p.wait_limit)) {
                         ok = false;
                         break;
                     }
@@ -447,7 +450,7 @@ __global__ void __launch_bounds__(kBlock, 1) sb_fused_kernel(const __grid_consta
             const uint32_t accd = tmem_base + 256u + 64u * w;
             uint32_t accum = 0u;
             for (int i = 0; i < n_d && ok; ++i) {
-                if (!tc::mbar_wait(full_bar(stage), phase, abort_flag, p.status)) {
+                if (!tc::mbar_wait(full_bar(stage), phase, abort_flag, p.status, p.wait_limit)) {
                     ok = false;
                     break;
                 }
@@ -481,7 +484,7 @@ __global__ void __launch_bounds__(kBlock, 1) sb_fused_kernel(const __grid_consta
             const bool two = n_gu >= 2;  // the second issuer had stages of its own
             uint32_t kept0 = 0u;         // MoC 2:8: bit i = this lane's channel is kept by token i of the warp's first item
             // ---- gate values
-            ok = __all_sync(0xffffffffu, tc::mbar_wait(tfull_g, 0u, abort_flag, p.status));
+            ok = __all_sync(0xffffffffu, tc::mbar_wait(tfull_g, 0u, abort_flag, p.status, p.wait_limit));
             if (ok) {
                 tc::tc_fence_after();
                 for (int item = half; item < items; item += 2) {
@@ -528,12 +531,13 @@ __global__ void __launch_bounds__(kBlock, 1) sb_fused_kernel(const __grid_consta
             } else {
                 __threadfence();
                 asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
-                if (etid == 0) atomicAdd(p.flags, 1u);
+                if (etid == 0 && !*abort_flag) atomicAdd(p.flags, 1u);  // (a CTA that gave up is never counted: those that
+                                                                          //  wait for it give up in turn, nothing half-done is read)
             }
             MOC_TL_IF(1024 + (int)blockIdx.x, etid == 0);
             // ---- Z' = SiLU(g) u on the kept channels.  The products are formed for every channel as soon as the up
             // projection is complete; the bitmaps, which usually arrive last, then only decide which of them are stored.
-            ok = ok && __all_sync(0xffffffffu, tc::mbar_wait(tfull_u, 0u, abort_flag, p.status));
+            ok = ok && __all_sync(0xffffffffu, tc::mbar_wait(tfull_u, 0u, abort_flag, p.status, p.wait_limit));
             // (the CTAs of a problem with at most 128 channels per CTA and at most 16 tokens have one item per warp)
             const int item0 = half;
             const int tile0 = item0 / chunks, t00 = (item0 - tile0 * chunks) << 4;
@@ -551,7 +555,7 @@ __global__ void __launch_bounds__(kBlock, 1) sb_fused_kernel(const __grid_consta
             }
             if (!p.grouped) {
                 int fine = 1;
-                if (lane == 0) fine = ok && flag_wait(p.flags + 1, (unsigned int)p.T, abort_flag, p.status) ? 1 : 0;
+                if (lane == 0) fine = ok && flag_wait(p.flags + 1, (unsigned int)p.T, abort_flag, p.status, p.wait_limit) ? 1 : 0;
                 ok = __shfl_sync(0xffffffffu, fine, 0) != 0;
             }
             if (ok) {
@@ -608,12 +612,12 @@ __global__ void __launch_bounds__(kBlock, 1) sb_fused_kernel(const __grid_consta
             }
             __threadfence();
             asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
-            if (etid == 0) atomicAdd(p.flags + 2, 1u);
+            if (etid == 0 && !*abort_flag) atomicAdd(p.flags + 2, 1u);
             MOC_TL_IF(2048 + (int)blockIdx.x, etid == 0);
         }
         // ---- D: partial sums into the fp32 accumulator, the last CTA of the column block rounds
         if (has_d) {
-            const bool done = ok && __all_sync(0xffffffffu, tc::mbar_wait(tfull_d, 0u, abort_flag, p.status));
+            const bool done = ok && __all_sync(0xffffffffu, tc::mbar_wait(tfull_d, 0u, abort_flag, p.status, p.wait_limit));
             if (done) {
                 tc::tc_fence_after();
                 const bool two = n_d >= 2;
@@ -657,7 +661,7 @@ __global__ void __launch_bounds__(kBlock, 1) sb_fused_kernel(const __grid_consta
             }
             __threadfence();
             asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
-            if (etid == 0) s_last = atomicAdd(&p.counters[m_blk], 1) == p.splits - 1;
+            if (etid == 0) s_last = !*abort_flag && atomicAdd(&p.counters[m_blk], 1) == p.splits - 1;
             asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
             if (s_last) {
                 __threadfence();

@@ -191,3 +191,36 @@ def test_one_kernel_form_with_the_2_of_8_mask(T, d, F):
     ref = orc.forward_given_idx(x64, wg64, wu64, wd64, idx_np.astype(np.int32))["out"]
     for o in outs:
         parity.assert_close(syn.to_f64(o), ref, "bf16", "decode, 2 of 8")
+
+
+def test_one_kernel_form_gives_up_cleanly_when_a_wait_cannot_complete():
+    """The kernel's CTAs wait on one another through counters in global memory.  The test hook tells the selector CTAs
+    to wait for one streamer more than exists and shortens every wait's limit to 100 M cycles (about 50 ms): every CTA
+    then meets a wait that nothing completes, gives up, raises MOC_ERR_TIMEOUT and returns -- nothing hangs, traps or
+    faults, `out` is not written, the context stays usable, and the next calls on the same workspace (which find no
+    "clean" mark and prepare the counters themselves) are right."""
+    import time
+    w = syn.Workload("sbf-stall", "bf16", 8, 256, 1000, 1000, 125, seed=31)
+    wg, wu, wd = syn.make_weights(w)
+    x = syn.make_x(w)
+    xd, wgd, wud, wdd = (t.cuda() for t in (x, wg, wu, wd))
+    desc = B.make_desc(w.tokens, w.d_model, w.d_ff, w.k, xd.dtype)
+    ws = B.alloc_workspace(desc, B.MOC_OP_DECODE, xd.device)
+    first = B.moc_ffn_decode(xd, wgd, wud, wdd, w.k, workspace=ws).clone()   # leaves the workspace's counters marked clean
+    assert B.moc_last_device_status() == B.MOC_OK
+    out = torch.full_like(xd, 7.0)
+    t0 = time.perf_counter()
+    B.moc_test_small_batch_stall(xd, wgd, wud, wdd, w.k, 100_000_000, out=out, workspace=ws)
+    assert B.moc_last_device_status() == B.MOC_ERR_TIMEOUT          # synchronises, reports, clears
+    assert time.perf_counter() - t0 < 5.0
+    assert B.moc_last_device_status() == B.MOC_OK
+    assert torch.all(out == 7.0)
+    with pytest.raises(B.MocError):
+        B.moc_test_small_batch_stall(xd, wgd, wud, wdd, w.k, 0, out=out, workspace=ws)   # limit out of range: nothing launched
+    for rep in range(2):
+        names = _kernels_of(lambda: out.copy_(B.moc_ffn_decode(xd, wgd, wud, wdd, w.k, workspace=ws)))
+        assert "sb_fused" in names, names
+        torch.cuda.synchronize()
+        _oracle_check(out, x, wg, wu, wd, w.d_ff, w.k, f"after the time-out, call {rep}")
+        torch.testing.assert_close(out.float(), first.float(), rtol=2e-2, atol=1e-3 * float(first.float().abs().max()))
+    assert B.moc_last_device_status() == B.MOC_OK
