@@ -1359,18 +1359,20 @@ int forward_small_batch_fused(const moc_ffn_desc &d, const SmallBatchLayout &L, 
     int *status = device_status_ptr();
     if (!status) return MOC_ERR_CUDA;
     int rc;
-    if ((rc = set_smem(sbf::sb_fused_kernel, FL.smem, 2048)) != MOC_OK) return rc;
-    // all CTAs must be resident at once (the launch would be refused otherwise); asked once per shared-memory size
+    const bool grouped = (d.flags & MOC_FLAG_SELECT_2_OF_8) != 0;
+    void (*const kern)(sbf::FusedParams) = grouped ? sbf::sb_fused_kernel<true> : sbf::sb_fused_kernel<false>;
+    if ((rc = set_smem(kern, FL.smem, 2048)) != MOC_OK) return rc;
+    // all CTAs must be resident at once (the launch would be refused otherwise); asked once per form and shared-memory size
     static std::mutex mu;
     static std::unordered_map<size_t, int> per_sm_of;
     int per_sm = 0;
     {
         std::lock_guard<std::mutex> lock(mu);
-        auto it = per_sm_of.find(FL.smem);
+        auto it = per_sm_of.find(2 * FL.smem + (grouped ? 1 : 0));
         if (it == per_sm_of.end()) {
-            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, sbf::sb_fused_kernel, sbf::kBlock, FL.smem) != cudaSuccess)
+            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, sbf::kBlock, FL.smem) != cudaSuccess)
                 return MOC_ERR_CUDA;
-            per_sm_of[FL.smem] = per_sm;
+            per_sm_of[2 * FL.smem + (grouped ? 1 : 0)] = per_sm;
         } else {
             per_sm = it->second;
         }
@@ -1388,7 +1390,7 @@ int forward_small_batch_fused(const moc_ffn_desc &d, const SmallBatchLayout &L, 
     fp.K = d.k;
     fp.d = dm;
     fp.tn = FL.tn;
-    fp.grouped = (d.flags & MOC_FLAG_SELECT_2_OF_8) ? 1 : 0;
+    fp.grouped = grouped ? 1 : 0;
     fp.n_stream = FL.n_stream;
     fp.n_gu = FL.n_gu;
     fp.rows = FL.rows;
@@ -1437,7 +1439,7 @@ int forward_small_batch_fused(const moc_ffn_desc &d, const SmallBatchLayout &L, 
     cudaError_t err = cudaErrorUnknown;
     if (pdl_ok.load(std::memory_order_relaxed)) {
         cfg.numAttrs = 2;
-        MOC_LAUNCH(KID_SB_FUSED, st, err = cudaLaunchKernelExC(&cfg, reinterpret_cast<const void *>(sbf::sb_fused_kernel), args));
+        MOC_LAUNCH(KID_SB_FUSED, st, err = cudaLaunchKernelExC(&cfg, reinterpret_cast<const void *>(kern), args));
         if (err != cudaSuccess) {
             (void)cudaGetLastError();
             pdl_ok.store(0, std::memory_order_relaxed);
@@ -1445,7 +1447,7 @@ int forward_small_batch_fused(const moc_ffn_desc &d, const SmallBatchLayout &L, 
     }
     if (err != cudaSuccess) {
         cfg.numAttrs = 1;
-        MOC_LAUNCH(KID_SB_FUSED, st, err = cudaLaunchKernelExC(&cfg, reinterpret_cast<const void *>(sbf::sb_fused_kernel), args));
+        MOC_LAUNCH(KID_SB_FUSED, st, err = cudaLaunchKernelExC(&cfg, reinterpret_cast<const void *>(kern), args));
     }
     return err == cudaSuccess ? launch_ok() : MOC_ERR_CUDA;
 }

@@ -221,6 +221,8 @@ __device__ __forceinline__ void selector_role(const FusedParams &p, uint32_t *dy
 }
 
 // ------------------------------------------------------------------------------------------------ the kernel
+// GROUPED: the MoC 2:8 mask (p.grouped; a template parameter so that the Top-K form carries none of its code or registers)
+template <bool GROUPED>
 __global__ void __launch_bounds__(kBlock, 1) sb_fused_kernel(const __grid_constant__ FusedParams p) {
     namespace cg = cooperative_groups;
     extern __shared__ __align__(16) uint8_t smem_raw[];
@@ -483,6 +485,24 @@ __global__ void __launch_bounds__(kBlock, 1) sb_fused_kernel(const __grid_consta
             const int items = (extra ? 2 : 1) * chunks;
             const bool two = n_gu >= 2;  // the second issuer had stages of its own
             uint32_t kept0 = 0u;         // MoC 2:8: bit i = this lane's channel is kept by token i of the warp's first item
+            // MoC 2:8: the kept bits of tokens t0 .. t0 + 15 for this lane's channel, from the gate values in shared memory.
+            // The 8 channels of a group sit in 8 adjacent lanes: a channel is kept when fewer than two of its group come
+            // before it in (key descending, channel ascending) order.  (A plain loop: few registers are live.)
+            auto group_mask = [&](int row, bool mine, int t0) {
+                uint32_t bits = 0u;
+#pragma unroll 1
+                for (int i = 0; i < 16; ++i) {
+                    const uint32_t key = (mine && t0 + i < p.T) ? gate_key(sg[(t0 + i) * p.rows + row]) : 0u;
+                    int before = 0;
+#pragma unroll
+                    for (int m = 1; m < 8; ++m) {
+                        const uint32_t other = __shfl_xor_sync(0xffffffffu, key, m);
+                        before += (other > key || (other == key && ((lane ^ m) & 7) < (lane & 7))) ? 1 : 0;
+                    }
+                    bits |= (before < kGroupKeep ? 1u : 0u) << i;
+                }
+                return bits;
+            };
             // ---- gate values
             ok = __all_sync(0xffffffffu, tc::mbar_wait(tfull_g, 0u, abort_flag, p.status, p.wait_limit));
             if (ok) {
@@ -499,30 +519,22 @@ __global__ void __launch_bounds__(kBlock, 1) sb_fused_kernel(const __grid_consta
 #pragma unroll
                         for (int i = 0; i < 16; ++i) {
                             if (t0 + i < p.T) {
-                                if (!p.grouped) dst[(int64_t)i * p.ldf] = g[i];  // a warp's store: 128 contiguous bytes
+                                if (!GROUPED) dst[(int64_t)i * p.ldf] = g[i];  // a warp's store: 128 contiguous bytes
                                 sg[(t0 + i) * p.rows + row] = g[i];
                             }
                         }
                     }
-                    if (p.grouped && item == half) {
-                        // The 2-of-8 mask needs the gate values only: it is worked out now, while the up projection
-                        // streams, not after it.  The 8 channels of a group sit in 8 adjacent lanes: a channel is kept
-                        // when fewer than two of its group come before it in (key descending, channel ascending) order.
-#pragma unroll
-                        for (int i = 0; i < 16; ++i) {
-                            const uint32_t key = (mine && t0 + i < p.T) ? gate_key(g[i]) : 0u;
-                            int before = 0;
-#pragma unroll
-                            for (int m = 1; m < 8; ++m) {
-                                const uint32_t other = __shfl_xor_sync(0xffffffffu, key, m);
-                                before += (other > key || (other == key && ((lane ^ m) & 7) < (lane & 7))) ? 1 : 0;
-                            }
-                            kept0 |= (before < kGroupKeep ? 1u : 0u) << i;
-                        }
-                    }
                 }
             }
-            if (p.grouped) {
+            if (GROUPED && ok && half < items && !((half / chunks) == 1 && quarter * 32 + 31 < kTile - extra)) {
+                // the mask needs the gate values only: for the warp's first item it is worked out now, while the up
+                // projection streams, not after it
+                const int tile = half / chunks, t0 = (half - tile * chunks) << 4;
+                const int row = tile == 0 ? trow : extra + trow;
+                __syncwarp();
+                kept0 = group_mask(row, (tile == 0 ? trow < p.rows : trow >= kTile - extra) && row < valid, t0);
+            }
+            if (GROUPED) {
                 // no selector CTAs: the streamers clear the output accumulator, a slice each (ordered before every
                 // addition to it by the count of streamers whose Z' is written, which each joins only afterwards)
                 const int64_t vecs = (int64_t)p.T * p.d / 4;
@@ -553,7 +565,7 @@ __global__ void __launch_bounds__(kBlock, 1) sb_fused_kernel(const __grid_consta
                         if (t00 + i < p.T) z0[i] *= silu_f(key_to_float(gate_key(sg[(t00 + i) * p.rows + row])));
                 }
             }
-            if (!p.grouped) {
+            if (!GROUPED) {
                 int fine = 1;
                 if (lane == 0) fine = ok && flag_wait(p.flags + 1, (unsigned int)p.T, abort_flag, p.status, p.wait_limit) ? 1 : 0;
                 ok = __shfl_sync(0xffffffffu, fine, 0) != 0;
@@ -569,7 +581,7 @@ __global__ void __launch_bounds__(kBlock, 1) sb_fused_kernel(const __grid_consta
                     // t0 + i (one trip to L2 for the whole warp), the loop below hands them round
                     const int ch_lo = ch0 + (tile == 0 ? quarter * 32 : extra + quarter * 32);  // lane 0's channel
                     uint32_t w_lo = 0u, w_hi = 0u;
-                    if (!p.grouped && lane < 16 && t0 + lane < p.T && (ch_lo >> 5) < p.kept_words) {
+                    if (!GROUPED && lane < 16 && t0 + lane < p.T && (ch_lo >> 5) < p.kept_words) {
                         const uint32_t *kb = p.kept_bits + (int64_t)(t0 + lane) * p.kept_words + (ch_lo >> 5);
                         w_lo = __ldcg(kb);
                         if ((ch_lo >> 5) + 1 < p.kept_words) w_hi = __ldcg(kb + 1);
@@ -587,21 +599,13 @@ __global__ void __launch_bounds__(kBlock, 1) sb_fused_kernel(const __grid_consta
                         }
                     }
                     const int bit = (ch_lo & 31) + lane;  // position in the 64-bit pair
+                    const uint32_t kmask = !GROUPED ? 0u : item == item0 ? kept0 : group_mask(row, mine, t0);
                     __nv_bfloat16 *dst = p.Z + ch_lo + lane + (int64_t)t0 * p.ldz;
 #pragma unroll
                     for (int i = 0; i < 16; ++i) {
                         bool kept;
-                        if (p.grouped && item == item0) {
-                            kept = ((kept0 >> i) & 1u) != 0u;
-                        } else if (p.grouped) {
-                            const uint32_t key = (mine && t0 + i < p.T) ? gate_key(sg[(t0 + i) * p.rows + row]) : 0u;
-                            int before = 0;
-#pragma unroll
-                            for (int m = 1; m < 8; ++m) {
-                                const uint32_t other = __shfl_xor_sync(0xffffffffu, key, m);
-                                before += (other > key || (other == key && ((lane ^ m) & 7) < (lane & 7))) ? 1 : 0;
-                            }
-                            kept = before < kGroupKeep;
+                        if (GROUPED) {
+                            kept = ((kmask >> i) & 1u) != 0u;
                         } else {
                             const uint32_t lo = __shfl_sync(0xffffffffu, w_lo, i), hi = __shfl_sync(0xffffffffu, w_hi, i);
                             kept = ((bit < 32 ? lo >> bit : hi >> (bit - 32)) & 1u) != 0u;
