@@ -1354,7 +1354,8 @@ FusedLayout fused_layout(const moc_ffn_desc &d, bool saving, bool &ok) {
 int forward_small_batch_fused(const moc_ffn_desc &d, const SmallBatchLayout &L, const FusedLayout &FL, const __nv_bfloat16 *x,
                               const __nv_bfloat16 *wg, const __nv_bfloat16 *wu, const __nv_bfloat16 *wd, __nv_bfloat16 *out,
                               char *wsp, cudaStream_t st, const __nv_bfloat16 *resid, long long wait_limit = tc::kWaitLimitCycles,
-                              int stall = 0) {
+                              int stall = 0, const __nv_bfloat16 *rms_h = nullptr, const __nv_bfloat16 *rms_w = nullptr,
+                              float rms_eps = 0.f) {
     const int T = (int)d.tokens, F = d.d_ff, dm = d.d_model;
     int *status = device_status_ptr();
     if (!status) return MOC_ERR_CUDA;
@@ -1420,6 +1421,13 @@ int forward_small_batch_fused(const moc_ffn_desc &d, const SmallBatchLayout &L, 
     fp.status = status;
     fp.wait_limit = wait_limit;
     fp.stall = stall;
+    if (rms_w) {  // x is where the selector CTAs will write RMSNorm(rms_h)
+        if (grouped) return MOC_ERR_UNSUPPORTED;
+        fp.rms_h = rms_h;
+        fp.rms_w = rms_w;
+        fp.rms_eps = rms_eps;
+        fp.xn = const_cast<__nv_bfloat16 *>(x);
+    }
     // cooperative, and allowed to become resident while the previous kernel in the stream drains (the kernel waits for
     // that kernel's completion before it touches anything but the weights); a driver that refuses the combination gets
     // the plain cooperative launch from then on
@@ -1795,6 +1803,19 @@ int moc_ffn_decode_block(const moc_ffn_desc *desc, const void *h, const void *rm
     // otherwise a small kernel writes RMSNorm(h) behind the decode workspace, the plan's first kernel reads it as
     // its x, and the plan's last step adds h before it rounds
     T *xn = reinterpret_cast<T *>(wsp + align_up(moc_ffn_workspace_bytes(desc, MOC_OP_DECODE), 256));
+    if (!use_decode_plan(*desc) && !(desc->flags & MOC_FLAG_SELECT_2_OF_8)) {
+        // 6 to 32 tokens: the one-kernel form, whose selector CTAs -- idle until the gate values exist -- normalise the
+        // tokens themselves
+        bool fused_ok = false;
+        const FusedLayout FL = fused_layout(*desc, false, fused_ok);
+        if (fused_ok) {
+            const SmallBatchLayout L = small_batch_layout(*desc);
+            const int rc2 = forward_small_batch_fused(*desc, L, FL, xn, (const T *)w_gate, (const T *)w_up, (const T *)w_down,
+                                                      (T *)out, wsp, st, (const T *)h, tc::kWaitLimitCycles, 0, (const T *)h,
+                                                      (const T *)rms_weight, rms_eps);
+            if (rc2 != MOC_ERR_UNSUPPORTED) return rc2;
+        }
+    }
     MOC_LAUNCH(KID_DEC_RMSNORM, st,
                launch_pdl(dec::rmsnorm_rows_kernel, dim3((unsigned)desc->tokens), 256, 0, st, (const T *)h,
                           (const T *)rms_weight, rms_eps, desc->d_model, xn));

@@ -843,40 +843,51 @@ __global__ void __launch_bounds__(kGemvThreads, 2) down_rows_kernel(const __nv_b
 }
 
 // RMSNorm of the residual stream in front of the layer (Section 2, "RMSNorm"): y = h / sqrt(mean(h^2) + eps) . weight
-// per token, rounded to bf16 (the layer's input type).  One CTA per token.
+// for one token, rounded to bf16 (the layer's input type), by the first 256 threads of a CTA (all of its threads call:
+// there is a block-wide barrier inside).  s_part: 8 floats of shared memory.
+__device__ __forceinline__ void rmsnorm_row(const __nv_bfloat16 *__restrict__ row, const __nv_bfloat16 *__restrict__ weight,
+                                            float eps, int d, __nv_bfloat16 *__restrict__ y, float *s_part) {
+    const int tid = threadIdx.x;
+    float ss = 0.f;
+    if (tid < 256) {
+        for (int i = tid * 8; i < d; i += 256 * 8) {  // d is a multiple of 8
+            float v[8];
+            Vec8<__nv_bfloat16>::load(row + i, v);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) ss = fmaf(v[e], v[e], ss);
+        }
+        ss = warp_sum(ss);
+        if ((tid & 31) == 0) s_part[tid >> 5] = ss;
+    }
+    __syncthreads();
+    if (tid < 256) {
+        float tot = 0.f;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) tot += s_part[w];
+        const float scale = rsqrtf(tot / (float)d + eps);
+        for (int i = tid * 8; i < d; i += 256 * 8) {
+            float v[8], g[8];
+            Vec8<__nv_bfloat16>::load(row + i, v);
+            Vec8<__nv_bfloat16>::load(weight + i, g);
+            uint32_t w4[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) w4[e] = tc::pack_bf16(v[2 * e] * scale * g[2 * e], v[2 * e + 1] * scale * g[2 * e + 1]);
+            *reinterpret_cast<uint4 *>(y + i) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+        }
+    }
+}
+
+// One CTA per token.
 __global__ void __launch_bounds__(256) rmsnorm_rows_kernel(const __nv_bfloat16 *__restrict__ h,
                                                            const __nv_bfloat16 *__restrict__ weight, float eps, int d,
                                                            __nv_bfloat16 *__restrict__ y) {
     __shared__ float s_part[8];
-    const int tid = threadIdx.x, t = blockIdx.x;
+    const int t = blockIdx.x;
     tc::pdl_launch_dependents();
     // waits although h is an input of the call: the kernels after this one wait for THIS kernel only, and rely on
     // everything before it in the stream being over when it is
     tc::pdl_wait();
-    const __nv_bfloat16 *row = h + (int64_t)t * d;
-    float ss = 0.f;
-    for (int i = tid * 8; i < d; i += 256 * 8) {  // d is a multiple of 8
-        float v[8];
-        Vec8<__nv_bfloat16>::load(row + i, v);
-#pragma unroll
-        for (int e = 0; e < 8; ++e) ss = fmaf(v[e], v[e], ss);
-    }
-    ss = warp_sum(ss);
-    if ((tid & 31) == 0) s_part[tid >> 5] = ss;
-    __syncthreads();
-    float tot = 0.f;
-#pragma unroll
-    for (int w = 0; w < 8; ++w) tot += s_part[w];
-    const float scale = rsqrtf(tot / (float)d + eps);
-    for (int i = tid * 8; i < d; i += 256 * 8) {
-        float v[8], g[8];
-        Vec8<__nv_bfloat16>::load(row + i, v);
-        Vec8<__nv_bfloat16>::load(weight + i, g);
-        uint32_t w4[4];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) w4[e] = tc::pack_bf16(v[2 * e] * scale * g[2 * e], v[2 * e + 1] * scale * g[2 * e + 1]);
-        *reinterpret_cast<uint4 *>(y + (int64_t)t * d + i) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
-    }
+    rmsnorm_row(h + (int64_t)t * d, weight, eps, d, y + (int64_t)t * d, s_part);
 }
 
 

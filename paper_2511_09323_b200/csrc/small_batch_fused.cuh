@@ -83,9 +83,15 @@ struct FusedParams {
     float *acc;                  // [T, d] fp32
     __nv_bfloat16 *out;
     const __nv_bfloat16 *resid;  // the block form's residual, or nullptr
+    // the block form with the normalisation inside the kernel (Top-K form only): the selector CTAs, idle until the gate
+    // values exist, first write xn = RMSNorm(rms_h; rms_w, rms_eps) -- the array x_map reads -- a token each, and the
+    // producers request activation boxes only once flags[5] counts all of them.  rms_w == nullptr: x is given.
+    const __nv_bfloat16 *rms_h, *rms_w;
+    __nv_bfloat16 *xn;
+    float rms_eps;
     int *counters;               // [kStateCounters], of which m_tiles are used
     unsigned int *flags;         // [0] streamers done with G, [1] tokens selected, [2] streamers done with Z', [3] CTAs that
-                                 // have read the mark, [4] CTAs that have finished, [6..7] the mark (8-byte aligned)
+                                 // have read the mark, [4] CTAs that have finished, [5] tokens normalised, [6..7] the mark (8-byte aligned)
     int *status;
     long long wait_limit;        // cycles after which a wait gives up (tc::kWaitLimitCycles; shorter in the time-out test)
     int stall;                   // the time-out test: the selectors wait for this many streamers more than exist
@@ -161,7 +167,7 @@ __device__ __forceinline__ void cta_finished(const FusedParams &p) {
     __threadfence();
     if (atomicAdd(p.flags + 4, 1u) == gridDim.x - 1) {
 #pragma unroll
-        for (int i = 0; i < 5; ++i) p.flags[i] = 0u;
+        for (int i = 0; i < 6; ++i) p.flags[i] = 0u;
         __threadfence();
         *reinterpret_cast<volatile unsigned long long *>(p.flags + 6) = kCleanMark;
     }
@@ -177,6 +183,13 @@ __device__ __forceinline__ void selector_role(const FusedParams &p, uint32_t *dy
     uint32_t *keys = dyn, *lists = dyn + Fp, *bits = lists;
     auto &sm = *reinterpret_cast<SelectSmemT<kBlock / 32> *>(
         (reinterpret_cast<uintptr_t>(lists + 2 * dec::kSelListCap) + 15) & ~(uintptr_t)15);
+    if (p.rms_w) {  // the layer's input for this token: the streamers' first stages wait for it
+        __shared__ float s_part[8];
+        dec::rmsnorm_row(p.rms_h + (int64_t)t * p.d, p.rms_w, p.rms_eps, p.d, p.xn + (int64_t)t * p.d, s_part);
+        __threadfence();
+        __syncthreads();
+        if (tid == 0) atomicAdd(p.flags + 5, 1u);
+    }
     for (int i = tid; i < p.d / 4; i += kBlock)  // the token's row of the output accumulator
         reinterpret_cast<float4 *>(p.acc + (int64_t)t * p.d)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     if (tid == 0) {
@@ -327,7 +340,7 @@ __global__ void __launch_bounds__(kBlock, 1) sb_fused_kernel(const __grid_consta
     }
     // everything below touches what earlier kernels in the stream may still read or write (x, the workspace, out)
     tc::pdl_wait();
-    if (streamer && threadIdx.x == 0) {
+    if (streamer && threadIdx.x == 0 && !p.rms_w) {
         for (int i = 0; i < ahead; ++i) {
             issue_gu_x(i, i);
             pr_next();
@@ -360,6 +373,14 @@ __global__ void __launch_bounds__(kBlock, 1) sb_fused_kernel(const __grid_consta
         // ------------------------------------------------------------------ producer
         if (lane == 0) {
             bool ok = true;
+            if (p.rms_w) {  // the first ring's activation boxes: once the selector CTAs have normalised every token
+                ok = flag_wait(p.flags + 5, (unsigned int)p.T, abort_flag, p.status, p.wait_limit);
+                asm volatile("fence.proxy.async;" ::: "memory");
+                for (int i = 0; i < ahead && ok; ++i) {
+                    issue_gu_x(i, i);
+                    pr_next();
+                }
+            }
             while (ok && pr_item < 2 * n_gu) {  // W_gate, then W_up
                 if (!tc::mbar_wait(empty_bar(pr_stage), pr_phase ^ 1u, abort_flag, p.status, p.wait_limit)) {
                     ok = false;
