@@ -122,3 +122,29 @@ def test_block_argument_errors():
     with pytest.raises(B.MocError):   # negative eps
         B.moc_ffn_decode_block(hd, gd, -1.0, wgd, wud, wdd, w.k)
     assert B.moc_last_device_status() == B.MOC_OK
+
+
+@pytest.mark.parametrize("T,d,F,F_ld,K", [
+    (6, 264, 333, 336, 41),        # ragged everything, one stage per matrix
+    (16, 2048, 5461, 5464, 683),   # the LLaMA-1B layer
+    (32, 1024, 2048, 2048, 256),   # the largest batch of the one-kernel form
+])
+def test_block_in_one_kernel_for_6_to_32_tokens(T, d, F, F_ld, K):
+    """6 to 32 tokens: one cooperative kernel, no normalisation kernel in front (its selector CTAs normalise the
+    tokens); `out` may be `h`; a second call on the same workspace gives the same."""
+    w = syn.Workload(f"blk1-{T}-{d}-{F}", "bf16", T, d, F, F_ld, K, seed=4300 + T)
+    h, gamma, wg, wu, wd = _inputs(w)
+    hd, gd, wgd, wud, wdd = (t.cuda() for t in (h, gamma, wg, wu, wd))
+    B.moc_profile_enable(True)
+    out = B.moc_ffn_decode_block(hd, gd, 1e-5, wgd, wud, wdd, K, d_ff=F)
+    prof = B.moc_profile_collect()
+    B.moc_profile_enable(False)
+    names = {k for k, (n, _) in prof.items() if n}
+    assert names == {"sb_fused"}, names
+    torch.cuda.synchronize()
+    _check(out, h, gamma, 1e-5, wg, wu, wd, K, f"one-kernel block T={T}")
+    inplace = hd.clone()
+    B.moc_ffn_decode_block(inplace, gd, 1e-5, wgd, wud, wdd, K, d_ff=F, out=inplace)
+    torch.cuda.synchronize()
+    torch.testing.assert_close(inplace.float(), out.float(), rtol=2e-2, atol=1e-3 * float(out.float().abs().max()))
+    assert B.moc_last_device_status() == B.MOC_OK
