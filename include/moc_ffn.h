@@ -183,7 +183,7 @@ MOC_API int moc_ffn_recompute_up(const moc_ffn_desc *desc, const void *x, const 
  * (more: MOC_ERR_UNSUPPORTED; use moc_ffn_forward).  Up to 16 tokens it is organised so that only the
  * gate matrix and the selected rows of w_up / w_down are read from HBM (d d_ffn + 2 K d weight
  * elements per token instead of 3 d d_ffn).  From 17 tokens on the union of the tokens' channel sets
- * covers nearly every channel (from 6 tokens on at least half of them), and all three matrices are
+ * covers nearly every channel (from 5 tokens on nearly half of them at K = d_ff / 8), and all three matrices are
  * streamed once through tensor-core kernels whose tiles are shaped for a few dozen tokens;
  * moc_ffn_forward takes the same path for such batches.
  * In both forms the partial sums of the down projection meet in an fp32 accumulator in an order that

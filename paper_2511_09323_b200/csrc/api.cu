@@ -1173,8 +1173,9 @@ SmallBatchLayout small_batch_layout(const moc_ffn_desc &d) {
 
 // Which of the two small-batch forms reads fewer bytes: the decode plan reads W_gate and the rows of W_up / W_down
 // that some token selected, (1 + 2 u) F d elements with u = 1 - (1 - K/F)^T the expected share of used channels; the
-// small-batch plan reads all 3 F d but has one kernel less and no gathers.  Measured on the LLaMA-7B shape the two
-// cross where u reaches one half (6 tokens at K = F/8); from 17 tokens on only the small-batch plan exists.
+// small-batch plan reads all 3 F d but is one kernel without gathers.  Measured on the LLaMA-7B shape the two cross
+// between 4 and 5 tokens at K = F/8 (58.3 / 63.4 us for the chain, 58.9 / 59.7 us for the one-kernel form), i.e. where u
+// passes 0.45; from 17 tokens on only the small-batch plan exists.
 // MOC_FFN_SB_MIN_TOKENS=n in the environment moves the boundary to n tokens (measurements only).
 bool small_batch_preferred(const moc_ffn_desc &d) {
     static const int forced = [] {
@@ -1184,7 +1185,7 @@ bool small_batch_preferred(const moc_ffn_desc &d) {
     if (forced >= 1) return d.tokens >= forced;
     if (d.tokens > 16) return true;
     const double unused = std::pow(1.0 - (double)d.k / (double)d.d_ff, (double)d.tokens);
-    return 1.0 - unused >= 0.5;
+    return 1.0 - unused >= 0.45;
 }
 
 // moc_ffn_forward takes the small-batch plan for every bf16 batch it can serve (the tensor-core plan's tiles need

@@ -129,8 +129,8 @@ def test_block_argument_errors():
     (16, 2048, 5461, 5464, 683),   # the LLaMA-1B layer
     (32, 1024, 2048, 2048, 256),   # the largest batch of the one-kernel form
 ])
-def test_block_in_one_kernel_for_6_to_32_tokens(T, d, F, F_ld, K):
-    """6 to 32 tokens: one cooperative kernel, no normalisation kernel in front (its selector CTAs normalise the
+def test_block_in_one_kernel_for_a_few_dozen_tokens(T, d, F, F_ld, K):
+    """5 to 32 tokens (at K = d_ff / 8): one cooperative kernel, no normalisation kernel in front (its selector CTAs normalise the
     tokens); `out` may be `h`; a second call on the same workspace gives the same."""
     w = syn.Workload(f"blk1-{T}-{d}-{F}", "bf16", T, d, F, F_ld, K, seed=4300 + T)
     h, gamma, wg, wu, wd = _inputs(w)
