@@ -201,11 +201,13 @@ __device__ __forceinline__ void selector_role(const FusedParams &p, uint32_t *dy
     if (s_abort) return;
     MOC_TL_CTA(1280);
     if (!dec::cta_stage_rows(&s_bar, &s_abort, p.status, keys, p.G + (int64_t)t * p.ldf, (uint32_t)Fp * 4u)) return;
+    MOC_TL_CTA(3072);
     uint32_t tau;
     int need;
     bool ties_cut;
     uint32_t kreg[dec::kSelCached];
     dec::cta_select_threshold(nullptr, p.F, p.K, keys, lists, sm, tau, need, ties_cut, kreg);
+    MOC_TL_CTA(3328);
     uint32_t *my_bits = p.kept_bits + (int64_t)t * p.kept_words;
     constexpr int NW = kBlock / 32;
     if (!ties_cut) {
@@ -228,6 +230,7 @@ __device__ __forceinline__ void selector_role(const FusedParams &p, uint32_t *dy
     __syncthreads();
     if (tid == 0) {
         atomicAdd(p.flags + 1, 1u);
+        MOC_TL_CTA_ANY(3840);
         cta_finished(p);
     }
     MOC_TL_CTA(1536);

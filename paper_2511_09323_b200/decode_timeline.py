@@ -25,7 +25,8 @@ REGIONS = [(256, "gate start"), (512, "gate mma done"), (768, "gate end"), (1024
            (2560, "down after wait"), (2816, "down mma done"), (3072, "down end")]
 # the one-kernel form (streamer CTAs, then the selector CTAs, in one grid)
 REGIONS_FUSED = [(256, "start"), (512, "after grid barrier"), (768, "gate mma done"), (1024, "gate values stored"),
-                 (1280, "select: row wait over"), (1536, "select end"), (1792, "up mma done"), (2048, "Z' stored"),
+                 (1280, "select: row wait over"), (3072, "select: row staged"), (3328, "select: threshold found"),
+                 (3840, "select: bitmap signalled"), (1536, "select end"), (1792, "up mma done"), (2048, "Z' stored"),
                  (2304, "down: Z' complete"), (2560, "down mma done"), (2816, "end")]
 # the one-kernel decode form for one or two tokens
 REGIONS_COOP = [(256, "start"), (512, "x staged, arrays cleared"), (768, "gate rows done, barrier 0"), (1024, "histogram complete (barrier 1)"),
