@@ -605,18 +605,9 @@ __global__ void __launch_bounds__(256) split_sum_kernel(const float *__restrict_
     }
 }
 
-// A GEMM whose output has so few tiles that half of the CTA pairs would idle (a few hundred tokens: 32 tiles of
-// 256 x 256 for 512 tokens and d_model = 4096, each with the whole d_ffn to contract) is split in two along its
-// contraction: the halves run as two problems of one launch into fp32 partial outputs, which split_sum_kernel adds.
-// MOC_FFN_SPLIT_K=0 in the environment switches the split off (comparisons).
+// (see tc::split_contraction_pays) -- here with the room the caller has for the partial outputs
 bool split_contraction(int64_t T, int n_cols, size_t scratch_floats) {
-    static const bool on = [] {
-        const char *e = getenv("MOC_FFN_SPLIT_K");
-        return !(e && atoi(e) == 0);
-    }();
-    if (!on || !tc::pair_mode() || (n_cols & 7)) return false;
-    const int tiles = (ceil_div(T, tc::BM) + 1) / 2 * ceil_div(n_cols, tc::BN);
-    return 2 * tiles <= tc::sm_count() / 2 && (size_t)2 * T * n_cols <= scratch_floats;
+    return tc::split_contraction_pays(T, n_cols) && (size_t)2 * T * n_cols <= scratch_floats;
 }
 
 int launch_split_sum(const float *partial, int64_t T, int n_cols, __nv_bfloat16 *out, cudaStream_t st) {
@@ -897,19 +888,33 @@ int backward_tc(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat
         if (!map_k_major(&p.a_map[0], dGp, T, F, L.ldf, BM) || !map_k_major(&p.a_map[1], dUp, T, F, L.ldf, BM) ||
             !map_mn_major(&p.b_map[0], wg, F, dm, dm) || !map_mn_major(&p.b_map[1], wu, F, dm, dm))
             return MOC_ERR_CUDA;
-        p.k_segments = 2;
-        p.a_idx[0][1] = 1;
-        p.b_idx[0][1] = 1;
         p.k_blocks = ceil_div(F, BK);
         p.M = (int)T;
         p.N = dm;
         p.m_tiles = ceil_div(T, BM);
         p.n_tiles = ceil_div(dm, BN);
-        p.c[0] = gx;
-        p.ldc[0] = dm;
         p.status = status;
-        MOC_LAUNCH(KID_TC_DX_GEMM, st, (rc = launch_gemm<false, true, EPI_BF16>(p, st)));
-        if (rc != MOC_OK) return rc;
+        if (L.split_bytes) {
+            // a few hundred tokens: the two segments as two problems of the launch, fp32 partial outputs, added behind it
+            float *partial = reinterpret_cast<float *>(ws + L.off_split);
+            p.num_problems = 2;
+            p.a_idx[1][0] = 1;
+            p.b_idx[1][0] = 1;
+            p.c[0] = partial;
+            p.c[1] = partial + T * dm;
+            p.ldc[0] = p.ldc[1] = dm;
+            MOC_LAUNCH(KID_TC_DX_GEMM, st, (rc = launch_gemm<false, true, EPI_F32>(p, st)));
+            if (rc != MOC_OK) return rc;
+            if ((rc = launch_split_sum(partial, T, dm, gx, st)) != MOC_OK) return rc;
+        } else {
+            p.k_segments = 2;
+            p.a_idx[0][1] = 1;
+            p.b_idx[0][1] = 1;
+            p.c[0] = gx;
+            p.ldc[0] = dm;
+            MOC_LAUNCH(KID_TC_DX_GEMM, st, (rc = launch_gemm<false, true, EPI_BF16>(p, st)));
+            if (rc != MOC_OK) return rc;
+        }
     }
     return MOC_OK;
 }

@@ -961,6 +961,7 @@ struct TcBackwardLayout {
     // MoC 2:8 with grad_x on the sparse MMA: dG' and dU' in compressed form [T, F / 2] with their metadata (sp_bytes == 0:
     // not used)
     size_t off_gc, off_uc, off_gmeta, off_umeta, sp_bytes;
+    size_t off_split, split_bytes;        // a few hundred tokens: two fp32 partial outputs [T, d] of the grad_x GEMM
 };
 
 inline int round_up8(int v) { return (v + 7) & ~7; }
@@ -1010,6 +1011,20 @@ inline TcForwardLayout tc_forward_layout(const moc_ffn_desc &d) {
     return L;
 }
 
+// A GEMM whose output has so few tiles that half of the CTA pairs would idle (a few hundred tokens: 32 tiles of
+// 256 x 256 for 512 tokens and d_model = 4096, each with the whole d_ffn to contract) is split in two along its
+// contraction: the halves run as two problems of one launch into fp32 partial outputs, which a small kernel adds.
+// MOC_FFN_SPLIT_K=0 in the environment switches the split off (comparisons).
+inline bool split_contraction_pays(int64_t T, int n_cols) {
+    static const bool on = [] {
+        const char *e = getenv("MOC_FFN_SPLIT_K");
+        return !(e && atoi(e) == 0);
+    }();
+    if (!on || !pair_mode() || (n_cols & 7)) return false;
+    const int64_t tiles = ((T + BM - 1) / BM + 1) / 2 * ((n_cols + BN - 1) / BN);
+    return 2 * tiles <= sm_count() / 2;
+}
+
 inline TcBackwardLayout tc_backward_layout(const moc_ffn_desc &d) {
     TcBackwardLayout L{};
     L.ldf = round_up8(d.d_ff);
@@ -1036,6 +1051,11 @@ inline TcBackwardLayout tc_backward_layout(const moc_ffn_desc &d) {
         L.sp_bytes = 2 * comp + 2 * meta;
         off += L.sp_bytes;
     }
+    // fp32 partial outputs of the grad_x GEMM when its contraction is split (its two segments as two problems)
+    L.off_split = off;
+    L.split_bytes = (!L.small_bytes && !L.sp_bytes && split_contraction_pays(d.tokens, d.d_model))
+                        ? align_up((size_t)2 * d.tokens * d.d_model * sizeof(float), 256) : 0;
+    off += L.split_bytes;
     L.total = off;
     return L;
 }

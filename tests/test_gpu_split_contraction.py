@@ -50,3 +50,30 @@ def test_forward_with_split_down_projection(T, d, F, F_ld, K):
     out_big = B.moc_ffn_forward(big, wgd, wud, wdd, K, d_ff=F, save=False)[0]
     torch.cuda.synchronize()
     torch.testing.assert_close(out.float(), out_big[:T].float(), rtol=2e-2, atol=2e-3 * float(out.float().abs().max()))
+
+
+@pytest.mark.parametrize("T,d,F,F_ld,K", [
+    (400, 1024, 2048, 2048, 256),
+    (257, 520, 2000, 2048, 250),     # output 520 columns wide: three column tiles, the last 8 wide; padding rows
+])
+def test_backward_with_split_grad_x(T, d, F, F_ld, K):
+    """The grad_x GEMM of the same range: its two contraction segments (dG' Wg and dU' Wu, Eq. (bp-5)) run as two
+    problems of one launch into fp32 partial outputs, which the same small kernel adds."""
+    w = syn.Workload(f"splitb-{T}-{d}-{F}", "bf16", T, d, F, F_ld, K, seed=7100 + T)
+    wg, wu, wd = syn.make_weights(w)
+    x, dD = syn.make_x(w), syn.make_grad_out(w)
+    xd, wgd, wud, wdd, dDd = (t.cuda() for t in (x, wg, wu, wd, dD))
+    out, idx, tg, tu = B.moc_ffn_forward(xd, wgd, wud, wdd, K, d_ff=F)
+    B.moc_profile_enable(True)
+    grads = B.moc_ffn_backward(xd, wgd, wud, wdd, idx, tg, tu, dDd, d_ff=F)
+    prof = B.moc_profile_collect()
+    B.moc_profile_enable(False)
+    assert prof.get("tc_split_sum", (0, 0))[0] == 1 and prof.get("tc_dx_gemm", (0, 0))[0] == 1, prof
+    torch.cuda.synchronize()
+    x64, wg64, wu64, wd64, dD64 = map(syn.to_f64, (x, wg[:F], wu[:F], wd[:F], dD))
+    gdev = {k: syn.to_f64(v) for k, v in grads.items()}
+    parity.check_backward(gdev, x64, wg64, wu64, wd64, idx.cpu().numpy(), syn.to_f64(tg), syn.to_f64(tu), dD64, F, w.dtype)
+    # only grad_x asked for: the same path, the same bits (the halves are added in a fixed order)
+    gx = B.moc_ffn_backward(xd, wgd, wud, wdd, idx, tg, tu, dDd, d_ff=F, want=("x",))["grad_x"]
+    torch.cuda.synchronize()
+    assert torch.equal(gx, grads["grad_x"])
