@@ -1039,8 +1039,13 @@ int launch_coop(const dc::Params &prm, const CoopLayout &L, cudaStream_t st) {
     if (per_sm < 1 || L.grid > per_sm * tc::sm_count()) return MOC_ERR_UNSUPPORTED;
     dc::Params local = prm;
     void *args[] = {&local};
+    cudaError_t err = cudaSuccess;
     MOC_LAUNCH(KID_DEC_COOP, st,
-               cudaLaunchCooperativeKernel(reinterpret_cast<void *>(kern), dim3(L.grid), dim3(dc::kThreads), args, L.smem, st));
+               err = cudaLaunchCooperativeKernel(reinterpret_cast<void *>(kern), dim3(L.grid), dim3(dc::kThreads), args, L.smem, st));
+    if (err != cudaSuccess) {  // refused: nothing ran, the four-kernel plan serves the call
+        (void)cudaGetLastError();
+        return MOC_ERR_UNSUPPORTED;
+    }
     return launch_ok();
 }
 
@@ -1463,7 +1468,11 @@ int forward_small_batch_fused(const moc_ffn_desc &d, const SmallBatchLayout &L, 
         cfg.numAttrs = 1;
         MOC_LAUNCH(KID_SB_FUSED, st, err = cudaLaunchKernelExC(&cfg, reinterpret_cast<const void *>(kern), args));
     }
-    return err == cudaSuccess ? launch_ok() : MOC_ERR_CUDA;
+    if (err != cudaSuccess) {  // the launch was refused (SMs reserved by others, ...): nothing ran, the multi-kernel forms serve the call
+        (void)cudaGetLastError();
+        return MOC_ERR_UNSUPPORTED;
+    }
+    return launch_ok();
 }
 
 int forward_small_batch(const moc_ffn_desc &d, const __nv_bfloat16 *x, const __nv_bfloat16 *wg,
