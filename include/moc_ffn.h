@@ -42,7 +42,7 @@
  *            behind the first, or anywhere once the first has completed.  Its contents between calls are the
  *            caller's (nothing in it outlives a call).  For batches of up to 32 tokens the library keeps three
  *            counters per workspace ADDRESS in its own statically allocated device memory (they are left zero by
- *            every call that completes, so a call can start without clearing them); 256 addresses per device are
+ *            every call that completes, so a call can start without clearing them); 1024 addresses per device are
  *            served that way, further ones by the kernels that need no such state.
  * Co-op      Two kernels are launched cooperatively (cudaLaunchCooperativeKernel: their CTAs wait on one another, so
  *            all must be resident): the one-kernel forms of moc_ffn_decode / moc_ffn_forward for one or two tokens

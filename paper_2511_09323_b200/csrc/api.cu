@@ -48,7 +48,7 @@ int *device_status_ptr() {
 // flags its CTAs signal with and a mark that says both are zero): kept in the library's own device memory rather than
 // in the caller's workspace, whose contents between calls are the caller's.  One block of kFusedStateWords words per
 // workspace address -- a workspace serves one call at a time, so a block is never used by two runs at once.
-constexpr int kFusedStateWords = 128, kFusedStateSlots = 256;
+constexpr int kFusedStateWords = 128, kFusedStateSlots = 1024;
 __device__ unsigned int g_fused_state[kFusedStateSlots * kFusedStateWords];
 
 unsigned int *fused_state_for(const void *workspace) {
